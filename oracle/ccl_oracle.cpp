@@ -1,0 +1,425 @@
+// Chiplet-Contiguous Layout (CCL) -- CPU oracle.
+//
+// TEST INFRASTRUCTURE ONLY.  This file is the slow, plain, obviously-correct
+// statement of what the CUDA library computes.  It shares no code, header,
+// table or helper with the CUDA path and is never called by the product path;
+// only the test-suite, the smoke check and the benchmark's CPU-baseline leg
+// load it.
+//
+// Every function cites the passage of the paper it restates:
+//   Eq. 1  : g = floor(n / w), n' = n mod w, w = N / G
+//   Eq. 2  : index_row(k, n) = k*N + n
+//   Eq. 3  : index_CCL(k, n) = g*K*w + k*w + n'
+//   Sec. 3.2 (last paragraph): a strip of K*w elements may be aligned to the
+//            placement granularity (strip_align_bytes below)
+//   Sec. 2.2: C = A*B, one CTA per output tile streaming A and B along K;
+//            a column region of a column-major operand is already contiguous
+//            (PART_ROWS below)
+//   Sec. 4.1: page-granularity placement policies (round-robin interleave,
+//            coarse G-block placement) and the remote-traffic metric, here
+//            WITHOUT the L2 filter: every byte a CTA touches is counted.
+//
+// Pinning status (tests/test_oracle_*.py, no GPU needed):
+//   map / inverse : pinned (bijection, stride form of Sec. 3.3, Fig. 4(a)
+//                   worked example, reshape/permute, slice sizes of Sec. 2.2)
+//   repack        : pinned (permutation, round trip, strided-slice copies)
+//   gemm          : pinned (identity, all-ones, library matmul, fp64 bound)
+//   traffic       : pinned by invariants, closed forms and a hand-enumerated
+//                   tiny case; against the paper's Fig. 6 ratios it is
+//                   PARITY UNPINNED (they need the unreleased L2 simulator).
+//
+// Build: g++ -O2 -std=c++17 -shared -fPIC -pthread (see oracle/build.py).
+
+#include <cstdint>
+#include <cstring>
+#include <cstdlib>
+#include <vector>
+#include <thread>
+#include <algorithm>
+
+extern "C" {
+
+enum { ORC_ROWMAJOR = 0, ORC_CCL = 1 };
+enum { ORC_PART_NONE = 0, ORC_PART_ROWS = 1, ORC_PART_COLS = 2 };
+enum { ORC_PLACE_RR = 0, ORC_PLACE_BLOCK = 1, ORC_PLACE_BEST = 2 };
+enum { ORC_ASSIGN_N = 0, ORC_ASSIGN_M = 1, ORC_ASSIGN_EXPLICIT = 2 };
+
+// A stored matrix: rows x cols, cols contiguous in the row-major view.
+typedef struct {
+    int64_t rows, cols;
+    int32_t elem_bytes;
+    int32_t P;                  // the paper's G
+    int32_t part;               // which stored dimension is split over chiplets
+    int32_t layout;             // physical order of the buffer
+    int64_t strip_align_bytes;  // 0 = packed (Eq. 3 literally)
+} orc_mat;
+
+typedef struct {
+    int64_t M, N, K;
+    int32_t BM, BN;
+    orc_mat A, B, C;
+    int32_t a_trans, b_trans;
+    int32_t P;
+    int64_t page_bytes;
+    int32_t place[3];
+    int32_t assign;
+    int32_t strip_tiling;
+} orc_traffic_desc;
+
+}  // extern "C"
+
+namespace {
+
+bool mat_ok(const orc_mat& m) {
+    if (m.rows <= 0 || m.cols <= 0 || m.P < 1) return false;
+    if (m.elem_bytes != 1 && m.elem_bytes != 2 && m.elem_bytes != 4) return false;
+    if (m.layout != ORC_ROWMAJOR && m.layout != ORC_CCL) return false;
+    if (m.part < 0 || m.part > 2) return false;
+    if (m.strip_align_bytes < 0 || m.strip_align_bytes % m.elem_bytes) return false;
+    if (m.layout == ORC_CCL) {
+        if (m.part == ORC_PART_COLS && m.cols % m.P) return false;  // w = N/G must be whole
+        if (m.part == ORC_PART_ROWS && m.rows % m.P) return false;
+    }
+    return true;
+}
+
+bool is_ccl(const orc_mat& m) { return m.layout == ORC_CCL && m.part != ORC_PART_NONE; }
+
+// Elements between the bases of two consecutive strips.  Packed: K*w (Eq. 3);
+// aligned: K*w*e rounded up to the alignment (Sec. 3.2, last paragraph).
+int64_t strip_stride(const orc_mat& m) {
+    int64_t packed = (m.part == ORC_PART_COLS) ? m.rows * (m.cols / m.P) : (m.rows / m.P) * m.cols;
+    if (m.strip_align_bytes == 0) return packed;
+    int64_t bytes = packed * m.elem_bytes;
+    int64_t up = (bytes + m.strip_align_bytes - 1) / m.strip_align_bytes * m.strip_align_bytes;
+    return up / m.elem_bytes;
+}
+
+int64_t buffer_elems(const orc_mat& m) {
+    if (!is_ccl(m)) return m.rows * m.cols;
+    return (int64_t)m.P * strip_stride(m);
+}
+
+// Eq. 2 (row-major) or Eq. 1 + Eq. 3 (CCL) applied to stored coordinates.
+int64_t map_offset(const orc_mat& m, int64_t r, int64_t c) {
+    if (!is_ccl(m)) return r * m.cols + c;            // Eq. 2
+    if (m.part == ORC_PART_COLS) {
+        int64_t w = m.cols / m.P;                      // per-chiplet width
+        int64_t g = c / w;                             // Eq. 1
+        int64_t cp = c % w;                            // Eq. 1
+        return g * strip_stride(m) + r * w + cp;       // Eq. 3
+    }
+    // Split along rows: each strip is h whole rows, already contiguous (Sec. 2.2).
+    int64_t h = m.rows / m.P;
+    return (r / h) * strip_stride(m) + (r % h) * m.cols + c;
+}
+
+int map_inverse(const orc_mat& m, int64_t off, int64_t* r, int64_t* c) {
+    if (off < 0 || off >= buffer_elems(m)) return -1;
+    if (!is_ccl(m)) { *r = off / m.cols; *c = off % m.cols; return 0; }
+    int64_t st = strip_stride(m);
+    int64_t g = off / st, rem = off % st;
+    if (m.part == ORC_PART_COLS) {
+        int64_t w = m.cols / m.P;
+        if (rem >= m.rows * w) return -2;              // inside the padding of strip g
+        *r = rem / w; *c = g * w + rem % w; return 0;
+    }
+    int64_t h = m.rows / m.P;
+    if (rem >= h * m.cols) return -2;
+    *r = g * h + rem / m.cols; *c = rem % m.cols; return 0;
+}
+
+inline float bf16_to_f32(uint16_t h) { uint32_t u = (uint32_t)h << 16; float f; std::memcpy(&f, &u, 4); return f; }
+inline uint16_t f32_to_bf16_rne(float f) {
+    uint32_t u; std::memcpy(&u, &f, 4);
+    u += 0x7FFFu + ((u >> 16) & 1u);                   // round to nearest, ties to even (finite inputs)
+    return (uint16_t)(u >> 16);
+}
+
+// ---- tile grid of the execution model (Sec. 2.2 / Sec. 4.1: one CTA per output tile) ----
+struct Seg { int64_t lo, hi; };
+
+// Tiles of one dimension.  strip_tiled: every strip of len/P is tiled on its own,
+// so that no tile straddles two strips; otherwise plain ceil(len/B) tiles.
+std::vector<Seg> tile_dim(int64_t len, int64_t B, int P, bool strip_tiled) {
+    std::vector<Seg> v;
+    if (!strip_tiled) { for (int64_t s = 0; s < len; s += B) v.push_back({s, std::min(len, s + B)}); return v; }
+    int64_t w = len / P;
+    for (int g = 0; g < P; ++g)
+        for (int64_t s = 0; s < w; s += B) v.push_back({g * w + s, g * w + std::min(w, s + B)});
+    return v;
+}
+
+struct Tile { int64_t m0, m1, n0, n1; int32_t q; };
+
+int enumerate_tiles(const orc_traffic_desc& d, const int32_t* explicit_q, std::vector<Tile>& out) {
+    if (d.M <= 0 || d.N <= 0 || d.K <= 0 || d.BM <= 0 || d.BN <= 0 || d.P < 1) return -1;
+    bool n_strips = d.assign == ORC_ASSIGN_N, m_strips = d.assign == ORC_ASSIGN_M;
+    if (n_strips && d.N % d.P) return -1;
+    if (m_strips && d.M % d.P) return -1;
+    if (d.assign == ORC_ASSIGN_EXPLICIT && !explicit_q) return -1;
+    if (d.assign < 0 || d.assign > 2) return -1;
+    auto tm = tile_dim(d.M, d.BM, d.P, m_strips && d.strip_tiling);
+    auto tn = tile_dim(d.N, d.BN, d.P, n_strips && d.strip_tiling);
+    for (size_t i = 0; i < tm.size(); ++i)
+        for (size_t j = 0; j < tn.size(); ++j) {
+            Tile t{tm[i].lo, tm[i].hi, tn[j].lo, tn[j].hi, 0};
+            int64_t idx = (int64_t)i * (int64_t)tn.size() + (int64_t)j;
+            if (n_strips) t.q = (int32_t)(t.n0 / (d.N / d.P));       // chiplet owning the tile's columns
+            else if (m_strips) t.q = (int32_t)(t.m0 / (d.M / d.P));
+            else { t.q = explicit_q[idx]; if (t.q < 0 || t.q >= d.P) return -1; }
+            out.push_back(t);
+        }
+    return 0;
+}
+
+// Stored-coordinate rectangle an output tile touches in operand X (0=A, 1=B, 2=C).
+void tile_rect(const orc_traffic_desc& d, const Tile& t, int X, int64_t& r0, int64_t& r1, int64_t& c0, int64_t& c1) {
+    if (X == 0) { if (!d.a_trans) { r0 = t.m0; r1 = t.m1; c0 = 0; c1 = d.K; } else { r0 = 0; r1 = d.K; c0 = t.m0; c1 = t.m1; } }
+    else if (X == 1) { if (!d.b_trans) { r0 = 0; r1 = d.K; c0 = t.n0; c1 = t.n1; } else { r0 = t.n0; r1 = t.n1; c0 = 0; c1 = d.K; } }
+    else { r0 = t.m0; r1 = t.m1; c0 = t.n0; c1 = t.n1; }
+}
+
+bool traffic_desc_ok(const orc_traffic_desc& d) {
+    if (!mat_ok(d.A) || !mat_ok(d.B) || !mat_ok(d.C)) return false;
+    if (d.page_bytes <= 0) return false;
+    const orc_mat* ms[3] = {&d.A, &d.B, &d.C};
+    for (int X = 0; X < 3; ++X) {
+        if (d.page_bytes % ms[X]->elem_bytes) return false;
+        if (d.place[X] < 0 || d.place[X] > 2) return false;
+    }
+    int64_t ar = d.a_trans ? d.K : d.M, ac = d.a_trans ? d.M : d.K;
+    int64_t br = d.b_trans ? d.N : d.K, bc = d.b_trans ? d.K : d.N;
+    return d.A.rows == ar && d.A.cols == ac && d.B.rows == br && d.B.cols == bc && d.C.rows == d.M && d.C.cols == d.N;
+}
+
+int64_t pages_of(const orc_mat& m, int64_t S) { return (buffer_elems(m) * m.elem_bytes + S - 1) / S; }
+
+// Owner of a page under the fixed (address-driven) policies of Sec. 4.1.
+//   RR   : consecutive fixed-size regions go to chiplets in address order.
+//   BLOCK: the buffer is cut into P equal contiguous address blocks (coarse
+//          placement); a page belongs to the block that holds its first byte.
+int32_t fixed_owner(int place, int64_t page, int64_t S, int P, int64_t bytes_total) {
+    if (place == ORC_PLACE_RR) return (int32_t)(page % P);
+    int64_t o = (page * S * P) / bytes_total;
+    return (int32_t)std::min<int64_t>(P - 1, o);
+}
+
+struct Visit { int64_t byte, len; };   // a contiguous piece inside one page
+
+template <class F>
+void for_each_piece_elem(const orc_traffic_desc& d, const orc_mat& m, int64_t r0, int64_t r1, int64_t c0, int64_t c1, F&& f) {
+    for (int64_t r = r0; r < r1; ++r)
+        for (int64_t c = c0; c < c1; ++c) f(map_offset(m, r, c) * m.elem_bytes, (int64_t)m.elem_bytes);
+    (void)d;
+}
+
+// Run level: a stored row of the rectangle is contiguous inside one strip; cut it
+// at strip boundaries (PART_COLS) and then at page boundaries.
+template <class F>
+void for_each_piece_run(const orc_traffic_desc& d, const orc_mat& m, int64_t r0, int64_t r1, int64_t c0, int64_t c1, F&& f) {
+    int64_t S = d.page_bytes, e = m.elem_bytes;
+    int64_t w = (is_ccl(m) && m.part == ORC_PART_COLS) ? m.cols / m.P : m.cols;
+    for (int64_t r = r0; r < r1; ++r) {
+        int64_t c = c0;
+        while (c < c1) {
+            int64_t cend = std::min(c1, (c / w + 1) * w);
+            int64_t b = map_offset(m, r, c) * e, bend = b + (cend - c) * e;
+            while (b < bend) {
+                int64_t pend = std::min(bend, (b / S + 1) * S);
+                f(b, pend - b);
+                b = pend;
+            }
+            c = cend;
+        }
+    }
+}
+
+template <bool RUNS>
+int traffic_impl(const orc_traffic_desc& d, const int32_t* explicit_q, uint64_t* per_cta, uint64_t* const* per_page_out,
+                 uint8_t* const* owner_out, uint64_t* totals) {
+    if (!traffic_desc_ok(d)) return -1;
+    std::vector<Tile> tiles;
+    if (enumerate_tiles(d, explicit_q, tiles)) return -1;
+    const orc_mat* ms[3] = {&d.A, &d.B, &d.C};
+    int64_t S = d.page_bytes;
+    int P = d.P;
+    std::vector<uint64_t> hist[3];
+    std::vector<uint8_t> own[3];
+    for (int X = 0; X < 3; ++X) { hist[X].assign((size_t)pages_of(*ms[X], S) * P, 0); own[X].assign((size_t)pages_of(*ms[X], S), 0); }
+    // pass 1: bytes of every page demanded by every chiplet
+    for (const Tile& t : tiles)
+        for (int X = 0; X < 3; ++X) {
+            int64_t r0, r1, c0, c1; tile_rect(d, t, X, r0, r1, c0, c1);
+            auto add = [&](int64_t byte, int64_t len) { hist[X][(size_t)(byte / S) * P + t.q] += (uint64_t)len; };
+            if (RUNS) for_each_piece_run(d, *ms[X], r0, r1, c0, c1, add); else for_each_piece_elem(d, *ms[X], r0, r1, c0, c1, add);
+        }
+    // owner of every page
+    for (int X = 0; X < 3; ++X) {
+        int64_t np = pages_of(*ms[X], S), bytes_total = buffer_elems(*ms[X]) * ms[X]->elem_bytes;
+        for (int64_t p = 0; p < np; ++p) {
+            if (d.place[X] == ORC_PLACE_BEST) {        // best any page-granular mapping can do: the largest demander
+                int best = 0;
+                for (int q = 1; q < P; ++q) if (hist[X][(size_t)p * P + q] > hist[X][(size_t)p * P + best]) best = q;
+                own[X][p] = (uint8_t)best;
+            } else own[X][p] = (uint8_t)fixed_owner(d.place[X], p, S, P, bytes_total);
+        }
+    }
+    // pass 2: classify every touched byte as local or remote
+    for (int i = 0; i < 6; ++i) totals[i] = 0;
+    for (size_t ti = 0; ti < tiles.size(); ++ti) {
+        const Tile& t = tiles[ti];
+        for (int X = 0; X < 3; ++X) {
+            uint64_t loc = 0, rem = 0;
+            int64_t r0, r1, c0, c1; tile_rect(d, t, X, r0, r1, c0, c1);
+            auto cls = [&](int64_t byte, int64_t len) { if (own[X][(size_t)(byte / S)] == t.q) loc += (uint64_t)len; else rem += (uint64_t)len; };
+            if (RUNS) for_each_piece_run(d, *ms[X], r0, r1, c0, c1, cls); else for_each_piece_elem(d, *ms[X], r0, r1, c0, c1, cls);
+            per_cta[ti * 6 + X * 2 + 0] = loc; per_cta[ti * 6 + X * 2 + 1] = rem;
+            totals[X * 2 + 0] += loc; totals[X * 2 + 1] += rem;
+        }
+    }
+    for (int X = 0; X < 3; ++X) {
+        if (per_page_out && per_page_out[X]) std::memcpy(per_page_out[X], hist[X].data(), hist[X].size() * 8);
+        if (owner_out && owner_out[X]) std::memcpy(owner_out[X], own[X].data(), own[X].size());
+    }
+    return 0;
+}
+
+}  // namespace
+
+extern "C" {
+
+int orc_mat_valid(const orc_mat* m) { return mat_ok(*m) ? 1 : 0; }
+
+// Eq. 1-3.  Returns 0 and the element offset, or -1 on a bad descriptor / coordinate.
+int orc_map_offset(const orc_mat* m, int64_t r, int64_t c, int64_t* off) {
+    if (!mat_ok(*m) || r < 0 || c < 0 || r >= m->rows || c >= m->cols) return -1;
+    *off = map_offset(*m, r, c); return 0;
+}
+
+// Inverse of Eq. 3.  -2 when the offset falls into alignment padding.
+int orc_map_inverse(const orc_mat* m, int64_t off, int64_t* r, int64_t* c) {
+    if (!mat_ok(*m)) return -1;
+    return map_inverse(*m, off, r, c);
+}
+
+int orc_strip_stride(const orc_mat* m, int64_t* elems) { if (!mat_ok(*m) || !is_ccl(*m)) return -1; *elems = strip_stride(*m); return 0; }
+int orc_buffer_bytes(const orc_mat* m, int64_t* bytes) { if (!mat_ok(*m)) return -1; *bytes = buffer_elems(*m) * m->elem_bytes; return 0; }
+
+// Whole map as a table: out[r*cols + c] = offset (for bijection / stride-form pins).
+int orc_map_table(const orc_mat* m, int64_t* out) {
+    if (!mat_ok(*m)) return -1;
+    for (int64_t r = 0; r < m->rows; ++r) for (int64_t c = 0; c < m->cols; ++c) out[r * m->cols + c] = map_offset(*m, r, c);
+    return 0;
+}
+
+// Repack (Sec. 3.3: operands "adopt CCL" by a permutation copy).
+// dir 0: dst[map(r,c)] = src[r*C + c], padding bytes = 0.  dir 1: dst[r*C + c] = src[map(r,c)].
+int orc_repack(const orc_mat* m, const void* src, void* dst, int dir) {
+    if (!mat_ok(*m)) return -1;
+    int64_t e = m->elem_bytes;
+    const uint8_t* s = (const uint8_t*)src; uint8_t* d = (uint8_t*)dst;
+    if (dir == 0) std::memset(d, 0, (size_t)(buffer_elems(*m) * e));
+    for (int64_t r = 0; r < m->rows; ++r)
+        for (int64_t c = 0; c < m->cols; ++c) {
+            int64_t lin = (r * m->cols + c) * e, off = map_offset(*m, r, c) * e;
+            if (dir == 0) std::memcpy(d + off, s + lin, (size_t)e); else std::memcpy(d + lin, s + off, (size_t)e);
+        }
+    return 0;
+}
+
+// GEMM of Sec. 2.2, C = A*B, from the LOGICAL operands (never from CCL buffers):
+//   ref32[m][n] = sum_k float(A[m][k]) * float(B[k][n]), k ascending, fp32 accumulate
+//   ref64       = the same sum in double (bounds the fp32 oracle's own error)
+//   out_bf16    = ref32 rounded to bf16, nearest-even
+// A is stored row-major [M x K] (a_trans = 0) or [K x M] (a_trans = 1);
+// B is stored row-major [K x N] (b_trans = 0) or [N x K] (b_trans = 1).
+// Only the block rows [m0,m1) x cols [n0,n1) is produced, densely packed.
+int orc_gemm(int64_t M, int64_t N, int64_t K, const uint16_t* A, int a_trans, const uint16_t* B, int b_trans,
+             int64_t m0, int64_t m1, int64_t n0, int64_t n1, float* ref32, double* ref64, uint16_t* out_bf16, int threads) {
+    if (M <= 0 || N <= 0 || K <= 0 || m0 < 0 || n0 < 0 || m1 > M || n1 > N || m0 >= m1 || n0 >= n1) return -1;
+    int64_t nb = n1 - n0, mb = m1 - m0;
+    // gather the needed columns of B as floats, [K x nb] (pure data movement)
+    std::vector<float> Bf((size_t)(K * nb));
+    for (int64_t k = 0; k < K; ++k)
+        for (int64_t j = 0; j < nb; ++j)
+            Bf[(size_t)(k * nb + j)] = bf16_to_f32(b_trans ? B[(n0 + j) * K + k] : B[k * N + n0 + j]);
+    if (threads < 1) threads = 1;
+    threads = (int)std::min<int64_t>(threads, mb);
+    auto work = [&](int64_t lo, int64_t hi) {
+        std::vector<float> acc((size_t)nb);
+        std::vector<double> acc64(ref64 ? (size_t)nb : 0);
+        for (int64_t i = lo; i < hi; ++i) {
+            std::fill(acc.begin(), acc.end(), 0.0f);
+            std::fill(acc64.begin(), acc64.end(), 0.0);
+            for (int64_t k = 0; k < K; ++k) {
+                float a = bf16_to_f32(a_trans ? A[k * M + (m0 + i)] : A[(m0 + i) * K + k]);
+                const float* brow = &Bf[(size_t)(k * nb)];
+                for (int64_t j = 0; j < nb; ++j) acc[(size_t)j] += a * brow[j];
+                if (ref64) for (int64_t j = 0; j < nb; ++j) acc64[(size_t)j] += (double)a * (double)brow[j];
+            }
+            for (int64_t j = 0; j < nb; ++j) {
+                if (ref32) ref32[i * nb + j] = acc[(size_t)j];
+                if (ref64) ref64[i * nb + j] = acc64[(size_t)j];
+                if (out_bf16) out_bf16[i * nb + j] = f32_to_bf16_rne(acc[(size_t)j]);
+            }
+        }
+    };
+    std::vector<std::thread> pool;
+    int64_t per = (mb + threads - 1) / threads;
+    for (int t = 0; t < threads; ++t) {
+        int64_t lo = t * per, hi = std::min(mb, lo + per);
+        if (lo < hi) pool.emplace_back(work, lo, hi);
+    }
+    for (auto& th : pool) th.join();
+    return 0;
+}
+
+uint16_t orc_f32_to_bf16(float f) { return f32_to_bf16_rne(f); }
+
+// Number of output tiles and of pages per operand.
+int orc_traffic_sizes(const orc_traffic_desc* d, int64_t* ntiles, int64_t* pages) {
+    if (!traffic_desc_ok(*d)) return -1;
+    std::vector<Tile> tiles;
+    std::vector<int32_t> zeros;
+    const int32_t* q = nullptr;
+    if (d->assign == ORC_ASSIGN_EXPLICIT) {   // count only: any valid assignment will do
+        int64_t n = (int64_t)tile_dim(d->M, d->BM, d->P, false).size() * (int64_t)tile_dim(d->N, d->BN, d->P, false).size();
+        zeros.assign((size_t)n, 0); q = zeros.data();
+    }
+    if (enumerate_tiles(*d, q, tiles)) return -1;
+    *ntiles = (int64_t)tiles.size();
+    pages[0] = pages_of(d->A, d->page_bytes); pages[1] = pages_of(d->B, d->page_bytes); pages[2] = pages_of(d->C, d->page_bytes);
+    return 0;
+}
+
+// Tile rectangles and chiplets, [ntiles][5] = m0, m1, n0, n1, q (for sampling and tests).
+int orc_traffic_tiles(const orc_traffic_desc* d, const int32_t* explicit_q, int64_t* out) {
+    if (!traffic_desc_ok(*d)) return -1;
+    std::vector<Tile> tiles;
+    if (enumerate_tiles(*d, explicit_q, tiles)) return -1;
+    for (size_t i = 0; i < tiles.size(); ++i) {
+        out[i * 5 + 0] = tiles[i].m0; out[i * 5 + 1] = tiles[i].m1; out[i * 5 + 2] = tiles[i].n0; out[i * 5 + 3] = tiles[i].n1; out[i * 5 + 4] = tiles[i].q;
+    }
+    return 0;
+}
+
+// Remote-traffic count (Sec. 4.1 metric without the L2 filter), element by element.
+//   per_cta  [ntiles][3 operands A,B,C][local, remote] bytes
+//   per_page [X][pages_X][P] bytes of the page demanded by each chiplet (any entry may be NULL)
+//   owner    [X][pages_X] chiplet the policy maps the page to
+//   totals   [3][2]
+int orc_traffic_elem(const orc_traffic_desc* d, const int32_t* explicit_q, uint64_t* per_cta, uint64_t* const* per_page,
+                     uint8_t* const* owner, uint64_t* totals) {
+    return traffic_impl<false>(*d, explicit_q, per_cta, per_page, owner, totals);
+}
+
+// The same count taken run by run (a stored row of a tile is one contiguous run per strip,
+// cut at page boundaries).  Validated against orc_traffic_elem in the tests; used at sizes
+// where the element walk would take minutes.
+int orc_traffic_runs(const orc_traffic_desc* d, const int32_t* explicit_q, uint64_t* per_cta, uint64_t* const* per_page,
+                     uint8_t* const* owner, uint64_t* totals) {
+    return traffic_impl<true>(*d, explicit_q, per_cta, per_page, owner, totals);
+}
+
+}  // extern "C"

@@ -1,0 +1,167 @@
+"""Pins for the oracle's address map (Eq. 1-3) and repack.  No GPU."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle as orc
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def ccl_cols(R, Cc, P, e=2, align=0):
+    return orc.Mat(R, Cc, e, P, orc.PART_COLS, orc.CCL, align)
+
+
+def ccl_rows(R, Cc, P, e=2, align=0):
+    return orc.Mat(R, Cc, e, P, orc.PART_ROWS, orc.CCL, align)
+
+
+def test_fig4a_worked_example():
+    rows = [l.split() for l in open(os.path.join(GOLD, "fig4a_ccl_index.txt")) if l.strip() and not l.startswith("#")]
+    hdr = {k: int(v) for k, v in rows[:3]}
+    table = np.array(rows[3:], dtype=np.int64)
+    assert table.shape == (hdr["K"], hdr["N"])
+    m = ccl_cols(hdr["K"], hdr["N"], hdr["G"])
+    np.testing.assert_array_equal(orc.map_table(m), table)
+    assert orc.map_offset(m, 1, 5) == 21           # row-major would give 13
+    # interleave granularity: 4 elements in row-major, 16 in CCL (contiguous run of one chiplet)
+    inv = np.empty(32, dtype=np.int64)
+    chip = np.repeat(np.arange(2), 4)[None, :].repeat(4, 0)           # chiplet of column n
+    inv[table.reshape(-1)] = chip.reshape(-1)
+    assert (inv[:16] == 0).all() and (inv[16:] == 1).all()
+    rm = chip.reshape(-1)                                              # row-major memory order
+    assert max(len(list(g)) for g in np.split(rm, np.flatnonzero(np.diff(rm)) + 1)) == 4
+
+
+@pytest.mark.parametrize("R,Cc,P", [(4, 8, 2), (7, 12, 3), (5, 200, 2), (64, 1536, 4), (33, 768, 8), (2048, 1536, 4), (768, 2048, 2)])
+def test_bijection_and_strips_packed(R, Cc, P):
+    m = ccl_cols(R, Cc, P)
+    t = orc.map_table(m)
+    flat = np.sort(t.reshape(-1))
+    np.testing.assert_array_equal(flat, np.arange(R * Cc))            # bijection onto [0, R*C)
+    w = Cc // P
+    for g in range(P):                                                # strip g is exactly [g*K*w, (g+1)*K*w)
+        s = t[:, g * w:(g + 1) * w]
+        assert s.min() == g * R * w and s.max() == (g + 1) * R * w - 1
+    assert orc.buffer_bytes(m) == R * Cc * 2
+
+
+@pytest.mark.parametrize("R,Cc,P", [(4, 8, 2), (7, 12, 3), (64, 1536, 4), (16, 768, 8)])
+def test_stride_form(R, Cc, P):
+    """Sec. 3.3: the view (K, G, N/G) with strides (w, K*w, 1)."""
+    w = Cc // P
+    k, g, n = np.meshgrid(np.arange(R), np.arange(P), np.arange(w), indexing="ij")
+    stride_form = (k * w + g * (R * w) + n * 1).reshape(R, Cc)
+    np.testing.assert_array_equal(orc.map_table(ccl_cols(R, Cc, P)), stride_form)
+
+
+def test_identity_cases():
+    R, Cc = 12, 40
+    rm = np.arange(R * Cc).reshape(R, Cc)
+    np.testing.assert_array_equal(orc.map_table(orc.Mat(R, Cc)), rm)                        # Eq. 2
+    np.testing.assert_array_equal(orc.map_table(ccl_cols(R, Cc, 1)), rm)                   # G = 1
+    np.testing.assert_array_equal(orc.map_table(ccl_rows(R, Cc, 4)), rm)                   # split along rows: already contiguous
+    np.testing.assert_array_equal(orc.map_table(orc.Mat(R, Cc, 2, 4, orc.PART_COLS, orc.ROWMAJOR)), rm)
+
+
+def test_slice_sizes_of_sec_2_2():
+    # widths 768, 4096, 14336; bf16; four chiplets -> row slices of 384 B, 2 KB, 7168 B
+    for width, nbytes in [(768, 384), (4096, 2048), (14336, 7168)]:
+        m = ccl_cols(3, width, 4)
+        run = orc.map_offset(m, 1, 0) - orc.map_offset(m, 0, 0)       # elements between consecutive rows of one strip
+        assert run * 2 == nbytes
+        assert orc.map_offset(m, 0, width // 4) == 3 * (width // 4)   # next chiplet's slice starts a new strip
+    # fused gate/up width 1536 over 4 chiplets -> 384-element slices (Fig. 3(a))
+    assert orc.map_offset(ccl_cols(2, 1536, 4), 1, 0) == 384
+
+
+@pytest.mark.parametrize("part", ["cols", "rows"])
+@pytest.mark.parametrize("align", [64, 4096])
+def test_aligned_strips_injective_and_inverse(part, align):
+    R, Cc, P = 6, 36, 3
+    m = ccl_cols(R, Cc, P, 2, align) if part == "cols" else ccl_rows(R, Cc, P, 2, align)
+    t = orc.map_table(m)
+    assert len(np.unique(t)) == R * Cc
+    st = orc.strip_stride(m)
+    assert (st * 2) % align == 0 and st * 2 >= R * Cc * 2 // P
+    assert orc.buffer_bytes(m) == P * st * 2
+    hit = np.zeros(P * st, dtype=bool)
+    hit[t.reshape(-1)] = True
+    for off in range(P * st):
+        rc, r, c = orc.map_inverse(m, off)
+        if hit[off]:
+            assert rc == 0 and t[r, c] == off
+        else:
+            assert rc == -2                                           # padding hole
+    assert orc.map_inverse(m, P * st)[0] == -1
+
+
+def test_inverse_packed_roundtrip():
+    m = ccl_cols(9, 40, 5)
+    t = orc.map_table(m)
+    for off in range(9 * 40):
+        rc, r, c = orc.map_inverse(m, off)
+        assert rc == 0 and t[r, c] == off
+
+
+def test_rejects_bad_descriptors():
+    with pytest.raises(ValueError):
+        orc.map_table(ccl_cols(4, 10, 4))          # w = N/G not whole
+    with pytest.raises(ValueError):
+        orc.map_table(ccl_rows(5, 8, 2))
+    with pytest.raises(ValueError):
+        orc.map_offset(ccl_cols(4, 8, 2), 4, 0)    # out of range
+    with pytest.raises(ValueError):
+        orc.map_table(orc.Mat(4, 8, 3))            # element size
+
+
+# ---------------------------------------------------------------- repack
+
+def _rand_u16(R, Cc, seed=0):
+    return np.random.default_rng(seed).integers(0, 65536, size=(R, Cc), dtype=np.uint16)
+
+
+@pytest.mark.parametrize("R,Cc,P", [(4, 8, 2), (130, 384, 4), (130, 384, 2), (5, 200, 2), (77, 96, 3), (256, 1536, 8)])
+def test_repack_is_reshape_permute(R, Cc, P):
+    x = _rand_u16(R, Cc, 1)
+    got = orc.repack(ccl_cols(R, Cc, P), x, 0)
+    want = torch.from_numpy(x.view(np.int16)).reshape(R, P, Cc // P).permute(1, 0, 2).contiguous().numpy().view(np.uint16)
+    np.testing.assert_array_equal(got, want.reshape(-1))
+    # equals P strided 2-D copies: strip g = columns [g*w, (g+1)*w) of every row
+    w = Cc // P
+    for g in range(P):
+        np.testing.assert_array_equal(got[g * R * w:(g + 1) * R * w].reshape(R, w), x[:, g * w:(g + 1) * w])
+    # a permutation: same multiset
+    np.testing.assert_array_equal(np.sort(got), np.sort(x.reshape(-1)))
+    # round trip
+    np.testing.assert_array_equal(orc.repack(ccl_cols(R, Cc, P), got, 1).reshape(R, Cc), x)
+
+
+def test_repack_p1_and_rows_are_memcpy():
+    x = _rand_u16(33, 50, 2)
+    np.testing.assert_array_equal(orc.repack(ccl_cols(33, 50, 1), x, 0), x.reshape(-1))
+    np.testing.assert_array_equal(orc.repack(ccl_rows(33, 50, 3), x, 0), x.reshape(-1))
+
+
+@pytest.mark.parametrize("e,dt", [(1, np.uint8), (2, np.uint16), (4, np.uint32)])
+def test_repack_aligned_padding_is_zero(e, dt):
+    R, Cc, P, align = 7, 24, 3, 256
+    x = np.random.default_rng(3).integers(1, 200, size=(R, Cc)).astype(dt)    # no zeros in the payload
+    m = ccl_cols(R, Cc, P, e, align)
+    got = orc.repack(m, x, 0)
+    st = orc.strip_stride(m)
+    assert got.size == P * st
+    w = Cc // P
+    for g in range(P):
+        np.testing.assert_array_equal(got[g * st:g * st + R * w].reshape(R, w), x[:, g * w:(g + 1) * w])
+        assert (got[g * st + R * w:(g + 1) * st] == 0).all()
+    np.testing.assert_array_equal(orc.repack(m, got, 1).reshape(R, Cc), x)
+    mr = ccl_rows(6, Cc, P, e, align)
+    xr = x[:6]
+    gr = orc.repack(mr, xr, 0)
+    sr = orc.strip_stride(mr)
+    for g in range(P):
+        np.testing.assert_array_equal(gr[g * sr:g * sr + 2 * Cc].reshape(2, Cc), xr[2 * g:2 * g + 2])
+        assert (gr[g * sr + 2 * Cc:(g + 1) * sr] == 0).all()
