@@ -1,0 +1,196 @@
+/*
+ * ccl.h -- C ABI of the B200 (sm_100a) hot path of Chiplet-Contiguous Layout (CCL).
+ *
+ * CCL stores a matrix so that the data consumed by one chiplet ("strip") is one
+ * contiguous region (paper Sec. 3).  This library provides the four operations on
+ * that path: the address map, the row-major <-> CCL repack, a bf16 GEMM whose
+ * operands and output are read/written in CCL, and a counter of local/remote HBM
+ * bytes that scores a layout against page-granularity placement.
+ *
+ * Conventions (all entry points)
+ *  - A "stored matrix" is rows x cols with cols contiguous in its row-major view.
+ *  - P is the chiplet count (the paper's G).  e = elem_bytes.
+ *  - Pointers named *_dev are DEVICE pointers on the current CUDA device; everything
+ *    else is a host pointer.  The caller owns every buffer; the library never
+ *    allocates or frees device memory and keeps no reference after a call returns.
+ *  - Device work is enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL =
+ *    the legacy default stream) and is asynchronous; no entry point synchronises.
+ *  - Input and output buffers of one call must not overlap.
+ *  - Every call returns a ccl_status and never aborts, throws or prints.  Arguments
+ *    are validated on the host before any launch; on error nothing is launched.
+ *    ccl_last_error() gives a thread-local message for the last failing call.
+ *  - There is no CPU fallback: without a CUDA device the device entry points return
+ *    CCL_ERR_CUDA.
+ */
+#ifndef CCL_H_
+#define CCL_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    CCL_OK = 0,
+    CCL_ERR_INVALID_ARG = 1, /* NULL pointer, unknown enum value, negative size                  */
+    CCL_ERR_SHAPE = 2,       /* split dimension not divisible by P, operand shapes inconsistent */
+    CCL_ERR_ALIGN = 3,       /* pointer / stride not aligned as the operation needs             */
+    CCL_ERR_UNSUPPORTED = 4, /* valid request this build cannot run (e.g. GEMM with w % 8 != 0) */
+    CCL_ERR_CUDA = 5,        /* a CUDA runtime/driver call failed                               */
+    CCL_ERR_WORKSPACE = 6,   /* workspace / required output buffer missing or too small        */
+    CCL_ERR_TIMEOUT = 7,     /* a bounded device-side wait expired (see ccl_gemm_status)        */
+    CCL_ERR_PADDING = 8      /* inverse map: the offset lies in alignment padding               */
+} ccl_status;
+
+typedef enum { CCL_ROWMAJOR = 0, CCL_CCL = 1 } ccl_layout;                   /* physical order of a buffer */
+typedef enum { CCL_PART_NONE = 0, CCL_PART_ROWS = 1, CCL_PART_COLS = 2 } ccl_part; /* stored dim split over chiplets */
+
+/*
+ * Descriptor of one stored matrix.
+ *   layout = CCL_ROWMAJOR : offset(r,c) = r*cols + c                         (Eq. 2)
+ *   layout = CCL_CCL, part = CCL_PART_COLS (the paper's case, Eq. 1 + Eq. 3):
+ *       w = cols/P, g = c / w, c' = c mod w, offset = g*stride + r*w + c'
+ *       stride = rows*w when strip_align_bytes == 0 (packed, Eq. 3 literally), else
+ *       rows*w*e rounded up to strip_align_bytes (Sec. 3.2: a strip can be aligned to
+ *       the placement granularity).  Padding elements belong to no (r,c).
+ *   layout = CCL_CCL, part = CCL_PART_ROWS (split along the non-contiguous dimension,
+ *       which Sec. 2.2 calls coarse-grained: already contiguous):
+ *       h = rows/P, offset = (r / h)*stride + (r mod h)*cols + c, stride = h*cols
+ *       (rounded up likewise).
+ *   layout = CCL_CCL with part = CCL_PART_NONE behaves as CCL_ROWMAJOR.
+ * Requirements: rows, cols > 0; elem_bytes in {1,2,4}; P >= 1; the split dimension
+ * divisible by P (else CCL_ERR_SHAPE); strip_align_bytes >= 0 and a multiple of e.
+ */
+typedef struct ccl_mat {
+    int64_t rows, cols;
+    int32_t elem_bytes;
+    int32_t P;
+    int32_t part;   /* ccl_part   */
+    int32_t layout; /* ccl_layout */
+    int64_t strip_align_bytes;
+} ccl_mat;
+
+/* ---- address map (Eq. 1-3; host, pure, O(1)) ------------------------------------------- */
+
+/* Element offset of stored coordinate (r,c). CCL_ERR_INVALID_ARG if (r,c) is out of range. */
+ccl_status ccl_map_offset(const ccl_mat* m, int64_t r, int64_t c, int64_t* elem_off);
+/* Inverse of the above. CCL_ERR_PADDING if elem_off is a padding element. */
+ccl_status ccl_map_inverse(const ccl_mat* m, int64_t elem_off, int64_t* r, int64_t* c);
+/* Size in bytes of the buffer the descriptor addresses, padding included (P*stride*e for CCL). */
+ccl_status ccl_buffer_bytes(const ccl_mat* m, int64_t* bytes);
+/* Elements between the bases of consecutive strips (CCL layouts only). */
+ccl_status ccl_strip_stride(const ccl_mat* m, int64_t* elems);
+
+/* ---- repack (Sec. 3.3: operands adopt CCL at load time or are repacked) ---------------- */
+
+/*
+ * Permutation copy on the device.
+ *   dir = 0: src_dev is row-major [rows x cols]; dst_dev receives the layout `m` describes
+ *            (ccl_buffer_bytes(m) bytes); padding bytes are written as zero.
+ *   dir = 1: src_dev is in the layout `m` describes; dst_dev receives row-major.
+ * Any shape the map accepts is accepted; base pointers must be aligned to elem_bytes.
+ * 16-byte aligned bases with (w*e) % 16 == 0 and (stride*e) % 16 == 0 take the fast path.
+ */
+ccl_status ccl_repack(const ccl_mat* m, const void* src_dev, void* dst_dev, int dir, void* cuda_stream);
+
+/* ---- GEMM on CCL operands (Sec. 2.2 execution model, Sec. 3.3 "only the address map changes") */
+
+/*
+ * C[M x N] = A[M x K] * B[K x N]; bf16 inputs, fp32 accumulation, bf16 output rounded to
+ * nearest-even.  Each operand is described by its own ccl_mat and may be row-major or CCL:
+ *   A stored [M x K] (a_trans = 0) or [K x M] (a_trans = 1);
+ *   B stored [K x N] (b_trans = 0) or [N x K] (b_trans = 1);   C stored [M x N].
+ * out_part / P / grouped_raster describe how C is partitioned over chiplets and whether CTA
+ * group g computes only strip g of C (Sec. 3.1: each CTA runs on the chiplet that owns its
+ * output tile): out_part = CCL_PART_COLS splits N, CCL_PART_ROWS splits M, CCL_PART_NONE (or
+ * grouped_raster = 0) uses one plain raster.  The result does not depend on these choices.
+ * Requirements (else CCL_ERR_UNSUPPORTED / CCL_ERR_ALIGN, nothing launched): elem_bytes = 2;
+ * every contiguous extent a tile row lives in (cols, or w for CCL_PART_COLS) a multiple of 8
+ * elements; strip strides multiples of 16 bytes; base pointers 16-byte aligned.
+ */
+typedef struct ccl_gemm_desc {
+    int64_t M, N, K;
+    ccl_mat A, B, C;
+    int32_t a_trans, b_trans;
+    int32_t out_part; /* ccl_part */
+    int32_t P;
+    int32_t grouped_raster;
+} ccl_gemm_desc;
+
+/* Bytes of device workspace ccl_gemm needs for this problem (0 when none). */
+ccl_status ccl_gemm_workspace(const ccl_gemm_desc* d, size_t* bytes);
+/*
+ * Enqueue the GEMM.  ws_dev may be NULL when ccl_gemm_workspace reports 0.
+ * Device-side waits are bounded; if one expires the kernel stores a non-zero code in an
+ * internal status word and returns early (C is then incomplete): see ccl_gemm_status.
+ */
+ccl_status ccl_gemm(const ccl_gemm_desc* d, const void* A_dev, const void* B_dev, void* C_dev, void* ws_dev,
+                    size_t ws_bytes, void* cuda_stream);
+/*
+ * Synchronises `cuda_stream`, then reports and clears the status word of GEMMs finished on
+ * the current device: CCL_OK, or CCL_ERR_TIMEOUT with *detail = the raw device code.
+ * detail may be NULL.
+ */
+ccl_status ccl_gemm_status(void* cuda_stream, int32_t* detail);
+
+/* ---- remote-traffic counter (Sec. 4.1 metric, every touched byte counted: no L2 filter) */
+
+typedef enum { CCL_PLACE_RR = 0, CCL_PLACE_BLOCK = 1, CCL_PLACE_BEST = 2 } ccl_place;
+typedef enum { CCL_ASSIGN_N_STRIPS = 0, CCL_ASSIGN_M_STRIPS = 1, CCL_ASSIGN_EXPLICIT = 2 } ccl_assign;
+
+/*
+ * One CTA per BM x BN output tile (Sec. 2.2); it reads its rows of A over all K, its
+ * columns of B over all K, and writes its tile of C.  Every operand is an allocation of
+ * its own whose base is page 0.  A page of `page_bytes` is owned by one chiplet:
+ *   CCL_PLACE_RR    : owner = page mod P            (fixed round-robin interleave, Sec. 4.1)
+ *   CCL_PLACE_BLOCK : owner = min(P-1, page*page_bytes*P / buffer_bytes): P equal contiguous
+ *                     address blocks (coarse placement, Sec. 4.1); on a CCL buffer whose
+ *                     strips are whole pages this is "page -> its strip's chiplet"
+ *   CCL_PLACE_BEST  : owner = the chiplet that demands most bytes of the page (ties: lowest
+ *                     index; untouched pages: 0): the best any page-granular mapping can do.
+ * Tile -> chiplet: CCL_ASSIGN_N_STRIPS: the strip (width N/P) holding the tile's first column;
+ * CCL_ASSIGN_M_STRIPS likewise along M; CCL_ASSIGN_EXPLICIT: cta_chiplet_dev[tile].
+ * strip_tiling = 1 tiles every strip of the assignment dimension on its own (tiles never
+ * straddle strips, the last tile of a strip may be partial); 0 tiles globally.  Tiles are
+ * numbered tile_m * tiles_n + tile_n.  Partial tiles touch only valid elements.
+ */
+typedef struct ccl_traffic_desc {
+    int64_t M, N, K;
+    int32_t BM, BN;
+    ccl_mat A, B, C;
+    int32_t a_trans, b_trans;
+    int32_t P;
+    int64_t page_bytes; /* > 0, multiple of every operand's elem_bytes */
+    int32_t place[3];   /* ccl_place for A, B, C */
+    int32_t assign;     /* ccl_assign */
+    int32_t strip_tiling;
+} ccl_traffic_desc;
+
+/* Number of tiles and of pages per operand (sizes of the output arrays below). */
+ccl_status ccl_traffic_sizes(const ccl_traffic_desc* d, int64_t* ntiles, int64_t pages[3]);
+/*
+ * Outputs (device; every one is fully overwritten):
+ *   per_cta_dev  uint64 [ntiles][3 (A,B,C)][2 (local, remote)] bytes        (required)
+ *   per_page_dev[X] uint64 [pages_X][P] bytes of page demanded per chiplet  (NULL = not wanted;
+ *                required for an operand placed with CCL_PLACE_BEST, else CCL_ERR_WORKSPACE)
+ *   owner_dev[X] uint8 [pages_X] owning chiplet                              (same rule)
+ *   totals_dev   uint64 [3][2]                                               (required)
+ * per_page_dev / owner_dev are HOST arrays of three device pointers (or NULL altogether).
+ * cta_chiplet_dev: int32 [ntiles], values in [0,P); only read for CCL_ASSIGN_EXPLICIT.
+ * Out-of-range entries are counted as chiplet 0 ... never dereferenced out of bounds.
+ */
+ccl_status ccl_traffic(const ccl_traffic_desc* d, const int32_t* cta_chiplet_dev, uint64_t* per_cta_dev,
+                       uint64_t* const per_page_dev[3], uint8_t* const owner_dev[3], uint64_t* totals_dev,
+                       void* cuda_stream);
+
+/* Message for the last non-OK status returned on this thread ("" if none). Static storage. */
+const char* ccl_last_error(void);
+/* Library version, "major.minor". */
+const char* ccl_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CCL_H_ */

@@ -1,0 +1,164 @@
+"""Thin ctypes binding of the C-ABI library declared in include/ccl.h.
+
+Argument marshalling only: every step runs in the CUDA kernels of libccl.so.  Tensors are
+torch CUDA tensors used as plain device buffers; the stream is torch's current stream.
+There is no CPU fallback: if libccl.so is missing the import of this module's functions
+raises, and device entry points fail without a CUDA device.
+"""
+import ctypes as C
+import os
+
+import torch
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libccl.so")
+
+OK, ERR_INVALID_ARG, ERR_SHAPE, ERR_ALIGN, ERR_UNSUPPORTED, ERR_CUDA, ERR_WORKSPACE, ERR_TIMEOUT, ERR_PADDING = range(9)
+ROWMAJOR, CCL = 0, 1
+PART_NONE, PART_ROWS, PART_COLS = 0, 1, 2
+PLACE_RR, PLACE_BLOCK, PLACE_BEST = 0, 1, 2
+ASSIGN_N_STRIPS, ASSIGN_M_STRIPS, ASSIGN_EXPLICIT = 0, 1, 2
+
+EXPORTS = ["ccl_map_offset", "ccl_map_inverse", "ccl_buffer_bytes", "ccl_strip_stride", "ccl_repack", "ccl_gemm_workspace",
+           "ccl_gemm", "ccl_gemm_status", "ccl_traffic_sizes", "ccl_traffic", "ccl_last_error", "ccl_version"]
+
+
+class CclError(RuntimeError):
+    def __init__(self, status, message):
+        super().__init__(f"ccl status {status}: {message}")
+        self.status = status
+
+
+class Mat(C.Structure):
+    """ccl_mat"""
+    _fields_ = [("rows", C.c_int64), ("cols", C.c_int64), ("elem_bytes", C.c_int32), ("P", C.c_int32),
+                ("part", C.c_int32), ("layout", C.c_int32), ("strip_align_bytes", C.c_int64)]
+
+    def __init__(self, rows=0, cols=0, elem_bytes=2, P=1, part=PART_NONE, layout=ROWMAJOR, strip_align_bytes=0):
+        super().__init__(rows, cols, elem_bytes, P, part, layout, strip_align_bytes)
+
+
+class GemmDesc(C.Structure):
+    """ccl_gemm_desc"""
+    _fields_ = [("M", C.c_int64), ("N", C.c_int64), ("K", C.c_int64), ("A", Mat), ("B", Mat), ("C", Mat),
+                ("a_trans", C.c_int32), ("b_trans", C.c_int32), ("out_part", C.c_int32), ("P", C.c_int32),
+                ("grouped_raster", C.c_int32)]
+
+
+class TrafficDesc(C.Structure):
+    """ccl_traffic_desc"""
+    _fields_ = [("M", C.c_int64), ("N", C.c_int64), ("K", C.c_int64), ("BM", C.c_int32), ("BN", C.c_int32),
+                ("A", Mat), ("B", Mat), ("C", Mat), ("a_trans", C.c_int32), ("b_trans", C.c_int32), ("P", C.c_int32),
+                ("page_bytes", C.c_int64), ("place", C.c_int32 * 3), ("assign", C.c_int32), ("strip_tiling", C.c_int32)]
+
+
+_lib = None
+
+
+def lib():
+    """Loads libccl.so (built by paper_2606_11718_b200.build); raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} not found: build it with `python -m paper_2606_11718_b200.build` "
+                              "(there is no fallback path)")
+        l = C.CDLL(LIB_PATH)
+        l.ccl_last_error.restype = C.c_char_p
+        l.ccl_version.restype = C.c_char_p
+        l.ccl_map_offset.argtypes = [C.POINTER(Mat), C.c_int64, C.c_int64, C.POINTER(C.c_int64)]
+        l.ccl_map_inverse.argtypes = [C.POINTER(Mat), C.c_int64, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
+        l.ccl_buffer_bytes.argtypes = [C.POINTER(Mat), C.POINTER(C.c_int64)]
+        l.ccl_strip_stride.argtypes = [C.POINTER(Mat), C.POINTER(C.c_int64)]
+        l.ccl_repack.argtypes = [C.POINTER(Mat), C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]
+        l.ccl_gemm_workspace.argtypes = [C.POINTER(GemmDesc), C.POINTER(C.c_size_t)]
+        l.ccl_gemm.argtypes = [C.POINTER(GemmDesc), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+        l.ccl_gemm_status.argtypes = [C.c_void_p, C.POINTER(C.c_int32)]
+        l.ccl_traffic_sizes.argtypes = [C.POINTER(TrafficDesc), C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
+        l.ccl_traffic.argtypes = [C.POINTER(TrafficDesc), C.c_void_p, C.c_void_p, C.POINTER(C.c_void_p), C.POINTER(C.c_void_p),
+                                  C.c_void_p, C.c_void_p]
+        _lib = l
+    return _lib
+
+
+def _check(status):
+    if status != OK:
+        raise CclError(status, lib().ccl_last_error().decode())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _ptr(t):
+    return C.c_void_p(t.data_ptr()) if t is not None else None
+
+
+def ccl_version():
+    return lib().ccl_version().decode()
+
+
+def ccl_map_offset(m, r, c):
+    off = C.c_int64()
+    _check(lib().ccl_map_offset(C.byref(m), r, c, C.byref(off)))
+    return off.value
+
+
+def ccl_map_inverse(m, elem_off):
+    r, c = C.c_int64(), C.c_int64()
+    _check(lib().ccl_map_inverse(C.byref(m), elem_off, C.byref(r), C.byref(c)))
+    return r.value, c.value
+
+
+def ccl_buffer_bytes(m):
+    b = C.c_int64()
+    _check(lib().ccl_buffer_bytes(C.byref(m), C.byref(b)))
+    return b.value
+
+
+def ccl_strip_stride(m):
+    b = C.c_int64()
+    _check(lib().ccl_strip_stride(C.byref(m), C.byref(b)))
+    return b.value
+
+
+def ccl_repack(m, src, dst, direction=0):
+    """src, dst: CUDA tensors (any dtype; only their bytes matter)."""
+    need_src = m.rows * m.cols * m.elem_bytes if direction == 0 else ccl_buffer_bytes(m)
+    need_dst = ccl_buffer_bytes(m) if direction == 0 else m.rows * m.cols * m.elem_bytes
+    if src.numel() * src.element_size() < need_src or dst.numel() * dst.element_size() < need_dst:
+        raise ValueError("ccl_repack: buffer too small")
+    _check(lib().ccl_repack(C.byref(m), _ptr(src), _ptr(dst), direction, _stream()))
+
+
+def ccl_gemm_workspace(d):
+    n = C.c_size_t()
+    _check(lib().ccl_gemm_workspace(C.byref(d), C.byref(n)))
+    return n.value
+
+
+def ccl_gemm(d, A, B, Cout, ws=None):
+    for t, m in ((A, d.A), (B, d.B), (Cout, d.C)):
+        if t.numel() * t.element_size() < ccl_buffer_bytes(m):
+            raise ValueError("ccl_gemm: operand buffer too small")
+    ws_bytes = ws.numel() * ws.element_size() if ws is not None else 0
+    _check(lib().ccl_gemm(C.byref(d), _ptr(A), _ptr(B), _ptr(Cout), _ptr(ws), ws_bytes, _stream()))
+
+
+def ccl_gemm_status():
+    detail = C.c_int32()
+    st = lib().ccl_gemm_status(_stream(), C.byref(detail))
+    return st, detail.value
+
+
+def ccl_traffic_sizes(d):
+    nt = C.c_int64()
+    pages = (C.c_int64 * 3)()
+    _check(lib().ccl_traffic_sizes(C.byref(d), C.byref(nt), pages))
+    return nt.value, list(pages)
+
+
+def ccl_traffic(d, per_cta, totals, per_page=None, owner=None, cta_chiplet=None):
+    """per_cta: uint64-sized CUDA tensor [ntiles,3,2]; totals [3,2]; per_page / owner: lists of 3 tensors or None."""
+    pp = (C.c_void_p * 3)(*[(t.data_ptr() if t is not None else None) for t in per_page]) if per_page is not None else None
+    ow = (C.c_void_p * 3)(*[(t.data_ptr() if t is not None else None) for t in owner]) if owner is not None else None
+    _check(lib().ccl_traffic(C.byref(d), _ptr(cta_chiplet), _ptr(per_cta), pp, ow, _ptr(totals), _stream()))

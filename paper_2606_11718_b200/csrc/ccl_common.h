@@ -1,0 +1,59 @@
+// Internal helpers of the CCL library: status/error text, descriptor validation and the
+// address-map arithmetic (Eq. 1-3) shared by the host entry points and the kernels.
+#pragma once
+
+#include <cstdarg>
+#include <cstdint>
+#include <cstdio>
+
+#include <cuda_runtime.h>
+
+#include "ccl.h"
+
+#if defined(__CUDACC__)
+#define CCL_HD __host__ __device__ __forceinline__
+#else
+#define CCL_HD inline
+#endif
+
+namespace ccl {
+
+ccl_status fail(ccl_status s, const char* fmt, ...);   // records the thread-local message, returns s
+void clear_error();
+
+#define CCL_CUDA_TRY(expr)                                                                      \
+    do {                                                                                        \
+        cudaError_t e__ = (expr);                                                               \
+        if (e__ != cudaSuccess) return ::ccl::fail(CCL_ERR_CUDA, "%s: %s", #expr, cudaGetErrorString(e__)); \
+    } while (0)
+
+// Flattened view of a ccl_mat: everything a kernel needs to address it.
+//   offset(r,c) = (r / h) * stride + (r % h) * w_row ... see map() below.
+struct MatView {
+    int64_t rows, cols;
+    int64_t w;        // width of a strip row in elements (cols/P for PART_COLS, else cols)
+    int64_t h;        // rows per strip (rows/P for PART_ROWS, else rows)
+    int64_t stride;   // elements between strip bases (0 when there is a single strip)
+    int64_t nstrips;  // P for CCL layouts, else 1
+    int32_t e;        // element bytes
+    int32_t split;    // 0 none, 1 rows, 2 cols (effective: 0 for row-major)
+};
+
+CCL_HD int64_t map(const MatView& v, int64_t r, int64_t c) {
+    if (v.split == 2) {                      // Eq. 1 + Eq. 3
+        int64_t g = c / v.w, cp = c - g * v.w;
+        return g * v.stride + r * v.w + cp;
+    }
+    if (v.split == 1) {                      // strips of h whole rows
+        int64_t g = r / v.h, rp = r - g * v.h;
+        return g * v.stride + rp * v.cols + c;
+    }
+    return r * v.cols + c;                   // Eq. 2
+}
+
+CCL_HD int64_t buffer_elems(const MatView& v) { return v.split ? v.nstrips * v.stride : v.rows * v.cols; }
+
+// Validates a descriptor and flattens it.  `what` names the argument in error messages.
+ccl_status make_view(const ccl_mat* m, const char* what, MatView* out);
+
+}  // namespace ccl

@@ -1,0 +1,115 @@
+// Host-only entry points: the address map (Eq. 1-3), sizes, error text.
+#include <cstring>
+
+#include "ccl_common.h"
+
+namespace ccl {
+
+static thread_local char g_err[512] = "";
+
+ccl_status fail(ccl_status s, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return s;
+}
+
+void clear_error() { g_err[0] = 0; }
+
+ccl_status make_view(const ccl_mat* m, const char* what, MatView* out) {
+    if (!m) return fail(CCL_ERR_INVALID_ARG, "%s: NULL descriptor", what);
+    if (m->rows <= 0 || m->cols <= 0) return fail(CCL_ERR_INVALID_ARG, "%s: rows and cols must be positive", what);
+    if (m->elem_bytes != 1 && m->elem_bytes != 2 && m->elem_bytes != 4)
+        return fail(CCL_ERR_INVALID_ARG, "%s: elem_bytes must be 1, 2 or 4", what);
+    if (m->P < 1) return fail(CCL_ERR_INVALID_ARG, "%s: P must be >= 1", what);
+    if (m->layout != CCL_ROWMAJOR && m->layout != CCL_CCL) return fail(CCL_ERR_INVALID_ARG, "%s: unknown layout", what);
+    if (m->part != CCL_PART_NONE && m->part != CCL_PART_ROWS && m->part != CCL_PART_COLS)
+        return fail(CCL_ERR_INVALID_ARG, "%s: unknown part", what);
+    if (m->strip_align_bytes < 0 || m->strip_align_bytes % m->elem_bytes)
+        return fail(CCL_ERR_INVALID_ARG, "%s: strip_align_bytes must be a non-negative multiple of elem_bytes", what);
+    // keep every byte offset comfortably inside int64
+    if (m->rows > (INT64_C(1) << 40) || m->cols > (INT64_C(1) << 40) ||
+        (double)m->rows * (double)m->cols * m->elem_bytes > 9.0e17)
+        return fail(CCL_ERR_INVALID_ARG, "%s: matrix too large", what);
+    MatView v;
+    v.rows = m->rows; v.cols = m->cols; v.e = m->elem_bytes;
+    v.w = m->cols; v.h = m->rows; v.stride = 0; v.nstrips = 1; v.split = 0;
+    if (m->layout == CCL_CCL && m->part != CCL_PART_NONE) {
+        int64_t packed;
+        if (m->part == CCL_PART_COLS) {
+            if (m->cols % m->P) return fail(CCL_ERR_SHAPE, "%s: cols (%lld) not divisible by P (%d)", what, (long long)m->cols, m->P);
+            v.w = m->cols / m->P; packed = m->rows * v.w; v.split = 2;
+        } else {
+            if (m->rows % m->P) return fail(CCL_ERR_SHAPE, "%s: rows (%lld) not divisible by P (%d)", what, (long long)m->rows, m->P);
+            v.h = m->rows / m->P; packed = v.h * m->cols; v.split = 1;
+        }
+        v.nstrips = m->P;
+        if (m->strip_align_bytes) {
+            int64_t a = m->strip_align_bytes, bytes = packed * m->elem_bytes;
+            v.stride = (bytes + a - 1) / a * a / m->elem_bytes;
+        } else {
+            v.stride = packed;
+        }
+    }
+    *out = v;
+    return CCL_OK;
+}
+
+}  // namespace ccl
+
+using namespace ccl;
+
+extern "C" {
+
+ccl_status ccl_map_offset(const ccl_mat* m, int64_t r, int64_t c, int64_t* elem_off) {
+    MatView v;
+    ccl_status s = make_view(m, "ccl_map_offset", &v);
+    if (s) return s;
+    if (!elem_off) return fail(CCL_ERR_INVALID_ARG, "ccl_map_offset: NULL output");
+    if (r < 0 || c < 0 || r >= v.rows || c >= v.cols) return fail(CCL_ERR_INVALID_ARG, "ccl_map_offset: (r,c) out of range");
+    *elem_off = map(v, r, c);
+    return CCL_OK;
+}
+
+ccl_status ccl_map_inverse(const ccl_mat* m, int64_t off, int64_t* r, int64_t* c) {
+    MatView v;
+    ccl_status s = make_view(m, "ccl_map_inverse", &v);
+    if (s) return s;
+    if (!r || !c) return fail(CCL_ERR_INVALID_ARG, "ccl_map_inverse: NULL output");
+    if (off < 0 || off >= buffer_elems(v)) return fail(CCL_ERR_INVALID_ARG, "ccl_map_inverse: offset out of range");
+    if (v.split == 0) { *r = off / v.cols; *c = off % v.cols; return CCL_OK; }
+    int64_t g = off / v.stride, rem = off % v.stride;
+    if (v.split == 2) {
+        if (rem >= v.rows * v.w) return fail(CCL_ERR_PADDING, "ccl_map_inverse: offset lies in the padding of strip %lld", (long long)g);
+        *r = rem / v.w; *c = g * v.w + rem % v.w;
+    } else {
+        if (rem >= v.h * v.cols) return fail(CCL_ERR_PADDING, "ccl_map_inverse: offset lies in the padding of strip %lld", (long long)g);
+        *r = g * v.h + rem / v.cols; *c = rem % v.cols;
+    }
+    return CCL_OK;
+}
+
+ccl_status ccl_buffer_bytes(const ccl_mat* m, int64_t* bytes) {
+    MatView v;
+    ccl_status s = make_view(m, "ccl_buffer_bytes", &v);
+    if (s) return s;
+    if (!bytes) return fail(CCL_ERR_INVALID_ARG, "ccl_buffer_bytes: NULL output");
+    *bytes = buffer_elems(v) * v.e;
+    return CCL_OK;
+}
+
+ccl_status ccl_strip_stride(const ccl_mat* m, int64_t* elems) {
+    MatView v;
+    ccl_status s = make_view(m, "ccl_strip_stride", &v);
+    if (s) return s;
+    if (!elems) return fail(CCL_ERR_INVALID_ARG, "ccl_strip_stride: NULL output");
+    if (v.split == 0) return fail(CCL_ERR_INVALID_ARG, "ccl_strip_stride: not a CCL layout");
+    *elems = v.stride;
+    return CCL_OK;
+}
+
+const char* ccl_last_error(void) { return g_err; }
+const char* ccl_version(void) { return "0.1"; }
+
+}  // extern "C"

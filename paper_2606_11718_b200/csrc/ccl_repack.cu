@@ -1,0 +1,293 @@
+// ccl_repack: row-major <-> CCL permutation copy (Sec. 3.3).
+//
+// Both directions are one strided 3-D copy over (strip g, row r of the strip, bytes of the row):
+//   split along columns (Eq. 3): row-major side  g*w*e + r*C*e,   CCL side  g*stride*e + r*w*e
+//   split along rows           : row-major side  g*h*C*e + r*C*e, CCL side  g*stride*e + r*C*e
+// The work is pure HBM streaming (read once + write once).  Two kernels:
+//   * repack_tma_kernel  -- one thread per CTA drives a ring of TMA tile loads and TMA tile
+//     stores through shared memory (rank-3 tensor maps on both sides), so ~200 KB per SM
+//     is in flight with no per-byte instruction cost.  Needs 16-byte alignment everywhere.
+//   * repack_vec_kernel  -- plain vectorised loads/stores for every other shape
+//     (vector width = the largest power of two that divides all extents and addresses).
+#include <algorithm>
+#include <cstdlib>
+#include <cstring>
+
+#include "ccl_common.h"
+#include "ccl_tma.h"
+
+namespace ccl {
+
+struct CopyPlan {
+    int64_t nstrips, rows, row_bytes;         // rows per strip, bytes per strip row
+    int64_t src_g, src_r, dst_g, dst_r;       // byte strides
+    int64_t pad_off, pad_bytes, pad_g;        // dir 0: zero dst[g*pad_g + pad_off, +pad_bytes) for every strip
+};
+
+__device__ int g_repack_status = 0;
+
+// ------------------------------------------------------------------------------------------
+// Vector path
+// ------------------------------------------------------------------------------------------
+template <typename V>
+__device__ __forceinline__ V ld_stream(const V* p) { return __ldcs(p); }
+template <typename V>
+__device__ __forceinline__ void st_stream(V* p, V v) { __stcs(p, v); }
+template <>
+__device__ __forceinline__ unsigned char ld_stream(const unsigned char* p) { return *p; }
+template <>
+__device__ __forceinline__ void st_stream(unsigned char* p, unsigned char v) { *p = v; }
+template <>
+__device__ __forceinline__ unsigned short ld_stream(const unsigned short* p) { return *p; }
+template <>
+__device__ __forceinline__ void st_stream(unsigned short* p, unsigned short v) { *p = v; }
+
+constexpr int kVecThreads = 256;
+constexpr int kVecUnroll = 4;
+
+template <typename V, typename IDX>
+__global__ void __launch_bounds__(kVecThreads) repack_vec_kernel(const char* __restrict__ src, char* __restrict__ dst, CopyPlan p,
+                                                                 IDX chunks_per_row, IDX chunks_per_strip) {
+    const int64_t g = blockIdx.y;
+    const char* s = src + g * p.src_g;
+    char* d = dst + g * p.dst_g;
+    const IDX step = (IDX)gridDim.x * kVecThreads * kVecUnroll;
+    for (IDX base = (IDX)blockIdx.x * kVecThreads * kVecUnroll + threadIdx.x; base < chunks_per_strip; base += step) {
+        V v[kVecUnroll];
+        int64_t doff[kVecUnroll];
+#pragma unroll
+        for (int u = 0; u < kVecUnroll; ++u) {
+            IDX j = base + (IDX)u * kVecThreads;
+            doff[u] = -1;
+            if (j < chunks_per_strip) {
+                IDX r = j / chunks_per_row;
+                IDX x = j - r * chunks_per_row;
+                v[u] = ld_stream(reinterpret_cast<const V*>(s + (int64_t)r * p.src_r + (int64_t)x * (int64_t)sizeof(V)));
+                doff[u] = (int64_t)r * p.dst_r + (int64_t)x * (int64_t)sizeof(V);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kVecUnroll; ++u)
+            if (doff[u] >= 0) st_stream(reinterpret_cast<V*>(d + doff[u]), v[u]);
+    }
+}
+
+template <typename V>
+__global__ void zero_pad_kernel(char* dst, int64_t pad_g, int64_t pad_off, int64_t chunks) {
+    char* d = dst + (int64_t)blockIdx.y * pad_g + pad_off;
+    V z;
+    memset(&z, 0, sizeof(V));
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < chunks; i += (int64_t)gridDim.x * blockDim.x)
+        reinterpret_cast<V*>(d)[i] = z;
+}
+
+// ------------------------------------------------------------------------------------------
+// TMA path: tile = box of (bx 8-byte units) x (by rows) of one strip
+// ------------------------------------------------------------------------------------------
+constexpr int kTmaStages = 6;
+constexpr int kTmaStageBytes = 32768;
+
+struct TmaTiling {
+    uint32_t bx, by;              // box extents (8-byte units, rows)
+    uint32_t tiles_x, tiles_y;    // per strip
+    uint64_t ntiles;
+};
+
+__global__ void __launch_bounds__(32, 1) repack_tma_kernel(const __grid_constant__ CUtensorMap src_map,
+                                                           const __grid_constant__ CUtensorMap dst_map, TmaTiling t) {
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    // stage buffers first (128-byte aligned), barriers after them
+    unsigned char* stage0 = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
+    uint64_t* full = reinterpret_cast<uint64_t*>(stage0 + (size_t)kTmaStages * kTmaStageBytes);
+    if (threadIdx.x != 0) return;
+
+    prefetch_tmap(&src_map);
+    prefetch_tmap(&dst_map);
+    for (int s = 0; s < kTmaStages; ++s) mbar_init(&full[s], 1);
+    fence_barrier_init();
+
+    const uint32_t box_bytes = t.bx * t.by * 8u;
+    const uint64_t per_strip = (uint64_t)t.tiles_x * t.tiles_y;
+    auto issue_load = [&](uint64_t it) {
+        uint64_t tile = (uint64_t)blockIdx.x + it * gridDim.x;
+        if (tile >= t.ntiles) return;
+        uint32_t slot = (uint32_t)(it % kTmaStages);
+        uint32_t g = (uint32_t)(tile / per_strip);
+        uint32_t rem = (uint32_t)(tile - (uint64_t)g * per_strip);
+        uint32_t ty = rem / t.tiles_x, tx = rem - ty * t.tiles_x;
+        mbar_expect_tx(&full[slot], box_bytes);
+        tma_load_3d(stage0 + (size_t)slot * kTmaStageBytes, &src_map, &full[slot], (int)(tx * t.bx), (int)(ty * t.by), (int)g);
+    };
+
+    for (uint64_t it = 0; it < kTmaStages; ++it) issue_load(it);
+    for (uint64_t it = 0;; ++it) {
+        uint64_t tile = (uint64_t)blockIdx.x + it * gridDim.x;
+        if (tile >= t.ntiles) break;
+        uint32_t slot = (uint32_t)(it % kTmaStages);
+        uint32_t parity = (uint32_t)((it / kTmaStages) & 1);
+        if (!mbar_wait_bounded(&full[slot], parity)) { atomicExch(&g_repack_status, 1); break; }
+        uint32_t g = (uint32_t)(tile / per_strip);
+        uint32_t rem = (uint32_t)(tile - (uint64_t)g * per_strip);
+        uint32_t ty = rem / t.tiles_x, tx = rem - ty * t.tiles_x;
+        tma_store_3d(&dst_map, stage0 + (size_t)slot * kTmaStageBytes, (int)(tx * t.bx), (int)(ty * t.by), (int)g);
+        tma_store_commit();
+        // the store issued one iteration ago has now read its buffer: refill that slot
+        if (it >= 1) {
+            tma_store_wait_read<1>();
+            issue_load(it - 1 + kTmaStages);
+        }
+    }
+    tma_store_wait_all<0>();
+}
+
+// ------------------------------------------------------------------------------------------
+// Host side
+// ------------------------------------------------------------------------------------------
+static int64_t pow2_divisor(int64_t x, int64_t cap) {   // largest power of two <= cap dividing x (x = 0 -> cap)
+    int64_t v = cap;
+    while (v > 1 && (x % v)) v >>= 1;
+    return v;
+}
+
+static int g_sm_count = 0;
+static ccl_status sm_count(int* n) {
+    if (!g_sm_count) {
+        int dev;
+        CCL_CUDA_TRY(cudaGetDevice(&dev));
+        CCL_CUDA_TRY(cudaDeviceGetAttribute(&g_sm_count, cudaDevAttrMultiProcessorCount, dev));
+    }
+    *n = g_sm_count;
+    return CCL_OK;
+}
+
+template <typename V>
+static ccl_status launch_vec(const char* src, char* dst, const CopyPlan& p, int sms, cudaStream_t st) {
+    int64_t cpr = p.row_bytes / (int64_t)sizeof(V), cps = cpr * p.rows;
+    int64_t blocks_needed = (cps + (int64_t)kVecThreads * kVecUnroll - 1) / ((int64_t)kVecThreads * kVecUnroll);
+    int64_t target = ((int64_t)sms * 8 + p.nstrips - 1) / p.nstrips;
+    dim3 grid((unsigned)std::max<int64_t>(1, std::min(blocks_needed, target)), (unsigned)p.nstrips);
+    if (cps < (INT64_C(1) << 31))
+        repack_vec_kernel<V, uint32_t><<<grid, kVecThreads, 0, st>>>(src, dst, p, (uint32_t)cpr, (uint32_t)cps);
+    else
+        repack_vec_kernel<V, uint64_t><<<grid, kVecThreads, 0, st>>>(src, dst, p, (uint64_t)cpr, (uint64_t)cps);
+    CCL_CUDA_TRY(cudaGetLastError());
+    return CCL_OK;
+}
+
+template <typename V>
+static ccl_status launch_pad(char* dst, const CopyPlan& p, cudaStream_t st) {
+    int64_t chunks = p.pad_bytes / (int64_t)sizeof(V);
+    dim3 grid((unsigned)std::max<int64_t>(1, std::min<int64_t>((chunks + 255) / 256, 64)), (unsigned)p.nstrips);
+    zero_pad_kernel<V><<<grid, 256, 0, st>>>(dst, p.pad_g, p.pad_off, chunks);
+    CCL_CUDA_TRY(cudaGetLastError());
+    return CCL_OK;
+}
+
+static ccl_status launch_tma(const char* src, char* dst, const CopyPlan& p, int sms, cudaStream_t st) {
+    uint64_t dims[3] = {(uint64_t)(p.row_bytes / 8), (uint64_t)p.rows, (uint64_t)p.nstrips};
+    TmaTiling t;
+    t.bx = (uint32_t)std::min<uint64_t>(256, dims[0]);
+    t.by = (uint32_t)std::max<uint64_t>(1, std::min<uint64_t>(std::min<uint64_t>(256, dims[1]), kTmaStageBytes / (t.bx * 8ull)));
+    t.tiles_x = (uint32_t)((dims[0] + t.bx - 1) / t.bx);
+    t.tiles_y = (uint32_t)((dims[1] + t.by - 1) / t.by);
+    t.ntiles = (uint64_t)t.tiles_x * t.tiles_y * (uint64_t)p.nstrips;
+    uint32_t box[3] = {t.bx, t.by, 1};
+    // a strip stride is irrelevant (and may be 0) when there is one strip: give the encoder a valid value
+    uint64_t sstr[2] = {(uint64_t)p.src_r, (uint64_t)(p.nstrips > 1 ? p.src_g : p.src_r * p.rows)};
+    uint64_t dstr[2] = {(uint64_t)p.dst_r, (uint64_t)(p.nstrips > 1 ? p.dst_g : p.dst_r * p.rows)};
+    CUtensorMap sm, dm;
+    ccl_status s = encode_tmap(&sm, CU_TENSOR_MAP_DATA_TYPE_UINT64, 3, src, dims, sstr, box, CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (s) return s;
+    s = encode_tmap(&dm, CU_TENSOR_MAP_DATA_TYPE_UINT64, 3, dst, dims, dstr, box, CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (s) return s;
+    size_t smem = (size_t)kTmaStages * kTmaStageBytes + 128 + kTmaStages * sizeof(uint64_t);
+    static bool attr_set = false;
+    if (!attr_set) {
+        CCL_CUDA_TRY(cudaFuncSetAttribute(repack_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        attr_set = true;
+    }
+    unsigned grid = (unsigned)std::min<uint64_t>(t.ntiles, (uint64_t)sms);
+    repack_tma_kernel<<<grid, 32, smem, st>>>(sm, dm, t);
+    CCL_CUDA_TRY(cudaGetLastError());
+    return CCL_OK;
+}
+
+ccl_status repack_status_take(int* code) {
+    int v = 0, z = 0;
+    CCL_CUDA_TRY(cudaMemcpyFromSymbol(&v, g_repack_status, sizeof(int)));
+    if (v) CCL_CUDA_TRY(cudaMemcpyToSymbol(g_repack_status, &z, sizeof(int)));
+    *code = v;
+    return CCL_OK;
+}
+
+}  // namespace ccl
+
+using namespace ccl;
+
+extern "C" ccl_status ccl_repack(const ccl_mat* m, const void* src_dev, void* dst_dev, int dir, void* cuda_stream) {
+    MatView v;
+    ccl_status s = make_view(m, "ccl_repack", &v);
+    if (s) return s;
+    if (!src_dev || !dst_dev) return fail(CCL_ERR_INVALID_ARG, "ccl_repack: NULL buffer");
+    if (dir != 0 && dir != 1) return fail(CCL_ERR_INVALID_ARG, "ccl_repack: dir must be 0 or 1");
+    if (src_dev == dst_dev) return fail(CCL_ERR_INVALID_ARG, "ccl_repack: in-place repack is not supported");
+    if ((reinterpret_cast<uintptr_t>(src_dev) % v.e) || (reinterpret_cast<uintptr_t>(dst_dev) % v.e))
+        return fail(CCL_ERR_ALIGN, "ccl_repack: buffers must be aligned to elem_bytes");
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    int sms;
+    s = sm_count(&sms);
+    if (s) return s;
+
+    const int64_t e = v.e;
+    CopyPlan p;
+    std::memset(&p, 0, sizeof(p));
+    int64_t rm_g, rm_r, cc_g, cc_r;          // row-major side and CCL side strides (bytes)
+    if (v.split == 2) {
+        p.nstrips = v.nstrips; p.rows = v.rows; p.row_bytes = v.w * e;
+        rm_g = v.w * e; rm_r = v.cols * e; cc_g = v.stride * e; cc_r = v.w * e;
+    } else if (v.split == 1) {
+        p.nstrips = v.nstrips; p.rows = v.h; p.row_bytes = v.cols * e;
+        rm_g = v.h * v.cols * e; rm_r = v.cols * e; cc_g = v.stride * e; cc_r = v.cols * e;
+    } else {                                  // identity: a plain copy, treated as one strip
+        p.nstrips = 1; p.rows = v.rows; p.row_bytes = v.cols * e;
+        rm_g = 0; rm_r = v.cols * e; cc_g = 0; cc_r = v.cols * e;
+    }
+    if (p.nstrips > 65535) return fail(CCL_ERR_UNSUPPORTED, "ccl_repack: P > 65535");
+    if (dir == 0) { p.src_g = rm_g; p.src_r = rm_r; p.dst_g = cc_g; p.dst_r = cc_r; }
+    else          { p.src_g = cc_g; p.src_r = cc_r; p.dst_g = rm_g; p.dst_r = rm_r; }
+    if (dir == 0 && v.split) {
+        p.pad_off = p.rows * p.row_bytes; p.pad_bytes = v.stride * e - p.pad_off; p.pad_g = cc_g;
+    }
+
+    const char* src = static_cast<const char*>(src_dev);
+    char* dst = static_cast<char*>(dst_dev);
+    int64_t addr_bits = (int64_t)((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst)) & 15);
+    int64_t vec = pow2_divisor(p.row_bytes | p.src_g | p.src_r | p.dst_g | p.dst_r | addr_bits, 16);
+
+    // path choice: TMA when everything is 16-byte aligned and the copy is big enough to be worth a ring
+    const char* force = std::getenv("CCL_REPACK_PATH");
+    bool tma_ok = vec == 16 && p.rows < (INT64_C(1) << 31) && p.row_bytes / 8 < (INT64_C(1) << 31) &&
+                  std::max(std::max(p.src_g, p.src_r), std::max(p.dst_g, p.dst_r)) < (INT64_C(1) << 40);
+    bool use_tma = tma_ok && p.nstrips * p.rows * p.row_bytes >= (INT64_C(1) << 20);
+    if (force && !std::strcmp(force, "vec")) use_tma = false;
+    if (force && !std::strcmp(force, "tma") && tma_ok) use_tma = true;
+
+    if (use_tma) s = launch_tma(src, dst, p, sms, st);
+    else if (vec == 16) s = launch_vec<uint4>(src, dst, p, sms, st);
+    else if (vec == 8) s = launch_vec<uint2>(src, dst, p, sms, st);
+    else if (vec == 4) s = launch_vec<unsigned int>(src, dst, p, sms, st);
+    else if (vec == 2) s = launch_vec<unsigned short>(src, dst, p, sms, st);
+    else s = launch_vec<unsigned char>(src, dst, p, sms, st);
+    if (s) return s;
+
+    if (p.pad_bytes > 0) {
+        int64_t pv = pow2_divisor(p.pad_off | p.pad_bytes | p.pad_g | (int64_t)(reinterpret_cast<uintptr_t>(dst) & 15), 16);
+        if (pv == 16) s = launch_pad<uint4>(dst, p, st);
+        else if (pv == 8) s = launch_pad<uint2>(dst, p, st);
+        else if (pv == 4) s = launch_pad<unsigned int>(dst, p, st);
+        else if (pv == 2) s = launch_pad<unsigned short>(dst, p, st);
+        else s = launch_pad<unsigned char>(dst, p, st);
+        if (s) return s;
+    }
+    return CCL_OK;
+}

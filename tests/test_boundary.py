@@ -1,0 +1,163 @@
+"""C-ABI boundary on the CPU: the library loads, exports what include/ccl.h declares, its host-side
+address map agrees with the oracle, and bad input is rejected before any launch.  No GPU."""
+import ctypes as C
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle as orc
+from paper_2606_11718_b200 import binding as ccl
+from paper_2606_11718_b200 import build as ccl_build
+from helpers import gemm_desc, mat_pair, traffic_pair
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    ccl_build.build()
+
+
+def test_exports_match_header():
+    hdr = open(os.path.join(ROOT, "include", "ccl.h")).read()
+    hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
+    declared = sorted(set(re.findall(r"\b(ccl_[a-z_]+)\s*\(", hdr)))
+    assert declared == sorted(ccl.EXPORTS)
+    l = ccl.lib()
+    for name in declared:
+        assert getattr(l, name) is not None
+    assert ccl.ccl_version() == "0.1"
+
+
+def test_struct_sizes_match_c_layout():
+    # the ctypes mirrors follow the C rules; spot-check the sizes the header implies
+    assert C.sizeof(ccl.Mat) == 40
+    assert C.sizeof(ccl.GemmDesc) == 24 + 3 * 40 + 5 * 4 + 4
+    assert C.sizeof(ccl.TrafficDesc) == 24 + 8 + 3 * 40 + 12 + 4 + 8 + 12 + 4 + 4 + 4
+
+
+MAP_CASES = [
+    dict(rows=4, cols=8, P=2, part=2, layout=1),
+    dict(rows=7, cols=12, P=3, part=2, layout=1),
+    dict(rows=33, cols=768, P=8, part=2, layout=1),
+    dict(rows=64, cols=200, P=2, part=2, layout=1, e=4),
+    dict(rows=12, cols=40, P=4, part=1, layout=1),
+    dict(rows=12, cols=40, P=4, part=2, layout=0),
+    dict(rows=12, cols=40, P=1, part=0, layout=0, e=1),
+    dict(rows=6, cols=36, P=3, part=2, layout=1, align=256),
+    dict(rows=6, cols=36, P=3, part=1, layout=1, align=4096),
+    dict(rows=5, cols=30, P=5, part=2, layout=1, align=64, e=4),
+]
+
+
+@pytest.mark.parametrize("case", MAP_CASES)
+def test_host_map_equals_oracle(case):
+    mo, ml = mat_pair(**case)
+    table = orc.map_table(mo)
+    for r in range(mo.rows):
+        for c in range(mo.cols):
+            assert ccl.ccl_map_offset(ml, r, c) == table[r, c]
+    assert ccl.ccl_buffer_bytes(ml) == orc.buffer_bytes(mo)
+    if case["layout"] == 1 and case["part"] != 0:
+        assert ccl.ccl_strip_stride(ml) == orc.strip_stride(mo)
+    n = orc.buffer_bytes(mo) // mo.elem_bytes
+    for off in range(n):
+        rc, r, c = orc.map_inverse(mo, off)
+        if rc == 0:
+            assert ccl.ccl_map_inverse(ml, off) == (r, c)
+        else:
+            with pytest.raises(ccl.CclError) as ei:
+                ccl.ccl_map_inverse(ml, off)
+            assert ei.value.status == ccl.ERR_PADDING
+
+
+def test_large_offsets_use_64_bits():
+    mo, ml = mat_pair(1 << 20, 1 << 16, 2, 4, 2, 1)                    # 2^36 elements
+    for r, c in [(0, 0), (1 << 19, 40000), ((1 << 20) - 1, (1 << 16) - 1)]:
+        assert ccl.ccl_map_offset(ml, r, c) == orc.map_offset(mo, r, c)
+
+
+def expect(status, fn, *a, **k):
+    with pytest.raises(ccl.CclError) as ei:
+        fn(*a, **k)
+    assert ei.value.status == status, ei.value
+    assert ccl.lib().ccl_last_error() != b""
+
+
+def test_map_error_codes():
+    expect(ccl.ERR_SHAPE, ccl.ccl_map_offset, ccl.Mat(4, 10, 2, 4, 2, 1), 0, 0)
+    expect(ccl.ERR_SHAPE, ccl.ccl_buffer_bytes, ccl.Mat(5, 8, 2, 2, 1, 1))
+    expect(ccl.ERR_INVALID_ARG, ccl.ccl_map_offset, ccl.Mat(4, 8, 2, 2, 2, 1), 4, 0)
+    expect(ccl.ERR_INVALID_ARG, ccl.ccl_map_offset, ccl.Mat(4, 8, 3, 2, 2, 1), 0, 0)
+    expect(ccl.ERR_INVALID_ARG, ccl.ccl_map_offset, ccl.Mat(4, 8, 2, 0, 2, 1), 0, 0)
+    expect(ccl.ERR_INVALID_ARG, ccl.ccl_map_offset, ccl.Mat(4, 8, 2, 2, 2, 1, 3), 0, 0)
+    expect(ccl.ERR_INVALID_ARG, ccl.ccl_strip_stride, ccl.Mat(4, 8))
+    expect(ccl.ERR_INVALID_ARG, ccl.ccl_map_inverse, ccl.Mat(4, 8), 32)
+
+
+def test_repack_rejects_bad_input_before_any_launch():
+    l = ccl.lib()
+    m = ccl.Mat(4, 8, 2, 2, 2, 1)
+    assert l.ccl_repack(C.byref(m), None, None, 0, None) == ccl.ERR_INVALID_ARG
+    assert l.ccl_repack(C.byref(m), C.c_void_p(256), C.c_void_p(512), 2, None) == ccl.ERR_INVALID_ARG
+    assert l.ccl_repack(C.byref(m), C.c_void_p(256), C.c_void_p(256), 0, None) == ccl.ERR_INVALID_ARG
+    assert l.ccl_repack(C.byref(m), C.c_void_p(257), C.c_void_p(512), 0, None) == ccl.ERR_ALIGN
+    bad = ccl.Mat(4, 9, 2, 2, 2, 1)
+    assert l.ccl_repack(C.byref(bad), C.c_void_p(256), C.c_void_p(512), 0, None) == ccl.ERR_SHAPE
+
+
+def gemm_rc(d, a=4096, b=8192, c=16384):
+    return ccl.lib().ccl_gemm(C.byref(d), C.c_void_p(a), C.c_void_p(b), C.c_void_p(c), None, 0, None)
+
+
+def test_gemm_rejects_bad_input_before_any_launch():
+    ok = gemm_desc(256, 768, 2048, 4, ("row", "ccl", "ccl"), b_trans=1)
+    assert ccl.ccl_gemm_workspace(ok) == 0
+    assert ccl.lib().ccl_gemm(C.byref(ok), None, None, None, None, 0, None) == ccl.ERR_INVALID_ARG
+    assert gemm_rc(gemm_desc(128, 200, 64, 2, ("row", "ccl", "ccl"))) == ccl.ERR_UNSUPPORTED        # w = 100
+    assert gemm_rc(gemm_desc(128, 256, 100)) == ccl.ERR_UNSUPPORTED                                  # K % 8 for A rows
+    assert gemm_rc(ok, a=4100) == ccl.ERR_ALIGN
+    d = gemm_desc(128, 256, 64)
+    d.A.rows = 100
+    assert gemm_rc(d) == ccl.ERR_SHAPE
+    d = gemm_desc(128, 256, 64)
+    d.C.elem_bytes = 4
+    assert gemm_rc(d) == ccl.ERR_UNSUPPORTED
+    d = gemm_desc(128, 256, 64, 4, ("row", "ccl", "ccl"))
+    d.C.P = 2                                                                                        # B and C strips differ
+    assert gemm_rc(d) == ccl.ERR_UNSUPPORTED
+    d = gemm_desc(128, 256, 64, 3, ("row", "row", "row"))
+    assert gemm_rc(d) == ccl.ERR_SHAPE                                                               # N % P with a grouped raster
+    d = gemm_desc(128, 256, 64)
+    d.out_part = 7
+    assert gemm_rc(d) == ccl.ERR_INVALID_ARG
+    d = gemm_desc(128, 512, 96, 2, ("row", "ccl", "row"), parts=(0, 1, 0))                            # B split along K, 48-row strips
+    assert gemm_rc(d) == ccl.ERR_UNSUPPORTED
+    d = gemm_desc(128, 512, 64, 2, ("row", "ccl", "ccl"), align=8)
+    d.B.rows = 63; d.K = 63; d.A.cols = 63                                                           # strip stride 63*256*2 is fine; K=63 breaks A
+    assert gemm_rc(d) == ccl.ERR_UNSUPPORTED
+
+
+def test_traffic_sizes_and_rejections():
+    do, dl = traffic_pair(130, 384, 96, 4, 256, ("row", "ccl", "ccl"), (0, 1, 1))
+    assert ccl.ccl_traffic_sizes(dl) == tuple(orc.traffic_sizes(do))
+    do, dl = traffic_pair(130, 384, 96, 4, 256, strip_tiling=0)
+    assert ccl.ccl_traffic_sizes(dl) == tuple(orc.traffic_sizes(do))
+    do, dl = traffic_pair(128, 256, 64, 8, 512, assign=1, BM=16, BN=64, lay=("ccl", "row", "ccl"), align=1024)
+    assert ccl.ccl_traffic_sizes(dl) == tuple(orc.traffic_sizes(do))
+    l = ccl.lib()
+    _, bad = traffic_pair(8, 9, 4, 2, 16)
+    assert l.ccl_traffic(C.byref(bad), None, C.c_void_p(256), None, None, C.c_void_p(512), None) == ccl.ERR_SHAPE
+    _, d = traffic_pair(8, 8, 4, 2, 16)
+    assert l.ccl_traffic(C.byref(d), None, None, None, None, C.c_void_p(512), None) == ccl.ERR_INVALID_ARG
+    _, d = traffic_pair(8, 8, 4, 2, 16, place=(2, 2, 2))
+    assert l.ccl_traffic(C.byref(d), None, C.c_void_p(256), None, None, C.c_void_p(512), None) == ccl.ERR_WORKSPACE
+    _, d = traffic_pair(8, 8, 4, 2, 16, assign=2)
+    assert l.ccl_traffic(C.byref(d), None, C.c_void_p(256), None, None, C.c_void_p(512), None) == ccl.ERR_INVALID_ARG
+    _, d = traffic_pair(8, 8, 4, 2, 3)
+    assert l.ccl_traffic(C.byref(d), None, C.c_void_p(256), None, None, C.c_void_p(512), None) == ccl.ERR_INVALID_ARG
+    _, d = traffic_pair(8, 8, 4, 2, 16)
+    d.A.rows = 9
+    assert l.ccl_traffic(C.byref(d), None, C.c_void_p(256), None, None, C.c_void_p(512), None) == ccl.ERR_SHAPE

@@ -1,0 +1,193 @@
+"""GPU parity, through the C ABI: ccl_gemm against the fp32 oracle.
+
+Tolerance (stated by the benchmark spec): err = |C_gpu - ref32| / max(1, |ref32|) <= 1e-2 * sqrt(K / 1024),
+where ref32 is the oracle's fp32-accumulate sum from the logical (row-major) operands.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle as orc
+from paper_2606_11718_b200 import binding as ccl
+from paper_2606_11718_b200 import synth
+from helpers import gemm_desc
+
+pytestmark = pytest.mark.gpu
+
+
+def tol(K):
+    return 1e-2 * math.sqrt(K / 1024.0)
+
+
+def to_layout(x_bits, m):
+    """Host bits of a stored row-major operand -> device buffer in the layout `m` (library descriptor) describes.
+    Uses the oracle's repack on the host, so a wrong device-side map cannot cancel out."""
+    mo = orc.Mat(m.rows, m.cols, m.elem_bytes, m.P, m.part, m.layout, m.strip_align_bytes)
+    buf = orc.repack(mo, x_bits, 0)
+    return torch.from_numpy(buf.view(np.int16)).cuda()
+
+
+def from_layout(buf, m):
+    mo = orc.Mat(m.rows, m.cols, m.elem_bytes, m.P, m.part, m.layout, m.strip_align_bytes)
+    return orc.repack(mo, buf.cpu().numpy().view(np.uint16), 1).reshape(m.rows, m.cols)
+
+
+def run_gemm(d, A, B):
+    """A, B: bf16 CPU tensors as stored (row-major).  Returns C as uint16 bits [M x N] (logical order)."""
+    a_dev, b_dev = to_layout(synth.bits(A), d.A), to_layout(synth.bits(B), d.B)
+    c_dev = torch.full((ccl.ccl_buffer_bytes(d.C) // 2,), 0x7FC0, dtype=torch.int16, device="cuda")   # NaN poison
+    ccl.ccl_gemm(d, a_dev, b_dev, c_dev)
+    st, detail = ccl.ccl_gemm_status()
+    assert st == ccl.OK, detail
+    return from_layout(c_dev, d.C)
+
+
+def check(d, A, B, block=None):
+    got = run_gemm(d, A, B)
+    M, N, K = d.M, d.N, d.K
+    ref32, _, ref_bits = orc.gemm(synth.bits(A), synth.bits(B), M, N, K, d.a_trans, d.b_trans, block=block)
+    if block is not None:
+        got = got[block[0]:block[1], block[2]:block[3]]
+    g = synth.from_bits(got).to(torch.float32).numpy()
+    assert np.isfinite(g).all(), "unwritten (poisoned) output elements"
+    err = np.abs(g - ref32) / np.maximum(1.0, np.abs(ref32))
+    assert err.max() <= tol(K), (err.max(), tol(K))
+    return got, ref_bits
+
+
+SMALL = [
+    # M, N, K, P, layouts(A,B,C), a_trans, b_trans, out_part
+    (128, 256, 64, 1, ("row", "row", "row"), 0, 1, 0),     # one tile, both operands K-major
+    (128, 256, 64, 1, ("row", "row", "row"), 0, 0, 0),     # B N-contiguous (MN-major)
+    (128, 256, 64, 1, ("row", "row", "row"), 1, 0, 0),     # A M-contiguous
+    (128, 256, 64, 1, ("row", "row", "row"), 1, 1, 0),
+    (130, 384, 96, 2, ("row", "row", "row"), 0, 0, 2),     # partial tiles in M, K not a multiple of 64
+    (130, 384, 96, 2, ("row", "ccl", "ccl"), 0, 0, 2),     # w = 192
+    (130, 384, 96, 4, ("row", "ccl", "ccl"), 0, 0, 2),     # w = 96: partial 128-wide tiles inside every strip
+    (130, 384, 200, 4, ("row", "ccl", "ccl"), 0, 1, 2),    # B stored [N x K], N-split = row split
+    (264, 768, 328, 4, ("row", "ccl", "ccl"), 1, 0, 2),
+    (264, 768, 328, 3, ("row", "ccl", "ccl"), 1, 1, 2),    # P = 3, w = 256
+    (512, 1024, 256, 8, ("row", "ccl", "ccl"), 0, 0, 2),
+    (512, 512, 256, 4, ("ccl", "row", "ccl"), 0, 0, 1),    # M-partition: A and C split along rows
+    (512, 512, 256, 2, ("ccl", "row", "ccl"), 1, 0, 1),    # M-partition with A stored [K x M]: a column split of A
+    (1, 512, 256, 4, ("row", "ccl", "ccl"), 0, 0, 2),      # M = 1
+    (16, 512, 256, 2, ("row", "ccl", "ccl"), 0, 0, 2),
+    (640, 2560, 512, 2, ("row", "ccl", "ccl"), 0, 0, 2),   # several tiles per CTA group, 5 stages wrap
+    (256, 512, 128, 2, ("ccl", "ccl", "row"), 0, 0, 0),    # A and B split along K (parts below), plain raster
+]
+
+
+@pytest.mark.parametrize("M,N,K,P,lay,at,bt,op", SMALL)
+def test_gemm_small_shapes(M, N, K, P, lay, at, bt, op):
+    parts = None
+    if lay == ("ccl", "ccl", "row") and op == 0:
+        parts = (1 if at else 2, 2 if bt else 1, 0)                    # both operands split along K
+    A, B = synth.gemm_operands(M, N, K, at, bt, seed=0, tag="small")
+    for grouped in (1, 0):
+        d = gemm_desc(M, N, K, P, lay, at, bt, op, grouped, parts=parts)
+        check(d, A, B)
+    if any(l == "ccl" for l in lay) and parts is None:
+        d = gemm_desc(M, N, K, P, lay, at, bt, op, 1, align=4096)      # page-aligned strips
+        check(d, A, B)
+
+
+def test_gemm_exact_cases():
+    eye = synth.from_bits(synth.bits(torch.eye(256).to(torch.bfloat16)))
+    A = synth.randn_bf16(200, 256, 1.0, 0, "eye")
+    d = gemm_desc(200, 256, 256, 2, ("row", "ccl", "ccl"))
+    np.testing.assert_array_equal(run_gemm(d, A, eye), synth.bits(A))                  # B = I  =>  C = A, bit for bit
+    ones_a, ones_b = torch.ones(128, 256).to(torch.bfloat16), torch.ones(256, 512).to(torch.bfloat16)
+    d = gemm_desc(128, 512, 256, 4, ("row", "ccl", "ccl"))
+    got = synth.from_bits(run_gemm(d, ones_a, ones_b)).to(torch.float32)
+    assert (got == 256.0).all()                                                        # all ones => K, exactly
+
+
+@pytest.mark.parametrize("at,bt", [(0, 0), (0, 1), (1, 0)])
+def test_layout_invariance_and_strip_independence(at, bt):
+    """Sec. 3.3: the GEMM computation is unchanged, only the address map: same bits from CCL and row-major operands."""
+    M, N, K, P = 384, 1536, 512, 4
+    A, B = synth.gemm_operands(M, N, K, at, bt, seed=3, tag="inv")
+    c_row = run_gemm(gemm_desc(M, N, K, P, ("row", "row", "row"), at, bt, 2, 1), A, B)
+    c_ccl = run_gemm(gemm_desc(M, N, K, P, ("row", "ccl", "ccl"), at, bt, 2, 1), A, B)
+    c_pad = run_gemm(gemm_desc(M, N, K, P, ("row", "ccl", "ccl"), at, bt, 2, 0, align=65536), A, B)
+    np.testing.assert_array_equal(c_row, c_ccl)
+    np.testing.assert_array_equal(c_row, c_pad)
+    # zeroing strip 2 of B changes strip 2 of C only
+    w = N // P
+    B2 = B.clone()
+    if bt:
+        B2[2 * w:3 * w, :] = 0
+    else:
+        B2[:, 2 * w:3 * w] = 0
+    c2 = run_gemm(gemm_desc(M, N, K, P, ("row", "ccl", "ccl"), at, bt, 2, 1), A, B2)
+    keep = np.ones(N, dtype=bool)
+    keep[2 * w:3 * w] = False
+    np.testing.assert_array_equal(c2[:, keep], c_ccl[:, keep])
+    assert (c2[:, ~keep] == 0).all()
+
+
+def test_gemm_config1_expert_up_projection():
+    g = synth.config1_gemm()
+    A, B = synth.gemm_operands(g["M"], g["N"], g["K"], g["a_trans"], g["b_trans"], seed=0, tag=g["name"])
+    d = gemm_desc(g["M"], g["N"], g["K"], 4, ("row", "ccl", "ccl"), g["a_trans"], g["b_trans"], 2, 1)
+    got, ref_bits = check(d, A, B)
+    ulp = np.abs(got.astype(np.int32) - ref_bits.astype(np.int32))
+    big = np.abs(synth.from_bits(ref_bits).to(torch.float32).numpy()) > 1e-2
+    assert ulp[big].max() <= 2
+    # 1b: W^T materialised [K x N], w = 192 (384-byte slices)
+    Bt = B.T.contiguous()
+    check(gemm_desc(g["M"], g["N"], g["K"], 4, ("row", "ccl", "ccl"), 0, 0, 2, 1), A, Bt)
+
+
+@pytest.mark.parametrize("P", [2, 4])
+def test_gemm_qwen_config(P):
+    for g in synth.qwen_ffn_gemms():
+        A, B = synth.gemm_operands(g["M"], g["N"], g["K"], g["a_trans"], g["b_trans"], seed=0, tag=g["name"],
+                                   a_std=g["a_std"], b_std=g["b_std"])
+        d = gemm_desc(g["M"], g["N"], g["K"], P, ("row", "ccl", "ccl"), g["a_trans"], g["b_trans"], 2, 1, align=4096)
+        check(d, A, B)
+
+
+def sample_blocks(M, N, P, rng, n_random=8, bm=128, bn=128):
+    w = N // P
+    blocks = {(0, 0), (0, N - bn), (M - bm, 0), (M - bm, N - bn)}
+    for g in range(P):                                                 # first and last tile of every strip, and across its edges
+        blocks.add((0, g * w)); blocks.add((M - bm, (g + 1) * w - bn))
+        if g:
+            blocks.add((bm, g * w - bn // 2))
+    for _ in range(n_random):
+        blocks.add((int(rng.integers(0, M - bm + 1)), int(rng.integers(0, N - bn + 1))))
+    return [(m, m + bm, n, n + bn) for m, n in sorted(blocks)]
+
+
+@pytest.mark.parametrize("name,P", [("llama_fwd_down", 4), ("llama_wgrad", 2)])
+def test_gemm_llama_full_size_sampled(name, P):
+    """Full Llama-70B-size GEMM in the benchmark's launch configuration (CCL B and C, grouped raster): sampled
+    128x128 blocks against the oracle, plus a randomised projection check over the whole output."""
+    g = {x["name"]: x for x in synth.llama_fwd_gemms() + synth.llama_bwd_gemms()}[name]
+    M, N, K = g["M"], g["N"], g["K"]
+    A, B = synth.gemm_operands(M, N, K, g["a_trans"], g["b_trans"], seed=0, tag=name, a_std=g["a_std"], b_std=g["b_std"])
+    d = gemm_desc(M, N, K, P, ("row", "ccl", "ccl"), g["a_trans"], g["b_trans"], 2, 1)
+    got = run_gemm(d, A, B)
+    gf = synth.from_bits(got).to(torch.float32)
+    assert torch.isfinite(gf).all()
+    rng = np.random.default_rng(0)
+    for blk in sample_blocks(M, N, P, rng):
+        ref32, _, _ = orc.gemm(synth.bits(A), synth.bits(B), M, N, K, g["a_trans"], g["b_trans"], block=blk)
+        sub = gf[blk[0]:blk[1], blk[2]:blk[3]].numpy()
+        err = np.abs(sub - ref32) / np.maximum(1.0, np.abs(ref32))
+        assert err.max() <= tol(K), (blk, err.max())
+    # property over every output element: C v = A (B v) for random +-1 vectors (exact arithmetic up to rounding)
+    Al = (A.T if g["a_trans"] else A).to(torch.float32)
+    Bl = (B.T if g["b_trans"] else B).to(torch.float32)
+    sigma_c = g["a_std"] * g["b_std"] * math.sqrt(K)
+    for s in range(2):
+        v = torch.from_numpy(rng.choice([-1.0, 1.0], size=N).astype(np.float32))
+        lhs = gf.to(torch.float64) @ v.to(torch.float64)
+        rhs = Al.to(torch.float64) @ (Bl.to(torch.float64) @ v.to(torch.float64)) if K * N < 3e8 else \
+            (Al @ (Bl @ v)).to(torch.float64)
+        # bf16 rounding of C: each element off by <= 2^-9 relative; random signs -> sqrt(N) growth, 8 sigma margin
+        bound = 8 * math.sqrt(N) * sigma_c * 2.0 ** -8
+        assert (lhs - rhs).abs().max().item() <= bound

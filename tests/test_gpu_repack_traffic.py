@@ -1,0 +1,219 @@
+"""GPU parity, through the C ABI: ccl_repack and ccl_traffic against the oracle, bit for bit."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle as orc
+from paper_2606_11718_b200 import binding as ccl
+from helpers import mat_pair, traffic_pair
+
+pytestmark = pytest.mark.gpu
+DT = {1: (np.uint8, torch.uint8), 2: (np.uint16, torch.int16), 4: (np.uint32, torch.int32)}
+
+
+def dev(a):
+    return torch.from_numpy(a.view({1: np.uint8, 2: np.int16, 4: np.int32, 8: np.int64}[a.itemsize])).cuda()
+
+
+def host(t, np_dtype):
+    return t.cpu().numpy().view(np_dtype)
+
+
+def run_repack(case, path=None, seed=0):
+    mo, ml = mat_pair(**case)
+    npdt, _ = DT[mo.elem_bytes]
+    rng = np.random.default_rng(seed)
+    x = rng.integers(1, np.iinfo(npdt).max, size=(mo.rows, mo.cols), dtype=npdt)
+    want = orc.repack(mo, x, 0)
+    old = os.environ.pop("CCL_REPACK_PATH", None)
+    if path:
+        os.environ["CCL_REPACK_PATH"] = path
+    try:
+        src = dev(x)
+        dst = dev(np.full(want.size, 0x5A, dtype=npdt))                # poison: padding must be overwritten with zeros
+        ccl.ccl_repack(ml, src, dst, 0)
+        got = host(dst, npdt)
+        np.testing.assert_array_equal(got, want)
+        back = dev(np.zeros(mo.rows * mo.cols, dtype=npdt))
+        ccl.ccl_repack(ml, dst, back, 1)
+        np.testing.assert_array_equal(host(back, npdt).reshape(mo.rows, mo.cols), x)
+        np.testing.assert_array_equal(orc.repack(mo, want, 1).reshape(mo.rows, mo.cols), x)
+        assert ccl.ccl_gemm_status()[0] == ccl.OK
+    finally:
+        os.environ.pop("CCL_REPACK_PATH", None)
+        if old is not None:
+            os.environ["CCL_REPACK_PATH"] = old
+
+
+REPACK_CASES = [
+    dict(rows=4, cols=8, P=2, part=2, layout=1),                       # the Fig. 4(a) example
+    dict(rows=1, cols=16, P=2, part=2, layout=1),
+    dict(rows=130, cols=384, P=4, part=2, layout=1),                   # w = 96
+    dict(rows=130, cols=384, P=2, part=2, layout=1),                   # w = 192
+    dict(rows=64, cols=200, P=2, part=2, layout=1),                    # w = 100: 8-byte vectors only
+    dict(rows=33, cols=50, P=5, part=2, layout=1),                     # w = 10: 4-byte vectors
+    dict(rows=33, cols=21, P=3, part=2, layout=1),                     # w = 7: scalar
+    dict(rows=77, cols=96, P=3, part=2, layout=1, e=1),
+    dict(rows=77, cols=96, P=3, part=2, layout=1, e=4),
+    dict(rows=256, cols=1536, P=8, part=2, layout=1),
+    dict(rows=2048, cols=1536, P=4, part=2, layout=1),                 # Qwen gate/up weight, 384-element slices
+    dict(rows=768, cols=2048, P=4, part=2, layout=1),                  # Qwen down weight
+    dict(rows=768, cols=2048, P=1, part=2, layout=1),                  # G = 1: a plain copy
+    dict(rows=768, cols=2048, P=4, part=1, layout=1),                  # split along rows: a plain copy
+    dict(rows=768, cols=2048, P=4, part=1, layout=1, align=4096),
+    dict(rows=100, cols=2048, P=4, part=2, layout=1, align=4096),      # padded strips
+    dict(rows=7, cols=24, P=3, part=2, layout=1, align=256),
+    dict(rows=7, cols=24, P=3, part=2, layout=1, align=256, e=1),
+    dict(rows=1000, cols=4096, P=2, part=2, layout=1, align=65536),
+    dict(rows=4099, cols=2056, P=2, part=2, layout=1),                 # ragged: rows and box tails
+    dict(rows=300, cols=8192, P=2, part=2, layout=0),                  # row-major descriptor: identity
+]
+
+
+@pytest.mark.parametrize("case", REPACK_CASES)
+@pytest.mark.parametrize("path", ["vec", "tma", None])
+def test_repack_bit_exact(case, path):
+    run_repack(case, path)
+
+
+def test_repack_unaligned_base_pointer():
+    mo, ml = mat_pair(64, 256, 2, 4, 2, 1)
+    x = np.random.default_rng(1).integers(0, 65535, size=(64, 256), dtype=np.uint16)
+    buf = dev(np.zeros(64 * 256 + 8, dtype=np.uint16))
+    src = buf[1:1 + 64 * 256]                                          # 2-byte aligned only
+    src.copy_(dev(x).reshape(-1))
+    dst = dev(np.zeros(64 * 256 + 8, dtype=np.uint16))
+    ccl.ccl_repack(ml, src, dst[3:], 0)
+    np.testing.assert_array_equal(host(dst, np.uint16)[3:3 + 64 * 256], orc.repack(mo, x, 0))
+
+
+@pytest.mark.parametrize("P", [2, 4])
+def test_repack_llama_down_weight_full_size(P):
+    # [28672 x 8192] bf16 = 470 MB: the full-size matrix of the Llama down projection
+    R, Cc = 28672, 8192
+    mo, ml = mat_pair(R, Cc, 2, P, 2, 1)
+    x = np.random.default_rng(2).integers(0, 65535, size=(R, Cc), dtype=np.uint16)
+    src = dev(x)
+    dst = torch.empty(R * Cc, dtype=torch.int16, device="cuda")
+    ccl.ccl_repack(ml, src, dst, 0)
+    got = host(dst, np.uint16)
+    w = Cc // P
+    for g in range(P):                                                 # oracle definition, strip by strip (bounded host memory)
+        np.testing.assert_array_equal(got[g * R * w:(g + 1) * R * w].reshape(R, w), x[:, g * w:(g + 1) * w])
+    idx = np.random.default_rng(3).integers(0, R * Cc, size=2000)
+    for lin in idx:                                                    # sampled outputs through the oracle's own map
+        r, c = divmod(int(lin), Cc)
+        assert got[orc.map_offset(mo, r, c)] == x[r, c]
+
+
+# ------------------------------------------------------------------------------------------ traffic
+
+def run_traffic(do, dl, level="elem", explicit_q=None):
+    want = orc.traffic(do, explicit_q=explicit_q, level=level)
+    nt, pages = ccl.ccl_traffic_sizes(dl)
+    assert (nt, pages) == tuple(orc.traffic_sizes(do))
+    per_cta = torch.full((nt, 3, 2), -1, dtype=torch.int64, device="cuda")
+    totals = torch.full((3, 2), -1, dtype=torch.int64, device="cuda")
+    per_page = [torch.full((pages[x], dl.P), -1, dtype=torch.int64, device="cuda") for x in range(3)]
+    owner = [torch.full((pages[x],), 77, dtype=torch.uint8, device="cuda") for x in range(3)]
+    q = None if explicit_q is None else torch.from_numpy(np.asarray(explicit_q, dtype=np.int32)).cuda()
+    ccl.ccl_traffic(dl, per_cta, totals, per_page, owner, q)
+    np.testing.assert_array_equal(host(per_cta, np.uint64), want["per_cta"])
+    np.testing.assert_array_equal(host(totals, np.uint64), want["totals"])
+    for X in range(3):
+        np.testing.assert_array_equal(host(per_page[X], np.uint64), want["per_page"][X])
+        np.testing.assert_array_equal(host(owner[X], np.uint8), want["owner"][X])
+    # second call without the optional outputs (only legal when no operand uses BEST placement)
+    if 2 not in list(dl.place):
+        per_cta2 = torch.full((nt, 3, 2), -1, dtype=torch.int64, device="cuda")
+        totals2 = torch.full((3, 2), -1, dtype=torch.int64, device="cuda")
+        ccl.ccl_traffic(dl, per_cta2, totals2, None, None, q)
+        np.testing.assert_array_equal(host(per_cta2, np.uint64), want["per_cta"])
+        np.testing.assert_array_equal(host(totals2, np.uint64), want["totals"])
+    return want
+
+
+SHAPES = [
+    dict(M=4, N=8, K=4, P=2, S=16, BM=4, BN=4),                       # the hand-enumerated case
+    dict(M=130, N=384, K=96, P=4, S=256),
+    dict(M=130, N=384, K=96, P=2, S=4096),
+    dict(M=64, N=200, K=40, P=2, S=16),
+    dict(M=96, N=96, K=64, P=3, S=64, BM=32, BN=32),
+    dict(M=96, N=96, K=64, P=3, S=48, BM=32, BN=32),                   # page size not a power of two
+    dict(M=256, N=768, K=128, P=4, S=4096, b_trans=1),
+    dict(M=120, N=256, K=72, P=4, S=128, a_trans=1),
+    dict(M=128, N=256, K=64, P=8, S=512, assign=1, BM=16, BN=64),
+    dict(M=100, N=240, K=48, P=2, S=1 << 21),
+    dict(M=130, N=384, K=96, P=4, S=256, strip_tiling=0),
+    dict(M=1, N=512, K=256, P=4, S=4096),
+    dict(M=16, N=512, K=256, P=1, S=4096),
+]
+LAYS = [("row", "row", "row"), ("row", "ccl", "ccl"), ("ccl", "ccl", "ccl")]
+PLACES = [(0, 0, 0), (1, 1, 1), (2, 2, 2), (0, 1, 2)]
+
+
+@pytest.mark.parametrize("shape", SHAPES)
+@pytest.mark.parametrize("lay", LAYS)
+@pytest.mark.parametrize("place", PLACES)
+def test_traffic_bit_exact_small(shape, lay, place):
+    for align in (0, 1024):
+        do, dl = traffic_pair(lay=lay, place=place, align=align, **shape)
+        run_traffic(do, dl, "elem")
+
+
+def test_traffic_explicit_assignment():
+    do, dl = traffic_pair(64, 96, 32, 3, 64, BM=16, BN=32, assign=2, lay=("row", "ccl", "ccl"), place=(0, 1, 2),
+                          parts=(0, 2, 2))
+    nt, _ = ccl.ccl_traffic_sizes(dl)
+    q = np.random.default_rng(0).integers(0, 3, size=nt).astype(np.int32)
+    run_traffic(do, dl, "elem", explicit_q=q)
+
+
+def test_traffic_config1_expert_up_projection():
+    # X[256x2048] times W[768x2048]^T, P = 4, 128x128 tiles, 4 KB pages; remote traffic vs 4 KB round-robin
+    base = dict(M=256, N=768, K=2048, P=4, S=4096, b_trans=1)
+    rr = run_traffic(*traffic_pair(**base), level="elem")
+    cc = run_traffic(*traffic_pair(lay=("row", "ccl", "ccl"), place=(0, 1, 1), **base), level="elem")
+    assert cc["totals"][1, 1] == 0 and cc["totals"][2, 1] == 0         # B and C fully local under CCL
+    assert rr["totals"][:, 1].sum() > cc["totals"][:, 1].sum()
+    run_traffic(*traffic_pair(place=(2, 2, 2), **base), level="elem")
+    # 1b: W^T materialised [K x N], w = 192 -> 384-byte slices
+    base = dict(M=256, N=768, K=2048, P=4, S=4096)
+    run_traffic(*traffic_pair(**base), level="elem")
+    run_traffic(*traffic_pair(lay=("row", "ccl", "ccl"), place=(0, 1, 1), **base), level="elem")
+
+
+@pytest.mark.parametrize("P,S", [(2, 4096), (4, 4096), (4, 65536)])
+def test_traffic_qwen_config(P, S):
+    from paper_2606_11718_b200 import synth
+    for g in synth.qwen_ffn_gemms():
+        base = dict(M=g["M"], N=g["N"], K=g["K"], P=P, S=S, a_trans=g["a_trans"], b_trans=g["b_trans"])
+        for lay, place in [(("row", "row", "row"), (0, 0, 0)), (("row", "ccl", "ccl"), (0, 1, 1)), (("row", "row", "row"), (1, 1, 1))]:
+            run_traffic(*traffic_pair(lay=lay, place=place, **base), level="runs")
+
+
+@pytest.mark.parametrize("name,lay,place", [("row_rr", ("row", "row", "row"), (0, 0, 0)), ("ccl_block", ("row", "ccl", "ccl"), (0, 1, 1)),
+                                            ("row_best", ("row", "row", "row"), (2, 2, 2))])
+def test_traffic_llama_down_full_size(name, lay, place):
+    # [8192 x 28672] x [28672 x 8192], P = 4, 4 KB pages: 4096 tiles, ~1.2e8 run pieces
+    run_traffic(*traffic_pair(8192, 8192, 28672, 4, 4096, lay=lay, place=place), level="runs")
+
+
+def test_traffic_llama_gateup_full_size_closed_form():
+    # B [8192 x 57344] row-major under 4 KB round-robin, P = 4: remote is exactly 5/7 of the B bytes
+    do, dl = traffic_pair(8192, 57344, 8192, 4, 4096)
+    nt, pages = ccl.ccl_traffic_sizes(dl)
+    per_cta = torch.zeros((nt, 3, 2), dtype=torch.int64, device="cuda")
+    totals = torch.zeros((3, 2), dtype=torch.int64, device="cuda")
+    ccl.ccl_traffic(dl, per_cta, totals)
+    t = host(totals, np.uint64)
+    assert int(t[1].sum()) == 60_129_542_144 and int(t[1, 1]) == 42_949_672_960
+    assert int(t[2].sum()) == 8192 * 57344 * 2
+    pc = host(per_cta, np.uint64)
+    assert (pc.sum(axis=2) == np.array([128 * 8192 * 2, 8192 * 128 * 2, 128 * 128 * 2], dtype=np.uint64)).all()
+    # sampled tiles through the oracle: a descriptor restricted to one tile row gives the same per-CTA numbers
+    do1, _ = traffic_pair(128, 57344, 8192, 4, 4096)
+    want = orc.traffic(do1, level="runs")["per_cta"]
+    np.testing.assert_array_equal(pc[:448, 1:], want[:, 1:])          # B and C columns of tile row 0
