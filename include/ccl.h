@@ -179,7 +179,7 @@ ccl_status ccl_traffic_sizes(const ccl_traffic_desc* d, int64_t* ntiles, int64_t
  *   totals_dev   uint64 [3][2]                                               (required)
  * per_page_dev / owner_dev are HOST arrays of three device pointers (or NULL altogether).
  * cta_chiplet_dev: int32 [ntiles], values in [0,P); only read for CCL_ASSIGN_EXPLICIT.
- * Out-of-range entries are counted as chiplet 0 ... never dereferenced out of bounds.
+ * Entries outside [0,P) are clamped into the range.
  */
 ccl_status ccl_traffic(const ccl_traffic_desc* d, const int32_t* cta_chiplet_dev, uint64_t* per_cta_dev,
                        uint64_t* const per_page_dev[3], uint8_t* const owner_dev[3], uint64_t* totals_dev,
@@ -187,6 +187,8 @@ ccl_status ccl_traffic(const ccl_traffic_desc* d, const int32_t* cta_chiplet_dev
 
 /* Message for the last non-OK status returned on this thread ("" if none). Static storage. */
 const char* ccl_last_error(void);
+/* Number of CUDA kernels this library has launched in this process (all threads, all streams). */
+uint64_t ccl_launch_count(void);
 /* Library version, "major.minor". */
 const char* ccl_version(void);
 

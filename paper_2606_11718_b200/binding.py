@@ -20,7 +20,7 @@ PLACE_RR, PLACE_BLOCK, PLACE_BEST = 0, 1, 2
 ASSIGN_N_STRIPS, ASSIGN_M_STRIPS, ASSIGN_EXPLICIT = 0, 1, 2
 
 EXPORTS = ["ccl_map_offset", "ccl_map_inverse", "ccl_buffer_bytes", "ccl_strip_stride", "ccl_repack", "ccl_gemm_workspace",
-           "ccl_gemm", "ccl_gemm_status", "ccl_traffic_sizes", "ccl_traffic", "ccl_last_error", "ccl_version"]
+           "ccl_gemm", "ccl_gemm_status", "ccl_traffic_sizes", "ccl_traffic", "ccl_last_error", "ccl_launch_count", "ccl_version"]
 
 
 class CclError(RuntimeError):
@@ -65,6 +65,7 @@ def lib():
         l = C.CDLL(LIB_PATH)
         l.ccl_last_error.restype = C.c_char_p
         l.ccl_version.restype = C.c_char_p
+        l.ccl_launch_count.restype = C.c_uint64
         l.ccl_map_offset.argtypes = [C.POINTER(Mat), C.c_int64, C.c_int64, C.POINTER(C.c_int64)]
         l.ccl_map_inverse.argtypes = [C.POINTER(Mat), C.c_int64, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
         l.ccl_buffer_bytes.argtypes = [C.POINTER(Mat), C.POINTER(C.c_int64)]
@@ -95,6 +96,10 @@ def _ptr(t):
 
 def ccl_version():
     return lib().ccl_version().decode()
+
+
+def ccl_launch_count():
+    return int(lib().ccl_launch_count())
 
 
 def ccl_map_offset(m, r, c):

@@ -20,6 +20,7 @@ namespace ccl {
 
 ccl_status fail(ccl_status s, const char* fmt, ...);   // records the thread-local message, returns s
 void clear_error();
+void count_launch(int n = 1);                              // bookkeeping for ccl_launch_count()
 
 #define CCL_CUDA_TRY(expr)                                                                      \
     do {                                                                                        \

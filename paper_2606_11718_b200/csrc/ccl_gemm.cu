@@ -183,32 +183,48 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             uint32_t phase = 0;
             TileCoord t;
             bool ok = true;
+            // K runs along the tensor map's x for a K-contiguous operand and along y otherwise.  Unless
+            // the operand is split along K itself (rare), only that coordinate changes with kb, so
+            // the box coordinates are computed once per tile.
+            const bool a_ksplit = p.a_mn ? p.a.split == 1 : p.a.split == 2;
+            const bool b_ksplit = p.b_mn ? p.b.split == 1 : p.b.split == 2;
+            constexpr int NA = BM / 64, NB = BN / 64;
             for (int64_t i = sched.idx; ok && sched.get(i, t); i += sched.step) {
+                int ax[NA], ay[NA], az[NA], bx[NB], by[NB], bz[NB];
+                if (!p.a_mn) to_coords(p.a, t.m0, 0, ax[0], ay[0], az[0]);
+                else {
+#pragma unroll
+                    for (int c = 0; c < NA; ++c) to_coords(p.a, 0, t.m0 + 64 * c, ax[c], ay[c], az[c]);
+                }
+                if (!p.b_mn) to_coords(p.b, t.n0, 0, bx[0], by[0], bz[0]);
+                else {
+#pragma unroll
+                    for (int c = 0; c < NB; ++c) to_coords(p.b, 0, t.n0 + 64 * c, bx[c], by[c], bz[c]);
+                }
                 for (int kb = 0; kb < p.num_kb; ++kb) {
                     if (!mbar_wait_bounded(&empty[stage], phase ^ 1)) { atomicExch(&g_gemm_status, 1); *abort_flag = 1; ok = false; break; }
                     unsigned char* sa = smem + (size_t)stage * p.stage_bytes;
                     unsigned char* sb = sa + p.a_bytes;
                     mbar_expect_tx(&full[stage], p.stage_bytes);
                     const int k0 = kb * BK;
-                    int x, y, z;
                     if (!p.a_mn) {                      // A stored [M x K]: one box of 64 k x 128 m
-                        to_coords(p.a, t.m0, k0, x, y, z);
-                        tma_load_3d(sa, &map_a, &full[stage], x, y, z);
+                        if (a_ksplit) to_coords(p.a, t.m0, k0, ax[0], ay[0], az[0]);
+                        tma_load_3d(sa, &map_a, &full[stage], a_ksplit ? ax[0] : k0, ay[0], az[0]);
                     } else {                            // A stored [K x M]: boxes of 64 m x 64 k
 #pragma unroll
-                        for (int c = 0; c < BM / 64; ++c) {
-                            to_coords(p.a, k0, t.m0 + 64 * c, x, y, z);
-                            tma_load_3d(sa + c * (64 * BK * 2), &map_a, &full[stage], x, y, z);
+                        for (int c = 0; c < NA; ++c) {
+                            if (a_ksplit) to_coords(p.a, k0, t.m0 + 64 * c, ax[c], ay[c], az[c]);
+                            tma_load_3d(sa + c * (64 * BK * 2), &map_a, &full[stage], ax[c], a_ksplit ? ay[c] : k0, az[c]);
                         }
                     }
                     if (!p.b_mn) {                      // B stored [N x K]: one box of 64 k x BN n
-                        to_coords(p.b, t.n0, k0, x, y, z);
-                        tma_load_3d(sb, &map_b, &full[stage], x, y, z);
+                        if (b_ksplit) to_coords(p.b, t.n0, k0, bx[0], by[0], bz[0]);
+                        tma_load_3d(sb, &map_b, &full[stage], b_ksplit ? bx[0] : k0, by[0], bz[0]);
                     } else {                            // B stored [K x N]: boxes of 64 n x 64 k
 #pragma unroll
-                        for (int c = 0; c < BN / 64; ++c) {
-                            to_coords(p.b, k0, t.n0 + 64 * c, x, y, z);
-                            tma_load_3d(sb + c * (64 * BK * 2), &map_b, &full[stage], x, y, z);
+                        for (int c = 0; c < NB; ++c) {
+                            if (b_ksplit) to_coords(p.b, k0, t.n0 + 64 * c, bx[c], by[c], bz[c]);
+                            tma_load_3d(sb + c * (64 * BK * 2), &map_b, &full[stage], bx[c], b_ksplit ? by[c] : k0, bz[c]);
                         }
                     }
                     if (++stage == p.stages) { stage = 0; phase ^= 1; }
@@ -434,6 +450,7 @@ static ccl_status launch(const GemmPlan& plan, const CUtensorMap& ma, const CUte
         configured_for = (int)plan.smem_bytes;
     }
     ccl_gemm_kernel<BN><<<plan.grid, kGemmThreads, plan.smem_bytes, st>>>(ma, mb, plan.p);
+    count_launch();
     CCL_CUDA_TRY(cudaGetLastError());
     return CCL_OK;
 }

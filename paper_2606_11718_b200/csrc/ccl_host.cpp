@@ -1,4 +1,5 @@
 // Host-only entry points: the address map (Eq. 1-3), sizes, error text.
+#include <atomic>
 #include <cstring>
 
 #include "ccl_common.h"
@@ -16,6 +17,10 @@ ccl_status fail(ccl_status s, const char* fmt, ...) {
 }
 
 void clear_error() { g_err[0] = 0; }
+
+static std::atomic<uint64_t> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+uint64_t launches() { return g_launches.load(std::memory_order_relaxed); }
 
 ccl_status make_view(const ccl_mat* m, const char* what, MatView* out) {
     if (!m) return fail(CCL_ERR_INVALID_ARG, "%s: NULL descriptor", what);
@@ -110,6 +115,7 @@ ccl_status ccl_strip_stride(const ccl_mat* m, int64_t* elems) {
 }
 
 const char* ccl_last_error(void) { return g_err; }
+uint64_t ccl_launch_count(void) { return ccl::launches(); }
 const char* ccl_version(void) { return "0.1"; }
 
 }  // extern "C"

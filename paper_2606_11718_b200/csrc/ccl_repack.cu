@@ -170,6 +170,7 @@ static ccl_status launch_vec(const char* src, char* dst, const CopyPlan& p, int 
         repack_vec_kernel<V, uint32_t><<<grid, kVecThreads, 0, st>>>(src, dst, p, (uint32_t)cpr, (uint32_t)cps);
     else
         repack_vec_kernel<V, uint64_t><<<grid, kVecThreads, 0, st>>>(src, dst, p, (uint64_t)cpr, (uint64_t)cps);
+    count_launch();
     CCL_CUDA_TRY(cudaGetLastError());
     return CCL_OK;
 }
@@ -179,6 +180,7 @@ static ccl_status launch_pad(char* dst, const CopyPlan& p, cudaStream_t st) {
     int64_t chunks = p.pad_bytes / (int64_t)sizeof(V);
     dim3 grid((unsigned)std::max<int64_t>(1, std::min<int64_t>((chunks + 255) / 256, 64)), (unsigned)p.nstrips);
     zero_pad_kernel<V><<<grid, 256, 0, st>>>(dst, p.pad_g, p.pad_off, chunks);
+    count_launch();
     CCL_CUDA_TRY(cudaGetLastError());
     return CCL_OK;
 }
@@ -208,6 +210,7 @@ static ccl_status launch_tma(const char* src, char* dst, const CopyPlan& p, int 
     }
     unsigned grid = (unsigned)std::min<uint64_t>(t.ntiles, (uint64_t)sms);
     repack_tma_kernel<<<grid, 32, smem, st>>>(sm, dm, t);
+    count_launch();
     CCL_CUDA_TRY(cudaGetLastError());
     return CCL_OK;
 }

@@ -258,19 +258,23 @@ extern "C" ccl_status ccl_traffic(const ccl_traffic_desc* d, const int32_t* cta_
     z.p[0] = totals_dev; z.n[0] = 6;
     for (int X = 0; X < 3; ++X) if (p.per_page[X]) { z.p[1 + X] = p.per_page[X]; z.n[1 + X] = p.pages[X] * p.P; }
     traffic_prep_kernel<<<sms * 2, 256, 0, st>>>(z);
+    count_launch();
     CCL_CUDA_TRY(cudaGetLastError());
 
     int64_t nwork = p.ntiles * 3;
     unsigned grid = (unsigned)std::max<int64_t>(1, std::min<int64_t>((nwork + kWarpsPerBlock - 1) / kWarpsPerBlock, (int64_t)sms * 8));
     if (need_hist) {
         traffic_hist_kernel<<<grid, kWarpsPerBlock * 32, 0, st>>>(p);
+        count_launch();
         CCL_CUDA_TRY(cudaGetLastError());
     }
     if (need_owner) {
         traffic_owner_kernel<<<sms * 2, 256, 0, st>>>(p);
+        count_launch();
         CCL_CUDA_TRY(cudaGetLastError());
     }
     traffic_classify_kernel<<<grid, kWarpsPerBlock * 32, 0, st>>>(p);
+    count_launch();
     CCL_CUDA_TRY(cudaGetLastError());
     return CCL_OK;
 }
