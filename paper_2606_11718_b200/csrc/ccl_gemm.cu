@@ -6,17 +6,23 @@
 //     -- the view (K, G, N/G) with strides (w, K*w, 1) of Sec. 3.3 -- so the address
 //     translation costs nothing per access and a partial last tile of a strip is handled by
 //     TMA zero fill.
-//   * One persistent CTA per SM, warp-specialised: warp 0 = TMA producer, warp 1 = tcgen05.mma
-//     issuer (one elected thread) and TMEM owner, warps 2-5 = epilogue (TMEM -> registers ->
-//     bf16 -> global, addressing C through its own layout).
-//   * 128 x BN x 64 tiles (BN in {128,192,256}), SWIZZLE_128B shared-memory tiles, a ring of
-//     smem stages, two TMEM accumulators so the epilogue of tile i overlaps the main loop of
-//     tile i+1.
+//   * Persistent, warp-specialised CTAs: warp 0 = TMA producer, warp 1 = tcgen05.mma issuer
+//     (one elected thread) and TMEM owner, warps 2-5 = epilogue (TMEM -> registers -> bf16 ->
+//     global, addressing C through its own layout).
+//   * Two flavours of one kernel template:
+//       CTAS = 2: a cluster of two CTAs (one SM pair) computes a 256 x BN tile with
+//                 tcgen05.mma.cta_group::2; each CTA stages its own 128 rows of A and its own
+//                 half of the B columns, which halves the shared-memory traffic per flop
+//                 (the 1-CTA kernel is bound by it: ~61% tensor-pipe activity);
+//       CTAS = 1: one CTA per 128 x BN tile, for shapes whose M extent does not fill a pair.
+//   * SWIZZLE_128B shared-memory tiles, a ring of smem stages, two TMEM accumulators so the
+//     epilogue of tile i overlaps the main loop of tile i+1.
 //   * Chiplet-grouped raster (Sec. 3.1): the CTAs are cut into P groups and group g walks only
 //     the output tiles of strip g, i.e. it streams one contiguous region of B and C.
 //   * Every mbarrier wait is bounded; on expiry the kernel records a code in g_gemm_status,
 //     all roles leave their loops, TMEM is released and the kernel returns.
 #include <algorithm>
+#include <cstdlib>
 #include <cstring>
 
 #include <cuda_bf16.h>
@@ -26,11 +32,11 @@
 
 namespace ccl {
 
-constexpr int BM = 128;
+constexpr int BM = 128;                         // rows of the output tile one CTA owns
 constexpr int BK = 64;
 constexpr int kGemmThreads = 192;
 constexpr int kTmemCols = 512;
-constexpr uint32_t kSmemBudget = 200 * 1024;   // ring of operand stages
+constexpr uint32_t kSmemBudget = 200 * 1024;    // ring of operand stages
 
 __device__ int g_gemm_status = 0;
 
@@ -42,7 +48,7 @@ struct OpMap {          // how stored coordinates (r, c) of an operand become te
 struct GemmParams {
     int32_t M, N, K;
     int32_t Wm, Wn;                 // widths of the strips the tile grid respects (M / N when unsplit)
-    int32_t tps_m, tps_n;           // tiles per strip
+    int32_t tps_m, tps_n;           // tiles per strip (a tile is 128*CTAS x BN)
     int32_t tiles_m, tiles_n;
     int32_t num_kb;
     int32_t groups, group_dim;      // chiplet-grouped raster: number of CTA groups, 0 = along N, 1 = along M
@@ -54,26 +60,71 @@ struct GemmParams {
     uint16_t* C;
     uint32_t idesc;
     int32_t stages;
-    uint32_t stage_bytes, a_bytes;  // bytes per stage, bytes of the A part
+    uint32_t stage_bytes, a_bytes;  // bytes per stage per CTA, bytes of its A part
 };
 
-// ---- tcgen05 wrappers ---------------------------------------------------------------------
+// ---- PTX wrappers ---------------------------------------------------------------------------
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ uint32_t cluster_ctarank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
+__device__ __forceinline__ void cluster_sync() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// shared::cluster address of the same shared-memory offset in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+
+template <int CTAS>
 __device__ __forceinline__ void tmem_alloc(uint32_t* smem_dst, uint32_t ncols) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_dst)), "r"(ncols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (CTAS == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_dst)), "r"(ncols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    } else {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_dst)), "r"(ncols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
 }
+template <int CTAS>
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+    if (CTAS == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+    else asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
 }
+template <int CTAS>
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
-        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+    if (CTAS == 1)
+        asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+                     ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+    else
+        asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}"
+                     ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// Arrive on an mbarrier once every MMA issued so far by this thread has completed.  With two CTAs
+// the arrival is delivered to the barrier at the same offset in both CTAs of the pair.
+template <int CTAS>
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+    if (CTAS == 1)
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+    else
+        asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                     ::"r"(smem_u32(bar)), "h"((unsigned short)3) : "memory");
+}
+// TMA tile load whose completion bytes are credited to `bar_addr` (a shared::cluster address; with two
+// CTAs this is the leader's barrier, which the cta_group::2 form of the copy is allowed to signal).
+template <int CTAS>
+__device__ __forceinline__ void tma_load(void* smem_dst, const CUtensorMap* map, uint32_t bar_addr, int c0, int c1, int c2) {
+    if (CTAS == 1)
+        asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+                     ::"r"(smem_u32(smem_dst)), "l"(map), "r"(bar_addr), "r"(c0), "r"(c1), "r"(c2) : "memory");
+    else
+        asm volatile("cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+                     ::"r"(smem_u32(smem_dst)), "l"(map), "r"(bar_addr), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile(
@@ -104,179 +155,196 @@ __device__ __forceinline__ void to_coords(const OpMap& o, int r, int c, int& x, 
 
 struct TileCoord { int m0, m1, n0, n1; };
 
-// Tiles of this CTA: CTAs are cut into `groups` contiguous ranges; group g walks the tiles of its
-// strip range in panels of `panel` m-tiles (m fastest inside a panel, then n, then the next panel).
+// Tiles of this CTA (pair).  The schedulable units (CTAs, or CTA pairs) are cut into `groups`
+// contiguous ranges; group g owns the tiles of strip range g (chiplet-grouped raster) and walks
+// them in panels of `panel` m-tiles (m fastest inside a panel, then n, then the next panel).
+// Groups can differ by one unit, so the walk has two phases: `rounds` rounds in which every unit
+// takes tile (its index + round * group size) of its own group, then the few tiles each group
+// has left are pooled and dealt round-robin to all units, which keeps every unit equally busy.
 struct Scheduler {
     const GemmParams& p;
-    int gm, gn, tm_off, tn_off;     // sub-grid of this CTA's group
-    int idx, step, bn;
-    int64_t total;
-    __device__ Scheduler(const GemmParams& p_, int bn_) : p(p_), bn(bn_) {
-        int G = gridDim.x, c = blockIdx.x, g = 0, lo = 0, hi = G;
-        if (p.groups > 1) {
-            for (g = 0; g < p.groups; ++g) {
-                lo = (int)(((int64_t)g * G) / p.groups);
-                hi = (int)(((int64_t)(g + 1) * G) / p.groups);
-                if (c >= lo && c < hi) break;
-            }
+    int gm, gn;                     // tile grid of one group
+    int unit, units, my_g, idx, step, bm, bn, rounds;
+    int64_t per_group;
+    __device__ int lo(int g) const { return (int)(((int64_t)g * units) / p.groups); }
+    __device__ Scheduler(const GemmParams& p_, int unit_, int units_, int bm_, int bn_) : p(p_), unit(unit_), units(units_), bm(bm_), bn(bn_) {
+        gm = p.tiles_m; gn = p.tiles_n;
+        if (p.groups > 1) { if (p.group_dim == 0) gn = p.tiles_n / p.groups; else gm = p.tiles_m / p.groups; }
+        per_group = (int64_t)gm * gn;
+        my_g = 0; rounds = 0x7fffffff;
+        for (int g = 0; g < p.groups; ++g) {
+            int l = lo(g), h = lo(g + 1);
+            if (unit >= l && unit < h) { my_g = g; idx = unit - l; step = h - l; }
+            rounds = min(rounds, (int)(per_group / (h - l)));
         }
-        idx = c - lo; step = hi - lo;
-        gm = p.tiles_m; gn = p.tiles_n; tm_off = 0; tn_off = 0;
-        if (p.groups > 1) {
-            if (p.group_dim == 0) { gn = p.tiles_n / p.groups; tn_off = g * gn; }
-            else { gm = p.tiles_m / p.groups; tm_off = g * gm; }
-        }
-        total = (int64_t)gm * gn;
     }
-    __device__ bool get(int64_t i, TileCoord& t) const {
-        if (i >= total) return false;
+    __device__ bool get(int it, TileCoord& t) const {
+        int g = my_g;
+        int64_t i;
+        if (it < rounds) i = idx + (int64_t)it * step;
+        else {                                            // pooled leftovers of all groups
+            int64_t q = unit + (int64_t)(it - rounds) * units;
+            for (g = 0; g < p.groups; ++g) {
+                int64_t done = (int64_t)rounds * (lo(g + 1) - lo(g)), left = per_group - done;
+                if (q < left) { i = done + q; break; }
+                q -= left;
+            }
+            if (g == p.groups) return false;
+        }
         int64_t per_panel = (int64_t)p.panel * gn;
         int pn = (int)(i / per_panel);
         int rem = (int)(i - (int64_t)pn * per_panel);
         int ph = min(p.panel, gm - pn * p.panel);
         int ln = rem / ph, lm = pn * p.panel + (rem - ln * ph);
-        int tm = tm_off + lm, tn = tn_off + ln;
+        int tm = lm + (p.group_dim == 1 ? g * gm : 0), tn = ln + (p.group_dim == 0 && p.groups > 1 ? g * gn : 0);
         int sm = tm / p.tps_m, jm = tm - sm * p.tps_m;
         int sn = tn / p.tps_n, jn = tn - sn * p.tps_n;
-        t.m0 = sm * p.Wm + jm * BM; t.m1 = min(t.m0 + BM, (sm + 1) * p.Wm);
-        t.n0 = sn * p.Wn; t.n1 = (sn + 1) * p.Wn;     // strip bounds; the BN step is applied by the caller
-        t.n0 += jn * bn; t.n1 = min(t.n0 + bn, t.n1);
+        t.m0 = sm * p.Wm + jm * bm; t.m1 = min(t.m0 + bm, (sm + 1) * p.Wm);
+        t.n0 = sn * p.Wn + jn * bn; t.n1 = min(t.n0 + bn, (sn + 1) * p.Wn);
         return true;
     }
 };
 
-template <int BN>
+template <int BN, int CTAS>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const GemmParams p) {
+    // A tile wider than 256 columns is computed as NSUB sub-tiles of SUBN columns (one MMA each per
+    // k step) that fill TMEM; narrower tiles use the two 256-column halves of TMEM as a double buffer.
+    constexpr int NSUB = BN > 256 ? BN / 256 : 1;
+    constexpr int SUBN = BN / NSUB;
+    constexpr int SUBH = SUBN / CTAS;                // B columns of one sub-tile this CTA stages
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)p.stages * p.stage_bytes);
-    uint64_t* full = bars;
-    uint64_t* empty = bars + p.stages;
-    uint64_t* tmem_full = bars + 2 * p.stages;
-    uint64_t* tmem_empty = tmem_full + 2;
+    uint64_t* full = bars;                           // used in the leader CTA only
+    uint64_t* empty = bars + p.stages;               // one set per CTA
+    uint64_t* tmem_full = bars + 2 * p.stages;       // one set per CTA
+    uint64_t* tmem_empty = tmem_full + 2;            // used in the leader CTA only
     uint32_t* tmem_ptr = reinterpret_cast<uint32_t*>(tmem_empty + 2);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_ptr + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = CTAS == 2 ? cluster_ctarank() : 0;
+    const bool leader = rank == 0;
 
     if (threadIdx.x == 0) {
         prefetch_tmap(&map_a);
         prefetch_tmap(&map_b);
         for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(&tmem_full[a], 1); mbar_init(&tmem_empty[a], 4); }
-        *abort_flag = 0;
+        for (int a = 0; a < 2; ++a) { mbar_init(&tmem_full[a], 1); mbar_init(&tmem_empty[a], 4 * CTAS); }
         fence_barrier_init();
     }
-    if (warp == 1) tmem_alloc(tmem_ptr, kTmemCols);
+    if (warp == 1) tmem_alloc<CTAS>(tmem_ptr, kTmemCols);
     tc_fence_before();
     __syncthreads();
+    if (CTAS == 2) cluster_sync();                   // the peer's barriers exist before anything remote touches them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_ptr;
 
-    Scheduler sched(p, BN);
+    Scheduler sched(p, (int)(blockIdx.x / CTAS), (int)(gridDim.x / CTAS), BM * CTAS, BN);
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            int stage = 0;
-            uint32_t phase = 0;
-            TileCoord t;
-            bool ok = true;
-            // K runs along the tensor map's x for a K-contiguous operand and along y otherwise.  Unless
-            // the operand is split along K itself (rare), only that coordinate changes with kb, so
-            // the box coordinates are computed once per tile.
-            const bool a_ksplit = p.a_mn ? p.a.split == 1 : p.a.split == 2;
-            const bool b_ksplit = p.b_mn ? p.b.split == 1 : p.b.split == 2;
-            constexpr int NA = BM / 64, NB = BN / 64;
-            for (int64_t i = sched.idx; ok && sched.get(i, t); i += sched.step) {
-                int ax[NA], ay[NA], az[NA], bx[NB], by[NB], bz[NB];
-                if (!p.a_mn) to_coords(p.a, t.m0, 0, ax[0], ay[0], az[0]);
-                else {
-#pragma unroll
-                    for (int c = 0; c < NA; ++c) to_coords(p.a, 0, t.m0 + 64 * c, ax[c], ay[c], az[c]);
-                }
-                if (!p.b_mn) to_coords(p.b, t.n0, 0, bx[0], by[0], bz[0]);
-                else {
-#pragma unroll
-                    for (int c = 0; c < NB; ++c) to_coords(p.b, 0, t.n0 + 64 * c, bx[c], by[c], bz[c]);
-                }
-                for (int kb = 0; kb < p.num_kb; ++kb) {
-                    if (!mbar_wait_bounded(&empty[stage], phase ^ 1)) { atomicExch(&g_gemm_status, 1); *abort_flag = 1; ok = false; break; }
-                    unsigned char* sa = smem + (size_t)stage * p.stage_bytes;
-                    unsigned char* sb = sa + p.a_bytes;
-                    mbar_expect_tx(&full[stage], p.stage_bytes);
-                    const int k0 = kb * BK;
-                    if (!p.a_mn) {                      // A stored [M x K]: one box of 64 k x 128 m
-                        if (a_ksplit) to_coords(p.a, t.m0, k0, ax[0], ay[0], az[0]);
-                        tma_load_3d(sa, &map_a, &full[stage], a_ksplit ? ax[0] : k0, ay[0], az[0]);
-                    } else {                            // A stored [K x M]: boxes of 64 m x 64 k
-#pragma unroll
-                        for (int c = 0; c < NA; ++c) {
-                            if (a_ksplit) to_coords(p.a, k0, t.m0 + 64 * c, ax[c], ay[c], az[c]);
-                            tma_load_3d(sa + c * (64 * BK * 2), &map_a, &full[stage], ax[c], a_ksplit ? ay[c] : k0, az[c]);
-                        }
-                    }
-                    if (!p.b_mn) {                      // B stored [N x K]: one box of 64 k x BN n
-                        if (b_ksplit) to_coords(p.b, t.n0, k0, bx[0], by[0], bz[0]);
-                        tma_load_3d(sb, &map_b, &full[stage], b_ksplit ? bx[0] : k0, by[0], bz[0]);
-                    } else {                            // B stored [K x N]: boxes of 64 n x 64 k
-#pragma unroll
-                        for (int c = 0; c < NB; ++c) {
-                            if (b_ksplit) to_coords(p.b, k0, t.n0 + 64 * c, bx[c], by[c], bz[c]);
-                            tma_load_3d(sb + c * (64 * BK * 2), &map_b, &full[stage], bx[c], b_ksplit ? by[c] : k0, bz[c]);
-                        }
-                    }
-                    if (++stage == p.stages) { stage = 0; phase ^= 1; }
-                }
+        // One lane per TMA box of a stage (at most 6): the whole warp walks the tile/k loop, every lane
+        // polls the stage's "empty" barrier, lane 0 posts the byte count and each active lane issues its
+        // own box, so a stage is refilled in one issue slot instead of a serial chain.
+        constexpr int NA = BM / 64, NC = SUBH / 64;          // 64-wide boxes per MN-major A tile / B sub-tile
+        const int nA = p.a_mn ? NA : 1;
+        const int nB = p.b_mn ? NSUB * NC : NSUB;
+        const bool active = lane < nA + nB;
+        const bool isA = lane < nA;
+        const int bi = isA ? lane : lane - nA;                // box index within its operand
+        const CUtensorMap* map = isA ? &map_a : &map_b;
+        const OpMap om = isA ? p.a : p.b;
+        const bool mn = isA ? p.a_mn != 0 : p.b_mn != 0;
+        // K runs along the tensor map's x for a K-contiguous operand and along y otherwise; unless the
+        // operand is split along K itself (rare) only that coordinate changes from one k block to the next
+        const bool ksplit = mn ? om.split == 1 : om.split == 2;
+        uint32_t soff;                                        // byte offset of the box inside a stage
+        int off;                                              // offset of the box along M (A) or N (B) from the tile origin
+        if (isA) { soff = mn ? (uint32_t)bi * (64 * BK * 2) : 0u; off = (int)rank * BM + (mn ? 64 * bi : 0); }
+        else if (mn) { const int h = bi / NC, c = bi - h * NC; soff = p.a_bytes + (uint32_t)(h * SUBH * BK * 2 + c * 64 * BK * 2); off = h * SUBN + (int)rank * SUBH + 64 * c; }
+        else { soff = p.a_bytes + (uint32_t)(bi * SUBH * BK * 2); off = bi * SUBN + (int)rank * SUBH; }
+        const uint32_t full0 = CTAS == 2 ? map_to_cta(smem_u32(&full[0]), 0) : smem_u32(&full[0]);
+        int stage = 0;
+        uint32_t phase = 0;
+        TileCoord t;
+        bool ok = true;
+        for (int it = 0; ok && sched.get(it, t); ++it) {
+            const int base = (isA ? t.m0 : t.n0) + off;
+            int x, y, z;
+            if (mn) to_coords(om, 0, base, x, y, z); else to_coords(om, base, 0, x, y, z);
+            for (int kb = 0; kb < p.num_kb; ++kb) {
+                ok = mbar_wait_bounded(&empty[stage], phase ^ 1);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) { if (lane == 0) atomicExch(&g_gemm_status, 1); break; }
+                if (lane == 0 && leader) mbar_expect_tx(&full[stage], p.stage_bytes * CTAS);
+                __syncwarp();
+                const int k0 = kb * BK;
+                if (ksplit) { if (mn) to_coords(om, k0, base, x, y, z); else to_coords(om, base, k0, x, y, z); }
+                else if (mn) y = k0; else x = k0;
+                if (active) tma_load<CTAS>(smem + (size_t)stage * p.stage_bytes + soff, map, full0 + (uint32_t)stage * 8u, x, y, z);
+                if (++stage == p.stages) { stage = 0; phase ^= 1; }
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+        if (lane == 0 && leader) {
             int stage = 0;
             uint32_t phase = 0;
             TileCoord t;
             bool ok = true;
-            int it = 0;
-            // descriptor constants per operand
             const uint32_t a_lbo = p.a_mn ? 64 * BK * 2 : 16, b_lbo = p.b_mn ? 64 * BK * 2 : 16;
             const uint32_t a_kstep = p.a_mn ? (16 * 128) >> 4 : (16 * 2) >> 4;     // descriptor units (16 B) per UMMA_K = 16
             const uint32_t b_kstep = p.b_mn ? (16 * 128) >> 4 : (16 * 2) >> 4;
-            for (int64_t i = sched.idx; ok && sched.get(i, t); i += sched.step, ++it) {
-                const int acc = it & 1;
-                const uint32_t acc_phase = (uint32_t)(it >> 1) & 1;
-                if (!mbar_wait_bounded(&tmem_empty[acc], acc_phase ^ 1)) { atomicExch(&g_gemm_status, 2); *abort_flag = 1; break; }
-                tc_fence_after();
-                const uint32_t tmem_d = tmem_base + (uint32_t)acc * 256u;
-                for (int kb = 0; kb < p.num_kb; ++kb) {
-                    if (!mbar_wait_bounded(&full[stage], phase)) { atomicExch(&g_gemm_status, 3); *abort_flag = 1; ok = false; break; }
+            for (int it = 0; ok && sched.get(it, t); ++it) {
+                // NSUB == 1: TMEM half (it & 1) is this tile's accumulator, the other half is being drained.
+                // NSUB == 2: both halves belong to this tile; half h may be overwritten once the epilogue
+                //            of the previous tile has drained it.
+                const int acc0 = NSUB == 1 ? (it & 1) : 0;
+                const uint32_t acc_phase = NSUB == 1 ? ((uint32_t)(it >> 1) & 1) : ((uint32_t)it & 1);
+                for (int kb = 0; ok && kb < p.num_kb; ++kb) {
+                    if (!mbar_wait_bounded(&full[stage], phase)) { atomicExch(&g_gemm_status, 3); ok = false; break; }
                     tc_fence_after();
                     const uint32_t sa = smem_u32(smem + (size_t)stage * p.stage_bytes);
                     const uint64_t adesc = smem_desc(sa, a_lbo, 1024);
-                    const uint64_t bdesc = smem_desc(sa + p.a_bytes, b_lbo, 1024);
 #pragma unroll
-                    for (int k = 0; k < BK / 16; ++k)
-                        umma_bf16(tmem_d, adesc + (uint64_t)(k * a_kstep), bdesc + (uint64_t)(k * b_kstep), p.idesc, (kb | k) != 0);
-                    umma_commit(&empty[stage]);          // frees the stage once these MMAs have read it
+                    for (int h = 0; h < NSUB; ++h) {
+                        if (kb == 0) {
+                            if (!mbar_wait_bounded(&tmem_empty[acc0 + h], acc_phase ^ 1)) { atomicExch(&g_gemm_status, 2); ok = false; break; }
+                            tc_fence_after();
+                        }
+                        const uint32_t tmem_d = tmem_base + (uint32_t)(acc0 + h) * 256u;
+                        const uint64_t bdesc = smem_desc(sa + p.a_bytes + h * (SUBH * BK * 2), b_lbo, 1024);
+#pragma unroll
+                        for (int k = 0; k < BK / 16; ++k)
+                            umma_bf16<CTAS>(tmem_d, adesc + (uint64_t)(k * a_kstep), bdesc + (uint64_t)(k * b_kstep), p.idesc, (kb | k) != 0);
+                    }
+                    if (!ok) break;
+                    umma_commit<CTAS>(&empty[stage]);          // frees the stage (in both CTAs) once these MMAs have read it
                     if (++stage == p.stages) { stage = 0; phase ^= 1; }
                 }
-                if (ok) umma_commit(&tmem_full[acc]);    // accumulator complete
+                if (ok) {
+#pragma unroll
+                    for (int h = 0; h < NSUB; ++h) umma_commit<CTAS>(&tmem_full[acc0 + h]);   // accumulators complete (both CTAs)
+                }
             }
         }
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..5)
         const int quad = warp & 3;                       // TMEM lane quadrant this warp may read
+        const uint32_t tmem_empty0 = CTAS == 2 ? map_to_cta(smem_u32(&tmem_empty[0]), 0) : smem_u32(&tmem_empty[0]);
         TileCoord t;
-        int it = 0;
-        for (int64_t i = sched.idx; sched.get(i, t); i += sched.step, ++it) {
-            const int acc = it & 1;
-            const uint32_t acc_phase = (uint32_t)(it >> 1) & 1;
+        bool alive = true;
+        for (int it = 0; alive && sched.get(it, t); ++it) {
+          const int m = t.m0 + (int)rank * BM + quad * 32 + lane;
+          for (int h = 0; h < NSUB; ++h) {
+            const int acc = NSUB == 1 ? (it & 1) : h;
+            const uint32_t acc_phase = NSUB == 1 ? ((uint32_t)(it >> 1) & 1) : ((uint32_t)it & 1);
+            const int nb = t.n0 + h * SUBN;              // first column of this sub-tile
             bool ok = mbar_wait_bounded(&tmem_full[acc], acc_phase);
             ok = __all_sync(0xffffffffu, ok);
-            if (!ok) { if (lane == 0) { atomicExch(&g_gemm_status, 4); *abort_flag = 1; } break; }
+            if (!ok) { if (lane == 0) atomicExch(&g_gemm_status, 4); alive = false; break; }
             tc_fence_after();
-            const int m = t.m0 + quad * 32 + lane;
             // offset of (m, n) in C is row_base + n for every n of this tile
             int64_t row_base;
             if (p.c_split == 2) { int64_t g = t.n0 / p.c_w; row_base = g * p.c_stride + (int64_t)m * p.c_w - g * p.c_w; }
@@ -284,15 +352,15 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             else row_base = (int64_t)m * p.c_cols;
             const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)acc * 256u;
 #pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
-                if (t.n0 + c * 32 >= t.n1) break;        // warp-uniform: nothing valid further right
+            for (int c = 0; c < SUBN / 32; ++c) {
+                if (nb + c * 32 >= t.n1) break;          // warp-uniform: nothing valid further right
                 uint32_t r[32];
                 tmem_ld32(taddr + (uint32_t)(c * 32), r);
                 tmem_ld_wait();
                 if (m < t.m1) {
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        const int n = t.n0 + c * 32 + j * 8;
+                        const int n = nb + c * 32 + j * 8;
                         if (n < t.n1) {                  // n1 - n0 is a multiple of 8
                             uint4 v;
                             __nv_bfloat162 h;
@@ -307,15 +375,20 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&tmem_empty[acc]);
+            if (lane == 0) {
+                if (CTAS == 2) mbar_arrive_cluster(tmem_empty0 + (uint32_t)acc * 8u);
+                else mbar_arrive(&tmem_empty[acc]);
+            }
+          }
         }
     }
 
     tc_fence_before();
     __syncthreads();
+    if (CTAS == 2) cluster_sync();                   // neither CTA frees TMEM or exits while the other may still use it
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, kTmemCols);
+        tmem_dealloc<CTAS>(tmem_base, kTmemCols);
     }
 }
 
@@ -324,7 +397,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 // ------------------------------------------------------------------------------------------
 struct GemmPlan {
     GemmParams p;
-    int bn;
+    int bn, ctas;
     MatView va, vb, vc;
     uint32_t smem_bytes;
     unsigned grid;
@@ -341,7 +414,7 @@ static ccl_status check_operand(const MatView& v, const void* ptr, const char* n
     return CCL_OK;
 }
 
-// strip width an operand imposes on GEMM dimension `dim_is_rows ? stored rows : stored cols`
+// strip width an operand imposes on the GEMM dimension that runs along its stored rows / cols
 static int64_t split_width(const MatView& v, bool along_rows) {
     if (along_rows) return v.split == 1 ? v.h : 0;
     return v.split == 2 ? v.w : 0;
@@ -354,7 +427,10 @@ static ccl_status merge_width(int64_t* cur, int64_t w, const char* dim) {
     return CCL_OK;
 }
 
-static ccl_status make_plan(const ccl_gemm_desc* d, const void* A, const void* B, const void* C, int sms, GemmPlan* plan) {
+static int64_t padded(int64_t w, int64_t b) { return (w + b - 1) / b * b; }
+
+// units = schedulable CTAs (1-CTA kernel) or CTA pairs (2-CTA kernel) the device can hold at once
+static ccl_status make_plan(const ccl_gemm_desc* d, const void* A, const void* B, const void* C, int sms, int pairs, GemmPlan* plan) {
     if (!d) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: NULL descriptor");
     if (d->M <= 0 || d->N <= 0 || d->K <= 0) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: M, N, K must be positive");
     if (d->M >= (INT64_C(1) << 31) || d->N >= (INT64_C(1) << 31) || d->K >= (INT64_C(1) << 31)) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: dimension too large");
@@ -396,36 +472,50 @@ static ccl_status make_plan(const ccl_gemm_desc* d, const void* A, const void* B
     if (!Wm) Wm = d->M;
     if (!Wn) Wn = d->N;
 
-    // BN: least padded work per strip, ties to the wider tile
-    int best_bn = 256;
-    int64_t best_waste = -1;
-    for (int bn : {256, 192, 128}) {
-        int64_t waste = (Wn + bn - 1) / bn * bn - Wn;
-        if (best_waste < 0 || waste < best_waste) { best_waste = waste; best_bn = bn; }
-    }
-    plan->bn = best_bn;
+    // tile shape: least padded work per strip, ties to the wider tile; the 2-CTA kernel (256-row tiles,
+    // BN in {256,128}) is taken unless it pads noticeably more than the 1-CTA kernel (BN in {256,192,128})
+    int bn1 = 256, bn2 = 256;
+    for (int bn : {192, 128}) if (padded(Wn, bn) < padded(Wn, bn1)) bn1 = bn;
+    if (padded(Wn, 128) < padded(Wn, 256)) bn2 = 128;
+    // 256 x 512 pair tiles move 25% fewer operand bytes per flop (the L2 -> SM fill rate is what bounds
+    // the 256 x 256 kernel); they are worth a little padding, and need K long enough to amortise the
+    // epilogue that is only half overlapped
+    if (padded(Wn, 512) <= 1.05 * padded(Wn, bn2) && d->K >= 1024) bn2 = 512;
+    double work1 = (double)padded(Wm, 128) * (double)padded(Wn, bn1), work2 = (double)padded(Wm, 256) * (double)padded(Wn, bn2);
+    int ctas = (pairs > 0 && work2 <= 1.08 * work1) ? 2 : 1;
+    if (const char* f = std::getenv("CCL_GEMM_CTAS")) { if (f[0] == '1') ctas = 1; else if (f[0] == '2' && pairs > 0) ctas = 2; }
+    if (const char* f = std::getenv("CCL_GEMM_BN")) { int v = atoi(f); if (ctas == 2 && (v == 512 || v == 256 || v == 128)) bn2 = v; if (ctas == 1 && (v == 256 || v == 192 || v == 128)) bn1 = v; }
+    const int bn = ctas == 2 ? bn2 : bn1;
+    const int subn = bn > 256 ? 256 : bn;                // columns of one MMA / one TMEM accumulator
+    const int bm = BM * ctas;
+    plan->bn = bn; plan->ctas = ctas;
 
     GemmParams& p = plan->p;
     std::memset(&p, 0, sizeof(p));
     p.M = (int32_t)d->M; p.N = (int32_t)d->N; p.K = (int32_t)d->K;
     p.Wm = (int32_t)Wm; p.Wn = (int32_t)Wn;
-    p.tps_m = (int32_t)((Wm + BM - 1) / BM); p.tps_n = (int32_t)((Wn + best_bn - 1) / best_bn);
+    p.tps_m = (int32_t)((Wm + bm - 1) / bm); p.tps_n = (int32_t)((Wn + bn - 1) / bn);
     p.tiles_m = (int32_t)(d->M / Wm) * p.tps_m; p.tiles_n = (int32_t)(d->N / Wn) * p.tps_n;
     p.num_kb = (int32_t)((d->K + BK - 1) / BK);
     p.a.split = va.split; p.a.w = (int32_t)va.w; p.a.h = (int32_t)va.h;
     p.b.split = vb.split; p.b.w = (int32_t)vb.w; p.b.h = (int32_t)vb.h;
     p.a_mn = at ? 1 : 0; p.b_mn = bt ? 0 : 1;
     p.c_split = vc.split; p.c_w = vc.w; p.c_h = vc.h; p.c_stride = vc.stride; p.c_cols = vc.cols;
+    // instruction descriptor: D = f32, A = B = bf16, operand majors, N >> 3, M >> 4 (M spans the CTA pair)
     p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)p.a_mn << 15) | ((uint32_t)p.b_mn << 16) |
-              ((uint32_t)(best_bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
-    p.a_bytes = BM * BK * 2; p.stage_bytes = p.a_bytes + (uint32_t)best_bn * BK * 2;
-    p.stages = (int32_t)(kSmemBudget / p.stage_bytes);
+              ((uint32_t)(subn >> 3) << 17) | ((uint32_t)(bm >> 4) << 24);
+    p.a_bytes = BM * BK * 2; p.stage_bytes = p.a_bytes + (uint32_t)(bn / ctas) * BK * 2;
+    uint32_t budget = kSmemBudget;
+    if (const char* f = std::getenv("CCL_GEMM_SMEM_KB")) budget = (uint32_t)atoi(f) * 1024u;
+    p.stages = (int32_t)(budget / p.stage_bytes);
     if (p.stages > 8) p.stages = 8;
     p.panel = 16;
+    if (const char* f = std::getenv("CCL_GEMM_PANEL")) p.panel = std::max(1, atoi(f));
     int64_t ntiles = (int64_t)p.tiles_m * p.tiles_n;
-    plan->grid = (unsigned)std::min<int64_t>(ntiles, sms);
-    // grouped raster needs at least one CTA per group and whole strips per group
-    if (groups > 1 && (int)plan->grid >= groups && (group_dim == 0 ? p.tiles_n % groups == 0 : p.tiles_m % groups == 0)) {
+    int units = (int)std::min<int64_t>(ntiles, ctas == 2 ? pairs : sms);
+    plan->grid = (unsigned)(units * ctas);
+    // grouped raster needs at least one unit per group and whole strips per group
+    if (groups > 1 && units >= groups && (group_dim == 0 ? p.tiles_n % groups == 0 : p.tiles_m % groups == 0)) {
         p.groups = groups; p.group_dim = group_dim;
     } else { p.groups = 1; p.group_dim = 0; }
     plan->smem_bytes = (uint32_t)p.stages * p.stage_bytes + 1024 + (2 * p.stages + 4) * 8 + 16;
@@ -442,17 +532,52 @@ static ccl_status operand_tmap(CUtensorMap* m, const MatView& v, const void* bas
     return encode_tmap(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
-template <int BN>
-static ccl_status launch(const GemmPlan& plan, const CUtensorMap& ma, const CUtensorMap& mb, cudaStream_t st) {
-    static int configured_for = 0;
-    if (configured_for < (int)plan.smem_bytes) {
-        CCL_CUDA_TRY(cudaFuncSetAttribute(ccl_gemm_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem_bytes));
-        configured_for = (int)plan.smem_bytes;
+template <int BN, int CTAS>
+static ccl_status configure(uint32_t smem_bytes) {
+    static uint32_t configured_for = 0;
+    if (configured_for < smem_bytes) {
+        CCL_CUDA_TRY(cudaFuncSetAttribute(ccl_gemm_kernel<BN, CTAS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes));
+        configured_for = smem_bytes;
     }
-    ccl_gemm_kernel<BN><<<plan.grid, kGemmThreads, plan.smem_bytes, st>>>(ma, mb, plan.p);
-    count_launch();
-    CCL_CUDA_TRY(cudaGetLastError());
     return CCL_OK;
+}
+
+template <int BN, int CTAS>
+static ccl_status launch(const GemmPlan& plan, const CUtensorMap& ma, const CUtensorMap& mb, cudaStream_t st) {
+    ccl_status s = configure<BN, CTAS>(plan.smem_bytes);
+    if (s) return s;
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(plan.grid, 1, 1);
+    cfg.blockDim = dim3(kGemmThreads, 1, 1);
+    cfg.dynamicSmemBytes = plan.smem_bytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = CTAS; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    CCL_CUDA_TRY(cudaLaunchKernelEx(&cfg, ccl_gemm_kernel<BN, CTAS>, ma, mb, plan.p));
+    count_launch();
+    return CCL_OK;
+}
+
+// CTA pairs of the 2-CTA kernel that can be resident at once (0 if clusters cannot be launched)
+static int resident_pairs() {
+    static int pairs = -1;
+    if (pairs >= 0) return pairs;
+    uint32_t smem = 224 * 1024 + 2048;
+    if (configure<256, 2>(smem) != CCL_OK) { clear_error(); return pairs = 0; }
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(2, 1, 1); cfg.blockDim = dim3(kGemmThreads, 1, 1); cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, ccl_gemm_kernel<256, 2>, &cfg) != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
+    return pairs = n;
 }
 
 ccl_status repack_status_take(int* code);   // ccl_repack.cu
@@ -463,7 +588,7 @@ using namespace ccl;
 
 extern "C" ccl_status ccl_gemm_workspace(const ccl_gemm_desc* d, size_t* bytes) {
     GemmPlan plan;
-    ccl_status s = make_plan(d, nullptr, nullptr, nullptr, 148, &plan);
+    ccl_status s = make_plan(d, nullptr, nullptr, nullptr, 148, 74, &plan);
     if (s) return s;
     if (!bytes) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm_workspace: NULL output");
     *bytes = 0;
@@ -475,22 +600,27 @@ extern "C" ccl_status ccl_gemm(const ccl_gemm_desc* d, const void* A_dev, const 
     (void)ws_dev; (void)ws_bytes;
     if (!A_dev || !B_dev || !C_dev) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: NULL operand");
     GemmPlan plan;
-    ccl_status s = make_plan(d, A_dev, B_dev, C_dev, 148, &plan);     // validation first: no CUDA call on bad input
+    ccl_status s = make_plan(d, A_dev, B_dev, C_dev, 148, 74, &plan);     // validation first: no CUDA call on bad input
     if (s) return s;
     int dev, sms;
     CCL_CUDA_TRY(cudaGetDevice(&dev));
     CCL_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    if ((s = make_plan(d, A_dev, B_dev, C_dev, sms, &plan))) return s;
+    if ((s = make_plan(d, A_dev, B_dev, C_dev, sms, resident_pairs(), &plan))) return s;
     plan.p.C = static_cast<uint16_t*>(C_dev);
+    const uint32_t bnh = (uint32_t)((plan.bn > 256 ? 256 : plan.bn) / plan.ctas);   // B rows of one K-major box
     CUtensorMap ma, mb;
     if (!plan.p.a_mn) s = operand_tmap(&ma, plan.va, A_dev, BK, BM); else s = operand_tmap(&ma, plan.va, A_dev, 64, BK);
     if (s) return s;
-    if (!plan.p.b_mn) s = operand_tmap(&mb, plan.vb, B_dev, BK, (uint32_t)plan.bn); else s = operand_tmap(&mb, plan.vb, B_dev, 64, BK);
+    if (!plan.p.b_mn) s = operand_tmap(&mb, plan.vb, B_dev, BK, bnh); else s = operand_tmap(&mb, plan.vb, B_dev, 64, BK);
     if (s) return s;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
-    if (plan.bn == 256) return launch<256>(plan, ma, mb, st);
-    if (plan.bn == 192) return launch<192>(plan, ma, mb, st);
-    return launch<128>(plan, ma, mb, st);
+    if (plan.ctas == 2) {
+        if (plan.bn == 512) return launch<512, 2>(plan, ma, mb, st);
+        return plan.bn == 256 ? launch<256, 2>(plan, ma, mb, st) : launch<128, 2>(plan, ma, mb, st);
+    }
+    if (plan.bn == 256) return launch<256, 1>(plan, ma, mb, st);
+    if (plan.bn == 192) return launch<192, 1>(plan, ma, mb, st);
+    return launch<128, 1>(plan, ma, mb, st);
 }
 
 extern "C" ccl_status ccl_gemm_status(void* cuda_stream, int32_t* detail) {

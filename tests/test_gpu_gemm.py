@@ -4,6 +4,7 @@ Tolerance (stated by the benchmark spec): err = |C_gpu - ref32| / max(1, |ref32|) <= 1e-2 
 where ref32 is the oracle's fp32-accumulate sum from the logical (row-major) operands.
 """
 import math
+import os
 
 import numpy as np
 import pytest
@@ -79,8 +80,20 @@ SMALL = [
 ]
 
 
+@pytest.fixture(params=["auto", "1", "2"])
+def cta_mode(request):
+    """Forces the 1-CTA or the 2-CTA (cta_group::2 pair) kernel, or leaves the library's own choice."""
+    old = os.environ.pop("CCL_GEMM_CTAS", None)
+    if request.param != "auto":
+        os.environ["CCL_GEMM_CTAS"] = request.param
+    yield request.param
+    os.environ.pop("CCL_GEMM_CTAS", None)
+    if old is not None:
+        os.environ["CCL_GEMM_CTAS"] = old
+
+
 @pytest.mark.parametrize("M,N,K,P,lay,at,bt,op", SMALL)
-def test_gemm_small_shapes(M, N, K, P, lay, at, bt, op):
+def test_gemm_small_shapes(M, N, K, P, lay, at, bt, op, cta_mode):
     parts = None
     if lay == ("ccl", "ccl", "row") and op == 0:
         parts = (1 if at else 2, 2 if bt else 1, 0)                    # both operands split along K
