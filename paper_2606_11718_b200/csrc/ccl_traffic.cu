@@ -7,10 +7,11 @@
 //
 // Kernels (all integer):
 //   prep      zero the outputs that are accumulated into
-//   hist      per-page demand per chiplet (only when per-page output or BEST placement is asked)
+//   walk      every contiguous run a CTA touches is cut at strip and page boundaries; per piece the
+//             per-page demand is accumulated and/or the piece is classified local / remote.  A is
+//             walked once per tile row and B once per tile column (all tiles of the row / column
+//             touch the same bytes), C once per tile
 //   owner     page -> chiplet for every operand whose owner table is asked for / needed
-//   classify  one warp per (tile, operand): lanes walk the stored rows of the tile's rectangle,
-//             cut every contiguous run at strip and page boundaries, classify, warp-reduce
 #include <algorithm>
 #include <cstring>
 
@@ -104,21 +105,123 @@ __device__ __forceinline__ int32_t fixed_owner(const TrafficParams& p, int X, in
     return (int32_t)min((int64_t)(p.P - 1), o);
 }
 
-constexpr int kWarpsPerBlock = 8;
+constexpr int kWalkThreads = 256;
+constexpr int kWarpsPerBlock = kWalkThreads / 32;
 
-__global__ void __launch_bounds__(kWarpsPerBlock * 32) traffic_hist_kernel(TrafficParams p) {
-    const int lane = threadIdx.x & 31;
-    const int64_t nwork = p.ntiles * 3;
-    for (int64_t wk = (int64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5); wk < nwork; wk += (int64_t)gridDim.x * kWarpsPerBlock) {
-        int64_t t = wk / 3;
-        int X = (int)(wk - t * 3);
-        if (!p.per_page[X]) continue;
-        TileInfo ti = decode_tile(p, t);
+// One pass over every byte the CTAs touch.  HIST accumulates the per-page demand, CLASSIFY the
+// local / remote split.  The A rectangle of a tile depends only on its tile row and the B rectangle
+// only on its tile column, so they are walked ONCE per tile row / column by a whole block, which
+// records how many bytes each chiplet owns (and which chiplets the sharing tiles run on) and then
+// hands every tile of the row / column its numbers; only C is walked per tile (one warp each).
+//   blocks [0, tiles_m)                    : A of tile row j
+//   blocks [tiles_m, tiles_m + tiles_n)    : B of tile column j
+//   the rest                               : C, kWarpsPerBlock tiles per block
+template <bool HIST, bool CLASSIFY>
+__global__ void __launch_bounds__(kWalkThreads) traffic_walk_kernel(TrafficParams p) {
+    __shared__ unsigned long long own[256];       // bytes of the rectangle whose page belongs to chiplet o
+    __shared__ unsigned int cnt[256];             // tiles sharing the rectangle that run on chiplet q
+    __shared__ unsigned long long blk[6];
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int64_t item = blockIdx.x;
+    if (tid < 6) blk[tid] = 0;
+    if (item < p.tiles_m + p.tiles_n) {
+        const int X = item < p.tiles_m ? 0 : 1;
+        const int64_t j = X == 0 ? item : item - p.tiles_m;
+        const bool do_hist = HIST && p.per_page[X] != nullptr;
+        if (!do_hist && !CLASSIFY) return;
+        const int64_t nshare = X == 0 ? p.tiles_n : p.tiles_m;                  // tiles that touch this rectangle
+        const int64_t t_first = X == 0 ? j * p.tiles_n : j, t_step = X == 0 ? 1 : p.tiles_n;
+        for (int i = tid; i < p.P; i += kWalkThreads) { own[i] = 0; cnt[i] = 0; }
+        __syncthreads();
+        if (do_hist) {
+            for (int64_t o = tid; o < nshare; o += kWalkThreads) atomicAdd(&cnt[decode_tile(p, t_first + o * t_step).q], 1u);
+            __syncthreads();
+        }
+        const TileInfo ti = decode_tile(p, t_first);
         int64_t r0, r1, c0, c1;
         tile_rect(p, ti, X, r0, r1, c0, c1);
+        const bool table = p.place[X] == CCL_PLACE_BEST;
+        const uint8_t* own_tab = p.owner[X];
         unsigned long long* hist = reinterpret_cast<unsigned long long*>(p.per_page[X]);
-        for (int64_t r = r0 + lane; r < r1; r += 32)
-            walk_row(p, p.v[X], r, c0, c1, [&](int64_t page, int64_t len) { atomicAdd(&hist[page * p.P + ti.q], (unsigned long long)len); });
+        // bytes per owning chiplet: kept in registers while P <= 8 (the usual case; all threads of a block
+        // tend to hit the same owner, which would serialise shared-memory atomics), else in shared memory
+        const bool small_p = p.P <= 8;
+        unsigned long long acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        for (int64_t r = r0 + tid; r < r1; r += kWalkThreads)
+            walk_row(p, p.v[X], r, c0, c1, [&](int64_t page, int64_t len) {
+                if (do_hist)
+                    for (int q = 0; q < p.P; ++q) { const unsigned int n = cnt[q]; if (n) atomicAdd(&hist[page * p.P + q], (unsigned long long)len * n); }
+                if (CLASSIFY) {
+                    const int32_t o = table ? (int32_t)own_tab[page] : fixed_owner(p, X, page);
+                    if (small_p) {
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) acc[q] += (o == q) ? (unsigned long long)len : 0ull;
+                    } else atomicAdd(&own[o], (unsigned long long)len);
+                }
+            });
+        if (CLASSIFY && small_p) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                unsigned long long v = acc[q];
+#pragma unroll
+                for (int s2 = 16; s2 > 0; s2 >>= 1) v += __shfl_xor_sync(0xffffffffu, v, s2);
+                if (lane == 0 && v) atomicAdd(&own[q], v);
+            }
+        }
+        if (CLASSIFY) {
+            __syncthreads();
+            unsigned long long total = 0, loc_sum = 0, rem_sum = 0;
+            for (int o = 0; o < p.P; ++o) total += own[o];
+            for (int64_t o = tid; o < nshare; o += kWalkThreads) {
+                const int64_t t = t_first + o * t_step;
+                const unsigned long long loc = own[decode_tile(p, t).q];
+                p.per_cta[t * 6 + X * 2 + 0] = loc;
+                p.per_cta[t * 6 + X * 2 + 1] = total - loc;
+                loc_sum += loc; rem_sum += total - loc;
+            }
+            if (loc_sum) atomicAdd(&blk[X * 2 + 0], loc_sum);
+            if (rem_sum) atomicAdd(&blk[X * 2 + 1], rem_sum);
+        }
+    } else {
+        const int X = 2;
+        const bool do_hist = HIST && p.per_page[X] != nullptr;
+        if (!do_hist && !CLASSIFY) return;
+        __syncthreads();                                  // blk[] zeroed
+        const int64_t t = (item - p.tiles_m - p.tiles_n) * kWarpsPerBlock + (tid >> 5);
+        if (t < p.ntiles) {
+            const TileInfo ti = decode_tile(p, t);
+            int64_t r0, r1, c0, c1;
+            tile_rect(p, ti, X, r0, r1, c0, c1);
+            const bool table = p.place[X] == CCL_PLACE_BEST;
+            const uint8_t* own_tab = p.owner[X];
+            unsigned long long* hist = reinterpret_cast<unsigned long long*>(p.per_page[X]);
+            unsigned long long loc = 0, rem = 0;
+            for (int64_t r = r0 + lane; r < r1; r += 32)
+                walk_row(p, p.v[X], r, c0, c1, [&](int64_t page, int64_t len) {
+                    if (do_hist) atomicAdd(&hist[page * p.P + ti.q], (unsigned long long)len);
+                    if (CLASSIFY) {
+                        const int32_t o = table ? (int32_t)own_tab[page] : fixed_owner(p, X, page);
+                        if (o == ti.q) loc += (unsigned long long)len; else rem += (unsigned long long)len;
+                    }
+                });
+            if (CLASSIFY) {
+#pragma unroll
+                for (int s = 16; s > 0; s >>= 1) {
+                    loc += __shfl_xor_sync(0xffffffffu, loc, s);
+                    rem += __shfl_xor_sync(0xffffffffu, rem, s);
+                }
+                if (lane == 0) {
+                    p.per_cta[t * 6 + 4] = loc;
+                    p.per_cta[t * 6 + 5] = rem;
+                    atomicAdd(&blk[4], loc);
+                    atomicAdd(&blk[5], rem);
+                }
+            }
+        }
+    }
+    if (CLASSIFY) {
+        __syncthreads();
+        if (tid < 6 && blk[tid]) atomicAdd(reinterpret_cast<unsigned long long*>(p.totals) + tid, blk[tid]);
     }
 }
 
@@ -136,42 +239,6 @@ __global__ void traffic_owner_kernel(TrafficParams p) {
             p.owner[X][pg] = (uint8_t)o;
         }
     }
-}
-
-__global__ void __launch_bounds__(kWarpsPerBlock * 32) traffic_classify_kernel(TrafficParams p) {
-    __shared__ unsigned long long blk[6];
-    if (threadIdx.x < 6) blk[threadIdx.x] = 0;
-    __syncthreads();
-    const int lane = threadIdx.x & 31;
-    const int64_t nwork = p.ntiles * 3;
-    for (int64_t wk = (int64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5); wk < nwork; wk += (int64_t)gridDim.x * kWarpsPerBlock) {
-        int64_t t = wk / 3;
-        int X = (int)(wk - t * 3);
-        TileInfo ti = decode_tile(p, t);
-        int64_t r0, r1, c0, c1;
-        tile_rect(p, ti, X, r0, r1, c0, c1);
-        unsigned long long loc = 0, rem = 0;
-        const bool table = p.place[X] == CCL_PLACE_BEST;
-        const uint8_t* own = p.owner[X];
-        for (int64_t r = r0 + lane; r < r1; r += 32)
-            walk_row(p, p.v[X], r, c0, c1, [&](int64_t page, int64_t len) {
-                int32_t o = table ? (int32_t)own[page] : fixed_owner(p, X, page);
-                if (o == ti.q) loc += (unsigned long long)len; else rem += (unsigned long long)len;
-            });
-#pragma unroll
-        for (int s = 16; s > 0; s >>= 1) {
-            loc += __shfl_xor_sync(0xffffffffu, loc, s);
-            rem += __shfl_xor_sync(0xffffffffu, rem, s);
-        }
-        if (lane == 0) {
-            p.per_cta[t * 6 + X * 2 + 0] = loc;
-            p.per_cta[t * 6 + X * 2 + 1] = rem;
-            atomicAdd(&blk[X * 2 + 0], loc);
-            atomicAdd(&blk[X * 2 + 1], rem);
-        }
-    }
-    __syncthreads();
-    if (threadIdx.x < 6 && blk[threadIdx.x]) atomicAdd(reinterpret_cast<unsigned long long*>(p.totals) + threadIdx.x, blk[threadIdx.x]);
 }
 
 static ccl_status fill_params(const ccl_traffic_desc* d, TrafficParams* p) {
@@ -261,20 +328,31 @@ extern "C" ccl_status ccl_traffic(const ccl_traffic_desc* d, const int32_t* cta_
     count_launch();
     CCL_CUDA_TRY(cudaGetLastError());
 
-    int64_t nwork = p.ntiles * 3;
-    unsigned grid = (unsigned)std::max<int64_t>(1, std::min<int64_t>((nwork + kWarpsPerBlock - 1) / kWarpsPerBlock, (int64_t)sms * 8));
-    if (need_hist) {
-        traffic_hist_kernel<<<grid, kWarpsPerBlock * 32, 0, st>>>(p);
+    bool any_best = false;
+    for (int X = 0; X < 3; ++X) any_best |= p.place[X] == CCL_PLACE_BEST;
+    const int64_t nblocks = p.tiles_m + p.tiles_n + (p.ntiles + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    if (nblocks >= (INT64_C(1) << 31)) return fail(CCL_ERR_UNSUPPORTED, "ccl_traffic: too many tiles");
+    const unsigned grid = (unsigned)nblocks;
+    if (any_best) {                       // demand first, then the owner table, then the classification that reads it
+        traffic_walk_kernel<true, false><<<grid, kWalkThreads, 0, st>>>(p);
         count_launch();
         CCL_CUDA_TRY(cudaGetLastError());
-    }
-    if (need_owner) {
         traffic_owner_kernel<<<sms * 2, 256, 0, st>>>(p);
         count_launch();
         CCL_CUDA_TRY(cudaGetLastError());
+        traffic_walk_kernel<false, true><<<grid, kWalkThreads, 0, st>>>(p);
+        count_launch();
+        CCL_CUDA_TRY(cudaGetLastError());
+    } else {
+        if (need_hist) traffic_walk_kernel<true, true><<<grid, kWalkThreads, 0, st>>>(p);
+        else traffic_walk_kernel<false, true><<<grid, kWalkThreads, 0, st>>>(p);
+        count_launch();
+        CCL_CUDA_TRY(cudaGetLastError());
+        if (need_owner) {
+            traffic_owner_kernel<<<sms * 2, 256, 0, st>>>(p);
+            count_launch();
+            CCL_CUDA_TRY(cudaGetLastError());
+        }
     }
-    traffic_classify_kernel<<<grid, kWarpsPerBlock * 32, 0, st>>>(p);
-    count_launch();
-    CCL_CUDA_TRY(cudaGetLastError());
     return CCL_OK;
 }
