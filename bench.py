@@ -137,17 +137,13 @@ def run_cuda(args):
     import torch
     from paper_2606_11718_b200 import binding as ccl
     from paper_2606_11718_b200 import synth
+    from paper_2606_11718_b200 import dist as ccl_dist
 
-    rank = int(os.environ.get("RANK", 0))
-    world = int(os.environ.get("WORLD_SIZE", 1))
-    local = int(os.environ.get("LOCAL_RANK", 0))
+    rank, world, local = ccl_dist.env_world()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py: no CUDA device (there is no CPU fallback; use --impl reference for the oracle)")
     torch.cuda.set_device(local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    group = ccl_dist.Group("nccl", torch.device("cuda", local))
     ccl.lib()
     P, page = args.P, args.page
     descs = make_descs(ccl, P, page)
@@ -189,17 +185,7 @@ def run_cuda(args):
                 kernel_events["repack"].append((e[0], e[1])); kernel_events["gemm"].append((e[1], e[2]))
                 kernel_events["traffic"].append((e[2], e[3]))
 
-    def barrier():
-        if dist is not None:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    def max_over_ranks(ms):
-        if dist is None:
-            return ms
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    barrier, max_over_ranks = group.barrier, group.max_over_ranks
 
     # ---- device-resident timing
     for _ in range(args.warmup):
@@ -287,8 +273,7 @@ def run_cuda(args):
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = oracle_sample(P, page, synth, host)
         print(json.dumps(line), flush=True)
-    if dist is not None:
-        dist.destroy_process_group()
+    group.close()
 
 
 # ---------------------------------------------------------------------------------------------
