@@ -61,6 +61,8 @@ struct GemmParams {
     uint32_t idesc;
     int32_t stages;
     uint32_t stage_bytes, a_bytes;  // bytes per stage per CTA, bytes of its A part
+    int32_t splits, kb_per_split;   // split-K: each tile is computed by `splits` units over disjoint k-block ranges
+    float* ws;                      // split-K partial sums, [splits][M][N] fp32 (row-major, logical coordinates)
 };
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
@@ -153,7 +155,7 @@ __device__ __forceinline__ void to_coords(const OpMap& o, int r, int c, int& x, 
     else { x = c; y = r; z = 0; }
 }
 
-struct TileCoord { int m0, m1, n0, n1; };
+struct TileCoord { int m0, m1, n0, n1, split; };
 
 // Tiles of this CTA (pair).  The schedulable units (CTAs, or CTA pairs) are cut into `groups`
 // contiguous ranges; group g owns the tiles of strip range g (chiplet-grouped raster) and walks
@@ -170,7 +172,7 @@ struct Scheduler {
     __device__ Scheduler(const GemmParams& p_, int unit_, int units_, int bm_, int bn_) : p(p_), unit(unit_), units(units_), bm(bm_), bn(bn_) {
         gm = p.tiles_m; gn = p.tiles_n;
         if (p.groups > 1) { if (p.group_dim == 0) gn = p.tiles_n / p.groups; else gm = p.tiles_m / p.groups; }
-        per_group = (int64_t)gm * gn;
+        per_group = (int64_t)gm * gn * p.splits;
         my_g = 0; rounds = 0x7fffffff;
         for (int g = 0; g < p.groups; ++g) {
             int l = lo(g), h = lo(g + 1);
@@ -191,6 +193,8 @@ struct Scheduler {
             }
             if (g == p.groups) return false;
         }
+        t.split = (int)(i % p.splits);                   // the splits of one tile are neighbours in the walk
+        i /= p.splits;
         int64_t per_panel = (int64_t)p.panel * gn;
         int pn = (int)(i / per_panel);
         int rem = (int)(i - (int64_t)pn * per_panel);
@@ -273,7 +277,8 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             const int base = (isA ? t.m0 : t.n0) + off;
             int x, y, z;
             if (mn) to_coords(om, 0, base, x, y, z); else to_coords(om, base, 0, x, y, z);
-            for (int kb = 0; kb < p.num_kb; ++kb) {
+            const int kb0 = t.split * p.kb_per_split, kb1 = min(p.num_kb, kb0 + p.kb_per_split);
+            for (int kb = kb0; kb < kb1; ++kb) {
                 ok = mbar_wait_bounded(&empty[stage], phase ^ 1);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) { if (lane == 0) atomicExch(&g_gemm_status, 1); break; }
@@ -302,14 +307,15 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 //            of the previous tile has drained it.
                 const int acc0 = NSUB == 1 ? (it & 1) : 0;
                 const uint32_t acc_phase = NSUB == 1 ? ((uint32_t)(it >> 1) & 1) : ((uint32_t)it & 1);
-                for (int kb = 0; ok && kb < p.num_kb; ++kb) {
+                const int kb0 = t.split * p.kb_per_split, kb1 = min(p.num_kb, kb0 + p.kb_per_split);
+                for (int kb = kb0; ok && kb < kb1; ++kb) {
                     if (!mbar_wait_bounded(&full[stage], phase)) { atomicExch(&g_gemm_status, 3); ok = false; break; }
                     tc_fence_after();
                     const uint32_t sa = smem_u32(smem + (size_t)stage * p.stage_bytes);
                     const uint64_t adesc = smem_desc(sa, a_lbo, 1024);
 #pragma unroll
                     for (int h = 0; h < NSUB; ++h) {
-                        if (kb == 0) {
+                        if (kb == kb0) {
                             if (!mbar_wait_bounded(&tmem_empty[acc0 + h], acc_phase ^ 1)) { atomicExch(&g_gemm_status, 2); ok = false; break; }
                             tc_fence_after();
                         }
@@ -317,7 +323,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                         const uint64_t bdesc = smem_desc(sa + p.a_bytes + h * (SUBH * BK * 2), b_lbo, 1024);
 #pragma unroll
                         for (int k = 0; k < BK / 16; ++k)
-                            umma_bf16<CTAS>(tmem_d, adesc + (uint64_t)(k * a_kstep), bdesc + (uint64_t)(k * b_kstep), p.idesc, (kb | k) != 0);
+                            umma_bf16<CTAS>(tmem_d, adesc + (uint64_t)(k * a_kstep), bdesc + (uint64_t)(k * b_kstep), p.idesc, ((kb - kb0) | k) != 0);
                     }
                     if (!ok) break;
                     umma_commit<CTAS>(&empty[stage]);          // frees the stage (in both CTAs) once these MMAs have read it
@@ -357,7 +363,17 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 uint32_t r[32];
                 tmem_ld32(taddr + (uint32_t)(c * 32), r);
                 tmem_ld_wait();
-                if (m < t.m1) {
+                if (p.splits > 1) {                      // partial sums, summed in fixed order by splitk_reduce_kernel
+                    if (m < t.m1) {
+                        float* wrow = p.ws + ((int64_t)t.split * p.M + m) * (int64_t)p.N;
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            const int n = nb + c * 32 + j * 4;
+                            if (n < t.n1)
+                                *reinterpret_cast<uint4*>(wrow + n) = make_uint4(r[j * 4 + 0], r[j * 4 + 1], r[j * 4 + 2], r[j * 4 + 3]);
+                        }
+                    }
+                } else if (m < t.m1) {
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         const int n = nb + c * 32 + j * 8;
@@ -392,12 +408,42 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     }
 }
 
+// Split-K epilogue: C = bf16( ws[0] + ws[1] + ... + ws[splits-1] ), the sum taken in that fixed order so
+// the result is the same on every run.  One thread per 8 consecutive columns of a row.
+__global__ void __launch_bounds__(256) splitk_reduce_kernel(const GemmParams p) {
+    const int64_t n8 = p.N / 8, total = (int64_t)p.M * n8;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t m = i / n8, n = (i - m * n8) * 8;
+        float acc[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[j] = 0.0f;
+        for (int sp = 0; sp < p.splits; ++sp) {
+            const float4* src = reinterpret_cast<const float4*>(p.ws + ((int64_t)sp * p.M + m) * (int64_t)p.N + n);
+            const float4 x = src[0], y = src[1];
+            acc[0] += x.x; acc[1] += x.y; acc[2] += x.z; acc[3] += x.w;
+            acc[4] += y.x; acc[5] += y.y; acc[6] += y.z; acc[7] += y.w;
+        }
+        int64_t off;
+        if (p.c_split == 2) { int64_t g = n / p.c_w; off = g * p.c_stride + m * p.c_w + (n - g * p.c_w); }
+        else if (p.c_split == 1) { int64_t g = m / p.c_h; off = g * p.c_stride + (m - g * p.c_h) * p.c_cols + n; }
+        else off = m * p.c_cols + n;
+        uint4 v;
+        __nv_bfloat162 h;
+        h = __floats2bfloat162_rn(acc[0], acc[1]); v.x = *reinterpret_cast<uint32_t*>(&h);
+        h = __floats2bfloat162_rn(acc[2], acc[3]); v.y = *reinterpret_cast<uint32_t*>(&h);
+        h = __floats2bfloat162_rn(acc[4], acc[5]); v.z = *reinterpret_cast<uint32_t*>(&h);
+        h = __floats2bfloat162_rn(acc[6], acc[7]); v.w = *reinterpret_cast<uint32_t*>(&h);
+        *reinterpret_cast<uint4*>(p.C + off) = v;
+    }
+}
+
 // ------------------------------------------------------------------------------------------
 // Host side
 // ------------------------------------------------------------------------------------------
 struct GemmPlan {
     GemmParams p;
     int bn, ctas;
+    size_t ws_bytes;
     MatView va, vb, vc;
     uint32_t smem_bytes;
     unsigned grid;
@@ -472,23 +518,45 @@ static ccl_status make_plan(const ccl_gemm_desc* d, const void* A, const void* B
     if (!Wm) Wm = d->M;
     if (!Wn) Wn = d->N;
 
-    // tile shape: least padded work per strip, ties to the wider tile; the 2-CTA kernel (256-row tiles,
-    // BN in {256,128}) is taken unless it pads noticeably more than the 1-CTA kernel (BN in {256,192,128})
-    int bn1 = 256, bn2 = 256;
-    for (int bn : {192, 128}) if (padded(Wn, bn) < padded(Wn, bn1)) bn1 = bn;
-    if (padded(Wn, 128) < padded(Wn, 256)) bn2 = 128;
-    // 256 x 512 pair tiles move 25% fewer operand bytes per flop (the L2 -> SM fill rate is what bounds
-    // the 256 x 256 kernel); they are worth a little padding, and need K long enough to amortise the
-    // epilogue that is only half overlapped
-    if (padded(Wn, 512) <= 1.05 * padded(Wn, bn2) && d->K >= 1024) bn2 = 512;
-    double work1 = (double)padded(Wm, 128) * (double)padded(Wn, bn1), work2 = (double)padded(Wm, 256) * (double)padded(Wn, bn2);
-    int ctas = (pairs > 0 && work2 <= 1.08 * work1) ? 2 : 1;
-    if (const char* f = std::getenv("CCL_GEMM_CTAS")) { if (f[0] == '1') ctas = 1; else if (f[0] == '2' && pairs > 0) ctas = 2; }
-    if (const char* f = std::getenv("CCL_GEMM_BN")) { int v = atoi(f); if (ctas == 2 && (v == 512 || v == 256 || v == 128)) bn2 = v; if (ctas == 1 && (v == 256 || v == 192 || v == 128)) bn1 = v; }
-    const int bn = ctas == 2 ? bn2 : bn1;
+    // Tile shape, CTA pairing and split-K from a small cost model (cycles per unit):
+    //   a k block takes max(MMA time, time to pull this SM's operand bytes from L2 at ~50 B/clk);
+    //   a unit pays ~3000 cycles of pipeline fill + epilogue; split-K adds the partial-sum traffic.
+    // 256 x 512 pair tiles move the fewest bytes per flop; small problems prefer 1-CTA tiles and split-K.
+    const int64_t num_kb = (d->K + BK - 1) / BK;
+    const int64_t strips_m = d->M / Wm, strips_n = d->N / Wn;
+    int ctas = 1, bn = 256, splits = 1;
+    double best = -1.0;
+    const char* force_ctas = std::getenv("CCL_GEMM_CTAS");
+    const char* force_bn = std::getenv("CCL_GEMM_BN");
+    const char* force_split = std::getenv("CCL_GEMM_SPLITK");
+    for (int c = 1; c <= 2; ++c) {
+        if (c == 2 && pairs <= 0) continue;
+        if (force_ctas && atoi(force_ctas) != c) continue;
+        const int units = c == 2 ? pairs : sms;
+        for (int b : {512, 256, 192, 128}) {
+            if (c == 1 && b == 512) continue;
+            if (c == 2 && b == 192) continue;
+            if (force_bn && atoi(force_bn) != b) continue;
+            const int64_t tiles = strips_m * ((Wm + BM * c - 1) / (BM * c)) * strips_n * ((Wn + b - 1) / b);
+            const double t_kb = std::max((double)b / 256.0 * 512.0, (128.0 + (double)b / c) * 2.56);
+            for (int sp : {1, 2, 3, 4, 6, 8, 12, 16}) {
+                if (sp > 1 && (c == 2 || num_kb / sp < 2)) continue;
+                if (force_split && atoi(force_split) != sp) continue;
+                const int64_t kbps = (num_kb + sp - 1) / sp;
+                const int64_t sp_eff = (num_kb + kbps - 1) / kbps;          // every split owns at least one k block
+                if (sp_eff != sp) continue;
+                const int64_t waves = (tiles * sp + units - 1) / units;
+                double cost = (double)waves * ((double)kbps * t_kb + 3000.0);
+                if (sp > 1) cost += ((double)sp + 0.5) * (double)d->M * (double)d->N * 4.0 / 3400.0 + 4000.0;
+                if (best < 0 || cost < best) { best = cost; ctas = c; bn = b; splits = sp; }
+            }
+        }
+    }
+    if (best < 0) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: no kernel variant matches the forced CCL_GEMM_* settings");
     const int subn = bn > 256 ? 256 : bn;                // columns of one MMA / one TMEM accumulator
     const int bm = BM * ctas;
     plan->bn = bn; plan->ctas = ctas;
+    plan->ws_bytes = splits > 1 ? (size_t)splits * (size_t)d->M * (size_t)d->N * 4 : 0;
 
     GemmParams& p = plan->p;
     std::memset(&p, 0, sizeof(p));
@@ -496,7 +564,8 @@ static ccl_status make_plan(const ccl_gemm_desc* d, const void* A, const void* B
     p.Wm = (int32_t)Wm; p.Wn = (int32_t)Wn;
     p.tps_m = (int32_t)((Wm + bm - 1) / bm); p.tps_n = (int32_t)((Wn + bn - 1) / bn);
     p.tiles_m = (int32_t)(d->M / Wm) * p.tps_m; p.tiles_n = (int32_t)(d->N / Wn) * p.tps_n;
-    p.num_kb = (int32_t)((d->K + BK - 1) / BK);
+    p.num_kb = (int32_t)num_kb;
+    p.splits = splits; p.kb_per_split = (int32_t)((num_kb + splits - 1) / splits);
     p.a.split = va.split; p.a.w = (int32_t)va.w; p.a.h = (int32_t)va.h;
     p.b.split = vb.split; p.b.w = (int32_t)vb.w; p.b.h = (int32_t)vb.h;
     p.a_mn = at ? 1 : 0; p.b_mn = bt ? 0 : 1;
@@ -511,7 +580,7 @@ static ccl_status make_plan(const ccl_gemm_desc* d, const void* A, const void* B
     if (p.stages > 8) p.stages = 8;
     p.panel = 16;
     if (const char* f = std::getenv("CCL_GEMM_PANEL")) p.panel = std::max(1, atoi(f));
-    int64_t ntiles = (int64_t)p.tiles_m * p.tiles_n;
+    int64_t ntiles = (int64_t)p.tiles_m * p.tiles_n * splits;
     int units = (int)std::min<int64_t>(ntiles, ctas == 2 ? pairs : sms);
     plan->grid = (unsigned)(units * ctas);
     // grouped raster needs at least one unit per group and whole strips per group
@@ -586,18 +655,32 @@ ccl_status repack_status_take(int* code);   // ccl_repack.cu
 
 using namespace ccl;
 
+// SM count and resident CTA pairs of the current device; the figures of a B200 when no device is usable
+// (the planner then still validates and sizes the workspace the same way a B200 would).
+static void device_units(int* sms, int* pairs) {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) {
+        *sms = n; *pairs = resident_pairs();
+    } else {
+        (void)cudaGetLastError();
+        *sms = 148; *pairs = 74;
+    }
+}
+
 extern "C" ccl_status ccl_gemm_workspace(const ccl_gemm_desc* d, size_t* bytes) {
     GemmPlan plan;
-    ccl_status s = make_plan(d, nullptr, nullptr, nullptr, 148, 74, &plan);
+    ccl_status s = make_plan(d, nullptr, nullptr, nullptr, 148, 74, &plan);     // validation without any CUDA call
     if (s) return s;
     if (!bytes) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm_workspace: NULL output");
-    *bytes = 0;
+    int sms, pairs;
+    device_units(&sms, &pairs);
+    if ((s = make_plan(d, nullptr, nullptr, nullptr, sms, pairs, &plan))) return s;
+    *bytes = plan.ws_bytes;
     return CCL_OK;
 }
 
 extern "C" ccl_status ccl_gemm(const ccl_gemm_desc* d, const void* A_dev, const void* B_dev, void* C_dev, void* ws_dev,
                                size_t ws_bytes, void* cuda_stream) {
-    (void)ws_dev; (void)ws_bytes;
     if (!A_dev || !B_dev || !C_dev) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: NULL operand");
     GemmPlan plan;
     ccl_status s = make_plan(d, A_dev, B_dev, C_dev, 148, 74, &plan);     // validation first: no CUDA call on bad input
@@ -606,7 +689,13 @@ extern "C" ccl_status ccl_gemm(const ccl_gemm_desc* d, const void* A_dev, const 
     CCL_CUDA_TRY(cudaGetDevice(&dev));
     CCL_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     if ((s = make_plan(d, A_dev, B_dev, C_dev, sms, resident_pairs(), &plan))) return s;
+    if (plan.ws_bytes) {
+        if (!ws_dev || ws_bytes < plan.ws_bytes)
+            return fail(CCL_ERR_WORKSPACE, "ccl_gemm: this problem is split along K and needs %zu bytes of workspace (got %zu)", plan.ws_bytes, ws_dev ? ws_bytes : (size_t)0);
+        if (reinterpret_cast<uintptr_t>(ws_dev) & 15) return fail(CCL_ERR_ALIGN, "ccl_gemm: workspace is not 16-byte aligned");
+    }
     plan.p.C = static_cast<uint16_t*>(C_dev);
+    plan.p.ws = static_cast<float*>(ws_dev);
     const uint32_t bnh = (uint32_t)((plan.bn > 256 ? 256 : plan.bn) / plan.ctas);   // B rows of one K-major box
     CUtensorMap ma, mb;
     if (!plan.p.a_mn) s = operand_tmap(&ma, plan.va, A_dev, BK, BM); else s = operand_tmap(&ma, plan.va, A_dev, 64, BK);
@@ -615,12 +704,20 @@ extern "C" ccl_status ccl_gemm(const ccl_gemm_desc* d, const void* A_dev, const 
     if (s) return s;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
     if (plan.ctas == 2) {
-        if (plan.bn == 512) return launch<512, 2>(plan, ma, mb, st);
-        return plan.bn == 256 ? launch<256, 2>(plan, ma, mb, st) : launch<128, 2>(plan, ma, mb, st);
+        if (plan.bn == 512) s = launch<512, 2>(plan, ma, mb, st);
+        else s = plan.bn == 256 ? launch<256, 2>(plan, ma, mb, st) : launch<128, 2>(plan, ma, mb, st);
+    } else if (plan.bn == 256) s = launch<256, 1>(plan, ma, mb, st);
+    else if (plan.bn == 192) s = launch<192, 1>(plan, ma, mb, st);
+    else s = launch<128, 1>(plan, ma, mb, st);
+    if (s) return s;
+    if (plan.p.splits > 1) {
+        int64_t work = (int64_t)plan.p.M * (plan.p.N / 8);
+        unsigned grid = (unsigned)std::max<int64_t>(1, std::min<int64_t>((work + 255) / 256, (int64_t)sms * 8));
+        splitk_reduce_kernel<<<grid, 256, 0, st>>>(plan.p);
+        count_launch();
+        CCL_CUDA_TRY(cudaGetLastError());
     }
-    if (plan.bn == 256) return launch<256, 1>(plan, ma, mb, st);
-    if (plan.bn == 192) return launch<192, 1>(plan, ma, mb, st);
-    return launch<128, 1>(plan, ma, mb, st);
+    return CCL_OK;
 }
 
 extern "C" ccl_status ccl_gemm_status(void* cuda_stream, int32_t* detail) {

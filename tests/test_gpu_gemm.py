@@ -39,7 +39,9 @@ def run_gemm(d, A, B):
     """A, B: bf16 CPU tensors as stored (row-major).  Returns C as uint16 bits [M x N] (logical order)."""
     a_dev, b_dev = to_layout(synth.bits(A), d.A), to_layout(synth.bits(B), d.B)
     c_dev = torch.full((ccl.ccl_buffer_bytes(d.C) // 2,), 0x7FC0, dtype=torch.int16, device="cuda")   # NaN poison
-    ccl.ccl_gemm(d, a_dev, b_dev, c_dev)
+    need = ccl.ccl_gemm_workspace(d)
+    ws = torch.full((need // 4,), float("nan"), dtype=torch.float32, device="cuda") if need else None
+    ccl.ccl_gemm(d, a_dev, b_dev, c_dev, ws)
     st, detail = ccl.ccl_gemm_status()
     assert st == ccl.OK, detail
     return from_layout(c_dev, d.C)
@@ -204,3 +206,69 @@ def test_gemm_llama_full_size_sampled(name, P):
         # bf16 rounding of C: each element off by <= 2^-9 relative; random signs -> sqrt(N) growth, 8 sigma margin
         bound = 8 * math.sqrt(N) * sigma_c * 2.0 ** -8
         assert (lhs - rhs).abs().max().item() <= bound
+
+
+@pytest.fixture(params=["auto", "1", "2", "4", "8"])
+def split_mode(request):
+    """Forces the number of K splits of the 1-CTA kernel (partial sums in the workspace, fixed-order reduction)."""
+    keys = ("CCL_GEMM_SPLITK", "CCL_GEMM_CTAS")
+    old = {k: os.environ.pop(k, None) for k in keys}
+    if request.param != "auto":
+        os.environ["CCL_GEMM_SPLITK"] = request.param
+        os.environ["CCL_GEMM_CTAS"] = "1"
+    yield request.param
+    for k in keys:
+        os.environ.pop(k, None)
+        if old[k] is not None:
+            os.environ[k] = old[k]
+
+
+@pytest.mark.parametrize("M,N,K,P,at,bt", [(130, 384, 1000, 2, 0, 0), (16, 512, 2048, 4, 0, 1), (1, 768, 1536, 4, 0, 0),
+                                           (264, 768, 1088, 3, 1, 0)])
+def test_gemm_split_k(M, N, K, P, at, bt, split_mode):
+    A, B = synth.gemm_operands(M, N, K, at, bt, seed=5, tag="splitk")
+    d = gemm_desc(M, N, K, P, ("row", "ccl", "ccl"), at, bt, 2, 1)
+    try:
+        need = ccl.ccl_gemm_workspace(d)
+    except ccl.CclError as e:                                          # e.g. 8 splits of 17 k blocks: some split would be empty
+        assert e.status == ccl.ERR_UNSUPPORTED
+        pytest.skip("forced split count does not divide this K")
+    if split_mode not in ("auto", "1"):
+        assert need == int(split_mode) * M * N * 4
+    got1, _ = check(d, A, B)
+    got2, _ = check(d, A, B)
+    np.testing.assert_array_equal(got1, got2)                          # fixed-order reduction: run-to-run identical
+    if need:                                                           # too small a workspace is refused, nothing runs
+        a_dev, b_dev = to_layout(synth.bits(A), d.A), to_layout(synth.bits(B), d.B)
+        c_dev = torch.zeros(M * N, dtype=torch.int16, device="cuda")
+        with pytest.raises(ccl.CclError) as ei:
+            ccl.ccl_gemm(d, a_dev, b_dev, c_dev, torch.empty(need // 4 - 4, dtype=torch.float32, device="cuda"))
+        assert ei.value.status == ccl.ERR_WORKSPACE
+        with pytest.raises(ccl.CclError):
+            ccl.ccl_gemm(d, a_dev, b_dev, c_dev, None)
+
+
+@pytest.mark.parametrize("name", ["llama_fwd_down", "llama_fwd_gateup"])
+def test_gemm_small_m_sweep_llama_shapes(name):
+    """The token-count sweep at weight-streaming sizes: M in {1, 16, 128} on the full Llama weight matrices."""
+    g = {x["name"]: x for x in synth.llama_fwd_gemms()}[name]
+    N, K = g["N"], g["K"]
+    Bfull = synth.randn_bf16(K, N, synth.WEIGHT_STD, 0, name + "/B")
+    for M, Ps in ((1, (4,)), (16, (2, 8)), (128, (4,))):
+        A = synth.randn_bf16(M, K, synth.ACT_STD, 0, f"{name}/A{M}")
+        for P in Ps:
+            d = gemm_desc(M, N, K, P, ("row", "ccl", "ccl"), 0, 0, 2, 1)
+            got = run_gemm(d, A, Bfull)
+            gf = synth.from_bits(got).to(torch.float32).numpy()
+            assert np.isfinite(gf).all()
+            rng = np.random.default_rng(M * 10 + P)
+            cols = sorted({0, N - 256, *(int(c) for c in rng.integers(0, N // 256, size=6) * 256)})
+            for n0 in cols:                                            # sampled 256-column blocks, all rows
+                ref32, _, _ = orc.gemm(synth.bits(A), synth.bits(Bfull), M, N, K, 0, 0, block=(0, M, n0, n0 + 256))
+                err = np.abs(gf[:, n0:n0 + 256] - ref32) / np.maximum(1.0, np.abs(ref32))
+                assert err.max() <= tol(K), (M, P, n0, err.max())
+            # every column: projection on a random +-1 vector over rows is cheap here (M is small): full check in fp64
+            full = (A.to(torch.float64) @ Bfull.to(torch.float64)).numpy() if M <= 16 else None
+            if full is not None:
+                err = np.abs(gf - full) / np.maximum(1.0, np.abs(full))
+                assert err.max() <= tol(K)
