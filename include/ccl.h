@@ -135,6 +135,34 @@ ccl_status ccl_gemm(const ccl_gemm_desc* d, const void* A_dev, const void* B_dev
  */
 ccl_status ccl_gemm_status(void* cuda_stream, int32_t* detail);
 
+/*
+ * Variant of ccl_gemm for callers that must not allocate.  (The paper has no counterpart: this is
+ * a convenience of this library, not part of the method.)
+ *
+ * Who needs it: code that runs where a device allocation is off the table -- a serving loop whose
+ * host framework hands out every byte of device memory up front and treats any cudaMalloc as a bug,
+ * a plug-in called from inside another allocator, a latency-critical step that cannot afford the
+ * device-wide synchronisation and unbounded latency an allocation may bring.  Such a caller can
+ * still pass A, B and C (it owns them already) but has nowhere to get the split-K workspace from.
+ * This entry point therefore takes no workspace: small problems that ccl_gemm would split along K
+ * keep their partial sums in a scratch array of CCL_GEMM_STATIC_WS_BYTES that is compiled into the
+ * library image, so every GPU that loads the library carries those bytes until the process exits.
+ *
+ * Behaviour: identical results to ccl_gemm (same kernels, same plan).  A problem whose plan needs
+ * more than CCL_GEMM_STATIC_WS_BYTES is rejected with CCL_ERR_WORKSPACE before anything is
+ * launched (ccl_gemm_workspace(d) tells in advance); a problem that needs no workspace runs as
+ * usual.  The call performs no cudaMalloc / cudaFree and calls no allocating library routine.
+ * The first call on each device looks up the scratch array's device address (which may make the
+ * runtime load the library's device code), so make that first call outside any stream capture.
+ * All calls on a device share the one array and it keeps whatever the previous call left in it;
+ * the kernels overwrite every partial sum they later read, so nothing needs clearing, but two
+ * calls whose kernels can overlap on the GPU (different streams, no dependency) would race on
+ * it: serialise them.
+ */
+#define CCL_GEMM_STATIC_WS_BYTES (8u * 1024u * 1024u)
+ccl_status ccl_gemm_static_ws(const ccl_gemm_desc* d, const void* A_dev, const void* B_dev, void* C_dev,
+                              void* cuda_stream);
+
 /* ---- remote-traffic counter (Sec. 4.1 metric, every touched byte counted: no L2 filter) */
 
 typedef enum { CCL_PLACE_RR = 0, CCL_PLACE_BLOCK = 1, CCL_PLACE_BEST = 2 } ccl_place;

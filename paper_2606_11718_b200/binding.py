@@ -20,7 +20,7 @@ PLACE_RR, PLACE_BLOCK, PLACE_BEST = 0, 1, 2
 ASSIGN_N_STRIPS, ASSIGN_M_STRIPS, ASSIGN_EXPLICIT = 0, 1, 2
 
 EXPORTS = ["ccl_map_offset", "ccl_map_inverse", "ccl_buffer_bytes", "ccl_strip_stride", "ccl_repack", "ccl_gemm_workspace",
-           "ccl_gemm", "ccl_gemm_status", "ccl_traffic_sizes", "ccl_traffic", "ccl_last_error", "ccl_launch_count", "ccl_version"]
+           "ccl_gemm", "ccl_gemm_static_ws", "ccl_gemm_status", "ccl_traffic_sizes", "ccl_traffic", "ccl_last_error", "ccl_launch_count", "ccl_version"]
 
 
 class CclError(RuntimeError):
@@ -73,6 +73,7 @@ def lib():
         l.ccl_repack.argtypes = [C.POINTER(Mat), C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]
         l.ccl_gemm_workspace.argtypes = [C.POINTER(GemmDesc), C.POINTER(C.c_size_t)]
         l.ccl_gemm.argtypes = [C.POINTER(GemmDesc), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+        l.ccl_gemm_static_ws.argtypes = [C.POINTER(GemmDesc), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         l.ccl_gemm_status.argtypes = [C.c_void_p, C.POINTER(C.c_int32)]
         l.ccl_traffic_sizes.argtypes = [C.POINTER(TrafficDesc), C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
         l.ccl_traffic.argtypes = [C.POINTER(TrafficDesc), C.c_void_p, C.c_void_p, C.POINTER(C.c_void_p), C.POINTER(C.c_void_p),
@@ -147,6 +148,19 @@ def ccl_gemm(d, A, B, Cout, ws=None):
             raise ValueError("ccl_gemm: operand buffer too small")
     ws_bytes = ws.numel() * ws.element_size() if ws is not None else 0
     _check(lib().ccl_gemm(C.byref(d), _ptr(A), _ptr(B), _ptr(Cout), _ptr(ws), ws_bytes, _stream()))
+
+
+GEMM_STATIC_WS_BYTES = 8 * 1024 * 1024
+
+
+def ccl_gemm_static_ws(d, A, B, Cout):
+    """ccl_gemm without a workspace argument: split-K partial sums go to the scratch array built into the library
+    (for callers that cannot allocate device memory).  Raises CclError(ERR_WORKSPACE) if the problem needs more
+    than GEMM_STATIC_WS_BYTES."""
+    for t, m in ((A, d.A), (B, d.B), (Cout, d.C)):
+        if t.numel() * t.element_size() < ccl_buffer_bytes(m):
+            raise ValueError("ccl_gemm_static_ws: operand buffer too small")
+    _check(lib().ccl_gemm_static_ws(C.byref(d), _ptr(A), _ptr(B), _ptr(Cout), _stream()))
 
 
 def ccl_gemm_status():

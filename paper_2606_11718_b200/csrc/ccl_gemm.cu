@@ -24,6 +24,7 @@
 #include <algorithm>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 
 #include <cuda_bf16.h>
 
@@ -730,4 +731,50 @@ extern "C" ccl_status ccl_gemm_status(void* cuda_stream, int32_t* detail) {
     if (detail) *detail = v ? v : (rv ? 100 + rv : 0);
     if (v || rv) return fail(CCL_ERR_TIMEOUT, "a bounded device-side wait expired (code %d)", v ? v : 100 + rv);
     return CCL_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// ccl_gemm_static_ws: the split-K GEMM for callers that cannot allocate
+// ------------------------------------------------------------------------------------------
+// Scratch for the split-K partial sums, part of the library image: every GPU that loads the library
+// holds these bytes until the process ends.  Only device code may use the name as an address; on the
+// host the name is merely a handle that cudaGetSymbolAddress turns into the device pointer.
+static __device__ __align__(256) unsigned char g_static_ws[CCL_GEMM_STATIC_WS_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_ws_mutex;
+void* g_static_ws_addr[kMaxDevices] = {};
+
+// Device address of g_static_ws on the current device, looked up once per device.
+ccl_status static_ws_address(void** out) {
+    int dev = -1;
+    CCL_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return ccl::fail(CCL_ERR_UNSUPPORTED, "ccl_gemm_static_ws: device ordinal %d is beyond the %d this library tracks", dev, kMaxDevices);
+    std::lock_guard<std::mutex> lock(g_static_ws_mutex);
+    if (!g_static_ws_addr[dev]) {
+        void* ptr = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_ws);
+        if (e != cudaSuccess || !ptr)
+            return ccl::fail(CCL_ERR_CUDA, "ccl_gemm_static_ws: cudaGetSymbolAddress failed: %s", cudaGetErrorString(e));
+        g_static_ws_addr[dev] = ptr;
+    }
+    *out = g_static_ws_addr[dev];
+    return CCL_OK;
+}
+}  // namespace
+
+extern "C" ccl_status ccl_gemm_static_ws(const ccl_gemm_desc* d, const void* A_dev, const void* B_dev, void* C_dev,
+                                         void* cuda_stream) {
+    size_t need = 0;
+    ccl_status s = ccl_gemm_workspace(d, &need);
+    if (s) return s;
+    if (need > (size_t)CCL_GEMM_STATIC_WS_BYTES)
+        return ccl::fail(CCL_ERR_WORKSPACE, "ccl_gemm_static_ws: this problem needs %zu bytes of split-K workspace, the built-in scratch holds %u; "
+                         "use ccl_gemm with a caller-provided workspace", need, (unsigned)CCL_GEMM_STATIC_WS_BYTES);
+    void* ws = nullptr;
+    if (need) {
+        if ((s = static_ws_address(&ws))) return s;
+    }
+    return ccl_gemm(d, A_dev, B_dev, C_dev, ws, need ? (size_t)CCL_GEMM_STATIC_WS_BYTES : 0, cuda_stream);
 }
