@@ -115,10 +115,17 @@ def ccl_map_inverse(m, elem_off):
     return r.value, c.value
 
 
+_bytes_cache = {}
+
+
 def ccl_buffer_bytes(m):
-    b = C.c_int64()
-    _check(lib().ccl_buffer_bytes(C.byref(m), C.byref(b)))
-    return b.value
+    key = (m.rows, m.cols, m.elem_bytes, m.P, m.part, m.layout, m.strip_align_bytes)
+    v = _bytes_cache.get(key)
+    if v is None:
+        b = C.c_int64()
+        _check(lib().ccl_buffer_bytes(C.byref(m), C.byref(b)))
+        v = _bytes_cache[key] = b.value
+    return v
 
 
 def ccl_strip_stride(m):

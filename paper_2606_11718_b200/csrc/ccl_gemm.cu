@@ -37,7 +37,8 @@ constexpr int BM = 128;                         // rows of the output tile one C
 constexpr int BK = 64;
 constexpr int kGemmThreads = 192;
 constexpr int kTmemCols = 512;
-constexpr uint32_t kSmemBudget = 200 * 1024;    // ring of operand stages
+constexpr uint32_t kSmemBudget = 192 * 1024;    // ring of operand stages
+constexpr uint32_t kEpiBytes = 4 * 2 * 32 * 128; // epilogue staging: per warp two buffers of 32 rows x 128 B
 
 __device__ int g_gemm_status = 0;
 
@@ -212,7 +213,8 @@ struct Scheduler {
 
 template <int BN, int CTAS>
 __global__ void __launch_bounds__(kGemmThreads, 1)
-ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const GemmParams p) {
+ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                const __grid_constant__ CUtensorMap map_c, const GemmParams p) {
     // A tile wider than 256 columns is computed as NSUB sub-tiles of SUBN columns (one MMA each per
     // k step) that fill TMEM; narrower tiles use the two 256-column halves of TMEM as a double buffer.
     constexpr int NSUB = BN > 256 ? BN / 256 : 1;
@@ -220,7 +222,8 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     constexpr int SUBH = SUBN / CTAS;                // B columns of one sub-tile this CTA stages
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)p.stages * p.stage_bytes);
+    unsigned char* epi = smem + (size_t)p.stages * p.stage_bytes;     // 1024-byte aligned: stage sizes are multiples of 1 KB
+    uint64_t* bars = reinterpret_cast<uint64_t*>(epi + kEpiBytes);
     uint64_t* full = bars;                           // used in the leader CTA only
     uint64_t* empty = bars + p.stages;               // one set per CTA
     uint64_t* tmem_full = bars + 2 * p.stages;       // one set per CTA
@@ -234,6 +237,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     if (threadIdx.x == 0) {
         prefetch_tmap(&map_a);
         prefetch_tmap(&map_b);
+        prefetch_tmap(&map_c);
         for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(&tmem_full[a], 1); mbar_init(&tmem_empty[a], 4 * CTAS); }
         fence_barrier_init();
@@ -342,6 +346,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         const uint32_t tmem_empty0 = CTAS == 2 ? map_to_cta(smem_u32(&tmem_empty[0]), 0) : smem_u32(&tmem_empty[0]);
         TileCoord t;
         bool alive = true;
+        uint32_t epi_count = 0;                          // TMA-stored pieces so far (selects the staging buffer)
         for (int it = 0; alive && sched.get(it, t); ++it) {
           const int m = t.m0 + (int)rank * BM + quad * 32 + lane;
           for (int h = 0; h < NSUB; ++h) {
@@ -358,34 +363,69 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             else if (p.c_split == 1) { int64_t g = t.m0 / p.c_h; row_base = g * p.c_stride + ((int64_t)m - g * p.c_h) * p.c_cols; }
             else row_base = (int64_t)m * p.c_cols;
             const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)acc * 256u;
+            // Full 32-row x 64-column pieces go through shared memory (128-byte swizzle) and a TMA tile store
+            // addressed through C's own rank-3 map; ragged pieces (tile clipped by a strip or the matrix edge)
+            // and split-K partial sums are stored from registers.
+            const int row0 = t.m0 + (int)rank * BM + quad * 32;
+            const bool rows_full = row0 + 32 <= t.m1;
+            int cy, cz, cx0;                                 // C map coordinates of (row0, nb)
+            if (p.c_split == 2) { cz = nb / (int)p.c_w; cx0 = nb - cz * (int)p.c_w; cy = row0; }
+            else if (p.c_split == 1) { cz = row0 / (int)p.c_h; cy = row0 - cz * (int)p.c_h; cx0 = nb; }
+            else { cz = 0; cy = row0; cx0 = nb; }
 #pragma unroll 1
-            for (int c = 0; c < SUBN / 32; ++c) {
-                if (nb + c * 32 >= t.n1) break;          // warp-uniform: nothing valid further right
-                uint32_t r[32];
-                tmem_ld32(taddr + (uint32_t)(c * 32), r);
+            for (int c = 0; c < SUBN / 64; ++c) {
+                const int n64 = nb + c * 64;
+                if (n64 >= t.n1) break;                  // warp-uniform: nothing valid further right
+                uint32_t r[64];
+                tmem_ld32(taddr + (uint32_t)(c * 64), *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
+                tmem_ld32(taddr + (uint32_t)(c * 64 + 32), *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
                 tmem_ld_wait();
-                if (p.splits > 1) {                      // partial sums, summed in fixed order by splitk_reduce_kernel
-                    if (m < t.m1) {
-                        float* wrow = p.ws + ((int64_t)t.split * p.M + m) * (int64_t)p.N;
+                if (p.splits == 1 && rows_full && n64 + 64 <= t.n1) {
+                    unsigned char* buf = epi + (size_t)((warp - 2) * 2 + (epi_count & 1)) * (32 * 128);
+                    if (epi_count >= 2) { if (lane == 0) tma_store_wait_read<1>(); __syncwarp(); }   // buffer free again
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            const int n = nb + c * 32 + j * 4;
-                            if (n < t.n1)
-                                *reinterpret_cast<uint4*>(wrow + n) = make_uint4(r[j * 4 + 0], r[j * 4 + 1], r[j * 4 + 2], r[j * 4 + 3]);
-                        }
+                    for (int u = 0; u < 8; ++u) {
+                        uint4 v;
+                        __nv_bfloat162 hh;
+                        hh = __floats2bfloat162_rn(__uint_as_float(r[u * 8 + 0]), __uint_as_float(r[u * 8 + 1])); v.x = *reinterpret_cast<uint32_t*>(&hh);
+                        hh = __floats2bfloat162_rn(__uint_as_float(r[u * 8 + 2]), __uint_as_float(r[u * 8 + 3])); v.y = *reinterpret_cast<uint32_t*>(&hh);
+                        hh = __floats2bfloat162_rn(__uint_as_float(r[u * 8 + 4]), __uint_as_float(r[u * 8 + 5])); v.z = *reinterpret_cast<uint32_t*>(&hh);
+                        hh = __floats2bfloat162_rn(__uint_as_float(r[u * 8 + 6]), __uint_as_float(r[u * 8 + 7])); v.w = *reinterpret_cast<uint32_t*>(&hh);
+                        *reinterpret_cast<uint4*>(buf + lane * 128 + ((u ^ (lane & 7)) << 4)) = v;
                     }
-                } else if (m < t.m1) {
+                    fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) { tma_store_3d(&map_c, buf, cx0 + c * 64, cy, cz); tma_store_commit(); }
+                    ++epi_count;
+                    continue;
+                }
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const int n = nb + c * 32 + j * 8;
-                        if (n < t.n1) {                  // n1 - n0 is a multiple of 8
-                            uint4 v;
-                            __nv_bfloat162 h;
-                            h = __floats2bfloat162_rn(__uint_as_float(r[j * 8 + 0]), __uint_as_float(r[j * 8 + 1])); v.x = *reinterpret_cast<uint32_t*>(&h);
-                            h = __floats2bfloat162_rn(__uint_as_float(r[j * 8 + 2]), __uint_as_float(r[j * 8 + 3])); v.y = *reinterpret_cast<uint32_t*>(&h);
-                            h = __floats2bfloat162_rn(__uint_as_float(r[j * 8 + 4]), __uint_as_float(r[j * 8 + 5])); v.z = *reinterpret_cast<uint32_t*>(&h);
-                            h = __floats2bfloat162_rn(__uint_as_float(r[j * 8 + 6]), __uint_as_float(r[j * 8 + 7])); v.w = *reinterpret_cast<uint32_t*>(&h);
-                            *reinterpret_cast<uint4*>(p.C + row_base + n) = v;
+                for (int half = 0; half < 2; ++half) {
+                    const uint32_t* rr = &r[half * 32];
+                    const int n32 = n64 + half * 32;
+                    if (p.splits > 1) {                  // partial sums, summed in fixed order by splitk_reduce_kernel
+                        if (m < t.m1) {
+                            float* wrow = p.ws + ((int64_t)t.split * p.M + m) * (int64_t)p.N;
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                const int n = n32 + j * 4;
+                                if (n < t.n1)
+                                    *reinterpret_cast<uint4*>(wrow + n) = make_uint4(rr[j * 4 + 0], rr[j * 4 + 1], rr[j * 4 + 2], rr[j * 4 + 3]);
+                            }
+                        }
+                    } else if (m < t.m1) {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const int n = n32 + j * 8;
+                            if (n < t.n1) {              // n1 - n0 is a multiple of 8
+                                uint4 v;
+                                __nv_bfloat162 hh;
+                                hh = __floats2bfloat162_rn(__uint_as_float(rr[j * 8 + 0]), __uint_as_float(rr[j * 8 + 1])); v.x = *reinterpret_cast<uint32_t*>(&hh);
+                                hh = __floats2bfloat162_rn(__uint_as_float(rr[j * 8 + 2]), __uint_as_float(rr[j * 8 + 3])); v.y = *reinterpret_cast<uint32_t*>(&hh);
+                                hh = __floats2bfloat162_rn(__uint_as_float(rr[j * 8 + 4]), __uint_as_float(rr[j * 8 + 5])); v.z = *reinterpret_cast<uint32_t*>(&hh);
+                                hh = __floats2bfloat162_rn(__uint_as_float(rr[j * 8 + 6]), __uint_as_float(rr[j * 8 + 7])); v.w = *reinterpret_cast<uint32_t*>(&hh);
+                                *reinterpret_cast<uint4*>(p.C + row_base + n) = v;
+                            }
                         }
                     }
                 }
@@ -398,6 +438,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             }
           }
         }
+        if (lane == 0) tma_store_wait_all<0>();          // every tile store has left shared memory and landed
     }
 
     tc_fence_before();
@@ -588,7 +629,7 @@ static ccl_status make_plan(const ccl_gemm_desc* d, const void* A, const void* B
     if (groups > 1 && units >= groups && (group_dim == 0 ? p.tiles_n % groups == 0 : p.tiles_m % groups == 0)) {
         p.groups = groups; p.group_dim = group_dim;
     } else { p.groups = 1; p.group_dim = 0; }
-    plan->smem_bytes = (uint32_t)p.stages * p.stage_bytes + 1024 + (2 * p.stages + 4) * 8 + 16;
+    plan->smem_bytes = (uint32_t)p.stages * p.stage_bytes + kEpiBytes + 1024 + (2 * p.stages + 4) * 8 + 16;
     return CCL_OK;
 }
 
@@ -613,7 +654,7 @@ static ccl_status configure(uint32_t smem_bytes) {
 }
 
 template <int BN, int CTAS>
-static ccl_status launch(const GemmPlan& plan, const CUtensorMap& ma, const CUtensorMap& mb, cudaStream_t st) {
+static ccl_status launch(const GemmPlan& plan, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, cudaStream_t st) {
     ccl_status s = configure<BN, CTAS>(plan.smem_bytes);
     if (s) return s;
     cudaLaunchConfig_t cfg;
@@ -627,7 +668,7 @@ static ccl_status launch(const GemmPlan& plan, const CUtensorMap& ma, const CUte
     attr[0].val.clusterDim.x = CTAS; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    CCL_CUDA_TRY(cudaLaunchKernelEx(&cfg, ccl_gemm_kernel<BN, CTAS>, ma, mb, plan.p));
+    CCL_CUDA_TRY(cudaLaunchKernelEx(&cfg, ccl_gemm_kernel<BN, CTAS>, ma, mb, mc, plan.p));
     count_launch();
     return CCL_OK;
 }
@@ -656,6 +697,44 @@ ccl_status repack_status_take(int* code);   // ccl_repack.cu
 
 using namespace ccl;
 
+// ---- host-side cache of prepared calls (plan + encoded tensor maps) --------------------------------------
+struct PreparedKey {
+    int64_t f[32];          // every field of the descriptor, the three pointers, the device and the tuning overrides
+    int dev;
+    char env[60];
+};
+struct Prepared {
+    PreparedKey key;
+    GemmPlan plan;
+    CUtensorMap ma, mb, mc;
+    int sms;
+    bool valid = false;
+};
+constexpr int kPreparedSlots = 16;
+static Prepared g_prepared[kPreparedSlots];
+static int g_prepared_next = 0;
+static std::mutex g_prepared_mutex;
+
+static void put_mat(const ccl_mat& m, int64_t* f) {
+    f[0] = m.rows; f[1] = m.cols; f[2] = m.elem_bytes; f[3] = m.P; f[4] = m.part; f[5] = m.layout; f[6] = m.strip_align_bytes;
+}
+static void make_key(const ccl_gemm_desc* d, const void* A, const void* B, const void* C, PreparedKey* k) {
+    std::memset(k, 0, sizeof(*k));
+    k->f[0] = d->M; k->f[1] = d->N; k->f[2] = d->K;
+    put_mat(d->A, k->f + 3); put_mat(d->B, k->f + 10); put_mat(d->C, k->f + 17);
+    k->f[24] = d->a_trans; k->f[25] = d->b_trans; k->f[26] = d->out_part; k->f[27] = d->P; k->f[28] = d->grouped_raster;
+    k->f[29] = (int64_t)reinterpret_cast<uintptr_t>(A); k->f[30] = (int64_t)reinterpret_cast<uintptr_t>(B);
+    k->f[31] = (int64_t)reinterpret_cast<uintptr_t>(C);
+    k->dev = -1;
+    (void)cudaGetDevice(&k->dev);
+    size_t pos = 0;
+    for (const char* name : {"CCL_GEMM_CTAS", "CCL_GEMM_BN", "CCL_GEMM_SPLITK", "CCL_GEMM_SMEM_KB", "CCL_GEMM_PANEL"}) {
+        const char* v = std::getenv(name);
+        for (const char* c = v ? v : ""; *c && pos + 2 < sizeof(k->env); ++c) k->env[pos++] = *c;
+        if (pos + 1 < sizeof(k->env)) k->env[pos++] = ';';
+    }
+}
+
 // SM count and resident CTA pairs of the current device; the figures of a B200 when no device is usable
 // (the planner then still validates and sizes the workspace the same way a B200 would).
 static void device_units(int* sms, int* pairs) {
@@ -683,33 +762,56 @@ extern "C" ccl_status ccl_gemm_workspace(const ccl_gemm_desc* d, size_t* bytes) 
 extern "C" ccl_status ccl_gemm(const ccl_gemm_desc* d, const void* A_dev, const void* B_dev, void* C_dev, void* ws_dev,
                                size_t ws_bytes, void* cuda_stream) {
     if (!A_dev || !B_dev || !C_dev) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: NULL operand");
-    GemmPlan plan;
-    ccl_status s = make_plan(d, A_dev, B_dev, C_dev, 148, 74, &plan);     // validation first: no CUDA call on bad input
-    if (s) return s;
-    int dev, sms;
-    CCL_CUDA_TRY(cudaGetDevice(&dev));
-    CCL_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    if ((s = make_plan(d, A_dev, B_dev, C_dev, sms, resident_pairs(), &plan))) return s;
+    if (!d) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: NULL descriptor");
+    // Repeated calls with the same descriptor and buffers (the normal case in a training / serving loop)
+    // reuse the plan and the two encoded tensor maps: a host-side cache only, nothing is kept on the device.
+    PreparedKey key;
+    make_key(d, A_dev, B_dev, C_dev, &key);
+    Prepared prep;
+    bool hit = false;
+    {
+        std::lock_guard<std::mutex> lock(g_prepared_mutex);
+        for (int i = 0; i < kPreparedSlots; ++i)
+            if (g_prepared[i].valid && std::memcmp(&g_prepared[i].key, &key, sizeof(key)) == 0) { prep = g_prepared[i]; hit = true; break; }
+    }
+    ccl_status s;
+    if (!hit) {
+        GemmPlan& plan = prep.plan;
+        s = make_plan(d, A_dev, B_dev, C_dev, 148, 74, &plan);     // validation first: no CUDA call on bad input
+        if (s) return s;
+        int dev;
+        CCL_CUDA_TRY(cudaGetDevice(&dev));
+        CCL_CUDA_TRY(cudaDeviceGetAttribute(&prep.sms, cudaDevAttrMultiProcessorCount, dev));
+        if (dev != key.dev) make_key(d, A_dev, B_dev, C_dev, &key);
+        if ((s = make_plan(d, A_dev, B_dev, C_dev, prep.sms, resident_pairs(), &plan))) return s;
+        plan.p.C = static_cast<uint16_t*>(C_dev);
+        const uint32_t bnh = (uint32_t)((plan.bn > 256 ? 256 : plan.bn) / plan.ctas);   // B rows of one K-major box
+        if (!plan.p.a_mn) s = operand_tmap(&prep.ma, plan.va, A_dev, BK, BM); else s = operand_tmap(&prep.ma, plan.va, A_dev, 64, BK);
+        if (s) return s;
+        if (!plan.p.b_mn) s = operand_tmap(&prep.mb, plan.vb, B_dev, BK, bnh); else s = operand_tmap(&prep.mb, plan.vb, B_dev, 64, BK);
+        if (s) return s;
+        if ((s = operand_tmap(&prep.mc, plan.vc, C_dev, 64, 32))) return s;            // C: 64-column x 32-row store boxes
+        prep.key = key; prep.valid = true;
+        std::lock_guard<std::mutex> lock(g_prepared_mutex);
+        g_prepared[g_prepared_next] = prep;
+        g_prepared_next = (g_prepared_next + 1) % kPreparedSlots;
+    }
+    GemmPlan& plan = prep.plan;
+    const CUtensorMap &ma = prep.ma, &mb = prep.mb, &mc = prep.mc;
+    const int sms = prep.sms;
     if (plan.ws_bytes) {
         if (!ws_dev || ws_bytes < plan.ws_bytes)
             return fail(CCL_ERR_WORKSPACE, "ccl_gemm: this problem is split along K and needs %zu bytes of workspace (got %zu)", plan.ws_bytes, ws_dev ? ws_bytes : (size_t)0);
         if (reinterpret_cast<uintptr_t>(ws_dev) & 15) return fail(CCL_ERR_ALIGN, "ccl_gemm: workspace is not 16-byte aligned");
     }
-    plan.p.C = static_cast<uint16_t*>(C_dev);
     plan.p.ws = static_cast<float*>(ws_dev);
-    const uint32_t bnh = (uint32_t)((plan.bn > 256 ? 256 : plan.bn) / plan.ctas);   // B rows of one K-major box
-    CUtensorMap ma, mb;
-    if (!plan.p.a_mn) s = operand_tmap(&ma, plan.va, A_dev, BK, BM); else s = operand_tmap(&ma, plan.va, A_dev, 64, BK);
-    if (s) return s;
-    if (!plan.p.b_mn) s = operand_tmap(&mb, plan.vb, B_dev, BK, bnh); else s = operand_tmap(&mb, plan.vb, B_dev, 64, BK);
-    if (s) return s;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
     if (plan.ctas == 2) {
-        if (plan.bn == 512) s = launch<512, 2>(plan, ma, mb, st);
-        else s = plan.bn == 256 ? launch<256, 2>(plan, ma, mb, st) : launch<128, 2>(plan, ma, mb, st);
-    } else if (plan.bn == 256) s = launch<256, 1>(plan, ma, mb, st);
-    else if (plan.bn == 192) s = launch<192, 1>(plan, ma, mb, st);
-    else s = launch<128, 1>(plan, ma, mb, st);
+        if (plan.bn == 512) s = launch<512, 2>(plan, ma, mb, mc, st);
+        else s = plan.bn == 256 ? launch<256, 2>(plan, ma, mb, mc, st) : launch<128, 2>(plan, ma, mb, mc, st);
+    } else if (plan.bn == 256) s = launch<256, 1>(plan, ma, mb, mc, st);
+    else if (plan.bn == 192) s = launch<192, 1>(plan, ma, mb, mc, st);
+    else s = launch<128, 1>(plan, ma, mb, mc, st);
     if (s) return s;
     if (plan.p.splits > 1) {
         int64_t work = (int64_t)plan.p.M * (plan.p.N / 8);

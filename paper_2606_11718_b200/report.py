@@ -1,0 +1,219 @@
+"""Per-GEMM report over the five workload configurations (single GPU).
+
+    python -m paper_2606_11718_b200.report [--config 1..5 | all] [--out DIR] [--quick]
+
+For every GEMM of a configuration it measures, with CUDA events on the launching stream:
+  * ccl_repack of the B operand (row-major -> CCL), GB/s of read+write bytes;
+  * ccl_gemm with B and C in CCL under the chiplet-grouped raster, and with row-major operands
+    under the plain raster (Sec. 3.3: the layout should not change the speed);
+  * ccl_traffic under the policies of Sec. 4.1 -- row-major + round-robin at 4 KB (the baseline),
+    64 KB and 2 MB, row-major + coarse block placement, row-major + best page-granular placement,
+    CCL + page->strip placement, CCL + literal round-robin -- for the N- and the M-partition of C,
+    and prints remote bytes relative to the 4 KB round-robin baseline (no L2 filter: every byte a CTA
+    touches is counted, so the ratios are not the paper's simulated ones).
+Roofline per GEMM: min(tensor peak, HBM peak * arithmetic intensity), against the measured peaks in
+MEASURED_PEAKS.json when present.  One JSON object per GEMM is written to DIR/report_config<N>.json
+and a table is printed.  Nothing here calls the CPU oracle.
+"""
+import argparse
+import json
+import math
+import os
+
+import torch
+
+from . import binding as ccl
+from . import synth
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        j = json.load(open(p))
+        return dict(hbm=j["hbm_gbs"], tf=j["bf16_tflops"], src="measured")
+    return dict(hbm=6650.0, tf=1590.0, src="fallback")
+
+
+def configs(which, quick):
+    out = {}
+    g1 = synth.config1_gemm()
+    out[1] = [dict(g1, P=4, S=4096), dict(g1, name="qwen_expert_up_wT", b_trans=0, P=4, S=4096)]
+    out[2] = [dict(g, P=P, S=S) for g in synth.qwen_ffn_gemms() for P in (2, 4) for S in (4096, 65536)]
+    out[3] = [dict(g, P=P, S=4096) for g in synth.llama_fwd_gemms() for P in (2, 4)]
+    out[4] = [dict(g, P=P, S=4096) for g in synth.llama_bwd_gemms() for P in (2, 4)]
+    sweep = []
+    for g in synth.llama_fwd_gemms() + synth.qwen_ffn_gemms()[:2]:
+        for M in (1, 16, 128, 1024, 8192):
+            for P in ((4,) if quick else (2, 4, 8)):
+                sweep.append(dict(g, name=f"{g['name']}_M{M}", M=M, P=P, S=4096))
+    out[5] = sweep
+    return {k: v for k, v in out.items() if which in ("all", str(k))}
+
+
+def mats(g, layout_bc, align=0):
+    M, N, K, at, bt, P = g["M"], g["N"], g["K"], g["a_trans"], g["b_trans"], g["P"]
+    a_shape = (K, M) if at else (M, K)
+    b_shape = (N, K) if bt else (K, N)
+    b_part = ccl.PART_ROWS if bt else ccl.PART_COLS
+    mA = ccl.Mat(a_shape[0], a_shape[1], 2)
+    mB = ccl.Mat(b_shape[0], b_shape[1], 2, P, b_part, layout_bc, align if layout_bc == ccl.CCL else 0)
+    mC = ccl.Mat(M, N, 2, P, ccl.PART_COLS, layout_bc, align if layout_bc == ccl.CCL else 0)
+    return mA, mB, mC
+
+
+def timed(fn, reps, warm=2):
+    for _ in range(warm):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / reps
+
+
+def traffic_remote(g, layout_bc, place_bc, S, assign, align=0):
+    """Remote bytes (A, B, C) of one policy; None if the partition does not apply (M % P != 0)."""
+    M, N, K, P = g["M"], g["N"], g["K"], g["P"]
+    if assign == ccl.ASSIGN_M_STRIPS and (M % P or M < P):
+        return None
+    at, bt = g["a_trans"], g["b_trans"]
+    td = ccl.TrafficDesc()
+    td.M, td.N, td.K, td.BM, td.BN = M, N, K, 128, 128
+    a_shape = (K, M) if at else (M, K)
+    b_shape = (N, K) if bt else (K, N)
+    if assign == ccl.ASSIGN_N_STRIPS:                       # C split along N: B and C follow, A is shared
+        parts = (ccl.PART_NONE, ccl.PART_ROWS if bt else ccl.PART_COLS, ccl.PART_COLS)
+    else:                                                   # C split along M: A and C follow, B is shared
+        parts = (ccl.PART_COLS if at else ccl.PART_ROWS, ccl.PART_NONE, ccl.PART_ROWS)
+    shapes = (a_shape, b_shape, (M, N))
+    ms = []
+    for X in range(3):
+        is_ccl = layout_bc == ccl.CCL and parts[X] != ccl.PART_NONE
+        ms.append(ccl.Mat(shapes[X][0], shapes[X][1], 2, P, parts[X] if is_ccl else ccl.PART_NONE,
+                          ccl.CCL if is_ccl else ccl.ROWMAJOR, align if is_ccl else 0))
+    td.A, td.B, td.C = ms
+    td.a_trans, td.b_trans, td.P, td.page_bytes = at, bt, P, S
+    for X in range(3):
+        split = parts[X] != ccl.PART_NONE
+        td.place[X] = place_bc if split else (ccl.PLACE_RR if place_bc != ccl.PLACE_BEST else ccl.PLACE_BEST)
+    td.assign, td.strip_tiling = assign, 1
+    nt, pages = ccl.ccl_traffic_sizes(td)
+    per_cta = torch.empty((nt, 3, 2), dtype=torch.int64, device="cuda")
+    totals = torch.empty((3, 2), dtype=torch.int64, device="cuda")
+    pp = ow = None
+    if place_bc == ccl.PLACE_BEST:
+        pp = [torch.empty((pages[x], P), dtype=torch.int64, device="cuda") for x in range(3)]
+        ow = [torch.empty((pages[x],), dtype=torch.uint8, device="cuda") for x in range(3)]
+    ms_t = timed(lambda: ccl.ccl_traffic(td, per_cta, totals, pp, ow), 3, 1)
+    t = totals.cpu()
+    return dict(remote=[int(x) for x in t[:, 1]], total=int(t.sum()), ms=ms_t)
+
+
+def run_gemm(g, pk, reps):
+    M, N, K, at, bt, P, S = g["M"], g["N"], g["K"], g["a_trans"], g["b_trans"], g["P"], g["S"]
+    dev = "cuda"
+    A = torch.empty((K, M) if at else (M, K), dtype=torch.bfloat16, device=dev).normal_(0, g["a_std"])
+    B = torch.empty((N, K) if bt else (K, N), dtype=torch.bfloat16, device=dev).normal_(0, g["b_std"])
+    res = dict(name=g["name"], M=M, N=N, K=K, P=P, page=S, a_trans=at, b_trans=bt)
+    flop = 2.0 * M * N * K
+    bytes_alg = 2.0 * (M * K + K * N + M * N)
+    roof_tf = min(pk["tf"], pk["hbm"] * flop / bytes_alg / 1e3)
+    res.update(flop=flop, algorithmic_bytes=bytes_alg, roofline_tflops=roof_tf, roofline_bound="tensor" if roof_tf >= pk["tf"] else "hbm")
+    outs = {}
+    for tag, lay, grouped in (("ccl_grouped", ccl.CCL, 1), ("row_plain", ccl.ROWMAJOR, 0)):
+        mA, mB, mC = mats(g, lay, S)
+        d = ccl.GemmDesc()
+        d.M, d.N, d.K, d.A, d.B, d.C = M, N, K, mA, mB, mC
+        d.a_trans, d.b_trans, d.out_part, d.P, d.grouped_raster = at, bt, ccl.PART_COLS, P, grouped
+        try:
+            need = ccl.ccl_gemm_workspace(d)
+        except ccl.CclError as e:
+            res[tag] = dict(error=str(e))
+            continue
+        ws = torch.empty(max(need, 16) // 4, dtype=torch.float32, device=dev)
+        Bl = B
+        if lay == ccl.CCL:
+            Bl = torch.empty(ccl.ccl_buffer_bytes(mB) // 2, dtype=torch.bfloat16, device=dev)
+            rp_ms = timed(lambda: ccl.ccl_repack(mB, B, Bl, 0), reps)
+            rp_bytes = 2.0 * K * N * 2
+            res["repack"] = dict(ms=rp_ms, gbs=rp_bytes / rp_ms / 1e6, frac_of_hbm=rp_bytes / rp_ms / 1e6 / pk["hbm"])
+        Cb = torch.empty(ccl.ccl_buffer_bytes(mC) // 2, dtype=torch.bfloat16, device=dev)
+        ms_g = timed(lambda: ccl.ccl_gemm(d, A, Bl, Cb, ws), reps)
+        st, detail = ccl.ccl_gemm_status()
+        tf = flop / ms_g / 1e9
+        res[tag] = dict(ms=ms_g, tflops=tf, frac_of_roofline=tf / roof_tf, split_k_workspace=need, status=st)
+        if lay == ccl.CCL:
+            Cr = torch.empty(M * N, dtype=torch.bfloat16, device=dev)
+            ccl.ccl_repack(mC, Cb, Cr, 1)
+            outs[tag] = Cr
+        else:
+            outs[tag] = Cb
+    if len(outs) == 2:
+        res["ccl_equals_rowmajor_bits"] = bool(torch.equal(outs["ccl_grouped"], outs["row_plain"]))
+    # library matmul on the same operands: context only
+    Al = A.t() if at else A
+    Bm = B.t() if bt else B
+    ms_t = timed(lambda: torch.matmul(Al, Bm), reps)
+    res["torch_matmul_tflops"] = flop / ms_t / 1e9
+    # remote traffic under the placement policies
+    base = None
+    pol = {}
+    for tag, lay, place, Sp in (("row_rr4k", ccl.ROWMAJOR, ccl.PLACE_RR, 4096), ("row_rr64k", ccl.ROWMAJOR, ccl.PLACE_RR, 65536),
+                                ("row_rr2m", ccl.ROWMAJOR, ccl.PLACE_RR, 2 << 20), ("row_block", ccl.ROWMAJOR, ccl.PLACE_BLOCK, S),
+                                ("row_best", ccl.ROWMAJOR, ccl.PLACE_BEST, S), ("ccl_block", ccl.CCL, ccl.PLACE_BLOCK, S),
+                                ("ccl_rr", ccl.CCL, ccl.PLACE_RR, S)):
+        best = None
+        for assign in (ccl.ASSIGN_N_STRIPS, ccl.ASSIGN_M_STRIPS):
+            r = traffic_remote(g, lay, place, Sp, assign, align=Sp)
+            if r is None:
+                continue
+            r["partition"] = "N" if assign == ccl.ASSIGN_N_STRIPS else "M"
+            if best is None or sum(r["remote"]) < sum(best["remote"]):
+                best = r
+        pol[tag] = best
+        if tag == "row_rr4k":
+            base = sum(best["remote"])
+    for tag, r in pol.items():
+        r["ratio_vs_rr4k"] = (sum(r["remote"]) / base) if base else None
+    res["traffic"] = pol
+    return res
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--config", default="all")
+    ap.add_argument("--out", default=os.path.join(ROOT, "gpurun_out"))
+    ap.add_argument("--quick", action="store_true", help="fewer repetitions and P = 4 only in the sweep")
+    args = ap.parse_args()
+    assert torch.cuda.is_available(), "report needs a CUDA device"
+    pk = peaks()
+    os.makedirs(args.out, exist_ok=True)
+    for cfg, gemms in configs(args.config, args.quick).items():
+        rows = []
+        for g in gemms:
+            big = g["M"] * g["N"] * g["K"] > 1e11
+            r = run_gemm(g, pk, 3 if (big or args.quick) else 20)
+            rows.append(r)
+            c, rw = r.get("ccl_grouped", {}), r.get("row_plain", {})
+            t = r["traffic"]
+            print(f"cfg{cfg} {r['name']:24s} M{r['M']:5d} N{r['N']:5d} K{r['K']:5d} P{r['P']} S{r['page']:7d} | "
+                  f"gemm ccl {c.get('tflops', float('nan')):7.1f} row {rw.get('tflops', float('nan')):7.1f} torch {r['torch_matmul_tflops']:7.1f} TF "
+                  f"(roof {r['roofline_tflops']:6.1f} {r['roofline_bound']}, {100 * c.get('frac_of_roofline', float('nan')):5.1f}%) "
+                  f"bits_equal={r.get('ccl_equals_rowmajor_bits')} | repack {r.get('repack', {}).get('gbs', float('nan')):7.1f} GB/s | "
+                  f"remote/rr4k: rr64k {t['row_rr64k']['ratio_vs_rr4k']:.3f} rr2m {t['row_rr2m']['ratio_vs_rr4k']:.3f} "
+                  f"block {t['row_block']['ratio_vs_rr4k']:.3f} best {t['row_best']['ratio_vs_rr4k']:.3f} "
+                  f"CCL {t['ccl_block']['ratio_vs_rr4k']:.3f} ({t['ccl_block']['partition']}) ccl+rr {t['ccl_rr']['ratio_vs_rr4k']:.3f}", flush=True)
+        json.dump(dict(config=cfg, peaks=pk, gemms=rows), open(os.path.join(args.out, f"report_config{cfg}.json"), "w"), indent=1)
+        nz = [r["traffic"]["ccl_block"]["ratio_vs_rr4k"] for r in rows if r["traffic"]["ccl_block"]["ratio_vs_rr4k"]]
+        if nz:
+            print(f"cfg{cfg}: geometric mean of CCL/rr4k remote-traffic ratios over {len(nz)} GEMMs with non-zero ratio "
+                  f"({len(rows) - len(nz)} zero): {math.exp(sum(math.log(x) for x in nz) / len(nz)):.3f}", flush=True)
+
+
+if __name__ == "__main__":
+    main()
