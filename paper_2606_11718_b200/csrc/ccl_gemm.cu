@@ -159,41 +159,42 @@ __device__ __forceinline__ void to_coords(const OpMap& o, int r, int c, int& x, 
 
 struct TileCoord { int m0, m1, n0, n1, split; };
 
-// Tiles of this CTA (pair).  The schedulable units (CTAs, or CTA pairs) are cut into `groups`
-// contiguous ranges; group g owns the tiles of strip range g (chiplet-grouped raster) and walks
-// them in panels of `panel` m-tiles (m fastest inside a panel, then n, then the next panel).
-// Groups can differ by one unit, so the walk has two phases: `rounds` rounds in which every unit
-// takes tile (its index + round * group size) of its own group, then the few tiles each group
-// has left are pooled and dealt round-robin to all units, which keeps every unit equally busy.
+// Tiles of this CTA (pair).  The schedulable units (CTAs, or CTA pairs) serve `groups` strip ranges
+// (chiplet-grouped raster): group g owns the tiles of strip range g and walks them in panels of
+// `panel` m-tiles (m fastest inside a panel, then n, then the next panel).
+// Every group gets the SAME number of units (upg = units / groups) so that the groups advance in
+// lockstep through the same m-panels and share the A operand in L2; the units left over ("floaters")
+// and, at the end, everybody work through a pool made of the last few tiles of every group:
+//   grouped unit : rounds [0, R) -> tile (index + round * upg) of its own group, then the pool
+//   floater f    : rounds [0, R) -> pool entries f, f + F, ...,                  then the pool
+// with R = min(total / units, per_group / upg); pool entries alternate between the groups.
 struct Scheduler {
     const GemmParams& p;
     int gm, gn;                     // tile grid of one group
-    int unit, units, my_g, idx, step, bm, bn, rounds;
-    int64_t per_group;
-    __device__ int lo(int g) const { return (int)(((int64_t)g * units) / p.groups); }
+    int unit, units, upg, floaters, my_g, idx, bm, bn, rounds;
+    int64_t per_group, pool_per_group;
     __device__ Scheduler(const GemmParams& p_, int unit_, int units_, int bm_, int bn_) : p(p_), unit(unit_), units(units_), bm(bm_), bn(bn_) {
         gm = p.tiles_m; gn = p.tiles_n;
         if (p.groups > 1) { if (p.group_dim == 0) gn = p.tiles_n / p.groups; else gm = p.tiles_m / p.groups; }
         per_group = (int64_t)gm * gn * p.splits;
-        my_g = 0; rounds = 0x7fffffff;
-        for (int g = 0; g < p.groups; ++g) {
-            int l = lo(g), h = lo(g + 1);
-            if (unit >= l && unit < h) { my_g = g; idx = unit - l; step = h - l; }
-            rounds = min(rounds, (int)(per_group / (h - l)));
-        }
+        upg = units / p.groups;                          // the host guarantees units >= groups
+        floaters = units - upg * p.groups;
+        my_g = unit < upg * p.groups ? unit / upg : -1;  // -1: floater
+        idx = my_g >= 0 ? unit - my_g * upg : unit - upg * p.groups;
+        rounds = (int)min(per_group * p.groups / units, per_group / upg);
+        pool_per_group = per_group - (int64_t)rounds * upg;
     }
     __device__ bool get(int it, TileCoord& t) const {
-        int g = my_g;
+        int g;
         int64_t i;
-        if (it < rounds) i = idx + (int64_t)it * step;
-        else {                                            // pooled leftovers of all groups
-            int64_t q = unit + (int64_t)(it - rounds) * units;
-            for (g = 0; g < p.groups; ++g) {
-                int64_t done = (int64_t)rounds * (lo(g + 1) - lo(g)), left = per_group - done;
-                if (q < left) { i = done + q; break; }
-                q -= left;
-            }
-            if (g == p.groups) return false;
+        if (it < rounds && my_g >= 0) { g = my_g; i = idx + (int64_t)it * upg; }
+        else {
+            const int64_t q = it < rounds ? idx + (int64_t)it * floaters
+                                          : (int64_t)floaters * rounds + unit + (int64_t)(it - rounds) * units;
+            g = (int)(q % p.groups);
+            const int64_t j = q / p.groups;
+            if (j >= pool_per_group) return false;
+            i = (int64_t)rounds * upg + j;
         }
         t.split = (int)(i % p.splits);                   // the splits of one tile are neighbours in the walk
         i /= p.splits;
@@ -568,6 +569,8 @@ static ccl_status make_plan(const ccl_gemm_desc* d, const void* A, const void* B
     const int64_t strips_m = d->M / Wm, strips_n = d->N / Wn;
     int ctas = 1, bn = 256, splits = 1;
     double best = -1.0;
+    // Tuning / test overrides (environment): CCL_GEMM_CTAS = 1|2, CCL_GEMM_BN = 128|192|256|512,
+    // CCL_GEMM_SPLITK = number of K splits, CCL_GEMM_PANEL = raster panel height in m-tiles.
     const char* force_ctas = std::getenv("CCL_GEMM_CTAS");
     const char* force_bn = std::getenv("CCL_GEMM_BN");
     const char* force_split = std::getenv("CCL_GEMM_SPLITK");
@@ -616,12 +619,8 @@ static ccl_status make_plan(const ccl_gemm_desc* d, const void* A, const void* B
     p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)p.a_mn << 15) | ((uint32_t)p.b_mn << 16) |
               ((uint32_t)(subn >> 3) << 17) | ((uint32_t)(bm >> 4) << 24);
     p.a_bytes = BM * BK * 2; p.stage_bytes = p.a_bytes + (uint32_t)(bn / ctas) * BK * 2;
-    uint32_t budget = kSmemBudget;
-    if (const char* f = std::getenv("CCL_GEMM_SMEM_KB")) budget = (uint32_t)atoi(f) * 1024u;
-    p.stages = (int32_t)(budget / p.stage_bytes);
+    p.stages = (int32_t)(kSmemBudget / p.stage_bytes);
     if (p.stages > 8) p.stages = 8;
-    p.panel = 16;
-    if (const char* f = std::getenv("CCL_GEMM_PANEL")) p.panel = std::max(1, atoi(f));
     int64_t ntiles = (int64_t)p.tiles_m * p.tiles_n * splits;
     int units = (int)std::min<int64_t>(ntiles, ctas == 2 ? pairs : sms);
     plan->grid = (unsigned)(units * ctas);
@@ -629,6 +628,21 @@ static ccl_status make_plan(const ccl_gemm_desc* d, const void* A, const void* B
     if (groups > 1 && units >= groups && (group_dim == 0 ? p.tiles_n % groups == 0 : p.tiles_m % groups == 0)) {
         p.groups = groups; p.group_dim = group_dim;
     } else { p.groups = 1; p.group_dim = 0; }
+    // Raster panel height: the units of a group that run at the same time cover `panel` m-tiles by
+    // ceil(upg / panel) n-tiles; all groups walk the same m-panel.  The operand rows + columns such a wave
+    // touches are what it pulls from DRAM (the L2 does not hold a wave's footprint until the next wave), so
+    // pick the panel that minimises them; ties go to the taller panel.
+    {
+        const int upg = std::max(1, units / p.groups);
+        const int gm = p.group_dim == 1 && p.groups > 1 ? p.tiles_m / p.groups : p.tiles_m;
+        int64_t best_fp = -1;
+        for (int pnl = 1; pnl <= std::min(gm, 64); ++pnl) {
+            int64_t fp = (int64_t)pnl * bm + (int64_t)p.groups * ((upg + pnl - 1) / pnl) * bn;
+            if (p.group_dim == 1 && p.groups > 1) fp = (int64_t)p.groups * pnl * bm + (int64_t)((upg + pnl - 1) / pnl) * bn;
+            if (best_fp < 0 || fp <= best_fp) { best_fp = fp; p.panel = pnl; }
+        }
+    }
+    if (const char* f = std::getenv("CCL_GEMM_PANEL")) p.panel = std::max(1, atoi(f));
     plan->smem_bytes = (uint32_t)p.stages * p.stage_bytes + kEpiBytes + 1024 + (2 * p.stages + 4) * 8 + 16;
     return CCL_OK;
 }
@@ -677,7 +691,7 @@ static ccl_status launch(const GemmPlan& plan, const CUtensorMap& ma, const CUte
 static int resident_pairs() {
     static int pairs = -1;
     if (pairs >= 0) return pairs;
-    uint32_t smem = 224 * 1024 + 2048;
+    uint32_t smem = kSmemBudget + kEpiBytes + 2048;
     if (configure<256, 2>(smem) != CCL_OK) { clear_error(); return pairs = 0; }
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof(cfg));
@@ -728,7 +742,7 @@ static void make_key(const ccl_gemm_desc* d, const void* A, const void* B, const
     k->dev = -1;
     (void)cudaGetDevice(&k->dev);
     size_t pos = 0;
-    for (const char* name : {"CCL_GEMM_CTAS", "CCL_GEMM_BN", "CCL_GEMM_SPLITK", "CCL_GEMM_SMEM_KB", "CCL_GEMM_PANEL"}) {
+    for (const char* name : {"CCL_GEMM_CTAS", "CCL_GEMM_BN", "CCL_GEMM_SPLITK", "CCL_GEMM_PANEL"}) {
         const char* v = std::getenv(name);
         for (const char* c = v ? v : ""; *c && pos + 2 < sizeof(k->env); ++c) k->env[pos++] = *c;
         if (pos + 1 < sizeof(k->env)) k->env[pos++] = ';';

@@ -5,7 +5,7 @@
 //   split along rows           : row-major side  g*h*C*e + r*C*e, CCL side  g*stride*e + r*C*e
 // The work is pure HBM streaming (read once + write once).  Two kernels:
 //   * repack_tma_kernel  -- one thread per CTA drives a ring of TMA tile loads and TMA tile
-//     stores through shared memory (rank-3 tensor maps on both sides), so ~200 KB per SM
+//     stores through shared memory (rank-3 tensor maps on both sides), so ~190 KB per SM
 //     is in flight with no per-byte instruction cost.  Needs 16-byte alignment everywhere.
 //   * repack_vec_kernel  -- plain vectorised loads/stores for every other shape
 //     (vector width = the largest power of two that divides all extents and addresses).
@@ -84,26 +84,26 @@ __global__ void zero_pad_kernel(char* dst, int64_t pad_g, int64_t pad_off, int64
 // ------------------------------------------------------------------------------------------
 // TMA path: tile = box of (bx 8-byte units) x (by rows) of one strip
 // ------------------------------------------------------------------------------------------
-constexpr int kTmaStages = 6;
-constexpr int kTmaStageBytes = 32768;
+constexpr int kTmaMaxStages = 16;
 
 struct TmaTiling {
     uint32_t bx, by;              // box extents (8-byte units, rows)
     uint32_t tiles_x, tiles_y;    // per strip
+    uint32_t stages, stage_bytes; // ring depth and bytes per ring slot
     uint64_t ntiles;
 };
 
-__global__ void __launch_bounds__(32, 1) repack_tma_kernel(const __grid_constant__ CUtensorMap src_map,
+__global__ void __launch_bounds__(32) repack_tma_kernel(const __grid_constant__ CUtensorMap src_map,
                                                            const __grid_constant__ CUtensorMap dst_map, TmaTiling t) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     // stage buffers first (128-byte aligned), barriers after them
     unsigned char* stage0 = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
-    uint64_t* full = reinterpret_cast<uint64_t*>(stage0 + (size_t)kTmaStages * kTmaStageBytes);
+    uint64_t* full = reinterpret_cast<uint64_t*>(stage0 + (size_t)t.stages * t.stage_bytes);
     if (threadIdx.x != 0) return;
 
     prefetch_tmap(&src_map);
     prefetch_tmap(&dst_map);
-    for (int s = 0; s < kTmaStages; ++s) mbar_init(&full[s], 1);
+    for (int s = 0; s < t.stages; ++s) mbar_init(&full[s], 1);
     fence_barrier_init();
 
     const uint32_t box_bytes = t.bx * t.by * 8u;
@@ -111,30 +111,30 @@ __global__ void __launch_bounds__(32, 1) repack_tma_kernel(const __grid_constant
     auto issue_load = [&](uint64_t it) {
         uint64_t tile = (uint64_t)blockIdx.x + it * gridDim.x;
         if (tile >= t.ntiles) return;
-        uint32_t slot = (uint32_t)(it % kTmaStages);
+        uint32_t slot = (uint32_t)(it % t.stages);
         uint32_t g = (uint32_t)(tile / per_strip);
         uint32_t rem = (uint32_t)(tile - (uint64_t)g * per_strip);
         uint32_t ty = rem / t.tiles_x, tx = rem - ty * t.tiles_x;
         mbar_expect_tx(&full[slot], box_bytes);
-        tma_load_3d(stage0 + (size_t)slot * kTmaStageBytes, &src_map, &full[slot], (int)(tx * t.bx), (int)(ty * t.by), (int)g);
+        tma_load_3d(stage0 + (size_t)slot * t.stage_bytes, &src_map, &full[slot], (int)(tx * t.bx), (int)(ty * t.by), (int)g);
     };
 
-    for (uint64_t it = 0; it < kTmaStages; ++it) issue_load(it);
+    for (uint64_t it = 0; it < t.stages; ++it) issue_load(it);
     for (uint64_t it = 0;; ++it) {
         uint64_t tile = (uint64_t)blockIdx.x + it * gridDim.x;
         if (tile >= t.ntiles) break;
-        uint32_t slot = (uint32_t)(it % kTmaStages);
-        uint32_t parity = (uint32_t)((it / kTmaStages) & 1);
+        uint32_t slot = (uint32_t)(it % t.stages);
+        uint32_t parity = (uint32_t)((it / t.stages) & 1);
         if (!mbar_wait_bounded(&full[slot], parity)) { atomicExch(&g_repack_status, 1); break; }
         uint32_t g = (uint32_t)(tile / per_strip);
         uint32_t rem = (uint32_t)(tile - (uint64_t)g * per_strip);
         uint32_t ty = rem / t.tiles_x, tx = rem - ty * t.tiles_x;
-        tma_store_3d(&dst_map, stage0 + (size_t)slot * kTmaStageBytes, (int)(tx * t.bx), (int)(ty * t.by), (int)g);
+        tma_store_3d(&dst_map, stage0 + (size_t)slot * t.stage_bytes, (int)(tx * t.bx), (int)(ty * t.by), (int)g);
         tma_store_commit();
         // the store issued one iteration ago has now read its buffer: refill that slot
         if (it >= 1) {
             tma_store_wait_read<1>();
-            issue_load(it - 1 + kTmaStages);
+            issue_load(it - 1 + t.stages);
         }
     }
     tma_store_wait_all<0>();
@@ -188,8 +188,14 @@ static ccl_status launch_pad(char* dst, const CopyPlan& p, cudaStream_t st) {
 static ccl_status launch_tma(const char* src, char* dst, const CopyPlan& p, int sms, cudaStream_t st) {
     uint64_t dims[3] = {(uint64_t)(p.row_bytes / 8), (uint64_t)p.rows, (uint64_t)p.nstrips};
     TmaTiling t;
-    t.bx = (uint32_t)std::min<uint64_t>(256, dims[0]);
-    t.by = (uint32_t)std::max<uint64_t>(1, std::min<uint64_t>(std::min<uint64_t>(256, dims[1]), kTmaStageBytes / (t.bx * 8ull)));
+    t.stages = 4; t.stage_bytes = 49152;                  // 4 x 48 KB measured best (6 x 32 KB: -3 %, 12 x 16 KB: -10 %)
+    int ctas_per_sm = 1, max_bx = 256;
+    if (const char* f = std::getenv("CCL_REPACK_TUNE")) {   // "stages,stage_kb,ctas_per_sm,max_bx"
+        int a = 0, b = 0, c = 0, d2 = 0;
+        if (sscanf(f, "%d,%d,%d,%d", &a, &b, &c, &d2) == 4 && a > 0 && a <= kTmaMaxStages && b > 0 && c > 0 && d2 > 0) { t.stages = a; t.stage_bytes = b * 1024; ctas_per_sm = c; max_bx = d2; }
+    }
+    t.bx = (uint32_t)std::min<uint64_t>((uint64_t)max_bx, dims[0]);
+    t.by = (uint32_t)std::max<uint64_t>(1, std::min<uint64_t>(std::min<uint64_t>(256, dims[1]), t.stage_bytes / (t.bx * 8ull)));
     t.tiles_x = (uint32_t)((dims[0] + t.bx - 1) / t.bx);
     t.tiles_y = (uint32_t)((dims[1] + t.by - 1) / t.by);
     t.ntiles = (uint64_t)t.tiles_x * t.tiles_y * (uint64_t)p.nstrips;
@@ -202,13 +208,13 @@ static ccl_status launch_tma(const char* src, char* dst, const CopyPlan& p, int 
     if (s) return s;
     s = encode_tmap(&dm, CU_TENSOR_MAP_DATA_TYPE_UINT64, 3, dst, dims, dstr, box, CU_TENSOR_MAP_SWIZZLE_NONE);
     if (s) return s;
-    size_t smem = (size_t)kTmaStages * kTmaStageBytes + 128 + kTmaStages * sizeof(uint64_t);
-    static bool attr_set = false;
-    if (!attr_set) {
+    size_t smem = (size_t)t.stages * t.stage_bytes + 128 + t.stages * sizeof(uint64_t);
+    static size_t attr_set = 0;
+    if (attr_set < smem) {
         CCL_CUDA_TRY(cudaFuncSetAttribute(repack_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        attr_set = true;
+        attr_set = smem;
     }
-    unsigned grid = (unsigned)std::min<uint64_t>(t.ntiles, (uint64_t)sms);
+    unsigned grid = (unsigned)std::min<uint64_t>(t.ntiles, (uint64_t)sms * ctas_per_sm);
     repack_tma_kernel<<<grid, 32, smem, st>>>(sm, dm, t);
     count_launch();
     CCL_CUDA_TRY(cudaGetLastError());
