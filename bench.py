@@ -367,7 +367,7 @@ def main():
         args.warmup = args.warmup if args.warmup is not None else 1
         run_reference(args)
     else:
-        args.steps = args.steps if args.steps is not None else 20
+        args.steps = args.steps if args.steps is not None else 10
         args.warmup = max(3, args.warmup if args.warmup is not None else 3)
         run_cuda(args)
 
