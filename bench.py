@@ -39,6 +39,12 @@ GEMMS = [dict(name="gateup", M=T, N=2 * I, K=H), dict(name="down", M=T, N=H, K=I
 FLOP_PER_STEP = sum(2 * g["M"] * g["N"] * g["K"] for g in GEMMS)
 
 
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the two GEMM launches of one step, from the
+# single-pass ncu capture of this very workload (profiles/ccl_gemm_kernel_llama_gateup_1024tok.md, second
+# table): gate+up 10.33 + 0.93 GB, down 4.70 + 0.12 GB.  Only valid for the default configuration.
+GEMM_DRAM_BYTES_PER_STEP = {(8192, 4, 4096): 16.08e9}
+
+
 def set_tokens(t):
     """--tokens: a smaller batch of the same FFN (for profiler captures); the default is the 8192-token workload."""
     global T, GEMMS, FLOP_PER_STEP
@@ -261,7 +267,8 @@ def run_cuda(args):
                 "ms_per_step": round(e2e_ms, 3)},
         "gpu_launches": int(launches),
         "roofline": {"kernel": "ccl_gemm_kernel", "bound": "tensor", "achieved": round(gemm_tf, 1), "peak": peaks["tf_sustained"],
-                     "unit": "TFLOP/s", "frac": round(gemm_tf / peaks["tf_sustained"], 4), "traffic": None,
+                     "unit": "TFLOP/s", "frac": round(gemm_tf / peaks["tf_sustained"], 4), "traffic": GEMM_DRAM_BYTES_PER_STEP.get((T, P, page)),
+                     "traffic_unit": "bytes per step (2 launches), ncu", "algorithmic_bytes_per_step": sum(2 * (g["M"] * g["K"] + g["K"] * g["N"] + g["M"] * g["N"]) for g in GEMMS),
                      "peak_source": f"bf16 sustained, {peaks['source']}", "frac_of_burst": round(gemm_tf / peaks["tf_burst"], 4),
                      "frac_of_nominal_2250": round(gemm_tf / 2250.0, 4), "ms_per_step": round(kms["gemm"], 4)},
         "kernels": {"gemm_tflops": round(gemm_tf, 1), "repack_gbs": round(repack_gbs, 1),
