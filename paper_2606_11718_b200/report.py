@@ -187,7 +187,7 @@ def run_gemm(g, pk, reps):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--config", default="all")
-    ap.add_argument("--out", default=os.path.join(ROOT, "gpurun_out"))
+    ap.add_argument("--out", default=os.path.join(ROOT, "report_out"))
     ap.add_argument("--quick", action="store_true", help="fewer repetitions and P = 4 only in the sweep")
     args = ap.parse_args()
     assert torch.cuda.is_available(), "report needs a CUDA device"
