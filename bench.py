@@ -77,7 +77,7 @@ class ClockSampler:
             os.close(fd)
             self.proc = subprocess.Popen(["nvidia-smi", "-i", self.uuid, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
                                           "-lms", "20"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
-            time.sleep(0.05)                                           # let the first sample land before the timed region
+            time.sleep(0.4)                                            # nvidia-smi needs a moment before its first sample
         except Exception:
             self.proc = None
 
@@ -90,14 +90,14 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in open(self.path):
             f = [x.strip() for x in line.split(",")]
             if len(f) < 7:
                 continue
             try:
-                sm.append(float(f[0])); mx.append(float(f[1]))
+                sm.append(float(f[0])); mx.append(float(f[1])); pw.append(float(f[2]))
             except ValueError:
                 continue
             for n, v in zip(names, f[3:7]):
@@ -105,7 +105,7 @@ class ClockSampler:
                     reasons.add(n)
         os.unlink(self.path)
         if sm:
-            busy = [x for x in sm if x > 0.5 * max(sm)] or sm          # samples under load
+            busy = [c for c, w in zip(sm, pw) if w > 0.6 * max(pw)] or sm     # samples taken under load (by power draw)
             out.update(sm_mhz=statistics.median(busy), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
         return out
 
@@ -193,16 +193,16 @@ def run_cuda(args):
 
     barrier, max_over_ranks = group.barrier, group.max_over_ranks
 
-    # ---- device-resident timing
+    # ---- device-resident timing (the clock sampler runs from the warm-up on; idle samples are dropped by power draw)
+    uuid = "GPU-" + str(torch.cuda.get_device_properties(local).uuid).replace("GPU-", "")
+    sampler = ClockSampler(uuid)
+    sampler.start()
     for _ in range(args.warmup):
         step(False)
     st, detail = ccl.ccl_gemm_status()
     if st != ccl.OK:
         raise SystemExit(f"bench.py: device-side wait expired during warm-up (code {detail})")
-    uuid = "GPU-" + str(torch.cuda.get_device_properties(local).uuid).replace("GPU-", "")
-    sampler = ClockSampler(uuid)
     barrier()
-    sampler.start()
     launches0 = ccl.ccl_launch_count()
     t0, t1 = ev(), ev()
     t0.record()
@@ -232,20 +232,48 @@ def run_cuda(args):
     h2d = sum(v.numel() * 2 for v in host.values())
     d2h = sum(d["host_c"].numel() * 2 + 48 for d in descs)
 
-    def e2e_step():
-        for k in host:
-            devb[k].copy_(host[k], non_blocking=True)
-        step(False)
-        for d in descs:
-            d["host_c"].copy_(d["c_ccl"], non_blocking=True)
-            d["host_tot"].copy_(d["totals"], non_blocking=True)
+    # Three streams, two buffer slots: the host->device copy of step i+1 and the device->host copy of step i-1
+    # overlap the kernels of step i.  Every step still moves all of its inputs in and all of its results out.
+    s_in, s_out, s_cmp = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.current_stream()
+    slots = []
+    for sl in range(2):
+        dv = devb if sl == 0 else {k: torch.empty_like(v) for k, v in devb.items()}
+        outs = [dict(c_ccl=d["c_ccl"] if sl == 0 else torch.empty_like(d["c_ccl"]),
+                     totals=d["totals"] if sl == 0 else torch.empty_like(d["totals"]),
+                     per_cta=d["per_cta"] if sl == 0 else torch.empty_like(d["per_cta"])) for d in descs]
+        slots.append(dict(dev=dv, outs=outs, ev_in=torch.cuda.Event(), ev_cmp=torch.cuda.Event(), ev_out=torch.cuda.Event()))
+    for sl in slots:
+        sl["ev_cmp"].record(s_cmp); sl["ev_out"].record(s_cmp)
 
-    e2e_steps = max(2, min(args.steps, 5))
-    e2e_step()
+    def e2e_step(i):
+        sl = slots[i % 2]
+        with torch.cuda.stream(s_in):
+            s_in.wait_event(sl["ev_cmp"])                      # the kernels that last read this slot's inputs are done
+            for k in host:
+                sl["dev"][k].copy_(host[k], non_blocking=True)
+            sl["ev_in"].record(s_in)
+        s_cmp.wait_event(sl["ev_in"])
+        s_cmp.wait_event(sl["ev_out"])                         # this slot's previous results have left the device
+        for d, o in zip(descs, sl["outs"]):
+            ccl.ccl_repack(d["mB"], sl["dev"][d["w"]], d["w_ccl"], 0)
+            ccl.ccl_gemm(d["gd"], sl["dev"][d["a"]], d["w_ccl"], o["c_ccl"])
+            ccl.ccl_traffic(d["td"]["ccl"], o["per_cta"], o["totals"])
+        sl["ev_cmp"].record(s_cmp)
+        with torch.cuda.stream(s_out):
+            s_out.wait_event(sl["ev_cmp"])
+            for d, o in zip(descs, sl["outs"]):
+                d["host_c"].copy_(o["c_ccl"], non_blocking=True)
+                d["host_tot"].copy_(o["totals"], non_blocking=True)
+            sl["ev_out"].record(s_out)
+
+    e2e_steps = max(4, min(args.steps, 8))
+    e2e_step(0); e2e_step(1)
     barrier()
     t0.record()
-    for _ in range(e2e_steps):
-        e2e_step()
+    for i in range(e2e_steps):
+        e2e_step(i)
+    for sl in slots:
+        s_cmp.wait_event(sl["ev_out"])
     t1.record()
     barrier()
     e2e_ms = max_over_ranks(t0.elapsed_time(t1)) / e2e_steps
