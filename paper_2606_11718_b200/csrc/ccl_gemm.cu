@@ -373,14 +373,9 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             if (p.c_split == 2) { cz = nb / (int)p.c_w; cx0 = nb - cz * (int)p.c_w; cy = row0; }
             else if (p.c_split == 1) { cz = row0 / (int)p.c_h; cy = row0 - cz * (int)p.c_h; cx0 = nb; }
             else { cz = 0; cy = row0; cx0 = nb; }
-#pragma unroll 1
-            for (int c = 0; c < SUBN / 64; ++c) {
+            // One 64-column piece: registers -> C.  `r` holds 64 fp32 accumulators of this thread's row.
+            auto store_piece = [&](const uint32_t (&r)[64], int c) {
                 const int n64 = nb + c * 64;
-                if (n64 >= t.n1) break;                  // warp-uniform: nothing valid further right
-                uint32_t r[64];
-                tmem_ld32(taddr + (uint32_t)(c * 64), *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
-                tmem_ld32(taddr + (uint32_t)(c * 64 + 32), *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
-                tmem_ld_wait();
                 if (p.splits == 1 && rows_full && n64 + 64 <= t.n1) {
                     unsigned char* buf = epi + (size_t)((warp - 2) * 2 + (epi_count & 1)) * (32 * 128);
                     if (epi_count >= 2) { if (lane == 0) tma_store_wait_read<1>(); __syncwarp(); }   // buffer free again
@@ -398,7 +393,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     __syncwarp();
                     if (lane == 0) { tma_store_3d(&map_c, buf, cx0 + c * 64, cy, cz); tma_store_commit(); }
                     ++epi_count;
-                    continue;
+                    return;
                 }
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
@@ -429,6 +424,26 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                             }
                         }
                     }
+                }
+            };
+            // TMEM reads are software-pipelined: the load of piece c+1 is in flight while piece c is converted
+            // and stored (two register sets, so the loop is unrolled by two).
+            const int npieces = min(SUBN / 64, (t.n1 - nb + 63) / 64);      // warp-uniform
+            uint32_t ra[64], rb[64];
+            auto load_piece = [&](uint32_t (&r)[64], int c) {
+                tmem_ld32(taddr + (uint32_t)(c * 64), *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
+                tmem_ld32(taddr + (uint32_t)(c * 64 + 32), *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
+            };
+            if (npieces > 0) load_piece(ra, 0);
+#pragma unroll 1
+            for (int c = 0; c < npieces; c += 2) {
+                tmem_ld_wait();
+                if (c + 1 < npieces) load_piece(rb, c + 1);
+                store_piece(ra, c);
+                if (c + 1 < npieces) {
+                    tmem_ld_wait();
+                    if (c + 2 < npieces) load_piece(ra, c + 2);
+                    store_piece(rb, c + 1);
                 }
             }
             tc_fence_before();
