@@ -11,7 +11,7 @@ import numpy as np
 
 from . import build as _build
 
-ROWMAJOR, CCL = 0, 1
+ROWMAJOR, CCL, CCL_INTERLEAVED = 0, 1, 2
 PART_NONE, PART_ROWS, PART_COLS = 0, 1, 2
 PLACE_RR, PLACE_BLOCK, PLACE_BEST = 0, 1, 2
 ASSIGN_N, ASSIGN_M, ASSIGN_EXPLICIT = 0, 1, 2

@@ -15,6 +15,10 @@
 //   Sec. 2.2: C = A*B, one CTA per output tile streaming A and B along K;
 //            a column region of a column-major operand is already contiguous
 //            (PART_ROWS below)
+//   Sec. 3.3 / 4.1 ("plain 4 KB round-robin interleaving achieves the fine-grained locality"): the
+//            page-interleaved variant of CCL (layout ORC_CCL_INTERLEAVED): strip g's j-th chunk of
+//            strip_align_bytes is stored at chunk j*G + g, so an address-driven "chunk mod G" mapping
+//            sends every strip to its own chiplet
 //   Sec. 4.1: page-granularity placement policies (round-robin interleave,
 //            coarse G-block placement) and the remote-traffic metric, here
 //            WITHOUT the L2 filter: every byte a CTA touches is counted.
@@ -39,7 +43,7 @@
 
 extern "C" {
 
-enum { ORC_ROWMAJOR = 0, ORC_CCL = 1 };
+enum { ORC_ROWMAJOR = 0, ORC_CCL = 1, ORC_CCL_INTERLEAVED = 2 };
 enum { ORC_PART_NONE = 0, ORC_PART_ROWS = 1, ORC_PART_COLS = 2 };
 enum { ORC_PLACE_RR = 0, ORC_PLACE_BLOCK = 1, ORC_PLACE_BEST = 2 };
 enum { ORC_ASSIGN_N = 0, ORC_ASSIGN_M = 1, ORC_ASSIGN_EXPLICIT = 2 };
@@ -51,7 +55,8 @@ typedef struct {
     int32_t P;                  // the paper's G
     int32_t part;               // which stored dimension is split over chiplets
     int32_t layout;             // physical order of the buffer
-    int64_t strip_align_bytes;  // 0 = packed (Eq. 3 literally)
+    int64_t strip_align_bytes;  // ORC_CCL: 0 = packed (Eq. 3 literally), else strip bases rounded up to it;
+                                // ORC_CCL_INTERLEAVED: the chunk size (required)
 } orc_mat;
 
 typedef struct {
@@ -73,22 +78,33 @@ namespace {
 bool mat_ok(const orc_mat& m) {
     if (m.rows <= 0 || m.cols <= 0 || m.P < 1) return false;
     if (m.elem_bytes != 1 && m.elem_bytes != 2 && m.elem_bytes != 4) return false;
-    if (m.layout != ORC_ROWMAJOR && m.layout != ORC_CCL) return false;
+    if (m.layout != ORC_ROWMAJOR && m.layout != ORC_CCL && m.layout != ORC_CCL_INTERLEAVED) return false;
     if (m.part < 0 || m.part > 2) return false;
     if (m.strip_align_bytes < 0 || m.strip_align_bytes % m.elem_bytes) return false;
-    if (m.layout == ORC_CCL) {
+    if (m.layout != ORC_ROWMAJOR) {
         if (m.part == ORC_PART_COLS && m.cols % m.P) return false;  // w = N/G must be whole
         if (m.part == ORC_PART_ROWS && m.rows % m.P) return false;
     }
+    if (m.layout == ORC_CCL_INTERLEAVED && m.part != ORC_PART_NONE && m.strip_align_bytes <= 0) return false;
     return true;
 }
 
-bool is_ccl(const orc_mat& m) { return m.layout == ORC_CCL && m.part != ORC_PART_NONE; }
+bool is_ccl(const orc_mat& m) { return m.layout != ORC_ROWMAJOR && m.part != ORC_PART_NONE; }
+bool is_interleaved(const orc_mat& m) { return m.layout == ORC_CCL_INTERLEAVED && m.part != ORC_PART_NONE; }
+
+// Elements of one strip (K*w in the paper's notation).
+int64_t strip_elems(const orc_mat& m) {
+    return (m.part == ORC_PART_COLS) ? m.rows * (m.cols / m.P) : (m.rows / m.P) * m.cols;
+}
+// Interleaved layout: chunks of strip_align_bytes each strip needs.
+int64_t strip_chunks(const orc_mat& m) {
+    return (strip_elems(m) * m.elem_bytes + m.strip_align_bytes - 1) / m.strip_align_bytes;
+}
 
 // Elements between the bases of two consecutive strips.  Packed: K*w (Eq. 3);
 // aligned: K*w*e rounded up to the alignment (Sec. 3.2, last paragraph).
 int64_t strip_stride(const orc_mat& m) {
-    int64_t packed = (m.part == ORC_PART_COLS) ? m.rows * (m.cols / m.P) : (m.rows / m.P) * m.cols;
+    int64_t packed = strip_elems(m);
     if (m.strip_align_bytes == 0) return packed;
     int64_t bytes = packed * m.elem_bytes;
     int64_t up = (bytes + m.strip_align_bytes - 1) / m.strip_align_bytes * m.strip_align_bytes;
@@ -97,7 +113,15 @@ int64_t strip_stride(const orc_mat& m) {
 
 int64_t buffer_elems(const orc_mat& m) {
     if (!is_ccl(m)) return m.rows * m.cols;
+    if (is_interleaved(m)) return strip_chunks(m) * m.P * (m.strip_align_bytes / m.elem_bytes);
     return (int64_t)m.P * strip_stride(m);
+}
+
+// Interleaved layout: element `o` of strip g's packed contents (Eq. 3 inside the strip) lives in that strip's chunk
+// j = o*e / S, which is stored as chunk j*G + g of the buffer.
+int64_t interleave(const orc_mat& m, int64_t g, int64_t o) {
+    int64_t S = m.strip_align_bytes, b = o * m.elem_bytes;
+    return ((b / S * m.P + g) * S + b % S) / m.elem_bytes;
 }
 
 // Eq. 2 (row-major) or Eq. 1 + Eq. 3 (CCL) applied to stored coordinates.
@@ -107,18 +131,29 @@ int64_t map_offset(const orc_mat& m, int64_t r, int64_t c) {
         int64_t w = m.cols / m.P;                      // per-chiplet width
         int64_t g = c / w;                             // Eq. 1
         int64_t cp = c % w;                            // Eq. 1
+        if (is_interleaved(m)) return interleave(m, g, r * w + cp);
         return g * strip_stride(m) + r * w + cp;       // Eq. 3
     }
     // Split along rows: each strip is h whole rows, already contiguous (Sec. 2.2).
     int64_t h = m.rows / m.P;
+    if (is_interleaved(m)) return interleave(m, r / h, (r % h) * m.cols + c);
     return (r / h) * strip_stride(m) + (r % h) * m.cols + c;
 }
 
 int map_inverse(const orc_mat& m, int64_t off, int64_t* r, int64_t* c) {
     if (off < 0 || off >= buffer_elems(m)) return -1;
     if (!is_ccl(m)) { *r = off / m.cols; *c = off % m.cols; return 0; }
-    int64_t st = strip_stride(m);
-    int64_t g = off / st, rem = off % st;
+    int64_t st, g, rem;
+    if (is_interleaved(m)) {                           // undo the chunk interleave, then proceed as for a packed strip
+        int64_t S = m.strip_align_bytes, b = off * m.elem_bytes, chunk = b / S;
+        g = chunk % m.P;
+        rem = (chunk / m.P * S + b % S) / m.elem_bytes;
+        st = strip_elems(m);
+        if (rem >= st) return -2;
+    } else {
+        st = strip_stride(m);
+        g = off / st; rem = off % st;
+    }
     if (m.part == ORC_PART_COLS) {
         int64_t w = m.cols / m.P;
         if (rem >= m.rows * w) return -2;              // inside the padding of strip g
@@ -224,6 +259,14 @@ void for_each_piece_run(const orc_traffic_desc& d, const orc_mat& m, int64_t r0,
         int64_t c = c0;
         while (c < c1) {
             int64_t cend = std::min(c1, (c / w + 1) * w);
+            if (is_interleaved(m)) {                   // contiguity also ends at every chunk of the interleave
+                int64_t Si = m.strip_align_bytes;
+                int64_t rr = (m.part == ORC_PART_ROWS) ? r % (m.rows / m.P) : r;
+                int64_t roww = (m.part == ORC_PART_COLS) ? w : m.cols;
+                int64_t packed = (rr * roww + (m.part == ORC_PART_COLS ? c % w : c)) * e;   // byte inside the strip
+                int64_t sub = std::min<int64_t>((cend - c) * e, (packed / Si + 1) * Si - packed);
+                cend = c + sub / e;
+            }
             int64_t b = map_offset(m, r, c) * e, bend = b + (cend - c) * e;
             while (b < bend) {
                 int64_t pend = std::min(bend, (b / S + 1) * S);
@@ -303,7 +346,7 @@ int orc_map_inverse(const orc_mat* m, int64_t off, int64_t* r, int64_t* c) {
     return map_inverse(*m, off, r, c);
 }
 
-int orc_strip_stride(const orc_mat* m, int64_t* elems) { if (!mat_ok(*m) || !is_ccl(*m)) return -1; *elems = strip_stride(*m); return 0; }
+int orc_strip_stride(const orc_mat* m, int64_t* elems) { if (!mat_ok(*m) || !is_ccl(*m) || is_interleaved(*m)) return -1; *elems = strip_stride(*m); return 0; }
 int orc_buffer_bytes(const orc_mat* m, int64_t* bytes) { if (!mat_ok(*m)) return -1; *bytes = buffer_elems(*m) * m->elem_bytes; return 0; }
 
 // Whole map as a table: out[r*cols + c] = offset (for bijection / stride-form pins).
