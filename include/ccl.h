@@ -44,7 +44,7 @@ typedef enum {
     CCL_ERR_PADDING = 8      /* inverse map: the offset lies in alignment padding               */
 } ccl_status;
 
-typedef enum { CCL_ROWMAJOR = 0, CCL_CCL = 1 } ccl_layout;                   /* physical order of a buffer */
+typedef enum { CCL_ROWMAJOR = 0, CCL_CCL = 1, CCL_CCL_INTERLEAVED = 2 } ccl_layout; /* physical order of a buffer */
 typedef enum { CCL_PART_NONE = 0, CCL_PART_ROWS = 1, CCL_PART_COLS = 2 } ccl_part; /* stored dim split over chiplets */
 
 /*
@@ -59,7 +59,15 @@ typedef enum { CCL_PART_NONE = 0, CCL_PART_ROWS = 1, CCL_PART_COLS = 2 } ccl_par
  *       which Sec. 2.2 calls coarse-grained: already contiguous):
  *       h = rows/P, offset = (r / h)*stride + (r mod h)*cols + c, stride = h*cols
  *       (rounded up likewise).
- *   layout = CCL_CCL with part = CCL_PART_NONE behaves as CCL_ROWMAJOR.
+ *   layout = CCL_CCL_INTERLEAVED (either part): the page-interleaved form of CCL that makes a plain
+ *       address-driven round-robin mapping local (Sec. 3.3 / 4.1: "4 KB round-robin interleaving
+ *       achieves the fine-grained locality").  strip_align_bytes is the chunk size S (> 0).  Element
+ *       o of strip g's packed contents (o = r*w + c' resp. (r mod h)*cols + c, as above) sits in that
+ *       strip's chunk j = o*e / S, and chunk j of strip g is stored as chunk j*P + g of the buffer:
+ *       byte offset = (j*P + g)*S + (o*e mod S).  The buffer holds ceil(strip bytes / S)*P chunks;
+ *       the tail of every strip's last chunk is padding.  ccl_strip_stride is not defined for it.
+ *       ccl_gemm does not take this layout yet (CCL_ERR_UNSUPPORTED); map, repack and traffic do.
+ *   A CCL layout with part = CCL_PART_NONE behaves as CCL_ROWMAJOR.
  * Requirements: rows, cols > 0; elem_bytes in {1,2,4}; P >= 1; the split dimension
  * divisible by P (else CCL_ERR_SHAPE); strip_align_bytes >= 0 and a multiple of e.
  */

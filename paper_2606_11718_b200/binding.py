@@ -14,7 +14,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libccl.so")
 
 OK, ERR_INVALID_ARG, ERR_SHAPE, ERR_ALIGN, ERR_UNSUPPORTED, ERR_CUDA, ERR_WORKSPACE, ERR_TIMEOUT, ERR_PADDING = range(9)
-ROWMAJOR, CCL = 0, 1
+ROWMAJOR, CCL, CCL_INTERLEAVED = 0, 1, 2
 PART_NONE, PART_ROWS, PART_COLS = 0, 1, 2
 PLACE_RR, PLACE_BLOCK, PLACE_BEST = 0, 1, 2
 ASSIGN_N_STRIPS, ASSIGN_M_STRIPS, ASSIGN_EXPLICIT = 0, 1, 2

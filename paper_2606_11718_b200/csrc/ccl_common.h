@@ -38,21 +38,35 @@ struct MatView {
     int64_t nstrips;  // P for CCL layouts, else 1
     int32_t e;        // element bytes
     int32_t split;    // 0 none, 1 rows, 2 cols (effective: 0 for row-major)
+    int64_t ichunk;   // page-interleaved CCL: elements per chunk (0 = strips stored one after the other)
+    int64_t ichunks;  // page-interleaved CCL: chunks per strip
 };
+
+// Page-interleaved CCL: element o of strip g's packed contents -> element offset in the buffer
+// (chunk j of strip g is stored as chunk j*P + g).
+CCL_HD int64_t interleave(const MatView& v, int64_t g, int64_t o) {
+    int64_t j = o / v.ichunk;
+    return (j * v.nstrips + g) * v.ichunk + (o - j * v.ichunk);
+}
 
 CCL_HD int64_t map(const MatView& v, int64_t r, int64_t c) {
     if (v.split == 2) {                      // Eq. 1 + Eq. 3
         int64_t g = c / v.w, cp = c - g * v.w;
+        if (v.ichunk) return interleave(v, g, r * v.w + cp);
         return g * v.stride + r * v.w + cp;
     }
     if (v.split == 1) {                      // strips of h whole rows
         int64_t g = r / v.h, rp = r - g * v.h;
+        if (v.ichunk) return interleave(v, g, rp * v.cols + c);
         return g * v.stride + rp * v.cols + c;
     }
     return r * v.cols + c;                   // Eq. 2
 }
 
-CCL_HD int64_t buffer_elems(const MatView& v) { return v.split ? v.nstrips * v.stride : v.rows * v.cols; }
+CCL_HD int64_t buffer_elems(const MatView& v) {
+    if (v.ichunk) return v.ichunks * v.nstrips * v.ichunk;
+    return v.split ? v.nstrips * v.stride : v.rows * v.cols;
+}
 
 // Validates a descriptor and flattens it.  `what` names the argument in error messages.
 ccl_status make_view(const ccl_mat* m, const char* what, MatView* out);

@@ -509,6 +509,7 @@ struct GemmPlan {
 
 static ccl_status check_operand(const MatView& v, const void* ptr, const char* name) {
     if (v.e != 2) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: %s: only 2-byte (bf16) elements are supported", name);
+    if (v.ichunk) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: %s: the page-interleaved layout is not supported by the GEMM yet", name);
     int64_t inner = v.split == 2 ? v.w : v.cols;
     if (inner % 8) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: %s: contiguous extent %lld is not a multiple of 8 elements", name, (long long)inner);
     if (v.split && (v.stride * v.e) % 16) return fail(CCL_ERR_ALIGN, "ccl_gemm: %s: strip stride is not a multiple of 16 bytes", name);

@@ -28,7 +28,7 @@ ccl_status make_view(const ccl_mat* m, const char* what, MatView* out) {
     if (m->elem_bytes != 1 && m->elem_bytes != 2 && m->elem_bytes != 4)
         return fail(CCL_ERR_INVALID_ARG, "%s: elem_bytes must be 1, 2 or 4", what);
     if (m->P < 1) return fail(CCL_ERR_INVALID_ARG, "%s: P must be >= 1", what);
-    if (m->layout != CCL_ROWMAJOR && m->layout != CCL_CCL) return fail(CCL_ERR_INVALID_ARG, "%s: unknown layout", what);
+    if (m->layout != CCL_ROWMAJOR && m->layout != CCL_CCL && m->layout != CCL_CCL_INTERLEAVED) return fail(CCL_ERR_INVALID_ARG, "%s: unknown layout", what);
     if (m->part != CCL_PART_NONE && m->part != CCL_PART_ROWS && m->part != CCL_PART_COLS)
         return fail(CCL_ERR_INVALID_ARG, "%s: unknown part", what);
     if (m->strip_align_bytes < 0 || m->strip_align_bytes % m->elem_bytes)
@@ -39,8 +39,8 @@ ccl_status make_view(const ccl_mat* m, const char* what, MatView* out) {
         return fail(CCL_ERR_INVALID_ARG, "%s: matrix too large", what);
     MatView v;
     v.rows = m->rows; v.cols = m->cols; v.e = m->elem_bytes;
-    v.w = m->cols; v.h = m->rows; v.stride = 0; v.nstrips = 1; v.split = 0;
-    if (m->layout == CCL_CCL && m->part != CCL_PART_NONE) {
+    v.w = m->cols; v.h = m->rows; v.stride = 0; v.nstrips = 1; v.split = 0; v.ichunk = 0; v.ichunks = 0;
+    if (m->layout != CCL_ROWMAJOR && m->part != CCL_PART_NONE) {
         int64_t packed;
         if (m->part == CCL_PART_COLS) {
             if (m->cols % m->P) return fail(CCL_ERR_SHAPE, "%s: cols (%lld) not divisible by P (%d)", what, (long long)m->cols, m->P);
@@ -50,7 +50,12 @@ ccl_status make_view(const ccl_mat* m, const char* what, MatView* out) {
             v.h = m->rows / m->P; packed = v.h * m->cols; v.split = 1;
         }
         v.nstrips = m->P;
-        if (m->strip_align_bytes) {
+        if (m->layout == CCL_CCL_INTERLEAVED) {
+            if (m->strip_align_bytes <= 0) return fail(CCL_ERR_INVALID_ARG, "%s: the interleaved layout needs strip_align_bytes (the chunk size) > 0", what);
+            v.ichunk = m->strip_align_bytes / m->elem_bytes;
+            v.ichunks = (packed + v.ichunk - 1) / v.ichunk;
+            v.stride = packed;                 // strip-local extent; strips are not stored one after the other
+        } else if (m->strip_align_bytes) {
             int64_t a = m->strip_align_bytes, bytes = packed * m->elem_bytes;
             v.stride = (bytes + a - 1) / a * a / m->elem_bytes;
         } else {
@@ -84,7 +89,13 @@ ccl_status ccl_map_inverse(const ccl_mat* m, int64_t off, int64_t* r, int64_t* c
     if (!r || !c) return fail(CCL_ERR_INVALID_ARG, "ccl_map_inverse: NULL output");
     if (off < 0 || off >= buffer_elems(v)) return fail(CCL_ERR_INVALID_ARG, "ccl_map_inverse: offset out of range");
     if (v.split == 0) { *r = off / v.cols; *c = off % v.cols; return CCL_OK; }
-    int64_t g = off / v.stride, rem = off % v.stride;
+    int64_t g, rem;
+    if (v.ichunk) {                        // undo the chunk interleave, then proceed as for a packed strip
+        int64_t chunk = off / v.ichunk;
+        g = chunk % v.nstrips;
+        rem = (chunk / v.nstrips) * v.ichunk + off % v.ichunk;
+        if (rem >= v.stride) return fail(CCL_ERR_PADDING, "ccl_map_inverse: offset lies in the padding of strip %lld", (long long)g);
+    } else { g = off / v.stride; rem = off % v.stride; }
     if (v.split == 2) {
         if (rem >= v.rows * v.w) return fail(CCL_ERR_PADDING, "ccl_map_inverse: offset lies in the padding of strip %lld", (long long)g);
         *r = rem / v.w; *c = g * v.w + rem % v.w;
@@ -110,6 +121,7 @@ ccl_status ccl_strip_stride(const ccl_mat* m, int64_t* elems) {
     if (s) return s;
     if (!elems) return fail(CCL_ERR_INVALID_ARG, "ccl_strip_stride: NULL output");
     if (v.split == 0) return fail(CCL_ERR_INVALID_ARG, "ccl_strip_stride: not a CCL layout");
+    if (v.ichunk) return fail(CCL_ERR_INVALID_ARG, "ccl_strip_stride: not defined for the interleaved layout");
     *elems = v.stride;
     return CCL_OK;
 }

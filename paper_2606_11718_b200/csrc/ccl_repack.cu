@@ -22,7 +22,16 @@ struct CopyPlan {
     int64_t nstrips, rows, row_bytes;         // rows per strip, bytes per strip row
     int64_t src_g, src_r, dst_g, dst_r;       // byte strides
     int64_t pad_off, pad_bytes, pad_g;        // dir 0: zero dst[g*pad_g + pad_off, +pad_bytes) for every strip
+    // page-interleaved CCL side (il_chunk = 0: none): byte b of strip g's packed contents lives at
+    // g*il_chunk + (b / il_chunk)*il_chunk*il_P + b % il_chunk
+    int64_t il_chunk, il_P;
+    int32_t il_shift, il_dst;                 // log2(il_chunk) or -1; 1 = the destination is the interleaved side
 };
+
+__device__ __forceinline__ int64_t interleaved_off(const CopyPlan& p, int64_t g, int64_t b) {
+    const int64_t j = p.il_shift >= 0 ? (b >> p.il_shift) : (b / p.il_chunk);
+    return g * p.il_chunk + j * p.il_chunk * p.il_P + (b - j * p.il_chunk);
+}
 
 __device__ int g_repack_status = 0;
 
@@ -55,20 +64,27 @@ __global__ void __launch_bounds__(kVecThreads) repack_vec_kernel(const char* __r
     for (IDX base = (IDX)blockIdx.x * kVecThreads * kVecUnroll + threadIdx.x; base < chunks_per_strip; base += step) {
         V v[kVecUnroll];
         int64_t doff[kVecUnroll];
+        bool live[kVecUnroll];
 #pragma unroll
         for (int u = 0; u < kVecUnroll; ++u) {
             IDX j = base + (IDX)u * kVecThreads;
-            doff[u] = -1;
-            if (j < chunks_per_strip) {
+            live[u] = j < chunks_per_strip;
+            if (live[u]) {
                 IDX r = j / chunks_per_row;
                 IDX x = j - r * chunks_per_row;
-                v[u] = ld_stream(reinterpret_cast<const V*>(s + (int64_t)r * p.src_r + (int64_t)x * (int64_t)sizeof(V)));
-                doff[u] = (int64_t)r * p.dst_r + (int64_t)x * (int64_t)sizeof(V);
+                int64_t so = (int64_t)r * p.src_r + (int64_t)x * (int64_t)sizeof(V);
+                int64_t dn = (int64_t)r * p.dst_r + (int64_t)x * (int64_t)sizeof(V);
+                if (p.il_chunk) {                 // the CCL side is addressed through the chunk interleave
+                    const int64_t b = (int64_t)r * p.row_bytes + (int64_t)x * (int64_t)sizeof(V);
+                    if (p.il_dst) dn = interleaved_off(p, g, b) - g * p.dst_g; else so = interleaved_off(p, g, b) - g * p.src_g;
+                }
+                v[u] = ld_stream(reinterpret_cast<const V*>(s + so));
+                doff[u] = dn;
             }
         }
 #pragma unroll
         for (int u = 0; u < kVecUnroll; ++u)
-            if (doff[u] >= 0) st_stream(reinterpret_cast<V*>(d + doff[u]), v[u]);
+            if (live[u]) st_stream(reinterpret_cast<V*>(d + doff[u]), v[u]);
     }
 }
 
@@ -264,18 +280,27 @@ extern "C" ccl_status ccl_repack(const ccl_mat* m, const void* src_dev, void* ds
     if (p.nstrips > 65535) return fail(CCL_ERR_UNSUPPORTED, "ccl_repack: P > 65535");
     if (dir == 0) { p.src_g = rm_g; p.src_r = rm_r; p.dst_g = cc_g; p.dst_r = cc_r; }
     else          { p.src_g = cc_g; p.src_r = cc_r; p.dst_g = rm_g; p.dst_r = rm_r; }
-    if (dir == 0 && v.split) {
+    if (dir == 0 && v.split && !v.ichunk) {
         p.pad_off = p.rows * p.row_bytes; p.pad_bytes = v.stride * e - p.pad_off; p.pad_g = cc_g;
+    }
+    if (v.ichunk) {                           // page-interleaved CCL: chunk j of strip g is chunk j*P + g of the buffer
+        const int64_t S = v.ichunk * e, Bs = p.rows * p.row_bytes;
+        p.il_chunk = S; p.il_P = v.nstrips; p.il_dst = dir == 0;
+        p.il_shift = -1;
+        if ((S & (S - 1)) == 0) { int sh = 0; while ((INT64_C(1) << sh) < S) ++sh; p.il_shift = sh; }
+        if (dir == 0) {                       // the tail of every strip's last chunk is padding
+            p.pad_g = S; p.pad_off = (v.ichunks - 1) * v.nstrips * S + (Bs - (v.ichunks - 1) * S); p.pad_bytes = v.ichunks * S - Bs;
+        }
     }
 
     const char* src = static_cast<const char*>(src_dev);
     char* dst = static_cast<char*>(dst_dev);
     int64_t addr_bits = (int64_t)((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst)) & 15);
-    int64_t vec = pow2_divisor(p.row_bytes | p.src_g | p.src_r | p.dst_g | p.dst_r | addr_bits, 16);
+    int64_t vec = pow2_divisor(p.row_bytes | p.src_g | p.src_r | p.dst_g | p.dst_r | p.il_chunk | addr_bits, 16);
 
     // path choice: TMA when everything is 16-byte aligned and the copy is big enough to be worth a ring
     const char* force = std::getenv("CCL_REPACK_PATH");
-    bool tma_ok = vec == 16 && p.rows < (INT64_C(1) << 31) && p.row_bytes / 8 < (INT64_C(1) << 31) &&
+    bool tma_ok = vec == 16 && !p.il_chunk && p.rows < (INT64_C(1) << 31) && p.row_bytes / 8 < (INT64_C(1) << 31) &&
                   std::max(std::max(p.src_g, p.src_r), std::max(p.dst_g, p.dst_r)) < (INT64_C(1) << 40);
     bool use_tma = tma_ok && p.nstrips * p.rows * p.row_bytes >= (INT64_C(1) << 20);
     if (force && !std::strcmp(force, "vec")) use_tma = false;

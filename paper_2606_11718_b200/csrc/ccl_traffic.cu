@@ -82,7 +82,15 @@ __device__ __forceinline__ void walk_row(const TrafficParams& p, const MatView& 
         if (v.split == 2) {
             int64_t g = c / v.w;
             cend = min(c1, (g + 1) * v.w);
-            off = g * v.stride + r * v.w + (c - g * v.w);
+            if (v.ichunk) {                        // page-interleaved CCL: contiguity also ends at every chunk
+                const int64_t o = r * v.w + (c - g * v.w);
+                cend = min(cend, c + (o / v.ichunk + 1) * v.ichunk - o);
+                off = interleave(v, g, o);
+            } else off = g * v.stride + r * v.w + (c - g * v.w);
+        } else if (v.ichunk) {                     // split along rows, page-interleaved
+            const int64_t g = r / v.h, o = (r - g * v.h) * v.cols + c;
+            cend = min(c1, c + (o / v.ichunk + 1) * v.ichunk - o);
+            off = interleave(v, g, o);
         } else {
             cend = c1;
             off = map(v, r, c);

@@ -8,7 +8,8 @@ For every GEMM of a configuration it measures, with CUDA events on the launching
     under the plain raster (Sec. 3.3: the layout should not change the speed);
   * ccl_traffic under the policies of Sec. 4.1 -- row-major + round-robin at 4 KB (the baseline),
     64 KB and 2 MB, row-major + coarse block placement, row-major + best page-granular placement,
-    CCL + page->strip placement, CCL + literal round-robin -- for the N- and the M-partition of C,
+    CCL + page->strip placement, CCL + literal round-robin, page-interleaved CCL + literal round-robin
+    -- for the N- and the M-partition of C,
     and prints remote bytes relative to the 4 KB round-robin baseline (no L2 filter: every byte a CTA
     touches is counted, so the ratios are not the paper's simulated ones).
 Roofline per GEMM: min(tensor peak, HBM peak * arithmetic intensity), against the measured peaks in
@@ -93,9 +94,9 @@ def traffic_remote(g, layout_bc, place_bc, S, assign, align=0):
     shapes = (a_shape, b_shape, (M, N))
     ms = []
     for X in range(3):
-        is_ccl = layout_bc == ccl.CCL and parts[X] != ccl.PART_NONE
+        is_ccl = layout_bc != ccl.ROWMAJOR and parts[X] != ccl.PART_NONE
         ms.append(ccl.Mat(shapes[X][0], shapes[X][1], 2, P, parts[X] if is_ccl else ccl.PART_NONE,
-                          ccl.CCL if is_ccl else ccl.ROWMAJOR, align if is_ccl else 0))
+                          layout_bc if is_ccl else ccl.ROWMAJOR, align if is_ccl else 0))
     td.A, td.B, td.C = ms
     td.a_trans, td.b_trans, td.P, td.page_bytes = at, bt, P, S
     for X in range(3):
@@ -166,7 +167,7 @@ def run_gemm(g, pk, reps):
     for tag, lay, place, Sp in (("row_rr4k", ccl.ROWMAJOR, ccl.PLACE_RR, 4096), ("row_rr64k", ccl.ROWMAJOR, ccl.PLACE_RR, 65536),
                                 ("row_rr2m", ccl.ROWMAJOR, ccl.PLACE_RR, 2 << 20), ("row_block", ccl.ROWMAJOR, ccl.PLACE_BLOCK, S),
                                 ("row_best", ccl.ROWMAJOR, ccl.PLACE_BEST, S), ("ccl_block", ccl.CCL, ccl.PLACE_BLOCK, S),
-                                ("ccl_rr", ccl.CCL, ccl.PLACE_RR, S)):
+                                ("ccl_rr", ccl.CCL, ccl.PLACE_RR, S), ("ileave_rr", ccl.CCL_INTERLEAVED, ccl.PLACE_RR, S)):
         best = None
         for assign in (ccl.ASSIGN_N_STRIPS, ccl.ASSIGN_M_STRIPS):
             r = traffic_remote(g, lay, place, Sp, assign, align=Sp)
@@ -207,7 +208,8 @@ def main():
                   f"bits_equal={r.get('ccl_equals_rowmajor_bits')} | repack {r.get('repack', {}).get('gbs', float('nan')):7.1f} GB/s | "
                   f"remote/rr4k: rr64k {t['row_rr64k']['ratio_vs_rr4k']:.3f} rr2m {t['row_rr2m']['ratio_vs_rr4k']:.3f} "
                   f"block {t['row_block']['ratio_vs_rr4k']:.3f} best {t['row_best']['ratio_vs_rr4k']:.3f} "
-                  f"CCL {t['ccl_block']['ratio_vs_rr4k']:.3f} ({t['ccl_block']['partition']}) ccl+rr {t['ccl_rr']['ratio_vs_rr4k']:.3f}", flush=True)
+                  f"CCL {t['ccl_block']['ratio_vs_rr4k']:.3f} ({t['ccl_block']['partition']}) ccl+rr {t['ccl_rr']['ratio_vs_rr4k']:.3f} "
+                  f"interleaved-CCL+rr {t['ileave_rr']['ratio_vs_rr4k']:.3f}", flush=True)
         json.dump(dict(config=cfg, peaks=pk, gemms=rows), open(os.path.join(args.out, f"report_config{cfg}.json"), "w"), indent=1)
         nz = [r["traffic"]["ccl_block"]["ratio_vs_rr4k"] for r in rows if r["traffic"]["ccl_block"]["ratio_vs_rr4k"]]
         if nz:

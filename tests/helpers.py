@@ -35,8 +35,9 @@ def traffic_pair(M, N, K, P, S, lay=("row", "row", "row"), place=(0, 0, 0), a_tr
         d.M, d.N, d.K, d.BM, d.BN = M, N, K, BM, BN
         mats = []
         for X in range(3):
-            is_ccl = lay[X] == "ccl" and parts[X] != 0
-            mats.append(mod.Mat(shapes[X][0], shapes[X][1], e, P, parts[X] if is_ccl else 0, 1 if is_ccl else 0, align if is_ccl else 0))
+            is_ccl = lay[X] in ("ccl", "ileave") and parts[X] != 0      # "ileave": page-interleaved CCL, align = chunk size
+            mats.append(mod.Mat(shapes[X][0], shapes[X][1], e, P, parts[X] if is_ccl else 0,
+                                (2 if lay[X] == "ileave" else 1) if is_ccl else 0, align if is_ccl else 0))
         d.A, d.B, d.C = mats
         d.a_trans, d.b_trans, d.P, d.page_bytes = a_trans, b_trans, P, S
         d.place[0], d.place[1], d.place[2] = place

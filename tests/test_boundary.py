@@ -49,6 +49,10 @@ MAP_CASES = [
     dict(rows=6, cols=36, P=3, part=2, layout=1, align=256),
     dict(rows=6, cols=36, P=3, part=1, layout=1, align=4096),
     dict(rows=5, cols=30, P=5, part=2, layout=1, align=64, e=4),
+    dict(rows=4, cols=8, P=2, part=2, layout=2, align=16),                 # page-interleaved CCL, the hand example
+    dict(rows=7, cols=24, P=3, part=2, layout=2, align=64),
+    dict(rows=12, cols=40, P=4, part=1, layout=2, align=48, e=4),
+    dict(rows=33, cols=96, P=4, part=2, layout=2, align=256, e=1),
 ]
 
 
@@ -62,6 +66,9 @@ def test_host_map_equals_oracle(case):
     assert ccl.ccl_buffer_bytes(ml) == orc.buffer_bytes(mo)
     if case["layout"] == 1 and case["part"] != 0:
         assert ccl.ccl_strip_stride(ml) == orc.strip_stride(mo)
+    if case["layout"] == 2:
+        with pytest.raises(ccl.CclError):
+            ccl.ccl_strip_stride(ml)
     n = orc.buffer_bytes(mo) // mo.elem_bytes
     for off in range(n):
         rc, r, c = orc.map_inverse(mo, off)
@@ -94,6 +101,7 @@ def test_map_error_codes():
     expect(ccl.ERR_INVALID_ARG, ccl.ccl_map_offset, ccl.Mat(4, 8, 2, 0, 2, 1), 0, 0)
     expect(ccl.ERR_INVALID_ARG, ccl.ccl_map_offset, ccl.Mat(4, 8, 2, 2, 2, 1, 3), 0, 0)
     expect(ccl.ERR_INVALID_ARG, ccl.ccl_strip_stride, ccl.Mat(4, 8))
+    expect(ccl.ERR_INVALID_ARG, ccl.ccl_map_offset, ccl.Mat(4, 8, 2, 2, 2, 2, 0), 0, 0)      # interleaved layout without a chunk size
     expect(ccl.ERR_INVALID_ARG, ccl.ccl_map_inverse, ccl.Mat(4, 8), 32)
 
 
@@ -134,6 +142,9 @@ def test_gemm_rejects_bad_input_before_any_launch():
     assert gemm_rc(d) == ccl.ERR_UNSUPPORTED
     d = gemm_desc(128, 256, 64, 3, ("row", "row", "row"))
     assert gemm_rc(d) == ccl.ERR_SHAPE                                                               # N % P with a grouped raster
+    d = gemm_desc(128, 256, 64, 2, ("row", "ccl", "ccl"), align=4096)
+    d.B.layout = 2                                                                                   # page-interleaved operand
+    assert gemm_rc(d) == ccl.ERR_UNSUPPORTED
     d = gemm_desc(128, 256, 64)
     d.out_part = 7
     assert gemm_rc(d) == ccl.ERR_INVALID_ARG

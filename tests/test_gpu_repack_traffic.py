@@ -69,6 +69,14 @@ REPACK_CASES = [
     dict(rows=1000, cols=4096, P=2, part=2, layout=1, align=65536),
     dict(rows=4099, cols=2056, P=2, part=2, layout=1),                 # ragged: rows and box tails
     dict(rows=300, cols=8192, P=2, part=2, layout=0),                  # row-major descriptor: identity
+    dict(rows=4, cols=8, P=2, part=2, layout=2, align=16),             # page-interleaved CCL: the hand example
+    dict(rows=130, cols=384, P=4, part=2, layout=2, align=4096),       # strips are not whole chunks
+    dict(rows=2048, cols=1536, P=4, part=2, layout=2, align=4096),     # Qwen gate/up weight, 4 KB chunks
+    dict(rows=768, cols=2048, P=8, part=2, layout=2, align=65536),
+    dict(rows=768, cols=2048, P=4, part=1, layout=2, align=4096),
+    dict(rows=77, cols=96, P=3, part=2, layout=2, align=48, e=1),      # chunk size not a power of two
+    dict(rows=64, cols=200, P=2, part=2, layout=2, align=40),          # 8-byte vectors at most
+    dict(rows=4099, cols=2056, P=2, part=2, layout=2, align=2 << 20),
 ]
 
 
@@ -150,7 +158,7 @@ SHAPES = [
     dict(M=1, N=512, K=256, P=4, S=4096),
     dict(M=16, N=512, K=256, P=1, S=4096),
 ]
-LAYS = [("row", "row", "row"), ("row", "ccl", "ccl"), ("ccl", "ccl", "ccl")]
+LAYS = [("row", "row", "row"), ("row", "ccl", "ccl"), ("ccl", "ccl", "ccl"), ("row", "ileave", "ileave"), ("ileave", "ileave", "ileave")]
 PLACES = [(0, 0, 0), (1, 1, 1), (2, 2, 2), (0, 1, 2)]
 
 
@@ -158,9 +166,20 @@ PLACES = [(0, 0, 0), (1, 1, 1), (2, 2, 2), (0, 1, 2)]
 @pytest.mark.parametrize("lay", LAYS)
 @pytest.mark.parametrize("place", PLACES)
 def test_traffic_bit_exact_small(shape, lay, place):
-    for align in (0, 1024):
+    for align in ((64, 1024) if "ileave" in lay else (0, 1024)):       # the interleaved layout needs a chunk size
         do, dl = traffic_pair(lay=lay, place=place, align=align, **shape)
         run_traffic(do, dl, "elem")
+
+
+@pytest.mark.parametrize("P", [2, 4, 8])
+def test_traffic_interleaved_ccl_is_local_under_literal_round_robin(P):
+    """Sec. 3.3 / 4.1: with the page-interleaved CCL buffers, plain 4 KB round-robin puts B and C on their chiplets."""
+    from paper_2606_11718_b200 import synth
+    for g in synth.qwen_ffn_gemms()[:2] + [dict(M=1024, N=8192, K=28672, a_trans=0, b_trans=0)]:
+        base = dict(M=g["M"], N=g["N"], K=g["K"], P=P, S=4096, a_trans=g["a_trans"], b_trans=g["b_trans"])
+        r = run_traffic(*traffic_pair(lay=("row", "ileave", "ileave"), place=(0, 0, 0), align=4096, **base), level="runs")
+        assert r["totals"][1, 1] == 0 and r["totals"][2, 1] == 0
+        r = run_traffic(*traffic_pair(lay=("row", "ileave", "ileave"), place=(0, 0, 0), align=65536, **base), level="runs")
 
 
 def test_traffic_explicit_assignment():
