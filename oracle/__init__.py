@@ -150,5 +150,14 @@ def traffic(d, explicit_q=None, level="elem"):
     return dict(per_cta=per_cta, per_page=per_page, owner=owner, totals=totals)
 
 
+def traffic_ideal_l2(d, explicit_q=None):
+    """Local / remote bytes [3,2] when every chiplet fetches each byte at most once (ideal private L2)."""
+    totals = np.zeros((3, 2), dtype=np.uint64)
+    qarr = None if explicit_q is None else np.ascontiguousarray(explicit_q, dtype=np.int32)
+    if lib().orc_traffic_ideal_l2(C.byref(d), None if qarr is None else _p(qarr), _p(totals)):
+        raise ValueError("bad traffic descriptor (or a BEST placement)")
+    return totals
+
+
 def f32_to_bf16(x):
     return lib().orc_f32_to_bf16(C.c_float(x))

@@ -457,6 +457,39 @@ int orc_traffic_elem(const orc_traffic_desc* d, const int32_t* explicit_q, uint6
     return traffic_impl<false>(*d, explicit_q, per_cta, per_page, owner, totals);
 }
 
+// Remote traffic behind an IDEAL private L2 per chiplet (a step towards the metric of Sec. 4.1, which counts
+// only the reads that miss the chiplet's L2): a chiplet fetches every byte it needs at most once, however many of
+// its CTAs touch it; output writes are counted once each.  Brute force: one "touched" bitmap per chiplet and
+// operand, then every touched element is charged to local or remote by the owner of its page.
+//   totals [3 operands][local, remote] bytes, summed over chiplets.  Fixed placements only (RR, BLOCK).
+int orc_traffic_ideal_l2(const orc_traffic_desc* d, const int32_t* explicit_q, uint64_t* totals) {
+    if (!traffic_desc_ok(*d)) return -1;
+    std::vector<Tile> tiles;
+    if (enumerate_tiles(*d, explicit_q, tiles)) return -1;
+    const orc_mat* ms[3] = {&d->A, &d->B, &d->C};
+    for (int i = 0; i < 6; ++i) totals[i] = 0;
+    for (int X = 0; X < 3; ++X) {
+        if (d->place[X] == ORC_PLACE_BEST) return -1;
+        const orc_mat& m = *ms[X];
+        int64_t n = buffer_elems(m), bytes_total = n * m.elem_bytes;
+        for (int q = 0; q < d->P; ++q) {
+            std::vector<uint8_t> touched((size_t)n, 0);
+            for (const Tile& t : tiles) {
+                if (t.q != q) continue;
+                int64_t r0, r1, c0, c1; tile_rect(*d, t, X, r0, r1, c0, c1);
+                for (int64_t r = r0; r < r1; ++r) for (int64_t c = c0; c < c1; ++c) touched[(size_t)map_offset(m, r, c)] = 1;
+            }
+            for (int64_t off = 0; off < n; ++off) {
+                if (!touched[(size_t)off]) continue;
+                int64_t page = off * m.elem_bytes / d->page_bytes;
+                int32_t o = fixed_owner(d->place[X], page, d->page_bytes, d->P, bytes_total);
+                totals[X * 2 + (o == q ? 0 : 1)] += (uint64_t)m.elem_bytes;
+            }
+        }
+    }
+    return 0;
+}
+
 // The same count taken run by run (a stored row of a tile is one contiguous run per strip,
 // cut at page boundaries).  Validated against orc_traffic_elem in the tests; used at sizes
 // where the element walk would take minutes.
