@@ -221,6 +221,17 @@ ccl_status ccl_traffic(const ccl_traffic_desc* d, const int32_t* cta_chiplet_dev
                        uint64_t* const per_page_dev[3], uint8_t* const owner_dev[3], uint64_t* totals_dev,
                        void* cuda_stream);
 
+/*
+ * The same count behind an IDEAL private L2 per chiplet: a chiplet fetches every byte it needs at most once,
+ * however many of its CTAs read it (A is shared by the tiles of a tile row, B by those of a tile column), and
+ * every output byte is written once.  This is a step from the every-byte count above towards the metric of
+ * Sec. 4.1, which counts only the reads that miss the chiplet's L2 (finite there, unbounded here).
+ *   totals_l2_dev uint64 [3 (A,B,C)][2 (local, remote)], summed over chiplets (device, overwritten).
+ * Fixed placements only (CCL_PLACE_RR, CCL_PLACE_BLOCK; CCL_PLACE_BEST -> CCL_ERR_UNSUPPORTED).
+ */
+ccl_status ccl_traffic_l2(const ccl_traffic_desc* d, const int32_t* cta_chiplet_dev, uint64_t* totals_l2_dev,
+                          void* cuda_stream);
+
 /* Message for the last non-OK status returned on this thread ("" if none). Static storage. */
 const char* ccl_last_error(void);
 /* Number of CUDA kernels this library has launched in this process (all threads, all streams). */

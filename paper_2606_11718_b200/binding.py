@@ -20,7 +20,7 @@ PLACE_RR, PLACE_BLOCK, PLACE_BEST = 0, 1, 2
 ASSIGN_N_STRIPS, ASSIGN_M_STRIPS, ASSIGN_EXPLICIT = 0, 1, 2
 
 EXPORTS = ["ccl_map_offset", "ccl_map_inverse", "ccl_buffer_bytes", "ccl_strip_stride", "ccl_repack", "ccl_gemm_workspace",
-           "ccl_gemm", "ccl_gemm_static_ws", "ccl_gemm_status", "ccl_traffic_sizes", "ccl_traffic", "ccl_last_error", "ccl_launch_count", "ccl_version"]
+           "ccl_gemm", "ccl_gemm_static_ws", "ccl_gemm_status", "ccl_traffic_sizes", "ccl_traffic", "ccl_traffic_l2", "ccl_last_error", "ccl_launch_count", "ccl_version"]
 
 
 class CclError(RuntimeError):
@@ -78,6 +78,7 @@ def lib():
         l.ccl_traffic_sizes.argtypes = [C.POINTER(TrafficDesc), C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
         l.ccl_traffic.argtypes = [C.POINTER(TrafficDesc), C.c_void_p, C.c_void_p, C.POINTER(C.c_void_p), C.POINTER(C.c_void_p),
                                   C.c_void_p, C.c_void_p]
+        l.ccl_traffic_l2.argtypes = [C.POINTER(TrafficDesc), C.c_void_p, C.c_void_p, C.c_void_p]
         _lib = l
     return _lib
 
@@ -188,3 +189,8 @@ def ccl_traffic(d, per_cta, totals, per_page=None, owner=None, cta_chiplet=None)
     pp = (C.c_void_p * 3)(*[(t.data_ptr() if t is not None else None) for t in per_page]) if per_page is not None else None
     ow = (C.c_void_p * 3)(*[(t.data_ptr() if t is not None else None) for t in owner]) if owner is not None else None
     _check(lib().ccl_traffic(C.byref(d), _ptr(cta_chiplet), _ptr(per_cta), pp, ow, _ptr(totals), _stream()))
+
+
+def ccl_traffic_l2(d, totals_l2, cta_chiplet=None):
+    """Local / remote bytes [3,2] behind an ideal private L2 per chiplet (each chiplet fetches a byte at most once)."""
+    _check(lib().ccl_traffic_l2(C.byref(d), _ptr(cta_chiplet), _ptr(totals_l2), _stream()))

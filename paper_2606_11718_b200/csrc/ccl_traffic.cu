@@ -38,6 +38,7 @@ struct TrafficParams {
     uint64_t* per_page[3];
     uint8_t* owner[3];
     uint64_t* totals;
+    uint64_t* totals_l2;          // optional: totals behind an ideal private L2 per chiplet (each byte fetched once per chiplet)
 };
 
 struct ZeroSeg { uint64_t* p[4]; int64_t n[4]; };
@@ -128,10 +129,10 @@ template <bool HIST, bool CLASSIFY>
 __global__ void __launch_bounds__(kWalkThreads) traffic_walk_kernel(TrafficParams p) {
     __shared__ unsigned long long own[256];       // bytes of the rectangle whose page belongs to chiplet o
     __shared__ unsigned int cnt[256];             // tiles sharing the rectangle that run on chiplet q
-    __shared__ unsigned long long blk[6];
+    __shared__ unsigned long long blk[12];        // [0,6): totals, [6,12): totals behind the ideal L2
     const int tid = threadIdx.x, lane = tid & 31;
     const int64_t item = blockIdx.x;
-    if (tid < 6) blk[tid] = 0;
+    if (tid < 12) blk[tid] = 0;
     if (item < p.tiles_m + p.tiles_n) {
         const int X = item < p.tiles_m ? 0 : 1;
         const int64_t j = X == 0 ? item : item - p.tiles_m;
@@ -141,7 +142,7 @@ __global__ void __launch_bounds__(kWalkThreads) traffic_walk_kernel(TrafficParam
         const int64_t t_first = X == 0 ? j * p.tiles_n : j, t_step = X == 0 ? 1 : p.tiles_n;
         for (int i = tid; i < p.P; i += kWalkThreads) { own[i] = 0; cnt[i] = 0; }
         __syncthreads();
-        if (do_hist) {
+        if (do_hist || p.totals_l2) {
             for (int64_t o = tid; o < nshare; o += kWalkThreads) atomicAdd(&cnt[decode_tile(p, t_first + o * t_step).q], 1u);
             __syncthreads();
         }
@@ -183,10 +184,12 @@ __global__ void __launch_bounds__(kWalkThreads) traffic_walk_kernel(TrafficParam
             for (int64_t o = tid; o < nshare; o += kWalkThreads) {
                 const int64_t t = t_first + o * t_step;
                 const unsigned long long loc = own[decode_tile(p, t).q];
-                p.per_cta[t * 6 + X * 2 + 0] = loc;
-                p.per_cta[t * 6 + X * 2 + 1] = total - loc;
+                if (p.per_cta) { p.per_cta[t * 6 + X * 2 + 0] = loc; p.per_cta[t * 6 + X * 2 + 1] = total - loc; }
                 loc_sum += loc; rem_sum += total - loc;
             }
+            if (p.totals_l2)                              // a chiplet fetches this rectangle once, however many of its tiles share it
+                for (int q = tid; q < p.P; q += kWalkThreads)
+                    if (cnt[q]) { atomicAdd(&blk[6 + X * 2 + 0], own[q]); atomicAdd(&blk[6 + X * 2 + 1], total - own[q]); }
             if (loc_sum) atomicAdd(&blk[X * 2 + 0], loc_sum);
             if (rem_sum) atomicAdd(&blk[X * 2 + 1], rem_sum);
         }
@@ -219,17 +222,19 @@ __global__ void __launch_bounds__(kWalkThreads) traffic_walk_kernel(TrafficParam
                     rem += __shfl_xor_sync(0xffffffffu, rem, s);
                 }
                 if (lane == 0) {
-                    p.per_cta[t * 6 + 4] = loc;
-                    p.per_cta[t * 6 + 5] = rem;
+                    if (p.per_cta) { p.per_cta[t * 6 + 4] = loc; p.per_cta[t * 6 + 5] = rem; }
                     atomicAdd(&blk[4], loc);
                     atomicAdd(&blk[5], rem);
+                    atomicAdd(&blk[10], loc);                 // every output element is written once either way
+                    atomicAdd(&blk[11], rem);
                 }
             }
         }
     }
     if (CLASSIFY) {
         __syncthreads();
-        if (tid < 6 && blk[tid]) atomicAdd(reinterpret_cast<unsigned long long*>(p.totals) + tid, blk[tid]);
+        if (tid < 6 && blk[tid] && p.totals) atomicAdd(reinterpret_cast<unsigned long long*>(p.totals) + tid, blk[tid]);
+        if (tid >= 6 && tid < 12 && blk[tid] && p.totals_l2) atomicAdd(reinterpret_cast<unsigned long long*>(p.totals_l2) + (tid - 6), blk[tid]);
     }
 }
 
@@ -362,5 +367,33 @@ extern "C" ccl_status ccl_traffic(const ccl_traffic_desc* d, const int32_t* cta_
             CCL_CUDA_TRY(cudaGetLastError());
         }
     }
+    return CCL_OK;
+}
+
+extern "C" ccl_status ccl_traffic_l2(const ccl_traffic_desc* d, const int32_t* cta_chiplet_dev, uint64_t* totals_l2_dev,
+                                     void* cuda_stream) {
+    TrafficParams p;
+    ccl_status s = fill_params(d, &p);
+    if (s) return s;
+    if (!totals_l2_dev) return fail(CCL_ERR_INVALID_ARG, "ccl_traffic_l2: totals_l2_dev is required");
+    if (d->assign == CCL_ASSIGN_EXPLICIT && !cta_chiplet_dev) return fail(CCL_ERR_INVALID_ARG, "ccl_traffic_l2: explicit assignment needs cta_chiplet_dev");
+    for (int X = 0; X < 3; ++X)
+        if (p.place[X] == CCL_PLACE_BEST) return fail(CCL_ERR_UNSUPPORTED, "ccl_traffic_l2: CCL_PLACE_BEST is not supported here (use a fixed placement)");
+    p.q = cta_chiplet_dev; p.totals_l2 = totals_l2_dev;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    int dev, sms;
+    CCL_CUDA_TRY(cudaGetDevice(&dev));
+    CCL_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    ZeroSeg z;
+    std::memset(&z, 0, sizeof(z));
+    z.p[0] = totals_l2_dev; z.n[0] = 6;
+    traffic_prep_kernel<<<1, 32, 0, st>>>(z);
+    count_launch();
+    CCL_CUDA_TRY(cudaGetLastError());
+    const int64_t nblocks = p.tiles_m + p.tiles_n + (p.ntiles + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    if (nblocks >= (INT64_C(1) << 31)) return fail(CCL_ERR_UNSUPPORTED, "ccl_traffic_l2: too many tiles");
+    traffic_walk_kernel<false, true><<<(unsigned)nblocks, kWalkThreads, 0, st>>>(p);
+    count_launch();
+    CCL_CUDA_TRY(cudaGetLastError());
     return CCL_OK;
 }

@@ -112,7 +112,12 @@ def traffic_remote(g, layout_bc, place_bc, S, assign, align=0):
         ow = [torch.empty((pages[x],), dtype=torch.uint8, device="cuda") for x in range(3)]
     ms_t = timed(lambda: ccl.ccl_traffic(td, per_cta, totals, pp, ow), 3, 1)
     t = totals.cpu()
-    return dict(remote=[int(x) for x in t[:, 1]], total=int(t.sum()), ms=ms_t)
+    out = dict(remote=[int(x) for x in t[:, 1]], total=int(t.sum()), ms=ms_t)
+    if place_bc != ccl.PLACE_BEST:            # the same policy behind an ideal private L2 per chiplet
+        l2 = torch.empty((3, 2), dtype=torch.int64, device="cuda")
+        ccl.ccl_traffic_l2(td, l2)
+        out["remote_ideal_l2"] = [int(x) for x in l2.cpu()[:, 1]]
+    return out
 
 
 def run_gemm(g, pk, reps):
@@ -179,8 +184,11 @@ def run_gemm(g, pk, reps):
         pol[tag] = best
         if tag == "row_rr4k":
             base = sum(best["remote"])
+    base_l2 = sum(pol["row_rr4k"]["remote_ideal_l2"])
     for tag, r in pol.items():
         r["ratio_vs_rr4k"] = (sum(r["remote"]) / base) if base else None
+        if "remote_ideal_l2" in r:
+            r["ratio_vs_rr4k_ideal_l2"] = (sum(r["remote_ideal_l2"]) / base_l2) if base_l2 else None
     res["traffic"] = pol
     return res
 
@@ -209,7 +217,8 @@ def main():
                   f"remote/rr4k: rr64k {t['row_rr64k']['ratio_vs_rr4k']:.3f} rr2m {t['row_rr2m']['ratio_vs_rr4k']:.3f} "
                   f"block {t['row_block']['ratio_vs_rr4k']:.3f} best {t['row_best']['ratio_vs_rr4k']:.3f} "
                   f"CCL {t['ccl_block']['ratio_vs_rr4k']:.3f} ({t['ccl_block']['partition']}) ccl+rr {t['ccl_rr']['ratio_vs_rr4k']:.3f} "
-                  f"interleaved-CCL+rr {t['ileave_rr']['ratio_vs_rr4k']:.3f}", flush=True)
+                  f"interleaved-CCL+rr {t['ileave_rr']['ratio_vs_rr4k']:.3f} | behind an ideal L2: block {t['row_block']['ratio_vs_rr4k_ideal_l2']:.3f} "
+                  f"CCL {t['ccl_block']['ratio_vs_rr4k_ideal_l2']:.3f} interleaved-CCL+rr {t['ileave_rr']['ratio_vs_rr4k_ideal_l2']:.3f}", flush=True)
         json.dump(dict(config=cfg, peaks=pk, gemms=rows), open(os.path.join(args.out, f"report_config{cfg}.json"), "w"), indent=1)
         nz = [r["traffic"]["ccl_block"]["ratio_vs_rr4k"] for r in rows if r["traffic"]["ccl_block"]["ratio_vs_rr4k"]]
         if nz:

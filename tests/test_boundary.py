@@ -23,7 +23,7 @@ def built():
 def test_exports_match_header():
     hdr = open(os.path.join(ROOT, "include", "ccl.h")).read()
     hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
-    declared = sorted(set(re.findall(r"\b(ccl_[a-z_]+)\s*\(", hdr)))
+    declared = sorted(set(re.findall(r"\b(ccl_[a-z0-9_]+)\s*\(", hdr)))
     assert declared == sorted(ccl.EXPORTS)
     l = ccl.lib()
     for name in declared:
