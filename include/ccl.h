@@ -66,7 +66,8 @@ typedef enum { CCL_PART_NONE = 0, CCL_PART_ROWS = 1, CCL_PART_COLS = 2 } ccl_par
  *       strip's chunk j = o*e / S, and chunk j of strip g is stored as chunk j*P + g of the buffer:
  *       byte offset = (j*P + g)*S + (o*e mod S).  The buffer holds ceil(strip bytes / S)*P chunks;
  *       the tail of every strip's last chunk is padding.  ccl_strip_stride is not defined for it.
- *       ccl_gemm does not take this layout yet (CCL_ERR_UNSUPPORTED); map, repack and traffic do.
+ *       Map, repack and traffic take every such layout; ccl_gemm takes those whose chunks line up with the
+ *       strip rows (see ccl_gemm).
  *   A CCL layout with part = CCL_PART_NONE behaves as CCL_ROWMAJOR.
  * Requirements: rows, cols > 0; elem_bytes in {1,2,4}; P >= 1; the split dimension
  * divisible by P (else CCL_ERR_SHAPE); strip_align_bytes >= 0 and a multiple of e.
@@ -117,6 +118,12 @@ ccl_status ccl_repack(const ccl_mat* m, const void* src_dev, void* dst_dev, int 
  * Requirements (else CCL_ERR_UNSUPPORTED / CCL_ERR_ALIGN, nothing launched): elem_bytes = 2;
  * every contiguous extent a tile row lives in (cols, or w for CCL_PART_COLS) a multiple of 8
  * elements; strip strides multiples of 16 bytes; base pointers 16-byte aligned.
+ * A CCL_CCL_INTERLEAVED operand is taken when its chunks line up with its strip rows, so that a tile is an
+ * affine box of the buffer: either a chunk holds a power-of-two number of whole strip rows, or a strip row is
+ * made of whole chunks of a multiple of 64 elements; the chunk size a multiple of 16 bytes.  (With chunks of
+ * whole rows, an operand whose rows run along K must have K a multiple of 64 or rows-per-strip a multiple of
+ * the rows per chunk: the padding of a strip's last chunk is not read as zero.)  Other chunkings ->
+ * CCL_ERR_UNSUPPORTED.
  */
 typedef struct ccl_gemm_desc {
     int64_t M, N, K;

@@ -2,10 +2,11 @@
 // Chiplet-Contiguous Layout (Sec. 2.2 execution model; Sec. 3.3: only the address map changes).
 //
 // Design (sm_100a):
-//   * CCL is folded into rank-3 TMA tensor maps {strip-local contiguous extent, rows, strip}
+//   * CCL is folded into TMA tensor maps {strip-local contiguous extent, rows, strip, 1}
 //     -- the view (K, G, N/G) with strides (w, K*w, 1) of Sec. 3.3 -- so the address
 //     translation costs nothing per access and a partial last tile of a strip is handled by
-//     TMA zero fill.
+//     TMA zero fill.  The page-interleaved form of CCL uses the fourth dimension: the chunk
+//     index (chunks of whole rows) or the chunk within a row (rows of whole chunks).
 //   * Persistent, warp-specialised CTAs: warp 0 = TMA producer, warp 1 = tcgen05.mma issuer
 //     (one elected thread) and TMEM owner, warps 2-5 = epilogue (TMEM -> registers -> bf16 ->
 //     global, addressing C through its own layout).
@@ -45,6 +46,11 @@ __device__ int g_gemm_status = 0;
 struct OpMap {          // how stored coordinates (r, c) of an operand become tensor-map coordinates
     int32_t split;      // 0 none, 1 rows, 2 cols
     int32_t w, h;       // strip width (split 2) / strip height (split 1)
+    // page-interleaved CCL (chunk of il_sc elements; chunk j of strip g stored as chunk j*P + g):
+    //   il_mode 1: a chunk holds il_kr whole strip rows  -> map {x, row % kr, strip, row / kr}
+    //   il_mode 2: a strip row spans whole chunks        -> map {x % sc, x / sc, row, strip}
+    //   il_mode 0: strips stored one after the other     -> map {x, row, strip, 1}
+    int32_t il_mode, il_kr, il_sc;
 };
 
 struct GemmParams {
@@ -57,8 +63,9 @@ struct GemmParams {
     int32_t panel;                  // m-tiles per raster panel
     OpMap a, b;
     int32_t a_mn, b_mn;             // 1 = MN-major operand tile in shared memory
+    OpMap c;                        // C addressed through its own map as well (TMA tile stores)
     int32_t c_split;
-    int64_t c_w, c_h, c_stride, c_cols;
+    int64_t c_w, c_h, c_stride, c_cols, c_ichunk, c_nstrips;
     uint16_t* C;
     uint32_t idesc;
     int32_t stages;
@@ -122,13 +129,17 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
 // TMA tile load whose completion bytes are credited to `bar_addr` (a shared::cluster address; with two
 // CTAs this is the leader's barrier, which the cta_group::2 form of the copy is allowed to signal).
 template <int CTAS>
-__device__ __forceinline__ void tma_load(void* smem_dst, const CUtensorMap* map, uint32_t bar_addr, int c0, int c1, int c2) {
+__device__ __forceinline__ void tma_load(void* smem_dst, const CUtensorMap* map, uint32_t bar_addr, int c0, int c1, int c2, int c3) {
     if (CTAS == 1)
-        asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-                     ::"r"(smem_u32(smem_dst)), "l"(map), "r"(bar_addr), "r"(c0), "r"(c1), "r"(c2) : "memory");
+        asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+                     ::"r"(smem_u32(smem_dst)), "l"(map), "r"(bar_addr), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
     else
-        asm volatile("cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-                     ::"r"(smem_u32(smem_dst)), "l"(map), "r"(bar_addr), "r"(c0), "r"(c1), "r"(c2) : "memory");
+        asm volatile("cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+                     ::"r"(smem_u32(smem_dst)), "l"(map), "r"(bar_addr), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, const void* smem_src, int c0, int c1, int c2, int c3) {
+    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+                 ::"l"(map), "r"(smem_u32(smem_src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
 }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile(
@@ -151,10 +162,24 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint3
     return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) | (1ull << 46) | (2ull << 61);
 }
 
-__device__ __forceinline__ void to_coords(const OpMap& o, int r, int c, int& x, int& y, int& z) {
-    if (o.split == 2) { z = c / o.w; x = c - z * o.w; y = r; }
-    else if (o.split == 1) { z = r / o.h; y = r - z * o.h; x = c; }
-    else { x = c; y = r; z = 0; }
+// Stored coordinates (r, c) of an operand -> coordinates of its rank-4 tensor map.
+__device__ __forceinline__ void to_coords(const OpMap& o, int r, int c, int& x, int& y, int& z, int& u) {
+    int g, rr, xx;                                   // strip, row inside the strip, column inside the strip row
+    if (o.split == 2) { g = c / o.w; xx = c - g * o.w; rr = r; }
+    else if (o.split == 1) { g = r / o.h; rr = r - g * o.h; xx = c; }
+    else { g = 0; rr = r; xx = c; }
+    if (o.il_mode == 1) { u = rr / o.il_kr; y = rr - u * o.il_kr; x = xx; z = g; }
+    else if (o.il_mode == 2) { y = xx / o.il_sc; x = xx - y * o.il_sc; z = rr; u = g; }
+    else { x = xx; y = rr; z = g; u = 0; }
+}
+// Element offset of C[m][n] in its buffer (any layout).
+__device__ __forceinline__ int64_t c_offset(const GemmParams& p, int64_t m, int64_t n) {
+    int64_t g = 0, o;
+    if (p.c_split == 2) { g = n / p.c_w; o = m * p.c_w + (n - g * p.c_w); }
+    else if (p.c_split == 1) { g = m / p.c_h; o = (m - g * p.c_h) * p.c_cols + n; }
+    else o = m * p.c_cols + n;
+    if (p.c_ichunk) { const int64_t j = o / p.c_ichunk; return (j * p.c_nstrips + g) * p.c_ichunk + (o - j * p.c_ichunk); }
+    return g * p.c_stride + o;
 }
 
 struct TileCoord { int m0, m1, n0, n1, split; };
@@ -268,7 +293,8 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         const bool mn = isA ? p.a_mn != 0 : p.b_mn != 0;
         // K runs along the tensor map's x for a K-contiguous operand and along y otherwise; unless the
         // operand is split along K itself (rare) only that coordinate changes from one k block to the next
-        const bool ksplit = mn ? om.split == 1 : om.split == 2;
+        // (a page-interleaved operand recomputes its coordinates every k block as well)
+        const bool ksplit = (mn ? om.split == 1 : om.split == 2) || om.il_mode != 0;
         uint32_t soff;                                        // byte offset of the box inside a stage
         int off;                                              // offset of the box along M (A) or N (B) from the tile origin
         if (isA) { soff = mn ? (uint32_t)bi * (64 * BK * 2) : 0u; off = (int)rank * BM + (mn ? 64 * bi : 0); }
@@ -281,8 +307,8 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         bool ok = true;
         for (int it = 0; ok && sched.get(it, t); ++it) {
             const int base = (isA ? t.m0 : t.n0) + off;
-            int x, y, z;
-            if (mn) to_coords(om, 0, base, x, y, z); else to_coords(om, base, 0, x, y, z);
+            int x, y, z, u;
+            if (mn) to_coords(om, 0, base, x, y, z, u); else to_coords(om, base, 0, x, y, z, u);
             const int kb0 = t.split * p.kb_per_split, kb1 = min(p.num_kb, kb0 + p.kb_per_split);
             for (int kb = kb0; kb < kb1; ++kb) {
                 ok = mbar_wait_bounded(&empty[stage], phase ^ 1);
@@ -291,9 +317,9 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 if (lane == 0 && leader) mbar_expect_tx(&full[stage], p.stage_bytes * CTAS);
                 __syncwarp();
                 const int k0 = kb * BK;
-                if (ksplit) { if (mn) to_coords(om, k0, base, x, y, z); else to_coords(om, base, k0, x, y, z); }
+                if (ksplit) { if (mn) to_coords(om, k0, base, x, y, z, u); else to_coords(om, base, k0, x, y, z, u); }
                 else if (mn) y = k0; else x = k0;
-                if (active) tma_load<CTAS>(smem + (size_t)stage * p.stage_bytes + soff, map, full0 + (uint32_t)stage * 8u, x, y, z);
+                if (active) tma_load<CTAS>(smem + (size_t)stage * p.stage_bytes + soff, map, full0 + (uint32_t)stage * 8u, x, y, z, u);
                 if (++stage == p.stages) { stage = 0; phase ^= 1; }
             }
         }
@@ -365,14 +391,10 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             else row_base = (int64_t)m * p.c_cols;
             const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)acc * 256u;
             // Full 32-row x 64-column pieces go through shared memory (128-byte swizzle) and a TMA tile store
-            // addressed through C's own rank-3 map; ragged pieces (tile clipped by a strip or the matrix edge)
+            // addressed through C's own tensor map; ragged pieces (tile clipped by a strip or the matrix edge)
             // and split-K partial sums are stored from registers.
             const int row0 = t.m0 + (int)rank * BM + quad * 32;
             const bool rows_full = row0 + 32 <= t.m1;
-            int cy, cz, cx0;                                 // C map coordinates of (row0, nb)
-            if (p.c_split == 2) { cz = nb / (int)p.c_w; cx0 = nb - cz * (int)p.c_w; cy = row0; }
-            else if (p.c_split == 1) { cz = row0 / (int)p.c_h; cy = row0 - cz * (int)p.c_h; cx0 = nb; }
-            else { cz = 0; cy = row0; cx0 = nb; }
             // One 64-column piece: registers -> C.  `r` holds 64 fp32 accumulators of this thread's row.
             auto store_piece = [&](const uint32_t (&r)[64], int c) {
                 const int n64 = nb + c * 64;
@@ -391,7 +413,12 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     }
                     fence_proxy_async();
                     __syncwarp();
-                    if (lane == 0) { tma_store_3d(&map_c, buf, cx0 + c * 64, cy, cz); tma_store_commit(); }
+                    if (lane == 0) {
+                        int cx, cy, cz, cu;                      // C map coordinates of (row0, n64)
+                        to_coords(p.c, row0, n64, cx, cy, cz, cu);
+                        tma_store_4d(&map_c, buf, cx, cy, cz, cu);
+                        tma_store_commit();
+                    }
                     ++epi_count;
                     return;
                 }
@@ -420,7 +447,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                                 hh = __floats2bfloat162_rn(__uint_as_float(rr[j * 8 + 2]), __uint_as_float(rr[j * 8 + 3])); v.y = *reinterpret_cast<uint32_t*>(&hh);
                                 hh = __floats2bfloat162_rn(__uint_as_float(rr[j * 8 + 4]), __uint_as_float(rr[j * 8 + 5])); v.z = *reinterpret_cast<uint32_t*>(&hh);
                                 hh = __floats2bfloat162_rn(__uint_as_float(rr[j * 8 + 6]), __uint_as_float(rr[j * 8 + 7])); v.w = *reinterpret_cast<uint32_t*>(&hh);
-                                *reinterpret_cast<uint4*>(p.C + row_base + n) = v;
+                                *reinterpret_cast<uint4*>(p.C + (p.c_ichunk ? c_offset(p, m, n) : row_base + n)) = v;
                             }
                         }
                     }
@@ -481,10 +508,7 @@ __global__ void __launch_bounds__(256) splitk_reduce_kernel(const GemmParams p) 
             acc[0] += x.x; acc[1] += x.y; acc[2] += x.z; acc[3] += x.w;
             acc[4] += y.x; acc[5] += y.y; acc[6] += y.z; acc[7] += y.w;
         }
-        int64_t off;
-        if (p.c_split == 2) { int64_t g = n / p.c_w; off = g * p.c_stride + m * p.c_w + (n - g * p.c_w); }
-        else if (p.c_split == 1) { int64_t g = m / p.c_h; off = g * p.c_stride + (m - g * p.c_h) * p.c_cols + n; }
-        else off = m * p.c_cols + n;
+        const int64_t off = c_offset(p, m, n);
         uint4 v;
         __nv_bfloat162 h;
         h = __floats2bfloat162_rn(acc[0], acc[1]); v.x = *reinterpret_cast<uint32_t*>(&h);
@@ -507,12 +531,38 @@ struct GemmPlan {
     unsigned grid;
 };
 
-static ccl_status check_operand(const MatView& v, const void* ptr, const char* name) {
+// How a page-interleaved operand is expressed as a rank-4 tensor map (OpMap::il_mode): 0 = not interleaved,
+// 1 = a chunk holds *kr whole strip rows, 2 = a strip row spans whole chunks, -1 = neither (no affine map exists).
+static int interleave_mode(const MatView& v, int64_t* kr) {
+    *kr = 0;
+    if (!v.ichunk) return 0;
+    const int64_t row = v.split == 2 ? v.w : v.cols;
+    if (v.ichunk % row == 0) { *kr = v.ichunk / row; return 1; }
+    if (row % v.ichunk == 0 && v.ichunk % 64 == 0) return 2;
+    return -1;
+}
+
+// k_along_rows: the GEMM's K dimension runs along the stored rows of this operand (never for C)
+static ccl_status check_operand(const MatView& v, const void* ptr, const char* name, bool k_along_rows, int64_t K) {
     if (v.e != 2) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: %s: only 2-byte (bf16) elements are supported", name);
-    if (v.ichunk) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: %s: the page-interleaved layout is not supported by the GEMM yet", name);
     int64_t inner = v.split == 2 ? v.w : v.cols;
     if (inner % 8) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: %s: contiguous extent %lld is not a multiple of 8 elements", name, (long long)inner);
-    if (v.split && (v.stride * v.e) % 16) return fail(CCL_ERR_ALIGN, "ccl_gemm: %s: strip stride is not a multiple of 16 bytes", name);
+    if (v.ichunk) {
+        int64_t kr;
+        const int mode = interleave_mode(v, &kr);
+        if (mode < 0)
+            return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: %s: page-interleaved layout: a chunk (%lld elements) must hold whole strip rows (%lld elements), "
+                        "or a strip row whole chunks of a multiple of 64 elements", name, (long long)v.ichunk, (long long)inner);
+        if (mode == 1 && (kr & (kr - 1)))
+            return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: %s: page-interleaved layout: %lld strip rows per chunk is not a power of two", name, (long long)kr);
+        const int64_t R = v.split == 1 ? v.h : v.rows;
+        // rows past the strip's end inside its last chunk are padding, not zeros: a ragged K tail must not read them
+        if (mode == 1 && k_along_rows && K % BK && R % kr)
+            return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: %s: page-interleaved layout: K (%lld) is not a multiple of %d and ends inside a chunk", name, (long long)K, BK);
+        if ((v.ichunk * v.e) % 16) return fail(CCL_ERR_ALIGN, "ccl_gemm: %s: chunk size is not a multiple of 16 bytes", name);
+        if ((double)v.nstrips * (double)std::max(v.ichunk, inner) * v.e >= (double)(INT64_C(1) << 40))
+            return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: %s: extent too large for a tensor map", name);
+    } else if (v.split && (v.stride * v.e) % 16) return fail(CCL_ERR_ALIGN, "ccl_gemm: %s: strip stride is not a multiple of 16 bytes", name);
     if (ptr && (reinterpret_cast<uintptr_t>(ptr) & 15)) return fail(CCL_ERR_ALIGN, "ccl_gemm: %s: base pointer is not 16-byte aligned", name);
     if (v.rows >= (INT64_C(1) << 31) || v.cols >= (INT64_C(1) << 31) || v.stride * v.e >= (INT64_C(1) << 40))
         return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: %s: extent too large for a tensor map", name);
@@ -550,9 +600,13 @@ static ccl_status make_plan(const ccl_gemm_desc* d, const void* A, const void* B
     int64_t ar = at ? d->K : d->M, ac = at ? d->M : d->K, br = bt ? d->N : d->K, bc = bt ? d->K : d->N;
     if (va.rows != ar || va.cols != ac || vb.rows != br || vb.cols != bc || vc.rows != d->M || vc.cols != d->N)
         return fail(CCL_ERR_SHAPE, "ccl_gemm: operand shapes do not match M, N, K and the transpose flags");
-    if ((s = check_operand(va, A, "A"))) return s;
-    if ((s = check_operand(vb, B, "B"))) return s;
-    if ((s = check_operand(vc, C, "C"))) return s;
+    if ((s = check_operand(va, A, "A", at, d->K))) return s;
+    if ((s = check_operand(vb, B, "B", !bt, d->K))) return s;
+    if ((s = check_operand(vc, C, "C", false, d->K))) return s;
+    int64_t kr_a, kr_b, kr_c;
+    const int il_a = interleave_mode(va, &kr_a), il_b = interleave_mode(vb, &kr_b), il_c = interleave_mode(vc, &kr_c);
+    // a 192-row box of a K-contiguous B cannot be cut into chunks of more than 64 rows
+    const bool no_192 = il_b == 1 && bt && kr_b > 64;
 
     // strips along M, N (tiles must not straddle them) and along K (a 64-wide k block must not)
     int64_t Wm = 0, Wn = 0;
@@ -597,6 +651,7 @@ static ccl_status make_plan(const ccl_gemm_desc* d, const void* A, const void* B
         for (int b : {512, 256, 192, 128}) {
             if (c == 1 && b == 512) continue;
             if (c == 2 && b == 192) continue;
+            if (b == 192 && no_192) continue;
             if (force_bn && atoi(force_bn) != b) continue;
             const int64_t tiles = strips_m * ((Wm + BM * c - 1) / (BM * c)) * strips_n * ((Wn + b - 1) / b);
             const double t_kb = std::max((double)b / 256.0 * 512.0, (128.0 + (double)b / c) * 2.56);
@@ -630,7 +685,12 @@ static ccl_status make_plan(const ccl_gemm_desc* d, const void* A, const void* B
     p.a.split = va.split; p.a.w = (int32_t)va.w; p.a.h = (int32_t)va.h;
     p.b.split = vb.split; p.b.w = (int32_t)vb.w; p.b.h = (int32_t)vb.h;
     p.a_mn = at ? 1 : 0; p.b_mn = bt ? 0 : 1;
+    p.a.il_mode = il_a; p.a.il_kr = (int32_t)std::max<int64_t>(kr_a, 1); p.a.il_sc = (int32_t)std::max<int64_t>(va.ichunk, 1);
+    p.b.il_mode = il_b; p.b.il_kr = (int32_t)std::max<int64_t>(kr_b, 1); p.b.il_sc = (int32_t)std::max<int64_t>(vb.ichunk, 1);
+    p.c.split = vc.split; p.c.w = (int32_t)vc.w; p.c.h = (int32_t)vc.h;
+    p.c.il_mode = il_c; p.c.il_kr = (int32_t)std::max<int64_t>(kr_c, 1); p.c.il_sc = (int32_t)std::max<int64_t>(vc.ichunk, 1);
     p.c_split = vc.split; p.c_w = vc.w; p.c_h = vc.h; p.c_stride = vc.stride; p.c_cols = vc.cols;
+    p.c_ichunk = vc.ichunk; p.c_nstrips = vc.nstrips;
     // instruction descriptor: D = f32, A = B = bf16, operand majors, N >> 3, M >> 4 (M spans the CTA pair)
     p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)p.a_mn << 15) | ((uint32_t)p.b_mn << 16) |
               ((uint32_t)(subn >> 3) << 17) | ((uint32_t)(bm >> 4) << 24);
@@ -663,14 +723,38 @@ static ccl_status make_plan(const ccl_gemm_desc* d, const void* A, const void* B
     return CCL_OK;
 }
 
-// tensor map of an operand: {contiguous extent, rows (per strip), strips}
+// Rank-4 tensor map of an operand (coordinates as to_coords() produces them), for boxes of box_inner contiguous
+// elements by box_rows strip rows:
+//   strips one after the other : {strip row extent, rows per strip, strips, 1}
+//   interleaved, mode 1        : {strip row extent, rows per chunk kr, strips, chunk index}; a box of more than kr
+//                                rows takes kr rows from each of box_rows / kr consecutive chunks of its strip
+//   interleaved, mode 2        : {chunk extent, chunks per strip row, rows per strip, strips}
 static ccl_status operand_tmap(CUtensorMap* m, const MatView& v, const void* base, uint32_t box_inner, uint32_t box_rows) {
-    uint64_t dims[3], strides[2];
-    if (v.split == 2) { dims[0] = v.w; dims[1] = v.rows; dims[2] = v.nstrips; strides[0] = v.w * 2; strides[1] = v.stride * 2; }
-    else if (v.split == 1) { dims[0] = v.cols; dims[1] = v.h; dims[2] = v.nstrips; strides[0] = v.cols * 2; strides[1] = v.stride * 2; }
-    else { dims[0] = v.cols; dims[1] = v.rows; dims[2] = 1; strides[0] = v.cols * 2; strides[1] = v.cols * 2 * v.rows; }
-    uint32_t box[3] = {box_inner, box_rows, 1};
-    return encode_tmap(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B);
+    const uint64_t row = (uint64_t)(v.split == 2 ? v.w : v.cols);      // elements of a strip row
+    const uint64_t R = (uint64_t)(v.split == 1 ? v.h : v.rows);        // rows per strip
+    const uint64_t S = (uint64_t)v.nstrips, sc = (uint64_t)v.ichunk;
+    uint64_t dims[4], strides[3];
+    uint32_t box[4];
+    int64_t kr;
+    const int mode = interleave_mode(v, &kr);
+    if (mode == 1) {
+        const uint64_t k = (uint64_t)kr;
+        dims[0] = row; dims[1] = k; dims[2] = S; dims[3] = (R + k - 1) / k;
+        strides[0] = row * 2; strides[1] = sc * 2; strides[2] = S * sc * 2;
+        if (box_rows <= k) { if (k % box_rows) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: a %u-row box does not divide a chunk of %llu rows", box_rows, (unsigned long long)k); }
+        else if (box_rows % k) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: a %u-row box is not made of whole chunks of %llu rows", box_rows, (unsigned long long)k);
+        box[0] = box_inner; box[2] = 1;
+        if (box_rows <= k) { box[1] = box_rows; box[3] = 1; } else { box[1] = (uint32_t)k; box[3] = box_rows / (uint32_t)k; }
+    } else if (mode == 2) {
+        dims[0] = sc; dims[1] = row / sc; dims[2] = R; dims[3] = S;
+        strides[0] = S * sc * 2; strides[1] = row * S * 2; strides[2] = sc * 2;
+        box[0] = box_inner; box[1] = 1; box[2] = box_rows; box[3] = 1;
+    } else if (mode == 0) {
+        dims[0] = row; dims[1] = R; dims[2] = v.split ? S : 1; dims[3] = 1;
+        strides[0] = row * 2; strides[1] = v.split ? (uint64_t)v.stride * 2 : row * 2; strides[2] = strides[1];
+        box[0] = box_inner; box[1] = box_rows; box[2] = 1; box[3] = 1;
+    } else return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: this page-interleaved layout has no tensor map");
+    return encode_tmap(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
 template <int BN, int CTAS>

@@ -47,7 +47,8 @@ def traffic_pair(M, N, K, P, S, lay=("row", "row", "row"), place=(0, 0, 0), a_tr
 
 
 def gemm_desc(M, N, K, P=1, lay=("row", "row", "row"), a_trans=0, b_trans=0, out_part=2, grouped=1, align=0, parts=None):
-    """Library GEMM descriptor; lay[X] == "ccl" stores operand X in CCL split as `parts` says
+    """Library GEMM descriptor; lay[X] == "ccl" ("ileave": page-interleaved CCL with chunks of `align` bytes) stores
+    operand X in CCL split as `parts` says
     (default: the split an N- or M-partition of C implies)."""
     if parts is None:
         parts = m_split_parts(a_trans, b_trans) if out_part == 1 else n_split_parts(a_trans, b_trans)
@@ -56,8 +57,9 @@ def gemm_desc(M, N, K, P=1, lay=("row", "row", "row"), a_trans=0, b_trans=0, out
     d.M, d.N, d.K = M, N, K
     mats = []
     for X in range(3):
-        is_ccl = lay[X] == "ccl" and parts[X] != 0
-        mats.append(ccl.Mat(shapes[X][0], shapes[X][1], 2, P, parts[X] if is_ccl else 0, 1 if is_ccl else 0, align if is_ccl else 0))
+        is_ccl = lay[X] in ("ccl", "ileave") and parts[X] != 0
+        layout = (2 if lay[X] == "ileave" else 1) if is_ccl else 0
+        mats.append(ccl.Mat(shapes[X][0], shapes[X][1], 2, P, parts[X] if is_ccl else 0, layout, align if is_ccl else 0))
     d.A, d.B, d.C = mats
     d.a_trans, d.b_trans, d.out_part, d.P, d.grouped_raster = a_trans, b_trans, out_part, P, grouped
     return d

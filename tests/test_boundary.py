@@ -142,9 +142,11 @@ def test_gemm_rejects_bad_input_before_any_launch():
     assert gemm_rc(d) == ccl.ERR_UNSUPPORTED
     d = gemm_desc(128, 256, 64, 3, ("row", "row", "row"))
     assert gemm_rc(d) == ccl.ERR_SHAPE                                                               # N % P with a grouped raster
-    d = gemm_desc(128, 256, 64, 2, ("row", "ccl", "ccl"), align=4096)
-    d.B.layout = 2                                                                                   # page-interleaved operand
-    assert gemm_rc(d) == ccl.ERR_UNSUPPORTED
+    # page-interleaved operands: chunks must line up with the strip rows (w = 96 elements = 192 bytes here)
+    assert gemm_rc(gemm_desc(128, 192, 64, 2, ("row", "ileave", "ccl"), align=256)) == ccl.ERR_UNSUPPORTED    # neither divides
+    assert gemm_rc(gemm_desc(128, 192, 64, 2, ("row", "ileave", "ccl"), align=576)) == ccl.ERR_UNSUPPORTED    # 3 rows per chunk
+    assert gemm_rc(gemm_desc(128, 192, 64, 2, ("row", "ccl", "ileave"), align=64)) == ccl.ERR_UNSUPPORTED     # 3 chunks of 32 elements
+    assert gemm_rc(gemm_desc(128, 512, 72, 2, ("row", "ileave", "ccl"), align=8192)) == ccl.ERR_UNSUPPORTED   # K tail ends inside a chunk
     d = gemm_desc(128, 256, 64)
     d.out_part = 7
     assert gemm_rc(d) == ccl.ERR_INVALID_ARG

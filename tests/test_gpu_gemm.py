@@ -108,6 +108,36 @@ def test_gemm_small_shapes(M, N, K, P, lay, at, bt, op, cta_mode):
         check(d, A, B)
 
 
+INTERLEAVED = [
+    # M, N, K, P, layouts(A,B,C), a_trans, b_trans, out_part, chunk bytes
+    (130, 384, 96, 2, ("row", "ileave", "ileave"), 0, 0, 2, 1536),      # w = 192: 4 strip rows per chunk
+    (130, 384, 96, 4, ("row", "ileave", "ileave"), 0, 0, 2, 768),       # w = 96: ragged tiles inside every strip, 4 rows per chunk
+    (264, 1024, 328, 4, ("row", "ileave", "ileave"), 0, 0, 2, 256),     # w = 256: a strip row is 2 chunks
+    (264, 1024, 328, 4, ("row", "ileave", "ileave"), 1, 0, 2, 128),     # ... 4 chunks of 64 elements
+    (264, 1024, 328, 4, ("row", "ileave", "ileave"), 0, 0, 2, 512),     # a chunk is exactly one strip row
+    (200, 512, 256, 4, ("row", "ileave", "ileave"), 0, 1, 2, 4096),     # B stored [N x K]: 8 of its rows per chunk; 16 rows of C
+    (520, 1024, 256, 2, ("row", "ileave", "ileave"), 0, 1, 2, 65536),   # 128 B rows per chunk for B, 64 for C
+    (512, 512, 256, 4, ("ileave", "row", "ileave"), 0, 0, 1, 2048),     # M-partition: A and C split along rows
+    (512, 512, 256, 2, ("ileave", "row", "ileave"), 1, 0, 1, 256),      # A stored [K x M], split along its columns (w = 256)
+    (512, 512, 192, 2, ("ileave", "row", "ileave"), 1, 0, 1, 2048),     # ... 4 rows of A per chunk, 2 rows of C
+    (16, 1024, 2048, 2, ("row", "ileave", "ileave"), 0, 0, 2, 4096),    # split along K: the reduction writes interleaved C
+    (640, 2560, 512, 2, ("row", "ileave", "ileave"), 0, 0, 2, 10240),   # several tiles per CTA group, 4 rows per chunk
+    (256, 4096, 512, 4, ("row", "ileave", "ileave"), 0, 0, 2, 4096),    # the common case: 4 KB pages, 2 KB strip rows
+]
+
+
+@pytest.mark.parametrize("M,N,K,P,lay,at,bt,op,chunk", INTERLEAVED)
+def test_gemm_page_interleaved_operands(M, N, K, P, lay, at, bt, op, chunk, cta_mode):
+    """The page-interleaved form of CCL changes the address map only: same bits as from packed CCL operands."""
+    A, B = synth.gemm_operands(M, N, K, at, bt, seed=5, tag="ileave")
+    plain = tuple("ccl" if l == "ileave" else l for l in lay)
+    want = run_gemm(gemm_desc(M, N, K, P, plain, at, bt, op, 1), A, B)
+    for grouped in (1, 0):
+        d = gemm_desc(M, N, K, P, lay, at, bt, op, grouped, align=chunk)
+        got, _ = check(d, A, B)
+        np.testing.assert_array_equal(got, want)
+
+
 def test_gemm_exact_cases():
     eye = synth.from_bits(synth.bits(torch.eye(256).to(torch.bfloat16)))
     A = synth.randn_bf16(200, 256, 1.0, 0, "eye")
