@@ -43,14 +43,52 @@ constexpr uint32_t kEpiBytes = 4 * 2 * 32 * 128; // epilogue staging: per warp t
 
 __device__ int g_gemm_status = 0;
 
+#ifdef CCL_GEMM_TRACE   // development aid: per-CTA timestamps of the kernel's phases (not compiled into the library)
+__device__ unsigned long long g_trace[296][32];
+#define CCL_TRACE(slot) do { g_trace[blockIdx.x][slot] = global_timer_ns(); g_trace[blockIdx.x][16 + (slot)] = (unsigned long long)clock64(); } while (0)
+__device__ unsigned long long g_trace2[296][64];
+#define CCL_TRACE2(cond, slot) do { if (cond) g_trace2[blockIdx.x][slot] = (unsigned long long)clock64(); } while (0)
+#else
+#define CCL_TRACE(slot) do { } while (0)
+#define CCL_TRACE2(cond, slot) do { } while (0)
+#endif
+
+// Division of a non-negative int by a launch constant as a multiply-high and a shift (an integer division costs a few
+// hundred cycles, and the tile walk of a short GEMM is nothing but divisions).  For d >= 2: l = ceil(log2 d),
+// mul = ceil(2^(31+l) / d), n / d = umulhi(n, mul) >> (l - 1), exact for 0 <= n < 2^31; d = 1: mul = 0, shr = 0.
+struct FastDiv {
+    uint32_t d, mul, shr;
+    __host__ __device__ int div(int n) const {
+#ifdef __CUDA_ARCH__
+        return mul ? (int)(__umulhi((uint32_t)n, mul) >> shr) : n;
+#else
+        return mul ? (int)(((uint64_t)(uint32_t)n * mul) >> 32 >> shr) : n;
+#endif
+    }
+    __host__ __device__ void divmod(int n, int& q, int& r) const { q = div(n); r = n - q * (int)d; }
+};
+static FastDiv make_fastdiv(int64_t d) {
+    FastDiv f;
+    if (d < 1) d = 1;
+    f.d = (uint32_t)d; f.mul = 0; f.shr = 0;
+    if (d == 1) return f;
+    int l = 0;
+    while ((INT64_C(1) << l) < d) ++l;
+    const unsigned __int128 one = 1;
+    f.mul = (uint32_t)(((one << (31 + l)) + (unsigned __int128)d - 1) / (unsigned __int128)d);
+    f.shr = (uint32_t)(l - 1);
+    return f;
+}
+
 struct OpMap {          // how stored coordinates (r, c) of an operand become tensor-map coordinates
     int32_t split;      // 0 none, 1 rows, 2 cols
-    int32_t w, h;       // strip width (split 2) / strip height (split 1)
+    FastDiv w, h;       // strip width (split 2) / strip height (split 1)
     // page-interleaved CCL (chunk of il_sc elements; chunk j of strip g stored as chunk j*P + g):
     //   il_mode 1: a chunk holds il_kr whole strip rows  -> map {x, row % kr, strip, row / kr}
     //   il_mode 2: a strip row spans whole chunks        -> map {x % sc, x / sc, row, strip}
     //   il_mode 0: strips stored one after the other     -> map {x, row, strip, 1}
-    int32_t il_mode, il_kr, il_sc;
+    int32_t il_mode;
+    FastDiv il_kr, il_sc;
 };
 
 struct GemmParams {
@@ -61,6 +99,9 @@ struct GemmParams {
     int32_t num_kb;
     int32_t groups, group_dim;      // chiplet-grouped raster: number of CTA groups, 0 = along N, 1 = along M
     int32_t panel;                  // m-tiles per raster panel
+    // raster constants the host derives from the grid it launches (see Scheduler)
+    int32_t sch_units, sch_gm, sch_gn, sch_upg, sch_floaters, sch_rounds, sch_per_group, sch_pool_per_group;
+    FastDiv fd_upg, fd_groups, fd_splits, fd_per_panel, fd_panel, fd_tps_m, fd_tps_n;
     OpMap a, b;
     int32_t a_mn, b_mn;             // 1 = MN-major operand tile in shared memory
     OpMap c;                        // C addressed through its own map as well (TMA tile stores)
@@ -165,11 +206,11 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint3
 // Stored coordinates (r, c) of an operand -> coordinates of its rank-4 tensor map.
 __device__ __forceinline__ void to_coords(const OpMap& o, int r, int c, int& x, int& y, int& z, int& u) {
     int g, rr, xx;                                   // strip, row inside the strip, column inside the strip row
-    if (o.split == 2) { g = c / o.w; xx = c - g * o.w; rr = r; }
-    else if (o.split == 1) { g = r / o.h; rr = r - g * o.h; xx = c; }
+    if (o.split == 2) { o.w.divmod(c, g, xx); rr = r; }
+    else if (o.split == 1) { o.h.divmod(r, g, rr); xx = c; }
     else { g = 0; rr = r; xx = c; }
-    if (o.il_mode == 1) { u = rr / o.il_kr; y = rr - u * o.il_kr; x = xx; z = g; }
-    else if (o.il_mode == 2) { y = xx / o.il_sc; x = xx - y * o.il_sc; z = rr; u = g; }
+    if (o.il_mode == 1) { o.il_kr.divmod(rr, u, y); x = xx; z = g; }
+    else if (o.il_mode == 2) { o.il_sc.divmod(xx, y, x); z = rr; u = g; }
     else { x = xx; y = rr; z = g; u = 0; }
 }
 // Element offset of C[m][n] in its buffer (any layout).
@@ -193,44 +234,41 @@ struct TileCoord { int m0, m1, n0, n1, split; };
 //   grouped unit : rounds [0, R) -> tile (index + round * upg) of its own group, then the pool
 //   floater f    : rounds [0, R) -> pool entries f, f + F, ...,                  then the pool
 // with R = min(total / units, per_group / upg); pool entries alternate between the groups.
+// The per-launch constants (units, upg, floaters, R, pool size) come from the host; tiles x splits < 2^31.
 struct Scheduler {
     const GemmParams& p;
     int gm, gn;                     // tile grid of one group
-    int unit, units, upg, floaters, my_g, idx, bm, bn, rounds;
-    int64_t per_group, pool_per_group;
-    __device__ Scheduler(const GemmParams& p_, int unit_, int units_, int bm_, int bn_) : p(p_), unit(unit_), units(units_), bm(bm_), bn(bn_) {
-        gm = p.tiles_m; gn = p.tiles_n;
-        if (p.groups > 1) { if (p.group_dim == 0) gn = p.tiles_n / p.groups; else gm = p.tiles_m / p.groups; }
-        per_group = (int64_t)gm * gn * p.splits;
-        upg = units / p.groups;                          // the host guarantees units >= groups
-        floaters = units - upg * p.groups;
-        my_g = unit < upg * p.groups ? unit / upg : -1;  // -1: floater
+    int unit, units, upg, floaters, my_g, idx, bm, bn, rounds, pool_per_group;
+    __device__ Scheduler(const GemmParams& p_, int unit_, int bm_, int bn_) : p(p_), unit(unit_), bm(bm_), bn(bn_) {
+        gm = p.sch_gm; gn = p.sch_gn; units = p.sch_units; upg = p.sch_upg; floaters = p.sch_floaters;
+        rounds = p.sch_rounds; pool_per_group = p.sch_pool_per_group;
+        my_g = unit < upg * p.groups ? p.fd_upg.div(unit) : -1;  // -1: floater
         idx = my_g >= 0 ? unit - my_g * upg : unit - upg * p.groups;
-        rounds = (int)min(per_group * p.groups / units, per_group / upg);
-        pool_per_group = per_group - (int64_t)rounds * upg;
     }
     __device__ bool get(int it, TileCoord& t) const {
-        int g;
-        int64_t i;
-        if (it < rounds && my_g >= 0) { g = my_g; i = idx + (int64_t)it * upg; }
+        int g, i;
+        if (it < rounds && my_g >= 0) { g = my_g; i = idx + it * upg; }
         else {
-            const int64_t q = it < rounds ? idx + (int64_t)it * floaters
-                                          : (int64_t)floaters * rounds + unit + (int64_t)(it - rounds) * units;
-            g = (int)(q % p.groups);
-            const int64_t j = q / p.groups;
+            const int q = it < rounds ? idx + it * floaters : floaters * rounds + unit + (it - rounds) * units;
+            int j = q;
+            g = 0;
+            if (p.groups > 1) p.fd_groups.divmod(q, j, g);
             if (j >= pool_per_group) return false;
-            i = (int64_t)rounds * upg + j;
+            i = rounds * upg + j;
         }
-        t.split = (int)(i % p.splits);                   // the splits of one tile are neighbours in the walk
-        i /= p.splits;
-        int64_t per_panel = (int64_t)p.panel * gn;
-        int pn = (int)(i / per_panel);
-        int rem = (int)(i - (int64_t)pn * per_panel);
-        int ph = min(p.panel, gm - pn * p.panel);
-        int ln = rem / ph, lm = pn * p.panel + (rem - ln * ph);
+        t.split = 0;
+        if (p.splits > 1) { int ii; p.fd_splits.divmod(i, ii, t.split); i = ii; }   // the splits of one tile are neighbours in the walk
+        int pn, rem;
+        p.fd_per_panel.divmod(i, pn, rem);
+        const bool tail = gm - pn * p.panel < p.panel;   // the last panel may be lower
+        const int ph = tail ? gm - pn * p.panel : p.panel;
+        int ln, lr;
+        if (tail) { ln = rem / ph; lr = rem - ln * ph; } else p.fd_panel.divmod(rem, ln, lr);
+        int lm = pn * p.panel + lr;
         int tm = lm + (p.group_dim == 1 ? g * gm : 0), tn = ln + (p.group_dim == 0 && p.groups > 1 ? g * gn : 0);
-        int sm = tm / p.tps_m, jm = tm - sm * p.tps_m;
-        int sn = tn / p.tps_n, jn = tn - sn * p.tps_n;
+        int sm, jm, sn, jn;
+        p.fd_tps_m.divmod(tm, sm, jm);
+        p.fd_tps_n.divmod(tn, sn, jn);
         t.m0 = sm * p.Wm + jm * bm; t.m1 = min(t.m0 + bm, (sm + 1) * p.Wm);
         t.n0 = sn * p.Wn + jn * bn; t.n1 = min(t.n0 + bn, (sn + 1) * p.Wn);
         return true;
@@ -240,7 +278,16 @@ struct Scheduler {
 template <int BN, int CTAS>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                const __grid_constant__ CUtensorMap map_c, const GemmParams p) {
+                const __grid_constant__ CUtensorMap map_c, const __grid_constant__ GemmParams gp) {
+    // The parameters are read from shared memory: the threads fetch the block's words side by side, so
+    // the cold constant-cache misses at kernel start overlap instead of queueing up in every role's set-up.
+    __shared__ GemmParams p;
+    {
+        static_assert(sizeof(GemmParams) % 4 == 0, "GemmParams is copied word by word");
+        const uint32_t* src = reinterpret_cast<const uint32_t*>(&gp);
+        uint32_t* dst = reinterpret_cast<uint32_t*>(&p);
+        for (int i = threadIdx.x; i < (int)(sizeof(GemmParams) / 4); i += kGemmThreads) dst[i] = src[i];
+    }
     // A tile wider than 256 columns is computed as NSUB sub-tiles of SUBN columns (one MMA each per
     // k step) that fill TMEM; narrower tiles use the two 256-column halves of TMEM as a double buffer.
     constexpr int NSUB = BN > 256 ? BN / 256 : 1;
@@ -248,11 +295,11 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     constexpr int SUBH = SUBN / CTAS;                // B columns of one sub-tile this CTA stages
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    unsigned char* epi = smem + (size_t)p.stages * p.stage_bytes;     // 1024-byte aligned: stage sizes are multiples of 1 KB
+    unsigned char* epi = smem + (size_t)gp.stages * gp.stage_bytes;     // 1024-byte aligned: stage sizes are multiples of 1 KB
     uint64_t* bars = reinterpret_cast<uint64_t*>(epi + kEpiBytes);
     uint64_t* full = bars;                           // used in the leader CTA only
-    uint64_t* empty = bars + p.stages;               // one set per CTA
-    uint64_t* tmem_full = bars + 2 * p.stages;       // one set per CTA
+    uint64_t* empty = bars + gp.stages;               // one set per CTA
+    uint64_t* tmem_full = bars + 2 * gp.stages;       // one set per CTA
     uint64_t* tmem_empty = tmem_full + 2;            // used in the leader CTA only
     uint32_t* tmem_ptr = reinterpret_cast<uint32_t*>(tmem_empty + 2);
 
@@ -261,10 +308,11 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     const bool leader = rank == 0;
 
     if (threadIdx.x == 0) {
+        CCL_TRACE(0);
         prefetch_tmap(&map_a);
         prefetch_tmap(&map_b);
         prefetch_tmap(&map_c);
-        for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        for (int s = 0; s < gp.stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(&tmem_full[a], 1); mbar_init(&tmem_empty[a], 4 * CTAS); }
         fence_barrier_init();
     }
@@ -274,8 +322,10 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     if (CTAS == 2) cluster_sync();                   // the peer's barriers exist before anything remote touches them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_ptr;
+    if (threadIdx.x == 0) CCL_TRACE(1);
 
-    Scheduler sched(p, (int)(blockIdx.x / CTAS), (int)(gridDim.x / CTAS), BM * CTAS, BN);
+    Scheduler sched(p, (int)(blockIdx.x / CTAS), BM * CTAS, BN);
+    if (threadIdx.x == 0) CCL_TRACE(10);
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -310,16 +360,20 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             int x, y, z, u;
             if (mn) to_coords(om, 0, base, x, y, z, u); else to_coords(om, base, 0, x, y, z, u);
             const int kb0 = t.split * p.kb_per_split, kb1 = min(p.num_kb, kb0 + p.kb_per_split);
+            if (lane == 0 && it == 0) CCL_TRACE(11);
             for (int kb = kb0; kb < kb1; ++kb) {
                 ok = mbar_wait_bounded(&empty[stage], phase ^ 1);
                 ok = __all_sync(0xffffffffu, ok);
+                if (lane == 0 && it == 0 && kb == kb0) CCL_TRACE(12);
                 if (!ok) { if (lane == 0) atomicExch(&g_gemm_status, 1); break; }
                 if (lane == 0 && leader) mbar_expect_tx(&full[stage], p.stage_bytes * CTAS);
                 __syncwarp();
                 const int k0 = kb * BK;
                 if (ksplit) { if (mn) to_coords(om, k0, base, x, y, z, u); else to_coords(om, base, k0, x, y, z, u); }
                 else if (mn) y = k0; else x = k0;
+                if (lane == 0 && it == 0 && kb == kb0) CCL_TRACE(13);
                 if (active) tma_load<CTAS>(smem + (size_t)stage * p.stage_bytes + soff, map, full0 + (uint32_t)stage * 8u, x, y, z, u);
+                if (lane == 0 && it == 0 && kb == kb0) CCL_TRACE(2);
                 if (++stage == p.stages) { stage = 0; phase ^= 1; }
             }
         }
@@ -343,6 +397,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 for (int kb = kb0; ok && kb < kb1; ++kb) {
                     if (!mbar_wait_bounded(&full[stage], phase)) { atomicExch(&g_gemm_status, 3); ok = false; break; }
                     tc_fence_after();
+                    if (it == 0 && kb == kb0) CCL_TRACE(3);
                     const uint32_t sa = smem_u32(smem + (size_t)stage * p.stage_bytes);
                     const uint64_t adesc = smem_desc(sa, a_lbo, 1024);
 #pragma unroll
@@ -362,8 +417,8 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     if (++stage == p.stages) { stage = 0; phase ^= 1; }
                 }
                 if (ok) {
-#pragma unroll
-                    for (int h = 0; h < NSUB; ++h) umma_commit<CTAS>(&tmem_full[acc0 + h]);   // accumulators complete (both CTAs)
+                    umma_commit<CTAS>(&tmem_full[acc0]);   // accumulator(s) complete (both CTAs); the sub-tiles of a wide tile finish together
+                    if (it == 0) CCL_TRACE(4);
                 }
             }
         }
@@ -376,31 +431,36 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         uint32_t epi_count = 0;                          // TMA-stored pieces so far (selects the staging buffer)
         for (int it = 0; alive && sched.get(it, t); ++it) {
           const int m = t.m0 + (int)rank * BM + quad * 32 + lane;
+#pragma unroll 1                                         // one copy of the (large) drain code: a short GEMM pays for every instruction-cache miss
           for (int h = 0; h < NSUB; ++h) {
             const int acc = NSUB == 1 ? (it & 1) : h;
             const uint32_t acc_phase = NSUB == 1 ? ((uint32_t)(it >> 1) & 1) : ((uint32_t)it & 1);
             const int nb = t.n0 + h * SUBN;              // first column of this sub-tile
-            bool ok = mbar_wait_bounded(&tmem_full[acc], acc_phase);
+            bool ok = h > 0 || mbar_wait_bounded(&tmem_full[acc], acc_phase);   // one "full" barrier per tile
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) { if (lane == 0) atomicExch(&g_gemm_status, 4); alive = false; break; }
             tc_fence_after();
-            // offset of (m, n) in C is row_base + n for every n of this tile
-            int64_t row_base;
-            if (p.c_split == 2) { int64_t g = t.n0 / p.c_w; row_base = g * p.c_stride + (int64_t)m * p.c_w - g * p.c_w; }
-            else if (p.c_split == 1) { int64_t g = t.m0 / p.c_h; row_base = g * p.c_stride + ((int64_t)m - g * p.c_h) * p.c_cols; }
-            else row_base = (int64_t)m * p.c_cols;
+            if (warp == 2 && lane == 0 && it == 0 && h == 0) CCL_TRACE(5);
+            if (warp == 2 && lane == 0 && it == 0 && h == 1) CCL_TRACE(14);
             const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)acc * 256u;
             // Full 32-row x 64-column pieces go through shared memory (128-byte swizzle) and a TMA tile store
             // addressed through C's own tensor map; ragged pieces (tile clipped by a strip or the matrix edge)
             // and split-K partial sums are stored from registers.
             const int row0 = t.m0 + (int)rank * BM + quad * 32;
             const bool rows_full = row0 + 32 <= t.m1;
+            // C map coordinates of (row0, nb): a tile lies inside one strip, so only x moves from piece to piece
+            // (unless a strip row is cut into chunks, which puts the chunk index in y as well)
+            int cx0, cy0, cz0, cu0;
+            to_coords(p.c, row0, nb, cx0, cy0, cz0, cu0);
+            const bool c_chunked = p.c.il_mode == 2;
             // One 64-column piece: registers -> C.  `r` holds 64 fp32 accumulators of this thread's row.
             auto store_piece = [&](const uint32_t (&r)[64], int c) {
                 const int n64 = nb + c * 64;
                 if (p.splits == 1 && rows_full && n64 + 64 <= t.n1) {
                     unsigned char* buf = epi + (size_t)((warp - 2) * 2 + (epi_count & 1)) * (32 * 128);
+                    CCL_TRACE2(warp == 2 && lane == 0 && epi_count < 12, epi_count * 5 + 0);
                     if (epi_count >= 2) { if (lane == 0) tma_store_wait_read<1>(); __syncwarp(); }   // buffer free again
+                    CCL_TRACE2(warp == 2 && lane == 0 && epi_count < 12, epi_count * 5 + 1);
 #pragma unroll
                     for (int u = 0; u < 8; ++u) {
                         uint4 v;
@@ -411,17 +471,22 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                         hh = __floats2bfloat162_rn(__uint_as_float(r[u * 8 + 6]), __uint_as_float(r[u * 8 + 7])); v.w = *reinterpret_cast<uint32_t*>(&hh);
                         *reinterpret_cast<uint4*>(buf + lane * 128 + ((u ^ (lane & 7)) << 4)) = v;
                     }
+                    CCL_TRACE2(warp == 2 && lane == 0 && epi_count < 12, epi_count * 5 + 2);
                     fence_proxy_async();
                     __syncwarp();
+                    CCL_TRACE2(warp == 2 && lane == 0 && epi_count < 12, epi_count * 5 + 3);
                     if (lane == 0) {
-                        int cx, cy, cz, cu;                      // C map coordinates of (row0, n64)
-                        to_coords(p.c, row0, n64, cx, cy, cz, cu);
+                        int cx = cx0 + c * 64, cy = cy0, cz = cz0, cu = cu0;
+                        if (c_chunked) to_coords(p.c, row0, n64, cx, cy, cz, cu);
                         tma_store_4d(&map_c, buf, cx, cy, cz, cu);
                         tma_store_commit();
                     }
+                    CCL_TRACE2(warp == 2 && lane == 0 && epi_count < 12, epi_count * 5 + 4);
                     ++epi_count;
                     return;
                 }
+                // a 64-column piece of a row is contiguous in every layout the GEMM accepts
+                const int64_t piece_off = p.splits > 1 || m >= t.m1 ? 0 : c_offset(p, m, n64);
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
                     const uint32_t* rr = &r[half * 32];
@@ -447,7 +512,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                                 hh = __floats2bfloat162_rn(__uint_as_float(rr[j * 8 + 2]), __uint_as_float(rr[j * 8 + 3])); v.y = *reinterpret_cast<uint32_t*>(&hh);
                                 hh = __floats2bfloat162_rn(__uint_as_float(rr[j * 8 + 4]), __uint_as_float(rr[j * 8 + 5])); v.z = *reinterpret_cast<uint32_t*>(&hh);
                                 hh = __floats2bfloat162_rn(__uint_as_float(rr[j * 8 + 6]), __uint_as_float(rr[j * 8 + 7])); v.w = *reinterpret_cast<uint32_t*>(&hh);
-                                *reinterpret_cast<uint4*>(p.C + (p.c_ichunk ? c_offset(p, m, n) : row_base + n)) = v;
+                                *reinterpret_cast<uint4*>(p.C + piece_off + (n - n64)) = v;
                             }
                         }
                     }
@@ -475,21 +540,28 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             }
             tc_fence_before();
             __syncwarp();
+            if (warp == 2 && lane == 0 && it == 0 && h == NSUB - 1) CCL_TRACE(6);
+            if (warp == 2 && lane == 0 && it == 0 && h == 0) CCL_TRACE(15);
             if (lane == 0) {
                 if (CTAS == 2) mbar_arrive_cluster(tmem_empty0 + (uint32_t)acc * 8u);
                 else mbar_arrive(&tmem_empty[acc]);
             }
           }
         }
-        if (lane == 0) tma_store_wait_all<0>();          // every tile store has left shared memory and landed
+        // every tile store has read its shared-memory source; the writes themselves are complete, like any other
+        // store of the kernel, when the kernel is
+        if (lane == 0) tma_store_wait_read<0>();
+        if (warp == 2 && lane == 0) CCL_TRACE(7);
     }
 
     tc_fence_before();
     __syncthreads();
     if (CTAS == 2) cluster_sync();                   // neither CTA frees TMEM or exits while the other may still use it
+    if (threadIdx.x == 0) CCL_TRACE(8);
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc<CTAS>(tmem_base, kTmemCols);
+        if (lane == 0) CCL_TRACE(9);
     }
 }
 
@@ -682,13 +754,13 @@ static ccl_status make_plan(const ccl_gemm_desc* d, const void* A, const void* B
     p.tiles_m = (int32_t)(d->M / Wm) * p.tps_m; p.tiles_n = (int32_t)(d->N / Wn) * p.tps_n;
     p.num_kb = (int32_t)num_kb;
     p.splits = splits; p.kb_per_split = (int32_t)((num_kb + splits - 1) / splits);
-    p.a.split = va.split; p.a.w = (int32_t)va.w; p.a.h = (int32_t)va.h;
-    p.b.split = vb.split; p.b.w = (int32_t)vb.w; p.b.h = (int32_t)vb.h;
+    p.a.split = va.split; p.a.w = make_fastdiv(va.w); p.a.h = make_fastdiv(va.h);
+    p.b.split = vb.split; p.b.w = make_fastdiv(vb.w); p.b.h = make_fastdiv(vb.h);
     p.a_mn = at ? 1 : 0; p.b_mn = bt ? 0 : 1;
-    p.a.il_mode = il_a; p.a.il_kr = (int32_t)std::max<int64_t>(kr_a, 1); p.a.il_sc = (int32_t)std::max<int64_t>(va.ichunk, 1);
-    p.b.il_mode = il_b; p.b.il_kr = (int32_t)std::max<int64_t>(kr_b, 1); p.b.il_sc = (int32_t)std::max<int64_t>(vb.ichunk, 1);
-    p.c.split = vc.split; p.c.w = (int32_t)vc.w; p.c.h = (int32_t)vc.h;
-    p.c.il_mode = il_c; p.c.il_kr = (int32_t)std::max<int64_t>(kr_c, 1); p.c.il_sc = (int32_t)std::max<int64_t>(vc.ichunk, 1);
+    p.a.il_mode = il_a; p.a.il_kr = make_fastdiv(kr_a); p.a.il_sc = make_fastdiv(va.ichunk);
+    p.b.il_mode = il_b; p.b.il_kr = make_fastdiv(kr_b); p.b.il_sc = make_fastdiv(vb.ichunk);
+    p.c.split = vc.split; p.c.w = make_fastdiv(vc.w); p.c.h = make_fastdiv(vc.h);
+    p.c.il_mode = il_c; p.c.il_kr = make_fastdiv(kr_c); p.c.il_sc = make_fastdiv(vc.ichunk);
     p.c_split = vc.split; p.c_w = vc.w; p.c_h = vc.h; p.c_stride = vc.stride; p.c_cols = vc.cols;
     p.c_ichunk = vc.ichunk; p.c_nstrips = vc.nstrips;
     // instruction descriptor: D = f32, A = B = bf16, operand majors, N >> 3, M >> 4 (M spans the CTA pair)
@@ -704,6 +776,16 @@ static ccl_status make_plan(const ccl_gemm_desc* d, const void* A, const void* B
     if (groups > 1 && units >= groups && (group_dim == 0 ? p.tiles_n % groups == 0 : p.tiles_m % groups == 0)) {
         p.groups = groups; p.group_dim = group_dim;
     } else { p.groups = 1; p.group_dim = 0; }
+    {   // raster constants (see Scheduler): equal-size groups, floaters, full rounds and the pooled tail
+        if (ntiles >= (INT64_C(1) << 31) - 2 * units) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: too many tiles");
+        const int gm = p.group_dim == 1 && p.groups > 1 ? p.tiles_m / p.groups : p.tiles_m;
+        const int gn = p.group_dim == 0 && p.groups > 1 ? p.tiles_n / p.groups : p.tiles_n;
+        const int64_t per_group = (int64_t)gm * gn * splits;
+        const int upg = units / p.groups;
+        const int64_t rounds = std::min(per_group * p.groups / units, per_group / upg);
+        p.sch_units = units; p.sch_gm = gm; p.sch_gn = gn; p.sch_upg = upg; p.sch_floaters = units - upg * p.groups;
+        p.sch_rounds = (int32_t)rounds; p.sch_per_group = (int32_t)per_group; p.sch_pool_per_group = (int32_t)(per_group - rounds * upg);
+    }
     // Raster panel height: the units of a group that run at the same time cover `panel` m-tiles by
     // ceil(upg / panel) n-tiles; all groups walk the same m-panel.  The operand rows + columns such a wave
     // touches are what it pulls from DRAM (the L2 does not hold a wave's footprint until the next wave), so
@@ -719,6 +801,9 @@ static ccl_status make_plan(const ccl_gemm_desc* d, const void* A, const void* B
         }
     }
     if (const char* f = std::getenv("CCL_GEMM_PANEL")) p.panel = std::max(1, atoi(f));
+    p.fd_upg = make_fastdiv(p.sch_upg); p.fd_groups = make_fastdiv(p.groups); p.fd_splits = make_fastdiv(p.splits);
+    p.fd_per_panel = make_fastdiv((int64_t)p.panel * p.sch_gn); p.fd_panel = make_fastdiv(p.panel);
+    p.fd_tps_m = make_fastdiv(p.tps_m); p.fd_tps_n = make_fastdiv(p.tps_n);
     plan->smem_bytes = (uint32_t)p.stages * p.stage_bytes + kEpiBytes + 1024 + (2 * p.stages + 4) * 8 + 16;
     return CCL_OK;
 }
@@ -994,3 +1079,12 @@ extern "C" ccl_status ccl_gemm_static_ws(const ccl_gemm_desc* d, const void* A_d
     }
     return ccl_gemm(d, A_dev, B_dev, C_dev, ws, need ? (size_t)CCL_GEMM_STATIC_WS_BYTES : 0, cuda_stream);
 }
+
+#ifdef CCL_GEMM_TRACE
+extern "C" int ccl_debug_trace_read(void* host_out, size_t bytes) {
+    return (int)cudaMemcpyFromSymbol(host_out, ccl::g_trace, bytes < sizeof(ccl::g_trace) ? bytes : sizeof(ccl::g_trace));
+}
+extern "C" int ccl_debug_trace2_read(void* host_out, size_t bytes) {
+    return (int)cudaMemcpyFromSymbol(host_out, ccl::g_trace2, bytes < sizeof(ccl::g_trace2) ? bytes : sizeof(ccl::g_trace2));
+}
+#endif
