@@ -46,7 +46,7 @@ __device__ int g_gemm_status = 0;
 #ifdef CCL_GEMM_TRACE   // development aid: per-CTA timestamps of the kernel's phases (not compiled into the library)
 __device__ unsigned long long g_trace[296][32];
 #define CCL_TRACE(slot) do { g_trace[blockIdx.x][slot] = global_timer_ns(); g_trace[blockIdx.x][16 + (slot)] = (unsigned long long)clock64(); } while (0)
-__device__ unsigned long long g_trace2[296][64];
+__device__ unsigned long long g_trace2[296][128];
 #define CCL_TRACE2(cond, slot) do { if (cond) g_trace2[blockIdx.x][slot] = (unsigned long long)clock64(); } while (0)
 #else
 #define CCL_TRACE(slot) do { } while (0)
@@ -292,6 +292,8 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     // k step) that fill TMEM; narrower tiles use the two 256-column halves of TMEM as a double buffer.
     constexpr int NSUB = BN > 256 ? BN / 256 : 1;
     constexpr int SUBN = BN / NSUB;
+    constexpr int ACC_COLS = NSUB == 1 ? 256 : SUBN;  // TMEM columns between accumulators
+    constexpr int NACC = NSUB == 1 ? 2 : NSUB;        // accumulator barriers in use
     constexpr int SUBH = SUBN / CTAS;                // B columns of one sub-tile this CTA stages
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -300,8 +302,8 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     uint64_t* full = bars;                           // used in the leader CTA only
     uint64_t* empty = bars + gp.stages;               // one set per CTA
     uint64_t* tmem_full = bars + 2 * gp.stages;       // one set per CTA
-    uint64_t* tmem_empty = tmem_full + 2;            // used in the leader CTA only
-    uint32_t* tmem_ptr = reinterpret_cast<uint32_t*>(tmem_empty + 2);
+    uint64_t* tmem_empty = tmem_full + 4;            // used in the leader CTA only
+    uint32_t* tmem_ptr = reinterpret_cast<uint32_t*>(tmem_empty + 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = CTAS == 2 ? cluster_ctarank() : 0;
@@ -313,7 +315,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         prefetch_tmap(&map_b);
         prefetch_tmap(&map_c);
         for (int s = 0; s < gp.stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(&tmem_full[a], 1); mbar_init(&tmem_empty[a], 4 * CTAS); }
+        for (int a = 0; a < NACC; ++a) { mbar_init(&tmem_full[a], 1); mbar_init(&tmem_empty[a], 4 * CTAS); }
         fence_barrier_init();
     }
     if (warp == 1) tmem_alloc<CTAS>(tmem_ptr, kTmemCols);
@@ -355,26 +357,32 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         uint32_t phase = 0;
         TileCoord t;
         bool ok = true;
+        // loop constants in registers (the asm statements below are memory barriers to the compiler)
+        const int stages = p.stages, num_kb = p.num_kb, kbps = p.kb_per_split;
+        const uint32_t stage_bytes = p.stage_bytes;
+        const bool post_tx = lane == 0 && leader;
         for (int it = 0; ok && sched.get(it, t); ++it) {
             const int base = (isA ? t.m0 : t.n0) + off;
             int x, y, z, u;
             if (mn) to_coords(om, 0, base, x, y, z, u); else to_coords(om, base, 0, x, y, z, u);
-            const int kb0 = t.split * p.kb_per_split, kb1 = min(p.num_kb, kb0 + p.kb_per_split);
+            const int kb0 = t.split * kbps, kb1 = min(num_kb, kb0 + kbps);
             if (lane == 0 && it == 0) CCL_TRACE(11);
             for (int kb = kb0; kb < kb1; ++kb) {
                 ok = mbar_wait_bounded(&empty[stage], phase ^ 1);
                 ok = __all_sync(0xffffffffu, ok);
                 if (lane == 0 && it == 0 && kb == kb0) CCL_TRACE(12);
+                CCL_TRACE2(lane == 0 && it == 0 && kb - kb0 < 16, 64 + (kb - kb0) * 2);
                 if (!ok) { if (lane == 0) atomicExch(&g_gemm_status, 1); break; }
-                if (lane == 0 && leader) mbar_expect_tx(&full[stage], p.stage_bytes * CTAS);
-                __syncwarp();
+                // (the byte count may be posted after a copy has completed: the phase cannot end before this arrival)
+                if (post_tx) mbar_expect_tx(&full[stage], stage_bytes * CTAS);
                 const int k0 = kb * BK;
                 if (ksplit) { if (mn) to_coords(om, k0, base, x, y, z, u); else to_coords(om, base, k0, x, y, z, u); }
                 else if (mn) y = k0; else x = k0;
                 if (lane == 0 && it == 0 && kb == kb0) CCL_TRACE(13);
-                if (active) tma_load<CTAS>(smem + (size_t)stage * p.stage_bytes + soff, map, full0 + (uint32_t)stage * 8u, x, y, z, u);
+                if (active) tma_load<CTAS>(smem + (size_t)stage * stage_bytes + soff, map, full0 + (uint32_t)stage * 8u, x, y, z, u);
                 if (lane == 0 && it == 0 && kb == kb0) CCL_TRACE(2);
-                if (++stage == p.stages) { stage = 0; phase ^= 1; }
+                CCL_TRACE2(lane == 0 && it == 0 && kb - kb0 < 16, 64 + (kb - kb0) * 2 + 1);
+                if (++stage == stages) { stage = 0; phase ^= 1; }
             }
         }
     } else if (warp == 1) {
@@ -387,18 +395,23 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             const uint32_t a_lbo = p.a_mn ? 64 * BK * 2 : 16, b_lbo = p.b_mn ? 64 * BK * 2 : 16;
             const uint32_t a_kstep = p.a_mn ? (16 * 128) >> 4 : (16 * 2) >> 4;     // descriptor units (16 B) per UMMA_K = 16
             const uint32_t b_kstep = p.b_mn ? (16 * 128) >> 4 : (16 * 2) >> 4;
+            // loop constants in registers (the asm statements below are memory barriers to the compiler)
+            const int stages = p.stages, num_kb = p.num_kb, kbps = p.kb_per_split;
+            const uint32_t stage_bytes = p.stage_bytes, a_bytes = p.a_bytes, idesc = p.idesc, smem0 = smem_u32(smem);
             for (int it = 0; ok && sched.get(it, t); ++it) {
                 // NSUB == 1: TMEM half (it & 1) is this tile's accumulator, the other half is being drained.
                 // NSUB == 2: both halves belong to this tile; half h may be overwritten once the epilogue
                 //            of the previous tile has drained it.
                 const int acc0 = NSUB == 1 ? (it & 1) : 0;
                 const uint32_t acc_phase = NSUB == 1 ? ((uint32_t)(it >> 1) & 1) : ((uint32_t)it & 1);
-                const int kb0 = t.split * p.kb_per_split, kb1 = min(p.num_kb, kb0 + p.kb_per_split);
+                const int kb0 = t.split * kbps, kb1 = min(num_kb, kb0 + kbps);
                 for (int kb = kb0; ok && kb < kb1; ++kb) {
+                    // (the copies' completion on the barrier orders the operand bytes before the MMAs that read them;
+                    // tcgen05 fences are only needed around the accumulator hand-over below)
                     if (!mbar_wait_bounded(&full[stage], phase)) { atomicExch(&g_gemm_status, 3); ok = false; break; }
-                    tc_fence_after();
                     if (it == 0 && kb == kb0) CCL_TRACE(3);
-                    const uint32_t sa = smem_u32(smem + (size_t)stage * p.stage_bytes);
+                    CCL_TRACE2(it == 0 && kb - kb0 < 16, 96 + (kb - kb0) * 2);
+                    const uint32_t sa = smem0 + (uint32_t)stage * stage_bytes;
                     const uint64_t adesc = smem_desc(sa, a_lbo, 1024);
 #pragma unroll
                     for (int h = 0; h < NSUB; ++h) {
@@ -406,15 +419,16 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                             if (!mbar_wait_bounded(&tmem_empty[acc0 + h], acc_phase ^ 1)) { atomicExch(&g_gemm_status, 2); ok = false; break; }
                             tc_fence_after();
                         }
-                        const uint32_t tmem_d = tmem_base + (uint32_t)(acc0 + h) * 256u;
-                        const uint64_t bdesc = smem_desc(sa + p.a_bytes + h * (SUBH * BK * 2), b_lbo, 1024);
+                        const uint32_t tmem_d = tmem_base + (uint32_t)((acc0 + h) * ACC_COLS);
+                        const uint64_t bdesc = smem_desc(sa + a_bytes + h * (SUBH * BK * 2), b_lbo, 1024);
 #pragma unroll
                         for (int k = 0; k < BK / 16; ++k)
-                            umma_bf16<CTAS>(tmem_d, adesc + (uint64_t)(k * a_kstep), bdesc + (uint64_t)(k * b_kstep), p.idesc, ((kb - kb0) | k) != 0);
+                            umma_bf16<CTAS>(tmem_d, adesc + (uint64_t)(k * a_kstep), bdesc + (uint64_t)(k * b_kstep), idesc, ((kb - kb0) | k) != 0);
                     }
                     if (!ok) break;
                     umma_commit<CTAS>(&empty[stage]);          // frees the stage (in both CTAs) once these MMAs have read it
-                    if (++stage == p.stages) { stage = 0; phase ^= 1; }
+                    CCL_TRACE2(it == 0 && kb - kb0 < 16, 96 + (kb - kb0) * 2 + 1);
+                    if (++stage == stages) { stage = 0; phase ^= 1; }
                 }
                 if (ok) {
                     umma_commit<CTAS>(&tmem_full[acc0]);   // accumulator(s) complete (both CTAs); the sub-tiles of a wide tile finish together
@@ -442,7 +456,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             tc_fence_after();
             if (warp == 2 && lane == 0 && it == 0 && h == 0) CCL_TRACE(5);
             if (warp == 2 && lane == 0 && it == 0 && h == 1) CCL_TRACE(14);
-            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)acc * 256u;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * ACC_COLS);
             // Full 32-row x 64-column pieces go through shared memory (128-byte swizzle) and a TMA tile store
             // addressed through C's own tensor map; ragged pieces (tile clipped by a strip or the matrix edge)
             // and split-K partial sums are stored from registers.
@@ -596,7 +610,7 @@ __global__ void __launch_bounds__(256) splitk_reduce_kernel(const GemmParams p) 
 // ------------------------------------------------------------------------------------------
 struct GemmPlan {
     GemmParams p;
-    int bn, ctas;
+    int bn, ctas, subn;
     size_t ws_bytes;
     MatView va, vb, vc;
     uint32_t smem_bytes;
@@ -677,8 +691,8 @@ static ccl_status make_plan(const ccl_gemm_desc* d, const void* A, const void* B
     if ((s = check_operand(vc, C, "C", false, d->K))) return s;
     int64_t kr_a, kr_b, kr_c;
     const int il_a = interleave_mode(va, &kr_a), il_b = interleave_mode(vb, &kr_b), il_c = interleave_mode(vc, &kr_c);
-    // a 192-row box of a K-contiguous B cannot be cut into chunks of more than 64 rows
-    const bool no_192 = il_b == 1 && bt && kr_b > 64;
+    // a 192-row (96-row for a CTA pair) box of a K-contiguous B cannot be cut into chunks of more than 64 (32) rows
+    const bool no_192 = il_b == 1 && bt && kr_b > 64, no_192_pair = il_b == 1 && bt && kr_b > 32;
 
     // strips along M, N (tiles must not straddle them) and along K (a 64-wide k block must not)
     int64_t Wm = 0, Wn = 0;
@@ -704,9 +718,14 @@ static ccl_status make_plan(const ccl_gemm_desc* d, const void* A, const void* B
     if (!Wn) Wn = d->N;
 
     // Tile shape, CTA pairing and split-K from a small cost model (cycles per unit):
-    //   a k block takes max(MMA time, time to pull this SM's operand bytes from L2 at ~50 B/clk);
-    //   a unit pays ~3000 cycles of pipeline fill + epilogue; split-K adds the partial-sum traffic.
-    // 256 x 512 pair tiles move the fewest bytes per flop; small problems prefer 1-CTA tiles and split-K.
+    //   a k block of a one-accumulator tile takes ~600 cycles whatever its width (four MMAs are issued in ~350
+    //   cycles and the barrier round trip adds ~250), a 256 x 512 pair tile ~1050 (its eight MMAs keep the
+    //   tensor pipe busy for 1024); a tile that nobody shares its B columns with (one row of tiles) streams
+    //   them from HBM at this SM's share of the bandwidth, ~27 B/clk;
+    //   a one-accumulator tile hides its drain behind the next tile's main loop (TMEM double buffer), the wide
+    //   tile exposes it (~7000 cycles); split-K adds the partial-sum traffic and a second launch.
+    // 256 x 512 pair tiles move the fewest bytes per flop and win once K is long; short problems prefer the
+    // variant whose tile count fills the machine.
     const int64_t num_kb = (d->K + BK - 1) / BK;
     const int64_t strips_m = d->M / Wm, strips_n = d->N / Wn;
     int ctas = 1, bn = 256, splits = 1;
@@ -721,27 +740,31 @@ static ccl_status make_plan(const ccl_gemm_desc* d, const void* A, const void* B
         if (force_ctas && atoi(force_ctas) != c) continue;
         const int units = c == 2 ? pairs : sms;
         for (int b : {512, 256, 192, 128}) {
-            if (c == 1 && b == 512) continue;
-            if (c == 2 && b == 192) continue;
-            if (b == 192 && no_192) continue;
+            if (c == 1 && b > 256) continue;
+            if (c == 2 && b == 192 && !bt) continue;             // 96 columns per CTA are not made of 64-column boxes of an N-contiguous B
+            if (b == 192 && (c == 2 ? no_192_pair : no_192)) continue;
             if (force_bn && atoi(force_bn) != b) continue;
-            const int64_t tiles = strips_m * ((Wm + BM * c - 1) / (BM * c)) * strips_n * ((Wn + b - 1) / b);
-            const double t_kb = std::max((double)b / 256.0 * 512.0, (128.0 + (double)b / c) * 2.56);
+            const int64_t tiles_m_all = strips_m * ((Wm + BM * c - 1) / (BM * c));
+            const int64_t tiles = tiles_m_all * strips_n * ((Wn + b - 1) / b);
+            double t_kb = b == 512 ? 1050.0 : (c == 1 && b == 256 ? 680.0 : (c == 1 ? 570.0 : 620.0));
+            if (tiles_m_all == 1) t_kb = std::max(t_kb, (double)(b / c) * (BK * 2) / 27.0);
+            const double t_drain = b == 512 ? 7000.0 : 1500.0;
             for (int sp : {1, 2, 3, 4, 6, 8, 12, 16}) {
-                if (sp > 1 && (c == 2 || num_kb / sp < 2)) continue;
+                if (sp > 1 && num_kb / sp < 2) continue;
                 if (force_split && atoi(force_split) != sp) continue;
                 const int64_t kbps = (num_kb + sp - 1) / sp;
                 const int64_t sp_eff = (num_kb + kbps - 1) / kbps;          // every split owns at least one k block
                 if (sp_eff != sp) continue;
                 const int64_t waves = (tiles * sp + units - 1) / units;
-                double cost = (double)waves * ((double)kbps * t_kb + 3000.0);
-                if (sp > 1) cost += ((double)sp + 0.5) * (double)d->M * (double)d->N * 4.0 / 3400.0 + 4000.0;
+                double cost = (double)waves * ((double)kbps * t_kb + (sp > 1 ? 2.0 * t_drain : t_drain)) + 3000.0;
+                if (sp > 1) cost += ((double)sp + 0.5) * (double)d->M * (double)d->N * 4.0 / 3400.0 + 14000.0;
                 if (best < 0 || cost < best) { best = cost; ctas = c; bn = b; splits = sp; }
             }
         }
     }
     if (best < 0) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: no kernel variant matches the forced CCL_GEMM_* settings");
     const int subn = bn > 256 ? 256 : bn;                // columns of one MMA / one TMEM accumulator
+    plan->subn = subn;
     const int bm = BM * ctas;
     plan->bn = bn; plan->ctas = ctas;
     plan->ws_bytes = splits > 1 ? (size_t)splits * (size_t)d->M * (size_t)d->N * 4 : 0;
@@ -804,7 +827,7 @@ static ccl_status make_plan(const ccl_gemm_desc* d, const void* A, const void* B
     p.fd_upg = make_fastdiv(p.sch_upg); p.fd_groups = make_fastdiv(p.groups); p.fd_splits = make_fastdiv(p.splits);
     p.fd_per_panel = make_fastdiv((int64_t)p.panel * p.sch_gn); p.fd_panel = make_fastdiv(p.panel);
     p.fd_tps_m = make_fastdiv(p.tps_m); p.fd_tps_n = make_fastdiv(p.tps_n);
-    plan->smem_bytes = (uint32_t)p.stages * p.stage_bytes + kEpiBytes + 1024 + (2 * p.stages + 4) * 8 + 16;
+    plan->smem_bytes = (uint32_t)p.stages * p.stage_bytes + kEpiBytes + 1024 + (2 * p.stages + 8) * 8 + 16;
     return CCL_OK;
 }
 
@@ -984,7 +1007,7 @@ extern "C" ccl_status ccl_gemm(const ccl_gemm_desc* d, const void* A_dev, const 
         if (dev != key.dev) make_key(d, A_dev, B_dev, C_dev, &key);
         if ((s = make_plan(d, A_dev, B_dev, C_dev, prep.sms, resident_pairs(), &plan))) return s;
         plan.p.C = static_cast<uint16_t*>(C_dev);
-        const uint32_t bnh = (uint32_t)((plan.bn > 256 ? 256 : plan.bn) / plan.ctas);   // B rows of one K-major box
+        const uint32_t bnh = (uint32_t)(plan.subn / plan.ctas);   // B rows of one K-major box
         if (!plan.p.a_mn) s = operand_tmap(&prep.ma, plan.va, A_dev, BK, BM); else s = operand_tmap(&prep.ma, plan.va, A_dev, 64, BK);
         if (s) return s;
         if (!plan.p.b_mn) s = operand_tmap(&prep.mb, plan.vb, B_dev, BK, bnh); else s = operand_tmap(&prep.mb, plan.vb, B_dev, 64, BK);
@@ -1007,6 +1030,7 @@ extern "C" ccl_status ccl_gemm(const ccl_gemm_desc* d, const void* A_dev, const 
     cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
     if (plan.ctas == 2) {
         if (plan.bn == 512) s = launch<512, 2>(plan, ma, mb, mc, st);
+        else if (plan.bn == 192) s = launch<192, 2>(plan, ma, mb, mc, st);
         else s = plan.bn == 256 ? launch<256, 2>(plan, ma, mb, mc, st) : launch<128, 2>(plan, ma, mb, mc, st);
     } else if (plan.bn == 256) s = launch<256, 1>(plan, ma, mb, mc, st);
     else if (plan.bn == 192) s = launch<192, 1>(plan, ma, mb, mc, st);

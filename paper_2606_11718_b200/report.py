@@ -65,10 +65,14 @@ def mats(g, layout_bc, align=0):
 
 
 def timed(fn, reps, warm=2):
+    """Mean device time of `fn` in ms over `reps` back-to-back launches (CUDA events on the current stream).
+    The launches are queued behind a short device-side spin, so that a kernel of a few microseconds is not
+    timed at the rate the host can issue it."""
     for _ in range(warm):
         fn()
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda._sleep(min(200_000_000, 1_000_000 + 40_000 * reps))      # cycles; ~20 us of head start per launch
     e0.record()
     for _ in range(reps):
         fn()

@@ -238,14 +238,41 @@ def test_gemm_llama_full_size_sampled(name, P):
         assert (lhs - rhs).abs().max().item() <= bound
 
 
-@pytest.fixture(params=["auto", "1", "2", "4", "8"])
+@pytest.fixture(params=[(1, 128), (1, 192), (1, 256), (2, 128), (2, 192), (2, 256), (2, 512)], ids=lambda v: f"c{v[0]}b{v[1]}")
+def tile_mode(request):
+    """Forces one kernel variant: CTAs per tile (1, or a cta_group::2 pair) and tile width."""
+    keys = ("CCL_GEMM_CTAS", "CCL_GEMM_BN")
+    old = {k: os.environ.pop(k, None) for k in keys}
+    os.environ["CCL_GEMM_CTAS"], os.environ["CCL_GEMM_BN"] = str(request.param[0]), str(request.param[1])
+    yield request.param
+    for k in keys:
+        os.environ.pop(k, None)
+        if old[k] is not None:
+            os.environ[k] = old[k]
+
+
+@pytest.mark.parametrize("M,N,K,P,at,bt", [(520, 1536, 328, 4, 0, 0), (300, 2304, 512, 2, 0, 1), (512, 768, 192, 1, 1, 0),
+                                           (256, 3072, 1024, 4, 1, 1)])
+def test_gemm_every_tile_shape(M, N, K, P, at, bt, tile_mode):
+    """Each kernel variant on shapes with ragged tiles in M and N, several tiles per CTA and both operand majors."""
+    A, B = synth.gemm_operands(M, N, K, at, bt, seed=7, tag="tiles")
+    d = gemm_desc(M, N, K, P, ("row", "ccl", "ccl"), at, bt, 2, 1)
+    try:
+        ccl.ccl_gemm_workspace(d)
+    except ccl.CclError as e:                      # e.g. 192-wide pair tiles need a K-contiguous B
+        assert e.status == ccl.ERR_UNSUPPORTED
+        pytest.skip("variant not available for this operand layout")
+    check(d, A, B)
+
+
+@pytest.fixture(params=["auto", "1", "2", "4", "8", "2p", "4p"])
 def split_mode(request):
-    """Forces the number of K splits of the 1-CTA kernel (partial sums in the workspace, fixed-order reduction)."""
+    """Forces the number of K splits (partial sums in the workspace, fixed-order reduction); "2p", "4p": with CTA pairs."""
     keys = ("CCL_GEMM_SPLITK", "CCL_GEMM_CTAS")
     old = {k: os.environ.pop(k, None) for k in keys}
     if request.param != "auto":
-        os.environ["CCL_GEMM_SPLITK"] = request.param
-        os.environ["CCL_GEMM_CTAS"] = "1"
+        os.environ["CCL_GEMM_SPLITK"] = request.param.rstrip("p")
+        os.environ["CCL_GEMM_CTAS"] = "2" if request.param.endswith("p") else "1"
     yield request.param
     for k in keys:
         os.environ.pop(k, None)
@@ -264,7 +291,7 @@ def test_gemm_split_k(M, N, K, P, at, bt, split_mode):
         assert e.status == ccl.ERR_UNSUPPORTED
         pytest.skip("forced split count does not divide this K")
     if split_mode not in ("auto", "1"):
-        assert need == int(split_mode) * M * N * 4
+        assert need == int(split_mode.rstrip("p")) * M * N * 4
     got1, _ = check(d, A, B)
     got2, _ = check(d, A, B)
     np.testing.assert_array_equal(got1, got2)                          # fixed-order reduction: run-to-run identical

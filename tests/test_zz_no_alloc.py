@@ -6,7 +6,9 @@ ccl_gemm gives with a caller-provided workspace -- same kernels, same plan -- on
 that share the built-in scratch array, the second one a different problem that finds the first one's
 partial sums still lying there.
 """
+import contextlib
 import ctypes as C
+import os
 
 import numpy as np
 import pytest
@@ -17,6 +19,22 @@ from paper_2606_11718_b200 import synth
 from helpers import gemm_desc
 
 pytestmark = pytest.mark.gpu
+
+
+@contextlib.contextmanager
+def forced_split(n):
+    """Pins the plan to n K-splits of the 1-CTA kernel, so that the test does not depend on the planner's taste."""
+    keys = {"CCL_GEMM_SPLITK": str(n), "CCL_GEMM_CTAS": "1"}
+    old = {k: os.environ.get(k) for k in keys}
+    os.environ.update(keys)
+    try:
+        yield
+    finally:
+        for k, v in old.items():
+            if v is None:
+                os.environ.pop(k, None)
+            else:
+                os.environ[k] = v
 
 
 def via_existing_entry(d, a, b):
@@ -39,6 +57,11 @@ def via_no_alloc_entry(d, a, b):
 
 
 def test_static_workspace_entry_matches_ccl_gemm_on_two_calls_in_a_row():
+    with forced_split(4):
+        check_two_calls_in_a_row()
+
+
+def check_two_calls_in_a_row():
     problems = [(256, 768, 2048, 4, 1), (16, 1024, 4096, 2, 0)]          # M, N, K, P, b_trans: both get split along K
     expected, operands = [], []
     for M, N, K, P, bt in problems:
@@ -63,10 +86,11 @@ def test_static_workspace_entry_matches_ccl_gemm_on_two_calls_in_a_row():
 
 def test_static_workspace_entry_rejects_what_does_not_fit():
     d = gemm_desc(128, 8192, 28672, 4, ("row", "row", "row"), 0, 0, 2, 1)      # weight streaming, long K: 16 MB of partial sums
-    assert ccl.ccl_gemm_workspace(d) > ccl.GEMM_STATIC_WS_BYTES
-    rc = ccl.lib().ccl_gemm_static_ws(C.byref(d), C.c_void_p(256), C.c_void_p(512), C.c_void_p(1024), None)
-    assert rc == ccl.ERR_WORKSPACE
-    assert b"built-in scratch" in ccl.lib().ccl_last_error()
+    with forced_split(4):
+        assert ccl.ccl_gemm_workspace(d) > ccl.GEMM_STATIC_WS_BYTES
+        rc = ccl.lib().ccl_gemm_static_ws(C.byref(d), C.c_void_p(256), C.c_void_p(512), C.c_void_p(1024), None)
+        assert rc == ccl.ERR_WORKSPACE
+        assert b"built-in scratch" in ccl.lib().ccl_last_error()
     big = gemm_desc(1024, 1024, 1024, 1, ("row", "row", "row"), 0, 0, 0, 0)    # needs no workspace at all: runs as usual
     assert ccl.ccl_gemm_workspace(big) == 0
     A, B = synth.gemm_operands(1024, 1024, 1024, 0, 0, seed=8, tag="noalloc2")
