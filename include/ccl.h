@@ -144,6 +144,22 @@ ccl_status ccl_gemm_workspace(const ccl_gemm_desc* d, size_t* bytes);
 ccl_status ccl_gemm(const ccl_gemm_desc* d, const void* A_dev, const void* B_dev, void* C_dev, void* ws_dev,
                     size_t ws_bytes, void* cuda_stream);
 /*
+ * `batch` independent GEMMs of one shape and one set of layouts in a single launch, e.g. the expert
+ * projections of a mixture-of-experts FFN (Sec. 4.1 evaluates the Qwen expert GEMMs one at a time; the
+ * paper has no batched call: the batch only amortises the launch and fills the machine with small problems).
+ * Problem e (0 <= e < batch) reads A_dev + e*a_stride_bytes and B_dev + e*b_stride_bytes and writes
+ * C_dev + e*c_stride_bytes, each buffer laid out as `d` says; results are those of `batch` ccl_gemm calls,
+ * bit for bit.  A stride of 0 for A or B means every problem shares that operand.  Otherwise a stride must
+ * be a multiple of 16 bytes and at least ccl_buffer_bytes of the operand (CCL_ERR_ALIGN / CCL_ERR_INVALID_ARG);
+ * 1 <= batch <= 65536.  With batch = 1 the strides are ignored and the call equals ccl_gemm.
+ * Workspace: ccl_gemm_batched_workspace bytes (0 when the plan does not split K).  All buffers are the
+ * caller's; nothing is allocated.  Errors as for ccl_gemm, nothing launched on error.
+ */
+ccl_status ccl_gemm_batched_workspace(const ccl_gemm_desc* d, int32_t batch, size_t* bytes);
+ccl_status ccl_gemm_batched(const ccl_gemm_desc* d, int32_t batch, const void* A_dev, int64_t a_stride_bytes,
+                            const void* B_dev, int64_t b_stride_bytes, void* C_dev, int64_t c_stride_bytes,
+                            void* ws_dev, size_t ws_bytes, void* cuda_stream);
+/*
  * Synchronises `cuda_stream`, then reports and clears the status word of GEMMs finished on
  * the current device: CCL_OK, or CCL_ERR_TIMEOUT with *detail = the raw device code.
  * detail may be NULL.

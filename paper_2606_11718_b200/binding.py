@@ -20,7 +20,7 @@ PLACE_RR, PLACE_BLOCK, PLACE_BEST = 0, 1, 2
 ASSIGN_N_STRIPS, ASSIGN_M_STRIPS, ASSIGN_EXPLICIT = 0, 1, 2
 
 EXPORTS = ["ccl_map_offset", "ccl_map_inverse", "ccl_buffer_bytes", "ccl_strip_stride", "ccl_repack", "ccl_gemm_workspace",
-           "ccl_gemm", "ccl_gemm_static_ws", "ccl_gemm_status", "ccl_traffic_sizes", "ccl_traffic", "ccl_traffic_l2", "ccl_last_error", "ccl_launch_count", "ccl_version"]
+           "ccl_gemm", "ccl_gemm_batched_workspace", "ccl_gemm_batched", "ccl_gemm_static_ws", "ccl_gemm_status", "ccl_traffic_sizes", "ccl_traffic", "ccl_traffic_l2", "ccl_last_error", "ccl_launch_count", "ccl_version"]
 
 
 class CclError(RuntimeError):
@@ -73,6 +73,9 @@ def lib():
         l.ccl_repack.argtypes = [C.POINTER(Mat), C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]
         l.ccl_gemm_workspace.argtypes = [C.POINTER(GemmDesc), C.POINTER(C.c_size_t)]
         l.ccl_gemm.argtypes = [C.POINTER(GemmDesc), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+        l.ccl_gemm_batched_workspace.argtypes = [C.POINTER(GemmDesc), C.c_int32, C.POINTER(C.c_size_t)]
+        l.ccl_gemm_batched.argtypes = [C.POINTER(GemmDesc), C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64,
+                                       C.c_void_p, C.c_size_t, C.c_void_p]
         l.ccl_gemm_static_ws.argtypes = [C.POINTER(GemmDesc), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         l.ccl_gemm_status.argtypes = [C.c_void_p, C.POINTER(C.c_int32)]
         l.ccl_traffic_sizes.argtypes = [C.POINTER(TrafficDesc), C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
@@ -156,6 +159,21 @@ def ccl_gemm(d, A, B, Cout, ws=None):
             raise ValueError("ccl_gemm: operand buffer too small")
     ws_bytes = ws.numel() * ws.element_size() if ws is not None else 0
     _check(lib().ccl_gemm(C.byref(d), _ptr(A), _ptr(B), _ptr(Cout), _ptr(ws), ws_bytes, _stream()))
+
+
+def ccl_gemm_batched_workspace(d, batch):
+    n = C.c_size_t()
+    _check(lib().ccl_gemm_batched_workspace(C.byref(d), batch, C.byref(n)))
+    return n.value
+
+
+def ccl_gemm_batched(d, batch, A, a_stride, B, b_stride, Cout, c_stride, ws=None):
+    """`batch` GEMMs of one shape in one launch; X_stride: bytes between consecutive problems' buffers (0: shared A / B)."""
+    for t, m, st in ((A, d.A, a_stride), (B, d.B, b_stride), (Cout, d.C, c_stride)):
+        if t.numel() * t.element_size() < (batch - 1) * st + ccl_buffer_bytes(m):
+            raise ValueError("ccl_gemm_batched: operand buffer too small")
+    ws_bytes = ws.numel() * ws.element_size() if ws is not None else 0
+    _check(lib().ccl_gemm_batched(C.byref(d), batch, _ptr(A), a_stride, _ptr(B), b_stride, _ptr(Cout), c_stride, _ptr(ws), ws_bytes, _stream()))
 
 
 GEMM_STATIC_WS_BYTES = 8 * 1024 * 1024

@@ -89,6 +89,7 @@ struct OpMap {          // how stored coordinates (r, c) of an operand become te
     //   il_mode 0: strips stored one after the other     -> map {x, row, strip, 1}
     int32_t il_mode;
     FastDiv il_kr, il_sc;
+    int32_t batched;    // 1: each problem of a batch has its own buffer, 0: all problems share this operand
 };
 
 struct GemmParams {
@@ -102,6 +103,11 @@ struct GemmParams {
     // raster constants the host derives from the grid it launches (see Scheduler)
     int32_t sch_units, sch_gm, sch_gn, sch_upg, sch_floaters, sch_rounds, sch_per_group, sch_pool_per_group;
     FastDiv fd_upg, fd_groups, fd_splits, fd_per_panel, fd_panel, fd_tps_m, fd_tps_n;
+    // batch of independent problems of one shape (ccl_gemm_batched): the tile walk of a group runs through its
+    // tiles of problem 0, then of problem 1, ...; problem e is coordinate e of every tensor map's last dimension
+    int32_t batch;
+    FastDiv fd_tiles_per_problem;   // tiles of one problem inside one group
+    int64_t c_batch_stride;         // elements between the C buffers of consecutive problems
     OpMap a, b;
     int32_t a_mn, b_mn;             // 1 = MN-major operand tile in shared memory
     OpMap c;                        // C addressed through its own map as well (TMA tile stores)
@@ -170,17 +176,17 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
 // TMA tile load whose completion bytes are credited to `bar_addr` (a shared::cluster address; with two
 // CTAs this is the leader's barrier, which the cta_group::2 form of the copy is allowed to signal).
 template <int CTAS>
-__device__ __forceinline__ void tma_load(void* smem_dst, const CUtensorMap* map, uint32_t bar_addr, int c0, int c1, int c2, int c3) {
+__device__ __forceinline__ void tma_load(void* smem_dst, const CUtensorMap* map, uint32_t bar_addr, int c0, int c1, int c2, int c3, int c4) {
     if (CTAS == 1)
-        asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-                     ::"r"(smem_u32(smem_dst)), "l"(map), "r"(bar_addr), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+        asm volatile("cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+                     ::"r"(smem_u32(smem_dst)), "l"(map), "r"(bar_addr), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4) : "memory");
     else
-        asm volatile("cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-                     ::"r"(smem_u32(smem_dst)), "l"(map), "r"(bar_addr), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+        asm volatile("cp.async.bulk.tensor.5d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+                     ::"r"(smem_u32(smem_dst)), "l"(map), "r"(bar_addr), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4) : "memory");
 }
-__device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, const void* smem_src, int c0, int c1, int c2, int c3) {
-    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
-                 ::"l"(map), "r"(smem_u32(smem_src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+__device__ __forceinline__ void tma_store_5d(const CUtensorMap* map, const void* smem_src, int c0, int c1, int c2, int c3, int c4) {
+    asm volatile("cp.async.bulk.tensor.5d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5, %6}], [%1];"
+                 ::"l"(map), "r"(smem_u32(smem_src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4) : "memory");
 }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile(
@@ -203,7 +209,7 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint3
     return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) | (1ull << 46) | (2ull << 61);
 }
 
-// Stored coordinates (r, c) of an operand -> coordinates of its rank-4 tensor map.
+// Stored coordinates (r, c) of an operand -> the first four coordinates of its tensor map (the fifth is the problem of a batch).
 __device__ __forceinline__ void to_coords(const OpMap& o, int r, int c, int& x, int& y, int& z, int& u) {
     int g, rr, xx;                                   // strip, row inside the strip, column inside the strip row
     if (o.split == 2) { o.w.divmod(c, g, xx); rr = r; }
@@ -223,7 +229,7 @@ __device__ __forceinline__ int64_t c_offset(const GemmParams& p, int64_t m, int6
     return g * p.c_stride + o;
 }
 
-struct TileCoord { int m0, m1, n0, n1, split; };
+struct TileCoord { int m0, m1, n0, n1, split, e; };   // e: problem of the batch
 
 // Tiles of this CTA (pair).  The schedulable units (CTAs, or CTA pairs) serve `groups` strip ranges
 // (chiplet-grouped raster): group g owns the tiles of strip range g and walks them in panels of
@@ -258,6 +264,8 @@ struct Scheduler {
         }
         t.split = 0;
         if (p.splits > 1) { int ii; p.fd_splits.divmod(i, ii, t.split); i = ii; }   // the splits of one tile are neighbours in the walk
+        t.e = 0;
+        if (p.batch > 1) { int ii; p.fd_tiles_per_problem.divmod(i, t.e, ii); i = ii; }
         int pn, rem;
         p.fd_per_panel.divmod(i, pn, rem);
         const bool tail = gm - pn * p.panel < p.panel;   // the last panel may be lower
@@ -379,7 +387,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 if (ksplit) { if (mn) to_coords(om, k0, base, x, y, z, u); else to_coords(om, base, k0, x, y, z, u); }
                 else if (mn) y = k0; else x = k0;
                 if (lane == 0 && it == 0 && kb == kb0) CCL_TRACE(13);
-                if (active) tma_load<CTAS>(smem + (size_t)stage * stage_bytes + soff, map, full0 + (uint32_t)stage * 8u, x, y, z, u);
+                if (active) tma_load<CTAS>(smem + (size_t)stage * stage_bytes + soff, map, full0 + (uint32_t)stage * 8u, x, y, z, u, t.e * om.batched);
                 if (lane == 0 && it == 0 && kb == kb0) CCL_TRACE(2);
                 CCL_TRACE2(lane == 0 && it == 0 && kb - kb0 < 16, 64 + (kb - kb0) * 2 + 1);
                 if (++stage == stages) { stage = 0; phase ^= 1; }
@@ -492,7 +500,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     if (lane == 0) {
                         int cx = cx0 + c * 64, cy = cy0, cz = cz0, cu = cu0;
                         if (c_chunked) to_coords(p.c, row0, n64, cx, cy, cz, cu);
-                        tma_store_4d(&map_c, buf, cx, cy, cz, cu);
+                        tma_store_5d(&map_c, buf, cx, cy, cz, cu, t.e);
                         tma_store_commit();
                     }
                     CCL_TRACE2(warp == 2 && lane == 0 && epi_count < 12, epi_count * 5 + 4);
@@ -500,14 +508,14 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     return;
                 }
                 // a 64-column piece of a row is contiguous in every layout the GEMM accepts
-                const int64_t piece_off = p.splits > 1 || m >= t.m1 ? 0 : c_offset(p, m, n64);
+                const int64_t piece_off = p.splits > 1 || m >= t.m1 ? 0 : c_offset(p, m, n64) + (int64_t)t.e * p.c_batch_stride;
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
                     const uint32_t* rr = &r[half * 32];
                     const int n32 = n64 + half * 32;
                     if (p.splits > 1) {                  // partial sums, summed in fixed order by splitk_reduce_kernel
                         if (m < t.m1) {
-                            float* wrow = p.ws + ((int64_t)t.split * p.M + m) * (int64_t)p.N;
+                            float* wrow = p.ws + (((int64_t)t.e * p.splits + t.split) * p.M + m) * (int64_t)p.N;
 #pragma unroll
                             for (int j = 0; j < 8; ++j) {
                                 const int n = n32 + j * 4;
@@ -582,19 +590,20 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 // Split-K epilogue: C = bf16( ws[0] + ws[1] + ... + ws[splits-1] ), the sum taken in that fixed order so
 // the result is the same on every run.  One thread per 8 consecutive columns of a row.
 __global__ void __launch_bounds__(256) splitk_reduce_kernel(const GemmParams p) {
-    const int64_t n8 = p.N / 8, total = (int64_t)p.M * n8;
+    const int64_t n8 = p.N / 8, per_problem = (int64_t)p.M * n8, total = per_problem * p.batch;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t m = i / n8, n = (i - m * n8) * 8;
+        const int64_t e = i / per_problem, r = i - e * per_problem;
+        const int64_t m = r / n8, n = (r - m * n8) * 8;
         float acc[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) acc[j] = 0.0f;
         for (int sp = 0; sp < p.splits; ++sp) {
-            const float4* src = reinterpret_cast<const float4*>(p.ws + ((int64_t)sp * p.M + m) * (int64_t)p.N + n);
+            const float4* src = reinterpret_cast<const float4*>(p.ws + ((e * p.splits + sp) * p.M + m) * (int64_t)p.N + n);
             const float4 x = src[0], y = src[1];
             acc[0] += x.x; acc[1] += x.y; acc[2] += x.z; acc[3] += x.w;
             acc[4] += y.x; acc[5] += y.y; acc[6] += y.z; acc[7] += y.w;
         }
-        const int64_t off = c_offset(p, m, n);
+        const int64_t off = c_offset(p, m, n) + e * p.c_batch_stride;
         uint4 v;
         __nv_bfloat162 h;
         h = __floats2bfloat162_rn(acc[0], acc[1]); v.x = *reinterpret_cast<uint32_t*>(&h);
@@ -671,7 +680,7 @@ static ccl_status merge_width(int64_t* cur, int64_t w, const char* dim) {
 static int64_t padded(int64_t w, int64_t b) { return (w + b - 1) / b * b; }
 
 // units = schedulable CTAs (1-CTA kernel) or CTA pairs (2-CTA kernel) the device can hold at once
-static ccl_status make_plan(const ccl_gemm_desc* d, const void* A, const void* B, const void* C, int sms, int pairs, GemmPlan* plan) {
+static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, const void* A, const void* B, const void* C, int sms, int pairs, GemmPlan* plan) {
     if (!d) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: NULL descriptor");
     if (d->M <= 0 || d->N <= 0 || d->K <= 0) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: M, N, K must be positive");
     if (d->M >= (INT64_C(1) << 31) || d->N >= (INT64_C(1) << 31) || d->K >= (INT64_C(1) << 31)) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: dimension too large");
@@ -745,7 +754,7 @@ static ccl_status make_plan(const ccl_gemm_desc* d, const void* A, const void* B
             if (b == 192 && (c == 2 ? no_192_pair : no_192)) continue;
             if (force_bn && atoi(force_bn) != b) continue;
             const int64_t tiles_m_all = strips_m * ((Wm + BM * c - 1) / (BM * c));
-            const int64_t tiles = tiles_m_all * strips_n * ((Wn + b - 1) / b);
+            const int64_t tiles = tiles_m_all * strips_n * ((Wn + b - 1) / b) * batch;
             double t_kb = b == 512 ? 1050.0 : (c == 1 && b == 256 ? 680.0 : (c == 1 ? 570.0 : 620.0));
             if (tiles_m_all == 1) t_kb = std::max(t_kb, (double)(b / c) * (BK * 2) / 27.0);
             const double t_drain = b == 512 ? 7000.0 : 1500.0;
@@ -757,7 +766,7 @@ static ccl_status make_plan(const ccl_gemm_desc* d, const void* A, const void* B
                 if (sp_eff != sp) continue;
                 const int64_t waves = (tiles * sp + units - 1) / units;
                 double cost = (double)waves * ((double)kbps * t_kb + (sp > 1 ? 2.0 * t_drain : t_drain)) + 3000.0;
-                if (sp > 1) cost += ((double)sp + 0.5) * (double)d->M * (double)d->N * 4.0 / 3400.0 + 14000.0;
+                if (sp > 1) cost += ((double)sp + 0.5) * (double)batch * (double)d->M * (double)d->N * 4.0 / 3400.0 + 14000.0;
                 if (best < 0 || cost < best) { best = cost; ctas = c; bn = b; splits = sp; }
             }
         }
@@ -767,7 +776,7 @@ static ccl_status make_plan(const ccl_gemm_desc* d, const void* A, const void* B
     plan->subn = subn;
     const int bm = BM * ctas;
     plan->bn = bn; plan->ctas = ctas;
-    plan->ws_bytes = splits > 1 ? (size_t)splits * (size_t)d->M * (size_t)d->N * 4 : 0;
+    plan->ws_bytes = splits > 1 ? (size_t)batch * (size_t)splits * (size_t)d->M * (size_t)d->N * 4 : 0;
 
     GemmParams& p = plan->p;
     std::memset(&p, 0, sizeof(p));
@@ -792,7 +801,8 @@ static ccl_status make_plan(const ccl_gemm_desc* d, const void* A, const void* B
     p.a_bytes = BM * BK * 2; p.stage_bytes = p.a_bytes + (uint32_t)(bn / ctas) * BK * 2;
     p.stages = (int32_t)(kSmemBudget / p.stage_bytes);
     if (p.stages > 8) p.stages = 8;
-    int64_t ntiles = (int64_t)p.tiles_m * p.tiles_n * splits;
+    int64_t ntiles = (int64_t)p.tiles_m * p.tiles_n * splits * batch;
+    p.batch = (int32_t)batch;
     int units = (int)std::min<int64_t>(ntiles, ctas == 2 ? pairs : sms);
     plan->grid = (unsigned)(units * ctas);
     // grouped raster needs at least one unit per group and whole strips per group
@@ -803,7 +813,8 @@ static ccl_status make_plan(const ccl_gemm_desc* d, const void* A, const void* B
         if (ntiles >= (INT64_C(1) << 31) - 2 * units) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: too many tiles");
         const int gm = p.group_dim == 1 && p.groups > 1 ? p.tiles_m / p.groups : p.tiles_m;
         const int gn = p.group_dim == 0 && p.groups > 1 ? p.tiles_n / p.groups : p.tiles_n;
-        const int64_t per_group = (int64_t)gm * gn * splits;
+        const int64_t per_group = (int64_t)gm * gn * splits * batch;
+        p.fd_tiles_per_problem = make_fastdiv((int64_t)gm * gn);
         const int upg = units / p.groups;
         const int64_t rounds = std::min(per_group * p.groups / units, per_group / upg);
         p.sch_units = units; p.sch_gm = gm; p.sch_gn = gn; p.sch_upg = upg; p.sch_floaters = units - upg * p.groups;
@@ -831,20 +842,22 @@ static ccl_status make_plan(const ccl_gemm_desc* d, const void* A, const void* B
     return CCL_OK;
 }
 
-// Rank-4 tensor map of an operand (coordinates as to_coords() produces them), for boxes of box_inner contiguous
-// elements by box_rows strip rows:
+// Rank-5 tensor map of an operand (four coordinates as to_coords() produces them, then the problem of a batch), for
+// boxes of box_inner contiguous elements by box_rows strip rows:
 //   strips one after the other : {strip row extent, rows per strip, strips, 1}
 //   interleaved, mode 1        : {strip row extent, rows per chunk kr, strips, chunk index}; a box of more than kr
 //                                rows takes kr rows from each of box_rows / kr consecutive chunks of its strip
 //   interleaved, mode 2        : {chunk extent, chunks per strip row, rows per strip, strips}
-static ccl_status operand_tmap(CUtensorMap* m, const MatView& v, const void* base, uint32_t box_inner, uint32_t box_rows) {
+static ccl_status operand_tmap(CUtensorMap* m, const MatView& v, const void* base, uint32_t box_inner, uint32_t box_rows, int64_t batch, int64_t batch_stride_bytes) {
     const uint64_t row = (uint64_t)(v.split == 2 ? v.w : v.cols);      // elements of a strip row
     const uint64_t R = (uint64_t)(v.split == 1 ? v.h : v.rows);        // rows per strip
     const uint64_t S = (uint64_t)v.nstrips, sc = (uint64_t)v.ichunk;
-    uint64_t dims[4], strides[3];
-    uint32_t box[4];
+    uint64_t dims[5], strides[4];
+    uint32_t box[5];
     int64_t kr;
     const int mode = interleave_mode(v, &kr);
+    // last dimension: the problems of a batch (a single entry when the operand is not batched)
+    dims[4] = batch > 1 && batch_stride_bytes ? (uint64_t)batch : 1; box[4] = 1;
     if (mode == 1) {
         const uint64_t k = (uint64_t)kr;
         dims[0] = row; dims[1] = k; dims[2] = S; dims[3] = (R + k - 1) / k;
@@ -862,7 +875,8 @@ static ccl_status operand_tmap(CUtensorMap* m, const MatView& v, const void* bas
         strides[0] = row * 2; strides[1] = v.split ? (uint64_t)v.stride * 2 : row * 2; strides[2] = strides[1];
         box[0] = box_inner; box[1] = box_rows; box[2] = 1; box[3] = 1;
     } else return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: this page-interleaved layout has no tensor map");
-    return encode_tmap(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B);
+    strides[3] = dims[4] > 1 ? (uint64_t)batch_stride_bytes : strides[0];
+    return encode_tmap(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, base, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
 template <int BN, int CTAS>
@@ -921,7 +935,7 @@ using namespace ccl;
 
 // ---- host-side cache of prepared calls (plan + encoded tensor maps) --------------------------------------
 struct PreparedKey {
-    int64_t f[32];          // every field of the descriptor, the three pointers, the device and the tuning overrides
+    int64_t f[36];          // every field of the descriptor, the batch, the three pointers, the device and the tuning overrides
     int dev;
     char env[60];
 };
@@ -940,8 +954,9 @@ static std::mutex g_prepared_mutex;
 static void put_mat(const ccl_mat& m, int64_t* f) {
     f[0] = m.rows; f[1] = m.cols; f[2] = m.elem_bytes; f[3] = m.P; f[4] = m.part; f[5] = m.layout; f[6] = m.strip_align_bytes;
 }
-static void make_key(const ccl_gemm_desc* d, const void* A, const void* B, const void* C, PreparedKey* k) {
+static void make_key(const ccl_gemm_desc* d, const int64_t* batch4, const void* A, const void* B, const void* C, PreparedKey* k) {
     std::memset(k, 0, sizeof(*k));
+    for (int i = 0; i < 4; ++i) k->f[32 + i] = batch4[i];          // batch, strides of A, B, C
     k->f[0] = d->M; k->f[1] = d->N; k->f[2] = d->K;
     put_mat(d->A, k->f + 3); put_mat(d->B, k->f + 10); put_mat(d->C, k->f + 17);
     k->f[24] = d->a_trans; k->f[25] = d->b_trans; k->f[26] = d->out_part; k->f[27] = d->P; k->f[28] = d->grouped_raster;
@@ -969,26 +984,35 @@ static void device_units(int* sms, int* pairs) {
     }
 }
 
-extern "C" ccl_status ccl_gemm_workspace(const ccl_gemm_desc* d, size_t* bytes) {
+constexpr int64_t kMaxBatch = 65536;
+
+static ccl_status workspace_impl(const ccl_gemm_desc* d, int64_t batch, size_t* bytes) {
+    if (batch < 1 || batch > kMaxBatch) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: batch must be in [1, %lld]", (long long)kMaxBatch);
     GemmPlan plan;
-    ccl_status s = make_plan(d, nullptr, nullptr, nullptr, 148, 74, &plan);     // validation without any CUDA call
+    ccl_status s = make_plan(d, batch, nullptr, nullptr, nullptr, 148, 74, &plan);     // validation without any CUDA call
     if (s) return s;
     if (!bytes) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm_workspace: NULL output");
     int sms, pairs;
     device_units(&sms, &pairs);
-    if ((s = make_plan(d, nullptr, nullptr, nullptr, sms, pairs, &plan))) return s;
+    if ((s = make_plan(d, batch, nullptr, nullptr, nullptr, sms, pairs, &plan))) return s;
     *bytes = plan.ws_bytes;
     return CCL_OK;
 }
 
-extern "C" ccl_status ccl_gemm(const ccl_gemm_desc* d, const void* A_dev, const void* B_dev, void* C_dev, void* ws_dev,
-                               size_t ws_bytes, void* cuda_stream) {
+extern "C" ccl_status ccl_gemm_workspace(const ccl_gemm_desc* d, size_t* bytes) { return workspace_impl(d, 1, bytes); }
+extern "C" ccl_status ccl_gemm_batched_workspace(const ccl_gemm_desc* d, int32_t batch, size_t* bytes) { return workspace_impl(d, batch, bytes); }
+
+// strides[X]: bytes between the buffers of operand X (A, B, C) of consecutive problems; 0 = shared (A and B only)
+static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, const int64_t* strides, const void* A_dev, const void* B_dev, void* C_dev,
+                            void* ws_dev, size_t ws_bytes, void* cuda_stream) {
     if (!A_dev || !B_dev || !C_dev) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: NULL operand");
     if (!d) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: NULL descriptor");
+    if (batch < 1 || batch > kMaxBatch) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: batch must be in [1, %lld]", (long long)kMaxBatch);
+    const int64_t batch4[4] = {batch, batch > 1 ? strides[0] : 0, batch > 1 ? strides[1] : 0, batch > 1 ? strides[2] : 0};
     // Repeated calls with the same descriptor and buffers (the normal case in a training / serving loop)
     // reuse the plan and the two encoded tensor maps: a host-side cache only, nothing is kept on the device.
     PreparedKey key;
-    make_key(d, A_dev, B_dev, C_dev, &key);
+    make_key(d, batch4, A_dev, B_dev, C_dev, &key);
     Prepared prep;
     bool hit = false;
     {
@@ -999,20 +1023,33 @@ extern "C" ccl_status ccl_gemm(const ccl_gemm_desc* d, const void* A_dev, const 
     ccl_status s;
     if (!hit) {
         GemmPlan& plan = prep.plan;
-        s = make_plan(d, A_dev, B_dev, C_dev, 148, 74, &plan);     // validation first: no CUDA call on bad input
+        s = make_plan(d, batch, A_dev, B_dev, C_dev, 148, 74, &plan);     // validation first: no CUDA call on bad input
         if (s) return s;
+        if (batch > 1) {
+            const MatView* views[3] = {&plan.va, &plan.vb, &plan.vc};
+            const char* names[3] = {"A", "B", "C"};
+            for (int X = 0; X < 3; ++X) {
+                const int64_t st = batch4[1 + X], need = buffer_elems(*views[X]) * 2;
+                if (st == 0 && X < 2) continue;                     // an operand every problem shares
+                if (st < need) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm_batched: stride of %s (%lld bytes) is smaller than its buffer (%lld bytes)", names[X], (long long)st, (long long)need);
+                if (st % 16) return fail(CCL_ERR_ALIGN, "ccl_gemm_batched: stride of %s is not a multiple of 16 bytes", names[X]);
+                if (st >= (INT64_C(1) << 40)) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm_batched: stride of %s too large for a tensor map", names[X]);
+            }
+        }
         int dev;
         CCL_CUDA_TRY(cudaGetDevice(&dev));
         CCL_CUDA_TRY(cudaDeviceGetAttribute(&prep.sms, cudaDevAttrMultiProcessorCount, dev));
-        if (dev != key.dev) make_key(d, A_dev, B_dev, C_dev, &key);
-        if ((s = make_plan(d, A_dev, B_dev, C_dev, prep.sms, resident_pairs(), &plan))) return s;
+        if (dev != key.dev) make_key(d, batch4, A_dev, B_dev, C_dev, &key);
+        if ((s = make_plan(d, batch, A_dev, B_dev, C_dev, prep.sms, resident_pairs(), &plan))) return s;
         plan.p.C = static_cast<uint16_t*>(C_dev);
+        plan.p.a.batched = batch4[1] != 0; plan.p.b.batched = batch4[2] != 0; plan.p.c.batched = 1;
+        plan.p.c_batch_stride = batch4[3] / 2;
         const uint32_t bnh = (uint32_t)(plan.subn / plan.ctas);   // B rows of one K-major box
-        if (!plan.p.a_mn) s = operand_tmap(&prep.ma, plan.va, A_dev, BK, BM); else s = operand_tmap(&prep.ma, plan.va, A_dev, 64, BK);
+        if (!plan.p.a_mn) s = operand_tmap(&prep.ma, plan.va, A_dev, BK, BM, batch, batch4[1]); else s = operand_tmap(&prep.ma, plan.va, A_dev, 64, BK, batch, batch4[1]);
         if (s) return s;
-        if (!plan.p.b_mn) s = operand_tmap(&prep.mb, plan.vb, B_dev, BK, bnh); else s = operand_tmap(&prep.mb, plan.vb, B_dev, 64, BK);
+        if (!plan.p.b_mn) s = operand_tmap(&prep.mb, plan.vb, B_dev, BK, bnh, batch, batch4[2]); else s = operand_tmap(&prep.mb, plan.vb, B_dev, 64, BK, batch, batch4[2]);
         if (s) return s;
-        if ((s = operand_tmap(&prep.mc, plan.vc, C_dev, 64, 32))) return s;            // C: 64-column x 32-row store boxes
+        if ((s = operand_tmap(&prep.mc, plan.vc, C_dev, 64, 32, batch, batch4[3]))) return s;   // C: 64-column x 32-row store boxes
         prep.key = key; prep.valid = true;
         std::lock_guard<std::mutex> lock(g_prepared_mutex);
         g_prepared[g_prepared_next] = prep;
@@ -1037,13 +1074,27 @@ extern "C" ccl_status ccl_gemm(const ccl_gemm_desc* d, const void* A_dev, const 
     else s = launch<128, 1>(plan, ma, mb, mc, st);
     if (s) return s;
     if (plan.p.splits > 1) {
-        int64_t work = (int64_t)plan.p.M * (plan.p.N / 8);
+        int64_t work = (int64_t)plan.p.batch * plan.p.M * (plan.p.N / 8);
         unsigned grid = (unsigned)std::max<int64_t>(1, std::min<int64_t>((work + 255) / 256, (int64_t)sms * 8));
         splitk_reduce_kernel<<<grid, 256, 0, st>>>(plan.p);
         count_launch();
         CCL_CUDA_TRY(cudaGetLastError());
     }
     return CCL_OK;
+}
+
+extern "C" ccl_status ccl_gemm(const ccl_gemm_desc* d, const void* A_dev, const void* B_dev, void* C_dev, void* ws_dev,
+                               size_t ws_bytes, void* cuda_stream) {
+    const int64_t none[3] = {0, 0, 0};
+    return gemm_impl(d, 1, none, A_dev, B_dev, C_dev, ws_dev, ws_bytes, cuda_stream);
+}
+
+extern "C" ccl_status ccl_gemm_batched(const ccl_gemm_desc* d, int32_t batch, const void* A_dev, int64_t a_stride_bytes, const void* B_dev,
+                                       int64_t b_stride_bytes, void* C_dev, int64_t c_stride_bytes, void* ws_dev, size_t ws_bytes,
+                                       void* cuda_stream) {
+    if (a_stride_bytes < 0 || b_stride_bytes < 0 || c_stride_bytes < 0) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm_batched: negative stride");
+    const int64_t strides[3] = {a_stride_bytes, b_stride_bytes, c_stride_bytes};
+    return gemm_impl(d, batch, strides, A_dev, B_dev, C_dev, ws_dev, ws_bytes, cuda_stream);
 }
 
 extern "C" ccl_status ccl_gemm_status(void* cuda_stream, int32_t* detail) {

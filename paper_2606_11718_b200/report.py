@@ -210,7 +210,7 @@ def main():
         rows = []
         for g in gemms:
             big = g["M"] * g["N"] * g["K"] > 1e11
-            r = run_gemm(g, pk, 3 if (big or args.quick) else 20)
+            r = run_gemm(g, pk, 3 if (big or args.quick) else 100)
             rows.append(r)
             c, rw = r.get("ccl_grouped", {}), r.get("row_plain", {})
             t = r["traffic"]
