@@ -202,6 +202,7 @@ def main():
     ap.add_argument("--config", default="all")
     ap.add_argument("--out", default=os.path.join(ROOT, "report_out"))
     ap.add_argument("--quick", action="store_true", help="fewer repetitions and P = 4 only in the sweep")
+    ap.add_argument("--only", default=None, help="run only the GEMMs whose name contains this text (e.g. for a profiler capture)")
     args = ap.parse_args()
     assert torch.cuda.is_available(), "report needs a CUDA device"
     pk = peaks()
@@ -209,6 +210,8 @@ def main():
     for cfg, gemms in configs(args.config, args.quick).items():
         rows = []
         for g in gemms:
+            if args.only and args.only not in g["name"]:
+                continue
             big = g["M"] * g["N"] * g["K"] > 1e11
             r = run_gemm(g, pk, 3 if (big or args.quick) else 100)
             rows.append(r)
