@@ -28,6 +28,7 @@
 //                   worked example, reshape/permute, slice sizes of Sec. 2.2)
 //   repack        : pinned (permutation, round trip, strided-slice copies)
 //   gemm          : pinned (identity, all-ones, library matmul, fp64 bound)
+//   gemm_swiglu   : pinned (gate/up pairing enumerated by hand, silu closed forms, numpy in float64)
 //   traffic       : pinned by invariants, closed forms and a hand-enumerated
 //                   tiny case; against the paper's Fig. 6 ratios it is
 //                   PARITY UNPINNED (they need the unreleased L2 simulator).
@@ -37,6 +38,7 @@
 #include <cstdint>
 #include <cstring>
 #include <cstdlib>
+#include <cmath>
 #include <vector>
 #include <thread>
 #include <algorithm>
@@ -419,6 +421,30 @@ int orc_gemm(int64_t M, int64_t N, int64_t K, const uint16_t* A, int a_trans, co
 }
 
 uint16_t orc_f32_to_bf16(float f) { return f32_to_bf16_rne(f); }
+
+// Gated FFN activation on the product of a fused gate/up operand (the operand of Fig. 3; Sec. 3.3: activations are
+// produced directly by upstream kernels).  H = A*B is [M x N], N even, its columns cut into P strips of width
+// Wp = N/P (P = 1: one strip); strip g holds gate columns in its first half and up columns in its second half.
+//   out[m][g*Wp/2 + j] = silu(H[m][g*Wp + j]) * H[m][g*Wp + Wp/2 + j],  0 <= j < Wp/2,  silu(x) = x / (1 + exp(-x)).
+// H is the fp32 sequential-k sum of orc_gemm; silu and the product are evaluated in double from that fp32 value and
+// rounded once to fp32 (ref32) and to bf16 (out_bf16).  The standard definition of the activation is used; the paper
+// does not define one.
+int orc_gemm_swiglu(int64_t M, int64_t N, int64_t K, int64_t P, const uint16_t* A, int a_trans, const uint16_t* B, int b_trans,
+                    float* ref32, uint16_t* out_bf16, int threads) {
+    if (M <= 0 || N <= 0 || K <= 0 || P < 1 || N % P || (N / P) % 2) return -1;
+    std::vector<float> H((size_t)(M * N));
+    if (orc_gemm(M, N, K, A, a_trans, B, b_trans, 0, M, 0, N, H.data(), nullptr, nullptr, threads)) return -1;
+    const int64_t Wp = N / P, half = Wp / 2, No = N / 2;
+    for (int64_t m = 0; m < M; ++m)
+        for (int64_t g = 0; g < P; ++g)
+            for (int64_t j = 0; j < half; ++j) {
+                const double x = (double)H[(size_t)(m * N + g * Wp + j)], u = (double)H[(size_t)(m * N + g * Wp + half + j)];
+                const float v = (float)(x / (1.0 + std::exp(-x)) * u);
+                if (ref32) ref32[m * No + g * half + j] = v;
+                if (out_bf16) out_bf16[m * No + g * half + j] = f32_to_bf16_rne(v);
+            }
+    return 0;
+}
 
 // Number of output tiles and of pages per operand.
 int orc_traffic_sizes(const orc_traffic_desc* d, int64_t* ntiles, int64_t* pages) {
