@@ -160,6 +160,21 @@ ccl_status ccl_gemm_batched(const ccl_gemm_desc* d, int32_t batch, const void* A
                             const void* B_dev, int64_t b_stride_bytes, void* C_dev, int64_t c_stride_bytes,
                             void* ws_dev, size_t ws_bytes, void* cuda_stream);
 /*
+ * GEMM on a fused gate/up weight with the gated activation applied in the epilogue, so that the activation the
+ * next GEMM consumes is produced directly in its layout (Sec. 3.3: activations are "produced directly by upstream
+ * kernels in CCL layout"; Fig. 3 shows the fused up/gate operand and its per-chiplet strips).  The activation
+ * itself, silu(x) = x / (1 + exp(-x)), is the standard one of these FFNs; the paper does not define it.
+ *   H[M x N] = A * B as in ccl_gemm (fp32 accumulation), N even.  The N columns form S strips of width Wp = N/S,
+ *   S = d->P if d->out_part == CCL_PART_COLS and d->P > 1, else S = 1; a strip holds its gate columns in its first
+ *   half and its up columns in its second half.
+ *   C[m][g*Wp/2 + j] = bf16( silu(H[m][g*Wp + j]) * H[m][g*Wp + Wp/2 + j] ),  0 <= j < Wp/2  (fp32, one rounding).
+ * d->A and d->B describe the operands as for ccl_gemm; d->C describes the OUTPUT, [M x N/2].  If B is in CCL split
+ * along N its strips must be these S strips (width Wp), if C is in CCL split along its columns, strips of Wp/2;
+ * Wp/2 a multiple of 8.  Page-interleaved operands -> CCL_ERR_UNSUPPORTED.  No workspace (K is never split).
+ * Other requirements, asynchrony, bounded waits and errors as for ccl_gemm.
+ */
+ccl_status ccl_gemm_swiglu(const ccl_gemm_desc* d, const void* A_dev, const void* B_dev, void* C_dev, void* cuda_stream);
+/*
  * Synchronises `cuda_stream`, then reports and clears the status word of GEMMs finished on
  * the current device: CCL_OK, or CCL_ERR_TIMEOUT with *detail = the raw device code.
  * detail may be NULL.

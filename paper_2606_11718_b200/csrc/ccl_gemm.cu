@@ -107,12 +107,17 @@ struct GemmParams {
     // tiles of problem 0, then of problem 1, ...; problem e is coordinate e of every tensor map's last dimension
     int32_t batch;
     FastDiv fd_tiles_per_problem;   // tiles of one problem inside one group
+    // gated activation (ccl_gemm_swiglu): N, Wn and the tile walk refer to the OUTPUT columns; the accumulators of a
+    // tile hold the gate columns (sub-tile 0) and the up columns (sub-tile 1) of the same outputs, pair_dist B columns
+    // apart inside a strip of 2 * pair_dist
+    int32_t pair_dist;
+    FastDiv fd_wn;
     int64_t c_batch_stride;         // elements between the C buffers of consecutive problems
     OpMap a, b;
     int32_t a_mn, b_mn;             // 1 = MN-major operand tile in shared memory
     OpMap c;                        // C addressed through its own map as well (TMA tile stores)
-    int32_t c_split;
-    int64_t c_w, c_h, c_stride, c_cols, c_ichunk, c_nstrips;
+    int64_t c_row, c_stride, c_ichunk, c_nstrips;   // C: elements of a strip row, between strips, per chunk; strips
+    int32_t c_cpr;                  // page-interleaved C whose strip rows span chunks: chunks per strip row
     uint16_t* C;
     uint32_t idesc;
     int32_t stages;
@@ -199,7 +204,20 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
           "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr) : "memory");
 }
+// 16-byte global store under a predicate, without a branch: the epilogue's TMEM loads and waits are warp-wide
+// (.sync.aligned) and must never be reached by a warp that the compiler has split by a per-lane row test.
+__device__ __forceinline__ void st_global_v4_if(void* ptr, uint4 v, bool pred) {
+    asm volatile("{\n .reg .pred q;\n setp.ne.b32 q, %5, 0;\n @q st.global.v4.b32 [%0], {%1, %2, %3, %4};\n}"
+                 ::"l"(ptr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w), "r"((uint32_t)pred) : "memory");
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// The loaded registers only hold their values once the wait above has run, but to the compiler they were defined by
+// the load statement: nothing stops it from moving an instruction that reads them above the wait.  Passing them
+// through an (empty) volatile statement placed after the wait makes every later use depend on that statement.
+__device__ __forceinline__ void tmem_regs_ready(uint32_t (&r)[64]) {
+    asm volatile("" : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]), "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31]));
+    asm volatile("" : "+r"(r[32]), "+r"(r[33]), "+r"(r[34]), "+r"(r[35]), "+r"(r[36]), "+r"(r[37]), "+r"(r[38]), "+r"(r[39]), "+r"(r[40]), "+r"(r[41]), "+r"(r[42]), "+r"(r[43]), "+r"(r[44]), "+r"(r[45]), "+r"(r[46]), "+r"(r[47]), "+r"(r[48]), "+r"(r[49]), "+r"(r[50]), "+r"(r[51]), "+r"(r[52]), "+r"(r[53]), "+r"(r[54]), "+r"(r[55]), "+r"(r[56]), "+r"(r[57]), "+r"(r[58]), "+r"(r[59]), "+r"(r[60]), "+r"(r[61]), "+r"(r[62]), "+r"(r[63]));
+}
 
 // Shared-memory matrix descriptor, SWIZZLE_128B, descriptor version 1 (sm_100).
 //   K-major : rows of 128 B (64 bf16 along K); 8-row groups every `sbo` bytes.
@@ -221,12 +239,21 @@ __device__ __forceinline__ void to_coords(const OpMap& o, int r, int c, int& x, 
 }
 // Element offset of C[m][n] in its buffer (any layout).
 __device__ __forceinline__ int64_t c_offset(const GemmParams& p, int64_t m, int64_t n) {
-    int64_t g = 0, o;
-    if (p.c_split == 2) { g = n / p.c_w; o = m * p.c_w + (n - g * p.c_w); }
-    else if (p.c_split == 1) { g = m / p.c_h; o = (m - g * p.c_h) * p.c_cols + n; }
-    else o = m * p.c_cols + n;
-    if (p.c_ichunk) { const int64_t j = o / p.c_ichunk; return (j * p.c_nstrips + g) * p.c_ichunk + (o - j * p.c_ichunk); }
-    return g * p.c_stride + o;
+    // (multiply-shift divisions only: a 64-bit division is a subroutine of several hundred cycles)
+    int g = 0, rr = (int)m, xx = (int)n;             // strip, row inside the strip, column inside the strip row
+    if (p.c.split == 2) p.c.w.divmod((int)n, g, xx);
+    else if (p.c.split == 1) p.c.h.divmod((int)m, g, rr);
+    if (p.c.il_mode == 1) {                          // a chunk holds il_kr whole strip rows
+        int j, y;
+        p.c.il_kr.divmod(rr, j, y);
+        return ((int64_t)j * p.c_nstrips + g) * p.c_ichunk + (int64_t)y * p.c_row + xx;
+    }
+    if (p.c.il_mode == 2) {                          // a strip row spans c_cpr whole chunks
+        int cj, x;
+        p.c.il_sc.divmod(xx, cj, x);
+        return (((int64_t)rr * p.c_cpr + cj) * p.c_nstrips + g) * p.c_ichunk + x;
+    }
+    return (int64_t)g * p.c_stride + (int64_t)rr * p.c_row + xx;
 }
 
 struct TileCoord { int m0, m1, n0, n1, split, e; };   // e: problem of the batch
@@ -283,7 +310,7 @@ struct Scheduler {
     }
 };
 
-template <int BN, int CTAS>
+template <int BN, int CTAS, bool SWIGLU = false>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                 const __grid_constant__ CUtensorMap map_c, const __grid_constant__ GemmParams gp) {
@@ -302,6 +329,8 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     constexpr int SUBN = BN / NSUB;
     constexpr int ACC_COLS = NSUB == 1 ? 256 : SUBN;  // TMEM columns between accumulators
     constexpr int NACC = NSUB == 1 ? 2 : NSUB;        // accumulator barriers in use
+    static_assert(!SWIGLU || NSUB == 2, "the gated activation pairs the two accumulators of a wide tile");
+    constexpr int TILE_N = SWIGLU ? SUBN : BN;        // tile width in the columns the tile walk counts (output columns)
     constexpr int SUBH = SUBN / CTAS;                // B columns of one sub-tile this CTA stages
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -334,7 +363,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     const uint32_t tmem_base = *tmem_ptr;
     if (threadIdx.x == 0) CCL_TRACE(1);
 
-    Scheduler sched(p, (int)(blockIdx.x / CTAS), BM * CTAS, BN);
+    Scheduler sched(p, (int)(blockIdx.x / CTAS), BM * CTAS, TILE_N);
     if (threadIdx.x == 0) CCL_TRACE(10);
 
     if (warp == 0) {
@@ -357,9 +386,11 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         const bool ksplit = (mn ? om.split == 1 : om.split == 2) || om.il_mode != 0;
         uint32_t soff;                                        // byte offset of the box inside a stage
         int off;                                              // offset of the box along M (A) or N (B) from the tile origin
+        int hsel = 0;                                         // sub-tile of a B box
         if (isA) { soff = mn ? (uint32_t)bi * (64 * BK * 2) : 0u; off = (int)rank * BM + (mn ? 64 * bi : 0); }
-        else if (mn) { const int h = bi / NC, c = bi - h * NC; soff = p.a_bytes + (uint32_t)(h * SUBH * BK * 2 + c * 64 * BK * 2); off = h * SUBN + (int)rank * SUBH + 64 * c; }
-        else { soff = p.a_bytes + (uint32_t)(bi * SUBH * BK * 2); off = bi * SUBN + (int)rank * SUBH; }
+        else if (mn) { const int h = bi / NC, c = bi - h * NC; hsel = h; soff = p.a_bytes + (uint32_t)(h * SUBH * BK * 2 + c * 64 * BK * 2); off = h * SUBN + (int)rank * SUBH + 64 * c; }
+        else { hsel = bi; soff = p.a_bytes + (uint32_t)(bi * SUBH * BK * 2); off = bi * SUBN + (int)rank * SUBH; }
+        if (SWIGLU && !isA) off -= hsel * SUBN;               // sub-tile 1 is not 256 columns on but pair_dist (below)
         const uint32_t full0 = CTAS == 2 ? map_to_cta(smem_u32(&full[0]), 0) : smem_u32(&full[0]);
         int stage = 0;
         uint32_t phase = 0;
@@ -370,7 +401,9 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         const uint32_t stage_bytes = p.stage_bytes;
         const bool post_tx = lane == 0 && leader;
         for (int it = 0; ok && sched.get(it, t); ++it) {
-            const int base = (isA ? t.m0 : t.n0) + off;
+            int base = (isA ? t.m0 : t.n0) + off;
+            // output column n0 of strip g -> B column n0 + g * pair_dist (gate) and one pair_dist further (up)
+            if (SWIGLU && !isA) base += (p.fd_wn.div(t.n0) + hsel) * p.pair_dist;
             int x, y, z, u;
             if (mn) to_coords(om, 0, base, x, y, z, u); else to_coords(om, base, 0, x, y, z, u);
             const int kb0 = t.split * kbps, kb1 = min(num_kb, kb0 + kbps);
@@ -454,10 +487,10 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         for (int it = 0; alive && sched.get(it, t); ++it) {
           const int m = t.m0 + (int)rank * BM + quad * 32 + lane;
 #pragma unroll 1                                         // one copy of the (large) drain code: a short GEMM pays for every instruction-cache miss
-          for (int h = 0; h < NSUB; ++h) {
+          for (int h = 0; h < (SWIGLU ? 1 : NSUB); ++h) {
             const int acc = NSUB == 1 ? (it & 1) : h;
             const uint32_t acc_phase = NSUB == 1 ? ((uint32_t)(it >> 1) & 1) : ((uint32_t)it & 1);
-            const int nb = t.n0 + h * SUBN;              // first column of this sub-tile
+            const int nb = t.n0 + h * SUBN;              // first (output) column of this sub-tile
             bool ok = h > 0 || mbar_wait_bounded(&tmem_full[acc], acc_phase);   // one "full" barrier per tile
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) { if (lane == 0) atomicExch(&g_gemm_status, 4); alive = false; break; }
@@ -476,23 +509,27 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             to_coords(p.c, row0, nb, cx0, cy0, cz0, cu0);
             const bool c_chunked = p.c.il_mode == 2;
             // One 64-column piece: registers -> C.  `r` holds 64 fp32 accumulators of this thread's row.
-            auto store_piece = [&](const uint32_t (&r)[64], int c) {
+            // One 64-column piece of this warp's 32 rows -> C.  `pk` holds the piece already rounded to bf16 (two
+            // values per word); full pieces go through shared memory and a TMA tile store, ragged ones are stored
+            // from registers.  (The accumulator registers are packed right after the TMEM wait: nothing else reads
+            // the registers a tcgen05.ld has written.)
+            auto pack = [&](const uint32_t (&r)[64], uint32_t (&pk)[32]) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
+                    pk[i] = *reinterpret_cast<const uint32_t*>(&hh);
+                }
+            };
+            auto store_packed = [&](const uint32_t (&pk)[32], int c) {
                 const int n64 = nb + c * 64;
-                if (p.splits == 1 && rows_full && n64 + 64 <= t.n1) {
+                if (rows_full && n64 + 64 <= t.n1) {
                     unsigned char* buf = epi + (size_t)((warp - 2) * 2 + (epi_count & 1)) * (32 * 128);
                     CCL_TRACE2(warp == 2 && lane == 0 && epi_count < 12, epi_count * 5 + 0);
                     if (epi_count >= 2) { if (lane == 0) tma_store_wait_read<1>(); __syncwarp(); }   // buffer free again
                     CCL_TRACE2(warp == 2 && lane == 0 && epi_count < 12, epi_count * 5 + 1);
 #pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        uint4 v;
-                        __nv_bfloat162 hh;
-                        hh = __floats2bfloat162_rn(__uint_as_float(r[u * 8 + 0]), __uint_as_float(r[u * 8 + 1])); v.x = *reinterpret_cast<uint32_t*>(&hh);
-                        hh = __floats2bfloat162_rn(__uint_as_float(r[u * 8 + 2]), __uint_as_float(r[u * 8 + 3])); v.y = *reinterpret_cast<uint32_t*>(&hh);
-                        hh = __floats2bfloat162_rn(__uint_as_float(r[u * 8 + 4]), __uint_as_float(r[u * 8 + 5])); v.z = *reinterpret_cast<uint32_t*>(&hh);
-                        hh = __floats2bfloat162_rn(__uint_as_float(r[u * 8 + 6]), __uint_as_float(r[u * 8 + 7])); v.w = *reinterpret_cast<uint32_t*>(&hh);
-                        *reinterpret_cast<uint4*>(buf + lane * 128 + ((u ^ (lane & 7)) << 4)) = v;
-                    }
+                    for (int u = 0; u < 8; ++u)
+                        *reinterpret_cast<uint4*>(buf + lane * 128 + ((u ^ (lane & 7)) << 4)) = make_uint4(pk[4 * u], pk[4 * u + 1], pk[4 * u + 2], pk[4 * u + 3]);
                     CCL_TRACE2(warp == 2 && lane == 0 && epi_count < 12, epi_count * 5 + 2);
                     fence_proxy_async();
                     __syncwarp();
@@ -507,38 +544,31 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     ++epi_count;
                     return;
                 }
-                // a 64-column piece of a row is contiguous in every layout the GEMM accepts
-                const int64_t piece_off = p.splits > 1 || m >= t.m1 ? 0 : c_offset(p, m, n64) + (int64_t)t.e * p.c_batch_stride;
+                // a 64-column piece of a row is contiguous in every layout the GEMM accepts; rows past the tile's end
+                // compute the address of its last row and store nothing (the row test only ever predicates a store:
+                // the TMEM loads and waits around this code are warp-wide)
+                const bool row_ok = m < t.m1;
+                unsigned short* dst = p.C + c_offset(p, min(m, t.m1 - 1), n64) + (int64_t)t.e * p.c_batch_stride;
 #pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    const uint32_t* rr = &r[half * 32];
-                    const int n32 = n64 + half * 32;
-                    if (p.splits > 1) {                  // partial sums, summed in fixed order by splitk_reduce_kernel
-                        if (m < t.m1) {
-                            float* wrow = p.ws + (((int64_t)t.e * p.splits + t.split) * p.M + m) * (int64_t)p.N;
+                for (int j = 0; j < 8; ++j)
+                    if (n64 + j * 8 < t.n1)              // the same for the whole warp; n1 - n0 is a multiple of 8
+                        st_global_v4_if(dst + j * 8, make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]), row_ok);
+            };
+            // split-K: the fp32 partial sums of a piece, summed in fixed order by splitk_reduce_kernel
+            auto store_partial = [&](const uint32_t (&r)[64], int c) {
+                const int n64 = nb + c * 64;
+                const bool row_ok = m < t.m1;
+                float* wrow = p.ws + (((int64_t)t.e * p.splits + t.split) * p.M + min(m, t.m1 - 1)) * (int64_t)p.N;
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) {
-                                const int n = n32 + j * 4;
-                                if (n < t.n1)
-                                    *reinterpret_cast<uint4*>(wrow + n) = make_uint4(rr[j * 4 + 0], rr[j * 4 + 1], rr[j * 4 + 2], rr[j * 4 + 3]);
-                            }
-                        }
-                    } else if (m < t.m1) {
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const int n = n32 + j * 8;
-                            if (n < t.n1) {              // n1 - n0 is a multiple of 8
-                                uint4 v;
-                                __nv_bfloat162 hh;
-                                hh = __floats2bfloat162_rn(__uint_as_float(rr[j * 8 + 0]), __uint_as_float(rr[j * 8 + 1])); v.x = *reinterpret_cast<uint32_t*>(&hh);
-                                hh = __floats2bfloat162_rn(__uint_as_float(rr[j * 8 + 2]), __uint_as_float(rr[j * 8 + 3])); v.y = *reinterpret_cast<uint32_t*>(&hh);
-                                hh = __floats2bfloat162_rn(__uint_as_float(rr[j * 8 + 4]), __uint_as_float(rr[j * 8 + 5])); v.z = *reinterpret_cast<uint32_t*>(&hh);
-                                hh = __floats2bfloat162_rn(__uint_as_float(rr[j * 8 + 6]), __uint_as_float(rr[j * 8 + 7])); v.w = *reinterpret_cast<uint32_t*>(&hh);
-                                *reinterpret_cast<uint4*>(p.C + piece_off + (n - n64)) = v;
-                            }
-                        }
-                    }
-                }
+                for (int j = 0; j < 16; ++j)
+                    if (n64 + j * 4 < t.n1)
+                        st_global_v4_if(wrow + n64 + j * 4, make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]), row_ok);
+            };
+            auto store_piece = [&](uint32_t (&r)[64], int c) {
+                if (p.splits > 1) { store_partial(r, c); return; }
+                uint32_t pk[32];
+                pack(r, pk);
+                store_packed(pk, c);
             };
             // TMEM reads are software-pipelined: the load of piece c+1 is in flight while piece c is converted
             // and stored (two register sets, so the loop is unrolled by two).
@@ -548,17 +578,42 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 tmem_ld32(taddr + (uint32_t)(c * 64), *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
                 tmem_ld32(taddr + (uint32_t)(c * 64 + 32), *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
             };
+            if (SWIGLU) {
+                // piece c of accumulator 0 holds the gate values, piece c of accumulator 1 the up values of the same
+                // 64 output columns: out = gate / (1 + exp(-gate)) * up, in fp32, then the usual bf16 store
+#pragma unroll 1
+                for (int c = 0; c < npieces; ++c) {
+                    load_piece(ra, c);
+                    load_piece(rb, c + ACC_COLS / 64);
+                    tmem_ld_wait();
+                    tmem_regs_ready(ra);
+                    tmem_regs_ready(rb);
+                    uint32_t pk[32];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const float g0 = __uint_as_float(ra[2 * i]), g1 = __uint_as_float(ra[2 * i + 1]);
+                        const float u0 = __uint_as_float(rb[2 * i]), u1 = __uint_as_float(rb[2 * i + 1]);
+                        const __nv_bfloat162 hh = __floats2bfloat162_rn(__fdividef(g0, 1.0f + __expf(-g0)) * u0,
+                                                                        __fdividef(g1, 1.0f + __expf(-g1)) * u1);
+                        pk[i] = *reinterpret_cast<const uint32_t*>(&hh);
+                    }
+                    store_packed(pk, c);
+                }
+            } else {
             if (npieces > 0) load_piece(ra, 0);
 #pragma unroll 1
             for (int c = 0; c < npieces; c += 2) {
                 tmem_ld_wait();
+                tmem_regs_ready(ra);
                 if (c + 1 < npieces) load_piece(rb, c + 1);
                 store_piece(ra, c);
                 if (c + 1 < npieces) {
                     tmem_ld_wait();
+                    tmem_regs_ready(rb);
                     if (c + 2 < npieces) load_piece(ra, c + 2);
                     store_piece(rb, c + 1);
                 }
+            }
             }
             tc_fence_before();
             __syncwarp();
@@ -567,6 +622,10 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             if (lane == 0) {
                 if (CTAS == 2) mbar_arrive_cluster(tmem_empty0 + (uint32_t)acc * 8u);
                 else mbar_arrive(&tmem_empty[acc]);
+                if (SWIGLU) {                            // both accumulators of the tile have been read
+                    if (CTAS == 2) mbar_arrive_cluster(tmem_empty0 + 8u);
+                    else mbar_arrive(&tmem_empty[1]);
+                }
             }
           }
         }
@@ -680,7 +739,7 @@ static ccl_status merge_width(int64_t* cur, int64_t w, const char* dim) {
 static int64_t padded(int64_t w, int64_t b) { return (w + b - 1) / b * b; }
 
 // units = schedulable CTAs (1-CTA kernel) or CTA pairs (2-CTA kernel) the device can hold at once
-static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, const void* A, const void* B, const void* C, int sms, int pairs, GemmPlan* plan) {
+static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, const void* A, const void* B, const void* C, int sms, int pairs, GemmPlan* plan) {
     if (!d) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: NULL descriptor");
     if (d->M <= 0 || d->N <= 0 || d->K <= 0) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: M, N, K must be positive");
     if (d->M >= (INT64_C(1) << 31) || d->N >= (INT64_C(1) << 31) || d->K >= (INT64_C(1) << 31)) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: dimension too large");
@@ -693,8 +752,12 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, const void* A
     const MatView &va = plan->va, &vb = plan->vb, &vc = plan->vc;
     const bool at = d->a_trans != 0, bt = d->b_trans != 0;
     int64_t ar = at ? d->K : d->M, ac = at ? d->M : d->K, br = bt ? d->N : d->K, bc = bt ? d->K : d->N;
-    if (va.rows != ar || va.cols != ac || vb.rows != br || vb.cols != bc || vc.rows != d->M || vc.cols != d->N)
+    if (swiglu && d->N % 2) return fail(CCL_ERR_SHAPE, "ccl_gemm_swiglu: N (gate + up columns) must be even");
+    const int64_t Nc = swiglu ? d->N / 2 : d->N;        // columns of C, which the tile walk counts
+    if (va.rows != ar || va.cols != ac || vb.rows != br || vb.cols != bc || vc.rows != d->M || vc.cols != Nc)
         return fail(CCL_ERR_SHAPE, "ccl_gemm: operand shapes do not match M, N, K and the transpose flags");
+    if (swiglu && (va.ichunk || vb.ichunk || vc.ichunk))
+        return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm_swiglu: page-interleaved operands are not supported");
     if ((s = check_operand(va, A, "A", at, d->K))) return s;
     if ((s = check_operand(vb, B, "B", !bt, d->K))) return s;
     if ((s = check_operand(vc, C, "C", false, d->K))) return s;
@@ -707,13 +770,23 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, const void* A
     int64_t Wm = 0, Wn = 0;
     if ((s = merge_width(&Wm, split_width(va, !at), "M"))) return s;
     if ((s = merge_width(&Wm, split_width(vc, true), "M"))) return s;
-    if ((s = merge_width(&Wn, split_width(vb, bt), "N"))) return s;
+    if (swiglu) {
+        // a strip of B holds the gate and the up columns of one strip of C: twice as wide
+        const int64_t wb = split_width(vb, bt);
+        if (wb % 2) return fail(CCL_ERR_SHAPE, "ccl_gemm_swiglu: strips of B have an odd width");
+        if ((s = merge_width(&Wn, wb / 2, "N"))) return s;
+        // the gate | up halves follow the output partition whether or not the raster is grouped
+        if (d->out_part == CCL_PART_COLS && d->P > 1) {
+            if (Nc % d->P) return fail(CCL_ERR_SHAPE, "ccl_gemm_swiglu: N/2 not divisible by P");
+            if ((s = merge_width(&Wn, Nc / d->P, "N"))) return s;
+        }
+    } else if ((s = merge_width(&Wn, split_width(vb, bt), "N"))) return s;
     if ((s = merge_width(&Wn, split_width(vc, false), "N"))) return s;
     int groups = 1, group_dim = 0;
     if (d->grouped_raster && d->P > 1 && d->out_part != CCL_PART_NONE) {
         if (d->out_part == CCL_PART_COLS) {
-            if (d->N % d->P) return fail(CCL_ERR_SHAPE, "ccl_gemm: N not divisible by P");
-            if ((s = merge_width(&Wn, d->N / d->P, "N"))) return s;
+            if (Nc % d->P) return fail(CCL_ERR_SHAPE, "ccl_gemm: N not divisible by P");
+            if ((s = merge_width(&Wn, Nc / d->P, "N"))) return s;
             groups = d->P; group_dim = 0;
         } else {
             if (d->M % d->P) return fail(CCL_ERR_SHAPE, "ccl_gemm: M not divisible by P");
@@ -724,7 +797,13 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, const void* A
     int64_t ka = split_width(va, at), kb = split_width(vb, !bt);
     if ((ka && ka % BK) || (kb && kb % BK)) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: an operand split along K needs strips that are multiples of %d", BK);
     if (!Wm) Wm = d->M;
-    if (!Wn) Wn = d->N;
+    if (!Wn) Wn = Nc;
+    if (swiglu) {
+        const int64_t pd = d->out_part == CCL_PART_COLS && d->P > 1 ? Nc / d->P : Nc;      // gate -> up distance in B
+        if (Wn != pd) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm_swiglu: strips of B / C (%lld output columns) differ from the gate | up halves (%lld)", (long long)Wn, (long long)pd);
+        if (pd % 8) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm_swiglu: gate | up halves of %lld columns are not a multiple of 8", (long long)pd);
+        if (pairs <= 0) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm_swiglu: needs 2-CTA clusters");
+    }
 
     // Tile shape, CTA pairing and split-K from a small cost model (cycles per unit):
     //   a k block of a one-accumulator tile takes ~600 cycles whatever its width (four MMAs are issued in ~350
@@ -736,7 +815,7 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, const void* A
     // 256 x 512 pair tiles move the fewest bytes per flop and win once K is long; short problems prefer the
     // variant whose tile count fills the machine.
     const int64_t num_kb = (d->K + BK - 1) / BK;
-    const int64_t strips_m = d->M / Wm, strips_n = d->N / Wn;
+    const int64_t strips_m = d->M / Wm, strips_n = Nc / Wn;
     int ctas = 1, bn = 256, splits = 1;
     double best = -1.0;
     // Tuning / test overrides (environment): CCL_GEMM_CTAS = 1|2, CCL_GEMM_BN = 128|192|256|512,
@@ -753,13 +832,15 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, const void* A
             if (c == 2 && b == 192 && !bt) continue;             // 96 columns per CTA are not made of 64-column boxes of an N-contiguous B
             if (b == 192 && (c == 2 ? no_192_pair : no_192)) continue;
             if (force_bn && atoi(force_bn) != b) continue;
+            if (swiglu && !(c == 2 && b == 512)) continue;          // the gated activation pairs the two accumulators of the wide tile
             const int64_t tiles_m_all = strips_m * ((Wm + BM * c - 1) / (BM * c));
-            const int64_t tiles = tiles_m_all * strips_n * ((Wn + b - 1) / b) * batch;
+            const int bs = swiglu ? 256 : b;                        // tile width in C columns
+            const int64_t tiles = tiles_m_all * strips_n * ((Wn + bs - 1) / bs) * batch;
             double t_kb = b == 512 ? 1050.0 : (c == 1 && b == 256 ? 680.0 : (c == 1 ? 570.0 : 620.0));
             if (tiles_m_all == 1) t_kb = std::max(t_kb, (double)(b / c) * (BK * 2) / 27.0);
             const double t_drain = b == 512 ? 7000.0 : 1500.0;
             for (int sp : {1, 2, 3, 4, 6, 8, 12, 16}) {
-                if (sp > 1 && num_kb / sp < 2) continue;
+                if (sp > 1 && (swiglu || num_kb / sp < 2)) continue;
                 if (force_split && atoi(force_split) != sp) continue;
                 const int64_t kbps = (num_kb + sp - 1) / sp;
                 const int64_t sp_eff = (num_kb + kbps - 1) / kbps;          // every split owns at least one k block
@@ -780,10 +861,12 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, const void* A
 
     GemmParams& p = plan->p;
     std::memset(&p, 0, sizeof(p));
-    p.M = (int32_t)d->M; p.N = (int32_t)d->N; p.K = (int32_t)d->K;
+    p.M = (int32_t)d->M; p.N = (int32_t)Nc; p.K = (int32_t)d->K;
+    const int bn_walk = swiglu ? 256 : bn;              // tile width in C columns
+    p.pair_dist = swiglu ? (int32_t)Wn : 0; p.fd_wn = make_fastdiv(Wn);
     p.Wm = (int32_t)Wm; p.Wn = (int32_t)Wn;
-    p.tps_m = (int32_t)((Wm + bm - 1) / bm); p.tps_n = (int32_t)((Wn + bn - 1) / bn);
-    p.tiles_m = (int32_t)(d->M / Wm) * p.tps_m; p.tiles_n = (int32_t)(d->N / Wn) * p.tps_n;
+    p.tps_m = (int32_t)((Wm + bm - 1) / bm); p.tps_n = (int32_t)((Wn + bn_walk - 1) / bn_walk);
+    p.tiles_m = (int32_t)(d->M / Wm) * p.tps_m; p.tiles_n = (int32_t)(Nc / Wn) * p.tps_n;
     p.num_kb = (int32_t)num_kb;
     p.splits = splits; p.kb_per_split = (int32_t)((num_kb + splits - 1) / splits);
     p.a.split = va.split; p.a.w = make_fastdiv(va.w); p.a.h = make_fastdiv(va.h);
@@ -793,8 +876,9 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, const void* A
     p.b.il_mode = il_b; p.b.il_kr = make_fastdiv(kr_b); p.b.il_sc = make_fastdiv(vb.ichunk);
     p.c.split = vc.split; p.c.w = make_fastdiv(vc.w); p.c.h = make_fastdiv(vc.h);
     p.c.il_mode = il_c; p.c.il_kr = make_fastdiv(kr_c); p.c.il_sc = make_fastdiv(vc.ichunk);
-    p.c_split = vc.split; p.c_w = vc.w; p.c_h = vc.h; p.c_stride = vc.stride; p.c_cols = vc.cols;
+    p.c_row = vc.split == 2 ? vc.w : vc.cols; p.c_stride = vc.stride;
     p.c_ichunk = vc.ichunk; p.c_nstrips = vc.nstrips;
+    p.c_cpr = il_c == 2 ? (int32_t)(p.c_row / vc.ichunk) : 0;
     // instruction descriptor: D = f32, A = B = bf16, operand majors, N >> 3, M >> 4 (M spans the CTA pair)
     p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)p.a_mn << 15) | ((uint32_t)p.b_mn << 16) |
               ((uint32_t)(subn >> 3) << 17) | ((uint32_t)(bm >> 4) << 24);
@@ -879,19 +963,19 @@ static ccl_status operand_tmap(CUtensorMap* m, const MatView& v, const void* bas
     return encode_tmap(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, base, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
-template <int BN, int CTAS>
+template <int BN, int CTAS, bool SWIGLU = false>
 static ccl_status configure(uint32_t smem_bytes) {
     static uint32_t configured_for = 0;
     if (configured_for < smem_bytes) {
-        CCL_CUDA_TRY(cudaFuncSetAttribute(ccl_gemm_kernel<BN, CTAS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes));
+        CCL_CUDA_TRY(cudaFuncSetAttribute(ccl_gemm_kernel<BN, CTAS, SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes));
         configured_for = smem_bytes;
     }
     return CCL_OK;
 }
 
-template <int BN, int CTAS>
+template <int BN, int CTAS, bool SWIGLU = false>
 static ccl_status launch(const GemmPlan& plan, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, cudaStream_t st) {
-    ccl_status s = configure<BN, CTAS>(plan.smem_bytes);
+    ccl_status s = configure<BN, CTAS, SWIGLU>(plan.smem_bytes);
     if (s) return s;
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof(cfg));
@@ -904,7 +988,7 @@ static ccl_status launch(const GemmPlan& plan, const CUtensorMap& ma, const CUte
     attr[0].val.clusterDim.x = CTAS; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    CCL_CUDA_TRY(cudaLaunchKernelEx(&cfg, ccl_gemm_kernel<BN, CTAS>, ma, mb, mc, plan.p));
+    CCL_CUDA_TRY(cudaLaunchKernelEx(&cfg, ccl_gemm_kernel<BN, CTAS, SWIGLU>, ma, mb, mc, plan.p));
     count_launch();
     return CCL_OK;
 }
@@ -937,6 +1021,7 @@ using namespace ccl;
 struct PreparedKey {
     int64_t f[36];          // every field of the descriptor, the batch, the three pointers, the device and the tuning overrides
     int dev;
+    int mode;               // 0 plain, 1 gated activation
     char env[60];
 };
 struct Prepared {
@@ -989,12 +1074,12 @@ constexpr int64_t kMaxBatch = 65536;
 static ccl_status workspace_impl(const ccl_gemm_desc* d, int64_t batch, size_t* bytes) {
     if (batch < 1 || batch > kMaxBatch) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: batch must be in [1, %lld]", (long long)kMaxBatch);
     GemmPlan plan;
-    ccl_status s = make_plan(d, batch, nullptr, nullptr, nullptr, 148, 74, &plan);     // validation without any CUDA call
+    ccl_status s = make_plan(d, batch, false, nullptr, nullptr, nullptr, 148, 74, &plan);     // validation without any CUDA call
     if (s) return s;
     if (!bytes) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm_workspace: NULL output");
     int sms, pairs;
     device_units(&sms, &pairs);
-    if ((s = make_plan(d, batch, nullptr, nullptr, nullptr, sms, pairs, &plan))) return s;
+    if ((s = make_plan(d, batch, false, nullptr, nullptr, nullptr, sms, pairs, &plan))) return s;
     *bytes = plan.ws_bytes;
     return CCL_OK;
 }
@@ -1003,7 +1088,7 @@ extern "C" ccl_status ccl_gemm_workspace(const ccl_gemm_desc* d, size_t* bytes) 
 extern "C" ccl_status ccl_gemm_batched_workspace(const ccl_gemm_desc* d, int32_t batch, size_t* bytes) { return workspace_impl(d, batch, bytes); }
 
 // strides[X]: bytes between the buffers of operand X (A, B, C) of consecutive problems; 0 = shared (A and B only)
-static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, const int64_t* strides, const void* A_dev, const void* B_dev, void* C_dev,
+static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, const int64_t* strides, const void* A_dev, const void* B_dev, void* C_dev,
                             void* ws_dev, size_t ws_bytes, void* cuda_stream) {
     if (!A_dev || !B_dev || !C_dev) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: NULL operand");
     if (!d) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: NULL descriptor");
@@ -1013,6 +1098,7 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, const int64_t
     // reuse the plan and the two encoded tensor maps: a host-side cache only, nothing is kept on the device.
     PreparedKey key;
     make_key(d, batch4, A_dev, B_dev, C_dev, &key);
+    key.mode = swiglu ? 1 : 0;
     Prepared prep;
     bool hit = false;
     {
@@ -1023,7 +1109,7 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, const int64_t
     ccl_status s;
     if (!hit) {
         GemmPlan& plan = prep.plan;
-        s = make_plan(d, batch, A_dev, B_dev, C_dev, 148, 74, &plan);     // validation first: no CUDA call on bad input
+        s = make_plan(d, batch, swiglu, A_dev, B_dev, C_dev, 148, 74, &plan);     // validation first: no CUDA call on bad input
         if (s) return s;
         if (batch > 1) {
             const MatView* views[3] = {&plan.va, &plan.vb, &plan.vc};
@@ -1039,8 +1125,8 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, const int64_t
         int dev;
         CCL_CUDA_TRY(cudaGetDevice(&dev));
         CCL_CUDA_TRY(cudaDeviceGetAttribute(&prep.sms, cudaDevAttrMultiProcessorCount, dev));
-        if (dev != key.dev) make_key(d, batch4, A_dev, B_dev, C_dev, &key);
-        if ((s = make_plan(d, batch, A_dev, B_dev, C_dev, prep.sms, resident_pairs(), &plan))) return s;
+        if (dev != key.dev) { make_key(d, batch4, A_dev, B_dev, C_dev, &key); key.mode = swiglu ? 1 : 0; }
+        if ((s = make_plan(d, batch, swiglu, A_dev, B_dev, C_dev, prep.sms, resident_pairs(), &plan))) return s;
         plan.p.C = static_cast<uint16_t*>(C_dev);
         plan.p.a.batched = batch4[1] != 0; plan.p.b.batched = batch4[2] != 0; plan.p.c.batched = 1;
         plan.p.c_batch_stride = batch4[3] / 2;
@@ -1065,7 +1151,8 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, const int64_t
     }
     plan.p.ws = static_cast<float*>(ws_dev);
     cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
-    if (plan.ctas == 2) {
+    if (swiglu) s = launch<512, 2, true>(plan, ma, mb, mc, st);
+    else if (plan.ctas == 2) {
         if (plan.bn == 512) s = launch<512, 2>(plan, ma, mb, mc, st);
         else if (plan.bn == 192) s = launch<192, 2>(plan, ma, mb, mc, st);
         else s = plan.bn == 256 ? launch<256, 2>(plan, ma, mb, mc, st) : launch<128, 2>(plan, ma, mb, mc, st);
@@ -1086,7 +1173,7 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, const int64_t
 extern "C" ccl_status ccl_gemm(const ccl_gemm_desc* d, const void* A_dev, const void* B_dev, void* C_dev, void* ws_dev,
                                size_t ws_bytes, void* cuda_stream) {
     const int64_t none[3] = {0, 0, 0};
-    return gemm_impl(d, 1, none, A_dev, B_dev, C_dev, ws_dev, ws_bytes, cuda_stream);
+    return gemm_impl(d, 1, false, none, A_dev, B_dev, C_dev, ws_dev, ws_bytes, cuda_stream);
 }
 
 extern "C" ccl_status ccl_gemm_batched(const ccl_gemm_desc* d, int32_t batch, const void* A_dev, int64_t a_stride_bytes, const void* B_dev,
@@ -1094,7 +1181,12 @@ extern "C" ccl_status ccl_gemm_batched(const ccl_gemm_desc* d, int32_t batch, co
                                        void* cuda_stream) {
     if (a_stride_bytes < 0 || b_stride_bytes < 0 || c_stride_bytes < 0) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm_batched: negative stride");
     const int64_t strides[3] = {a_stride_bytes, b_stride_bytes, c_stride_bytes};
-    return gemm_impl(d, batch, strides, A_dev, B_dev, C_dev, ws_dev, ws_bytes, cuda_stream);
+    return gemm_impl(d, batch, false, strides, A_dev, B_dev, C_dev, ws_dev, ws_bytes, cuda_stream);
+}
+
+extern "C" ccl_status ccl_gemm_swiglu(const ccl_gemm_desc* d, const void* A_dev, const void* B_dev, void* C_dev, void* cuda_stream) {
+    const int64_t none[3] = {0, 0, 0};
+    return gemm_impl(d, 1, true, none, A_dev, B_dev, C_dev, nullptr, 0, cuda_stream);
 }
 
 extern "C" ccl_status ccl_gemm_status(void* cuda_stream, int32_t* detail) {

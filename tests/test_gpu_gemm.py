@@ -18,6 +18,9 @@ from helpers import gemm_desc
 pytestmark = pytest.mark.gpu
 
 
+GUARD = 8192        # elements of untouched memory that must stay untouched behind every output buffer
+
+
 def tol(K):
     return 1e-2 * math.sqrt(K / 1024.0)
 
@@ -38,13 +41,15 @@ def from_layout(buf, m):
 def run_gemm(d, A, B):
     """A, B: bf16 CPU tensors as stored (row-major).  Returns C as uint16 bits [M x N] (logical order)."""
     a_dev, b_dev = to_layout(synth.bits(A), d.A), to_layout(synth.bits(B), d.B)
-    c_dev = torch.full((ccl.ccl_buffer_bytes(d.C) // 2,), 0x7FC0, dtype=torch.int16, device="cuda")   # NaN poison
+    nc = ccl.ccl_buffer_bytes(d.C) // 2
+    c_dev = torch.full((nc + GUARD,), 0x7FC0, dtype=torch.int16, device="cuda")   # NaN poison, and a guard zone behind C
     need = ccl.ccl_gemm_workspace(d)
     ws = torch.full((need // 4,), float("nan"), dtype=torch.float32, device="cuda") if need else None
     ccl.ccl_gemm(d, a_dev, b_dev, c_dev, ws)
     st, detail = ccl.ccl_gemm_status()
     assert st == ccl.OK, detail
-    return from_layout(c_dev, d.C)
+    assert (c_dev[nc:] == 0x7FC0).all(), "the kernel wrote past the end of C"
+    return from_layout(c_dev[:nc], d.C)
 
 
 def check(d, A, B, block=None):
