@@ -1,0 +1,71 @@
+"""The device entry points are plain stream work: after one eager call (which fills the library's host-side plan cache
+and configures the kernels) a whole step -- repack, GEMM, split-K GEMM, batched GEMM, gated-activation GEMM, traffic
+count -- can be captured into a CUDA graph and replayed, with the same bits as the eager calls."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2606_11718_b200 import binding as ccl
+from paper_2606_11718_b200 import synth
+from helpers import gemm_desc, traffic_pair
+from test_gpu_gemm_swiglu import swiglu_desc
+
+pytestmark = pytest.mark.gpu
+
+
+def test_step_replays_from_a_cuda_graph():
+    M, N, K, P, E = 384, 1536, 512, 4, 3
+    A, B = synth.gemm_operands(M, N, K, 0, 0, seed=31, tag="graph", b_std=0.05)
+    a, b = A.cuda(), B.cuda()
+    d = gemm_desc(M, N, K, P, ("row", "ccl", "ccl"), 0, 0, 2, 1, align=4096)
+    ds = swiglu_desc(M, N, K, P, ("row", "ccl", "ccl"), 0, 0, 2, 1, align=4096)
+    dk = gemm_desc(16, N, 2048, P, ("row", "ccl", "ccl"), 0, 0, 2, 1)                    # split along K
+    Ak, Bk = synth.gemm_operands(16, N, 2048, 0, 0, seed=32, tag="graphk")
+    ak, bk_row = Ak.cuda(), Bk.cuda()
+    nb, nc = ccl.ccl_buffer_bytes(d.B) // 2, ccl.ccl_buffer_bytes(d.C) // 2
+    b_ccl = torch.empty(nb, dtype=torch.bfloat16, device="cuda")
+    bk_ccl = torch.empty(ccl.ccl_buffer_bytes(dk.B) // 2, dtype=torch.bfloat16, device="cuda")
+    c1 = torch.zeros(nc, dtype=torch.bfloat16, device="cuda")
+    c2 = torch.zeros(ccl.ccl_buffer_bytes(ds.C) // 2, dtype=torch.bfloat16, device="cuda")
+    ck = torch.zeros(ccl.ccl_buffer_bytes(dk.C) // 2, dtype=torch.bfloat16, device="cuda")
+    need = ccl.ccl_gemm_workspace(dk)
+    assert need > 0
+    ws = torch.empty(need // 4, dtype=torch.float32, device="cuda")
+    ab = a.repeat(E, 1).contiguous()
+    cb = torch.zeros(E * nc, dtype=torch.bfloat16, device="cuda")
+    needb = ccl.ccl_gemm_batched_workspace(d, E)
+    wsb = torch.empty(max(needb, 4) // 4, dtype=torch.float32, device="cuda")
+    _, td = traffic_pair(M, N, K, P, 4096, ("row", "ccl", "ccl"), (0, 1, 1), align=4096)
+    nt, _ = ccl.ccl_traffic_sizes(td)
+    per_cta = torch.zeros((nt, 3, 2), dtype=torch.int64, device="cuda")
+    totals = torch.zeros((3, 2), dtype=torch.int64, device="cuda")
+
+    def step():
+        ccl.ccl_repack(d.B, b, b_ccl, 0)
+        ccl.ccl_repack(dk.B, bk_row, bk_ccl, 0)
+        ccl.ccl_gemm(d, a, b_ccl, c1)
+        ccl.ccl_gemm_swiglu(ds, a, b_ccl, c2)
+        ccl.ccl_gemm(dk, ak, bk_ccl, ck, ws)
+        ccl.ccl_gemm_batched(d, E, ab, M * K * 2, b_ccl, 0, cb, nc * 2, wsb if needb else None)
+        ccl.ccl_traffic(td, per_cta, totals)
+
+    outs = (c1, c2, ck, cb, per_cta, totals)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        step()                                                   # eager: plans cached, kernels configured
+        side.synchronize()
+        assert ccl.ccl_gemm_status()[0] == ccl.OK
+        want = [o.clone() for o in outs]
+        for o in outs:
+            o.zero_()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            step()
+    for _ in range(3):
+        for o in outs:
+            o.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        for o, w in zip(outs, want):
+            assert torch.equal(o, w)
+    assert ccl.ccl_gemm_status()[0] == ccl.OK
