@@ -36,7 +36,11 @@ namespace ccl {
 
 constexpr int BM = 128;                         // rows of the output tile one CTA owns
 constexpr int BK = 64;
-constexpr int kGemmThreads = 192;
+#ifndef CCL_EPI_WARPS
+#define CCL_EPI_WARPS 4
+#endif
+constexpr int kEpiWarps = CCL_EPI_WARPS;        // 4, or 8: two warps per TMEM lane quadrant taking alternate 64-column pieces
+constexpr int kGemmThreads = 64 + 32 * kEpiWarps;
 constexpr int kTmemCols = 512;
 constexpr uint32_t kSmemBudget = 192 * 1024;    // ring of operand stages
 constexpr uint32_t kEpiBytes = 4 * 2 * 32 * 128; // epilogue staging: per warp two buffers of 32 rows x 128 B
@@ -352,7 +356,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         prefetch_tmap(&map_b);
         prefetch_tmap(&map_c);
         for (int s = 0; s < gp.stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-        for (int a = 0; a < NACC; ++a) { mbar_init(&tmem_full[a], 1); mbar_init(&tmem_empty[a], 4 * CTAS); }
+        for (int a = 0; a < NACC; ++a) { mbar_init(&tmem_full[a], 1); mbar_init(&tmem_empty[a], kEpiWarps * CTAS); }
         fence_barrier_init();
     }
     if (warp == 1) tmem_alloc<CTAS>(tmem_ptr, kTmemCols);
@@ -480,6 +484,8 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..5)
         const int quad = warp & 3;                       // TMEM lane quadrant this warp may read
+        constexpr int EW = kEpiWarps / 4;                // warps per quadrant
+        const int hf = (warp - 2) >> 2;                  // which of them this one is
         const uint32_t tmem_empty0 = CTAS == 2 ? map_to_cta(smem_u32(&tmem_empty[0]), 0) : smem_u32(&tmem_empty[0]);
         TileCoord t;
         bool alive = true;
@@ -523,9 +529,10 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             auto store_packed = [&](const uint32_t (&pk)[32], int c) {
                 const int n64 = nb + c * 64;
                 if (rows_full && n64 + 64 <= t.n1) {
-                    unsigned char* buf = epi + (size_t)((warp - 2) * 2 + (epi_count & 1)) * (32 * 128);
+                    // staging: 32 KB in all -- two buffers per warp with four warps, one with eight
+                    unsigned char* buf = epi + (size_t)(EW == 1 ? (warp - 2) * 2 + (epi_count & 1) : (warp - 2)) * (32 * 128);
                     CCL_TRACE2(warp == 2 && lane == 0 && epi_count < 12, epi_count * 5 + 0);
-                    if (epi_count >= 2) { if (lane == 0) tma_store_wait_read<1>(); __syncwarp(); }   // buffer free again
+                    if (epi_count >= 2 / EW) { if (lane == 0) tma_store_wait_read<2 / EW - 1>(); __syncwarp(); }   // buffer free again
                     CCL_TRACE2(warp == 2 && lane == 0 && epi_count < 12, epi_count * 5 + 1);
 #pragma unroll
                     for (int u = 0; u < 8; ++u)
@@ -582,7 +589,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 // piece c of accumulator 0 holds the gate values, piece c of accumulator 1 the up values of the same
                 // 64 output columns: out = gate / (1 + exp(-gate)) * up, in fp32, then the usual bf16 store
 #pragma unroll 1
-                for (int c = 0; c < npieces; ++c) {
+                for (int c = hf; c < npieces; c += EW) {
                     load_piece(ra, c);
                     load_piece(rb, c + ACC_COLS / 64);
                     tmem_ld_wait();
@@ -598,6 +605,14 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                         pk[i] = *reinterpret_cast<const uint32_t*>(&hh);
                     }
                     store_packed(pk, c);
+                }
+            } else if (EW > 1) {
+#pragma unroll 1
+                for (int c = hf; c < npieces; c += EW) {
+                    load_piece(ra, c);
+                    tmem_ld_wait();
+                    tmem_regs_ready(ra);
+                    store_piece(ra, c);
                 }
             } else {
             if (npieces > 0) load_piece(ra, 0);
