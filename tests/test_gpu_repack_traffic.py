@@ -32,13 +32,17 @@ def run_repack(case, path=None, seed=0):
         os.environ["CCL_REPACK_PATH"] = path
     try:
         src = dev(x)
-        dst = dev(np.full(want.size, 0x5A, dtype=npdt))                # poison: padding must be overwritten with zeros
+        guard = 4096                                                   # elements behind each output that must stay untouched
+        dst = dev(np.full(want.size + guard, 0x5A, dtype=npdt))        # poison: padding must be overwritten with zeros
         ccl.ccl_repack(ml, src, dst, 0)
         got = host(dst, npdt)
-        np.testing.assert_array_equal(got, want)
-        back = dev(np.zeros(mo.rows * mo.cols, dtype=npdt))
+        np.testing.assert_array_equal(got[:want.size], want)
+        assert (got[want.size:] == 0x5A).all(), "repack wrote past the end of its output"
+        back = dev(np.full(mo.rows * mo.cols + guard, 0x5A, dtype=npdt))
         ccl.ccl_repack(ml, dst, back, 1)
-        np.testing.assert_array_equal(host(back, npdt).reshape(mo.rows, mo.cols), x)
+        hb = host(back, npdt)
+        np.testing.assert_array_equal(hb[:mo.rows * mo.cols].reshape(mo.rows, mo.cols), x)
+        assert (hb[mo.rows * mo.cols:] == 0x5A).all(), "repack wrote past the end of its output"
         np.testing.assert_array_equal(orc.repack(mo, want, 1).reshape(mo.rows, mo.cols), x)
         assert ccl.ccl_gemm_status()[0] == ccl.OK
     finally:
