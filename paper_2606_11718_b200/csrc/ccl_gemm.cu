@@ -23,6 +23,7 @@
 //   * Every mbarrier wait is bounded; on expiry the kernel records a code in g_gemm_status,
 //     all roles leave their loops, TMEM is released and the kernel returns.
 #include <algorithm>
+#include <cstdio>
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
@@ -851,9 +852,13 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
             const int64_t tiles_m_all = strips_m * ((Wm + BM * c - 1) / (BM * c));
             const int bs = swiglu ? 256 : b;                        // tile width in C columns
             const int64_t tiles = tiles_m_all * strips_n * ((Wn + bs - 1) / bs) * batch;
-            double t_kb = b == 512 ? 1050.0 : (c == 1 && b == 256 ? 680.0 : (c == 1 ? 570.0 : 620.0));
-            if (tiles_m_all == 1) t_kb = std::max(t_kb, (double)(b / c) * (BK * 2) / 27.0);
+            const double t_kb = b == 512 ? 1050.0 : (c == 1 && b == 256 ? 680.0 : (c == 1 ? 570.0 : 620.0));
             const double t_drain = b == 512 ? 7000.0 : 1500.0;
+            // one row of tiles: nobody shares the B columns, the problem streams B from HBM at ~29 B/clk per SM in
+            // aggregate however the units are cut (a ragged last wave still saturates the memory); wider boxes are
+            // fetched a little more efficiently (measured: 128 / 192 columns cost ~10 % / ~4 % more time per byte)
+            const double stream_clk = tiles_m_all == 1 ? (double)tiles * (double)num_kb * (double)b * (BK * 2) / (sms * 29.0) *
+                                                             (b <= 128 ? 1.10 : (b <= 192 ? 1.04 : 1.0)) : 0.0;
             for (int sp : {1, 2, 3, 4, 6, 8, 12, 16}) {
                 if (sp > 1 && (swiglu || num_kb / sp < 2)) continue;
                 if (force_split && atoi(force_split) != sp) continue;
@@ -861,13 +866,19 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
                 const int64_t sp_eff = (num_kb + kbps - 1) / kbps;          // every split owns at least one k block
                 if (sp_eff != sp) continue;
                 const int64_t waves = (tiles * sp + units - 1) / units;
-                double cost = (double)waves * ((double)kbps * t_kb + (sp > 1 ? 2.0 * t_drain : t_drain)) + 3000.0;
+                // (a last wave that leaves SMs idle streams a little slower: measured ~5 % between 96 and 128 busy SMs)
+                const double last = (double)(tiles * sp - (waves - 1) * units) / (double)units;
+                double cost = std::max((double)waves * ((double)kbps * t_kb + (sp > 1 ? 2.0 * t_drain : t_drain)),
+                                       stream_clk * (1.0 + 0.1 * (1.0 - last))) + 3000.0;
                 if (sp > 1) cost += ((double)sp + 0.5) * (double)batch * (double)d->M * (double)d->N * 4.0 / 3400.0 + 14000.0;
                 if (best < 0 || cost < best) { best = cost; ctas = c; bn = b; splits = sp; }
             }
         }
     }
     if (best < 0) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: no kernel variant matches the forced CCL_GEMM_* settings");
+    if (std::getenv("CCL_GEMM_VERBOSE"))
+        std::fprintf(stderr, "ccl_gemm plan: %lld x %lld x %lld batch %lld -> %d CTA(s) per tile, tile width %d, %d K split(s), modelled %.0f cycles\n",
+                     (long long)d->M, (long long)d->N, (long long)d->K, (long long)batch, ctas, bn, splits, best);
     const int subn = bn > 256 ? 256 : bn;                // columns of one MMA / one TMEM accumulator
     plan->subn = subn;
     const int bm = BM * ctas;
