@@ -752,8 +752,6 @@ static ccl_status merge_width(int64_t* cur, int64_t w, const char* dim) {
     return CCL_OK;
 }
 
-static int64_t padded(int64_t w, int64_t b) { return (w + b - 1) / b * b; }
-
 // units = schedulable CTAs (1-CTA kernel) or CTA pairs (2-CTA kernel) the device can hold at once
 static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, const void* A, const void* B, const void* C, int sms, int pairs, GemmPlan* plan) {
     if (!d) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: NULL descriptor");
@@ -1003,8 +1001,7 @@ template <int BN, int CTAS, bool SWIGLU = false>
 static ccl_status launch(const GemmPlan& plan, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, cudaStream_t st) {
     ccl_status s = configure<BN, CTAS, SWIGLU>(plan.smem_bytes);
     if (s) return s;
-    cudaLaunchConfig_t cfg;
-    std::memset(&cfg, 0, sizeof(cfg));
+    cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(plan.grid, 1, 1);
     cfg.blockDim = dim3(kGemmThreads, 1, 1);
     cfg.dynamicSmemBytes = plan.smem_bytes;
@@ -1025,8 +1022,7 @@ static int resident_pairs() {
     if (pairs >= 0) return pairs;
     uint32_t smem = kSmemBudget + kEpiBytes + 2048;
     if (configure<256, 2>(smem) != CCL_OK) { clear_error(); return pairs = 0; }
-    cudaLaunchConfig_t cfg;
-    std::memset(&cfg, 0, sizeof(cfg));
+    cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2, 1, 1); cfg.blockDim = dim3(kGemmThreads, 1, 1); cfg.dynamicSmemBytes = smem;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;

@@ -259,7 +259,7 @@ extern "C" ccl_status ccl_repack(const ccl_mat* m, const void* src_dev, void* ds
     if ((reinterpret_cast<uintptr_t>(src_dev) % v.e) || (reinterpret_cast<uintptr_t>(dst_dev) % v.e))
         return fail(CCL_ERR_ALIGN, "ccl_repack: buffers must be aligned to elem_bytes");
     cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
-    int sms;
+    int sms = 0;
     s = sm_count(&sms);
     if (s) return s;
 
