@@ -116,6 +116,23 @@ def gemm(A, B, M, N, K, a_trans=0, b_trans=0, block=None, want64=False, threads=
     return ref32, ref64, out
 
 
+def gemm_axpby(A, B, Cin, M, N, K, alpha, beta, a_trans=0, b_trans=0, threads=None):
+    """alpha * A*B + beta * Cin (Cin: logical [M x N] bf16 bits).  Returns (ref32, out_bf16_bits)."""
+    A = np.ascontiguousarray(A, dtype=np.uint16).reshape(-1)
+    B = np.ascontiguousarray(B, dtype=np.uint16).reshape(-1)
+    Cin = np.ascontiguousarray(Cin, dtype=np.uint16).reshape(-1)
+    assert A.size == M * K and B.size == K * N and Cin.size == M * N
+    ref32 = np.empty((M, N), dtype=np.float32)
+    out = np.empty((M, N), dtype=np.uint16)
+    if threads is None:
+        threads = os.cpu_count() or 1
+    rc = lib().orc_gemm_axpby(C.c_int64(M), C.c_int64(N), C.c_int64(K), _p(A), C.c_int(a_trans), _p(B), C.c_int(b_trans),
+                              C.c_double(alpha), C.c_double(beta), _p(Cin), _p(ref32), _p(out), C.c_int(threads))
+    if rc:
+        raise ValueError("orc_gemm_axpby rejected the arguments")
+    return ref32, out
+
+
 def gemm_swiglu(A, B, M, N, K, P=1, a_trans=0, b_trans=0, threads=None):
     """silu(gate) * up on the product of a fused gate/up operand whose column strips (P of them) hold gate | up halves.
     Returns (ref32 [M x N/2], out_bf16_bits)."""

@@ -28,6 +28,7 @@
 //                   worked example, reshape/permute, slice sizes of Sec. 2.2)
 //   repack        : pinned (permutation, round trip, strided-slice copies)
 //   gemm          : pinned (identity, all-ones, library matmul, fp64 bound)
+//   gemm_axpby    : pinned (alpha = 1, beta = 0 is gemm; alpha = 0, beta = 1 returns C; exact small integers)
 //   gemm_swiglu   : pinned (gate/up pairing enumerated by hand, silu closed forms, numpy in float64)
 //   traffic       : pinned by invariants, closed forms and a hand-enumerated
 //                   tiny case; against the paper's Fig. 6 ratios it is
@@ -421,6 +422,22 @@ int orc_gemm(int64_t M, int64_t N, int64_t K, const uint16_t* A, int a_trans, co
 }
 
 uint16_t orc_f32_to_bf16(float f) { return f32_to_bf16_rne(f); }
+
+// The BLAS form of Sec. 2.2: C <- alpha * A*B + beta * C ("the scalars do not affect placement and the C read shares
+// the partitioning of the output write").  Cin is the logical [M x N] bf16 matrix read; the fp32 sequential-k sum of
+// orc_gemm is scaled and added to beta * Cin in double, then rounded once to fp32 (ref32) and to bf16 (out_bf16).
+int orc_gemm_axpby(int64_t M, int64_t N, int64_t K, const uint16_t* A, int a_trans, const uint16_t* B, int b_trans,
+                   double alpha, double beta, const uint16_t* Cin, float* ref32, uint16_t* out_bf16, int threads) {
+    if (!Cin) return -1;
+    std::vector<float> H((size_t)(M * N));
+    if (orc_gemm(M, N, K, A, a_trans, B, b_trans, 0, M, 0, N, H.data(), nullptr, nullptr, threads)) return -1;
+    for (int64_t i = 0; i < M * N; ++i) {
+        const float v = (float)(alpha * (double)H[(size_t)i] + beta * (double)bf16_to_f32(Cin[i]));
+        if (ref32) ref32[i] = v;
+        if (out_bf16) out_bf16[i] = f32_to_bf16_rne(v);
+    }
+    return 0;
+}
 
 // Gated FFN activation on the product of a fused gate/up operand (the operand of Fig. 3; Sec. 3.3: activations are
 // produced directly by upstream kernels).  H = A*B is [M x N], N even, its columns cut into P strips of width

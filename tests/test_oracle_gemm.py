@@ -83,3 +83,42 @@ def test_block_equals_slice_of_full():
     np.testing.assert_array_equal(blk, full[10:50, 33:80])
     one, _, _ = orc.gemm(synth.bits(A), synth.bits(B), M, N, K, threads=1)
     np.testing.assert_array_equal(one, full)
+
+
+def test_axpby_special_cases_and_exact_integers():
+    """alpha * A*B + beta * C (Sec. 2.2): reduces to the pinned GEMM, to C itself, and is exact on small integers."""
+    rng = np.random.default_rng(11)
+    M, N, K = 7, 10, 33
+
+    def bf(x):
+        u = np.asarray(x, dtype=np.float32).view(np.uint32)
+        return ((u + 0x7FFF + ((u >> 16) & 1)) >> 16).astype(np.uint16)
+
+    def f32(b):
+        return (np.asarray(b, dtype=np.uint16).astype(np.uint32) << 16).view(np.float32)
+
+    A = bf(rng.standard_normal((M, K)).astype(np.float32))
+    B = bf(rng.standard_normal((K, N)).astype(np.float32))
+    Cin = bf(rng.standard_normal((M, N)).astype(np.float32))
+    H32, _, Hb = orc.gemm(A, B, M, N, K)
+    r, o = orc.gemm_axpby(A, B, Cin, M, N, K, 1.0, 0.0)
+    np.testing.assert_array_equal(r, H32)
+    np.testing.assert_array_equal(o, Hb)
+    r, o = orc.gemm_axpby(A, B, Cin, M, N, K, 0.0, 1.0)
+    np.testing.assert_array_equal(o, Cin.reshape(M, N))                      # C comes back bit for bit
+    r2, _ = orc.gemm_axpby(A, B, Cin, M, N, K, 2.0, 0.0)
+    np.testing.assert_array_equal(r2, 2.0 * H32)                             # scaling by a power of two is exact
+    r3, _ = orc.gemm_axpby(A, B, Cin, M, N, K, -0.5, 3.0)
+    want = -0.5 * H32.astype(np.float64) + 3.0 * f32(Cin).reshape(M, N).astype(np.float64)
+    np.testing.assert_allclose(r3, want, rtol=1e-7, atol=0)
+    # small integers: everything exact
+    Ai = bf(rng.integers(-3, 4, size=(M, K)).astype(np.float32))
+    Bi = bf(rng.integers(-3, 4, size=(K, N)).astype(np.float32))
+    Ci = bf(rng.integers(-8, 9, size=(M, N)).astype(np.float32))
+    ri, _ = orc.gemm_axpby(Ai, Bi, Ci, M, N, K, 2.0, -3.0)
+    wi = 2.0 * (f32(Ai).reshape(M, K).astype(np.int64) @ f32(Bi).reshape(K, N).astype(np.int64)) - 3.0 * f32(Ci).reshape(M, N)
+    np.testing.assert_array_equal(ri, wi.astype(np.float32))
+    # transposed storage of A and B changes nothing
+    rT, _ = orc.gemm_axpby(np.ascontiguousarray(A.reshape(M, K).T), np.ascontiguousarray(B.reshape(K, N).T), Cin, M, N, K, -0.5, 3.0,
+                           a_trans=1, b_trans=1)
+    np.testing.assert_array_equal(rT, r3)
