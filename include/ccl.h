@@ -144,6 +144,16 @@ ccl_status ccl_gemm_workspace(const ccl_gemm_desc* d, size_t* bytes);
 ccl_status ccl_gemm(const ccl_gemm_desc* d, const void* A_dev, const void* B_dev, void* C_dev, void* ws_dev,
                     size_t ws_bytes, void* cuda_stream);
 /*
+ * The BLAS form (Sec. 2.2: "the extension to alpha*A*B + beta*C is straightforward, since the scalars do not affect
+ * placement and the C read shares the same partitioning as the output write"):
+ *   C <- bf16( alpha * (A*B) + beta * C ),  fp32 arithmetic on the fp32 accumulator, one rounding.
+ * C is read (only when beta != 0) and written through the same descriptor d->C; every tile reads its own part
+ * of C before it writes it, so C_dev may hold anything when beta = 0.  alpha = 1, beta = 0 is ccl_gemm, bit for
+ * bit.  Workspace, requirements, asynchrony and errors as for ccl_gemm; NaN scalars -> CCL_ERR_INVALID_ARG.
+ */
+ccl_status ccl_gemm_axpby(const ccl_gemm_desc* d, float alpha, float beta, const void* A_dev, const void* B_dev,
+                          void* C_dev, void* ws_dev, size_t ws_bytes, void* cuda_stream);
+/*
  * `batch` independent GEMMs of one shape and one set of layouts in a single launch, e.g. the expert
  * projections of a mixture-of-experts FFN (Sec. 4.1 evaluates the Qwen expert GEMMs one at a time; the
  * paper has no batched call: the batch only amortises the launch and fills the machine with small problems).

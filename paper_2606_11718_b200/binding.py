@@ -20,7 +20,7 @@ PLACE_RR, PLACE_BLOCK, PLACE_BEST = 0, 1, 2
 ASSIGN_N_STRIPS, ASSIGN_M_STRIPS, ASSIGN_EXPLICIT = 0, 1, 2
 
 EXPORTS = ["ccl_map_offset", "ccl_map_inverse", "ccl_buffer_bytes", "ccl_strip_stride", "ccl_repack", "ccl_gemm_workspace",
-           "ccl_gemm", "ccl_gemm_batched_workspace", "ccl_gemm_batched", "ccl_gemm_swiglu", "ccl_gemm_static_ws", "ccl_gemm_status", "ccl_traffic_sizes", "ccl_traffic", "ccl_traffic_l2", "ccl_last_error", "ccl_launch_count", "ccl_version"]
+           "ccl_gemm", "ccl_gemm_batched_workspace", "ccl_gemm_batched", "ccl_gemm_axpby", "ccl_gemm_swiglu", "ccl_gemm_static_ws", "ccl_gemm_status", "ccl_traffic_sizes", "ccl_traffic", "ccl_traffic_l2", "ccl_last_error", "ccl_launch_count", "ccl_version"]
 
 
 class CclError(RuntimeError):
@@ -76,6 +76,7 @@ def lib():
         l.ccl_gemm_batched_workspace.argtypes = [C.POINTER(GemmDesc), C.c_int32, C.POINTER(C.c_size_t)]
         l.ccl_gemm_batched.argtypes = [C.POINTER(GemmDesc), C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64,
                                        C.c_void_p, C.c_size_t, C.c_void_p]
+        l.ccl_gemm_axpby.argtypes = [C.POINTER(GemmDesc), C.c_float, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         l.ccl_gemm_swiglu.argtypes = [C.POINTER(GemmDesc), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         l.ccl_gemm_static_ws.argtypes = [C.POINTER(GemmDesc), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         l.ccl_gemm_status.argtypes = [C.c_void_p, C.POINTER(C.c_int32)]
@@ -175,6 +176,15 @@ def ccl_gemm_batched(d, batch, A, a_stride, B, b_stride, Cout, c_stride, ws=None
             raise ValueError("ccl_gemm_batched: operand buffer too small")
     ws_bytes = ws.numel() * ws.element_size() if ws is not None else 0
     _check(lib().ccl_gemm_batched(C.byref(d), batch, _ptr(A), a_stride, _ptr(B), b_stride, _ptr(Cout), c_stride, _ptr(ws), ws_bytes, _stream()))
+
+
+def ccl_gemm_axpby(d, alpha, beta, A, B, Cinout, ws=None):
+    """C <- alpha * A*B + beta * C."""
+    for t, m in ((A, d.A), (B, d.B), (Cinout, d.C)):
+        if t.numel() * t.element_size() < ccl_buffer_bytes(m):
+            raise ValueError("ccl_gemm_axpby: operand buffer too small")
+    ws_bytes = ws.numel() * ws.element_size() if ws is not None else 0
+    _check(lib().ccl_gemm_axpby(C.byref(d), alpha, beta, _ptr(A), _ptr(B), _ptr(Cinout), _ptr(ws), ws_bytes, _stream()))
 
 
 def ccl_gemm_swiglu(d, A, B, Cout):

@@ -117,6 +117,9 @@ struct GemmParams {
     // apart inside a strip of 2 * pair_dist
     int32_t pair_dist;
     FastDiv fd_wn;
+    // C <- alpha * A*B + beta * C (ccl_gemm_axpby); axpby = 0 when alpha = 1 and beta = 0 (C is then never read)
+    int32_t axpby;
+    float alpha, beta;
     int64_t c_batch_stride;         // elements between the C buffers of consecutive problems
     OpMap a, b;
     int32_t a_mn, b_mn;             // 1 = MN-major operand tile in shared memory
@@ -214,6 +217,13 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 __device__ __forceinline__ void st_global_v4_if(void* ptr, uint4 v, bool pred) {
     asm volatile("{\n .reg .pred q;\n setp.ne.b32 q, %5, 0;\n @q st.global.v4.b32 [%0], {%1, %2, %3, %4};\n}"
                  ::"l"(ptr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w), "r"((uint32_t)pred) : "memory");
+}
+// 16-byte global load under a predicate (zeros when it is off), without a branch
+__device__ __forceinline__ uint4 ld_global_v4_if(const void* ptr, bool pred) {
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    asm volatile("{\n .reg .pred q;\n setp.ne.b32 q, %5, 0;\n @q ld.global.v4.b32 {%0, %1, %2, %3}, [%4];\n}"
+                 : "+r"(v.x), "+r"(v.y), "+r"(v.z), "+r"(v.w) : "l"(ptr), "r"((uint32_t)pred) : "memory");
+    return v;
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 // The loaded registers only hold their values once the wait above has run, but to the compiler they were defined by
@@ -572,8 +582,28 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     if (n64 + j * 4 < t.n1)
                         st_global_v4_if(wrow + n64 + j * 4, make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]), row_ok);
             };
+            // acc <- alpha * acc + beta * C for this lane's 64 columns (C read in its own layout, fp32 arithmetic)
+            auto axpby_piece = [&](uint32_t (&r)[64], int c) {
+                const int n64 = nb + c * 64;
+                const bool row_ok = m < t.m1;
+                const unsigned short* src = p.C + c_offset(p, min(m, t.m1 - 1), n64) + (int64_t)t.e * p.c_batch_stride;
+                const float alpha = p.alpha, beta = p.beta;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    uint4 cv = make_uint4(0u, 0u, 0u, 0u);
+                    if (beta != 0.0f && n64 + j * 8 < t.n1) cv = ld_global_v4_if(src + j * 8, row_ok);
+                    const uint32_t w[4] = {cv.x, cv.y, cv.z, cv.w};
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {                       // bf16 -> fp32 is a shift
+                        const float c0 = __uint_as_float(w[i] << 16), c1 = __uint_as_float(w[i] & 0xFFFF0000u);
+                        r[j * 8 + 2 * i] = __float_as_uint(fmaf(alpha, __uint_as_float(r[j * 8 + 2 * i]), beta * c0));
+                        r[j * 8 + 2 * i + 1] = __float_as_uint(fmaf(alpha, __uint_as_float(r[j * 8 + 2 * i + 1]), beta * c1));
+                    }
+                }
+            };
             auto store_piece = [&](uint32_t (&r)[64], int c) {
                 if (p.splits > 1) { store_partial(r, c); return; }
+                if (p.axpby) axpby_piece(r, c);
                 uint32_t pk[32];
                 pack(r, pk);
                 store_packed(pk, c);
@@ -679,6 +709,16 @@ __global__ void __launch_bounds__(256) splitk_reduce_kernel(const GemmParams p) 
             acc[4] += y.x; acc[5] += y.y; acc[6] += y.z; acc[7] += y.w;
         }
         const int64_t off = c_offset(p, m, n) + e * p.c_batch_stride;
+        if (p.axpby) {
+            uint4 cv = make_uint4(0u, 0u, 0u, 0u);
+            if (p.beta != 0.0f) cv = *reinterpret_cast<const uint4*>(p.C + off);
+            const uint32_t w[4] = {cv.x, cv.y, cv.z, cv.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                acc[2 * i] = fmaf(p.alpha, acc[2 * i], p.beta * __uint_as_float(w[i] << 16));
+                acc[2 * i + 1] = fmaf(p.alpha, acc[2 * i + 1], p.beta * __uint_as_float(w[i] & 0xFFFF0000u));
+            }
+        }
         uint4 v;
         __nv_bfloat162 h;
         h = __floats2bfloat162_rn(acc[0], acc[1]); v.x = *reinterpret_cast<uint32_t*>(&h);
@@ -1044,6 +1084,7 @@ struct PreparedKey {
     int64_t f[36];          // every field of the descriptor, the batch, the three pointers, the device and the tuning overrides
     int dev;
     int mode;               // 0 plain, 1 gated activation
+    float alpha, beta;
     char env[60];
 };
 struct Prepared {
@@ -1111,7 +1152,7 @@ extern "C" ccl_status ccl_gemm_batched_workspace(const ccl_gemm_desc* d, int32_t
 
 // strides[X]: bytes between the buffers of operand X (A, B, C) of consecutive problems; 0 = shared (A and B only)
 static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, const int64_t* strides, const void* A_dev, const void* B_dev, void* C_dev,
-                            void* ws_dev, size_t ws_bytes, void* cuda_stream) {
+                            void* ws_dev, size_t ws_bytes, void* cuda_stream, float alpha = 1.0f, float beta = 0.0f) {
     if (!A_dev || !B_dev || !C_dev) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: NULL operand");
     if (!d) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: NULL descriptor");
     if (batch < 1 || batch > kMaxBatch) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: batch must be in [1, %lld]", (long long)kMaxBatch);
@@ -1120,7 +1161,7 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     // reuse the plan and the two encoded tensor maps: a host-side cache only, nothing is kept on the device.
     PreparedKey key;
     make_key(d, batch4, A_dev, B_dev, C_dev, &key);
-    key.mode = swiglu ? 1 : 0;
+    key.mode = swiglu ? 1 : 0; key.alpha = alpha; key.beta = beta;
     Prepared prep;
     bool hit = false;
     {
@@ -1147,11 +1188,12 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
         int dev;
         CCL_CUDA_TRY(cudaGetDevice(&dev));
         CCL_CUDA_TRY(cudaDeviceGetAttribute(&prep.sms, cudaDevAttrMultiProcessorCount, dev));
-        if (dev != key.dev) { make_key(d, batch4, A_dev, B_dev, C_dev, &key); key.mode = swiglu ? 1 : 0; }
+        if (dev != key.dev) { make_key(d, batch4, A_dev, B_dev, C_dev, &key); key.mode = swiglu ? 1 : 0; key.alpha = alpha; key.beta = beta; }
         if ((s = make_plan(d, batch, swiglu, A_dev, B_dev, C_dev, prep.sms, resident_pairs(), &plan))) return s;
         plan.p.C = static_cast<uint16_t*>(C_dev);
         plan.p.a.batched = batch4[1] != 0; plan.p.b.batched = batch4[2] != 0; plan.p.c.batched = 1;
         plan.p.c_batch_stride = batch4[3] / 2;
+        plan.p.alpha = alpha; plan.p.beta = beta; plan.p.axpby = (alpha != 1.0f || beta != 0.0f) ? 1 : 0;
         const uint32_t bnh = (uint32_t)(plan.subn / plan.ctas);   // B rows of one K-major box
         if (!plan.p.a_mn) s = operand_tmap(&prep.ma, plan.va, A_dev, BK, BM, batch, batch4[1]); else s = operand_tmap(&prep.ma, plan.va, A_dev, 64, BK, batch, batch4[1]);
         if (s) return s;
@@ -1204,6 +1246,13 @@ extern "C" ccl_status ccl_gemm_batched(const ccl_gemm_desc* d, int32_t batch, co
     if (a_stride_bytes < 0 || b_stride_bytes < 0 || c_stride_bytes < 0) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm_batched: negative stride");
     const int64_t strides[3] = {a_stride_bytes, b_stride_bytes, c_stride_bytes};
     return gemm_impl(d, batch, false, strides, A_dev, B_dev, C_dev, ws_dev, ws_bytes, cuda_stream);
+}
+
+extern "C" ccl_status ccl_gemm_axpby(const ccl_gemm_desc* d, float alpha, float beta, const void* A_dev, const void* B_dev, void* C_dev,
+                                     void* ws_dev, size_t ws_bytes, void* cuda_stream) {
+    if (!(alpha == alpha) || !(beta == beta)) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm_axpby: alpha / beta is NaN");
+    const int64_t none[3] = {0, 0, 0};
+    return gemm_impl(d, 1, false, none, A_dev, B_dev, C_dev, ws_dev, ws_bytes, cuda_stream, alpha, beta);
 }
 
 extern "C" ccl_status ccl_gemm_swiglu(const ccl_gemm_desc* d, const void* A_dev, const void* B_dev, void* C_dev, void* cuda_stream) {

@@ -334,3 +334,57 @@ def test_gemm_small_m_sweep_llama_shapes(name):
             if full is not None:
                 err = np.abs(gf - full) / np.maximum(1.0, np.abs(full))
                 assert err.max() <= tol(K)
+
+
+AXPBY = [
+    # M, N, K, P, layouts, a_trans, b_trans, out_part, alpha, beta
+    (130, 384, 96, 2, ("row", "ccl", "ccl"), 0, 0, 2, 0.5, 2.0),          # ragged tiles, CCL output read and written
+    (264, 768, 328, 4, ("row", "ccl", "row"), 1, 0, 2, -1.25, 0.75),
+    (512, 1024, 256, 4, ("row", "ccl", "ccl"), 0, 1, 2, 1.0, 1.0),         # accumulation into C (e.g. weight gradients)
+    (16, 1024, 2048, 2, ("row", "ccl", "ccl"), 0, 0, 2, 2.0, -0.5),        # split along K: the reduction applies the scalars
+    (300, 1024, 256, 4, ("row", "ileave", "ileave"), 0, 0, 2, 0.25, 3.0),  # page-interleaved C
+    (640, 2560, 512, 2, ("row", "ccl", "ccl"), 0, 0, 2, 3.0, 0.0),         # beta = 0: C is not read
+]
+
+
+@pytest.mark.parametrize("M,N,K,P,lay,at,bt,op,alpha,beta", AXPBY)
+def test_gemm_axpby(M, N, K, P, lay, at, bt, op, alpha, beta, cta_mode):
+    """C <- alpha * A*B + beta * C (Sec. 2.2) against the oracle; tolerance: the GEMM's, scaled by |alpha|, plus the bf16
+    rounding of the result (2^-8 relative)."""
+    A, B = synth.gemm_operands(M, N, K, at, bt, seed=9, tag="axpby")
+    Cin = synth.randn_bf16(M, N, 1.0, 9, "axpby/C")
+    d = gemm_desc(M, N, K, P, lay, at, bt, op, 1, align=1024 if "ileave" in lay else 0)
+    a_dev, b_dev = to_layout(synth.bits(A), d.A), to_layout(synth.bits(B), d.B)
+    nc = ccl.ccl_buffer_bytes(d.C) // 2
+    c_dev = torch.full((nc + GUARD,), 0x7FC0, dtype=torch.int16, device="cuda")
+    if beta != 0.0:
+        c_dev[:nc] = to_layout(synth.bits(Cin), d.C)
+    need = ccl.ccl_gemm_workspace(d)
+    ws = torch.full((need // 4,), float("nan"), dtype=torch.float32, device="cuda") if need else None
+    ccl.ccl_gemm_axpby(d, alpha, beta, a_dev, b_dev, c_dev, ws)
+    assert ccl.ccl_gemm_status()[0] == ccl.OK
+    assert (c_dev[nc:] == 0x7FC0).all(), "the kernel wrote past the end of C"
+    got = synth.from_bits(from_layout(c_dev[:nc], d.C)).to(torch.float32).numpy()
+    ref32, _ = orc.gemm_axpby(synth.bits(A), synth.bits(B), synth.bits(Cin), M, N, K, alpha, beta, at, bt)
+    assert np.isfinite(got).all()
+    err = np.abs(got - ref32) / np.maximum(1.0, np.abs(ref32))
+    assert err.max() <= abs(alpha) * tol(K) + 2.0 ** -8, err.max()
+
+
+def test_gemm_axpby_identity_scalars_equal_plain_gemm():
+    M, N, K, P = 384, 1536, 512, 4
+    A, B = synth.gemm_operands(M, N, K, 0, 0, seed=10, tag="axpby1")
+    d = gemm_desc(M, N, K, P, ("row", "ccl", "ccl"), 0, 0, 2, 1)
+    want = run_gemm(d, A, B)
+    a_dev, b_dev = to_layout(synth.bits(A), d.A), to_layout(synth.bits(B), d.B)
+    c_dev = torch.full((ccl.ccl_buffer_bytes(d.C) // 2,), 0x7FC0, dtype=torch.int16, device="cuda")
+    ccl.ccl_gemm_axpby(d, 1.0, 0.0, a_dev, b_dev, c_dev)
+    np.testing.assert_array_equal(from_layout(c_dev, d.C), want)
+    # alpha = 0, beta = 1 leaves C as it was
+    Cin = synth.randn_bf16(M, N, 1.0, 10, "axpby1/C")
+    c_dev = to_layout(synth.bits(Cin), d.C)
+    ccl.ccl_gemm_axpby(d, 0.0, 1.0, a_dev, b_dev, c_dev)
+    np.testing.assert_array_equal(from_layout(c_dev, d.C), synth.bits(Cin))
+    with pytest.raises(ccl.CclError) as ei:
+        ccl.ccl_gemm_axpby(d, float("nan"), 0.0, a_dev, b_dev, c_dev)
+    assert ei.value.status == ccl.ERR_INVALID_ARG
