@@ -150,6 +150,22 @@ def gemm_swiglu(A, B, M, N, K, P=1, a_trans=0, b_trans=0, threads=None):
     return ref32, out
 
 
+class L2Model(C.Structure):
+    """orc_l2_model"""
+    _fields_ = [("capacity_bytes", C.c_int64), ("line_bytes", C.c_int32), ("ways", C.c_int32), ("traversal", C.c_int32)]
+
+    def __init__(self, capacity_bytes=8 << 20, line_bytes=128, ways=16, traversal=0):
+        super().__init__(capacity_bytes, line_bytes, ways, traversal)
+
+
+def traffic_lru(d, l2):
+    """Local / remote bytes [3,2] behind a finite LRU L2 per chiplet (the model stated in ccl_oracle.cpp)."""
+    totals = np.zeros((3, 2), dtype=np.uint64)
+    if lib().orc_traffic_lru(C.byref(d), C.byref(l2), _p(totals)):
+        raise ValueError("orc_traffic_lru rejected the arguments")
+    return totals
+
+
 def traffic_sizes(d):
     nt = C.c_int64()
     pages = (C.c_int64 * 3)()

@@ -30,6 +30,9 @@
 //   gemm          : pinned (identity, all-ones, library matmul, fp64 bound)
 //   gemm_axpby    : pinned (alpha = 1, beta = 0 is gemm; alpha = 0, beta = 1 returns C; exact small integers)
 //   gemm_swiglu   : pinned (gate/up pairing enumerated by hand, silu closed forms, numpy in float64)
+//   traffic_lru   : the finite-L2 model is this file's own reading of Sec. 4.1; pinned by its limits (one-line cache =
+//                   uncached count in whole lines, unbounded cache = ideal-L2 count, monotone in the ways) and a
+//                   hand-run example; against the paper's Fig. 6 numbers it is PARITY UNPINNED (unreleased simulator)
 //   traffic       : pinned by invariants, closed forms and a hand-enumerated
 //                   tiny case; against the paper's Fig. 6 ratios it is
 //                   PARITY UNPINNED (they need the unreleased L2 simulator).
@@ -536,6 +539,86 @@ int orc_traffic_ideal_l2(const orc_traffic_desc* d, const int32_t* explicit_q, u
 // The same count taken run by run (a stored row of a tile is one contiguous run per strip,
 // cut at page boundaries).  Validated against orc_traffic_elem in the tests; used at sizes
 // where the element walk would take minutes.
+// Remote traffic behind a FINITE private L2 per chiplet (Sec. 4.1: "per-chiplet L2 caches", 8 MB, 128-byte lines,
+// 16 ways; the metric counts "remote operand reads that miss in L2, and remote output writes").  What the paper
+// leaves open is fixed here as the simplest tile-level model:
+//   * every chiplet has its own cache of capacity_bytes / (line_bytes * ways) sets, set = line number mod sets,
+//     LRU replacement inside a set; the lines of A and of B are numbered from the start of their own buffers
+//     (assumed line-aligned) and carry the operand in their tag;
+//   * the CTAs of a chiplet (its tiles, as enumerate_tiles assigns them) run one after the other, in row-major
+//     order of the tile grid (traversal 0: n fastest) or column-major (traversal 1: m fastest);
+//   * a CTA touches every line of its A rectangle in address order, then every line of its B rectangle in address
+//     order (each line once per CTA); a hit costs nothing, a miss fetches the whole line from the page's owner:
+//     line_bytes local or remote bytes; page_bytes must be a multiple of line_bytes;
+//   * C is written once, past the cache: the C row of the totals is the one of the uncached count.
+// Placement policies: RR and BLOCK.
+typedef struct { int64_t capacity_bytes; int32_t line_bytes; int32_t ways; int32_t traversal; } orc_l2_model;
+
+int orc_traffic_lru(const orc_traffic_desc* d, const orc_l2_model* l2, uint64_t* totals) {
+    if (!traffic_desc_ok(*d) || !l2) return -1;
+    if (l2->line_bytes <= 0 || l2->ways <= 0 || l2->capacity_bytes <= 0 || (l2->traversal != 0 && l2->traversal != 1)) return -1;
+    if (l2->capacity_bytes % ((int64_t)l2->line_bytes * l2->ways) || d->page_bytes % l2->line_bytes) return -1;
+    if (d->assign == ORC_ASSIGN_EXPLICIT) return -1;
+    const int64_t L = l2->line_bytes, sets = l2->capacity_bytes / (L * l2->ways);
+    std::vector<Tile> tiles;
+    if (enumerate_tiles(*d, nullptr, tiles)) return -1;
+    const orc_mat* ms[3] = {&d->A, &d->B, &d->C};
+    for (int i = 0; i < 6; ++i) totals[i] = 0;
+    for (int X = 0; X < 3; ++X) if (d->place[X] == ORC_PLACE_BEST) return -1;
+    // C: written once, uncached
+    {
+        const orc_mat& m = d->C;
+        const int64_t bytes_total = buffer_elems(m) * m.elem_bytes;
+        for (const Tile& t : tiles)
+            for (int64_t r = t.m0; r < t.m1; ++r)
+                for (int64_t c = t.n0; c < t.n1; ++c) {
+                    const int64_t page = map_offset(m, r, c) * m.elem_bytes / d->page_bytes;
+                    totals[4 + (fixed_owner(d->place[2], page, d->page_bytes, d->P, bytes_total) == t.q ? 0 : 1)] += (uint64_t)m.elem_bytes;
+                }
+    }
+    // the order in which a chiplet runs its tiles
+    std::vector<size_t> order(tiles.size());
+    for (size_t i = 0; i < tiles.size(); ++i) order[i] = i;
+    std::stable_sort(order.begin(), order.end(), [&](size_t a, size_t b) {
+        const Tile &x = tiles[a], &y = tiles[b];
+        if (l2->traversal == 0) return x.m0 != y.m0 ? x.m0 < y.m0 : x.n0 < y.n0;
+        return x.n0 != y.n0 ? x.n0 < y.n0 : x.m0 < y.m0;
+    });
+    for (int q = 0; q < d->P; ++q) {
+        // cache[set] = tags from most to least recently used; tag = line * 2 + operand
+        std::vector<std::vector<int64_t>> cache((size_t)sets);
+        for (size_t oi : order) {
+            const Tile& t = tiles[oi];
+            if (t.q != q) continue;
+            for (int X = 0; X < 2; ++X) {
+                const orc_mat& m = *ms[X];
+                const int64_t bytes_total = buffer_elems(m) * m.elem_bytes;
+                int64_t r0, r1, c0, c1; tile_rect(*d, t, X, r0, r1, c0, c1);
+                std::vector<int64_t> lines;
+                for (int64_t r = r0; r < r1; ++r)
+                    for (int64_t c = c0; c < c1; ++c) {
+                        const int64_t b = map_offset(m, r, c) * m.elem_bytes;
+                        lines.push_back(b / L);
+                        lines.push_back((b + m.elem_bytes - 1) / L);
+                    }
+                std::sort(lines.begin(), lines.end());
+                lines.erase(std::unique(lines.begin(), lines.end()), lines.end());
+                for (int64_t line : lines) {
+                    std::vector<int64_t>& set = cache[(size_t)(line % sets)];
+                    const int64_t tag = line * 2 + X;
+                    auto it = std::find(set.begin(), set.end(), tag);
+                    if (it != set.end()) { set.erase(it); set.insert(set.begin(), tag); continue; }      // hit
+                    set.insert(set.begin(), tag);
+                    if ((int64_t)set.size() > l2->ways) set.pop_back();
+                    const int64_t page = line * L / d->page_bytes;
+                    totals[X * 2 + (fixed_owner(d->place[X], page, d->page_bytes, d->P, bytes_total) == q ? 0 : 1)] += (uint64_t)L;
+                }
+            }
+        }
+    }
+    return 0;
+}
+
 int orc_traffic_runs(const orc_traffic_desc* d, const int32_t* explicit_q, uint64_t* per_cta, uint64_t* const* per_page,
                      uint8_t* const* owner, uint64_t* totals) {
     return traffic_impl<true>(*d, explicit_q, per_cta, per_page, owner, totals);

@@ -1,0 +1,73 @@
+"""Pins of the oracle's finite-L2 traffic model (orc_traffic_lru): a hand-run access string, and the two limits in
+which it must reduce to counts that are pinned elsewhere -- a one-line cache (nothing is ever reused: the uncached
+count, in whole lines) and an unbounded cache (every chiplet fetches a line once: the ideal-L2 count).  No GPU."""
+import os
+
+import numpy as np
+import pytest
+
+import oracle as orc
+from helpers import traffic_pair
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+
+
+def test_hand_run():
+    do, _ = traffic_pair(2, 2, 64, 1, 4096, BM=1, BN=1)
+    for line in open(os.path.join(HERE, "golden", "lru_hand_run.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        sets, ways, a_bytes, b_bytes = (int(x) for x in line.split())
+        t = orc.traffic_lru(do, orc.L2Model(sets * ways * 128, 128, ways, 0))
+        assert (int(t[0].sum()), int(t[1].sum())) == (a_bytes, b_bytes), (sets, ways, t)
+        assert int(t[2].sum()) == 2 * 2 * 2                         # C: every element written once
+
+
+CASES = [
+    # M, N, K, P, page, layouts, placement: every tile row segment is a whole number of 128-byte lines
+    (256, 512, 128, 2, 4096, ("row", "row", "row"), (0, 0, 0)),
+    (256, 512, 128, 2, 4096, ("row", "ccl", "ccl"), (0, 1, 1)),
+    (384, 1024, 192, 4, 1024, ("row", "ccl", "ccl"), (0, 0, 0)),
+    (256, 512, 128, 4, 4096, ("ccl", "row", "ccl"), (1, 0, 1)),
+]
+
+
+@pytest.mark.parametrize("M,N,K,P,S,lay,place", CASES)
+@pytest.mark.parametrize("assign", [0, 1])
+@pytest.mark.parametrize("traversal", [0, 1])
+def test_limits(M, N, K, P, S, lay, place, assign, traversal):
+    do, _ = traffic_pair(M, N, K, P, S, lay, place, assign=assign, BM=128, BN=64, align=S)
+    plain = orc.traffic(do, level="runs")["totals"]
+    ideal = orc.traffic_ideal_l2(do)
+    one_line = orc.traffic_lru(do, orc.L2Model(128, 128, 1, traversal))
+    np.testing.assert_array_equal(one_line, plain)                  # no reuse at all
+    lines = sum(orc.buffer_bytes(m) for m in (do.A, do.B)) // 128
+    unbounded = orc.traffic_lru(do, orc.L2Model(128 * 2 * lines, 128, 2 * lines, traversal))
+    np.testing.assert_array_equal(unbounded, ideal)                 # each chiplet fetches a line once
+    # more ways over the same sets never miss more (LRU stack inclusion), and the C row never changes
+    prev = None
+    for ways in (1, 2, 4, 16):
+        t = orc.traffic_lru(do, orc.L2Model(8 * ways * 128, 128, ways, traversal))
+        np.testing.assert_array_equal(t[2], plain[2])
+        total = int(t[0].sum() + t[1].sum())
+        assert int(ideal[0].sum() + ideal[1].sum()) <= total <= int(plain[0].sum() + plain[1].sum())
+        if prev is not None:
+            assert total <= prev
+        prev = total
+
+
+def test_traversal_matters_and_rejections():
+    # one chiplet, a cache that holds one tile row of A but not all of B: row-major order reuses A, column-major B
+    do, _ = traffic_pair(512, 512, 256, 1, 4096, BM=128, BN=128)
+    cap = 128 * 256 * 2 + 128 * 256 * 2 + 4096                     # one A tile row + one B tile column + a little
+    cap -= cap % (128 * 16)
+    row = orc.traffic_lru(do, orc.L2Model(cap, 128, 16, 0))
+    col = orc.traffic_lru(do, orc.L2Model(cap, 128, 16, 1))
+    assert row[0].sum() < col[0].sum() and row[1].sum() > col[1].sum()
+    with pytest.raises(ValueError):
+        orc.traffic_lru(do, orc.L2Model(1000, 128, 16, 0))         # capacity not a whole number of sets
+    with pytest.raises(ValueError):
+        orc.traffic_lru(do, orc.L2Model(8 << 20, 128, 16, 2))      # unknown traversal
+    db, _ = traffic_pair(512, 512, 256, 2, 4096, place=(2, 2, 2))
+    with pytest.raises(ValueError):
+        orc.traffic_lru(db, orc.L2Model(8 << 20, 128, 16, 0))      # BEST placement is not modelled
