@@ -280,6 +280,36 @@ ccl_status ccl_traffic(const ccl_traffic_desc* d, const int32_t* cta_chiplet_dev
 ccl_status ccl_traffic_l2(const ccl_traffic_desc* d, const int32_t* cta_chiplet_dev, uint64_t* totals_l2_dev,
                           void* cuda_stream);
 
+/*
+ * The same count behind a FINITE private L2 per chiplet: the metric of Sec. 4.1 ("remote operand reads that miss in
+ * L2, and remote output writes"; 8 MB, 128-byte lines, 16 ways per chiplet).  The paper's simulator is not public;
+ * this is a tile-level model with everything it leaves open stated here:
+ *   - a chiplet's CTAs (its tiles under `assign`) run one after the other, in row-major order of the tile grid
+ *     (traversal = 0, n fastest) or column-major (traversal = 1, m fastest); the paper sweeps the traversal and
+ *     reports the best;
+ *   - a CTA touches every line of its A rectangle in address order, then every line of its B rectangle;
+ *   - each chiplet's cache has capacity_bytes / (line_bytes * ways) sets, LRU in a set; lines are numbered from the
+ *     start of each operand's buffer (assumed line-aligned) and the operand is part of the tag; set index:
+ *     hash = 0: line mod sets (the textbook index; power-of-two row pitches then pile up in a few sets),
+ *     hash = 1: (line + H(line div sets)) mod sets, H(b) = high 32 bits of b * 0x9E3779B97F4A7C15 -- a skew per
+ *     block of `sets` consecutive lines that stands in for the address hashing of a real L2;
+ *   - a miss fetches one whole line from the owner of its page: line_bytes local or remote bytes;
+ *   - C is written once, past the cache.
+ * totals_dev: uint64[3][2] (A, B, C) x (local, remote) bytes.
+ * Requirements: capacity a whole number of sets, ways <= 32, page_bytes a multiple of line_bytes (else
+ * CCL_ERR_INVALID_ARG / CCL_ERR_UNSUPPORTED); fixed placements only; CCL_ASSIGN_N_STRIPS or _M_STRIPS;
+ * A and B row-major or CCL (page-interleaved -> CCL_ERR_UNSUPPORTED).
+ * One thread simulates one cache set of one chiplet; cost grows with tiles x lines per tile / sets.
+ */
+typedef struct ccl_l2_model {
+    int64_t capacity_bytes; /* per chiplet */
+    int32_t line_bytes;
+    int32_t ways;
+    int32_t traversal;      /* 0 row-major over the tile grid, 1 column-major */
+    int32_t hash;           /* 0 set = line mod sets, 1 skewed index (see above) */
+} ccl_l2_model;
+ccl_status ccl_traffic_lru(const ccl_traffic_desc* d, const ccl_l2_model* m, uint64_t* totals_dev, void* cuda_stream);
+
 /* Message for the last non-OK status returned on this thread ("" if none). Static storage. */
 const char* ccl_last_error(void);
 /* Number of CUDA kernels this library has launched in this process (all threads, all streams). */

@@ -542,9 +542,11 @@ int orc_traffic_ideal_l2(const orc_traffic_desc* d, const int32_t* explicit_q, u
 // Remote traffic behind a FINITE private L2 per chiplet (Sec. 4.1: "per-chiplet L2 caches", 8 MB, 128-byte lines,
 // 16 ways; the metric counts "remote operand reads that miss in L2, and remote output writes").  What the paper
 // leaves open is fixed here as the simplest tile-level model:
-//   * every chiplet has its own cache of capacity_bytes / (line_bytes * ways) sets, set = line number mod sets,
-//     LRU replacement inside a set; the lines of A and of B are numbered from the start of their own buffers
-//     (assumed line-aligned) and carry the operand in their tag;
+//   * every chiplet has its own cache of capacity_bytes / (line_bytes * ways) sets, LRU replacement inside a set;
+//     the lines of A and of B are numbered from the start of their own buffers (assumed line-aligned) and carry the
+//     operand in their tag; set index: hash = 0: line mod sets (the textbook index: power-of-two row pitches pile up
+//     in a few sets); hash = 1: (line + H(line div sets)) mod sets with H(b) = high 32 bits of b * 0x9E3779B97F4A7C15
+//     (a skew per block of `sets` consecutive lines, standing in for the address hashing of a real L2);
 //   * the CTAs of a chiplet (its tiles, as enumerate_tiles assigns them) run one after the other, in row-major
 //     order of the tile grid (traversal 0: n fastest) or column-major (traversal 1: m fastest);
 //   * a CTA touches every line of its A rectangle in address order, then every line of its B rectangle in address
@@ -552,11 +554,19 @@ int orc_traffic_ideal_l2(const orc_traffic_desc* d, const int32_t* explicit_q, u
 //     line_bytes local or remote bytes; page_bytes must be a multiple of line_bytes;
 //   * C is written once, past the cache: the C row of the totals is the one of the uncached count.
 // Placement policies: RR and BLOCK.
-typedef struct { int64_t capacity_bytes; int32_t line_bytes; int32_t ways; int32_t traversal; } orc_l2_model;
+typedef struct { int64_t capacity_bytes; int32_t line_bytes; int32_t ways; int32_t traversal; int32_t hash; } orc_l2_model;
+
+static int64_t lru_set_index(int64_t line, int64_t sets, int hash) {
+    if (!hash) return line % sets;
+    const uint64_t block = (uint64_t)(line / sets);
+    const uint64_t skew = (block * 0x9E3779B97F4A7C15ull) >> 32;
+    return (int64_t)(((uint64_t)(line % sets) + skew % (uint64_t)sets) % (uint64_t)sets);
+}
 
 int orc_traffic_lru(const orc_traffic_desc* d, const orc_l2_model* l2, uint64_t* totals) {
     if (!traffic_desc_ok(*d) || !l2) return -1;
     if (l2->line_bytes <= 0 || l2->ways <= 0 || l2->capacity_bytes <= 0 || (l2->traversal != 0 && l2->traversal != 1)) return -1;
+    if (l2->hash != 0 && l2->hash != 1) return -1;
     if (l2->capacity_bytes % ((int64_t)l2->line_bytes * l2->ways) || d->page_bytes % l2->line_bytes) return -1;
     if (d->assign == ORC_ASSIGN_EXPLICIT) return -1;
     const int64_t L = l2->line_bytes, sets = l2->capacity_bytes / (L * l2->ways);
@@ -604,7 +614,7 @@ int orc_traffic_lru(const orc_traffic_desc* d, const orc_l2_model* l2, uint64_t*
                 std::sort(lines.begin(), lines.end());
                 lines.erase(std::unique(lines.begin(), lines.end()), lines.end());
                 for (int64_t line : lines) {
-                    std::vector<int64_t>& set = cache[(size_t)(line % sets)];
+                    std::vector<int64_t>& set = cache[(size_t)lru_set_index(line, sets, l2->hash)];
                     const int64_t tag = line * 2 + X;
                     auto it = std::find(set.begin(), set.end(), tag);
                     if (it != set.end()) { set.erase(it); set.insert(set.begin(), tag); continue; }      // hit

@@ -20,7 +20,7 @@ PLACE_RR, PLACE_BLOCK, PLACE_BEST = 0, 1, 2
 ASSIGN_N_STRIPS, ASSIGN_M_STRIPS, ASSIGN_EXPLICIT = 0, 1, 2
 
 EXPORTS = ["ccl_map_offset", "ccl_map_inverse", "ccl_buffer_bytes", "ccl_strip_stride", "ccl_repack", "ccl_gemm_workspace",
-           "ccl_gemm", "ccl_gemm_batched_workspace", "ccl_gemm_batched", "ccl_gemm_axpby", "ccl_gemm_swiglu", "ccl_gemm_static_ws", "ccl_gemm_status", "ccl_traffic_sizes", "ccl_traffic", "ccl_traffic_l2", "ccl_last_error", "ccl_launch_count", "ccl_version"]
+           "ccl_gemm", "ccl_gemm_batched_workspace", "ccl_gemm_batched", "ccl_gemm_axpby", "ccl_gemm_swiglu", "ccl_gemm_static_ws", "ccl_gemm_status", "ccl_traffic_sizes", "ccl_traffic", "ccl_traffic_l2", "ccl_traffic_lru", "ccl_last_error", "ccl_launch_count", "ccl_version"]
 
 
 class CclError(RuntimeError):
@@ -50,6 +50,15 @@ class TrafficDesc(C.Structure):
     _fields_ = [("M", C.c_int64), ("N", C.c_int64), ("K", C.c_int64), ("BM", C.c_int32), ("BN", C.c_int32),
                 ("A", Mat), ("B", Mat), ("C", Mat), ("a_trans", C.c_int32), ("b_trans", C.c_int32), ("P", C.c_int32),
                 ("page_bytes", C.c_int64), ("place", C.c_int32 * 3), ("assign", C.c_int32), ("strip_tiling", C.c_int32)]
+
+
+class L2Model(C.Structure):
+    """ccl_l2_model"""
+    _fields_ = [("capacity_bytes", C.c_int64), ("line_bytes", C.c_int32), ("ways", C.c_int32), ("traversal", C.c_int32),
+                ("hash", C.c_int32)]
+
+    def __init__(self, capacity_bytes=8 << 20, line_bytes=128, ways=16, traversal=0, hash=0):
+        super().__init__(capacity_bytes, line_bytes, ways, traversal, hash)
 
 
 _lib = None
@@ -84,6 +93,7 @@ def lib():
         l.ccl_traffic.argtypes = [C.POINTER(TrafficDesc), C.c_void_p, C.c_void_p, C.POINTER(C.c_void_p), C.POINTER(C.c_void_p),
                                   C.c_void_p, C.c_void_p]
         l.ccl_traffic_l2.argtypes = [C.POINTER(TrafficDesc), C.c_void_p, C.c_void_p, C.c_void_p]
+        l.ccl_traffic_lru.argtypes = [C.POINTER(TrafficDesc), C.POINTER(L2Model), C.c_void_p, C.c_void_p]
         _lib = l
     return _lib
 
@@ -226,6 +236,11 @@ def ccl_traffic(d, per_cta, totals, per_page=None, owner=None, cta_chiplet=None)
     pp = (C.c_void_p * 3)(*[(t.data_ptr() if t is not None else None) for t in per_page]) if per_page is not None else None
     ow = (C.c_void_p * 3)(*[(t.data_ptr() if t is not None else None) for t in owner]) if owner is not None else None
     _check(lib().ccl_traffic(C.byref(d), _ptr(cta_chiplet), _ptr(per_cta), pp, ow, _ptr(totals), _stream()))
+
+
+def ccl_traffic_lru(d, model, totals):
+    """Local / remote bytes [3,2] behind a finite LRU L2 per chiplet (tile-level model, see include/ccl.h)."""
+    _check(lib().ccl_traffic_lru(C.byref(d), C.byref(model), _ptr(totals), _stream()))
 
 
 def ccl_traffic_l2(d, totals_l2, cta_chiplet=None):

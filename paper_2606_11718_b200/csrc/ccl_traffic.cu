@@ -254,6 +254,114 @@ __global__ void traffic_owner_kernel(TrafficParams p) {
     }
 }
 
+// ---- finite private L2 per chiplet (tile-level LRU model) --------------------------------------------------
+// Sec. 4.1 scores "remote operand reads that miss in L2, and remote output writes" with an 8 MB, 16-way, 128-byte-line
+// L2 per chiplet.  Model: the CTAs of a chiplet run one after the other in row-major (traversal 0) or column-major
+// (traversal 1) order of the tile grid; a CTA touches the lines of its A rectangle in address order, then those of
+// its B rectangle; lines are numbered from the start of each operand's buffer and the operand is part of the tag,
+// LRU inside a set; a miss moves one whole line from the page's owner.
+// Sets are independent, so one warp simulates one set of one chiplet over the whole run: it enumerates, tile by
+// tile, only the lines that fall into its own set (32 blocks of lines per step) and lane 0 keeps the set's tags,
+// most recently used first, in its own local array.  Set index: line mod sets, or (hash = 1) skewed per block of `sets` lines, which stands in for the
+// address hashing of a real L2 (with the plain index, power-of-two row pitches pile up in a few sets).
+struct LruParams {
+    int64_t sets;
+    int32_t line, ways, traversal, hash;
+    uint64_t* out;                 // [2][2]: A local, A remote, B local, B remote
+};
+
+constexpr int kLruMaxWays = 32;
+
+struct LruSet {
+    uint64_t tag[kLruMaxWays];
+    int n;
+    // returns true on a miss
+    __device__ __forceinline__ bool touch(uint64_t t, int ways) {
+        int i = 0;
+        while (i < n && tag[i] != t) ++i;
+        const bool miss = i == n;
+        if (miss) { if (n < ways) ++n; i = n - 1; }
+        for (; i > 0; --i) tag[i] = tag[i - 1];
+        tag[0] = t;
+        return miss;
+    }
+};
+
+__global__ void __launch_bounds__(128) traffic_lru_kernel(TrafficParams p, LruParams l) {
+    // one WARP per (chiplet, set): the lanes scan 32 blocks of a piece at a time for the set's line, lane 0 owns the
+    // set's state and applies the hits in address order
+    const int lane = threadIdx.x & 31;
+    const int64_t wid = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (wid >= l.sets * p.P) return;                                        // whole warps leave together
+    const int32_t q = (int32_t)(wid / l.sets);
+    const int64_t s = wid - (int64_t)q * l.sets;
+    const int64_t L = l.line;
+    LruSet set;
+    set.n = 0;
+    uint64_t cnt[4] = {0, 0, 0, 0};
+    auto hit_line = [&](int X, int64_t line) {                              // lane 0 only
+        if (set.touch(((uint64_t)line << 1) | (uint64_t)X, l.ways)) {
+            const int64_t b = line * L;
+            const int64_t page = p.s_shift >= 0 ? (b >> p.s_shift) : (b / p.S);
+            cnt[X * 2 + (fixed_owner(p, X, page) == q ? 0 : 1)] += (uint64_t)L;
+        }
+    };
+    // The lines of rows [0, rows) of one contiguous piece that fall into this warp's set, in address order.
+    // Every block of `sets` consecutive lines holds exactly one line of each set (the index is the line's position
+    // in its block plus a skew that depends on the block only), so the piece is scanned block by block.
+    auto piece = [&](int X, int64_t base, int64_t rows, int64_t pitch, int64_t len) {
+        if (rows <= 0 || len <= 0) return;
+        const int64_t l0 = base / L, l1 = (base + (rows - 1) * pitch + len - 1) / L;
+        for (int64_t blk0 = l0 / l.sets; blk0 * l.sets <= l1; blk0 += 32) {
+            const int64_t blk = blk0 + lane;
+            const int64_t skew = l.hash ? (int64_t)((((uint64_t)blk * 0x9E3779B97F4A7C15ull) >> 32) % (uint64_t)l.sets) : 0;
+            const int64_t line = blk * l.sets + ((s - skew) % l.sets + l.sets) % l.sets;
+            bool in = line >= l0 && line <= l1;
+            if (in) {
+                // does the line [line*L, line*L + L) hold a byte of some row [base + r*pitch, + len) ?
+                const int64_t b0 = line * L, b1 = b0 + L;
+                int64_t r = b0 > base ? (b0 - base) / pitch : 0;             // the last row that starts at or before the line
+                if (r >= rows) r = rows - 1;
+                in = base + r * pitch < b1 && base + r * pitch + len > b0;
+                if (!in && r + 1 < rows) in = base + (r + 1) * pitch < b1;   // or the next row starts inside it
+            }
+            unsigned hits = __ballot_sync(0xffffffffu, in);
+            while (hits) {                                                   // ascending lanes = ascending addresses
+                const int src = __ffs(hits) - 1;
+                hits &= hits - 1;
+                const int64_t ln = __shfl_sync(0xffffffffu, line, src);
+                if (lane == 0) hit_line(X, ln);
+            }
+        }
+    };
+    const int64_t outer = l.traversal == 0 ? p.tiles_m : p.tiles_n, inner = l.traversal == 0 ? p.tiles_n : p.tiles_m;
+    for (int64_t o = 0; o < outer; ++o)
+        for (int64_t i = 0; i < inner; ++i) {
+            const int64_t tm = l.traversal == 0 ? o : i, tn = l.traversal == 0 ? i : o;
+            const TileInfo t = decode_tile(p, tm * p.tiles_n + tn);
+            if (t.q != q) continue;
+            for (int X = 0; X < 2; ++X) {
+                const MatView& v = p.v[X];
+                int64_t r0, r1, c0, c1;
+                tile_rect(p, t, X, r0, r1, c0, c1);
+                if (v.split == 2) {                                           // strips of columns: one piece per strip touched
+                    for (int64_t g = c0 / v.w; g * v.w < c1; ++g) {
+                        const int64_t ca = max(c0, g * v.w), cb = min(c1, (g + 1) * v.w);
+                        piece(X, (g * v.stride + r0 * v.w + (ca - g * v.w)) * v.e, r1 - r0, v.w * v.e, (cb - ca) * v.e);
+                    }
+                } else if (v.split == 1) {                                    // strips of rows
+                    for (int64_t g = r0 / v.h; g * v.h < r1; ++g) {
+                        const int64_t ra = max(r0, g * v.h), rb = min(r1, (g + 1) * v.h);
+                        piece(X, (g * v.stride + (ra - g * v.h) * v.cols + c0) * v.e, rb - ra, v.cols * v.e, (c1 - c0) * v.e);
+                    }
+                } else piece(X, (r0 * v.cols + c0) * v.e, r1 - r0, v.cols * v.e, (c1 - c0) * v.e);
+            }
+        }
+    if (lane == 0)
+        for (int k = 0; k < 4; ++k)
+            if (cnt[k]) atomicAdd(reinterpret_cast<unsigned long long*>(&l.out[k]), (unsigned long long)cnt[k]);
+}
+
 static ccl_status fill_params(const ccl_traffic_desc* d, TrafficParams* p) {
     if (!d) return fail(CCL_ERR_INVALID_ARG, "ccl_traffic: NULL descriptor");
     std::memset(p, 0, sizeof(*p));
@@ -397,3 +505,51 @@ extern "C" ccl_status ccl_traffic_l2(const ccl_traffic_desc* d, const int32_t* c
     CCL_CUDA_TRY(cudaGetLastError());
     return CCL_OK;
 }
+
+extern "C" ccl_status ccl_traffic_lru(const ccl_traffic_desc* d, const ccl_l2_model* m, uint64_t* totals_dev, void* cuda_stream) {
+    TrafficParams p;
+    ccl_status s = fill_params(d, &p);
+    if (s) return s;
+    if (!m || !totals_dev) return fail(CCL_ERR_INVALID_ARG, "ccl_traffic_lru: NULL model or output");
+    if (m->line_bytes <= 0 || m->ways <= 0 || m->capacity_bytes <= 0 || (m->traversal != 0 && m->traversal != 1))
+        return fail(CCL_ERR_INVALID_ARG, "ccl_traffic_lru: line_bytes, ways, capacity_bytes must be positive and traversal 0 or 1");
+    if (m->hash != 0 && m->hash != 1) return fail(CCL_ERR_INVALID_ARG, "ccl_traffic_lru: hash must be 0 or 1");
+    if (m->ways > kLruMaxWays) return fail(CCL_ERR_UNSUPPORTED, "ccl_traffic_lru: at most %d ways", kLruMaxWays);
+    if (m->capacity_bytes % ((int64_t)m->line_bytes * m->ways)) return fail(CCL_ERR_INVALID_ARG, "ccl_traffic_lru: capacity is not a whole number of sets");
+    if (d->page_bytes % m->line_bytes) return fail(CCL_ERR_INVALID_ARG, "ccl_traffic_lru: page_bytes is not a multiple of line_bytes");
+    if (d->assign == CCL_ASSIGN_EXPLICIT) return fail(CCL_ERR_UNSUPPORTED, "ccl_traffic_lru: explicit CTA assignment is not supported");
+    for (int X = 0; X < 3; ++X) {
+        if (p.place[X] == CCL_PLACE_BEST) return fail(CCL_ERR_UNSUPPORTED, "ccl_traffic_lru: CCL_PLACE_BEST is not supported here (use a fixed placement)");
+        if (X < 2 && p.v[X].ichunk) return fail(CCL_ERR_UNSUPPORTED, "ccl_traffic_lru: page-interleaved operands are not supported");
+    }
+    LruParams l;
+    std::memset(&l, 0, sizeof(l));
+    l.line = m->line_bytes; l.ways = m->ways; l.traversal = m->traversal; l.hash = m->hash;
+    l.sets = m->capacity_bytes / ((int64_t)m->line_bytes * m->ways);
+    if (l.sets * d->P >= (INT64_C(1) << 31) * 128) return fail(CCL_ERR_UNSUPPORTED, "ccl_traffic_lru: too many sets");
+    l.out = totals_dev;
+    p.totals_l2 = totals_dev;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    ZeroSeg z;
+    std::memset(&z, 0, sizeof(z));
+    z.p[0] = totals_dev; z.n[0] = 6;
+    traffic_prep_kernel<<<1, 32, 0, st>>>(z);
+    count_launch();
+    CCL_CUDA_TRY(cudaGetLastError());
+    // C is written once, past the cache: its row is the one of the walk behind an ideal L2 (= the uncached one)
+    const int64_t nblocks = p.tiles_m + p.tiles_n + (p.ntiles + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    if (nblocks >= (INT64_C(1) << 31)) return fail(CCL_ERR_UNSUPPORTED, "ccl_traffic_lru: too many tiles");
+    traffic_walk_kernel<false, true><<<(unsigned)nblocks, kWalkThreads, 0, st>>>(p);
+    count_launch();
+    CCL_CUDA_TRY(cudaGetLastError());
+    z.n[0] = 4;                                  // A and B come from the cache model
+    traffic_prep_kernel<<<1, 32, 0, st>>>(z);
+    count_launch();
+    CCL_CUDA_TRY(cudaGetLastError());
+    const int64_t threads = l.sets * d->P * 32;          // a warp per (chiplet, set)
+    traffic_lru_kernel<<<(unsigned)((threads + 127) / 128), 128, 0, st>>>(p, l);
+    count_launch();
+    CCL_CUDA_TRY(cudaGetLastError());
+    return CCL_OK;
+}
+

@@ -124,7 +124,52 @@ def traffic_remote(g, layout_bc, place_bc, S, assign, align=0):
     return out
 
 
-def run_gemm(g, pk, reps):
+def traffic_desc(g, layout_bc, place_bc, S, assign, align=0):
+    """Library descriptor of one placement policy; None if the partition does not apply (M % P != 0)."""
+    M, N, K, P = g["M"], g["N"], g["K"], g["P"]
+    if assign == ccl.ASSIGN_M_STRIPS and (M % P or M < P):
+        return None
+    at, bt = g["a_trans"], g["b_trans"]
+    td = ccl.TrafficDesc()
+    td.M, td.N, td.K, td.BM, td.BN = M, N, K, 128, 128
+    a_shape = (K, M) if at else (M, K)
+    b_shape = (N, K) if bt else (K, N)
+    if assign == ccl.ASSIGN_N_STRIPS:
+        parts = (ccl.PART_NONE, ccl.PART_ROWS if bt else ccl.PART_COLS, ccl.PART_COLS)
+    else:
+        parts = (ccl.PART_COLS if at else ccl.PART_ROWS, ccl.PART_NONE, ccl.PART_ROWS)
+    shapes = (a_shape, b_shape, (M, N))
+    ms = []
+    for X in range(3):
+        is_ccl = layout_bc != ccl.ROWMAJOR and parts[X] != ccl.PART_NONE
+        ms.append(ccl.Mat(shapes[X][0], shapes[X][1], 2, P, parts[X] if is_ccl else ccl.PART_NONE,
+                          layout_bc if is_ccl else ccl.ROWMAJOR, align if is_ccl else 0))
+    td.A, td.B, td.C = ms
+    td.a_trans, td.b_trans, td.P, td.page_bytes = at, bt, P, S
+    for X in range(3):
+        td.place[X] = place_bc if parts[X] != ccl.PART_NONE else ccl.PLACE_RR
+    td.assign, td.strip_tiling = assign, 1
+    return td
+
+
+def traffic_lru_best(g, layout_bc, place_bc, S, model_kw):
+    """Remote bytes (A, B, C) behind a finite LRU L2 per chiplet: the best of both output partitions and both CTA
+    traversals, as the paper reports (Sec. 4.1: "we sweep CTA traversal and output-partition choices")."""
+    best = None
+    for assign in (ccl.ASSIGN_N_STRIPS, ccl.ASSIGN_M_STRIPS):
+        td = traffic_desc(g, layout_bc, place_bc, S, assign, align=S)
+        if td is None:
+            continue
+        for traversal in (0, 1):
+            t = torch.empty((3, 2), dtype=torch.int64, device="cuda")
+            ccl.ccl_traffic_lru(td, ccl.L2Model(traversal=traversal, **model_kw), t)
+            r = [int(x) for x in t.cpu()[:, 1]]
+            if best is None or sum(r) < sum(best["remote"]):
+                best = dict(remote=r, partition="N" if assign == ccl.ASSIGN_N_STRIPS else "M", traversal=traversal)
+    return best
+
+
+def run_gemm(g, pk, reps, lru=False):
     M, N, K, at, bt, P, S = g["M"], g["N"], g["K"], g["a_trans"], g["b_trans"], g["P"], g["S"]
     dev = "cuda"
     A = torch.empty((K, M) if at else (M, K), dtype=torch.bfloat16, device=dev).normal_(0, g["a_std"])
@@ -194,6 +239,14 @@ def run_gemm(g, pk, reps):
         if "remote_ideal_l2" in r:
             r["ratio_vs_rr4k_ideal_l2"] = (sum(r["remote_ideal_l2"]) / base_l2) if base_l2 else None
     res["traffic"] = pol
+    if lru:                                       # the paper's metric: behind an 8 MB, 16-way, 128-byte-line L2 per chiplet
+        kw = dict(capacity_bytes=8 << 20, line_bytes=128, ways=16, hash=1)
+        fin = {tag: traffic_lru_best(g, lay, place, Sp, kw) for tag, lay, place, Sp in
+               (("row_rr4k", ccl.ROWMAJOR, ccl.PLACE_RR, 4096), ("row_block", ccl.ROWMAJOR, ccl.PLACE_BLOCK, S), ("ccl_block", ccl.CCL, ccl.PLACE_BLOCK, S))}
+        b = sum(fin["row_rr4k"]["remote"])
+        for r in fin.values():
+            r["ratio_vs_rr4k"] = sum(r["remote"]) / b if b else None
+        res["traffic_finite_l2"] = fin
     return res
 
 
@@ -202,6 +255,7 @@ def main():
     ap.add_argument("--config", default="all")
     ap.add_argument("--out", default=os.path.join(ROOT, "report_out"))
     ap.add_argument("--quick", action="store_true", help="fewer repetitions and P = 4 only in the sweep")
+    ap.add_argument("--lru", action="store_true", help="also score the placements behind a finite LRU L2 per chiplet (slow at Llama sizes)")
     ap.add_argument("--only", default=None, help="run only the GEMMs whose name contains this text (e.g. for a profiler capture)")
     args = ap.parse_args()
     assert torch.cuda.is_available(), "report needs a CUDA device"
@@ -213,7 +267,7 @@ def main():
             if args.only and args.only not in g["name"]:
                 continue
             big = g["M"] * g["N"] * g["K"] > 1e11
-            r = run_gemm(g, pk, 3 if (big or args.quick) else 100)
+            r = run_gemm(g, pk, 3 if (big or args.quick) else 100, lru=args.lru)
             rows.append(r)
             c, rw = r.get("ccl_grouped", {}), r.get("row_plain", {})
             t = r["traffic"]
@@ -225,12 +279,20 @@ def main():
                   f"block {t['row_block']['ratio_vs_rr4k']:.3f} best {t['row_best']['ratio_vs_rr4k']:.3f} "
                   f"CCL {t['ccl_block']['ratio_vs_rr4k']:.3f} ({t['ccl_block']['partition']}) ccl+rr {t['ccl_rr']['ratio_vs_rr4k']:.3f} "
                   f"interleaved-CCL+rr {t['ileave_rr']['ratio_vs_rr4k']:.3f} | behind an ideal L2: block {t['row_block']['ratio_vs_rr4k_ideal_l2']:.3f} "
-                  f"CCL {t['ccl_block']['ratio_vs_rr4k_ideal_l2']:.3f} interleaved-CCL+rr {t['ileave_rr']['ratio_vs_rr4k_ideal_l2']:.3f}", flush=True)
+                  f"CCL {t['ccl_block']['ratio_vs_rr4k_ideal_l2']:.3f} interleaved-CCL+rr {t['ileave_rr']['ratio_vs_rr4k_ideal_l2']:.3f}"
+                  + (f" | behind an 8 MB LRU L2 (best partition / traversal): block {r['traffic_finite_l2']['row_block']['ratio_vs_rr4k']:.3f} "
+                     f"CCL {r['traffic_finite_l2']['ccl_block']['ratio_vs_rr4k']:.3f}" if args.lru else ""), flush=True)
         json.dump(dict(config=cfg, peaks=pk, gemms=rows), open(os.path.join(args.out, f"report_config{cfg}.json"), "w"), indent=1)
         nz = [r["traffic"]["ccl_block"]["ratio_vs_rr4k"] for r in rows if r["traffic"]["ccl_block"]["ratio_vs_rr4k"]]
         if nz:
             print(f"cfg{cfg}: geometric mean of CCL/rr4k remote-traffic ratios over {len(nz)} GEMMs with non-zero ratio "
                   f"({len(rows) - len(nz)} zero): {math.exp(sum(math.log(x) for x in nz) / len(nz)):.3f}", flush=True)
+        if args.lru and rows:
+            for tag in ("row_block", "ccl_block"):
+                rs = [r["traffic_finite_l2"][tag]["ratio_vs_rr4k"] for r in rows if r["traffic_finite_l2"][tag]["ratio_vs_rr4k"]]
+                if rs:
+                    print(f"cfg{cfg}: behind an 8 MB LRU L2, geometric mean of {tag}/rr4k over {len(rs)} GEMMs: "
+                          f"{math.exp(sum(math.log(x) for x in rs) / len(rs)):.3f}", flush=True)
 
 
 if __name__ == "__main__":

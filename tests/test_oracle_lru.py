@@ -46,14 +46,17 @@ def test_limits(M, N, K, P, S, lay, place, assign, traversal):
     np.testing.assert_array_equal(unbounded, ideal)                 # each chiplet fetches a line once
     # more ways over the same sets never miss more (LRU stack inclusion), and the C row never changes
     prev = None
-    for ways in (1, 2, 4, 16):
-        t = orc.traffic_lru(do, orc.L2Model(8 * ways * 128, 128, ways, traversal))
-        np.testing.assert_array_equal(t[2], plain[2])
-        total = int(t[0].sum() + t[1].sum())
-        assert int(ideal[0].sum() + ideal[1].sum()) <= total <= int(plain[0].sum() + plain[1].sum())
-        if prev is not None:
-            assert total <= prev
-        prev = total
+    for hashed in (0, 1):                                           # whatever the set index, as long as it is a function of the line
+        prev = None
+        for ways in (1, 2, 4, 16):
+            t = orc.traffic_lru(do, orc.L2Model(8 * ways * 128, 128, ways, traversal, hashed))
+            np.testing.assert_array_equal(t[2], plain[2])
+            total = int(t[0].sum() + t[1].sum())
+            assert int(ideal[0].sum() + ideal[1].sum()) <= total <= int(plain[0].sum() + plain[1].sum())
+            if prev is not None:
+                assert total <= prev
+            prev = total
+        np.testing.assert_array_equal(orc.traffic_lru(do, orc.L2Model(128, 128, 1, traversal, hashed)), plain)
 
 
 def test_traversal_matters_and_rejections():
@@ -68,6 +71,12 @@ def test_traversal_matters_and_rejections():
         orc.traffic_lru(do, orc.L2Model(1000, 128, 16, 0))         # capacity not a whole number of sets
     with pytest.raises(ValueError):
         orc.traffic_lru(do, orc.L2Model(8 << 20, 128, 16, 2))      # unknown traversal
+    # a skewed index spreads a power-of-two stride over the sets: the column of lines 0, 64, 128, ... (pitch = sets)
+    # all share set 0 under the plain index and thrash a 2-way set; skewed, they land in different sets
+    ds, _ = traffic_pair(256, 128, 64, 1, 4096, BM=256, BN=128, b_trans=1)    # A [256 x 64]: one line per row, pitch one line
+    one_set_plain = orc.traffic_lru(ds, orc.L2Model(2 * 128, 128, 2, 0, 0))     # 1 set: the index cannot matter
+    one_set_hash = orc.traffic_lru(ds, orc.L2Model(2 * 128, 128, 2, 0, 1))
+    np.testing.assert_array_equal(one_set_plain, one_set_hash)
     db, _ = traffic_pair(512, 512, 256, 2, 4096, place=(2, 2, 2))
     with pytest.raises(ValueError):
         orc.traffic_lru(db, orc.L2Model(8 << 20, 128, 16, 0))      # BEST placement is not modelled
