@@ -250,17 +250,86 @@ def run_gemm(g, pk, reps, lru=False):
     return res
 
 
+def extras(out_dir, quick):
+    """The entry points around the plain GEMM, timed on the shapes they are meant for: the batch of expert GEMMs in one
+    launch, the gated activation fused into the gate/up GEMM, and alpha/beta accumulation."""
+    dev, rows = "cuda", []
+
+    def desc(M, N, K, P, bt=0, c_cols=None):
+        d = ccl.GemmDesc()
+        d.M, d.N, d.K = M, N, K
+        d.A = ccl.Mat(M, K, 2)
+        d.B = ccl.Mat(N, K, 2, P, ccl.PART_ROWS, ccl.CCL, 4096) if bt else ccl.Mat(K, N, 2, P, ccl.PART_COLS, ccl.CCL, 4096)
+        d.C = ccl.Mat(M, c_cols or N, 2, P, ccl.PART_COLS, ccl.CCL, 4096)
+        d.a_trans, d.b_trans, d.out_part, d.P, d.grouped_raster = 0, bt, ccl.PART_COLS, P, 1
+        return d
+
+    def buf(m, n=1):
+        return torch.empty(n * ccl.ccl_buffer_bytes(m) // 2, dtype=torch.bfloat16, device=dev).normal_(0, 0.05)
+
+    # 1. the experts of an MoE layer: one launch against one launch per expert and against torch.bmm
+    for E, M, N, K, bt in ((128, 256, 768, 2048, 1), (128, 256, 2048, 768, 0)) if not quick else ((32, 256, 768, 2048, 1),):
+        d = desc(M, N, K, 4, bt)
+        A, B, Cb = buf(d.A, E), buf(d.B, E), buf(d.C, E)
+        sa, sb, sc = (ccl.ccl_buffer_bytes(m) for m in (d.A, d.B, d.C))
+        need = ccl.ccl_gemm_batched_workspace(d, E)
+        ws = torch.empty(max(need, 16) // 4, dtype=torch.float32, device=dev)
+        t_b = timed(lambda: ccl.ccl_gemm_batched(d, E, A, sa, B, sb, Cb, sc, ws if need else None), 20)
+        need1 = ccl.ccl_gemm_workspace(d)
+        ws1 = torch.empty(max(need1, 16) // 4, dtype=torch.float32, device=dev)
+        views = [(A[e * sa // 2:(e + 1) * sa // 2], B[e * sb // 2:(e + 1) * sb // 2], Cb[e * sc // 2:(e + 1) * sc // 2]) for e in range(E)]
+
+        def one_by_one():
+            for a, b, c in views:
+                ccl.ccl_gemm(d, a, b, c, ws1 if need1 else None)
+        t_l = timed(one_by_one, 3)
+        Al = A.view(E, M, K)
+        Bl = B.view(E, N, K).transpose(1, 2) if bt else B.view(E, K, N)        # same bytes read as plain matrices: timing only
+        t_t = timed(lambda: torch.bmm(Al, Bl), 20)
+        fl = 2.0 * E * M * N * K
+        rows.append(dict(what="batched", E=E, M=M, N=N, K=K, batched_ms=t_b, launches_ms=t_l, torch_bmm_ms=t_t,
+                         batched_tflops=fl / t_b / 1e9, torch_bmm_tflops=fl / t_t / 1e9))
+        print(f"extras batched {E} x {M}x{N}x{K}: one launch {t_b * 1e3:8.1f} us ({fl / t_b / 1e9:6.0f} TFLOP/s) | {E} launches {t_l * 1e3:8.1f} us | "
+              f"torch.bmm {t_t * 1e3:8.1f} us", flush=True)
+    # 2. gate/up GEMM with the gated activation in the epilogue against GEMM + elementwise kernel
+    for M, N, K in ((8192, 57344, 8192), (16384, 1536, 2048)) if not quick else ((1024, 57344, 8192),):
+        d0, d1 = desc(M, N, K, 4), desc(M, N, K, 4, c_cols=N // 2)
+        A, B, C0, C1 = buf(d0.A), buf(d0.B), buf(d0.C), buf(d1.C)
+        reps = 5 if M * N * K > 1e11 else 50
+        t_g = timed(lambda: ccl.ccl_gemm(d0, A, B, C0), reps)
+        H = C0.view(M, N)
+        out = torch.empty(M, N // 2, dtype=torch.bfloat16, device=dev)
+        t_a = timed(lambda: torch.mul(torch.nn.functional.silu(H[:, :N // 2]), H[:, N // 2:], out=out), reps)
+        t_f = timed(lambda: ccl.ccl_gemm_swiglu(d1, A, B, C1), reps)
+        rows.append(dict(what="swiglu", M=M, N=N, K=K, gemm_ms=t_g, elementwise_ms=t_a, fused_ms=t_f))
+        print(f"extras gate/up {M}x{N}x{K}: GEMM {t_g * 1e3:8.1f} us + silu*mul kernel {t_a * 1e3:8.1f} us = {(t_g + t_a) * 1e3:8.1f} us | "
+              f"fused {t_f * 1e3:8.1f} us ({2.0 * M * N * K / t_f / 1e9:6.0f} TFLOP/s)", flush=True)
+    # 3. alpha / beta: what reading C in the epilogue costs
+    for M, N, K in ((8192, 8192, 8192),) if not quick else ((2048, 8192, 2048),):
+        d = desc(M, N, K, 4)
+        A, B, Cc = buf(d.A), buf(d.B), buf(d.C)
+        t_p = timed(lambda: ccl.ccl_gemm(d, A, B, Cc), 10)
+        t_x = timed(lambda: ccl.ccl_gemm_axpby(d, 1.0, 1.0, A, B, Cc), 10)
+        rows.append(dict(what="axpby", M=M, N=N, K=K, gemm_ms=t_p, axpby_ms=t_x))
+        print(f"extras accumulate {M}x{N}x{K}: C = A*B {t_p * 1e3:8.1f} us | C += A*B {t_x * 1e3:8.1f} us", flush=True)
+    json.dump(rows, open(os.path.join(out_dir, "report_extras.json"), "w"), indent=1)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--config", default="all")
     ap.add_argument("--out", default=os.path.join(ROOT, "report_out"))
     ap.add_argument("--quick", action="store_true", help="fewer repetitions and P = 4 only in the sweep")
     ap.add_argument("--lru", action="store_true", help="also score the placements behind a finite LRU L2 per chiplet (slow at Llama sizes)")
+    ap.add_argument("--extras", action="store_true", help="time the batched, gated-activation and alpha/beta entry points (then exit)")
     ap.add_argument("--only", default=None, help="run only the GEMMs whose name contains this text (e.g. for a profiler capture)")
     args = ap.parse_args()
     assert torch.cuda.is_available(), "report needs a CUDA device"
     pk = peaks()
     os.makedirs(args.out, exist_ok=True)
+    if args.extras:
+        extras(args.out, args.quick)
+        return
     for cfg, gemms in configs(args.config, args.quick).items():
         rows = []
         for g in gemms:
