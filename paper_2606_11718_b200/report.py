@@ -124,7 +124,7 @@ def traffic_remote(g, layout_bc, place_bc, S, assign, align=0):
     return out
 
 
-def traffic_desc(g, layout_bc, place_bc, S, assign, align=0):
+def traffic_desc(g, layout_bc, place_bc, S, assign, align=0, e=2):
     """Library descriptor of one placement policy; None if the partition does not apply (M % P != 0)."""
     M, N, K, P = g["M"], g["N"], g["K"], g["P"]
     if assign == ccl.ASSIGN_M_STRIPS and (M % P or M < P):
@@ -142,7 +142,7 @@ def traffic_desc(g, layout_bc, place_bc, S, assign, align=0):
     ms = []
     for X in range(3):
         is_ccl = layout_bc != ccl.ROWMAJOR and parts[X] != ccl.PART_NONE
-        ms.append(ccl.Mat(shapes[X][0], shapes[X][1], 2, P, parts[X] if is_ccl else ccl.PART_NONE,
+        ms.append(ccl.Mat(shapes[X][0], shapes[X][1], e, P, parts[X] if is_ccl else ccl.PART_NONE,
                           layout_bc if is_ccl else ccl.ROWMAJOR, align if is_ccl else 0))
     td.A, td.B, td.C = ms
     td.a_trans, td.b_trans, td.P, td.page_bytes = at, bt, P, S
@@ -152,12 +152,12 @@ def traffic_desc(g, layout_bc, place_bc, S, assign, align=0):
     return td
 
 
-def traffic_lru_best(g, layout_bc, place_bc, S, model_kw):
+def traffic_lru_best(g, layout_bc, place_bc, S, model_kw, e=2):
     """Remote bytes (A, B, C) behind a finite LRU L2 per chiplet: the best of both output partitions and both CTA
     traversals, as the paper reports (Sec. 4.1: "we sweep CTA traversal and output-partition choices")."""
     best = None
     for assign in (ccl.ASSIGN_N_STRIPS, ccl.ASSIGN_M_STRIPS):
-        td = traffic_desc(g, layout_bc, place_bc, S, assign, align=S)
+        td = traffic_desc(g, layout_bc, place_bc, S, assign, align=S, e=e)
         if td is None:
             continue
         for traversal in (0, 1):
@@ -250,6 +250,31 @@ def run_gemm(g, pk, reps, lru=False):
     return res
 
 
+def capacity_and_dtype_sweep(out_dir, quick):
+    """The two sweeps of the paper's last figure (Sec. 4.2: remote traffic against the per-chiplet L2 capacity with bf16
+    fixed, and against the data type with 8 MB fixed; average absolute traffic over the GEMMs at 4K tokens), under this
+    library's finite-L2 model: P = 4, 4 KB pages, best output partition and traversal per GEMM."""
+    T = 4096
+    gemms = [dict(g, P=4) for g in synth.qwen_ffn_gemms(T=T) + synth.llama_fwd_gemms(T=T) + synth.llama_bwd_gemms(T=T)]
+    if quick:
+        gemms = gemms[:6]
+    policies = (("rr4k", ccl.ROWMAJOR, ccl.PLACE_RR), ("coarse", ccl.ROWMAJOR, ccl.PLACE_BLOCK), ("ccl", ccl.CCL, ccl.PLACE_BLOCK))
+    settings = [("capacity", mb, 2) for mb in ((4, 8, 16) if quick else (2, 4, 8, 16, 32))] + [("dtype", 8, e) for e in (1, 4)]
+    table = []
+    for kind, mb, e in settings:
+        kw = dict(capacity_bytes=mb << 20, line_bytes=128, ways=16, hash=1)
+        avg = {}
+        for tag, lay, place in policies:
+            tot = 0
+            for g in gemms:
+                tot += sum(traffic_lru_best(g, lay, place, 4096, kw, e=e)["remote"])
+            avg[tag] = tot / len(gemms)
+        table.append(dict(sweep=kind, l2_mb=mb, elem_bytes=e, avg_remote_bytes=avg))
+        print(f"sweep {kind:8s} L2 {mb:2d} MB, {e}-byte elements: average remote bytes over {len(gemms)} GEMMs at {T} tokens: "
+              + "  ".join(f"{k} {v / 1e9:8.3f} GB" for k, v in avg.items()) + f"  | CCL / coarse = {avg['ccl'] / avg['coarse']:.3f}", flush=True)
+    json.dump(table, open(os.path.join(out_dir, "report_l2_sweep.json"), "w"), indent=1)
+
+
 def extras(out_dir, quick):
     """The entry points around the plain GEMM, timed on the shapes they are meant for: the batch of expert GEMMs in one
     launch, the gated activation fused into the gate/up GEMM, and alpha/beta accumulation."""
@@ -321,6 +346,7 @@ def main():
     ap.add_argument("--out", default=os.path.join(ROOT, "report_out"))
     ap.add_argument("--quick", action="store_true", help="fewer repetitions and P = 4 only in the sweep")
     ap.add_argument("--lru", action="store_true", help="also score the placements behind a finite LRU L2 per chiplet (slow at Llama sizes)")
+    ap.add_argument("--l2-sweep", action="store_true", help="remote traffic against L2 capacity and data type under the finite-L2 model (then exit)")
     ap.add_argument("--extras", action="store_true", help="time the batched, gated-activation and alpha/beta entry points (then exit)")
     ap.add_argument("--only", default=None, help="run only the GEMMs whose name contains this text (e.g. for a profiler capture)")
     args = ap.parse_args()
@@ -329,6 +355,9 @@ def main():
     os.makedirs(args.out, exist_ok=True)
     if args.extras:
         extras(args.out, args.quick)
+        return
+    if args.l2_sweep:
+        capacity_and_dtype_sweep(args.out, args.quick)
         return
     for cfg, gemms in configs(args.config, args.quick).items():
         rows = []
