@@ -153,10 +153,10 @@ def gemm_swiglu(A, B, M, N, K, P=1, a_trans=0, b_trans=0, threads=None):
 class L2Model(C.Structure):
     """orc_l2_model"""
     _fields_ = [("capacity_bytes", C.c_int64), ("line_bytes", C.c_int32), ("ways", C.c_int32), ("traversal", C.c_int32),
-                ("hash", C.c_int32)]
+                ("hash", C.c_int32), ("wave_ctas", C.c_int32), ("k_slice", C.c_int32)]
 
-    def __init__(self, capacity_bytes=8 << 20, line_bytes=128, ways=16, traversal=0, hash=0):
-        super().__init__(capacity_bytes, line_bytes, ways, traversal, hash)
+    def __init__(self, capacity_bytes=8 << 20, line_bytes=128, ways=16, traversal=0, hash=0, wave_ctas=1, k_slice=0):
+        super().__init__(capacity_bytes, line_bytes, ways, traversal, hash, wave_ctas, k_slice)
 
 
 def traffic_lru(d, l2):

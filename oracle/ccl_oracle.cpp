@@ -547,14 +547,18 @@ int orc_traffic_ideal_l2(const orc_traffic_desc* d, const int32_t* explicit_q, u
 //     operand in their tag; set index: hash = 0: line mod sets (the textbook index: power-of-two row pitches pile up
 //     in a few sets); hash = 1: (line + H(line div sets)) mod sets with H(b) = high 32 bits of b * 0x9E3779B97F4A7C15
 //     (a skew per block of `sets` consecutive lines, standing in for the address hashing of a real L2);
-//   * the CTAs of a chiplet (its tiles, as enumerate_tiles assigns them) run one after the other, in row-major
-//     order of the tile grid (traversal 0: n fastest) or column-major (traversal 1: m fastest);
-//   * a CTA touches every line of its A rectangle in address order, then every line of its B rectangle in address
-//     order (each line once per CTA); a hit costs nothing, a miss fetches the whole line from the page's owner:
-//     line_bytes local or remote bytes; page_bytes must be a multiple of line_bytes;
+//   * the CTAs of a chiplet (its tiles, as enumerate_tiles assigns them) are taken in row-major order of the tile
+//     grid (traversal 0: n fastest) or column-major (traversal 1: m fastest) and run in waves of wave_ctas
+//     consecutive CTAs; the CTAs of a wave advance through K in lockstep, k_slice elements at a time (0: all of K):
+//     for every k range, each CTA of the wave in turn touches every line of the A rows-by-k-range rectangle of its
+//     tile in address order, then every line of its B rectangle; wave_ctas = 1, k_slice = 0 is one CTA after the
+//     other, each reading all of A, then all of B;
+//   * a hit costs nothing, a miss fetches the whole line from the page's owner: line_bytes local or remote bytes;
+//     page_bytes must be a multiple of line_bytes;
 //   * C is written once, past the cache: the C row of the totals is the one of the uncached count.
 // Placement policies: RR and BLOCK.
-typedef struct { int64_t capacity_bytes; int32_t line_bytes; int32_t ways; int32_t traversal; int32_t hash; } orc_l2_model;
+typedef struct { int64_t capacity_bytes; int32_t line_bytes; int32_t ways; int32_t traversal; int32_t hash;
+                 int32_t wave_ctas; int32_t k_slice; } orc_l2_model;
 
 static int64_t lru_set_index(int64_t line, int64_t sets, int hash) {
     if (!hash) return line % sets;
@@ -567,6 +571,7 @@ int orc_traffic_lru(const orc_traffic_desc* d, const orc_l2_model* l2, uint64_t*
     if (!traffic_desc_ok(*d) || !l2) return -1;
     if (l2->line_bytes <= 0 || l2->ways <= 0 || l2->capacity_bytes <= 0 || (l2->traversal != 0 && l2->traversal != 1)) return -1;
     if (l2->hash != 0 && l2->hash != 1) return -1;
+    if (l2->wave_ctas < 1 || l2->k_slice < 0) return -1;
     if (l2->capacity_bytes % ((int64_t)l2->line_bytes * l2->ways) || d->page_bytes % l2->line_bytes) return -1;
     if (d->assign == ORC_ASSIGN_EXPLICIT) return -1;
     const int64_t L = l2->line_bytes, sets = l2->capacity_bytes / (L * l2->ways);
@@ -594,37 +599,46 @@ int orc_traffic_lru(const orc_traffic_desc* d, const orc_l2_model* l2, uint64_t*
         if (l2->traversal == 0) return x.m0 != y.m0 ? x.m0 < y.m0 : x.n0 < y.n0;
         return x.n0 != y.n0 ? x.n0 < y.n0 : x.m0 < y.m0;
     });
+    const int64_t W = l2->wave_ctas, ks = l2->k_slice > 0 ? l2->k_slice : d->K;
     for (int q = 0; q < d->P; ++q) {
         // cache[set] = tags from most to least recently used; tag = line * 2 + operand
         std::vector<std::vector<int64_t>> cache((size_t)sets);
-        for (size_t oi : order) {
-            const Tile& t = tiles[oi];
-            if (t.q != q) continue;
-            for (int X = 0; X < 2; ++X) {
-                const orc_mat& m = *ms[X];
-                const int64_t bytes_total = buffer_elems(m) * m.elem_bytes;
-                int64_t r0, r1, c0, c1; tile_rect(*d, t, X, r0, r1, c0, c1);
-                std::vector<int64_t> lines;
-                for (int64_t r = r0; r < r1; ++r)
-                    for (int64_t c = c0; c < c1; ++c) {
-                        const int64_t b = map_offset(m, r, c) * m.elem_bytes;
-                        lines.push_back(b / L);
-                        lines.push_back((b + m.elem_bytes - 1) / L);
+        std::vector<size_t> mine;                       // this chiplet's tiles in the order it runs them
+        for (size_t oi : order) if (tiles[oi].q == q) mine.push_back(oi);
+        // waves of W tiles run in lockstep: every tile of the wave reads its A slice and its B slice of the k range
+        // [k0, k0 + ks) before any of them moves on to the next range
+        for (size_t w0 = 0; w0 < mine.size(); w0 += (size_t)W)
+            for (int64_t k0 = 0; k0 < d->K; k0 += ks)
+                for (size_t j = w0; j < std::min(mine.size(), w0 + (size_t)W); ++j) {
+                    const Tile& t = tiles[mine[j]];
+                    const int64_t k1 = std::min(d->K, k0 + ks);
+                    for (int X = 0; X < 2; ++X) {
+                        const orc_mat& m = *ms[X];
+                        const int64_t bytes_total = buffer_elems(m) * m.elem_bytes;
+                        int64_t r0, r1, c0, c1; tile_rect(*d, t, X, r0, r1, c0, c1);
+                        const bool k_is_rows = X == 0 ? d->a_trans != 0 : d->b_trans == 0;
+                        if (k_is_rows) { r0 = k0; r1 = k1; } else { c0 = k0; c1 = k1; }
+                        std::vector<int64_t> lines;
+                        for (int64_t r = r0; r < r1; ++r)
+                            for (int64_t c = c0; c < c1; ++c) {
+                                const int64_t b = map_offset(m, r, c) * m.elem_bytes;
+                                lines.push_back(b / L);
+                                lines.push_back((b + m.elem_bytes - 1) / L);
+                            }
+                        std::sort(lines.begin(), lines.end());
+                        lines.erase(std::unique(lines.begin(), lines.end()), lines.end());
+                        for (int64_t line : lines) {
+                            std::vector<int64_t>& set = cache[(size_t)lru_set_index(line, sets, l2->hash)];
+                            const int64_t tag = line * 2 + X;
+                            auto it = std::find(set.begin(), set.end(), tag);
+                            if (it != set.end()) { set.erase(it); set.insert(set.begin(), tag); continue; }      // hit
+                            set.insert(set.begin(), tag);
+                            if ((int64_t)set.size() > l2->ways) set.pop_back();
+                            const int64_t page = line * L / d->page_bytes;
+                            totals[X * 2 + (fixed_owner(d->place[X], page, d->page_bytes, d->P, bytes_total) == q ? 0 : 1)] += (uint64_t)L;
+                        }
                     }
-                std::sort(lines.begin(), lines.end());
-                lines.erase(std::unique(lines.begin(), lines.end()), lines.end());
-                for (int64_t line : lines) {
-                    std::vector<int64_t>& set = cache[(size_t)lru_set_index(line, sets, l2->hash)];
-                    const int64_t tag = line * 2 + X;
-                    auto it = std::find(set.begin(), set.end(), tag);
-                    if (it != set.end()) { set.erase(it); set.insert(set.begin(), tag); continue; }      // hit
-                    set.insert(set.begin(), tag);
-                    if ((int64_t)set.size() > l2->ways) set.pop_back();
-                    const int64_t page = line * L / d->page_bytes;
-                    totals[X * 2 + (fixed_owner(d->place[X], page, d->page_bytes, d->P, bytes_total) == q ? 0 : 1)] += (uint64_t)L;
                 }
-            }
-        }
     }
     return 0;
 }

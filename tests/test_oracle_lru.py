@@ -23,6 +23,42 @@ def test_hand_run():
         assert int(t[2].sum()) == 2 * 2 * 2                         # C: every element written once
 
 
+def test_wave_hand_run():
+    do, _ = traffic_pair(2, 2, 64, 1, 4096, BM=1, BN=1)
+    for line in open(os.path.join(HERE, "golden", "lru_wave_hand_run.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        sets, ways, wave, ks, a_bytes, b_bytes = (int(x) for x in line.split())
+        t = orc.traffic_lru(do, orc.L2Model(sets * ways * 128, 128, ways, 0, 0, wave, ks))
+        assert (int(t[0].sum()), int(t[1].sum())) == (a_bytes, b_bytes), (sets, ways, wave, ks, t)
+
+
+def test_wave_shares_the_a_slice():
+    """Closed form: a fully associative cache of 300 lines, one chiplet, tiles 128 x 128, K = 256 (bf16).  One CTA
+    after the other, a tile's A rows (128 rows x 4 lines) and B columns (256 rows x 2 lines) are 512 lines each: no
+    line survives to the next tile, so every tile fetches its whole A and B rectangle.  In waves of one tile row
+    (4 CTAs) with k slices of 64, the 128 lines of an A slice come back after the 128 lines of one tile's B slice:
+    they hit, and A is fetched once in all; B slices are private to a tile and return only a whole wave later."""
+    M, N, K = 384, 512, 256
+    do, _ = traffic_pair(M, N, K, 1, 4096, BM=128, BN=128)
+    seq = orc.traffic_lru(do, orc.L2Model(300 * 128, 128, 300, 0))
+    assert int(seq[0].sum()) == (N // 128) * M * K * 2 and int(seq[1].sum()) == (M // 128) * K * N * 2
+    wav = orc.traffic_lru(do, orc.L2Model(300 * 128, 128, 300, 0, 0, 4, 64))
+    assert int(wav[0].sum()) == M * K * 2 and int(wav[1].sum()) == (M // 128) * K * N * 2
+    # a wave of two tile rows (8 CTAs): an A slice still returns after one B slice, while the B slice of a column
+    # returns in the second tile row only after three other B slices and two A slices (640 lines): same counts
+    w8 = orc.traffic_lru(do, orc.L2Model(300 * 128, 128, 300, 0, 0, 8, 64))
+    np.testing.assert_array_equal(w8, wav)
+    # ... and with room for all of that (4 B slices + 2 A slices = 768 lines) the second tile row of a wave finds
+    # its B slices: B is fetched once per wave (rows 0-1, row 2) instead of once per tile row
+    w8big = orc.traffic_lru(do, orc.L2Model(800 * 128, 128, 800, 0, 0, 8, 64))
+    assert int(w8big[0].sum()) == M * K * 2 and int(w8big[1].sum()) == 2 * K * N * 2
+    with pytest.raises(ValueError):
+        orc.traffic_lru(do, orc.L2Model(300 * 128, 128, 300, 0, 0, 0, 64))     # a wave holds at least one CTA
+    with pytest.raises(ValueError):
+        orc.traffic_lru(do, orc.L2Model(300 * 128, 128, 300, 0, 0, 4, -1))
+
+
 CASES = [
     # M, N, K, P, page, layouts, placement: every tile row segment is a whole number of 128-byte lines
     (256, 512, 128, 2, 4096, ("row", "row", "row"), (0, 0, 0)),
@@ -57,6 +93,10 @@ def test_limits(M, N, K, P, S, lay, place, assign, traversal):
                 assert total <= prev
             prev = total
         np.testing.assert_array_equal(orc.traffic_lru(do, orc.L2Model(128, 128, 1, traversal, hashed)), plain)
+    # both limits hold for waves in lockstep too (k slices of whole lines, so no line is shared by two slices)
+    for wave, ks in ((3, 64), (1, 64), (5, 0)):
+        np.testing.assert_array_equal(orc.traffic_lru(do, orc.L2Model(128, 128, 1, traversal, 0, wave, ks)), plain)
+        np.testing.assert_array_equal(orc.traffic_lru(do, orc.L2Model(128 * 2 * lines, 128, 2 * lines, traversal, 1, wave, ks)), ideal)
 
 
 def test_traversal_matters_and_rejections():
