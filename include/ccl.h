@@ -284,10 +284,12 @@ ccl_status ccl_traffic_l2(const ccl_traffic_desc* d, const int32_t* cta_chiplet_
  * The same count behind a FINITE private L2 per chiplet: the metric of Sec. 4.1 ("remote operand reads that miss in
  * L2, and remote output writes"; 8 MB, 128-byte lines, 16 ways per chiplet).  The paper's simulator is not public;
  * this is a tile-level model with everything it leaves open stated here:
- *   - a chiplet's CTAs (its tiles under `assign`) run one after the other, in row-major order of the tile grid
- *     (traversal = 0, n fastest) or column-major (traversal = 1, m fastest); the paper sweeps the traversal and
- *     reports the best;
- *   - a CTA touches every line of its A rectangle in address order, then every line of its B rectangle;
+ *   - a chiplet's CTAs (its tiles under `assign`) are taken in row-major order of the tile grid (traversal = 0,
+ *     n fastest) or column-major (traversal = 1, m fastest); the paper sweeps the traversal and reports the best;
+ *   - they run in waves of wave_ctas consecutive CTAs (the CTAs resident on the chiplet at one time) that advance
+ *     through K in lockstep, k_slice elements per step (0: all of K at once): in every step each CTA of the wave in
+ *     turn touches every line of the k range of its A rectangle in address order, then every line of the k range
+ *     of its B rectangle.  wave_ctas = 1, k_slice = 0: one CTA after the other, all of A, then all of B;
  *   - each chiplet's cache has capacity_bytes / (line_bytes * ways) sets, LRU in a set; lines are numbered from the
  *     start of each operand's buffer (assumed line-aligned) and the operand is part of the tag; set index:
  *     hash = 0: line mod sets (the textbook index; power-of-two row pitches then pile up in a few sets),
@@ -296,10 +298,10 @@ ccl_status ccl_traffic_l2(const ccl_traffic_desc* d, const int32_t* cta_chiplet_
  *   - a miss fetches one whole line from the owner of its page: line_bytes local or remote bytes;
  *   - C is written once, past the cache.
  * totals_dev: uint64[3][2] (A, B, C) x (local, remote) bytes.
- * Requirements: capacity a whole number of sets, ways <= 32, page_bytes a multiple of line_bytes (else
+ * Requirements: capacity a whole number of sets, ways <= 32, wave_ctas in [1, 256], page_bytes a multiple of line_bytes (else
  * CCL_ERR_INVALID_ARG / CCL_ERR_UNSUPPORTED); fixed placements only; CCL_ASSIGN_N_STRIPS or _M_STRIPS;
  * A and B row-major or CCL (page-interleaved -> CCL_ERR_UNSUPPORTED).
- * One thread simulates one cache set of one chiplet; cost grows with tiles x lines per tile / sets.
+ * One warp simulates one cache set of one chiplet; cost grows with tiles x K steps x lines per tile / sets.
  */
 typedef struct ccl_l2_model {
     int64_t capacity_bytes; /* per chiplet */
@@ -307,6 +309,8 @@ typedef struct ccl_l2_model {
     int32_t ways;
     int32_t traversal;      /* 0 row-major over the tile grid, 1 column-major */
     int32_t hash;           /* 0 set = line mod sets, 1 skewed index (see above) */
+    int32_t wave_ctas;      /* CTAs of a chiplet in flight together, 1..256 */
+    int32_t k_slice;        /* elements of K per lockstep step; 0 = all of K */
 } ccl_l2_model;
 ccl_status ccl_traffic_lru(const ccl_traffic_desc* d, const ccl_l2_model* m, uint64_t* totals_dev, void* cuda_stream);
 

@@ -256,21 +256,25 @@ __global__ void traffic_owner_kernel(TrafficParams p) {
 
 // ---- finite private L2 per chiplet (tile-level LRU model) --------------------------------------------------
 // Sec. 4.1 scores "remote operand reads that miss in L2, and remote output writes" with an 8 MB, 16-way, 128-byte-line
-// L2 per chiplet.  Model: the CTAs of a chiplet run one after the other in row-major (traversal 0) or column-major
-// (traversal 1) order of the tile grid; a CTA touches the lines of its A rectangle in address order, then those of
-// its B rectangle; lines are numbered from the start of each operand's buffer and the operand is part of the tag,
+// L2 per chiplet.  Model: the CTAs of a chiplet are taken in row-major (traversal 0) or column-major (traversal 1)
+// order of the tile grid and run in waves of `wave` consecutive CTAs that step through K together, `ks` elements at
+// a time; in each step every CTA of the wave in turn touches the lines of the k range of its A rectangle in address
+// order, then those of its B rectangle (wave = 1, ks = K: one CTA after the other); lines are numbered from the start of each operand's buffer and the operand is part of the tag,
 // LRU inside a set; a miss moves one whole line from the page's owner.
 // Sets are independent, so one warp simulates one set of one chiplet over the whole run: it enumerates, tile by
 // tile, only the lines that fall into its own set (32 blocks of lines per step) and lane 0 keeps the set's tags,
 // most recently used first, in its own local array.  Set index: line mod sets, or (hash = 1) skewed per block of `sets` lines, which stands in for the
 // address hashing of a real L2 (with the plain index, power-of-two row pitches pile up in a few sets).
 struct LruParams {
-    int64_t sets;
-    int32_t line, ways, traversal, hash;
+    int64_t sets, ks;              // ks: elements of K a wave consumes per step (K: everything at once)
+    int32_t line, ways, traversal, hash, wave;
+    int32_t line_shift, sets_shift;   // log2 when a power of two, else -1
     uint64_t* out;                 // [2][2]: A local, A remote, B local, B remote
 };
 
 constexpr int kLruMaxWays = 32;
+constexpr int kLruMaxWave = 256;
+constexpr int kLruWarps = 4;       // warps (sets) per block
 
 struct LruSet {
     uint64_t tag[kLruMaxWays];
@@ -287,7 +291,7 @@ struct LruSet {
     }
 };
 
-__global__ void __launch_bounds__(128) traffic_lru_kernel(TrafficParams p, LruParams l) {
+__global__ void __launch_bounds__(32 * kLruWarps) traffic_lru_kernel(TrafficParams p, LruParams l) {
     // one WARP per (chiplet, set): the lanes scan 32 blocks of a piece at a time for the set's line, lane 0 owns the
     // set's state and applies the hits in address order
     const int lane = threadIdx.x & 31;
@@ -311,11 +315,15 @@ __global__ void __launch_bounds__(128) traffic_lru_kernel(TrafficParams p, LruPa
     // in its block plus a skew that depends on the block only), so the piece is scanned block by block.
     auto piece = [&](int X, int64_t base, int64_t rows, int64_t pitch, int64_t len) {
         if (rows <= 0 || len <= 0) return;
-        const int64_t l0 = base / L, l1 = (base + (rows - 1) * pitch + len - 1) / L;
-        for (int64_t blk0 = l0 / l.sets; blk0 * l.sets <= l1; blk0 += 32) {
+        const int64_t last = base + (rows - 1) * pitch + len - 1;
+        const int64_t l0 = l.line_shift >= 0 ? base >> l.line_shift : base / L, l1 = l.line_shift >= 0 ? last >> l.line_shift : last / L;
+        for (int64_t blk0 = l.sets_shift >= 0 ? l0 >> l.sets_shift : l0 / l.sets; blk0 * l.sets <= l1; blk0 += 32) {
             const int64_t blk = blk0 + lane;
-            const int64_t skew = l.hash ? (int64_t)((((uint64_t)blk * 0x9E3779B97F4A7C15ull) >> 32) % (uint64_t)l.sets) : 0;
-            const int64_t line = blk * l.sets + ((s - skew) % l.sets + l.sets) % l.sets;
+            const uint64_t h = l.hash ? ((uint64_t)blk * 0x9E3779B97F4A7C15ull) >> 32 : 0;
+            int64_t pos;                                                     // position of the set's line in its block
+            if (l.sets_shift >= 0) pos = (s - (int64_t)h) & (l.sets - 1);
+            else { const int64_t skew = (int64_t)(h % (uint64_t)l.sets); pos = s - skew + (s < skew ? l.sets : 0); }
+            const int64_t line = blk * l.sets + pos;
             bool in = line >= l0 && line <= l1;
             if (in) {
                 // does the line [line*L, line*L + L) hold a byte of some row [base + r*pitch, + len) ?
@@ -334,29 +342,52 @@ __global__ void __launch_bounds__(128) traffic_lru_kernel(TrafficParams p, LruPa
             }
         }
     };
-    const int64_t outer = l.traversal == 0 ? p.tiles_m : p.tiles_n, inner = l.traversal == 0 ? p.tiles_n : p.tiles_m;
-    for (int64_t o = 0; o < outer; ++o)
-        for (int64_t i = 0; i < inner; ++i) {
+    // the k range [k0, k1) of tile t's rectangle of operand X
+    auto slice = [&](const TileInfo& t, int X, int64_t k0, int64_t k1) {
+        const MatView& v = p.v[X];
+        int64_t r0, r1, c0, c1;
+        tile_rect(p, t, X, r0, r1, c0, c1);
+        const bool k_is_rows = X == 0 ? p.a_trans : !p.b_trans;
+        if (k_is_rows) { r0 = k0; r1 = k1; } else { c0 = k0; c1 = k1; }
+        if (v.split == 2) {                                           // strips of columns: one piece per strip touched
+            for (int64_t g = c0 / v.w; g * v.w < c1; ++g) {
+                const int64_t ca = max(c0, g * v.w), cb = min(c1, (g + 1) * v.w);
+                piece(X, (g * v.stride + r0 * v.w + (ca - g * v.w)) * v.e, r1 - r0, v.w * v.e, (cb - ca) * v.e);
+            }
+        } else if (v.split == 1) {                                    // strips of rows
+            for (int64_t g = r0 / v.h; g * v.h < r1; ++g) {
+                const int64_t ra = max(r0, g * v.h), rb = min(r1, (g + 1) * v.h);
+                piece(X, (g * v.stride + (ra - g * v.h) * v.cols + c0) * v.e, rb - ra, v.cols * v.e, (c1 - c0) * v.e);
+            }
+        } else piece(X, (r0 * v.cols + c0) * v.e, r1 - r0, v.cols * v.e, (c1 - c0) * v.e);
+    };
+    // The chiplet's tiles in traversal order, a wave at a time: the warp gathers the next `wave` of its tiles into
+    // shared memory, then steps the whole wave through K.
+    __shared__ int64_t wave_tiles[kLruWarps][kLruMaxWave][4];
+    int64_t (*wt)[4] = wave_tiles[threadIdx.x >> 5];
+    const int64_t inner = l.traversal == 0 ? p.tiles_n : p.tiles_m;
+    int64_t o = 0, i = 0;
+    for (int64_t pos = 0; pos < p.ntiles;) {
+        int nw = 0;
+        for (; pos < p.ntiles && nw < l.wave; ++pos) {
             const int64_t tm = l.traversal == 0 ? o : i, tn = l.traversal == 0 ? i : o;
             const TileInfo t = decode_tile(p, tm * p.tiles_n + tn);
+            if (++i == inner) { i = 0; ++o; }
             if (t.q != q) continue;
-            for (int X = 0; X < 2; ++X) {
-                const MatView& v = p.v[X];
-                int64_t r0, r1, c0, c1;
-                tile_rect(p, t, X, r0, r1, c0, c1);
-                if (v.split == 2) {                                           // strips of columns: one piece per strip touched
-                    for (int64_t g = c0 / v.w; g * v.w < c1; ++g) {
-                        const int64_t ca = max(c0, g * v.w), cb = min(c1, (g + 1) * v.w);
-                        piece(X, (g * v.stride + r0 * v.w + (ca - g * v.w)) * v.e, r1 - r0, v.w * v.e, (cb - ca) * v.e);
-                    }
-                } else if (v.split == 1) {                                    // strips of rows
-                    for (int64_t g = r0 / v.h; g * v.h < r1; ++g) {
-                        const int64_t ra = max(r0, g * v.h), rb = min(r1, (g + 1) * v.h);
-                        piece(X, (g * v.stride + (ra - g * v.h) * v.cols + c0) * v.e, rb - ra, v.cols * v.e, (c1 - c0) * v.e);
-                    }
-                } else piece(X, (r0 * v.cols + c0) * v.e, r1 - r0, v.cols * v.e, (c1 - c0) * v.e);
-            }
+            if (lane == 0) { wt[nw][0] = t.m0; wt[nw][1] = t.m1; wt[nw][2] = t.n0; wt[nw][3] = t.n1; }
+            ++nw;
         }
+        __syncwarp();
+        for (int64_t k0 = 0; k0 < p.K; k0 += l.ks)
+            for (int j = 0; j < nw; ++j) {
+                TileInfo t;
+                t.m0 = wt[j][0]; t.m1 = wt[j][1]; t.n0 = wt[j][2]; t.n1 = wt[j][3]; t.q = q;
+                const int64_t k1 = min(p.K, k0 + l.ks);
+                slice(t, 0, k0, k1);
+                slice(t, 1, k0, k1);
+            }
+        __syncwarp();
+    }
     if (lane == 0)
         for (int k = 0; k < 4; ++k)
             if (cnt[k]) atomicAdd(reinterpret_cast<unsigned long long*>(&l.out[k]), (unsigned long long)cnt[k]);
@@ -514,6 +545,8 @@ extern "C" ccl_status ccl_traffic_lru(const ccl_traffic_desc* d, const ccl_l2_mo
     if (m->line_bytes <= 0 || m->ways <= 0 || m->capacity_bytes <= 0 || (m->traversal != 0 && m->traversal != 1))
         return fail(CCL_ERR_INVALID_ARG, "ccl_traffic_lru: line_bytes, ways, capacity_bytes must be positive and traversal 0 or 1");
     if (m->hash != 0 && m->hash != 1) return fail(CCL_ERR_INVALID_ARG, "ccl_traffic_lru: hash must be 0 or 1");
+    if (m->wave_ctas < 1 || m->k_slice < 0) return fail(CCL_ERR_INVALID_ARG, "ccl_traffic_lru: wave_ctas must be at least 1 and k_slice non-negative");
+    if (m->wave_ctas > kLruMaxWave) return fail(CCL_ERR_UNSUPPORTED, "ccl_traffic_lru: at most %d CTAs per wave", kLruMaxWave);
     if (m->ways > kLruMaxWays) return fail(CCL_ERR_UNSUPPORTED, "ccl_traffic_lru: at most %d ways", kLruMaxWays);
     if (m->capacity_bytes % ((int64_t)m->line_bytes * m->ways)) return fail(CCL_ERR_INVALID_ARG, "ccl_traffic_lru: capacity is not a whole number of sets");
     if (d->page_bytes % m->line_bytes) return fail(CCL_ERR_INVALID_ARG, "ccl_traffic_lru: page_bytes is not a multiple of line_bytes");
@@ -525,7 +558,13 @@ extern "C" ccl_status ccl_traffic_lru(const ccl_traffic_desc* d, const ccl_l2_mo
     LruParams l;
     std::memset(&l, 0, sizeof(l));
     l.line = m->line_bytes; l.ways = m->ways; l.traversal = m->traversal; l.hash = m->hash;
+    l.line_shift = l.sets_shift = -1;
+    l.wave = m->wave_ctas; l.ks = m->k_slice > 0 && m->k_slice < d->K ? m->k_slice : d->K;
     l.sets = m->capacity_bytes / ((int64_t)m->line_bytes * m->ways);
+    for (int b = 0; b < 62; ++b) {
+        if ((INT64_C(1) << b) == (int64_t)l.line) l.line_shift = b;
+        if ((INT64_C(1) << b) == l.sets) l.sets_shift = b;
+    }
     if (l.sets * d->P >= (INT64_C(1) << 31) * 128) return fail(CCL_ERR_UNSUPPORTED, "ccl_traffic_lru: too many sets");
     l.out = totals_dev;
     p.totals_l2 = totals_dev;
@@ -547,7 +586,7 @@ extern "C" ccl_status ccl_traffic_lru(const ccl_traffic_desc* d, const ccl_l2_mo
     count_launch();
     CCL_CUDA_TRY(cudaGetLastError());
     const int64_t threads = l.sets * d->P * 32;          // a warp per (chiplet, set)
-    traffic_lru_kernel<<<(unsigned)((threads + 127) / 128), 128, 0, st>>>(p, l);
+    traffic_lru_kernel<<<(unsigned)((threads + 32 * kLruWarps - 1) / (32 * kLruWarps)), 32 * kLruWarps, 0, st>>>(p, l);
     count_launch();
     CCL_CUDA_TRY(cudaGetLastError());
     return CCL_OK;

@@ -152,6 +152,9 @@ def traffic_desc(g, layout_bc, place_bc, S, assign, align=0, e=2):
     return td
 
 
+LRU_EXEC = dict(wave_ctas=1, k_slice=0)       # how a chiplet's CTAs run in the finite-L2 model (--lru-wave, --lru-kslice)
+
+
 def traffic_lru_best(g, layout_bc, place_bc, S, model_kw, e=2):
     """Remote bytes (A, B, C) behind a finite LRU L2 per chiplet: the best of both output partitions and both CTA
     traversals, as the paper reports (Sec. 4.1: "we sweep CTA traversal and output-partition choices")."""
@@ -162,7 +165,7 @@ def traffic_lru_best(g, layout_bc, place_bc, S, model_kw, e=2):
             continue
         for traversal in (0, 1):
             t = torch.empty((3, 2), dtype=torch.int64, device="cuda")
-            ccl.ccl_traffic_lru(td, ccl.L2Model(traversal=traversal, **model_kw), t)
+            ccl.ccl_traffic_lru(td, ccl.L2Model(traversal=traversal, **model_kw, **LRU_EXEC), t)
             r = [int(x) for x in t.cpu()[:, 1]]
             if best is None or sum(r) < sum(best["remote"]):
                 best = dict(remote=r, partition="N" if assign == ccl.ASSIGN_N_STRIPS else "M", traversal=traversal)
@@ -346,6 +349,8 @@ def main():
     ap.add_argument("--out", default=os.path.join(ROOT, "report_out"))
     ap.add_argument("--quick", action="store_true", help="fewer repetitions and P = 4 only in the sweep")
     ap.add_argument("--lru", action="store_true", help="also score the placements behind a finite LRU L2 per chiplet (slow at Llama sizes)")
+    ap.add_argument("--lru-wave", type=int, default=1, help="finite-L2 model: CTAs of a chiplet in flight together (1: one after the other)")
+    ap.add_argument("--lru-kslice", type=int, default=0, help="finite-L2 model: elements of K a wave consumes per lockstep step (0: all of K)")
     ap.add_argument("--l2-sweep", action="store_true", help="remote traffic against L2 capacity and data type under the finite-L2 model (then exit)")
     ap.add_argument("--extras", action="store_true", help="time the batched, gated-activation and alpha/beta entry points (then exit)")
     ap.add_argument("--only", default=None, help="run only the GEMMs whose name contains this text (e.g. for a profiler capture)")
@@ -353,6 +358,7 @@ def main():
     assert torch.cuda.is_available(), "report needs a CUDA device"
     pk = peaks()
     os.makedirs(args.out, exist_ok=True)
+    LRU_EXEC.update(wave_ctas=args.lru_wave, k_slice=args.lru_kslice)
     if args.extras:
         extras(args.out, args.quick)
         return

@@ -30,6 +30,16 @@ def test_hand_run_on_the_gpu():
         assert (int(t[0].sum()), int(t[1].sum()), int(t[2].sum())) == (a_bytes, b_bytes, 8)
 
 
+def test_wave_hand_run_on_the_gpu():
+    do, dl = traffic_pair(2, 2, 64, 1, 4096, BM=1, BN=1)
+    for line in open(os.path.join(HERE, "golden", "lru_wave_hand_run.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        sets, ways, wave, ks, a_bytes, b_bytes = (int(x) for x in line.split())
+        t = run(dl, ccl.L2Model(sets * ways * 128, 128, ways, 0, 0, wave, ks))
+        assert (int(t[0].sum()), int(t[1].sum()), int(t[2].sum())) == (a_bytes, b_bytes, 8)
+
+
 SHAPES = [
     # M, N, K, P, page, layouts, placement, BM, BN, a_trans, b_trans
     (256, 512, 128, 2, 4096, ("row", "row", "row"), (0, 0, 0), 128, 64, 0, 0),
@@ -58,6 +68,14 @@ def test_lru_bit_exact(M, N, K, P, S, lay, place, BM, BN, at, bt, assign):
             want = orc.traffic_lru(do, orc.L2Model(cap, line, ways, traversal, hashed))
             got = run(dl, ccl.L2Model(cap, line, ways, traversal, hashed))
             np.testing.assert_array_equal(got, want, err_msg=f"cache {cap}/{line}/{ways} traversal {traversal} hash {hashed}")
+    # waves of CTAs in lockstep through K: whole-line and ragged k slices, waves that divide the tile count or not
+    for cap, line, ways in ((8 * 1024, 128, 4), (96 * 1024, 128, 16), (1 << 20, 128, 16)):
+        if S % line:
+            continue
+        for wave, ks, traversal, hashed in ((4, 64, 0, 1), (3, 96, 1, 0), (7, 40, 0, 0), (256, 64, 1, 1), (2, 0, 0, 1), (1, 32, 1, 1)):
+            want = orc.traffic_lru(do, orc.L2Model(cap, line, ways, traversal, hashed, wave, ks))
+            got = run(dl, ccl.L2Model(cap, line, ways, traversal, hashed, wave, ks))
+            np.testing.assert_array_equal(got, want, err_msg=f"cache {cap}/{line}/{ways} traversal {traversal} hash {hashed} wave {wave} k_slice {ks}")
 
 
 def test_lru_llama_gateup_full_size_properties():
