@@ -107,8 +107,22 @@ struct TmaTiling {
     uint32_t tiles_x, tiles_y;    // per strip
     uint32_t stages, stage_bytes; // ring depth and bytes per ring slot
     uint64_t ntiles;
+    // page-interleaved CCL side (IL kernels): which side it is and how a tile's (x, row, strip) becomes coordinates
+    // of its rank-4 map.  il_mode 1: a chunk holds il_kr whole strip rows, map {x, row in chunk, strip, chunk};
+    // il_mode 2: a strip row is whole chunks of il_s8 8-byte units, map {x in chunk, chunk in row, row, strip}.
+    uint32_t il_mode, il_src, il_kr, il_s8;
 };
 
+struct Coord4 { int c[4]; };
+__device__ __forceinline__ Coord4 tile_coord(const TmaTiling& t, bool il_side, uint32_t x, uint32_t y, uint32_t g) {
+    Coord4 r;
+    if (!il_side) { r.c[0] = (int)x; r.c[1] = (int)y; r.c[2] = (int)g; r.c[3] = 0; }
+    else if (t.il_mode == 1) { r.c[0] = (int)x; r.c[1] = (int)(y % t.il_kr); r.c[2] = (int)g; r.c[3] = (int)(y / t.il_kr); }
+    else { r.c[0] = (int)(x % t.il_s8); r.c[1] = (int)(x / t.il_s8); r.c[2] = (int)y; r.c[3] = (int)g; }
+    return r;
+}
+
+template <bool IL>
 __global__ void __launch_bounds__(32) repack_tma_kernel(const __grid_constant__ CUtensorMap src_map,
                                                            const __grid_constant__ CUtensorMap dst_map, TmaTiling t) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
@@ -132,7 +146,11 @@ __global__ void __launch_bounds__(32) repack_tma_kernel(const __grid_constant__ 
         uint32_t rem = (uint32_t)(tile - (uint64_t)g * per_strip);
         uint32_t ty = rem / t.tiles_x, tx = rem - ty * t.tiles_x;
         mbar_expect_tx(&full[slot], box_bytes);
-        tma_load_3d(stage0 + (size_t)slot * t.stage_bytes, &src_map, &full[slot], (int)(tx * t.bx), (int)(ty * t.by), (int)g);
+        if (IL) {
+            const Coord4 c = tile_coord(t, t.il_src != 0, tx * t.bx, ty * t.by, g);
+            tma_load_4d(stage0 + (size_t)slot * t.stage_bytes, &src_map, &full[slot], c.c[0], c.c[1], c.c[2], c.c[3]);
+        } else
+            tma_load_3d(stage0 + (size_t)slot * t.stage_bytes, &src_map, &full[slot], (int)(tx * t.bx), (int)(ty * t.by), (int)g);
     };
 
     for (uint64_t it = 0; it < t.stages; ++it) issue_load(it);
@@ -145,7 +163,11 @@ __global__ void __launch_bounds__(32) repack_tma_kernel(const __grid_constant__ 
         uint32_t g = (uint32_t)(tile / per_strip);
         uint32_t rem = (uint32_t)(tile - (uint64_t)g * per_strip);
         uint32_t ty = rem / t.tiles_x, tx = rem - ty * t.tiles_x;
-        tma_store_3d(&dst_map, stage0 + (size_t)slot * t.stage_bytes, (int)(tx * t.bx), (int)(ty * t.by), (int)g);
+        if (IL) {
+            const Coord4 c = tile_coord(t, t.il_src == 0, tx * t.bx, ty * t.by, g);
+            tma_store_4d(&dst_map, stage0 + (size_t)slot * t.stage_bytes, c.c[0], c.c[1], c.c[2], c.c[3]);
+        } else
+            tma_store_3d(&dst_map, stage0 + (size_t)slot * t.stage_bytes, (int)(tx * t.bx), (int)(ty * t.by), (int)g);
         tma_store_commit();
         // the store issued one iteration ago has now read its buffer: refill that slot
         if (it >= 1) {
@@ -211,27 +233,69 @@ static ccl_status launch_tma(const char* src, char* dst, const CopyPlan& p, int 
         if (sscanf(f, "%d,%d,%d,%d", &a, &b, &c, &d2) == 4 && a > 0 && a <= kTmaMaxStages && b > 0 && c > 0 && d2 > 0) { t.stages = a; t.stage_bytes = b * 1024; ctas_per_sm = c; max_bx = d2; }
     }
     t.bx = (uint32_t)std::min<uint64_t>((uint64_t)max_bx, dims[0]);
+    t.il_mode = t.il_src = 0; t.il_kr = t.il_s8 = 1;
+    if (p.il_chunk) {
+        t.il_src = p.il_dst ? 0 : 1;
+        if (p.il_chunk % p.row_bytes == 0) { t.il_mode = 1; t.il_kr = (uint32_t)(p.il_chunk / p.row_bytes); }
+        else {                                           // whole chunks per strip row: a box stays inside one chunk
+            t.il_mode = 2; t.il_s8 = (uint32_t)(p.il_chunk / 8);
+            while (t.il_s8 % t.bx || (t.bx & 1)) --t.bx;          // even: a TMA copy starts on a 16-byte boundary
+        }
+    }
     t.by = (uint32_t)std::max<uint64_t>(1, std::min<uint64_t>(std::min<uint64_t>(256, dims[1]), t.stage_bytes / (t.bx * 8ull)));
+    uint32_t by_in = t.by, by_out = 1;                     // il_mode 1: rows of a box inside a chunk x chunks of a box
+    if (t.il_mode == 1) {
+        if (t.by >= t.il_kr) { by_in = t.il_kr; by_out = std::min<uint32_t>(t.by / t.il_kr, 256); }
+        else { while (t.il_kr % by_in) --by_in; }
+        t.by = by_in * by_out;
+    }
     t.tiles_x = (uint32_t)((dims[0] + t.bx - 1) / t.bx);
     t.tiles_y = (uint32_t)((dims[1] + t.by - 1) / t.by);
     t.ntiles = (uint64_t)t.tiles_x * t.tiles_y * (uint64_t)p.nstrips;
-    uint32_t box[3] = {t.bx, t.by, 1};
     // a strip stride is irrelevant (and may be 0) when there is one strip: give the encoder a valid value
-    uint64_t sstr[2] = {(uint64_t)p.src_r, (uint64_t)(p.nstrips > 1 ? p.src_g : p.src_r * p.rows)};
-    uint64_t dstr[2] = {(uint64_t)p.dst_r, (uint64_t)(p.nstrips > 1 ? p.dst_g : p.dst_r * p.rows)};
+    const uint64_t src_g = (uint64_t)(p.nstrips > 1 ? p.src_g : p.src_r * p.rows), dst_g = (uint64_t)(p.nstrips > 1 ? p.dst_g : p.dst_r * p.rows);
     CUtensorMap sm, dm;
-    ccl_status s = encode_tmap(&sm, CU_TENSOR_MAP_DATA_TYPE_UINT64, 3, src, dims, sstr, box, CU_TENSOR_MAP_SWIZZLE_NONE);
-    if (s) return s;
-    s = encode_tmap(&dm, CU_TENSOR_MAP_DATA_TYPE_UINT64, 3, dst, dims, dstr, box, CU_TENSOR_MAP_SWIZZLE_NONE);
-    if (s) return s;
+    ccl_status s;
+    if (!t.il_mode) {
+        uint32_t box[3] = {t.bx, t.by, 1};
+        uint64_t sstr[2] = {(uint64_t)p.src_r, src_g}, dstr[2] = {(uint64_t)p.dst_r, dst_g};
+        s = encode_tmap(&sm, CU_TENSOR_MAP_DATA_TYPE_UINT64, 3, src, dims, sstr, box, CU_TENSOR_MAP_SWIZZLE_NONE);
+        if (s) return s;
+        s = encode_tmap(&dm, CU_TENSOR_MAP_DATA_TYPE_UINT64, 3, dst, dims, dstr, box, CU_TENSOR_MAP_SWIZZLE_NONE);
+        if (s) return s;
+    } else {
+        // plain side: {x, row, strip, 1}; interleaved side: see TmaTiling.  Both boxes are by x bx dense in shared memory.
+        const uint64_t S = (uint64_t)p.il_chunk, P = (uint64_t)p.il_P, chunks = ((uint64_t)p.rows * p.row_bytes + S - 1) / S;
+        uint64_t pdims[4] = {dims[0], dims[1], dims[2], 1}, idims[4], istr[3];
+        uint32_t pbox[4] = {t.bx, t.by, 1, 1}, ibox[4];
+        if (t.il_mode == 1) {
+            idims[0] = dims[0]; idims[1] = t.il_kr; idims[2] = P; idims[3] = chunks;
+            istr[0] = (uint64_t)p.row_bytes; istr[1] = S; istr[2] = S * P;
+            ibox[0] = t.bx; ibox[1] = by_in; ibox[2] = 1; ibox[3] = by_out;
+        } else {
+            const uint64_t m = (uint64_t)p.row_bytes / S;
+            idims[0] = t.il_s8; idims[1] = m; idims[2] = dims[1]; idims[3] = P;
+            istr[0] = S * P; istr[1] = m * S * P; istr[2] = S;
+            ibox[0] = t.bx; ibox[1] = 1; ibox[2] = t.by; ibox[3] = 1;
+        }
+        const bool il_src = t.il_src != 0;
+        uint64_t pstr[3] = {(uint64_t)(il_src ? p.dst_r : p.src_r), il_src ? dst_g : src_g, (il_src ? dst_g : src_g) * dims[2]};
+        s = encode_tmap(&sm, CU_TENSOR_MAP_DATA_TYPE_UINT64, 4, src, il_src ? idims : pdims, il_src ? istr : pstr, il_src ? ibox : pbox, CU_TENSOR_MAP_SWIZZLE_NONE);
+        if (s) return s;
+        s = encode_tmap(&dm, CU_TENSOR_MAP_DATA_TYPE_UINT64, 4, dst, il_src ? pdims : idims, il_src ? pstr : istr, il_src ? pbox : ibox, CU_TENSOR_MAP_SWIZZLE_NONE);
+        if (s) return s;
+    }
     size_t smem = (size_t)t.stages * t.stage_bytes + 128 + t.stages * sizeof(uint64_t);
-    static size_t attr_set = 0;
-    if (attr_set < smem) {
-        CCL_CUDA_TRY(cudaFuncSetAttribute(repack_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        attr_set = smem;
+    static size_t attr_set[2] = {0, 0};
+    const int which = t.il_mode ? 1 : 0;
+    if (attr_set[which] < smem) {
+        if (which) CCL_CUDA_TRY(cudaFuncSetAttribute(repack_tma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        else CCL_CUDA_TRY(cudaFuncSetAttribute(repack_tma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        attr_set[which] = smem;
     }
     unsigned grid = (unsigned)std::min<uint64_t>(t.ntiles, (uint64_t)sms * ctas_per_sm);
-    repack_tma_kernel<<<grid, 32, smem, st>>>(sm, dm, t);
+    if (which) repack_tma_kernel<true><<<grid, 32, smem, st>>>(sm, dm, t);
+    else repack_tma_kernel<false><<<grid, 32, smem, st>>>(sm, dm, t);
     count_launch();
     CCL_CUDA_TRY(cudaGetLastError());
     return CCL_OK;
@@ -300,7 +364,9 @@ extern "C" ccl_status ccl_repack(const ccl_mat* m, const void* src_dev, void* ds
 
     // path choice: TMA when everything is 16-byte aligned and the copy is big enough to be worth a ring
     const char* force = std::getenv("CCL_REPACK_PATH");
-    bool tma_ok = vec == 16 && !p.il_chunk && p.rows < (INT64_C(1) << 31) && p.row_bytes / 8 < (INT64_C(1) << 31) &&
+    // (page-interleaved side: a chunk must hold whole strip rows, or a strip row whole chunks)
+    const bool il_ok = !p.il_chunk || p.il_chunk % p.row_bytes == 0 || p.row_bytes % p.il_chunk == 0;
+    bool tma_ok = vec == 16 && il_ok && p.rows < (INT64_C(1) << 31) && p.row_bytes / 8 < (INT64_C(1) << 31) &&
                   std::max(std::max(p.src_g, p.src_r), std::max(p.dst_g, p.dst_r)) < (INT64_C(1) << 40);
     bool use_tma = tma_ok && p.nstrips * p.rows * p.row_bytes >= (INT64_C(1) << 20);
     if (force && !std::strcmp(force, "vec")) use_tma = false;

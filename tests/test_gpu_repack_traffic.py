@@ -81,6 +81,11 @@ REPACK_CASES = [
     dict(rows=77, cols=96, P=3, part=2, layout=2, align=48, e=1),      # chunk size not a power of two
     dict(rows=64, cols=200, P=2, part=2, layout=2, align=40),          # 8-byte vectors at most
     dict(rows=4099, cols=2056, P=2, part=2, layout=2, align=2 << 20),
+    dict(rows=512, cols=8192, P=2, part=2, layout=2, align=4096),      # a strip row is two whole chunks
+    dict(rows=301, cols=7168, P=4, part=2, layout=2, align=512),       # ... seven chunks of 512 bytes, ragged rows
+    dict(rows=1001, cols=1024, P=4, part=2, layout=2, align=4096),     # a chunk holds 8 strip rows, the last chunk 1
+    dict(rows=1001, cols=1024, P=4, part=2, layout=2, align=16384, e=4),   # ... 16 rows of 4-byte elements
+    dict(rows=2100, cols=2048, P=4, part=1, layout=2, align=8192),     # strips of rows: a chunk holds two rows
 ]
 
 
