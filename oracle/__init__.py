@@ -96,6 +96,19 @@ def repack(m, src, direction=0):
     return dst
 
 
+def repack_transposed(m, src_t):
+    """Transposing repack (Sec. 3.3: an operand stored the other way round is repacked into CCL): src_t is the
+    row-major transpose [cols x rows] of the matrix `m` describes; element (r, c) of that matrix, src_t[c, r], goes to
+    offset index(r, c) of Eq. 1-3 (map_table); padding is zero.  Written from the map alone, one element at a time."""
+    src_t = np.ascontiguousarray(src_t).reshape(m.cols, m.rows)
+    assert src_t.itemsize == m.elem_bytes
+    table = map_table(m)
+    out = np.zeros(buffer_bytes(m) // m.elem_bytes, dtype=src_t.dtype)
+    for r in range(m.rows):
+        out[table[r]] = src_t[:, r]
+    return out
+
+
 def gemm(A, B, M, N, K, a_trans=0, b_trans=0, block=None, want64=False, threads=None):
     """A, B: uint16 (bf16 bit patterns), stored row-major as the flags say.
     Returns (ref32, ref64 or None, out_bf16_bits) for block = (m0, m1, n0, n1) or the whole C."""

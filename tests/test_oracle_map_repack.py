@@ -165,3 +165,22 @@ def test_repack_aligned_padding_is_zero(e, dt):
     for g in range(P):
         np.testing.assert_array_equal(gr[g * sr:g * sr + 2 * Cc].reshape(2, Cc), xr[2 * g:2 * g + 2])
         assert (gr[g * sr + 2 * Cc:(g + 1) * sr] == 0).all()
+
+
+def test_repack_transposed_hand_example_and_definition():
+    # the Fig. 4(a) example with the operand stored as [N x K] = [8 x 4], src_t[n, k] = 4n + k: position index(k, n)
+    # of the output holds 4n + k; by the table of the worked example the first strip (n < 4) is, row by row of k,
+    # 0 4 8 12 | 1 5 9 13 | 2 6 10 14 | 3 7 11 15 and the second strip the same plus 16
+    m = ccl_cols(4, 8, 2)
+    got = orc.repack_transposed(m, np.arange(32, dtype=np.uint16).reshape(8, 4))
+    first = np.array([0, 4, 8, 12, 1, 5, 9, 13, 2, 6, 10, 14, 3, 7, 11, 15], dtype=np.uint16)
+    np.testing.assert_array_equal(got, np.concatenate([first, first + 16]))
+    # in general it is the plain repack of the transposed array, padding included
+    for R, Cc, P, e, dt, align, lay in ((130, 384, 4, 2, np.uint16, 0, orc.CCL), (7, 24, 3, 1, np.uint8, 256, orc.CCL),
+                                        (33, 50, 5, 4, np.uint32, 0, orc.CCL), (64, 200, 2, 2, np.uint16, 40, orc.CCL_INTERLEAVED)):
+        x = np.random.default_rng(5).integers(1, 200, size=(R, Cc)).astype(dt)
+        for part in (orc.PART_COLS, orc.PART_ROWS):
+            if part == orc.PART_ROWS and R % P:
+                continue
+            mm = orc.Mat(R, Cc, e, P, part, lay, align)
+            np.testing.assert_array_equal(orc.repack_transposed(mm, np.ascontiguousarray(x.T)), orc.repack(mm, x, 0))
