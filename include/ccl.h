@@ -104,6 +104,26 @@ ccl_status ccl_strip_stride(const ccl_mat* m, int64_t* elems);
  */
 ccl_status ccl_repack(const ccl_mat* m, const void* src_dev, void* dst_dev, int dir, void* cuda_stream);
 
+/*
+ * The same copy for `batch` matrices of one descriptor in one launch (the expert weights of an MoE layer, Sec. 4.1):
+ * matrix i is read at src_dev + i * src_stride_bytes and written at dst_dev + i * dst_stride_bytes.
+ * batch in [1, 65535]; strides are multiples of elem_bytes (of 16 for the fast path); the destination stride is at
+ * least the size of one output (ccl_buffer_bytes(m) for dir = 0, rows*cols*elem_bytes for dir = 1) and the source
+ * stride is non-negative (0 repeats one source), else CCL_ERR_INVALID_ARG / CCL_ERR_ALIGN.  Bytes between the
+ * outputs are left untouched.
+ */
+ccl_status ccl_repack_batched(const ccl_mat* m, int32_t batch, const void* src_dev, int64_t src_stride_bytes, void* dst_dev,
+                              int64_t dst_stride_bytes, int dir, void* cuda_stream);
+
+/*
+ * Transposing repack: src_dev holds the row-major TRANSPOSE [cols x rows] of the matrix `m` describes (a weight
+ * kept as [N x K] that a GEMM wants as CCL [K x N], Sec. 3.3 "repacked when profitable"); dst_dev receives the layout
+ * `m` describes: element (r, c) of it is src[c * rows + r].  Padding bytes are written as zero.
+ * Any descriptor the map accepts; 2-byte elements with rows, cols, strip width, strip stride and chunk size all
+ * multiples of 8 elements and 16-byte aligned bases take the fast path (64 x 64 tiles through shared memory).
+ */
+ccl_status ccl_repack_transpose(const ccl_mat* m, const void* src_dev, void* dst_dev, void* cuda_stream);
+
 /* ---- GEMM on CCL operands (Sec. 2.2 execution model, Sec. 3.3 "only the address map changes") */
 
 /*

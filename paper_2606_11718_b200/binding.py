@@ -19,7 +19,7 @@ PART_NONE, PART_ROWS, PART_COLS = 0, 1, 2
 PLACE_RR, PLACE_BLOCK, PLACE_BEST = 0, 1, 2
 ASSIGN_N_STRIPS, ASSIGN_M_STRIPS, ASSIGN_EXPLICIT = 0, 1, 2
 
-EXPORTS = ["ccl_map_offset", "ccl_map_inverse", "ccl_buffer_bytes", "ccl_strip_stride", "ccl_repack", "ccl_gemm_workspace",
+EXPORTS = ["ccl_map_offset", "ccl_map_inverse", "ccl_buffer_bytes", "ccl_strip_stride", "ccl_repack", "ccl_repack_batched", "ccl_repack_transpose", "ccl_gemm_workspace",
            "ccl_gemm", "ccl_gemm_batched_workspace", "ccl_gemm_batched", "ccl_gemm_axpby", "ccl_gemm_swiglu", "ccl_gemm_static_ws", "ccl_gemm_status", "ccl_traffic_sizes", "ccl_traffic", "ccl_traffic_l2", "ccl_traffic_lru", "ccl_last_error", "ccl_launch_count", "ccl_version"]
 
 
@@ -80,6 +80,8 @@ def lib():
         l.ccl_buffer_bytes.argtypes = [C.POINTER(Mat), C.POINTER(C.c_int64)]
         l.ccl_strip_stride.argtypes = [C.POINTER(Mat), C.POINTER(C.c_int64)]
         l.ccl_repack.argtypes = [C.POINTER(Mat), C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]
+        l.ccl_repack_transpose.argtypes = [C.POINTER(Mat), C.c_void_p, C.c_void_p, C.c_void_p]
+        l.ccl_repack_batched.argtypes = [C.POINTER(Mat), C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_int, C.c_void_p]
         l.ccl_gemm_workspace.argtypes = [C.POINTER(GemmDesc), C.POINTER(C.c_size_t)]
         l.ccl_gemm.argtypes = [C.POINTER(GemmDesc), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         l.ccl_gemm_batched_workspace.argtypes = [C.POINTER(GemmDesc), C.c_int32, C.POINTER(C.c_size_t)]
@@ -157,6 +159,23 @@ def ccl_repack(m, src, dst, direction=0):
     if src.numel() * src.element_size() < need_src or dst.numel() * dst.element_size() < need_dst:
         raise ValueError("ccl_repack: buffer too small")
     _check(lib().ccl_repack(C.byref(m), _ptr(src), _ptr(dst), direction, _stream()))
+
+
+def ccl_repack_transpose(m, src, dst):
+    """src: the row-major transpose [cols x rows] of the matrix `m` describes; dst: the layout `m` describes."""
+    if src.numel() * src.element_size() < m.rows * m.cols * m.elem_bytes or dst.numel() * dst.element_size() < ccl_buffer_bytes(m):
+        raise ValueError("ccl_repack_transpose: buffer too small")
+    _check(lib().ccl_repack_transpose(C.byref(m), _ptr(src), _ptr(dst), _stream()))
+
+
+def ccl_repack_batched(m, batch, src, src_stride_bytes, dst, dst_stride_bytes, direction=0):
+    """`batch` matrices of one descriptor in one launch; matrix i at src + i * src_stride_bytes -> dst + i * dst_stride_bytes."""
+    need_src = m.rows * m.cols * m.elem_bytes if direction == 0 else ccl_buffer_bytes(m)
+    need_dst = ccl_buffer_bytes(m) if direction == 0 else m.rows * m.cols * m.elem_bytes
+    if batch >= 1 and (src.numel() * src.element_size() < (batch - 1) * src_stride_bytes + need_src
+                       or dst.numel() * dst.element_size() < (batch - 1) * dst_stride_bytes + need_dst):
+        raise ValueError("ccl_repack_batched: buffer too small")
+    _check(lib().ccl_repack_batched(C.byref(m), batch, _ptr(src), src_stride_bytes, _ptr(dst), dst_stride_bytes, direction, _stream()))
 
 
 def ccl_gemm_workspace(d):

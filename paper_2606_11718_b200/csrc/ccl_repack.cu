@@ -26,6 +26,7 @@ struct CopyPlan {
     // g*il_chunk + (b / il_chunk)*il_chunk*il_P + b % il_chunk
     int64_t il_chunk, il_P;
     int32_t il_shift, il_dst;                 // log2(il_chunk) or -1; 1 = the destination is the interleaved side
+    int64_t batch, src_b, dst_b;              // matrices per launch and the byte strides between them
 };
 
 __device__ __forceinline__ int64_t interleaved_off(const CopyPlan& p, int64_t g, int64_t b) {
@@ -58,8 +59,8 @@ template <typename V, typename IDX>
 __global__ void __launch_bounds__(kVecThreads) repack_vec_kernel(const char* __restrict__ src, char* __restrict__ dst, CopyPlan p,
                                                                  IDX chunks_per_row, IDX chunks_per_strip) {
     const int64_t g = blockIdx.y;
-    const char* s = src + g * p.src_g;
-    char* d = dst + g * p.dst_g;
+    const char* s = src + (int64_t)blockIdx.z * p.src_b + g * p.src_g;
+    char* d = dst + (int64_t)blockIdx.z * p.dst_b + g * p.dst_g;
     const IDX step = (IDX)gridDim.x * kVecThreads * kVecUnroll;
     for (IDX base = (IDX)blockIdx.x * kVecThreads * kVecUnroll + threadIdx.x; base < chunks_per_strip; base += step) {
         V v[kVecUnroll];
@@ -89,8 +90,8 @@ __global__ void __launch_bounds__(kVecThreads) repack_vec_kernel(const char* __r
 }
 
 template <typename V>
-__global__ void zero_pad_kernel(char* dst, int64_t pad_g, int64_t pad_off, int64_t chunks) {
-    char* d = dst + (int64_t)blockIdx.y * pad_g + pad_off;
+__global__ void zero_pad_kernel(char* dst, int64_t pad_g, int64_t pad_off, int64_t chunks, int64_t dst_b) {
+    char* d = dst + (int64_t)blockIdx.z * dst_b + (int64_t)blockIdx.y * pad_g + pad_off;
     V z;
     memset(&z, 0, sizeof(V));
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < chunks; i += (int64_t)gridDim.x * blockDim.x)
@@ -106,23 +107,26 @@ struct TmaTiling {
     uint32_t bx, by;              // box extents (8-byte units, rows)
     uint32_t tiles_x, tiles_y;    // per strip
     uint32_t stages, stage_bytes; // ring depth and bytes per ring slot
-    uint64_t ntiles;
-    // page-interleaved CCL side (IL kernels): which side it is and how a tile's (x, row, strip) becomes coordinates
-    // of its rank-4 map.  il_mode 1: a chunk holds il_kr whole strip rows, map {x, row in chunk, strip, chunk};
+    uint64_t ntiles;              // over all strips of all matrices of the batch
+    // page-interleaved CCL side: which side it is and how a tile's (x, row, strip) becomes coordinates of its map.
+    // il_mode 1: a chunk holds il_kr whole strip rows, map {x, row in chunk, strip, chunk};
     // il_mode 2: a strip row is whole chunks of il_s8 8-byte units, map {x in chunk, chunk in row, row, strip}.
-    uint32_t il_mode, il_src, il_kr, il_s8;
+    // The matrix of a batch is the coordinate after those (after {x, row, strip} on a plain side).
+    uint32_t il_mode, il_src, il_kr, il_s8, nstrips;
 };
 
-struct Coord4 { int c[4]; };
-__device__ __forceinline__ Coord4 tile_coord(const TmaTiling& t, bool il_side, uint32_t x, uint32_t y, uint32_t g) {
-    Coord4 r;
-    if (!il_side) { r.c[0] = (int)x; r.c[1] = (int)y; r.c[2] = (int)g; r.c[3] = 0; }
-    else if (t.il_mode == 1) { r.c[0] = (int)x; r.c[1] = (int)(y % t.il_kr); r.c[2] = (int)g; r.c[3] = (int)(y / t.il_kr); }
-    else { r.c[0] = (int)(x % t.il_s8); r.c[1] = (int)(x / t.il_s8); r.c[2] = (int)y; r.c[3] = (int)g; }
+struct Coord5 { int c[5]; };
+__device__ __forceinline__ Coord5 tile_coord(const TmaTiling& t, bool il_side, uint32_t x, uint32_t y, uint32_t g, uint32_t b) {
+    Coord5 r;
+    if (!il_side) { r.c[0] = (int)x; r.c[1] = (int)y; r.c[2] = (int)g; r.c[3] = (int)b; r.c[4] = 0; }
+    else if (t.il_mode == 1) { r.c[0] = (int)x; r.c[1] = (int)(y % t.il_kr); r.c[2] = (int)g; r.c[3] = (int)(y / t.il_kr); r.c[4] = (int)b; }
+    else { r.c[0] = (int)(x % t.il_s8); r.c[1] = (int)(x / t.il_s8); r.c[2] = (int)y; r.c[3] = (int)g; r.c[4] = (int)b; }
     return r;
 }
 
-template <bool IL>
+// RANK 3: one matrix, no interleaved side (maps {x, row, strip}); RANK 4: a batch of those, or one matrix with an
+// interleaved side; RANK 5: a batch with an interleaved side.
+template <int RANK>
 __global__ void __launch_bounds__(32) repack_tma_kernel(const __grid_constant__ CUtensorMap src_map,
                                                            const __grid_constant__ CUtensorMap dst_map, TmaTiling t) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
@@ -138,19 +142,30 @@ __global__ void __launch_bounds__(32) repack_tma_kernel(const __grid_constant__ 
 
     const uint32_t box_bytes = t.bx * t.by * 8u;
     const uint64_t per_strip = (uint64_t)t.tiles_x * t.tiles_y;
+    struct Tile { uint32_t x, y, g, b; };
+    auto decode = [&](uint64_t tile) {
+        Tile r;
+        uint64_t gi = tile / per_strip;                       // strip index over the whole batch
+        uint32_t rem = (uint32_t)(tile - gi * per_strip);
+        uint32_t ty = rem / t.tiles_x, tx = rem - ty * t.tiles_x;
+        r.x = tx * t.bx; r.y = ty * t.by;
+        if (RANK == 3) { r.g = (uint32_t)gi; r.b = 0; }
+        else { r.b = (uint32_t)(gi / t.nstrips); r.g = (uint32_t)(gi - (uint64_t)r.b * t.nstrips); }
+        return r;
+    };
     auto issue_load = [&](uint64_t it) {
         uint64_t tile = (uint64_t)blockIdx.x + it * gridDim.x;
         if (tile >= t.ntiles) return;
         uint32_t slot = (uint32_t)(it % t.stages);
-        uint32_t g = (uint32_t)(tile / per_strip);
-        uint32_t rem = (uint32_t)(tile - (uint64_t)g * per_strip);
-        uint32_t ty = rem / t.tiles_x, tx = rem - ty * t.tiles_x;
+        const Tile ti = decode(tile);
+        void* buf = stage0 + (size_t)slot * t.stage_bytes;
         mbar_expect_tx(&full[slot], box_bytes);
-        if (IL) {
-            const Coord4 c = tile_coord(t, t.il_src != 0, tx * t.bx, ty * t.by, g);
-            tma_load_4d(stage0 + (size_t)slot * t.stage_bytes, &src_map, &full[slot], c.c[0], c.c[1], c.c[2], c.c[3]);
-        } else
-            tma_load_3d(stage0 + (size_t)slot * t.stage_bytes, &src_map, &full[slot], (int)(tx * t.bx), (int)(ty * t.by), (int)g);
+        if (RANK == 3) tma_load_3d(buf, &src_map, &full[slot], (int)ti.x, (int)ti.y, (int)ti.g);
+        else {
+            const Coord5 c = tile_coord(t, t.il_mode && t.il_src, ti.x, ti.y, ti.g, ti.b);
+            if (RANK == 4) tma_load_4d(buf, &src_map, &full[slot], c.c[0], c.c[1], c.c[2], c.c[3]);
+            else tma_load_5d(buf, &src_map, &full[slot], c.c[0], c.c[1], c.c[2], c.c[3], c.c[4]);
+        }
     };
 
     for (uint64_t it = 0; it < t.stages; ++it) issue_load(it);
@@ -160,14 +175,14 @@ __global__ void __launch_bounds__(32) repack_tma_kernel(const __grid_constant__ 
         uint32_t slot = (uint32_t)(it % t.stages);
         uint32_t parity = (uint32_t)((it / t.stages) & 1);
         if (!mbar_wait_bounded(&full[slot], parity)) { atomicExch(&g_repack_status, 1); break; }
-        uint32_t g = (uint32_t)(tile / per_strip);
-        uint32_t rem = (uint32_t)(tile - (uint64_t)g * per_strip);
-        uint32_t ty = rem / t.tiles_x, tx = rem - ty * t.tiles_x;
-        if (IL) {
-            const Coord4 c = tile_coord(t, t.il_src == 0, tx * t.bx, ty * t.by, g);
-            tma_store_4d(&dst_map, stage0 + (size_t)slot * t.stage_bytes, c.c[0], c.c[1], c.c[2], c.c[3]);
-        } else
-            tma_store_3d(&dst_map, stage0 + (size_t)slot * t.stage_bytes, (int)(tx * t.bx), (int)(ty * t.by), (int)g);
+        const Tile ti = decode(tile);
+        const void* buf = stage0 + (size_t)slot * t.stage_bytes;
+        if (RANK == 3) tma_store_3d(&dst_map, buf, (int)ti.x, (int)ti.y, (int)ti.g);
+        else {
+            const Coord5 c = tile_coord(t, t.il_mode && !t.il_src, ti.x, ti.y, ti.g, ti.b);
+            if (RANK == 4) tma_store_4d(&dst_map, buf, c.c[0], c.c[1], c.c[2], c.c[3]);
+            else tma_store_5d_bulk(&dst_map, buf, c.c[0], c.c[1], c.c[2], c.c[3], c.c[4]);
+        }
         tma_store_commit();
         // the store issued one iteration ago has now read its buffer: refill that slot
         if (it >= 1) {
@@ -176,6 +191,96 @@ __global__ void __launch_bounds__(32) repack_tma_kernel(const __grid_constant__ 
         }
     }
     tma_store_wait_all<0>();
+}
+
+// ------------------------------------------------------------------------------------------
+// Transposing repack: the source is the row-major TRANSPOSE [cols x rows] of the described matrix (a weight kept as
+// [N x K] that a GEMM wants as CCL [K x N]); element (r, c) of the output comes from src[c * rows + r].
+// ------------------------------------------------------------------------------------------
+constexpr int kTrTile = 64, kTrThreads = 256, kTrStages = 4;
+
+// 2-byte elements, everything a multiple of 8 elements: 64 x 64 tiles through 8 KB of shared memory.  A tile is read
+// as 16-byte pieces of source rows (8 consecutive r at one c) and written as 16-byte pieces of output rows (8
+// consecutive c at one r).  Shared memory holds the tile as [c][r] with the 16-byte granule index XORed with c / 8,
+// which makes both the 16-byte stores of the first phase and the 2-byte gathers of the second free of bank conflicts.
+__global__ void __launch_bounds__(kTrThreads) repack_transpose_vec_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, MatView v,
+                                                                          int64_t tiles_c, int64_t ntiles, int il_shift) {
+    __shared__ __align__(16) uint16_t tile[kTrStages][kTrTile * kTrTile];
+    const int t = threadIdx.x, q = t & 7, o = t >> 3;                       // q: 16-byte piece of a 128-byte row, o: 0..31
+    // A CTA takes a contiguous run of tiles, c fastest: it fills 64 output rows from left to right (its 128-byte
+    // pieces of a row follow each other in time and leave L2 as whole rows), while the CTAs next to it read the
+    // neighbouring pieces of the same source rows.
+    const int64_t first = ntiles * blockIdx.x / gridDim.x, last = ntiles * (blockIdx.x + 1) / gridDim.x;
+    // source tiles arrive by 16-byte asynchronous copies straight into their (swizzled) place: kTrStages - 1 tiles
+    // of reads stay in flight per CTA without holding registers
+    auto load_tile = [&](int stage, int64_t ti) {                           // source row c0 + c, elements r0 + 8q .. + 8
+        const int64_t tr = ti / tiles_c, tc = ti - tr * tiles_c;
+        const int64_t r0 = tr * kTrTile, c0 = tc * kTrTile;
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+            const int c = o + 32 * k;
+            const bool in = c0 + c < v.cols && r0 + 8 * q < v.rows;        // outside: zero-filled (source size 0)
+            const uint16_t* g = in ? src + (c0 + c) * v.rows + r0 + 8 * q : src;
+            const uint32_t sm = smem_u32(&tile[stage][c * kTrTile + ((q ^ ((c >> 3) & 7)) << 3)]);
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(sm), "l"(g), "r"(in ? 16 : 0) : "memory");
+        }
+    };
+#pragma unroll
+    for (int d = 0; d < kTrStages - 1; ++d) {
+        if (first + d < last) load_tile(d, first + d);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    }
+    for (int64_t ti = first; ti < last; ++ti) {
+        const int stage = (int)((ti - first) % kTrStages);
+        const int64_t tr = ti / tiles_c, tc = ti - tr * tiles_c;
+        const int64_t r0 = tr * kTrTile, c0 = tc * kTrTile;
+        asm volatile("cp.async.wait_group %0;" ::"n"(kTrStages - 2) : "memory");
+        __syncthreads();                                                    // tile ti has landed; tile ti - 1 has been read out
+        if (ti + kTrStages - 1 < last) load_tile((int)((ti - first + kTrStages - 1) % kTrStages), ti + kTrStages - 1);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        const uint16_t* tl = tile[stage];
+        // packed strips of columns (Eq. 3): one division per thread and tile, rows are w apart
+        const bool strips = v.split == 2;
+        int64_t col_off = 0, g = 0;
+        if (strips) { const int64_t c = c0 + 8 * q; g = c / v.w; col_off = c - g * v.w; if (!v.ichunk) col_off += g * v.stride; }
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {                                       // output row r0 + r, columns c0 + 8q .. + 8
+            const int r = o + 32 * k;
+            if (r0 + r >= v.rows || c0 + 8 * q >= v.cols) continue;
+            uint16_t e[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) e[j] = tl[(8 * q + j) * kTrTile + ((((r >> 3) ^ q) & 7) << 3) + (r & 7)];
+            uint4 out;
+            out.x = e[0] | ((uint32_t)e[1] << 16); out.y = e[2] | ((uint32_t)e[3] << 16);
+            out.z = e[4] | ((uint32_t)e[5] << 16); out.w = e[6] | ((uint32_t)e[7] << 16);
+            int64_t off = col_off + (r0 + r) * v.w;
+            if (!strips) off = map(v, r0 + r, c0 + 8 * q);
+            else if (v.ichunk) {                                            // chunk j of strip g is chunk j * P + g of the buffer
+                const int64_t j = il_shift >= 0 ? off >> il_shift : off / v.ichunk;
+                off = (j * v.nstrips + g) * v.ichunk + (off - j * v.ichunk);
+            }
+            __stcs(reinterpret_cast<uint4*>(dst + off), out);
+        }
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+}
+
+// Any element size and shape: 32 x 32 tiles, one element per access.
+template <typename T>
+__global__ void __launch_bounds__(kTrThreads) repack_transpose_elem_kernel(const T* __restrict__ src, T* __restrict__ dst, MatView v,
+                                                                           int64_t tiles_r, int64_t ntiles) {
+    __shared__ T tile[32][33];
+    const int x = threadIdx.x & 31, y = threadIdx.x >> 5;                   // 8 rows of 32 threads
+    for (int64_t ti = blockIdx.x; ti < ntiles; ti += gridDim.x) {
+        const int64_t tc = ti / tiles_r, tr = ti - tc * tiles_r;
+        const int64_t r0 = tr * 32, c0 = tc * 32;
+        __syncthreads();
+        for (int k = y; k < 32; k += 8)
+            if (c0 + k < v.cols && r0 + x < v.rows) tile[k][x] = src[(c0 + k) * v.rows + r0 + x];
+        __syncthreads();
+        for (int k = y; k < 32; k += 8)
+            if (r0 + k < v.rows && c0 + x < v.cols) dst[map(v, r0 + k, c0 + x)] = tile[x][k];
+    }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -202,8 +307,8 @@ template <typename V>
 static ccl_status launch_vec(const char* src, char* dst, const CopyPlan& p, int sms, cudaStream_t st) {
     int64_t cpr = p.row_bytes / (int64_t)sizeof(V), cps = cpr * p.rows;
     int64_t blocks_needed = (cps + (int64_t)kVecThreads * kVecUnroll - 1) / ((int64_t)kVecThreads * kVecUnroll);
-    int64_t target = ((int64_t)sms * 8 + p.nstrips - 1) / p.nstrips;
-    dim3 grid((unsigned)std::max<int64_t>(1, std::min(blocks_needed, target)), (unsigned)p.nstrips);
+    int64_t target = ((int64_t)sms * 8 + p.nstrips * p.batch - 1) / (p.nstrips * p.batch);
+    dim3 grid((unsigned)std::max<int64_t>(1, std::min(blocks_needed, target)), (unsigned)p.nstrips, (unsigned)p.batch);
     if (cps < (INT64_C(1) << 31))
         repack_vec_kernel<V, uint32_t><<<grid, kVecThreads, 0, st>>>(src, dst, p, (uint32_t)cpr, (uint32_t)cps);
     else
@@ -216,8 +321,8 @@ static ccl_status launch_vec(const char* src, char* dst, const CopyPlan& p, int 
 template <typename V>
 static ccl_status launch_pad(char* dst, const CopyPlan& p, cudaStream_t st) {
     int64_t chunks = p.pad_bytes / (int64_t)sizeof(V);
-    dim3 grid((unsigned)std::max<int64_t>(1, std::min<int64_t>((chunks + 255) / 256, 64)), (unsigned)p.nstrips);
-    zero_pad_kernel<V><<<grid, 256, 0, st>>>(dst, p.pad_g, p.pad_off, chunks);
+    dim3 grid((unsigned)std::max<int64_t>(1, std::min<int64_t>((chunks + 255) / 256, 64)), (unsigned)p.nstrips, (unsigned)p.batch);
+    zero_pad_kernel<V><<<grid, 256, 0, st>>>(dst, p.pad_g, p.pad_off, chunks, p.dst_b);
     count_launch();
     CCL_CUDA_TRY(cudaGetLastError());
     return CCL_OK;
@@ -233,7 +338,7 @@ static ccl_status launch_tma(const char* src, char* dst, const CopyPlan& p, int 
         if (sscanf(f, "%d,%d,%d,%d", &a, &b, &c, &d2) == 4 && a > 0 && a <= kTmaMaxStages && b > 0 && c > 0 && d2 > 0) { t.stages = a; t.stage_bytes = b * 1024; ctas_per_sm = c; max_bx = d2; }
     }
     t.bx = (uint32_t)std::min<uint64_t>((uint64_t)max_bx, dims[0]);
-    t.il_mode = t.il_src = 0; t.il_kr = t.il_s8 = 1;
+    t.il_mode = t.il_src = 0; t.il_kr = t.il_s8 = 1; t.nstrips = (uint32_t)p.nstrips;
     if (p.il_chunk) {
         t.il_src = p.il_dst ? 0 : 1;
         if (p.il_chunk % p.row_bytes == 0) { t.il_mode = 1; t.il_kr = (uint32_t)(p.il_chunk / p.row_bytes); }
@@ -251,51 +356,47 @@ static ccl_status launch_tma(const char* src, char* dst, const CopyPlan& p, int 
     }
     t.tiles_x = (uint32_t)((dims[0] + t.bx - 1) / t.bx);
     t.tiles_y = (uint32_t)((dims[1] + t.by - 1) / t.by);
-    t.ntiles = (uint64_t)t.tiles_x * t.tiles_y * (uint64_t)p.nstrips;
-    // a strip stride is irrelevant (and may be 0) when there is one strip: give the encoder a valid value
+    t.ntiles = (uint64_t)t.tiles_x * t.tiles_y * (uint64_t)p.nstrips * (uint64_t)p.batch;
+    // a strip stride is irrelevant (and may be 0) when there is one strip, like the matrix stride of a batch of one:
+    // give the encoder valid values
     const uint64_t src_g = (uint64_t)(p.nstrips > 1 ? p.src_g : p.src_r * p.rows), dst_g = (uint64_t)(p.nstrips > 1 ? p.dst_g : p.dst_r * p.rows);
-    CUtensorMap sm, dm;
-    ccl_status s;
-    if (!t.il_mode) {
-        uint32_t box[3] = {t.bx, t.by, 1};
-        uint64_t sstr[2] = {(uint64_t)p.src_r, src_g}, dstr[2] = {(uint64_t)p.dst_r, dst_g};
-        s = encode_tmap(&sm, CU_TENSOR_MAP_DATA_TYPE_UINT64, 3, src, dims, sstr, box, CU_TENSOR_MAP_SWIZZLE_NONE);
-        if (s) return s;
-        s = encode_tmap(&dm, CU_TENSOR_MAP_DATA_TYPE_UINT64, 3, dst, dims, dstr, box, CU_TENSOR_MAP_SWIZZLE_NONE);
-        if (s) return s;
-    } else {
-        // plain side: {x, row, strip, 1}; interleaved side: see TmaTiling.  Both boxes are by x bx dense in shared memory.
+    const uint64_t src_b = (uint64_t)(p.batch > 1 ? p.src_b : 16), dst_b = (uint64_t)(p.batch > 1 ? p.dst_b : 16);
+    const int rank = 3 + (t.il_mode ? 1 : 0) + (p.batch > 1 ? 1 : 0);
+    // every map is built with 5 dimensions and encoded with the first `rank` of them (the rest have extent 1)
+    struct MapSpec { uint64_t dims[5], str[4]; uint32_t box[5]; };
+    auto plain_side = [&](uint64_t row_stride, uint64_t g_stride, uint64_t b_stride) {
+        MapSpec m = {{dims[0], dims[1], dims[2], (uint64_t)p.batch, 1}, {row_stride, g_stride, b_stride, 16}, {t.bx, t.by, 1, 1, 1}};
+        return m;
+    };
+    auto il_side = [&](uint64_t b_stride) {
         const uint64_t S = (uint64_t)p.il_chunk, P = (uint64_t)p.il_P, chunks = ((uint64_t)p.rows * p.row_bytes + S - 1) / S;
-        uint64_t pdims[4] = {dims[0], dims[1], dims[2], 1}, idims[4], istr[3];
-        uint32_t pbox[4] = {t.bx, t.by, 1, 1}, ibox[4];
+        MapSpec m;
         if (t.il_mode == 1) {
-            idims[0] = dims[0]; idims[1] = t.il_kr; idims[2] = P; idims[3] = chunks;
-            istr[0] = (uint64_t)p.row_bytes; istr[1] = S; istr[2] = S * P;
-            ibox[0] = t.bx; ibox[1] = by_in; ibox[2] = 1; ibox[3] = by_out;
+            m = {{dims[0], t.il_kr, P, chunks, (uint64_t)p.batch}, {(uint64_t)p.row_bytes, S, S * P, b_stride}, {t.bx, by_in, 1, by_out, 1}};
         } else {
-            const uint64_t m = (uint64_t)p.row_bytes / S;
-            idims[0] = t.il_s8; idims[1] = m; idims[2] = dims[1]; idims[3] = P;
-            istr[0] = S * P; istr[1] = m * S * P; istr[2] = S;
-            ibox[0] = t.bx; ibox[1] = 1; ibox[2] = t.by; ibox[3] = 1;
+            const uint64_t cpr = (uint64_t)p.row_bytes / S;
+            m = {{t.il_s8, cpr, dims[1], P, (uint64_t)p.batch}, {S * P, cpr * S * P, S, b_stride}, {t.bx, 1, t.by, 1, 1}};
         }
-        const bool il_src = t.il_src != 0;
-        uint64_t pstr[3] = {(uint64_t)(il_src ? p.dst_r : p.src_r), il_src ? dst_g : src_g, (il_src ? dst_g : src_g) * dims[2]};
-        s = encode_tmap(&sm, CU_TENSOR_MAP_DATA_TYPE_UINT64, 4, src, il_src ? idims : pdims, il_src ? istr : pstr, il_src ? ibox : pbox, CU_TENSOR_MAP_SWIZZLE_NONE);
-        if (s) return s;
-        s = encode_tmap(&dm, CU_TENSOR_MAP_DATA_TYPE_UINT64, 4, dst, il_src ? pdims : idims, il_src ? pstr : istr, il_src ? pbox : ibox, CU_TENSOR_MAP_SWIZZLE_NONE);
-        if (s) return s;
-    }
+        return m;
+    };
+    const MapSpec ss = t.il_mode && t.il_src ? il_side(src_b) : plain_side((uint64_t)p.src_r, src_g, src_b);
+    const MapSpec ds = t.il_mode && !t.il_src ? il_side(dst_b) : plain_side((uint64_t)p.dst_r, dst_g, dst_b);
+    CUtensorMap sm, dm;
+    ccl_status s = encode_tmap(&sm, CU_TENSOR_MAP_DATA_TYPE_UINT64, rank, src, ss.dims, ss.str, ss.box, CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (s) return s;
+    s = encode_tmap(&dm, CU_TENSOR_MAP_DATA_TYPE_UINT64, rank, dst, ds.dims, ds.str, ds.box, CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (s) return s;
     size_t smem = (size_t)t.stages * t.stage_bytes + 128 + t.stages * sizeof(uint64_t);
-    static size_t attr_set[2] = {0, 0};
-    const int which = t.il_mode ? 1 : 0;
-    if (attr_set[which] < smem) {
-        if (which) CCL_CUDA_TRY(cudaFuncSetAttribute(repack_tma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        else CCL_CUDA_TRY(cudaFuncSetAttribute(repack_tma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        attr_set[which] = smem;
+    static size_t attr_set[3] = {0, 0, 0};
+    const void* fn = rank == 3 ? (const void*)repack_tma_kernel<3> : rank == 4 ? (const void*)repack_tma_kernel<4> : (const void*)repack_tma_kernel<5>;
+    if (attr_set[rank - 3] < smem) {
+        CCL_CUDA_TRY(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        attr_set[rank - 3] = smem;
     }
     unsigned grid = (unsigned)std::min<uint64_t>(t.ntiles, (uint64_t)sms * ctas_per_sm);
-    if (which) repack_tma_kernel<true><<<grid, 32, smem, st>>>(sm, dm, t);
-    else repack_tma_kernel<false><<<grid, 32, smem, st>>>(sm, dm, t);
+    if (rank == 3) repack_tma_kernel<3><<<grid, 32, smem, st>>>(sm, dm, t);
+    else if (rank == 4) repack_tma_kernel<4><<<grid, 32, smem, st>>>(sm, dm, t);
+    else repack_tma_kernel<5><<<grid, 32, smem, st>>>(sm, dm, t);
     count_launch();
     CCL_CUDA_TRY(cudaGetLastError());
     return CCL_OK;
@@ -313,7 +414,30 @@ ccl_status repack_status_take(int* code) {
 
 using namespace ccl;
 
-extern "C" ccl_status ccl_repack(const ccl_mat* m, const void* src_dev, void* dst_dev, int dir, void* cuda_stream) {
+// Where the padding of a CCL destination lies (p->nstrips, rows, row_bytes set): the tail of every aligned strip, or,
+// page-interleaved, the tail of every strip's last chunk.
+static void set_padding(const MatView& v, CopyPlan* p) {
+    const int64_t e = v.e, Bs = p->rows * p->row_bytes;
+    if (v.ichunk) {
+        const int64_t S = v.ichunk * e;
+        p->pad_g = S; p->pad_off = (v.ichunks - 1) * v.nstrips * S + (Bs - (v.ichunks - 1) * S); p->pad_bytes = v.ichunks * S - Bs;
+    } else if (v.split) {
+        p->pad_off = Bs; p->pad_bytes = v.stride * e - Bs; p->pad_g = v.stride * e;
+    }
+}
+
+static ccl_status zero_padding(char* dst, const CopyPlan& p, cudaStream_t st) {
+    if (p.pad_bytes <= 0) return CCL_OK;
+    int64_t pv = pow2_divisor(p.pad_off | p.pad_bytes | p.pad_g | p.dst_b | (int64_t)(reinterpret_cast<uintptr_t>(dst) & 15), 16);
+    if (pv == 16) return launch_pad<uint4>(dst, p, st);
+    if (pv == 8) return launch_pad<uint2>(dst, p, st);
+    if (pv == 4) return launch_pad<unsigned int>(dst, p, st);
+    if (pv == 2) return launch_pad<unsigned short>(dst, p, st);
+    return launch_pad<unsigned char>(dst, p, st);
+}
+
+static ccl_status repack_impl(const ccl_mat* m, int64_t batch, const void* src_dev, int64_t src_b, void* dst_dev, int64_t dst_b, int dir,
+                              void* cuda_stream) {
     MatView v;
     ccl_status s = make_view(m, "ccl_repack", &v);
     if (s) return s;
@@ -322,6 +446,12 @@ extern "C" ccl_status ccl_repack(const ccl_mat* m, const void* src_dev, void* ds
     if (src_dev == dst_dev) return fail(CCL_ERR_INVALID_ARG, "ccl_repack: in-place repack is not supported");
     if ((reinterpret_cast<uintptr_t>(src_dev) % v.e) || (reinterpret_cast<uintptr_t>(dst_dev) % v.e))
         return fail(CCL_ERR_ALIGN, "ccl_repack: buffers must be aligned to elem_bytes");
+    if (batch < 1 || batch > 65535) return fail(CCL_ERR_INVALID_ARG, "ccl_repack_batched: batch must be in [1, 65535]");
+    if (batch > 1) {
+        const int64_t plain = v.rows * v.cols * v.e, packed = buffer_elems(v) * v.e;
+        if (src_b < 0 || dst_b < (dir == 0 ? packed : plain)) return fail(CCL_ERR_INVALID_ARG, "ccl_repack_batched: the outputs of a batch must not overlap (and strides must not be negative)");
+        if (src_b % v.e || dst_b % v.e) return fail(CCL_ERR_ALIGN, "ccl_repack_batched: strides must be multiples of elem_bytes");
+    } else src_b = dst_b = 0;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
     int sms = 0;
     s = sm_count(&sms);
@@ -330,6 +460,7 @@ extern "C" ccl_status ccl_repack(const ccl_mat* m, const void* src_dev, void* ds
     const int64_t e = v.e;
     CopyPlan p;
     std::memset(&p, 0, sizeof(p));
+    p.batch = batch; p.src_b = src_b; p.dst_b = dst_b;
     int64_t rm_g, rm_r, cc_g, cc_r;          // row-major side and CCL side strides (bytes)
     if (v.split == 2) {
         p.nstrips = v.nstrips; p.rows = v.rows; p.row_bytes = v.w * e;
@@ -344,31 +475,26 @@ extern "C" ccl_status ccl_repack(const ccl_mat* m, const void* src_dev, void* ds
     if (p.nstrips > 65535) return fail(CCL_ERR_UNSUPPORTED, "ccl_repack: P > 65535");
     if (dir == 0) { p.src_g = rm_g; p.src_r = rm_r; p.dst_g = cc_g; p.dst_r = cc_r; }
     else          { p.src_g = cc_g; p.src_r = cc_r; p.dst_g = rm_g; p.dst_r = rm_r; }
-    if (dir == 0 && v.split && !v.ichunk) {
-        p.pad_off = p.rows * p.row_bytes; p.pad_bytes = v.stride * e - p.pad_off; p.pad_g = cc_g;
-    }
+    if (dir == 0) set_padding(v, &p);
     if (v.ichunk) {                           // page-interleaved CCL: chunk j of strip g is chunk j*P + g of the buffer
-        const int64_t S = v.ichunk * e, Bs = p.rows * p.row_bytes;
+        const int64_t S = v.ichunk * e;
         p.il_chunk = S; p.il_P = v.nstrips; p.il_dst = dir == 0;
         p.il_shift = -1;
         if ((S & (S - 1)) == 0) { int sh = 0; while ((INT64_C(1) << sh) < S) ++sh; p.il_shift = sh; }
-        if (dir == 0) {                       // the tail of every strip's last chunk is padding
-            p.pad_g = S; p.pad_off = (v.ichunks - 1) * v.nstrips * S + (Bs - (v.ichunks - 1) * S); p.pad_bytes = v.ichunks * S - Bs;
-        }
     }
 
     const char* src = static_cast<const char*>(src_dev);
     char* dst = static_cast<char*>(dst_dev);
     int64_t addr_bits = (int64_t)((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst)) & 15);
-    int64_t vec = pow2_divisor(p.row_bytes | p.src_g | p.src_r | p.dst_g | p.dst_r | p.il_chunk | addr_bits, 16);
+    int64_t vec = pow2_divisor(p.row_bytes | p.src_g | p.src_r | p.dst_g | p.dst_r | p.il_chunk | p.src_b | p.dst_b | addr_bits, 16);
 
     // path choice: TMA when everything is 16-byte aligned and the copy is big enough to be worth a ring
     const char* force = std::getenv("CCL_REPACK_PATH");
     // (page-interleaved side: a chunk must hold whole strip rows, or a strip row whole chunks)
     const bool il_ok = !p.il_chunk || p.il_chunk % p.row_bytes == 0 || p.row_bytes % p.il_chunk == 0;
     bool tma_ok = vec == 16 && il_ok && p.rows < (INT64_C(1) << 31) && p.row_bytes / 8 < (INT64_C(1) << 31) &&
-                  std::max(std::max(p.src_g, p.src_r), std::max(p.dst_g, p.dst_r)) < (INT64_C(1) << 40);
-    bool use_tma = tma_ok && p.nstrips * p.rows * p.row_bytes >= (INT64_C(1) << 20);
+                  std::max(std::max(std::max(p.src_g, p.src_r), std::max(p.dst_g, p.dst_r)), std::max(p.src_b, p.dst_b)) < (INT64_C(1) << 40);
+    bool use_tma = tma_ok && p.batch * p.nstrips * p.rows * p.row_bytes >= (INT64_C(1) << 20);
     if (force && !std::strcmp(force, "vec")) use_tma = false;
     if (force && !std::strcmp(force, "tma") && tma_ok) use_tma = true;
 
@@ -380,14 +506,55 @@ extern "C" ccl_status ccl_repack(const ccl_mat* m, const void* src_dev, void* ds
     else s = launch_vec<unsigned char>(src, dst, p, sms, st);
     if (s) return s;
 
-    if (p.pad_bytes > 0) {
-        int64_t pv = pow2_divisor(p.pad_off | p.pad_bytes | p.pad_g | (int64_t)(reinterpret_cast<uintptr_t>(dst) & 15), 16);
-        if (pv == 16) s = launch_pad<uint4>(dst, p, st);
-        else if (pv == 8) s = launch_pad<uint2>(dst, p, st);
-        else if (pv == 4) s = launch_pad<unsigned int>(dst, p, st);
-        else if (pv == 2) s = launch_pad<unsigned short>(dst, p, st);
-        else s = launch_pad<unsigned char>(dst, p, st);
-        if (s) return s;
-    }
+    s = zero_padding(dst, p, st);
+    if (s) return s;
     return CCL_OK;
+}
+
+extern "C" ccl_status ccl_repack(const ccl_mat* m, const void* src_dev, void* dst_dev, int dir, void* cuda_stream) {
+    return repack_impl(m, 1, src_dev, 0, dst_dev, 0, dir, cuda_stream);
+}
+
+extern "C" ccl_status ccl_repack_batched(const ccl_mat* m, int32_t batch, const void* src_dev, int64_t src_stride_bytes, void* dst_dev,
+                                         int64_t dst_stride_bytes, int dir, void* cuda_stream) {
+    return repack_impl(m, batch, src_dev, src_stride_bytes, dst_dev, dst_stride_bytes, dir, cuda_stream);
+}
+
+extern "C" ccl_status ccl_repack_transpose(const ccl_mat* m, const void* src_dev, void* dst_dev, void* cuda_stream) {
+    MatView v;
+    ccl_status s = make_view(m, "ccl_repack_transpose", &v);
+    if (s) return s;
+    if (!src_dev || !dst_dev) return fail(CCL_ERR_INVALID_ARG, "ccl_repack_transpose: NULL buffer");
+    if (src_dev == dst_dev) return fail(CCL_ERR_INVALID_ARG, "ccl_repack_transpose: in-place repack is not supported");
+    if ((reinterpret_cast<uintptr_t>(src_dev) % v.e) || (reinterpret_cast<uintptr_t>(dst_dev) % v.e))
+        return fail(CCL_ERR_ALIGN, "ccl_repack_transpose: buffers must be aligned to elem_bytes");
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    int sms = 0;
+    s = sm_count(&sms);
+    if (s) return s;
+    CopyPlan p;
+    std::memset(&p, 0, sizeof(p));
+    p.batch = 1; p.nstrips = v.nstrips;
+    if (v.split == 2) { p.rows = v.rows; p.row_bytes = v.w * v.e; }
+    else if (v.split == 1) { p.rows = v.h; p.row_bytes = v.cols * v.e; }
+    else { p.rows = v.rows; p.row_bytes = v.cols * v.e; }
+    if (p.nstrips > 65535) return fail(CCL_ERR_UNSUPPORTED, "ccl_repack_transpose: P > 65535");
+    set_padding(v, &p);
+    char* dst = static_cast<char*>(dst_dev);
+    const bool aligned16 = ((reinterpret_cast<uintptr_t>(src_dev) | reinterpret_cast<uintptr_t>(dst_dev)) & 15) == 0;
+    const bool vec = v.e == 2 && aligned16 && v.rows % 8 == 0 && v.cols % 8 == 0 && v.w % 8 == 0 && v.stride % 8 == 0 && v.ichunk % 8 == 0;
+    const int64_t T = vec ? kTrTile : 32;
+    const int64_t tiles_r = (v.rows + T - 1) / T, tiles_c = (v.cols + T - 1) / T, ntiles = tiles_r * tiles_c;
+    int per_sm = 32, il_shift = -1;                           // short runs of tiles per CTA: 24-32 per SM measured best
+    if (v.ichunk && (v.ichunk & (v.ichunk - 1)) == 0) { il_shift = 0; while ((INT64_C(1) << il_shift) < v.ichunk) ++il_shift; }
+    if (const char* f = std::getenv("CCL_TRANSPOSE_CTAS")) { const int n = std::atoi(f); if (n > 0 && n <= 32) per_sm = n; }
+    const unsigned grid = (unsigned)std::min<int64_t>(ntiles, (int64_t)sms * per_sm);
+    if (vec) repack_transpose_vec_kernel<<<grid, kTrThreads, 0, st>>>(static_cast<const uint16_t*>(src_dev), reinterpret_cast<uint16_t*>(dst), v, tiles_c, ntiles, il_shift);
+    else if (v.e == 1) repack_transpose_elem_kernel<uint8_t><<<grid, kTrThreads, 0, st>>>(static_cast<const uint8_t*>(src_dev), reinterpret_cast<uint8_t*>(dst), v, tiles_r, ntiles);
+    else if (v.e == 2) repack_transpose_elem_kernel<uint16_t><<<grid, kTrThreads, 0, st>>>(static_cast<const uint16_t*>(src_dev), reinterpret_cast<uint16_t*>(dst), v, tiles_r, ntiles);
+    else if (v.e == 4) repack_transpose_elem_kernel<uint32_t><<<grid, kTrThreads, 0, st>>>(static_cast<const uint32_t*>(src_dev), reinterpret_cast<uint32_t*>(dst), v, tiles_r, ntiles);
+    else return fail(CCL_ERR_UNSUPPORTED, "ccl_repack_transpose: elem_bytes must be 1, 2 or 4");
+    count_launch();
+    CCL_CUDA_TRY(cudaGetLastError());
+    return zero_padding(dst, p, st);
 }

@@ -278,6 +278,40 @@ def capacity_and_dtype_sweep(out_dir, quick):
     json.dump(table, open(os.path.join(out_dir, "report_l2_sweep.json"), "w"), indent=1)
 
 
+def paper_sweep(out_dir, quick):
+    """The paper's headline experiment (Sec. 4.2) under this library's finite-L2 model: the six FFN GEMMs (gate/up and
+    down; forward, data gradient, weight gradient) of the Qwen-3-30B-style expert and the Llama-3.1-70B-style layer at
+    4K / 8K / 16K tokens (18 GEMMs per model), P = 4, 4 KB pages, 8 MB / 16-way / 128-byte L2 per chiplet, best output
+    partition and traversal per GEMM; remote traffic of coarse locality-aware placement and of CCL against 4 KB
+    round-robin, as geometric means; run for both execution models (one CTA after the other; waves in lockstep)."""
+    kw = dict(capacity_bytes=8 << 20, line_bytes=128, ways=16, hash=1)
+    policies = (("rr4k", ccl.ROWMAJOR, ccl.PLACE_RR), ("coarse", ccl.ROWMAJOR, ccl.PLACE_BLOCK), ("ccl", ccl.CCL, ccl.PLACE_BLOCK))
+    tokens = (4096,) if quick else (4096, 8192, 16384)
+    gm = lambda xs: math.exp(sum(math.log(x) for x in xs) / len(xs)) if xs else float("nan")
+    out = []
+    for exec_name, exec_kw in (("one CTA after the other", dict(wave_ctas=1, k_slice=0)), ("waves of 76 CTAs, 256 elements of K per step", dict(wave_ctas=76, k_slice=256))):
+        LRU_EXEC.update(exec_kw)
+        for model, H, I in (("qwen", 2048, 768), ("llama", 8192, 28672)):
+            rows = []
+            for T in tokens:
+                for g in synth.qwen_ffn_gemms(T=T, H=H, I=I):
+                    g = dict(g, P=4, name=g["name"].replace("qwen", model) + f"_T{T}")
+                    rem = {tag: sum(traffic_lru_best(g, lay, place, 4096, kw)["remote"]) for tag, lay, place in policies}
+                    rows.append(dict(name=g["name"], M=g["M"], N=g["N"], K=g["K"], remote_bytes=rem))
+                    print(f"  {g['name']:28s} M {g['M']:6d} N {g['N']:6d} K {g['K']:6d}: remote GB rr4k {rem['rr4k'] / 1e9:8.3f} coarse {rem['coarse'] / 1e9:8.3f} "
+                          f"CCL {rem['ccl'] / 1e9:8.3f}", flush=True)
+            pos = [r["remote_bytes"] for r in rows if min(r["remote_bytes"].values()) > 0]
+            fine = [r for r in pos if r["ccl"] < r["coarse"]]
+            summary = dict(exec=exec_name, model=model, gemms=len(rows), ccl_over_rr4k=gm([r["ccl"] / r["rr4k"] for r in pos]),
+                           coarse_over_rr4k=gm([r["coarse"] / r["rr4k"] for r in pos]), coarse_over_ccl=gm([r["coarse"] / r["ccl"] for r in pos]),
+                           fine_optimal=len(fine), max_coarse_over_ccl=max([r["coarse"] / r["ccl"] for r in pos], default=float("nan")))
+            out.append(dict(summary=summary, gemms=rows))
+            print(f"sweep [{exec_name}] {model}: {len(rows)} GEMMs ({len(rows) - len(pos)} with a zero count left out of the means): geometric mean CCL / rr4k "
+                  f"{summary['ccl_over_rr4k']:.3f}, coarse / rr4k {summary['coarse_over_rr4k']:.3f}, coarse / CCL {summary['coarse_over_ccl']:.2f}x "
+                  f"(max {summary['max_coarse_over_ccl']:.1f}x); CCL strictly below coarse on {len(fine)} GEMMs", flush=True)
+    json.dump(out, open(os.path.join(out_dir, "report_paper_sweep.json"), "w"), indent=1)
+
+
 def extras(out_dir, quick):
     """The entry points around the plain GEMM, timed on the shapes they are meant for: the batch of expert GEMMs in one
     launch, the gated activation fused into the gate/up GEMM, and alpha/beta accumulation."""
@@ -340,6 +374,36 @@ def extras(out_dir, quick):
         t_x = timed(lambda: ccl.ccl_gemm_axpby(d, 1.0, 1.0, A, B, Cc), 10)
         rows.append(dict(what="axpby", M=M, N=N, K=K, gemm_ms=t_p, axpby_ms=t_x))
         print(f"extras accumulate {M}x{N}x{K}: C = A*B {t_p * 1e3:8.1f} us | C += A*B {t_x * 1e3:8.1f} us", flush=True)
+    # 4. transposing repack: a weight kept as [N x K] becomes CCL [K x N]; against the plain repack and a strided copy
+    for name, R, Cc in (("llama_down", 28672, 8192), ("llama_gateup", 8192, 57344)) if not quick else (("qwen_x16", 2048, 16 * 1536),):
+        for layout, S in ((ccl.CCL, 0), (ccl.CCL_INTERLEAVED, 4096)):
+            m = ccl.Mat(R, Cc, 2, 4, ccl.PART_COLS, layout, S)
+            src = torch.empty(R * Cc, dtype=torch.int16, device=dev).random_()
+            dst = torch.empty(ccl.ccl_buffer_bytes(m) // 2, dtype=torch.int16, device=dev)
+            xt, y = src.view(Cc, R), torch.empty(R, Cc, dtype=torch.int16, device=dev)
+            t_t = timed(lambda: ccl.ccl_repack_transpose(m, src, dst), 10)
+            t_r = timed(lambda: ccl.ccl_repack(m, src, dst, 0), 10)
+            t_c = timed(lambda: y.copy_(xt.t()), 5)
+            gbs = lambda ms: 2 * R * Cc * 2 / (ms * 1e-3) / 1e9
+            rows.append(dict(what="repack_transpose", name=name, rows=R, cols=Cc, layout=layout, transpose_gbs=gbs(t_t), repack_gbs=gbs(t_r), torch_t_copy_gbs=gbs(t_c)))
+            print(f"extras transposing repack {name} [{Cc}x{R}] -> CCL [{R}x{Cc}] P 4 layout {layout}: {gbs(t_t):7.0f} GB/s | plain repack {gbs(t_r):7.0f} GB/s | "
+                  f"torch copy_(x.t()) {gbs(t_c):7.0f} GB/s", flush=True)
+    # 5. the weights of all experts in one launch
+    for R, Cc in ((2048, 1536), (768, 2048)):
+        E = 128 if not quick else 16
+        m = ccl.Mat(R, Cc, 2, 4, ccl.PART_COLS, ccl.CCL, 4096)
+        nb = ccl.ccl_buffer_bytes(m)
+        src = torch.empty(E * R * Cc, dtype=torch.int16, device=dev).random_()
+        dst = torch.empty(E * nb // 2, dtype=torch.int16, device=dev)
+        t_b = timed(lambda: ccl.ccl_repack_batched(m, E, src, R * Cc * 2, dst, nb, 0), 10)
+
+        def loop():
+            for i in range(E):
+                ccl.ccl_repack(m, src[i * R * Cc:(i + 1) * R * Cc], dst[i * nb // 2:(i + 1) * nb // 2], 0)
+        t_l = timed(loop, 5)
+        gbs = lambda ms: 2 * E * R * Cc * 2 / (ms * 1e-3) / 1e9
+        rows.append(dict(what="repack_batched", experts=E, rows=R, cols=Cc, batched_gbs=gbs(t_b), looped_gbs=gbs(t_l)))
+        print(f"extras repack of {E} expert weights [{R}x{Cc}]: one launch {gbs(t_b):7.0f} GB/s ({t_b * 1e3:7.1f} us) | {E} launches {gbs(t_l):7.0f} GB/s ({t_l * 1e3:7.1f} us)", flush=True)
     json.dump(rows, open(os.path.join(out_dir, "report_extras.json"), "w"), indent=1)
 
 
@@ -352,13 +416,17 @@ def main():
     ap.add_argument("--lru-wave", type=int, default=1, help="finite-L2 model: CTAs of a chiplet in flight together (1: one after the other)")
     ap.add_argument("--lru-kslice", type=int, default=0, help="finite-L2 model: elements of K a wave consumes per lockstep step (0: all of K)")
     ap.add_argument("--l2-sweep", action="store_true", help="remote traffic against L2 capacity and data type under the finite-L2 model (then exit)")
-    ap.add_argument("--extras", action="store_true", help="time the batched, gated-activation and alpha/beta entry points (then exit)")
+    ap.add_argument("--paper-sweep", action="store_true", help="the 2 x 18-GEMM sweep of Sec. 4.2 under the finite-L2 model, both execution models (then exit)")
+    ap.add_argument("--extras", action="store_true", help="time the batched, gated-activation, alpha/beta, transposing- and batched-repack entry points (then exit)")
     ap.add_argument("--only", default=None, help="run only the GEMMs whose name contains this text (e.g. for a profiler capture)")
     args = ap.parse_args()
     assert torch.cuda.is_available(), "report needs a CUDA device"
     pk = peaks()
     os.makedirs(args.out, exist_ok=True)
     LRU_EXEC.update(wave_ctas=args.lru_wave, k_slice=args.lru_kslice)
+    if args.paper_sweep:
+        paper_sweep(args.out, args.quick)
+        return
     if args.extras:
         extras(args.out, args.quick)
         return

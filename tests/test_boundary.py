@@ -114,6 +114,15 @@ def test_repack_rejects_bad_input_before_any_launch():
     assert l.ccl_repack(C.byref(m), C.c_void_p(257), C.c_void_p(512), 0, None) == ccl.ERR_ALIGN
     bad = ccl.Mat(4, 9, 2, 2, 2, 1)
     assert l.ccl_repack(C.byref(bad), C.c_void_p(256), C.c_void_p(512), 0, None) == ccl.ERR_SHAPE
+    # a batch: count in range, outputs that do not overlap, strides in whole elements
+    rb = lambda batch, ss, ds, d=0: l.ccl_repack_batched(C.byref(m), batch, C.c_void_p(256), ss, C.c_void_p(4096), ds, d, None)
+    assert rb(0, 64, 64) == ccl.ERR_INVALID_ARG
+    assert rb(70000, 64, 64) == ccl.ERR_INVALID_ARG
+    assert rb(2, 64, 62) == ccl.ERR_INVALID_ARG                    # 4 x 8 x 2 = 64 bytes per output
+    assert rb(2, -64, 64) == ccl.ERR_INVALID_ARG
+    assert rb(2, 65, 66) == ccl.ERR_ALIGN
+    padded = ccl.Mat(4, 8, 2, 2, 2, 1, 256)                        # strips padded to 256 bytes: 512 bytes per packed matrix
+    assert l.ccl_repack_batched(C.byref(padded), 2, C.c_void_p(256), 64, C.c_void_p(4096), 64, 0, None) == ccl.ERR_INVALID_ARG
 
 
 def gemm_rc(d, a=4096, b=8192, c=16384):

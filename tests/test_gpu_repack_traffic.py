@@ -95,6 +95,106 @@ def test_repack_bit_exact(case, path):
     run_repack(case, path)
 
 
+BATCHED = [
+    (dict(rows=2048, cols=1536, P=4, part=2, layout=1), 5),                # Qwen gate/up weights: rank-4 maps
+    (dict(rows=768, cols=2048, P=4, part=2, layout=1, align=4096), 3),
+    (dict(rows=1001, cols=1024, P=4, part=2, layout=2, align=4096), 3),    # page-interleaved: rank-5 maps
+    (dict(rows=301, cols=7168, P=4, part=2, layout=2, align=512), 2),
+    (dict(rows=33, cols=50, P=5, part=2, layout=1), 4),                    # 4-byte vectors
+    (dict(rows=77, cols=96, P=3, part=2, layout=2, align=48, e=1), 3),
+    (dict(rows=7, cols=24, P=3, part=2, layout=1, align=256), 6),          # padded strips
+]
+
+
+@pytest.mark.parametrize("case,batch", BATCHED)
+@pytest.mark.parametrize("path", ["vec", "tma", None])
+def test_repack_batched_bit_exact(case, batch, path):
+    """Every matrix of the batch equals the oracle's repack of it, the gaps between the outputs stay untouched, and the
+    way back restores the inputs."""
+    mo, ml = mat_pair(**case)
+    npdt, _ = DT[mo.elem_bytes]
+    e = mo.elem_bytes
+    rng = np.random.default_rng(11)
+    xs = rng.integers(1, np.iinfo(npdt).max, size=(batch, mo.rows, mo.cols), dtype=npdt)
+    want = [orc.repack(mo, xs[i], 0) for i in range(batch)]
+    plain, packed, gap = mo.rows * mo.cols, want[0].size, 4096 // e     # elements; 4 KB between consecutive outputs
+    old = os.environ.pop("CCL_REPACK_PATH", None)
+    if path:
+        os.environ["CCL_REPACK_PATH"] = path
+    try:
+        src = dev(np.ascontiguousarray(xs).reshape(-1))
+        dst = dev(np.full(batch * (packed + gap), 0x5A, dtype=npdt))
+        ccl.ccl_repack_batched(ml, batch, src, plain * e, dst, (packed + gap) * e, 0)
+        got = host(dst, npdt).reshape(batch, packed + gap)
+        for i in range(batch):
+            np.testing.assert_array_equal(got[i, :packed], want[i], err_msg=f"matrix {i}")
+        assert (got[:, packed:] == 0x5A).all(), "wrote between or past the outputs"
+        back = dev(np.full(batch * (plain + gap), 0x5A, dtype=npdt))
+        ccl.ccl_repack_batched(ml, batch, dst, (packed + gap) * e, back, (plain + gap) * e, 1)
+        hb = host(back, npdt).reshape(batch, plain + gap)
+        np.testing.assert_array_equal(hb[:, :plain].reshape(batch, mo.rows, mo.cols), xs)
+        assert (hb[:, plain:] == 0x5A).all(), "wrote between or past the outputs"
+        # one source repeated (stride 0)
+        ccl.ccl_repack_batched(ml, batch, src, 0, dst, (packed + gap) * e, 0)
+        got = host(dst, npdt).reshape(batch, packed + gap)
+        for i in range(batch):
+            np.testing.assert_array_equal(got[i, :packed], want[0])
+        assert ccl.ccl_gemm_status()[0] == ccl.OK
+    finally:
+        os.environ.pop("CCL_REPACK_PATH", None)
+        if old is not None:
+            os.environ["CCL_REPACK_PATH"] = old
+
+
+TRANSPOSED = [
+    dict(rows=4, cols=8, P=2, part=2, layout=1),                           # the Fig. 4(a) example
+    dict(rows=2048, cols=1536, P=4, part=2, layout=1),                     # Qwen gate/up weight kept as [1536 x 2048]
+    dict(rows=768, cols=2048, P=4, part=2, layout=1, align=4096),
+    dict(rows=136, cols=384, P=4, part=2, layout=1),                       # w = 96: a 64-wide tile straddles two strips
+    dict(rows=200, cols=1000, P=5, part=2, layout=1),                      # ragged tiles in both directions
+    dict(rows=768, cols=2048, P=4, part=1, layout=1, align=4096),          # strips of rows
+    dict(rows=1000, cols=1024, P=4, part=2, layout=2, align=4096),         # page-interleaved
+    dict(rows=130, cols=384, P=4, part=2, layout=1),                       # rows not a multiple of 8: element path
+    dict(rows=33, cols=50, P=5, part=2, layout=1),
+    dict(rows=77, cols=96, P=3, part=2, layout=1, e=1),
+    dict(rows=77, cols=96, P=3, part=2, layout=1, e=4, align=256),
+    dict(rows=300, cols=8192, P=2, part=2, layout=0),                      # row-major descriptor: a plain transpose
+]
+
+
+@pytest.mark.parametrize("case", TRANSPOSED)
+def test_repack_transpose_bit_exact(case):
+    mo, ml = mat_pair(**case)
+    npdt, _ = DT[mo.elem_bytes]
+    xt = np.random.default_rng(12).integers(1, np.iinfo(npdt).max, size=(mo.cols, mo.rows), dtype=npdt)
+    want = orc.repack_transposed(mo, xt)
+    guard = 4096
+    dst = dev(np.full(want.size + guard, 0x5A, dtype=npdt))
+    ccl.ccl_repack_transpose(ml, dev(xt), dst)
+    got = host(dst, npdt)
+    np.testing.assert_array_equal(got[:want.size], want)
+    assert (got[want.size:] == 0x5A).all(), "wrote past the end of its output"
+    back = dev(np.zeros(mo.rows * mo.cols, dtype=npdt))                # and the plain way back gives the transpose of the source
+    ccl.ccl_repack(ml, dst, back, 1)
+    np.testing.assert_array_equal(host(back, npdt).reshape(mo.rows, mo.cols), xt.T)
+
+
+def test_repack_transpose_llama_down_weight_full_size():
+    # the Llama down projection kept as [8192 x 28672] (470 MB), wanted as CCL [28672 x 8192] over 4 chiplets
+    R, Cc, P = 28672, 8192, 4
+    mo, ml = mat_pair(R, Cc, 2, P, 2, 1)
+    xt = np.random.default_rng(4).integers(0, 65535, size=(Cc, R), dtype=np.uint16)
+    dst = torch.empty(R * Cc, dtype=torch.int16, device="cuda")
+    ccl.ccl_repack_transpose(ml, dev(xt), dst)
+    got = host(dst, np.uint16)
+    w = Cc // P
+    for g in range(P):                                                 # strip g = rows g*w .. of the stored transpose, transposed
+        np.testing.assert_array_equal(got[g * R * w:(g + 1) * R * w].reshape(R, w), xt[g * w:(g + 1) * w].T)
+    for lin in np.random.default_rng(5).integers(0, R * Cc, size=2000):
+        r, c = divmod(int(lin), Cc)
+        assert got[orc.map_offset(mo, r, c)] == xt[c, r]
+
+
 def test_repack_unaligned_base_pointer():
     mo, ml = mat_pair(64, 256, 2, 4, 2, 1)
     x = np.random.default_rng(1).integers(0, 65535, size=(64, 256), dtype=np.uint16)
