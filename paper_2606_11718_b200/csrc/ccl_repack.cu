@@ -198,69 +198,79 @@ __global__ void __launch_bounds__(32) repack_tma_kernel(const __grid_constant__ 
 // [N x K] that a GEMM wants as CCL [K x N]); element (r, c) of the output comes from src[c * rows + r].
 // ------------------------------------------------------------------------------------------
 constexpr int kTrTile = 64, kTrThreads = 256, kTrStages = 4;
+#ifndef CCL_TR_MIN_CTAS
+#define CCL_TR_MIN_CTAS 5
+#endif
+constexpr int kTrMinCtas = CCL_TR_MIN_CTAS;
 
 // 2-byte elements, everything a multiple of 8 elements: 64 x 64 tiles through 8 KB of shared memory.  A tile is read
 // as 16-byte pieces of source rows (8 consecutive r at one c) and written as 16-byte pieces of output rows (8
 // consecutive c at one r).  Shared memory holds the tile as [c][r] with the 16-byte granule index XORed with c / 8,
 // which makes both the 16-byte stores of the first phase and the 2-byte gathers of the second free of bank conflicts.
-__global__ void __launch_bounds__(kTrThreads) repack_transpose_vec_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, MatView v,
-                                                                          int64_t tiles_c, int64_t ntiles, int il_shift) {
+__global__ void __launch_bounds__(kTrThreads, kTrMinCtas) repack_transpose_vec_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, MatView v,
+                                                                          uint32_t tiles_c, uint32_t ntiles, int il_shift) {
     __shared__ __align__(16) uint16_t tile[kTrStages][kTrTile * kTrTile];
-    const int t = threadIdx.x, q = t & 7, o = t >> 3;                       // q: 16-byte piece of a 128-byte row, o: 0..31
+    const uint32_t t = threadIdx.x, q = t & 7, o = t >> 3;                  // q: 16-byte piece of a 128-byte row, o: 0..31
+    const uint32_t rows = (uint32_t)v.rows, cols = (uint32_t)v.cols, w = (uint32_t)v.w;
     // A CTA takes a contiguous run of tiles, c fastest: it fills 64 output rows from left to right (its 128-byte
     // pieces of a row follow each other in time and leave L2 as whole rows), while the CTAs next to it read the
     // neighbouring pieces of the same source rows.
-    const int64_t first = ntiles * blockIdx.x / gridDim.x, last = ntiles * (blockIdx.x + 1) / gridDim.x;
+    const uint32_t first = (uint32_t)((uint64_t)ntiles * blockIdx.x / gridDim.x), last = (uint32_t)((uint64_t)ntiles * (blockIdx.x + 1) / gridDim.x);
     // source tiles arrive by 16-byte asynchronous copies straight into their (swizzled) place: kTrStages - 1 tiles
     // of reads stay in flight per CTA without holding registers
-    auto load_tile = [&](int stage, int64_t ti) {                           // source row c0 + c, elements r0 + 8q .. + 8
-        const int64_t tr = ti / tiles_c, tc = ti - tr * tiles_c;
-        const int64_t r0 = tr * kTrTile, c0 = tc * kTrTile;
+    uint32_t ltr = first / tiles_c, ltc = first - ltr * tiles_c;            // the next tile to load
+    auto load_next = [&](uint32_t stage) {                                  // source row c0 + c, elements r0 + 8q .. + 8
+        const uint32_t r = ltr * kTrTile + 8 * q;
 #pragma unroll
         for (int k = 0; k < 2; ++k) {
-            const int c = o + 32 * k;
-            const bool in = c0 + c < v.cols && r0 + 8 * q < v.rows;        // outside: zero-filled (source size 0)
-            const uint16_t* g = in ? src + (c0 + c) * v.rows + r0 + 8 * q : src;
-            const uint32_t sm = smem_u32(&tile[stage][c * kTrTile + ((q ^ ((c >> 3) & 7)) << 3)]);
+            const uint32_t cl = o + 32 * k, c = ltc * kTrTile + cl;
+            const bool in = c < cols && r < rows;                           // outside: zero-filled (source size 0)
+            const uint16_t* g = in ? src + (size_t)c * rows + r : src;
+            const uint32_t sm = smem_u32(&tile[stage][cl * kTrTile + ((q ^ ((cl >> 3) & 7)) << 3)]);
             asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(sm), "l"(g), "r"(in ? 16 : 0) : "memory");
         }
+        if (++ltc == tiles_c) { ltc = 0; ++ltr; }
     };
 #pragma unroll
-    for (int d = 0; d < kTrStages - 1; ++d) {
-        if (first + d < last) load_tile(d, first + d);
+    for (uint32_t d = 0; d < kTrStages - 1; ++d) {
+        if (first + d < last) load_next(d);
         asm volatile("cp.async.commit_group;" ::: "memory");
     }
-    for (int64_t ti = first; ti < last; ++ti) {
-        const int stage = (int)((ti - first) % kTrStages);
-        const int64_t tr = ti / tiles_c, tc = ti - tr * tiles_c;
-        const int64_t r0 = tr * kTrTile, c0 = tc * kTrTile;
+    uint32_t tr = first / tiles_c, tc = first - tr * tiles_c, stage = 0;
+    for (uint32_t ti = first; ti < last; ++ti) {
         asm volatile("cp.async.wait_group %0;" ::"n"(kTrStages - 2) : "memory");
         __syncthreads();                                                    // tile ti has landed; tile ti - 1 has been read out
-        if (ti + kTrStages - 1 < last) load_tile((int)((ti - first + kTrStages - 1) % kTrStages), ti + kTrStages - 1);
+        if (ti + kTrStages - 1 < last) load_next(stage == 0 ? kTrStages - 1 : stage - 1);
         asm volatile("cp.async.commit_group;" ::: "memory");
-        const uint16_t* tl = tile[stage];
-        // packed strips of columns (Eq. 3): one division per thread and tile, rows are w apart
-        const bool strips = v.split == 2;
-        int64_t col_off = 0, g = 0;
-        if (strips) { const int64_t c = c0 + 8 * q; g = c / v.w; col_off = c - g * v.w; if (!v.ichunk) col_off += g * v.stride; }
+        // This thread writes 16-byte pieces (columns c .. c + 8) of the output rows r and r + 1: one 32-bit word of
+        // shared memory holds both rows' elements of a column.
+        const uint32_t c = tc * kTrTile + 8 * q, rl = 2 * o, r = tr * kTrTile + rl;
+        if (c < cols && r < rows) {
+            const uint32_t* tw = reinterpret_cast<const uint32_t*>(tile[stage]);
+            uint32_t wd[8];
 #pragma unroll
-        for (int k = 0; k < 2; ++k) {                                       // output row r0 + r, columns c0 + 8q .. + 8
-            const int r = o + 32 * k;
-            if (r0 + r >= v.rows || c0 + 8 * q >= v.cols) continue;
-            uint16_t e[8];
-#pragma unroll
-            for (int j = 0; j < 8; ++j) e[j] = tl[(8 * q + j) * kTrTile + ((((r >> 3) ^ q) & 7) << 3) + (r & 7)];
-            uint4 out;
-            out.x = e[0] | ((uint32_t)e[1] << 16); out.y = e[2] | ((uint32_t)e[3] << 16);
-            out.z = e[4] | ((uint32_t)e[5] << 16); out.w = e[6] | ((uint32_t)e[7] << 16);
-            int64_t off = col_off + (r0 + r) * v.w;
-            if (!strips) off = map(v, r0 + r, c0 + 8 * q);
-            else if (v.ichunk) {                                            // chunk j of strip g is chunk j * P + g of the buffer
-                const int64_t j = il_shift >= 0 ? off >> il_shift : off / v.ichunk;
-                off = (j * v.nstrips + g) * v.ichunk + (off - j * v.ichunk);
-            }
-            __stcs(reinterpret_cast<uint4*>(dst + off), out);
+            for (int j = 0; j < 8; ++j) wd[j] = tw[((8 * q + j) * kTrTile + ((((rl >> 3) ^ q) & 7) << 3) + (rl & 7)) >> 1];
+            uint4 lo, hi;
+            lo.x = __byte_perm(wd[0], wd[1], 0x5410); hi.x = __byte_perm(wd[0], wd[1], 0x7632);
+            lo.y = __byte_perm(wd[2], wd[3], 0x5410); hi.y = __byte_perm(wd[2], wd[3], 0x7632);
+            lo.z = __byte_perm(wd[4], wd[5], 0x5410); hi.z = __byte_perm(wd[4], wd[5], 0x7632);
+            lo.w = __byte_perm(wd[6], wd[7], 0x5410); hi.w = __byte_perm(wd[6], wd[7], 0x7632);
+            // offset of (r, c): packed strips of columns are Eq. 3 with one 32-bit division; rows are w apart
+            int64_t off0, off1;
+            if (v.split == 2) {
+                const uint32_t g = c / w, cp = c - g * w;
+                off0 = (int64_t)r * w + cp; off1 = off0 + w;
+                if (v.ichunk) {                                             // chunk j of strip g is chunk j * P + g of the buffer
+                    const int64_t j0 = il_shift >= 0 ? off0 >> il_shift : off0 / v.ichunk, j1 = il_shift >= 0 ? off1 >> il_shift : off1 / v.ichunk;
+                    off0 = (j0 * v.nstrips + g) * v.ichunk + (off0 - j0 * v.ichunk);
+                    off1 = (j1 * v.nstrips + g) * v.ichunk + (off1 - j1 * v.ichunk);
+                } else { off0 += g * v.stride; off1 += g * v.stride; }
+            } else { off0 = map(v, r, c); off1 = r + 1 < rows ? map(v, r + 1, c) : 0; }
+            __stcs(reinterpret_cast<uint4*>(dst + off0), lo);
+            if (r + 1 < rows) __stcs(reinterpret_cast<uint4*>(dst + off1), hi);
         }
+        if (++tc == tiles_c) { tc = 0; ++tr; }
+        if (++stage == kTrStages) stage = 0;
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
 }
@@ -542,14 +552,24 @@ extern "C" ccl_status ccl_repack_transpose(const ccl_mat* m, const void* src_dev
     set_padding(v, &p);
     char* dst = static_cast<char*>(dst_dev);
     const bool aligned16 = ((reinterpret_cast<uintptr_t>(src_dev) | reinterpret_cast<uintptr_t>(dst_dev)) & 15) == 0;
-    const bool vec = v.e == 2 && aligned16 && v.rows % 8 == 0 && v.cols % 8 == 0 && v.w % 8 == 0 && v.stride % 8 == 0 && v.ichunk % 8 == 0;
+    const bool vec = v.e == 2 && aligned16 && v.rows % 8 == 0 && v.cols % 8 == 0 && v.w % 8 == 0 && v.stride % 8 == 0 && v.ichunk % 8 == 0 &&
+                     v.rows < (INT64_C(1) << 31) && v.cols < (INT64_C(1) << 31) && ((v.rows + 63) / 64) * ((v.cols + 63) / 64) < (INT64_C(1) << 31);
     const int64_t T = vec ? kTrTile : 32;
     const int64_t tiles_r = (v.rows + T - 1) / T, tiles_c = (v.cols + T - 1) / T, ntiles = tiles_r * tiles_c;
-    int per_sm = 32, il_shift = -1;                           // short runs of tiles per CTA: 24-32 per SM measured best
+    // a CTA takes a short run of tiles, all of whose reads it issues at once (the ring holds kTrStages - 1).  Measured
+    // on the Llama weights: runs of 1: 4.1-4.5 TB/s, 2: 5.6-6.0, 3: 5.9-6.2, 4: 5.9-6.15, 6: 5.9, 24: 5.6
+    int64_t run = kTrStages - 1;
+    int il_shift = -1;
     if (v.ichunk && (v.ichunk & (v.ichunk - 1)) == 0) { il_shift = 0; while ((INT64_C(1) << il_shift) < v.ichunk) ++il_shift; }
-    if (const char* f = std::getenv("CCL_TRANSPOSE_CTAS")) { const int n = std::atoi(f); if (n > 0 && n <= 32) per_sm = n; }
-    const unsigned grid = (unsigned)std::min<int64_t>(ntiles, (int64_t)sms * per_sm);
-    if (vec) repack_transpose_vec_kernel<<<grid, kTrThreads, 0, st>>>(static_cast<const uint16_t*>(src_dev), reinterpret_cast<uint16_t*>(dst), v, tiles_c, ntiles, il_shift);
+    if (const char* f = std::getenv("CCL_TRANSPOSE_RUN")) { const int n = std::atoi(f); if (n > 0) run = n; }
+    (void)sms;
+    const unsigned grid = (unsigned)std::min<int64_t>((ntiles + run - 1) / run, INT64_C(1) << 30);
+    static bool carveout_set = false;
+    if (vec && !carveout_set) {                               // room for as many 32 KB rings per SM as registers allow
+        CCL_CUDA_TRY(cudaFuncSetAttribute(repack_transpose_vec_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100));
+        carveout_set = true;
+    }
+    if (vec) repack_transpose_vec_kernel<<<grid, kTrThreads, 0, st>>>(static_cast<const uint16_t*>(src_dev), reinterpret_cast<uint16_t*>(dst), v, (uint32_t)tiles_c, (uint32_t)ntiles, il_shift);
     else if (v.e == 1) repack_transpose_elem_kernel<uint8_t><<<grid, kTrThreads, 0, st>>>(static_cast<const uint8_t*>(src_dev), reinterpret_cast<uint8_t*>(dst), v, tiles_r, ntiles);
     else if (v.e == 2) repack_transpose_elem_kernel<uint16_t><<<grid, kTrThreads, 0, st>>>(static_cast<const uint16_t*>(src_dev), reinterpret_cast<uint16_t*>(dst), v, tiles_r, ntiles);
     else if (v.e == 4) repack_transpose_elem_kernel<uint32_t><<<grid, kTrThreads, 0, st>>>(static_cast<const uint32_t*>(src_dev), reinterpret_cast<uint32_t*>(dst), v, tiles_r, ntiles);

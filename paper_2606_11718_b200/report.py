@@ -312,10 +312,11 @@ def paper_sweep(out_dir, quick):
     json.dump(out, open(os.path.join(out_dir, "report_paper_sweep.json"), "w"), indent=1)
 
 
-def extras(out_dir, quick):
+def extras(out_dir, quick, only=None):
     """The entry points around the plain GEMM, timed on the shapes they are meant for: the batch of expert GEMMs in one
     launch, the gated activation fused into the gate/up GEMM, and alpha/beta accumulation."""
     dev, rows = "cuda", []
+    want = lambda section: only is None or only in section       # --only batched | swiglu | axpby | transpose | experts
 
     def desc(M, N, K, P, bt=0, c_cols=None):
         d = ccl.GemmDesc()
@@ -330,7 +331,7 @@ def extras(out_dir, quick):
         return torch.empty(n * ccl.ccl_buffer_bytes(m) // 2, dtype=torch.bfloat16, device=dev).normal_(0, 0.05)
 
     # 1. the experts of an MoE layer: one launch against one launch per expert and against torch.bmm
-    for E, M, N, K, bt in ((128, 256, 768, 2048, 1), (128, 256, 2048, 768, 0)) if not quick else ((32, 256, 768, 2048, 1),):
+    for E, M, N, K, bt in (((128, 256, 768, 2048, 1), (128, 256, 2048, 768, 0)) if not quick else ((32, 256, 768, 2048, 1),)) if want("batched_gemm") else ():
         d = desc(M, N, K, 4, bt)
         A, B, Cb = buf(d.A, E), buf(d.B, E), buf(d.C, E)
         sa, sb, sc = (ccl.ccl_buffer_bytes(m) for m in (d.A, d.B, d.C))
@@ -354,7 +355,7 @@ def extras(out_dir, quick):
         print(f"extras batched {E} x {M}x{N}x{K}: one launch {t_b * 1e3:8.1f} us ({fl / t_b / 1e9:6.0f} TFLOP/s) | {E} launches {t_l * 1e3:8.1f} us | "
               f"torch.bmm {t_t * 1e3:8.1f} us", flush=True)
     # 2. gate/up GEMM with the gated activation in the epilogue against GEMM + elementwise kernel
-    for M, N, K in ((8192, 57344, 8192), (16384, 1536, 2048)) if not quick else ((1024, 57344, 8192),):
+    for M, N, K in (((8192, 57344, 8192), (16384, 1536, 2048)) if not quick else ((1024, 57344, 8192),)) if want("swiglu") else ():
         d0, d1 = desc(M, N, K, 4), desc(M, N, K, 4, c_cols=N // 2)
         A, B, C0, C1 = buf(d0.A), buf(d0.B), buf(d0.C), buf(d1.C)
         reps = 5 if M * N * K > 1e11 else 50
@@ -367,7 +368,7 @@ def extras(out_dir, quick):
         print(f"extras gate/up {M}x{N}x{K}: GEMM {t_g * 1e3:8.1f} us + silu*mul kernel {t_a * 1e3:8.1f} us = {(t_g + t_a) * 1e3:8.1f} us | "
               f"fused {t_f * 1e3:8.1f} us ({2.0 * M * N * K / t_f / 1e9:6.0f} TFLOP/s)", flush=True)
     # 3. alpha / beta: what reading C in the epilogue costs
-    for M, N, K in ((8192, 8192, 8192),) if not quick else ((2048, 8192, 2048),):
+    for M, N, K in (((8192, 8192, 8192),) if not quick else ((2048, 8192, 2048),)) if want("axpby") else ():
         d = desc(M, N, K, 4)
         A, B, Cc = buf(d.A), buf(d.B), buf(d.C)
         t_p = timed(lambda: ccl.ccl_gemm(d, A, B, Cc), 10)
@@ -375,7 +376,7 @@ def extras(out_dir, quick):
         rows.append(dict(what="axpby", M=M, N=N, K=K, gemm_ms=t_p, axpby_ms=t_x))
         print(f"extras accumulate {M}x{N}x{K}: C = A*B {t_p * 1e3:8.1f} us | C += A*B {t_x * 1e3:8.1f} us", flush=True)
     # 4. transposing repack: a weight kept as [N x K] becomes CCL [K x N]; against the plain repack and a strided copy
-    for name, R, Cc in (("llama_down", 28672, 8192), ("llama_gateup", 8192, 57344)) if not quick else (("qwen_x16", 2048, 16 * 1536),):
+    for name, R, Cc in ((("llama_down", 28672, 8192), ("llama_gateup", 8192, 57344)) if not quick else (("qwen_x16", 4096, 16 * 1536),)) if want("transpose") else ():
         for layout, S in ((ccl.CCL, 0), (ccl.CCL_INTERLEAVED, 4096)):
             m = ccl.Mat(R, Cc, 2, 4, ccl.PART_COLS, layout, S)
             src = torch.empty(R * Cc, dtype=torch.int16, device=dev).random_()
@@ -389,7 +390,7 @@ def extras(out_dir, quick):
             print(f"extras transposing repack {name} [{Cc}x{R}] -> CCL [{R}x{Cc}] P 4 layout {layout}: {gbs(t_t):7.0f} GB/s | plain repack {gbs(t_r):7.0f} GB/s | "
                   f"torch copy_(x.t()) {gbs(t_c):7.0f} GB/s", flush=True)
     # 5. the weights of all experts in one launch
-    for R, Cc in ((2048, 1536), (768, 2048)):
+    for R, Cc in (((2048, 1536), (768, 2048))) if want("experts_repack") else ():
         E = 128 if not quick else 16
         m = ccl.Mat(R, Cc, 2, 4, ccl.PART_COLS, ccl.CCL, 4096)
         nb = ccl.ccl_buffer_bytes(m)
@@ -428,7 +429,7 @@ def main():
         paper_sweep(args.out, args.quick)
         return
     if args.extras:
-        extras(args.out, args.quick)
+        extras(args.out, args.quick, args.only)
         return
     if args.l2_sweep:
         capacity_and_dtype_sweep(args.out, args.quick)
