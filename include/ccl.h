@@ -164,6 +164,23 @@ ccl_status ccl_gemm_workspace(const ccl_gemm_desc* d, size_t* bytes);
 ccl_status ccl_gemm(const ccl_gemm_desc* d, const void* A_dev, const void* B_dev, void* C_dev, void* ws_dev,
                     size_t ws_bytes, void* cuda_stream);
 /*
+ * A RAGGED batch (the experts of an MoE layer with their routed token counts, Sec. 4.1): `groups` problems share N and
+ * K; problem e multiplies rows [row_offsets[e], row_offsets[e+1]) of A [M x K] by its own B (problem e's buffer at
+ * B_dev + e * b_stride_bytes, in the layout d->B describes; stride 0 = one shared B) into the same rows of C [M x N].
+ * d->M is the total row count of A and C; rows no problem owns are left untouched.
+ *   row_offsets_dev  int32[groups + 1] on the DEVICE, non-decreasing, within [0, M]; read by the kernel, so the
+ *                    counts can come straight from a router kernel and the call can sit in a CUDA graph.
+ *   max_rows         host-known upper bound of the rows of any one problem (1 <= max_rows <= M); the tile grid
+ *                    is laid out for it and tiles past a problem's last row cost one loop iteration.
+ * A row-major [M x K] (a_trans = 0), not split along M; C row-major or CCL split along N (out_part != CCL_PART_ROWS);
+ * B as for ccl_gemm.  Never split along K: no workspace.  A problem whose offsets leave [0, M] or that has more rows
+ * than max_rows is not computed and ccl_gemm_status() then returns CCL_ERR_SHAPE (detail 5).
+ * Errors: as ccl_gemm; CCL_ERR_UNSUPPORTED for a_trans or operands split along M.
+ */
+ccl_status ccl_gemm_grouped(const ccl_gemm_desc* d, int32_t groups, int64_t max_rows, const int32_t* row_offsets_dev,
+                            const void* A_dev, const void* B_dev, int64_t b_stride_bytes, void* C_dev, void* cuda_stream);
+
+/*
  * The BLAS form (Sec. 2.2: "the extension to alpha*A*B + beta*C is straightforward, since the scalars do not affect
  * placement and the C read shares the same partitioning as the output write"):
  *   C <- bf16( alpha * (A*B) + beta * C ),  fp32 arithmetic on the fp32 accumulator, one rounding.

@@ -44,6 +44,7 @@ constexpr int kEpiWarps = CCL_EPI_WARPS;        // 4, or 8: two warps per TMEM l
 constexpr int kGemmThreads = 64 + 32 * kEpiWarps;
 constexpr int kTmemCols = 512;
 constexpr uint32_t kSmemBudget = 192 * 1024;    // ring of operand stages
+constexpr int64_t kRaggedDense = 4096;         // problems of a ragged batch whose tile prefix is kept in shared memory
 constexpr uint32_t kEpiBytes = 4 * 2 * 32 * 128; // epilogue staging: per warp two buffers of 32 rows x 128 B
 
 __device__ int g_gemm_status = 0;
@@ -121,6 +122,11 @@ struct GemmParams {
     int32_t axpby;
     float alpha, beta;
     int64_t c_batch_stride;         // elements between the C buffers of consecutive problems
+    // ragged batch (ccl_gemm_grouped): problem e owns rows [m_offs[e], m_offs[e + 1]) of A and C; the tile grid of a
+    // problem is laid out for Wm rows (the caller's bound) and tiles past a problem's last row are skipped
+    const int32_t* m_offs;
+    int32_t rag_dense;              // 1: the CTA builds a prefix of the problems' tile counts and walks only real tiles
+    FastDiv fd_tiles_n;
     OpMap a, b;
     int32_t a_mn, b_mn;             // 1 = MN-major operand tile in shared memory
     OpMap c;                        // C addressed through its own map as well (TMA tile stores)
@@ -271,7 +277,7 @@ __device__ __forceinline__ int64_t c_offset(const GemmParams& p, int64_t m, int6
     return (int64_t)g * p.c_stride + (int64_t)rr * p.c_row + xx;
 }
 
-struct TileCoord { int m0, m1, n0, n1, split, e; };   // e: problem of the batch
+struct TileCoord { int m0, m1, n0, n1, split, e; bool skip; };   // e: problem of the batch; skip: an empty tile of a ragged batch
 
 // Tiles of this CTA (pair).  The schedulable units (CTAs, or CTA pairs) serve `groups` strip ranges
 // (chiplet-grouped raster): group g owns the tiles of strip range g and walks them in panels of
@@ -287,13 +293,31 @@ struct Scheduler {
     const GemmParams& p;
     int gm, gn;                     // tile grid of one group
     int unit, units, upg, floaters, my_g, idx, bm, bn, rounds, pool_per_group;
-    __device__ Scheduler(const GemmParams& p_, int unit_, int bm_, int bn_) : p(p_), unit(unit_), bm(bm_), bn(bn_) {
+    const int* rag;                 // ragged batch, dense walk: rag[e] = m-tiles of the problems before e (shared memory)
+    __device__ Scheduler(const GemmParams& p_, int unit_, int bm_, int bn_, const int* rag_) : p(p_), unit(unit_), bm(bm_), bn(bn_), rag(rag_) {
         gm = p.sch_gm; gn = p.sch_gn; units = p.sch_units; upg = p.sch_upg; floaters = p.sch_floaters;
         rounds = p.sch_rounds; pool_per_group = p.sch_pool_per_group;
         my_g = unit < upg * p.groups ? p.fd_upg.div(unit) : -1;  // -1: floater
         idx = my_g >= 0 ? unit - my_g * upg : unit - upg * p.groups;
     }
+    // Ragged batch: tile q of the walk (n fastest, then the m-tiles of problem 0, 1, ...) by a search in the prefix.
+    __device__ bool get_ragged(int it, TileCoord& t) const {
+        const int E = p.batch, q = unit + it * units;
+        if (q >= rag[E] * p.tiles_n) return false;
+        int mt, tn;
+        p.fd_tiles_n.divmod(q, mt, tn);
+        int lo = 0, hi = E;                              // the last problem whose prefix is <= mt (empty problems share a prefix)
+        while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (rag[mid] <= mt) lo = mid; else hi = mid; }
+        const int o0 = __ldg(p.m_offs + lo), o1 = __ldg(p.m_offs + lo + 1);
+        int sn, jn;
+        p.fd_tps_n.divmod(tn, sn, jn);
+        t.e = lo; t.split = 0; t.skip = false;
+        t.m0 = o0 + (mt - rag[lo]) * bm; t.m1 = min(t.m0 + bm, o1);
+        t.n0 = sn * p.Wn + jn * bn; t.n1 = min(t.n0 + bn, (sn + 1) * p.Wn);
+        return true;
+    }
     __device__ bool get(int it, TileCoord& t) const {
+        if (rag) return get_ragged(it, t);
         int g, i;
         if (it < rounds && my_g >= 0) { g = my_g; i = idx + it * upg; }
         else {
@@ -321,6 +345,14 @@ struct Scheduler {
         p.fd_tps_n.divmod(tn, sn, jn);
         t.m0 = sm * p.Wm + jm * bm; t.m1 = min(t.m0 + bm, (sm + 1) * p.Wm);
         t.n0 = sn * p.Wn + jn * bn; t.n1 = min(t.n0 + bn, (sn + 1) * p.Wn);
+        t.skip = false;
+        if (p.m_offs) {                                  // rows of this problem inside the concatenated A and C
+            const int o0 = __ldg(p.m_offs + t.e), o1 = __ldg(p.m_offs + t.e + 1);
+            const bool bad = o0 < 0 || o1 > p.M || o1 - o0 > p.Wm;   // outside A / C, or more rows than the caller's bound:
+            if (bad && t.m0 == 0 && t.n0 == 0) atomicExch(&g_gemm_status, 5);   // reported, and the problem is left out
+            t.skip = bad || t.m0 >= o1 - o0;
+            t.m0 += o0; t.m1 = min(t.m0 + bm, o1);
+        }
         return true;
     }
 };
@@ -378,7 +410,33 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     const uint32_t tmem_base = *tmem_ptr;
     if (threadIdx.x == 0) CCL_TRACE(1);
 
-    Scheduler sched(p, (int)(blockIdx.x / CTAS), BM * CTAS, TILE_N);
+    // Ragged batch with a dense walk: m-tiles of every problem, as an exclusive prefix over the problems.
+    int* rag_prefix = nullptr;
+    if (p.rag_dense) {
+        int* part = reinterpret_cast<int*>(tmem_ptr + 4);           // one partial sum per thread, then the prefix itself
+        rag_prefix = part + kGemmThreads;
+        const int E = p.batch, bm = BM * CTAS, per = (E + kGemmThreads - 1) / kGemmThreads;
+        const int lo = min(E, (int)threadIdx.x * per), hi = min(E, lo + per);
+        auto tiles_of = [&](int e) {
+            const int o0 = __ldg(p.m_offs + e), o1 = __ldg(p.m_offs + e + 1);
+            if (o0 < 0 || o1 > p.M || o1 - o0 > p.Wm) { atomicExch(&g_gemm_status, 5); return 0; }   // reported, left out
+            return o1 > o0 ? (o1 - o0 + bm - 1) / bm : 0;
+        };
+        int sum = 0;
+        for (int e = lo; e < hi; ++e) sum += tiles_of(e);
+        part[threadIdx.x] = sum;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int run = 0;
+            for (int i = 0; i < kGemmThreads; ++i) { const int v = part[i]; part[i] = run; run += v; }
+            rag_prefix[E] = run;
+        }
+        __syncthreads();
+        int run = part[threadIdx.x];
+        for (int e = lo; e < hi; ++e) { rag_prefix[e] = run; run += tiles_of(e); }
+        __syncthreads();
+    }
+    Scheduler sched(p, (int)(blockIdx.x / CTAS), BM * CTAS, TILE_N, rag_prefix);
     if (threadIdx.x == 0) CCL_TRACE(10);
 
     if (warp == 0) {
@@ -416,6 +474,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         const uint32_t stage_bytes = p.stage_bytes;
         const bool post_tx = lane == 0 && leader;
         for (int it = 0; ok && sched.get(it, t); ++it) {
+            if (t.skip) continue;
             int base = (isA ? t.m0 : t.n0) + off;
             // output column n0 of strip g -> B column n0 + g * pair_dist (gate) and one pair_dist further (up)
             if (SWIGLU && !isA) base += (p.fd_wn.div(t.n0) + hsel) * p.pair_dist;
@@ -454,12 +513,15 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             // loop constants in registers (the asm statements below are memory barriers to the compiler)
             const int stages = p.stages, num_kb = p.num_kb, kbps = p.kb_per_split;
             const uint32_t stage_bytes = p.stage_bytes, a_bytes = p.a_bytes, idesc = p.idesc, smem0 = smem_u32(smem);
+            int done = 0;                                   // tiles computed so far (empty tiles of a ragged batch do not count)
             for (int it = 0; ok && sched.get(it, t); ++it) {
-                // NSUB == 1: TMEM half (it & 1) is this tile's accumulator, the other half is being drained.
+                if (t.skip) continue;
+                // NSUB == 1: TMEM half (done & 1) is this tile's accumulator, the other half is being drained.
                 // NSUB == 2: both halves belong to this tile; half h may be overwritten once the epilogue
                 //            of the previous tile has drained it.
-                const int acc0 = NSUB == 1 ? (it & 1) : 0;
-                const uint32_t acc_phase = NSUB == 1 ? ((uint32_t)(it >> 1) & 1) : ((uint32_t)it & 1);
+                const int acc0 = NSUB == 1 ? (done & 1) : 0;
+                const uint32_t acc_phase = NSUB == 1 ? ((uint32_t)(done >> 1) & 1) : ((uint32_t)done & 1);
+                ++done;
                 const int kb0 = t.split * kbps, kb1 = min(num_kb, kb0 + kbps);
                 for (int kb = kb0; ok && kb < kb1; ++kb) {
                     // (the copies' completion on the barrier orders the operand bytes before the MMAs that read them;
@@ -501,12 +563,15 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         TileCoord t;
         bool alive = true;
         uint32_t epi_count = 0;                          // TMA-stored pieces so far (selects the staging buffer)
+        int done = 0;                                    // tiles drained so far
         for (int it = 0; alive && sched.get(it, t); ++it) {
+          if (t.skip) continue;
+          const int tile_no = done++;
           const int m = t.m0 + (int)rank * BM + quad * 32 + lane;
 #pragma unroll 1                                         // one copy of the (large) drain code: a short GEMM pays for every instruction-cache miss
           for (int h = 0; h < (SWIGLU ? 1 : NSUB); ++h) {
-            const int acc = NSUB == 1 ? (it & 1) : h;
-            const uint32_t acc_phase = NSUB == 1 ? ((uint32_t)(it >> 1) & 1) : ((uint32_t)it & 1);
+            const int acc = NSUB == 1 ? (tile_no & 1) : h;
+            const uint32_t acc_phase = NSUB == 1 ? ((uint32_t)(tile_no >> 1) & 1) : ((uint32_t)tile_no & 1);
             const int nb = t.n0 + h * SUBN;              // first (output) column of this sub-tile
             bool ok = h > 0 || mbar_wait_bounded(&tmem_full[acc], acc_phase);   // one "full" barrier per tile
             ok = __all_sync(0xffffffffu, ok);
@@ -555,7 +620,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     if (lane == 0) {
                         int cx = cx0 + c * 64, cy = cy0, cz = cz0, cu = cu0;
                         if (c_chunked) to_coords(p.c, row0, n64, cx, cy, cz, cu);
-                        tma_store_5d(&map_c, buf, cx, cy, cz, cu, t.e);
+                        tma_store_5d(&map_c, buf, cx, cy, cz, cu, t.e * p.c.batched);
                         tma_store_commit();
                     }
                     CCL_TRACE2(warp == 2 && lane == 0 && epi_count < 12, epi_count * 5 + 4);
@@ -793,7 +858,9 @@ static ccl_status merge_width(int64_t* cur, int64_t w, const char* dim) {
 }
 
 // units = schedulable CTAs (1-CTA kernel) or CTA pairs (2-CTA kernel) the device can hold at once
-static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, const void* A, const void* B, const void* C, int sms, int pairs, GemmPlan* plan) {
+// cap > 0: a ragged batch -- the tile grid of one problem covers `cap` rows, d->M is the total row count of A and C
+static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, const void* A, const void* B, const void* C, int sms, int pairs, GemmPlan* plan,
+                            int64_t cap = 0) {
     if (!d) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: NULL descriptor");
     if (d->M <= 0 || d->N <= 0 || d->K <= 0) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: M, N, K must be positive");
     if (d->M >= (INT64_C(1) << 31) || d->N >= (INT64_C(1) << 31) || d->K >= (INT64_C(1) << 31)) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: dimension too large");
@@ -850,7 +917,9 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     }
     int64_t ka = split_width(va, at), kb = split_width(vb, !bt);
     if ((ka && ka % BK) || (kb && kb % BK)) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: an operand split along K needs strips that are multiples of %d", BK);
-    if (!Wm) Wm = d->M;
+    const int64_t Mt = cap > 0 ? cap : d->M;            // rows the tile grid of one problem covers
+    if (cap > 0 && Wm) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm_grouped: A and C must not be split along M");
+    if (!Wm) Wm = Mt;
     if (!Wn) Wn = Nc;
     if (swiglu) {
         const int64_t pd = d->out_part == CCL_PART_COLS && d->P > 1 ? Nc / d->P : Nc;      // gate -> up distance in B
@@ -869,7 +938,7 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     // 256 x 512 pair tiles move the fewest bytes per flop and win once K is long; short problems prefer the
     // variant whose tile count fills the machine.
     const int64_t num_kb = (d->K + BK - 1) / BK;
-    const int64_t strips_m = d->M / Wm, strips_n = Nc / Wn;
+    const int64_t strips_m = Mt / Wm, strips_n = Nc / Wn;
     int ctas = 1, bn = 256, splits = 1;
     double best = -1.0;
     // Tuning / test overrides (environment): CCL_GEMM_CTAS = 1|2, CCL_GEMM_BN = 128|192|256|512,
@@ -898,7 +967,7 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
             const double stream_clk = tiles_m_all == 1 ? (double)tiles * (double)num_kb * (double)b * (BK * 2) / (sms * 29.0) *
                                                              (b <= 128 ? 1.10 : (b <= 192 ? 1.04 : 1.0)) : 0.0;
             for (int sp : {1, 2, 3, 4, 6, 8, 12, 16}) {
-                if (sp > 1 && (swiglu || num_kb / sp < 2)) continue;
+                if (sp > 1 && (swiglu || cap > 0 || num_kb / sp < 2)) continue;
                 if (force_split && atoi(force_split) != sp) continue;
                 const int64_t kbps = (num_kb + sp - 1) / sp;
                 const int64_t sp_eff = (num_kb + kbps - 1) / kbps;          // every split owns at least one k block
@@ -908,7 +977,7 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
                 const double last = (double)(tiles * sp - (waves - 1) * units) / (double)units;
                 double cost = std::max((double)waves * ((double)kbps * t_kb + (sp > 1 ? 2.0 * t_drain : t_drain)),
                                        stream_clk * (1.0 + 0.1 * (1.0 - last))) + 3000.0;
-                if (sp > 1) cost += ((double)sp + 0.5) * (double)batch * (double)d->M * (double)d->N * 4.0 / 3400.0 + 14000.0;
+                if (sp > 1) cost += ((double)sp + 0.5) * (double)batch * (double)Mt * (double)d->N * 4.0 / 3400.0 + 14000.0;
                 if (best < 0 || cost < best) { best = cost; ctas = c; bn = b; splits = sp; }
             }
         }
@@ -930,7 +999,7 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     p.pair_dist = swiglu ? (int32_t)Wn : 0; p.fd_wn = make_fastdiv(Wn);
     p.Wm = (int32_t)Wm; p.Wn = (int32_t)Wn;
     p.tps_m = (int32_t)((Wm + bm - 1) / bm); p.tps_n = (int32_t)((Wn + bn_walk - 1) / bn_walk);
-    p.tiles_m = (int32_t)(d->M / Wm) * p.tps_m; p.tiles_n = (int32_t)(Nc / Wn) * p.tps_n;
+    p.tiles_m = (int32_t)(Mt / Wm) * p.tps_m; p.tiles_n = (int32_t)(Nc / Wn) * p.tps_n;
     p.num_kb = (int32_t)num_kb;
     p.splits = splits; p.kb_per_split = (int32_t)((num_kb + splits - 1) / splits);
     p.a.split = va.split; p.a.w = make_fastdiv(va.w); p.a.h = make_fastdiv(va.h);
@@ -947,7 +1016,13 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)p.a_mn << 15) | ((uint32_t)p.b_mn << 16) |
               ((uint32_t)(subn >> 3) << 17) | ((uint32_t)(bm >> 4) << 24);
     p.a_bytes = BM * BK * 2; p.stage_bytes = p.a_bytes + (uint32_t)(bn / ctas) * BK * 2;
-    p.stages = (int32_t)(kSmemBudget / p.stage_bytes);
+    // a ragged batch of up to kRaggedDense problems walks only real tiles: the prefix of their tile counts sits behind
+    // the barriers in shared memory, and the operand ring gives up that room
+    // (CCL_GEMM_RAGGED_DENSE=0: the fixed grid of max_rows per problem with empty tiles skipped, as for larger batches)
+    const char* rag_env = std::getenv("CCL_GEMM_RAGGED_DENSE");
+    const uint32_t rag_bytes = cap > 0 && batch <= kRaggedDense && !(rag_env && atoi(rag_env) == 0) ? (uint32_t)(4 * (kGemmThreads + batch + 1) + 1023) & ~1023u : 0;
+    p.rag_dense = rag_bytes ? 1 : 0;
+    p.stages = (int32_t)((kSmemBudget - rag_bytes) / p.stage_bytes);
     if (p.stages > 8) p.stages = 8;
     int64_t ntiles = (int64_t)p.tiles_m * p.tiles_n * splits * batch;
     p.batch = (int32_t)batch;
@@ -986,7 +1061,8 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     p.fd_upg = make_fastdiv(p.sch_upg); p.fd_groups = make_fastdiv(p.groups); p.fd_splits = make_fastdiv(p.splits);
     p.fd_per_panel = make_fastdiv((int64_t)p.panel * p.sch_gn); p.fd_panel = make_fastdiv(p.panel);
     p.fd_tps_m = make_fastdiv(p.tps_m); p.fd_tps_n = make_fastdiv(p.tps_n);
-    plan->smem_bytes = (uint32_t)p.stages * p.stage_bytes + kEpiBytes + 1024 + (2 * p.stages + 8) * 8 + 16;
+    plan->smem_bytes = (uint32_t)p.stages * p.stage_bytes + kEpiBytes + 1024 + (2 * p.stages + 8) * 8 + 16 + rag_bytes;
+    p.fd_tiles_n = make_fastdiv(p.tiles_n);
     return CCL_OK;
 }
 
@@ -1081,7 +1157,7 @@ using namespace ccl;
 
 // ---- host-side cache of prepared calls (plan + encoded tensor maps) --------------------------------------
 struct PreparedKey {
-    int64_t f[36];          // every field of the descriptor, the batch, the three pointers, the device and the tuning overrides
+    int64_t f[38];          // every field of the descriptor, the batch, the three pointers, the ragged-batch arguments
     int dev;
     int mode;               // 0 plain, 1 gated activation
     float alpha, beta;
@@ -1113,7 +1189,7 @@ static void make_key(const ccl_gemm_desc* d, const int64_t* batch4, const void* 
     k->dev = -1;
     (void)cudaGetDevice(&k->dev);
     size_t pos = 0;
-    for (const char* name : {"CCL_GEMM_CTAS", "CCL_GEMM_BN", "CCL_GEMM_SPLITK", "CCL_GEMM_PANEL"}) {
+    for (const char* name : {"CCL_GEMM_CTAS", "CCL_GEMM_BN", "CCL_GEMM_SPLITK", "CCL_GEMM_PANEL", "CCL_GEMM_RAGGED_DENSE"}) {
         const char* v = std::getenv(name);
         for (const char* c = v ? v : ""; *c && pos + 2 < sizeof(k->env); ++c) k->env[pos++] = *c;
         if (pos + 1 < sizeof(k->env)) k->env[pos++] = ';';
@@ -1151,8 +1227,10 @@ extern "C" ccl_status ccl_gemm_workspace(const ccl_gemm_desc* d, size_t* bytes) 
 extern "C" ccl_status ccl_gemm_batched_workspace(const ccl_gemm_desc* d, int32_t batch, size_t* bytes) { return workspace_impl(d, batch, bytes); }
 
 // strides[X]: bytes between the buffers of operand X (A, B, C) of consecutive problems; 0 = shared (A and B only)
+// m_offs / cap: ragged batch (ccl_gemm_grouped), else nullptr / 0
 static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, const int64_t* strides, const void* A_dev, const void* B_dev, void* C_dev,
-                            void* ws_dev, size_t ws_bytes, void* cuda_stream, float alpha = 1.0f, float beta = 0.0f) {
+                            void* ws_dev, size_t ws_bytes, void* cuda_stream, float alpha = 1.0f, float beta = 0.0f, const int32_t* m_offs = nullptr,
+                            int64_t cap = 0) {
     if (!A_dev || !B_dev || !C_dev) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: NULL operand");
     if (!d) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: NULL descriptor");
     if (batch < 1 || batch > kMaxBatch) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: batch must be in [1, %lld]", (long long)kMaxBatch);
@@ -1162,6 +1240,7 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     PreparedKey key;
     make_key(d, batch4, A_dev, B_dev, C_dev, &key);
     key.mode = swiglu ? 1 : 0; key.alpha = alpha; key.beta = beta;
+    key.f[36] = (int64_t)reinterpret_cast<uintptr_t>(m_offs); key.f[37] = cap;
     Prepared prep;
     bool hit = false;
     {
@@ -1172,14 +1251,14 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     ccl_status s;
     if (!hit) {
         GemmPlan& plan = prep.plan;
-        s = make_plan(d, batch, swiglu, A_dev, B_dev, C_dev, 148, 74, &plan);     // validation first: no CUDA call on bad input
+        s = make_plan(d, batch, swiglu, A_dev, B_dev, C_dev, 148, 74, &plan, cap);     // validation first: no CUDA call on bad input
         if (s) return s;
         if (batch > 1) {
             const MatView* views[3] = {&plan.va, &plan.vb, &plan.vc};
             const char* names[3] = {"A", "B", "C"};
             for (int X = 0; X < 3; ++X) {
                 const int64_t st = batch4[1 + X], need = buffer_elems(*views[X]) * 2;
-                if (st == 0 && X < 2) continue;                     // an operand every problem shares
+                if (st == 0 && (X < 2 || m_offs)) continue;         // an operand every problem shares (or, ragged, one concatenated C)
                 if (st < need) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm_batched: stride of %s (%lld bytes) is smaller than its buffer (%lld bytes)", names[X], (long long)st, (long long)need);
                 if (st % 16) return fail(CCL_ERR_ALIGN, "ccl_gemm_batched: stride of %s is not a multiple of 16 bytes", names[X]);
                 if (st >= (INT64_C(1) << 40)) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm_batched: stride of %s too large for a tensor map", names[X]);
@@ -1188,10 +1267,15 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
         int dev;
         CCL_CUDA_TRY(cudaGetDevice(&dev));
         CCL_CUDA_TRY(cudaDeviceGetAttribute(&prep.sms, cudaDevAttrMultiProcessorCount, dev));
-        if (dev != key.dev) { make_key(d, batch4, A_dev, B_dev, C_dev, &key); key.mode = swiglu ? 1 : 0; key.alpha = alpha; key.beta = beta; }
-        if ((s = make_plan(d, batch, swiglu, A_dev, B_dev, C_dev, prep.sms, resident_pairs(), &plan))) return s;
+        if (dev != key.dev) {
+            make_key(d, batch4, A_dev, B_dev, C_dev, &key);
+            key.mode = swiglu ? 1 : 0; key.alpha = alpha; key.beta = beta;
+            key.f[36] = (int64_t)reinterpret_cast<uintptr_t>(m_offs); key.f[37] = cap;
+        }
+        if ((s = make_plan(d, batch, swiglu, A_dev, B_dev, C_dev, prep.sms, resident_pairs(), &plan, cap))) return s;
         plan.p.C = static_cast<uint16_t*>(C_dev);
-        plan.p.a.batched = batch4[1] != 0; plan.p.b.batched = batch4[2] != 0; plan.p.c.batched = 1;
+        plan.p.a.batched = batch4[1] != 0; plan.p.b.batched = batch4[2] != 0; plan.p.c.batched = m_offs ? 0 : 1;
+        plan.p.m_offs = m_offs;
         plan.p.c_batch_stride = batch4[3] / 2;
         plan.p.alpha = alpha; plan.p.beta = beta; plan.p.axpby = (alpha != 1.0f || beta != 0.0f) ? 1 : 0;
         const uint32_t bnh = (uint32_t)(plan.subn / plan.ctas);   // B rows of one K-major box
@@ -1248,6 +1332,18 @@ extern "C" ccl_status ccl_gemm_batched(const ccl_gemm_desc* d, int32_t batch, co
     return gemm_impl(d, batch, false, strides, A_dev, B_dev, C_dev, ws_dev, ws_bytes, cuda_stream);
 }
 
+extern "C" ccl_status ccl_gemm_grouped(const ccl_gemm_desc* d, int32_t groups, int64_t max_rows, const int32_t* row_offsets_dev, const void* A_dev,
+                                       const void* B_dev, int64_t b_stride_bytes, void* C_dev, void* cuda_stream) {
+    if (!d) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm_grouped: NULL descriptor");
+    if (!row_offsets_dev) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm_grouped: NULL row offsets");
+    if (reinterpret_cast<uintptr_t>(row_offsets_dev) & 3) return fail(CCL_ERR_ALIGN, "ccl_gemm_grouped: row offsets are not 4-byte aligned");
+    if (max_rows < 1 || max_rows > d->M) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm_grouped: max_rows must be in [1, M]");
+    if (b_stride_bytes < 0) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm_grouped: negative stride");
+    if (d->a_trans) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm_grouped: A must be stored [M x K]");
+    const int64_t strides[3] = {0, b_stride_bytes, 0};
+    return gemm_impl(d, groups, false, strides, A_dev, B_dev, C_dev, nullptr, 0, cuda_stream, 1.0f, 0.0f, row_offsets_dev, max_rows);
+}
+
 extern "C" ccl_status ccl_gemm_axpby(const ccl_gemm_desc* d, float alpha, float beta, const void* A_dev, const void* B_dev, void* C_dev,
                                      void* ws_dev, size_t ws_bytes, void* cuda_stream) {
     if (!(alpha == alpha) || !(beta == beta)) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm_axpby: alpha / beta is NaN");
@@ -1268,6 +1364,7 @@ extern "C" ccl_status ccl_gemm_status(void* cuda_stream, int32_t* detail) {
     ccl_status s = repack_status_take(&rv);
     if (s) return s;
     if (detail) *detail = v ? v : (rv ? 100 + rv : 0);
+    if (v == 5) return fail(CCL_ERR_SHAPE, "ccl_gemm_grouped: row offsets outside [0, M] or a problem with more rows than max_rows (such problems were not computed)");
     if (v || rv) return fail(CCL_ERR_TIMEOUT, "a bounded device-side wait expired (code %d)", v ? v : 100 + rv);
     return CCL_OK;
 }

@@ -354,6 +354,31 @@ def extras(out_dir, quick, only=None):
                          batched_tflops=fl / t_b / 1e9, torch_bmm_tflops=fl / t_t / 1e9))
         print(f"extras batched {E} x {M}x{N}x{K}: one launch {t_b * 1e3:8.1f} us ({fl / t_b / 1e9:6.0f} TFLOP/s) | {E} launches {t_l * 1e3:8.1f} us | "
               f"torch.bmm {t_t * 1e3:8.1f} us", flush=True)
+    # 1b. the same experts with uneven (routed) token counts: the ragged batch in one launch
+    for E, T, N, K, bt in (((128, 32768, 768, 2048, 1), (128, 32768, 2048, 768, 0)) if not quick else ((32, 8192, 768, 2048, 1),)) if want("grouped_gemm") else ():
+        import numpy as np
+        for conc, label in ((1e6, "equal counts"), (2.0, "Dirichlet(2) counts"), (0.5, "Dirichlet(0.5) counts")):
+            wts = np.random.default_rng(3).dirichlet(np.full(E, conc))
+            counts = np.floor(wts * T).astype(np.int64)
+            counts[0] += T - counts.sum()
+            offs = torch.from_numpy(np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)).to(dev)
+            d = desc(T, N, K, 4, bt)
+            A, B, Cb = buf(d.A), buf(d.B, E), buf(d.C)
+            sb = ccl.ccl_buffer_bytes(d.B)
+            cap = int(counts.max())
+            t_g = timed(lambda: ccl.ccl_gemm_grouped(d, E, cap, offs, A, B, sb, Cb), 20)
+            Av, Bv = A.view(T, K), (B.view(E, N, K) if bt else B.view(E, K, N))
+            bounds = [int(x) for x in offs.cpu()]
+
+            def torch_loop():
+                for e in range(E):
+                    if bounds[e + 1] > bounds[e]:
+                        torch.matmul(Av[bounds[e]:bounds[e + 1]], Bv[e].t() if bt else Bv[e])
+            t_t = timed(torch_loop, 3)
+            tf = 2.0 * T * N * K / (t_g * 1e-3) / 1e12
+            rows.append(dict(what="grouped", experts=E, tokens=T, N=N, K=K, counts=label, max_count=cap, grouped_ms=t_g, torch_loop_ms=t_t, tflops=tf))
+            print(f"extras grouped {E} experts, {T} tokens x {N} x {K}, {label} (max {cap}): one launch {t_g * 1e3:8.1f} us ({tf:6.0f} TFLOP/s) | "
+                  f"torch.matmul per expert {t_t * 1e3:8.1f} us", flush=True)
     # 2. gate/up GEMM with the gated activation in the epilogue against GEMM + elementwise kernel
     for M, N, K in (((8192, 57344, 8192), (16384, 1536, 2048)) if not quick else ((1024, 57344, 8192),)) if want("swiglu") else ():
         d0, d1 = desc(M, N, K, 4), desc(M, N, K, 4, c_cols=N // 2)

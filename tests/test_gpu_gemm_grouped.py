@@ -1,0 +1,130 @@
+"""GPU parity, through the C ABI: ccl_gemm_grouped (a ragged batch: every problem its own row count and its own B)
+against the fp32 oracle problem by problem; rows no problem owns stay untouched."""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle as orc
+from paper_2606_11718_b200 import binding as ccl
+from paper_2606_11718_b200 import synth
+from helpers import gemm_desc
+from test_gpu_gemm import from_layout, to_layout, tol
+
+pytestmark = pytest.mark.gpu
+POISON = 0x7FC0
+
+
+def pad16(n):
+    return (n + 15) // 16 * 16
+
+
+def run_grouped(N, K, P, lay, bt, counts, first=0, slack=0, max_rows=None, expect=ccl.OK, share_b=False):
+    """counts[e] rows for problem e, the first problem starts at row `first`, `slack` unowned rows at the end.
+    Returns (C bits [M x N], offsets, As, Bs)."""
+    E = len(counts)
+    offs = np.concatenate([[first], first + np.cumsum(counts)]).astype(np.int32)
+    M = int(offs[-1]) + slack
+    d = gemm_desc(M, N, K, P, lay, 0, bt, 2, 1)
+    A = synth.gemm_operands(M, N, K, 0, bt, seed=5, tag="grouped")[0]
+    Bs = [synth.gemm_operands(8, N, K, 0, bt, seed=40 + e, tag="grouped")[1] for e in range(E)]
+    sb = pad16(ccl.ccl_buffer_bytes(d.B)) + 64
+    b_dev = torch.zeros((1 if share_b else E) * sb // 2, dtype=torch.int16, device="cuda")
+    for e in range(1 if share_b else E):
+        x = to_layout(synth.bits(Bs[e]), d.B)
+        b_dev[e * sb // 2: e * sb // 2 + x.numel()] = x
+    a_dev = to_layout(synth.bits(A), d.A)
+    nc = ccl.ccl_buffer_bytes(d.C) // 2
+    c_dev = torch.full((nc + 4096,), POISON, dtype=torch.int16, device="cuda")
+    ccl.ccl_gemm_grouped(d, E, max_rows if max_rows is not None else max(1, int(max(counts))), torch.from_numpy(offs).cuda(),
+                         a_dev, b_dev, 0 if share_b else sb, c_dev)
+    st, detail = ccl.ccl_gemm_status()
+    assert st == expect, (st, detail)
+    assert (c_dev[nc:] == POISON).all(), "wrote past the end of C"
+    return from_layout(c_dev[:nc], d.C), offs, A, Bs
+
+
+def check(Cbits, offs, A, Bs, N, K, bt, skip=()):
+    g = synth.from_bits(Cbits).to(torch.float32).numpy()
+    a_bits = synth.bits(A)
+    M = Cbits.shape[0]
+    owned = np.zeros(M, dtype=bool)
+    for e in range(len(Bs)):
+        o0, o1 = int(offs[e]), int(offs[e + 1])
+        if o1 <= o0 or e in skip:
+            continue
+        owned[o0:o1] = True
+        ref32, _, _ = orc.gemm(a_bits[o0:o1], synth.bits(Bs[e]), o1 - o0, N, K, 0, bt)
+        assert np.isfinite(g[o0:o1]).all(), f"problem {e}: unwritten output"
+        err = np.abs(g[o0:o1] - ref32) / np.maximum(1.0, np.abs(ref32))
+        assert err.max() <= tol(K), (e, err.max())
+    assert (Cbits[~owned] == POISON).all(), "rows no problem owns were written"
+
+
+CASES = [
+    # N, K, P, layouts, b_trans, counts, first, slack
+    (768, 512, 4, ("row", "ccl", "ccl"), 1, [256, 0, 37, 300, 1, 128, 513], 0, 0),     # expert up-projections, ragged token counts
+    (384, 200, 2, ("row", "ccl", "ccl"), 0, [130, 5, 260], 3, 9),                       # unowned rows before and after, ragged K
+    (512, 256, 1, ("row", "row", "row"), 0, [64, 64, 64, 64], 0, 0),                    # equal counts: a plain batch
+    (1024, 256, 4, ("row", "ccl", "row"), 0, [700, 20], 0, 0),                          # C row-major
+    (512, 1088, 2, ("row", "ccl", "ccl"), 1, [1, 2, 3, 250, 4], 8, 0),
+]
+
+
+@pytest.mark.parametrize("N,K,P,lay,bt,counts,first,slack", CASES)
+@pytest.mark.parametrize("tile", ["auto", "1,128", "1,256", "2,256", "2,512"])
+@pytest.mark.parametrize("walk", ["dense", "skip"])
+def test_grouped_equals_oracle(N, K, P, lay, bt, counts, first, slack, tile, walk):
+    """Both tile walks: the dense one (a prefix of the problems' tile counts) and the fixed grid of max_rows per problem
+    with empty tiles skipped, which batches of more than 4096 problems use."""
+    saved = {k: os.environ.pop(k, None) for k in ("CCL_GEMM_CTAS", "CCL_GEMM_BN", "CCL_GEMM_RAGGED_DENSE")}
+    if tile != "auto":
+        os.environ["CCL_GEMM_CTAS"], os.environ["CCL_GEMM_BN"] = tile.split(",")
+    if walk == "skip":
+        os.environ["CCL_GEMM_RAGGED_DENSE"] = "0"
+    try:
+        Cb, offs, A, Bs = run_grouped(N, K, P, lay, bt, counts, first, slack)
+        check(Cb, offs, A, Bs, N, K, bt)
+        # a looser bound on the rows per problem gives the same bits (more empty tiles, same tiles computed)
+        Cb2, _, _, _ = run_grouped(N, K, P, lay, bt, counts, first, slack, max_rows=min(int(offs[-1]) + slack, max(counts) + 300))
+        np.testing.assert_array_equal(Cb, Cb2)
+    finally:
+        for k, v in saved.items():
+            os.environ.pop(k, None)
+            if v is not None:
+                os.environ[k] = v
+
+
+def test_grouped_shared_b_is_one_gemm():
+    """With one shared B the ragged batch is a plain GEMM on the owned rows."""
+    N, K, P = 768, 320, 4
+    Cb, offs, A, Bs = run_grouped(N, K, P, ("row", "ccl", "ccl"), 0, [100, 28, 200], share_b=True)
+    check(Cb, offs, A, [Bs[0]] * 3, N, K, 0)
+
+
+def test_grouped_reports_a_problem_that_exceeds_the_bound():
+    """A problem with more rows than max_rows is left out and reported; the others are computed."""
+    N, K, P = 512, 256, 2
+    counts = [40, 300, 64]
+    Cb, offs, A, Bs = run_grouped(N, K, P, ("row", "ccl", "ccl"), 0, counts, max_rows=128, expect=ccl.ERR_SHAPE)
+    check(Cb, offs, A, Bs, N, K, 0, skip=(1,))
+    assert ccl.ccl_gemm_status()[0] == ccl.OK                      # the flag is cleared by the read
+
+
+def test_grouped_qwen_experts_full_size():
+    """128 experts of the Qwen-style layer with 32768 routed tokens (uneven counts): sampled problems in full."""
+    rng = np.random.default_rng(9)
+    w = rng.dirichlet(np.full(128, 2.0))
+    counts = np.floor(w * 32768).astype(np.int64)
+    counts[0] += 32768 - counts.sum()
+    Cb, offs, A, Bs = run_grouped(768, 2048, 4, ("row", "ccl", "ccl"), 1, [int(c) for c in counts], max_rows=int(counts.max()))
+    g = synth.from_bits(Cb).to(torch.float32).numpy()
+    assert np.isfinite(g).all()
+    a_bits = synth.bits(A)
+    for e in (0, 17, 64, 127):
+        o0, o1 = int(offs[e]), int(offs[e + 1])
+        ref32, _, _ = orc.gemm(a_bits[o0:o1], synth.bits(Bs[e]), o1 - o0, 768, 2048, 0, 1)
+        err = np.abs(g[o0:o1] - ref32) / np.maximum(1.0, np.abs(ref32))
+        assert err.max() <= tol(2048), (e, err.max())
