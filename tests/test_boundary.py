@@ -125,6 +125,21 @@ def test_repack_rejects_bad_input_before_any_launch():
     assert l.ccl_repack_batched(C.byref(padded), 2, C.c_void_p(256), 64, C.c_void_p(4096), 64, 0, None) == ccl.ERR_INVALID_ARG
 
 
+def test_gemm_grouped_rejects_bad_input_before_any_launch():
+    l = ccl.lib()
+    d = gemm_desc(1024, 768, 512, 4, ("row", "ccl", "ccl"), b_trans=1)
+    call = lambda dd, groups=4, cap=256, offs=65536, b_stride=1 << 20: l.ccl_gemm_grouped(
+        C.byref(dd), groups, cap, C.c_void_p(offs), C.c_void_p(4096), C.c_void_p(8192), b_stride, C.c_void_p(16384), None)
+    assert call(d, offs=None) == ccl.ERR_INVALID_ARG                 # no row offsets
+    assert call(d, offs=65538) == ccl.ERR_ALIGN
+    assert call(d, cap=0) == ccl.ERR_INVALID_ARG and call(d, cap=1025) == ccl.ERR_INVALID_ARG
+    assert call(d, b_stride=-16) == ccl.ERR_INVALID_ARG
+    assert call(d, groups=0) == ccl.ERR_INVALID_ARG
+    assert call(d, b_stride=1000) == ccl.ERR_INVALID_ARG             # smaller than one B
+    assert call(gemm_desc(1024, 768, 512, 4, ("row", "ccl", "ccl"), a_trans=1)) == ccl.ERR_UNSUPPORTED
+    assert call(gemm_desc(1024, 768, 512, 4, ("ccl", "row", "ccl"), out_part=1)) == ccl.ERR_UNSUPPORTED    # split along M
+
+
 def gemm_rc(d, a=4096, b=8192, c=16384):
     return ccl.lib().ccl_gemm(C.byref(d), C.c_void_p(a), C.c_void_p(b), C.c_void_p(c), None, 0, None)
 
