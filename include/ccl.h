@@ -179,6 +179,13 @@ ccl_status ccl_gemm(const ccl_gemm_desc* d, const void* A_dev, const void* B_dev
  */
 ccl_status ccl_gemm_grouped(const ccl_gemm_desc* d, int32_t groups, int64_t max_rows, const int32_t* row_offsets_dev,
                             const void* A_dev, const void* B_dev, int64_t b_stride_bytes, void* C_dev, void* cuda_stream);
+/*
+ * The ragged batch with the gated activation of ccl_gemm_swiglu in the epilogue: the first half of an MoE expert FFN
+ * in one launch.  d, A, B and C as for ccl_gemm_swiglu (d->N = gate + up columns of every B, C [M x N/2]), the batch
+ * arguments as for ccl_gemm_grouped; the conditions and errors of both apply.
+ */
+ccl_status ccl_gemm_grouped_swiglu(const ccl_gemm_desc* d, int32_t groups, int64_t max_rows, const int32_t* row_offsets_dev,
+                                   const void* A_dev, const void* B_dev, int64_t b_stride_bytes, void* C_dev, void* cuda_stream);
 
 /*
  * The BLAS form (Sec. 2.2: "the extension to alpha*A*B + beta*C is straightforward, since the scalars do not affect

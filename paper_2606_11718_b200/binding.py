@@ -20,7 +20,7 @@ PLACE_RR, PLACE_BLOCK, PLACE_BEST = 0, 1, 2
 ASSIGN_N_STRIPS, ASSIGN_M_STRIPS, ASSIGN_EXPLICIT = 0, 1, 2
 
 EXPORTS = ["ccl_map_offset", "ccl_map_inverse", "ccl_buffer_bytes", "ccl_strip_stride", "ccl_repack", "ccl_repack_batched", "ccl_repack_transpose", "ccl_gemm_workspace",
-           "ccl_gemm", "ccl_gemm_batched_workspace", "ccl_gemm_batched", "ccl_gemm_grouped", "ccl_gemm_axpby", "ccl_gemm_swiglu", "ccl_gemm_static_ws", "ccl_gemm_status", "ccl_traffic_sizes", "ccl_traffic", "ccl_traffic_l2", "ccl_traffic_lru", "ccl_last_error", "ccl_launch_count", "ccl_version"]
+           "ccl_gemm", "ccl_gemm_batched_workspace", "ccl_gemm_batched", "ccl_gemm_grouped", "ccl_gemm_grouped_swiglu", "ccl_gemm_axpby", "ccl_gemm_swiglu", "ccl_gemm_static_ws", "ccl_gemm_status", "ccl_traffic_sizes", "ccl_traffic", "ccl_traffic_l2", "ccl_traffic_lru", "ccl_last_error", "ccl_launch_count", "ccl_version"]
 
 
 class CclError(RuntimeError):
@@ -85,6 +85,7 @@ def lib():
         l.ccl_gemm_workspace.argtypes = [C.POINTER(GemmDesc), C.POINTER(C.c_size_t)]
         l.ccl_gemm.argtypes = [C.POINTER(GemmDesc), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         l.ccl_gemm_grouped.argtypes = [C.POINTER(GemmDesc), C.c_int32, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]
+        l.ccl_gemm_grouped_swiglu.argtypes = l.ccl_gemm_grouped.argtypes
         l.ccl_gemm_batched_workspace.argtypes = [C.POINTER(GemmDesc), C.c_int32, C.POINTER(C.c_size_t)]
         l.ccl_gemm_batched.argtypes = [C.POINTER(GemmDesc), C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64,
                                        C.c_void_p, C.c_size_t, C.c_void_p]
@@ -206,6 +207,13 @@ def ccl_gemm_batched(d, batch, A, a_stride, B, b_stride, Cout, c_stride, ws=None
             raise ValueError("ccl_gemm_batched: operand buffer too small")
     ws_bytes = ws.numel() * ws.element_size() if ws is not None else 0
     _check(lib().ccl_gemm_batched(C.byref(d), batch, _ptr(A), a_stride, _ptr(B), b_stride, _ptr(Cout), c_stride, _ptr(ws), ws_bytes, _stream()))
+
+
+def ccl_gemm_grouped_swiglu(d, groups, max_rows, row_offsets, A, B, b_stride_bytes, Cbuf):
+    """ccl_gemm_grouped with silu(gate) * up in the epilogue (d.N = gate + up columns, C [M x N/2])."""
+    if row_offsets.dtype != torch.int32 or not row_offsets.is_cuda or row_offsets.numel() < groups + 1:
+        raise ValueError("ccl_gemm_grouped_swiglu: row_offsets must be an int32 CUDA tensor with groups + 1 entries")
+    _check(lib().ccl_gemm_grouped_swiglu(C.byref(d), groups, max_rows, _ptr(row_offsets), _ptr(A), _ptr(B), b_stride_bytes, _ptr(Cbuf), _stream()))
 
 
 def ccl_gemm_grouped(d, groups, max_rows, row_offsets, A, B, b_stride_bytes, Cbuf):

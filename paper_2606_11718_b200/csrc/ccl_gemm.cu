@@ -1332,8 +1332,8 @@ extern "C" ccl_status ccl_gemm_batched(const ccl_gemm_desc* d, int32_t batch, co
     return gemm_impl(d, batch, false, strides, A_dev, B_dev, C_dev, ws_dev, ws_bytes, cuda_stream);
 }
 
-extern "C" ccl_status ccl_gemm_grouped(const ccl_gemm_desc* d, int32_t groups, int64_t max_rows, const int32_t* row_offsets_dev, const void* A_dev,
-                                       const void* B_dev, int64_t b_stride_bytes, void* C_dev, void* cuda_stream) {
+static ccl_status grouped_impl(const ccl_gemm_desc* d, bool swiglu, int32_t groups, int64_t max_rows, const int32_t* row_offsets_dev, const void* A_dev,
+                               const void* B_dev, int64_t b_stride_bytes, void* C_dev, void* cuda_stream) {
     if (!d) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm_grouped: NULL descriptor");
     if (!row_offsets_dev) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm_grouped: NULL row offsets");
     if (reinterpret_cast<uintptr_t>(row_offsets_dev) & 3) return fail(CCL_ERR_ALIGN, "ccl_gemm_grouped: row offsets are not 4-byte aligned");
@@ -1341,7 +1341,17 @@ extern "C" ccl_status ccl_gemm_grouped(const ccl_gemm_desc* d, int32_t groups, i
     if (b_stride_bytes < 0) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm_grouped: negative stride");
     if (d->a_trans) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm_grouped: A must be stored [M x K]");
     const int64_t strides[3] = {0, b_stride_bytes, 0};
-    return gemm_impl(d, groups, false, strides, A_dev, B_dev, C_dev, nullptr, 0, cuda_stream, 1.0f, 0.0f, row_offsets_dev, max_rows);
+    return gemm_impl(d, groups, swiglu, strides, A_dev, B_dev, C_dev, nullptr, 0, cuda_stream, 1.0f, 0.0f, row_offsets_dev, max_rows);
+}
+
+extern "C" ccl_status ccl_gemm_grouped(const ccl_gemm_desc* d, int32_t groups, int64_t max_rows, const int32_t* row_offsets_dev, const void* A_dev,
+                                       const void* B_dev, int64_t b_stride_bytes, void* C_dev, void* cuda_stream) {
+    return grouped_impl(d, false, groups, max_rows, row_offsets_dev, A_dev, B_dev, b_stride_bytes, C_dev, cuda_stream);
+}
+
+extern "C" ccl_status ccl_gemm_grouped_swiglu(const ccl_gemm_desc* d, int32_t groups, int64_t max_rows, const int32_t* row_offsets_dev,
+                                              const void* A_dev, const void* B_dev, int64_t b_stride_bytes, void* C_dev, void* cuda_stream) {
+    return grouped_impl(d, true, groups, max_rows, row_offsets_dev, A_dev, B_dev, b_stride_bytes, C_dev, cuda_stream);
 }
 
 extern "C" ccl_status ccl_gemm_axpby(const ccl_gemm_desc* d, float alpha, float beta, const void* A_dev, const void* B_dev, void* C_dev,

@@ -379,6 +379,31 @@ def extras(out_dir, quick, only=None):
             rows.append(dict(what="grouped", experts=E, tokens=T, N=N, K=K, counts=label, max_count=cap, grouped_ms=t_g, torch_loop_ms=t_t, tflops=tf))
             print(f"extras grouped {E} experts, {T} tokens x {N} x {K}, {label} (max {cap}): one launch {t_g * 1e3:8.1f} us ({tf:6.0f} TFLOP/s) | "
                   f"torch.matmul per expert {t_t * 1e3:8.1f} us", flush=True)
+    # 1c. a whole MoE expert FFN forward on routed tokens: gate/up with the activation fused, then down -- two launches
+    for E, T, H, I in (((128, 32768, 2048, 768),) if not quick else ((32, 8192, 2048, 768),)) if want("moe_ffn") else ():
+        import numpy as np
+        wts = np.random.default_rng(3).dirichlet(np.full(E, 2.0))
+        counts = np.floor(wts * T).astype(np.int64)
+        counts[0] += T - counts.sum()
+        offs = torch.from_numpy(np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)).to(dev)
+        cap = int(counts.max())
+        d1 = desc(T, 2 * I, H, 4, 0, c_cols=I)                       # X [T x H] * Wgu [H x 2I] -> silu(gate) * up [T x I]
+        d2 = desc(T, H, I, 4, 0)                                     # ... * Wd [I x H] -> [T x H]
+        d2.A = d1.C                                                  # the down GEMM reads the activation where the first wrote it
+        X, Wgu, Act, Wd, Y = buf(d1.A), buf(d1.B, E), buf(d1.C), buf(d2.B, E), buf(d2.C)
+        s1, s2 = ccl.ccl_buffer_bytes(d1.B), ccl.ccl_buffer_bytes(d2.B)
+        try:
+            def ffn():
+                ccl.ccl_gemm_grouped_swiglu(d1, E, cap, offs, X, Wgu, s1, Act)
+                ccl.ccl_gemm_grouped(d2, E, cap, offs, Act, Wd, s2, Y)
+            t_f = timed(ffn, 20)
+            t_1 = timed(lambda: ccl.ccl_gemm_grouped_swiglu(d1, E, cap, offs, X, Wgu, s1, Act), 20)
+            fl = 2.0 * T * (2 * I * H + H * I)
+            rows.append(dict(what="moe_ffn", experts=E, tokens=T, H=H, I=I, ffn_ms=t_f, gateup_ms=t_1, tflops=fl / (t_f * 1e-3) / 1e12))
+            print(f"extras MoE FFN forward, {E} experts, {T} routed tokens (Dirichlet(2), max {cap}), H {H} I {I}: gate/up + activation {t_1 * 1e3:7.1f} us, "
+                  f"with down {t_f * 1e3:7.1f} us ({fl / (t_f * 1e-3) / 1e12:6.0f} TFLOP/s)", flush=True)
+        except ccl.CclError as err:
+            print(f"extras MoE FFN forward: not supported in this form ({err})", flush=True)
     # 2. gate/up GEMM with the gated activation in the epilogue against GEMM + elementwise kernel
     for M, N, K in (((8192, 57344, 8192), (16384, 1536, 2048)) if not quick else ((1024, 57344, 8192),)) if want("swiglu") else ():
         d0, d1 = desc(M, N, K, 4), desc(M, N, K, 4, c_cols=N // 2)

@@ -128,3 +128,56 @@ def test_grouped_qwen_experts_full_size():
         ref32, _, _ = orc.gemm(a_bits[o0:o1], synth.bits(Bs[e]), o1 - o0, 768, 2048, 0, 1)
         err = np.abs(g[o0:o1] - ref32) / np.maximum(1.0, np.abs(ref32))
         assert err.max() <= tol(2048), (e, err.max())
+
+
+SWIGLU_CASES = [
+    # N (gate + up), K, P, layouts, b_trans, counts
+    (1536, 512, 4, ("row", "ccl", "ccl"), 1, [256, 0, 37, 300, 1, 130]),      # Qwen expert gate/up, strips of 192 | 192
+    (1024, 200, 2, ("row", "ccl", "ccl"), 0, [130, 5, 260]),
+    (512, 256, 1, ("row", "row", "row"), 0, [64, 200]),
+]
+
+
+@pytest.mark.parametrize("N,K,P,lay,bt,counts", SWIGLU_CASES)
+@pytest.mark.parametrize("walk", ["dense", "skip"])
+def test_grouped_swiglu_equals_oracle(N, K, P, lay, bt, counts, walk):
+    """The first half of an MoE expert FFN in one launch: per problem silu(gate) * up of its rows times its own B."""
+    saved = os.environ.pop("CCL_GEMM_RAGGED_DENSE", None)
+    if walk == "skip":
+        os.environ["CCL_GEMM_RAGGED_DENSE"] = "0"
+    try:
+        E = len(counts)
+        offs = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
+        M = int(offs[-1]) + 5                                         # five rows nobody owns
+        d = gemm_desc(M, N, K, P, lay, 0, bt, 2, 1)
+        c = d.C
+        d.C = ccl.Mat(M, N // 2, 2, c.P, c.part, c.layout, c.strip_align_bytes)
+        A = synth.gemm_operands(M, N, K, 0, bt, seed=6, tag="grouped_swiglu")[0]
+        Bs = [synth.gemm_operands(8, N, K, 0, bt, seed=60 + e, tag="grouped_swiglu", b_std=0.05)[1] for e in range(E)]
+        sb = pad16(ccl.ccl_buffer_bytes(d.B))
+        b_dev = torch.zeros(E * sb // 2, dtype=torch.int16, device="cuda")
+        for e in range(E):
+            x = to_layout(synth.bits(Bs[e]), d.B)
+            b_dev[e * sb // 2: e * sb // 2 + x.numel()] = x
+        nc = ccl.ccl_buffer_bytes(d.C) // 2
+        c_dev = torch.full((nc + 4096,), POISON, dtype=torch.int16, device="cuda")
+        ccl.ccl_gemm_grouped_swiglu(d, E, max(counts), torch.from_numpy(offs).cuda(), to_layout(synth.bits(A), d.A), b_dev, sb, c_dev)
+        assert ccl.ccl_gemm_status()[0] == ccl.OK
+        assert (c_dev[nc:] == POISON).all()
+        got = from_layout(c_dev[:nc], d.C)
+        g = synth.from_bits(got).to(torch.float32).numpy()
+        a_bits = synth.bits(A)
+        S = P if P > 1 else 1
+        for e in range(E):
+            o0, o1 = int(offs[e]), int(offs[e + 1])
+            if o1 == o0:
+                continue
+            ref32, _ = orc.gemm_swiglu(a_bits[o0:o1], synth.bits(Bs[e]), o1 - o0, N, K, P=S, a_trans=0, b_trans=bt)
+            assert np.isfinite(g[o0:o1]).all()
+            err = np.abs(g[o0:o1] - ref32) / np.maximum(1.0, np.abs(ref32))
+            assert err.max() <= tol(K) + 2.0 ** -8, (e, err.max())
+        assert (got[int(offs[-1]):] == POISON).all(), "rows no problem owns were written"
+    finally:
+        os.environ.pop("CCL_GEMM_RAGGED_DENSE", None)
+        if saved is not None:
+            os.environ["CCL_GEMM_RAGGED_DENSE"] = saved
