@@ -5,6 +5,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle as orc
 from paper_2606_11718_b200 import binding as ccl
 from paper_2606_11718_b200 import synth
 from helpers import gemm_desc, traffic_pair
@@ -68,4 +69,51 @@ def test_step_replays_from_a_cuda_graph():
         torch.cuda.synchronize()
         for o, w in zip(outs, want):
             assert torch.equal(o, w)
+    assert ccl.ccl_gemm_status()[0] == ccl.OK
+
+
+def test_ragged_batch_in_a_graph_follows_the_offsets_on_the_device():
+    """ccl_gemm_grouped reads the row offsets on the device: one captured launch serves whatever routing the offsets
+    hold at replay time (as long as no problem exceeds the bound the graph was captured with)."""
+    N, K, P, E, M = 768, 256, 4, 6, 1024
+    A, _ = synth.gemm_operands(M, N, K, 0, 1, seed=41, tag="graph_ragged")
+    Bs = [synth.gemm_operands(8, N, K, 0, 1, seed=50 + e, tag="graph_ragged")[1] for e in range(E)]
+    d = gemm_desc(M, N, K, P, ("row", "row", "row"), 0, 1, 2, 1)
+    a = A.cuda()
+    b = torch.stack(Bs).cuda().contiguous()                              # [E, N, K] row-major
+    c = torch.zeros(M * N, dtype=torch.bfloat16, device="cuda")
+    offs = torch.zeros(E + 1, dtype=torch.int32, device="cuda")
+    routings = [[100, 200, 0, 300, 24, 400], [400, 0, 0, 1, 223, 400], [170, 170, 170, 170, 170, 174]]
+
+    def set_offsets(counts):
+        offs.copy_(torch.tensor([0] + list(np.cumsum(counts)), dtype=torch.int32), non_blocking=False)
+
+    def expect(counts):                                                  # the oracle's GEMM, problem by problem
+        out = torch.zeros(M, N, dtype=torch.float32)
+        o = 0
+        for e, n in enumerate(counts):
+            if n:
+                out[o:o + n] = torch.from_numpy(orc.gemm(synth.bits(A)[o:o + n], synth.bits(Bs[e]), n, N, K, 0, 1)[0])
+            o += n
+        return out
+
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        set_offsets(routings[0])
+        ccl.ccl_gemm_grouped(d, E, 400, offs, a, b, N * K * 2, c)       # eager: plan cached, kernel configured
+        side.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            ccl.ccl_gemm_grouped(d, E, 400, offs, a, b, N * K * 2, c)
+    for counts in routings:
+        set_offsets(counts)
+        c.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        got = c.view(M, N).float().cpu()
+        want = expect(counts)
+        owned = sum(counts)
+        err = (got[:owned] - want[:owned]).abs() / want[:owned].abs().clamp(min=1.0)
+        assert err.max() <= 1e-2 * (K / 1024.0) ** 0.5 + 2.0 ** -8
+        assert (got[owned:] == 0).all()
     assert ccl.ccl_gemm_status()[0] == ccl.OK
