@@ -363,6 +363,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 const __grid_constant__ CUtensorMap map_c, const __grid_constant__ GemmParams gp) {
     // The parameters are read from shared memory: the threads fetch the block's words side by side, so
     // the cold constant-cache misses at kernel start overlap instead of queueing up in every role's set-up.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel's CTAs may be placed as SMs free up
     __shared__ GemmParams p;
     {
         static_assert(sizeof(GemmParams) % 4 == 0, "GemmParams is copied word by word");
@@ -409,6 +410,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     tc_fence_after();
     const uint32_t tmem_base = *tmem_ptr;
     if (threadIdx.x == 0) CCL_TRACE(1);
+    asm volatile("griddepcontrol.wait;" ::: "memory");   // everything before this overlapped the previous kernel's tail
 
     // Ragged batch with a dense walk: m-tiles of every problem, as an exclusive prefix over the problems.
     int* rag_prefix = nullptr;
@@ -1122,11 +1124,20 @@ static ccl_status launch(const GemmPlan& plan, const CUtensorMap& ma, const CUte
     cfg.blockDim = dim3(kGemmThreads, 1, 1);
     cfg.dynamicSmemBytes = plan.smem_bytes;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = CTAS; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    // Programmatic dependent launch (CCL_GEMM_PDL=0 turns it off): this kernel's CTAs may be placed, and run their set-up
+    // (parameters, barriers, TMEM, tensor-map prefetch), while the previous kernel in the stream drains; they touch
+    // global memory only after griddepcontrol.wait, i.e. after that kernel has completed and flushed.
+    static const bool pdl = []() { const char* f = std::getenv("CCL_GEMM_PDL"); return !f || atoi(f) != 0; }();
+    if (pdl) {
+        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[1].val.programmaticStreamSerializationAllowed = 1;
+        cfg.numAttrs = 2;
+    }
     CCL_CUDA_TRY(cudaLaunchKernelEx(&cfg, ccl_gemm_kernel<BN, CTAS, SWIGLU>, ma, mb, mc, plan.p));
     count_launch();
     return CCL_OK;
