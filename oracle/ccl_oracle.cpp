@@ -26,11 +26,13 @@
 // Pinning status (tests/test_oracle_*.py, no GPU needed):
 //   map / inverse : pinned (bijection, stride form of Sec. 3.3, Fig. 4(a)
 //                   worked example, reshape/permute, slice sizes of Sec. 2.2)
-//   repack        : pinned (permutation, round trip, strided-slice copies)
+//   repack        : pinned (permutation, round trip, strided-slice copies); the transposing form lives in
+//                   oracle/__init__.py (repack_transposed, written from the map; pinned by the Fig. 4(a) example)
 //   gemm          : pinned (identity, all-ones, library matmul, fp64 bound)
 //   gemm_axpby    : pinned (alpha = 1, beta = 0 is gemm; alpha = 0, beta = 1 returns C; exact small integers)
 //   gemm_swiglu   : pinned (gate/up pairing enumerated by hand, silu closed forms, numpy in float64)
-//   traffic_lru   : the finite-L2 model is this file's own reading of Sec. 4.1; pinned by its limits (one-line cache =
+//   traffic_lru   : the finite-L2 model (one CTA after the other, or waves in lockstep through K) is this file's own
+//                   reading of Sec. 4.1; pinned by its limits (one-line cache =
 //                   uncached count in whole lines, unbounded cache = ideal-L2 count, monotone in the ways) and a
 //                   hand-run example; against the paper's Fig. 6 numbers it is PARITY UNPINNED (unreleased simulator)
 //   traffic       : pinned by invariants, closed forms and a hand-enumerated
