@@ -358,6 +358,17 @@ typedef struct ccl_l2_model {
 } ccl_l2_model;
 ccl_status ccl_traffic_lru(const ccl_traffic_desc* d, const ccl_l2_model* m, uint64_t* totals_dev, void* cuda_stream);
 
+/*
+ * Experiment support (Sec. 2.1: chiplets with their own L2; a B200 is two dies behind one address space).  Launches
+ * `nctas` CTAs that cannot share an SM; CTA i records the SM it ran on in smid_dev[i] and, for each of `nlines` cache
+ * lines of a zero-filled device buffer (line j at byte offset j * stride_bytes), the mean round-trip time in SM clock
+ * cycles of 64 dependent loads that bypass L1, in lat_dev[i * nlines + j].  SMs of the die whose L2 partition holds
+ * a line see it faster than SMs of the other die: the rows of lat_dev cluster by die.
+ * zero_buf_dev must hold zeros over [0, (nlines - 1) * stride_bytes + 8); stride_bytes a positive multiple of 4.
+ */
+ccl_status ccl_probe_l2_latency(const void* zero_buf_dev, int32_t nlines, int64_t stride_bytes, int32_t nctas, float* lat_dev,
+                                int32_t* smid_dev, void* cuda_stream);
+
 /* Message for the last non-OK status returned on this thread ("" if none). Static storage. */
 const char* ccl_last_error(void);
 /* Number of CUDA kernels this library has launched in this process (all threads, all streams). */

@@ -20,7 +20,7 @@ PLACE_RR, PLACE_BLOCK, PLACE_BEST = 0, 1, 2
 ASSIGN_N_STRIPS, ASSIGN_M_STRIPS, ASSIGN_EXPLICIT = 0, 1, 2
 
 EXPORTS = ["ccl_map_offset", "ccl_map_inverse", "ccl_buffer_bytes", "ccl_strip_stride", "ccl_repack", "ccl_repack_batched", "ccl_repack_transpose", "ccl_gemm_workspace",
-           "ccl_gemm", "ccl_gemm_batched_workspace", "ccl_gemm_batched", "ccl_gemm_grouped", "ccl_gemm_grouped_swiglu", "ccl_gemm_axpby", "ccl_gemm_swiglu", "ccl_gemm_static_ws", "ccl_gemm_status", "ccl_traffic_sizes", "ccl_traffic", "ccl_traffic_l2", "ccl_traffic_lru", "ccl_last_error", "ccl_launch_count", "ccl_version"]
+           "ccl_gemm", "ccl_gemm_batched_workspace", "ccl_gemm_batched", "ccl_gemm_grouped", "ccl_gemm_grouped_swiglu", "ccl_gemm_axpby", "ccl_gemm_swiglu", "ccl_gemm_static_ws", "ccl_gemm_status", "ccl_traffic_sizes", "ccl_traffic", "ccl_traffic_l2", "ccl_traffic_lru", "ccl_probe_l2_latency", "ccl_last_error", "ccl_launch_count", "ccl_version"]
 
 
 class CclError(RuntimeError):
@@ -86,6 +86,7 @@ def lib():
         l.ccl_gemm.argtypes = [C.POINTER(GemmDesc), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         l.ccl_gemm_grouped.argtypes = [C.POINTER(GemmDesc), C.c_int32, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]
         l.ccl_gemm_grouped_swiglu.argtypes = l.ccl_gemm_grouped.argtypes
+        l.ccl_probe_l2_latency.argtypes = [C.c_void_p, C.c_int32, C.c_int64, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
         l.ccl_gemm_batched_workspace.argtypes = [C.POINTER(GemmDesc), C.c_int32, C.POINTER(C.c_size_t)]
         l.ccl_gemm_batched.argtypes = [C.POINTER(GemmDesc), C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64,
                                        C.c_void_p, C.c_size_t, C.c_void_p]
@@ -207,6 +208,16 @@ def ccl_gemm_batched(d, batch, A, a_stride, B, b_stride, Cout, c_stride, ws=None
             raise ValueError("ccl_gemm_batched: operand buffer too small")
     ws_bytes = ws.numel() * ws.element_size() if ws is not None else 0
     _check(lib().ccl_gemm_batched(C.byref(d), batch, _ptr(A), a_stride, _ptr(B), b_stride, _ptr(Cout), c_stride, _ptr(ws), ws_bytes, _stream()))
+
+
+def ccl_probe_l2_latency(zero_buf, nlines, stride_bytes, nctas):
+    """Returns (lat [nctas x nlines] float32 CUDA tensor of cycles per load, smid [nctas] int32 CUDA tensor)."""
+    if zero_buf.numel() * zero_buf.element_size() < (nlines - 1) * stride_bytes + 8:
+        raise ValueError("ccl_probe_l2_latency: buffer too small")
+    lat = torch.zeros((nctas, nlines), dtype=torch.float32, device=zero_buf.device)
+    smid = torch.zeros(nctas, dtype=torch.int32, device=zero_buf.device)
+    _check(lib().ccl_probe_l2_latency(_ptr(zero_buf), nlines, stride_bytes, nctas, _ptr(lat), _ptr(smid), _stream()))
+    return lat, smid
 
 
 def ccl_gemm_grouped_swiglu(d, groups, max_rows, row_offsets, A, B, b_stride_bytes, Cbuf):

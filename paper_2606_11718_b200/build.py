@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libccl.so")
-SOURCES = ["ccl_host.cpp", "ccl_tma.cpp", "ccl_repack.cu", "ccl_traffic.cu", "ccl_gemm.cu"]
+SOURCES = ["ccl_host.cpp", "ccl_tma.cpp", "ccl_repack.cu", "ccl_traffic.cu", "ccl_gemm.cu", "ccl_topo.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 
 

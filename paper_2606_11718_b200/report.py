@@ -312,6 +312,40 @@ def paper_sweep(out_dir, quick):
     json.dump(out, open(os.path.join(out_dir, "report_paper_sweep.json"), "w"), indent=1)
 
 
+def topology(out_dir):
+    """Which SMs share a die with which part of the L2 (an experiment, not part of the benchmark): every SM times
+    dependent L1-bypassing loads to 512 cache lines; after removing each line's and each SM's mean, the first singular
+    vector of the SM x line latency matrix splits the SMs and the lines into two sides."""
+    import numpy as np
+    nsm = torch.cuda.get_device_properties(0).multi_processor_count
+    nl = 512
+    buf = torch.zeros(8 << 20, dtype=torch.uint8, device="cuda")
+    sides = []
+    for rep in range(2):
+        lat, smid = ccl.ccl_probe_l2_latency(buf, nl, 4096 + 128 * rep, nsm)
+        torch.cuda.synchronize()
+        L, sm = lat.cpu().numpy().astype(np.float64), smid.cpu().numpy()
+        order = np.argsort(sm)
+        L, sm = L[order], sm[order]
+        X = L - L.mean(0, keepdims=True)
+        X = X - X.mean(1, keepdims=True)
+        U, S, Vt = np.linalg.svd(X, full_matrices=False)
+        side = U[:, 0] > 0
+        if not side[0]:
+            side = ~side
+        lines = X[side].mean(0) < 0                          # the lines this side of SMs reaches faster
+        near = (L[np.ix_(side, lines)].mean() + L[np.ix_(~side, ~lines)].mean()) / 2
+        far = (L[np.ix_(side, ~lines)].mean() + L[np.ix_(~side, lines)].mean()) / 2
+        sides.append(side)
+        print(f"topology run {rep}: {len(set(sm.tolist()))} SMs probed; singular values {S[0]:.0f}, {S[1]:.0f}, {S[2]:.0f}; sides of {int(side.sum())} and "
+              f"{int((~side).sum())} SMs; {int(lines.sum())} of {nl} lines nearer to the first side; mean load latency {near:.0f} cycles to the near "
+              f"half of the L2, {far:.0f} to the far half", flush=True)
+    agree = int((sides[0] == sides[1]).sum())
+    print(f"topology: the two runs put {agree} of {nsm} SMs on the same side; first side (by %smid): {sm[sides[0]].tolist()}", flush=True)
+    json.dump(dict(sm_count=nsm, side_of_sm={int(a): int(b) for a, b in zip(sm, sides[0])}, agree=agree),
+              open(os.path.join(out_dir, "report_topology.json"), "w"), indent=1)
+
+
 def extras(out_dir, quick, only=None):
     """The entry points around the plain GEMM, timed on the shapes they are meant for: the batch of expert GEMMs in one
     launch, the gated activation fused into the gate/up GEMM, and alpha/beta accumulation."""
@@ -468,6 +502,7 @@ def main():
     ap.add_argument("--lru-kslice", type=int, default=0, help="finite-L2 model: elements of K a wave consumes per lockstep step (0: all of K)")
     ap.add_argument("--l2-sweep", action="store_true", help="remote traffic against L2 capacity and data type under the finite-L2 model (then exit)")
     ap.add_argument("--paper-sweep", action="store_true", help="the 2 x 18-GEMM sweep of Sec. 4.2 under the finite-L2 model, both execution models (then exit)")
+    ap.add_argument("--topology", action="store_true", help="experiment: split the SMs into the two dies by their latency to the L2 (then exit)")
     ap.add_argument("--extras", action="store_true", help="time the batched, gated-activation, alpha/beta, transposing- and batched-repack entry points (then exit)")
     ap.add_argument("--only", default=None, help="run only the GEMMs whose name contains this text (e.g. for a profiler capture)")
     args = ap.parse_args()
@@ -477,6 +512,9 @@ def main():
     LRU_EXEC.update(wave_ctas=args.lru_wave, k_slice=args.lru_kslice)
     if args.paper_sweep:
         paper_sweep(args.out, args.quick)
+        return
+    if args.topology:
+        topology(args.out)
         return
     if args.extras:
         extras(args.out, args.quick, args.only)
