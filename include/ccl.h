@@ -188,6 +188,21 @@ ccl_status ccl_gemm_grouped_swiglu(const ccl_gemm_desc* d, int32_t groups, int64
                                    const void* A_dev, const void* B_dev, int64_t b_stride_bytes, void* C_dev, void* cuda_stream);
 
 /*
+ * A batch with RAGGED K: the weight gradients of the experts of an MoE layer (Sec. 4.1; dW_e = X_e^T * dY_e over the
+ * tokens routed to expert e).  Problem e contracts rows [k_offsets[e], k_offsets[e+1]) of A, stored [K x M]
+ * (a_trans = 1), and of B, stored [K x N] (b_trans = 0) -- K = d->K is the total row count of both -- into its own
+ * C [M x N] at C_dev + e * c_stride_bytes (layout d->C).  A problem without rows writes zeros.
+ *   k_offsets_dev  int32[groups + 1] on the DEVICE, non-decreasing, within [0, K]; read by the kernel.
+ * A and B row-major or CCL split along M / N, not split along K, not page-interleaved; C as for ccl_gemm_batched.
+ * The last 64-row block of a problem is cut at the problem's end: only its 16-row steps that hold rows of the problem
+ * are multiplied, and the rows of the last step that belong to the next problem are zeroed in shared memory first.
+ * Never split along K (no workspace); one CTA per tile.  Offsets outside [0, K] or decreasing: that problem's C is
+ * written as zeros and ccl_gemm_status() returns CCL_ERR_SHAPE (detail 5).
+ */
+ccl_status ccl_gemm_grouped_k(const ccl_gemm_desc* d, int32_t groups, const int32_t* k_offsets_dev, const void* A_dev,
+                              const void* B_dev, void* C_dev, int64_t c_stride_bytes, void* cuda_stream);
+
+/*
  * The BLAS form (Sec. 2.2: "the extension to alpha*A*B + beta*C is straightforward, since the scalars do not affect
  * placement and the C read shares the same partitioning as the output write"):
  *   C <- bf16( alpha * (A*B) + beta * C ),  fp32 arithmetic on the fp32 accumulator, one rounding.

@@ -20,7 +20,7 @@ PLACE_RR, PLACE_BLOCK, PLACE_BEST = 0, 1, 2
 ASSIGN_N_STRIPS, ASSIGN_M_STRIPS, ASSIGN_EXPLICIT = 0, 1, 2
 
 EXPORTS = ["ccl_map_offset", "ccl_map_inverse", "ccl_buffer_bytes", "ccl_strip_stride", "ccl_repack", "ccl_repack_batched", "ccl_repack_transpose", "ccl_gemm_workspace",
-           "ccl_gemm", "ccl_gemm_batched_workspace", "ccl_gemm_batched", "ccl_gemm_grouped", "ccl_gemm_grouped_swiglu", "ccl_gemm_axpby", "ccl_gemm_swiglu", "ccl_gemm_static_ws", "ccl_gemm_status", "ccl_traffic_sizes", "ccl_traffic", "ccl_traffic_l2", "ccl_traffic_lru", "ccl_probe_l2_latency", "ccl_last_error", "ccl_launch_count", "ccl_version"]
+           "ccl_gemm", "ccl_gemm_batched_workspace", "ccl_gemm_batched", "ccl_gemm_grouped", "ccl_gemm_grouped_swiglu", "ccl_gemm_grouped_k", "ccl_gemm_axpby", "ccl_gemm_swiglu", "ccl_gemm_static_ws", "ccl_gemm_status", "ccl_traffic_sizes", "ccl_traffic", "ccl_traffic_l2", "ccl_traffic_lru", "ccl_probe_l2_latency", "ccl_last_error", "ccl_launch_count", "ccl_version"]
 
 
 class CclError(RuntimeError):
@@ -87,6 +87,7 @@ def lib():
         l.ccl_gemm_grouped.argtypes = [C.POINTER(GemmDesc), C.c_int32, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]
         l.ccl_gemm_grouped_swiglu.argtypes = l.ccl_gemm_grouped.argtypes
         l.ccl_probe_l2_latency.argtypes = [C.c_void_p, C.c_int32, C.c_int64, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
+        l.ccl_gemm_grouped_k.argtypes = [C.POINTER(GemmDesc), C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]
         l.ccl_gemm_batched_workspace.argtypes = [C.POINTER(GemmDesc), C.c_int32, C.POINTER(C.c_size_t)]
         l.ccl_gemm_batched.argtypes = [C.POINTER(GemmDesc), C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64,
                                        C.c_void_p, C.c_size_t, C.c_void_p]
@@ -218,6 +219,13 @@ def ccl_probe_l2_latency(zero_buf, nlines, stride_bytes, nctas):
     smid = torch.zeros(nctas, dtype=torch.int32, device=zero_buf.device)
     _check(lib().ccl_probe_l2_latency(_ptr(zero_buf), nlines, stride_bytes, nctas, _ptr(lat), _ptr(smid), _stream()))
     return lat, smid
+
+
+def ccl_gemm_grouped_k(d, groups, k_offsets, A, B, Cbuf, c_stride_bytes):
+    """Ragged K: problem e contracts rows [k_offsets[e], k_offsets[e + 1]) of A [K x M] and B [K x N] into its own C."""
+    if k_offsets.dtype != torch.int32 or not k_offsets.is_cuda or k_offsets.numel() < groups + 1:
+        raise ValueError("ccl_gemm_grouped_k: k_offsets must be an int32 CUDA tensor with groups + 1 entries")
+    _check(lib().ccl_gemm_grouped_k(C.byref(d), groups, _ptr(k_offsets), _ptr(A), _ptr(B), _ptr(Cbuf), c_stride_bytes, _stream()))
 
 
 def ccl_gemm_grouped_swiglu(d, groups, max_rows, row_offsets, A, B, b_stride_bytes, Cbuf):

@@ -125,6 +125,8 @@ struct GemmParams {
     // ragged batch (ccl_gemm_grouped): problem e owns rows [m_offs[e], m_offs[e + 1]) of A and C; the tile grid of a
     // problem is laid out for Wm rows (the caller's bound) and tiles past a problem's last row are skipped
     const int32_t* m_offs;
+    // ragged K (ccl_gemm_grouped_k): problem e contracts rows [k_offs[e], k_offs[e + 1]) of A [K x M] and B [K x N]
+    const int32_t* k_offs;
     int32_t rag_dense;              // 1: the CTA builds a prefix of the problems' tile counts and walks only real tiles
     FastDiv fd_tiles_n;
     OpMap a, b;
@@ -275,6 +277,18 @@ __device__ __forceinline__ int64_t c_offset(const GemmParams& p, int64_t m, int6
         return (((int64_t)rr * p.c_cpr + cj) * p.c_nstrips + g) * p.c_ichunk + x;
     }
     return (int64_t)g * p.c_stride + (int64_t)rr * p.c_row + xx;
+}
+
+// Ragged K: first row, k blocks and rows of the last block of problem e (an empty or out-of-range problem: one block of
+// zero rows, so that its output is written as zeros).
+struct KRange { int k0, nkb, rem; };
+__device__ __forceinline__ KRange k_range(const int32_t* k_offs, int e, int Ktot) {
+    const int o0 = __ldg(k_offs + e), o1 = __ldg(k_offs + e + 1);
+    KRange r;
+    if (o0 < 0 || o1 > Ktot || o1 < o0) { atomicExch(&g_gemm_status, 5); r.k0 = 0; r.nkb = 1; r.rem = 0; return r; }
+    const int cnt = o1 - o0;
+    r.k0 = o0; r.nkb = cnt > 0 ? (cnt + BK - 1) / BK : 1; r.rem = cnt - (r.nkb - 1) * BK;
+    return r;
 }
 
 struct TileCoord { int m0, m1, n0, n1, split, e; bool skip; };   // e: problem of the batch; skip: an empty tile of a ragged batch
@@ -482,7 +496,8 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             if (SWIGLU && !isA) base += (p.fd_wn.div(t.n0) + hsel) * p.pair_dist;
             int x, y, z, u;
             if (mn) to_coords(om, 0, base, x, y, z, u); else to_coords(om, base, 0, x, y, z, u);
-            const int kb0 = t.split * kbps, kb1 = min(num_kb, kb0 + kbps);
+            int kb0 = t.split * kbps, kb1 = min(num_kb, kb0 + kbps), kbase = 0;
+            if (p.k_offs) { const KRange kr = k_range(p.k_offs, t.e, p.K); kb0 = 0; kb1 = kr.nkb; kbase = kr.k0; }
             if (lane == 0 && it == 0) CCL_TRACE(11);
             for (int kb = kb0; kb < kb1; ++kb) {
                 ok = mbar_wait_bounded(&empty[stage], phase ^ 1);
@@ -492,7 +507,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 if (!ok) { if (lane == 0) atomicExch(&g_gemm_status, 1); break; }
                 // (the byte count may be posted after a copy has completed: the phase cannot end before this arrival)
                 if (post_tx) mbar_expect_tx(&full[stage], stage_bytes * CTAS);
-                const int k0 = kb * BK;
+                const int k0 = kbase + kb * BK;
                 if (ksplit) { if (mn) to_coords(om, k0, base, x, y, z, u); else to_coords(om, base, k0, x, y, z, u); }
                 else if (mn) y = k0; else x = k0;
                 if (lane == 0 && it == 0 && kb == kb0) CCL_TRACE(13);
@@ -524,7 +539,8 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 const int acc0 = NSUB == 1 ? (done & 1) : 0;
                 const uint32_t acc_phase = NSUB == 1 ? ((uint32_t)(done >> 1) & 1) : ((uint32_t)done & 1);
                 ++done;
-                const int kb0 = t.split * kbps, kb1 = min(num_kb, kb0 + kbps);
+                int kb0 = t.split * kbps, kb1 = min(num_kb, kb0 + kbps), tail = BK;
+                if (p.k_offs) { const KRange kr = k_range(p.k_offs, t.e, p.K); kb0 = 0; kb1 = kr.nkb; tail = kr.rem; }
                 for (int kb = kb0; ok && kb < kb1; ++kb) {
                     // (the copies' completion on the barrier orders the operand bytes before the MMAs that read them;
                     // tcgen05 fences are only needed around the accumulator hand-over below)
@@ -533,6 +549,20 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     CCL_TRACE2(it == 0 && kb - kb0 < 16, 96 + (kb - kb0) * 2);
                     const uint32_t sa = smem0 + (uint32_t)stage * stage_bytes;
                     const uint64_t adesc = smem_desc(sa, a_lbo, 1024);
+                    // Ragged K, last block of a problem: only the 16-row k steps that hold rows of this problem are
+                    // issued, and the rows of the last step that belong to the next problem are zeroed in shared memory
+                    // (both operands are [k][64 columns] boxes of 128-byte rows here, so a k row is a whole line).
+                    int ksteps = BK / 16;
+                    if (tail < BK && kb == kb1 - 1) {
+                        ksteps = tail > 0 ? (tail + 15) / 16 : 1;
+                        const int nboxes = (int)(stage_bytes / (64 * BK * 2));
+                        for (int r = tail; r < ksteps * 16; ++r)
+                            for (int b = 0; b < nboxes; ++b)
+#pragma unroll
+                                for (int c = 0; c < 8; ++c)
+                                    asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(sa + (uint32_t)(b * 64 * BK * 2 + r * 128 + c * 16)), "r"(0u) : "memory");
+                        fence_proxy_async();
+                    }
 #pragma unroll
                     for (int h = 0; h < NSUB; ++h) {
                         if (kb == kb0) {
@@ -543,7 +573,8 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                         const uint64_t bdesc = smem_desc(sa + a_bytes + h * (SUBH * BK * 2), b_lbo, 1024);
 #pragma unroll
                         for (int k = 0; k < BK / 16; ++k)
-                            umma_bf16<CTAS>(tmem_d, adesc + (uint64_t)(k * a_kstep), bdesc + (uint64_t)(k * b_kstep), idesc, ((kb - kb0) | k) != 0);
+                            if (k < ksteps)
+                                umma_bf16<CTAS>(tmem_d, adesc + (uint64_t)(k * a_kstep), bdesc + (uint64_t)(k * b_kstep), idesc, ((kb - kb0) | k) != 0);
                     }
                     if (!ok) break;
                     umma_commit<CTAS>(&empty[stage]);          // frees the stage (in both CTAs) once these MMAs have read it
@@ -861,8 +892,9 @@ static ccl_status merge_width(int64_t* cur, int64_t w, const char* dim) {
 
 // units = schedulable CTAs (1-CTA kernel) or CTA pairs (2-CTA kernel) the device can hold at once
 // cap > 0: a ragged batch -- the tile grid of one problem covers `cap` rows, d->M is the total row count of A and C
+// ragk: a batch with ragged K -- d->K is the total row count of the concatenated A [K x M] and B [K x N]
 static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, const void* A, const void* B, const void* C, int sms, int pairs, GemmPlan* plan,
-                            int64_t cap = 0) {
+                            int64_t cap = 0, bool ragk = false) {
     if (!d) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: NULL descriptor");
     if (d->M <= 0 || d->N <= 0 || d->K <= 0) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: M, N, K must be positive");
     if (d->M >= (INT64_C(1) << 31) || d->N >= (INT64_C(1) << 31) || d->K >= (INT64_C(1) << 31)) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: dimension too large");
@@ -919,6 +951,8 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     }
     int64_t ka = split_width(va, at), kb = split_width(vb, !bt);
     if ((ka && ka % BK) || (kb && kb % BK)) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: an operand split along K needs strips that are multiples of %d", BK);
+    if (ragk && (!at || bt || ka || kb || il_a || il_b))
+        return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm_grouped_k: A must be stored [K x M] and B [K x N], neither split along K nor page-interleaved");
     const int64_t Mt = cap > 0 ? cap : d->M;            // rows the tile grid of one problem covers
     if (cap > 0 && Wm) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm_grouped: A and C must not be split along M");
     if (!Wm) Wm = Mt;
@@ -939,7 +973,7 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     //   tile exposes it (~7000 cycles); split-K adds the partial-sum traffic and a second launch.
     // 256 x 512 pair tiles move the fewest bytes per flop and win once K is long; short problems prefer the
     // variant whose tile count fills the machine.
-    const int64_t num_kb = (d->K + BK - 1) / BK;
+    const int64_t num_kb = ((ragk ? std::max<int64_t>(1, d->K / batch) : d->K) + BK - 1) / BK;   // (ragged K: the mean, for the cost model only)
     const int64_t strips_m = Mt / Wm, strips_n = Nc / Wn;
     int ctas = 1, bn = 256, splits = 1;
     double best = -1.0;
@@ -949,7 +983,7 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     const char* force_bn = std::getenv("CCL_GEMM_BN");
     const char* force_split = std::getenv("CCL_GEMM_SPLITK");
     for (int c = 1; c <= 2; ++c) {
-        if (c == 2 && pairs <= 0) continue;
+        if (c == 2 && (pairs <= 0 || ragk)) continue;          // (a ragged-K tail is zeroed by the CTA that issues the MMAs)
         if (force_ctas && atoi(force_ctas) != c) continue;
         const int units = c == 2 ? pairs : sms;
         for (int b : {512, 256, 192, 128}) {
@@ -969,7 +1003,7 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
             const double stream_clk = tiles_m_all == 1 ? (double)tiles * (double)num_kb * (double)b * (BK * 2) / (sms * 29.0) *
                                                              (b <= 128 ? 1.10 : (b <= 192 ? 1.04 : 1.0)) : 0.0;
             for (int sp : {1, 2, 3, 4, 6, 8, 12, 16}) {
-                if (sp > 1 && (swiglu || cap > 0 || num_kb / sp < 2)) continue;
+                if (sp > 1 && (swiglu || cap > 0 || ragk || num_kb / sp < 2)) continue;
                 if (force_split && atoi(force_split) != sp) continue;
                 const int64_t kbps = (num_kb + sp - 1) / sp;
                 const int64_t sp_eff = (num_kb + kbps - 1) / kbps;          // every split owns at least one k block
@@ -1241,7 +1275,7 @@ extern "C" ccl_status ccl_gemm_batched_workspace(const ccl_gemm_desc* d, int32_t
 // m_offs / cap: ragged batch (ccl_gemm_grouped), else nullptr / 0
 static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, const int64_t* strides, const void* A_dev, const void* B_dev, void* C_dev,
                             void* ws_dev, size_t ws_bytes, void* cuda_stream, float alpha = 1.0f, float beta = 0.0f, const int32_t* m_offs = nullptr,
-                            int64_t cap = 0) {
+                            int64_t cap = 0, const int32_t* k_offs = nullptr) {
     if (!A_dev || !B_dev || !C_dev) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: NULL operand");
     if (!d) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: NULL descriptor");
     if (batch < 1 || batch > kMaxBatch) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: batch must be in [1, %lld]", (long long)kMaxBatch);
@@ -1251,7 +1285,7 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     PreparedKey key;
     make_key(d, batch4, A_dev, B_dev, C_dev, &key);
     key.mode = swiglu ? 1 : 0; key.alpha = alpha; key.beta = beta;
-    key.f[36] = (int64_t)reinterpret_cast<uintptr_t>(m_offs); key.f[37] = cap;
+    key.f[36] = (int64_t)reinterpret_cast<uintptr_t>(m_offs) ^ ((int64_t)reinterpret_cast<uintptr_t>(k_offs) << 1); key.f[37] = cap + (k_offs ? (INT64_C(1) << 62) : 0);
     Prepared prep;
     bool hit = false;
     {
@@ -1262,7 +1296,7 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     ccl_status s;
     if (!hit) {
         GemmPlan& plan = prep.plan;
-        s = make_plan(d, batch, swiglu, A_dev, B_dev, C_dev, 148, 74, &plan, cap);     // validation first: no CUDA call on bad input
+        s = make_plan(d, batch, swiglu, A_dev, B_dev, C_dev, 148, 74, &plan, cap, k_offs != nullptr);     // validation first: no CUDA call on bad input
         if (s) return s;
         if (batch > 1) {
             const MatView* views[3] = {&plan.va, &plan.vb, &plan.vc};
@@ -1281,12 +1315,13 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
         if (dev != key.dev) {
             make_key(d, batch4, A_dev, B_dev, C_dev, &key);
             key.mode = swiglu ? 1 : 0; key.alpha = alpha; key.beta = beta;
-            key.f[36] = (int64_t)reinterpret_cast<uintptr_t>(m_offs); key.f[37] = cap;
+            key.f[36] = (int64_t)reinterpret_cast<uintptr_t>(m_offs) ^ ((int64_t)reinterpret_cast<uintptr_t>(k_offs) << 1); key.f[37] = cap + (k_offs ? (INT64_C(1) << 62) : 0);
         }
-        if ((s = make_plan(d, batch, swiglu, A_dev, B_dev, C_dev, prep.sms, resident_pairs(), &plan, cap))) return s;
+        if ((s = make_plan(d, batch, swiglu, A_dev, B_dev, C_dev, prep.sms, resident_pairs(), &plan, cap, k_offs != nullptr))) return s;
         plan.p.C = static_cast<uint16_t*>(C_dev);
         plan.p.a.batched = batch4[1] != 0; plan.p.b.batched = batch4[2] != 0; plan.p.c.batched = m_offs ? 0 : 1;
         plan.p.m_offs = m_offs;
+        plan.p.k_offs = k_offs;
         plan.p.c_batch_stride = batch4[3] / 2;
         plan.p.alpha = alpha; plan.p.beta = beta; plan.p.axpby = (alpha != 1.0f || beta != 0.0f) ? 1 : 0;
         const uint32_t bnh = (uint32_t)(plan.subn / plan.ctas);   // B rows of one K-major box
@@ -1363,6 +1398,16 @@ extern "C" ccl_status ccl_gemm_grouped(const ccl_gemm_desc* d, int32_t groups, i
 extern "C" ccl_status ccl_gemm_grouped_swiglu(const ccl_gemm_desc* d, int32_t groups, int64_t max_rows, const int32_t* row_offsets_dev,
                                               const void* A_dev, const void* B_dev, int64_t b_stride_bytes, void* C_dev, void* cuda_stream) {
     return grouped_impl(d, true, groups, max_rows, row_offsets_dev, A_dev, B_dev, b_stride_bytes, C_dev, cuda_stream);
+}
+
+extern "C" ccl_status ccl_gemm_grouped_k(const ccl_gemm_desc* d, int32_t groups, const int32_t* k_offsets_dev, const void* A_dev, const void* B_dev,
+                                         void* C_dev, int64_t c_stride_bytes, void* cuda_stream) {
+    if (!d) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm_grouped_k: NULL descriptor");
+    if (!k_offsets_dev) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm_grouped_k: NULL offsets");
+    if (reinterpret_cast<uintptr_t>(k_offsets_dev) & 3) return fail(CCL_ERR_ALIGN, "ccl_gemm_grouped_k: offsets are not 4-byte aligned");
+    if (c_stride_bytes < 0) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm_grouped_k: negative stride");
+    const int64_t strides[3] = {0, 0, c_stride_bytes};
+    return gemm_impl(d, groups, false, strides, A_dev, B_dev, C_dev, nullptr, 0, cuda_stream, 1.0f, 0.0f, nullptr, 0, k_offsets_dev);
 }
 
 extern "C" ccl_status ccl_gemm_axpby(const ccl_gemm_desc* d, float alpha, float beta, const void* A_dev, const void* B_dev, void* C_dev,

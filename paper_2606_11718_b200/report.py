@@ -438,6 +438,35 @@ def extras(out_dir, quick, only=None):
                   f"with down {t_f * 1e3:7.1f} us ({fl / (t_f * 1e-3) / 1e12:6.0f} TFLOP/s)", flush=True)
         except ccl.CclError as err:
             print(f"extras MoE FFN forward: not supported in this form ({err})", flush=True)
+    # 1d. the weight gradients of the experts: ragged K in one launch
+    for E, T, H, I in (((128, 32768, 2048, 768),) if not quick else ((32, 8192, 2048, 768),)) if want("moe_wgrad") else ():
+        import numpy as np
+        wts = np.random.default_rng(3).dirichlet(np.full(E, 2.0))
+        counts = np.floor(wts * T).astype(np.int64)
+        counts[0] += T - counts.sum()
+        offs = torch.from_numpy(np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)).to(dev)
+        bounds = [int(x) for x in offs.cpu()]
+        for name, M, N in (("down: act^T x dY", I, H), ("gate/up: X^T x dAct", H, 2 * I)):
+            d = ccl.GemmDesc()
+            d.M, d.N, d.K = M, N, T
+            d.A = ccl.Mat(T, M, 2)                                    # stored [K x M]
+            d.B = ccl.Mat(T, N, 2)
+            d.C = ccl.Mat(M, N, 2, 4, ccl.PART_COLS, ccl.CCL, 4096)   # the gradient in the layout of the weight
+            d.a_trans, d.b_trans, d.out_part, d.P, d.grouped_raster = 1, 0, ccl.PART_COLS, 4, 1
+            A, B, Cb = buf(d.A), buf(d.B), buf(d.C, E)
+            sc = ccl.ccl_buffer_bytes(d.C)
+            t_g = timed(lambda: ccl.ccl_gemm_grouped_k(d, E, offs, A, B, Cb, sc), 20)
+            Av, Bv = A.view(T, M), B.view(T, N)
+
+            def torch_loop():
+                for e in range(E):
+                    if bounds[e + 1] > bounds[e]:
+                        torch.matmul(Av[bounds[e]:bounds[e + 1]].t(), Bv[bounds[e]:bounds[e + 1]])
+            t_t = timed(torch_loop, 3)
+            tf = 2.0 * T * M * N / (t_g * 1e-3) / 1e12
+            rows.append(dict(what="moe_wgrad", name=name, experts=E, tokens=T, M=M, N=N, grouped_k_ms=t_g, torch_loop_ms=t_t, tflops=tf))
+            print(f"extras MoE weight gradient ({name}), {E} experts, {T} routed tokens, {M} x {N} each: one launch {t_g * 1e3:8.1f} us ({tf:6.0f} TFLOP/s) | "
+                  f"torch.matmul per expert {t_t * 1e3:8.1f} us", flush=True)
     # 2. gate/up GEMM with the gated activation in the epilogue against GEMM + elementwise kernel
     for M, N, K in (((8192, 57344, 8192), (16384, 1536, 2048)) if not quick else ((1024, 57344, 8192),)) if want("swiglu") else ():
         d0, d1 = desc(M, N, K, 4), desc(M, N, K, 4, c_cols=N // 2)

@@ -140,6 +140,19 @@ def test_gemm_grouped_rejects_bad_input_before_any_launch():
     assert call(gemm_desc(1024, 768, 512, 4, ("ccl", "row", "ccl"), out_part=1)) == ccl.ERR_UNSUPPORTED    # split along M
 
 
+def test_gemm_grouped_k_rejects_bad_input_before_any_launch():
+    l = ccl.lib()
+    d = gemm_desc(768, 2048, 4096, 4, ("row", "ccl", "ccl"), a_trans=1)
+    call = lambda dd, groups=4, offs=65536, c_stride=768 * 2048 * 2: l.ccl_gemm_grouped_k(
+        C.byref(dd), groups, C.c_void_p(offs), C.c_void_p(4096), C.c_void_p(8192), C.c_void_p(16384), c_stride, None)
+    assert call(d, offs=None) == ccl.ERR_INVALID_ARG
+    assert call(d, offs=65537) == ccl.ERR_ALIGN
+    assert call(d, c_stride=-2) == ccl.ERR_INVALID_ARG
+    assert call(d, c_stride=1024) == ccl.ERR_INVALID_ARG                                        # smaller than one C
+    assert call(gemm_desc(768, 2048, 4096, 4, ("row", "ccl", "ccl"))) == ccl.ERR_UNSUPPORTED   # A stored [M x K]
+    assert call(gemm_desc(768, 2048, 4096, 4, ("row", "ccl", "ccl"), a_trans=1, b_trans=1)) == ccl.ERR_UNSUPPORTED
+
+
 def gemm_rc(d, a=4096, b=8192, c=16384):
     return ccl.lib().ccl_gemm(C.byref(d), C.c_void_p(a), C.c_void_p(b), C.c_void_p(c), None, 0, None)
 

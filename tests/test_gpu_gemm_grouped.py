@@ -181,3 +181,75 @@ def test_grouped_swiglu_equals_oracle(N, K, P, lay, bt, counts, walk):
         os.environ.pop("CCL_GEMM_RAGGED_DENSE", None)
         if saved is not None:
             os.environ["CCL_GEMM_RAGGED_DENSE"] = saved
+
+
+RAGGED_K = [
+    # M, N, P, layouts, counts (rows of K per problem)
+    (768, 512, 4, ("row", "ccl", "ccl"), [256, 0, 37, 300, 1, 128, 64, 17]),      # expert weight gradients, ragged token counts
+    (256, 384, 2, ("row", "ccl", "ccl"), [130, 5, 260, 16, 15, 49]),
+    (128, 256, 1, ("row", "row", "row"), [64, 64, 128]),                          # whole blocks only
+    (256, 1024, 4, ("ccl", "ccl", "row"), [1000, 3]),                             # A split along M, C row-major
+]
+
+
+@pytest.mark.parametrize("M,N,P,lay,counts", RAGGED_K)
+@pytest.mark.parametrize("bn", ["auto", "128", "192", "256"])
+def test_grouped_k_equals_oracle(M, N, P, lay, counts, bn):
+    """Ragged K (the weight gradients of the experts): problem e contracts its own rows of A [K x M] and B [K x N]."""
+    saved = os.environ.pop("CCL_GEMM_BN", None)
+    if bn != "auto":
+        os.environ["CCL_GEMM_BN"] = bn
+    try:
+        E = len(counts)
+        offs = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
+        K = int(offs[-1]) + 11                                          # eleven rows no problem owns
+        parts = (2 if lay[0] == "ccl" else 0, 2, 2)                      # A [K x M] split along M, B [K x N] and C along N
+        d = gemm_desc(M, N, K, P, lay, 1, 0, 2, 1, parts=parts)
+        d.C = ccl.Mat(M, N, 2, d.C.P, d.C.part, d.C.layout, d.C.strip_align_bytes)
+        A, B = synth.gemm_operands(M, N, K, 1, 0, seed=7, tag="grouped_k")
+        a_bits, b_bits = synth.bits(A), synth.bits(B)
+        try:
+            sc = pad16(ccl.ccl_buffer_bytes(d.C)) + 64
+            c_dev = torch.full((E * sc // 2 + 4096,), POISON, dtype=torch.int16, device="cuda")
+            ccl.ccl_gemm_grouped_k(d, E, torch.from_numpy(offs).cuda(), to_layout(a_bits, d.A), to_layout(b_bits, d.B), c_dev, sc)
+        except ccl.CclError as e:
+            assert e.status == ccl.ERR_UNSUPPORTED
+            pytest.skip("tile width not available for this operand layout")
+        assert ccl.ccl_gemm_status()[0] == ccl.OK
+        nc = ccl.ccl_buffer_bytes(d.C) // 2
+        buf = c_dev[:E * sc // 2].view(E, sc // 2)
+        assert (buf[:, nc:] == POISON).all() and (c_dev[E * sc // 2:] == POISON).all(), "wrote between or past the outputs"
+        for e in range(E):
+            o0, o1 = int(offs[e]), int(offs[e + 1])
+            got = synth.from_bits(from_layout(buf[e, :nc], d.C)).to(torch.float32).numpy()
+            if o1 == o0:
+                assert (got == 0).all(), f"problem {e} has no rows: its output is zero"
+                continue
+            ref32, _, _ = orc.gemm(a_bits[o0:o1], b_bits[o0:o1], M, N, o1 - o0, 1, 0)
+            assert np.isfinite(got).all()
+            err = np.abs(got - ref32) / np.maximum(1.0, np.abs(ref32))
+            assert err.max() <= tol(max(o1 - o0, 64)), (e, o1 - o0, err.max())
+    finally:
+        os.environ.pop("CCL_GEMM_BN", None)
+        if saved is not None:
+            os.environ["CCL_GEMM_BN"] = saved
+
+
+def test_grouped_k_neighbours_do_not_leak():
+    """The rows after a problem's last row belong to its neighbour: huge values there must not reach the result."""
+    M, N, counts = 128, 256, [37, 90]
+    offs = np.array([0, 37, 127], dtype=np.int32)
+    K = 127
+    d = gemm_desc(M, N, K, 1, ("row", "row", "row"), 1, 0, 0, 0)
+    A, B = synth.gemm_operands(M, N, K, 1, 0, seed=8, tag="grouped_k_leak")
+    a_bits, b_bits = synth.bits(A).copy(), synth.bits(B).copy()
+    a_bits[37:40] = 0x7F00                                              # ~1.7e38 in the first rows of the second problem
+    b_bits[37:40] = 0x7F80                                              # +inf
+    nc = M * N
+    c_dev = torch.full((2 * nc,), POISON, dtype=torch.int16, device="cuda")
+    ccl.ccl_gemm_grouped_k(d, 2, torch.from_numpy(offs).cuda(), to_layout(a_bits, d.A), to_layout(b_bits, d.B), c_dev, nc * 2)
+    assert ccl.ccl_gemm_status()[0] == ccl.OK
+    got = synth.from_bits(c_dev[:nc].cpu().numpy().view(np.uint16).reshape(M, N)).to(torch.float32).numpy()
+    ref32, _, _ = orc.gemm(a_bits[:37], b_bits[:37], M, N, 37, 1, 0)
+    assert np.isfinite(got).all()
+    assert (np.abs(got - ref32) / np.maximum(1.0, np.abs(ref32))).max() <= tol(64)
