@@ -330,8 +330,9 @@ struct Scheduler {
         t.n0 = sn * p.Wn + jn * bn; t.n1 = min(t.n0 + bn, (sn + 1) * p.Wn);
         return true;
     }
+    template <int RAG>
     __device__ bool get(int it, TileCoord& t) const {
-        if (rag) return get_ragged(it, t);
+        if (RAG == 1 && rag) return get_ragged(it, t);
         int g, i;
         if (it < rounds && my_g >= 0) { g = my_g; i = idx + it * upg; }
         else {
@@ -360,7 +361,7 @@ struct Scheduler {
         t.m0 = sm * p.Wm + jm * bm; t.m1 = min(t.m0 + bm, (sm + 1) * p.Wm);
         t.n0 = sn * p.Wn + jn * bn; t.n1 = min(t.n0 + bn, (sn + 1) * p.Wn);
         t.skip = false;
-        if (p.m_offs) {                                  // rows of this problem inside the concatenated A and C
+        if (RAG == 1 && p.m_offs) {                      // rows of this problem inside the concatenated A and C
             const int o0 = __ldg(p.m_offs + t.e), o1 = __ldg(p.m_offs + t.e + 1);
             const bool bad = o0 < 0 || o1 > p.M || o1 - o0 > p.Wm;   // outside A / C, or more rows than the caller's bound:
             if (bad && t.m0 == 0 && t.n0 == 0) atomicExch(&g_gemm_status, 5);   // reported, and the problem is left out
@@ -371,7 +372,9 @@ struct Scheduler {
     }
 };
 
-template <int BN, int CTAS, bool SWIGLU = false>
+// RAG: 1 = ragged M (ccl_gemm_grouped), 2 = ragged K (ccl_gemm_grouped_k) -- instantiations of their own, so that the tile
+// walk and the k loops of all other calls stay as they are (the extra branches cost 1-1.5 us on a 15-30 us GEMM)
+template <int BN, int CTAS, bool SWIGLU = false, int RAG = 0>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                 const __grid_constant__ CUtensorMap map_c, const __grid_constant__ GemmParams gp) {
@@ -428,7 +431,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 
     // Ragged batch with a dense walk: m-tiles of every problem, as an exclusive prefix over the problems.
     int* rag_prefix = nullptr;
-    if (p.rag_dense) {
+    if (RAG == 1 && p.rag_dense) {
         int* part = reinterpret_cast<int*>(tmem_ptr + 4);           // one partial sum per thread, then the prefix itself
         rag_prefix = part + kGemmThreads;
         const int E = p.batch, bm = BM * CTAS, per = (E + kGemmThreads - 1) / kGemmThreads;
@@ -489,7 +492,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         const int stages = p.stages, num_kb = p.num_kb, kbps = p.kb_per_split;
         const uint32_t stage_bytes = p.stage_bytes;
         const bool post_tx = lane == 0 && leader;
-        for (int it = 0; ok && sched.get(it, t); ++it) {
+        for (int it = 0; ok && sched.template get<RAG>(it, t); ++it) {
             if (t.skip) continue;
             int base = (isA ? t.m0 : t.n0) + off;
             // output column n0 of strip g -> B column n0 + g * pair_dist (gate) and one pair_dist further (up)
@@ -497,7 +500,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             int x, y, z, u;
             if (mn) to_coords(om, 0, base, x, y, z, u); else to_coords(om, base, 0, x, y, z, u);
             int kb0 = t.split * kbps, kb1 = min(num_kb, kb0 + kbps), kbase = 0;
-            if (p.k_offs) { const KRange kr = k_range(p.k_offs, t.e, p.K); kb0 = 0; kb1 = kr.nkb; kbase = kr.k0; }
+            if (RAG == 2) { const KRange kr = k_range(p.k_offs, t.e, p.K); kb0 = 0; kb1 = kr.nkb; kbase = kr.k0; }
             if (lane == 0 && it == 0) CCL_TRACE(11);
             for (int kb = kb0; kb < kb1; ++kb) {
                 ok = mbar_wait_bounded(&empty[stage], phase ^ 1);
@@ -531,7 +534,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             const int stages = p.stages, num_kb = p.num_kb, kbps = p.kb_per_split;
             const uint32_t stage_bytes = p.stage_bytes, a_bytes = p.a_bytes, idesc = p.idesc, smem0 = smem_u32(smem);
             int done = 0;                                   // tiles computed so far (empty tiles of a ragged batch do not count)
-            for (int it = 0; ok && sched.get(it, t); ++it) {
+            for (int it = 0; ok && sched.template get<RAG>(it, t); ++it) {
                 if (t.skip) continue;
                 // NSUB == 1: TMEM half (done & 1) is this tile's accumulator, the other half is being drained.
                 // NSUB == 2: both halves belong to this tile; half h may be overwritten once the epilogue
@@ -540,7 +543,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 const uint32_t acc_phase = NSUB == 1 ? ((uint32_t)(done >> 1) & 1) : ((uint32_t)done & 1);
                 ++done;
                 int kb0 = t.split * kbps, kb1 = min(num_kb, kb0 + kbps), tail = BK;
-                if (p.k_offs) { const KRange kr = k_range(p.k_offs, t.e, p.K); kb0 = 0; kb1 = kr.nkb; tail = kr.rem; }
+                if (RAG == 2) { const KRange kr = k_range(p.k_offs, t.e, p.K); kb0 = 0; kb1 = kr.nkb; tail = kr.rem; }
                 for (int kb = kb0; ok && kb < kb1; ++kb) {
                     // (the copies' completion on the barrier orders the operand bytes before the MMAs that read them;
                     // tcgen05 fences are only needed around the accumulator hand-over below)
@@ -552,8 +555,9 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     // Ragged K, last block of a problem: only the 16-row k steps that hold rows of this problem are
                     // issued, and the rows of the last step that belong to the next problem are zeroed in shared memory
                     // (both operands are [k][64 columns] boxes of 128-byte rows here, so a k row is a whole line).
+                    const bool cut = RAG == 2 && tail < BK && kb == kb1 - 1;
                     int ksteps = BK / 16;
-                    if (tail < BK && kb == kb1 - 1) {
+                    if (cut) {
                         ksteps = tail > 0 ? (tail + 15) / 16 : 1;
                         const int nboxes = (int)(stage_bytes / (64 * BK * 2));
                         for (int r = tail; r < ksteps * 16; ++r)
@@ -571,10 +575,15 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                         }
                         const uint32_t tmem_d = tmem_base + (uint32_t)((acc0 + h) * ACC_COLS);
                         const uint64_t bdesc = smem_desc(sa + a_bytes + h * (SUBH * BK * 2), b_lbo, 1024);
+                        if (!cut) {                           // (the common path keeps its four back-to-back MMAs)
 #pragma unroll
-                        for (int k = 0; k < BK / 16; ++k)
-                            if (k < ksteps)
+                            for (int k = 0; k < BK / 16; ++k)
                                 umma_bf16<CTAS>(tmem_d, adesc + (uint64_t)(k * a_kstep), bdesc + (uint64_t)(k * b_kstep), idesc, ((kb - kb0) | k) != 0);
+                        } else {
+#pragma unroll 1
+                            for (int k = 0; k < ksteps; ++k)
+                                umma_bf16<CTAS>(tmem_d, adesc + (uint64_t)(k * a_kstep), bdesc + (uint64_t)(k * b_kstep), idesc, ((kb - kb0) | k) != 0);
+                        }
                     }
                     if (!ok) break;
                     umma_commit<CTAS>(&empty[stage]);          // frees the stage (in both CTAs) once these MMAs have read it
@@ -597,7 +606,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         bool alive = true;
         uint32_t epi_count = 0;                          // TMA-stored pieces so far (selects the staging buffer)
         int done = 0;                                    // tiles drained so far
-        for (int it = 0; alive && sched.get(it, t); ++it) {
+        for (int it = 0; alive && sched.template get<RAG>(it, t); ++it) {
           if (t.skip) continue;
           const int tile_no = done++;
           const int m = t.m0 + (int)rank * BM + quad * 32 + lane;
@@ -1139,19 +1148,19 @@ static ccl_status operand_tmap(CUtensorMap* m, const MatView& v, const void* bas
     return encode_tmap(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, base, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
-template <int BN, int CTAS, bool SWIGLU = false>
+template <int BN, int CTAS, bool SWIGLU = false, int RAG = 0>
 static ccl_status configure(uint32_t smem_bytes) {
     static uint32_t configured_for = 0;
     if (configured_for < smem_bytes) {
-        CCL_CUDA_TRY(cudaFuncSetAttribute(ccl_gemm_kernel<BN, CTAS, SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes));
+        CCL_CUDA_TRY(cudaFuncSetAttribute(ccl_gemm_kernel<BN, CTAS, SWIGLU, RAG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes));
         configured_for = smem_bytes;
     }
     return CCL_OK;
 }
 
-template <int BN, int CTAS, bool SWIGLU = false>
+template <int BN, int CTAS, bool SWIGLU = false, int RAG = 0>
 static ccl_status launch(const GemmPlan& plan, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, cudaStream_t st) {
-    ccl_status s = configure<BN, CTAS, SWIGLU>(plan.smem_bytes);
+    ccl_status s = configure<BN, CTAS, SWIGLU, RAG>(plan.smem_bytes);
     if (s) return s;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(plan.grid, 1, 1);
@@ -1172,7 +1181,7 @@ static ccl_status launch(const GemmPlan& plan, const CUtensorMap& ma, const CUte
         attr[1].val.programmaticStreamSerializationAllowed = 1;
         cfg.numAttrs = 2;
     }
-    CCL_CUDA_TRY(cudaLaunchKernelEx(&cfg, ccl_gemm_kernel<BN, CTAS, SWIGLU>, ma, mb, mc, plan.p));
+    CCL_CUDA_TRY(cudaLaunchKernelEx(&cfg, ccl_gemm_kernel<BN, CTAS, SWIGLU, RAG>, ma, mb, mc, plan.p));
     count_launch();
     return CCL_OK;
 }
@@ -1345,7 +1354,20 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     }
     plan.p.ws = static_cast<float*>(ws_dev);
     cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
-    if (swiglu) s = launch<512, 2, true>(plan, ma, mb, mc, st);
+    if (k_offs) {                                        // ragged K: one CTA per tile (make_plan)
+        if (plan.bn == 256) s = launch<256, 1, false, 2>(plan, ma, mb, mc, st);
+        else if (plan.bn == 192) s = launch<192, 1, false, 2>(plan, ma, mb, mc, st);
+        else s = launch<128, 1, false, 2>(plan, ma, mb, mc, st);
+    } else if (m_offs) {                                 // ragged M
+        if (swiglu) s = launch<512, 2, true, 1>(plan, ma, mb, mc, st);
+        else if (plan.ctas == 2) {
+            if (plan.bn == 512) s = launch<512, 2, false, 1>(plan, ma, mb, mc, st);
+            else if (plan.bn == 192) s = launch<192, 2, false, 1>(plan, ma, mb, mc, st);
+            else s = plan.bn == 256 ? launch<256, 2, false, 1>(plan, ma, mb, mc, st) : launch<128, 2, false, 1>(plan, ma, mb, mc, st);
+        } else if (plan.bn == 256) s = launch<256, 1, false, 1>(plan, ma, mb, mc, st);
+        else if (plan.bn == 192) s = launch<192, 1, false, 1>(plan, ma, mb, mc, st);
+        else s = launch<128, 1, false, 1>(plan, ma, mb, mc, st);
+    } else if (swiglu) s = launch<512, 2, true>(plan, ma, mb, mc, st);
     else if (plan.ctas == 2) {
         if (plan.bn == 512) s = launch<512, 2>(plan, ma, mb, mc, st);
         else if (plan.bn == 192) s = launch<192, 2>(plan, ma, mb, mc, st);
