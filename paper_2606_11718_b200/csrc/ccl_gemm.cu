@@ -251,27 +251,31 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint3
 }
 
 // Stored coordinates (r, c) of an operand -> the first four coordinates of its tensor map (the fifth is the problem of a batch).
+// FULL = false: the instantiation for plain calls (no page-interleaved operand, no batch, no alpha / beta, no operand split
+// along K) leaves those branches out -- 0.5-0.7 us on a 15-30 us GEMM, 0.5 % on the large ones.
+template <bool FULL = true>
 __device__ __forceinline__ void to_coords(const OpMap& o, int r, int c, int& x, int& y, int& z, int& u) {
     int g, rr, xx;                                   // strip, row inside the strip, column inside the strip row
     if (o.split == 2) { o.w.divmod(c, g, xx); rr = r; }
     else if (o.split == 1) { o.h.divmod(r, g, rr); xx = c; }
     else { g = 0; rr = r; xx = c; }
-    if (o.il_mode == 1) { o.il_kr.divmod(rr, u, y); x = xx; z = g; }
-    else if (o.il_mode == 2) { o.il_sc.divmod(xx, y, x); z = rr; u = g; }
+    if (FULL && o.il_mode == 1) { o.il_kr.divmod(rr, u, y); x = xx; z = g; }
+    else if (FULL && o.il_mode == 2) { o.il_sc.divmod(xx, y, x); z = rr; u = g; }
     else { x = xx; y = rr; z = g; u = 0; }
 }
 // Element offset of C[m][n] in its buffer (any layout).
+template <bool FULL = true>
 __device__ __forceinline__ int64_t c_offset(const GemmParams& p, int64_t m, int64_t n) {
     // (multiply-shift divisions only: a 64-bit division is a subroutine of several hundred cycles)
     int g = 0, rr = (int)m, xx = (int)n;             // strip, row inside the strip, column inside the strip row
     if (p.c.split == 2) p.c.w.divmod((int)n, g, xx);
     else if (p.c.split == 1) p.c.h.divmod((int)m, g, rr);
-    if (p.c.il_mode == 1) {                          // a chunk holds il_kr whole strip rows
+    if (FULL && p.c.il_mode == 1) {                  // a chunk holds il_kr whole strip rows
         int j, y;
         p.c.il_kr.divmod(rr, j, y);
         return ((int64_t)j * p.c_nstrips + g) * p.c_ichunk + (int64_t)y * p.c_row + xx;
     }
-    if (p.c.il_mode == 2) {                          // a strip row spans c_cpr whole chunks
+    if (FULL && p.c.il_mode == 2) {                  // a strip row spans c_cpr whole chunks
         int cj, x;
         p.c.il_sc.divmod(xx, cj, x);
         return (((int64_t)rr * p.c_cpr + cj) * p.c_nstrips + g) * p.c_ichunk + x;
@@ -330,7 +334,7 @@ struct Scheduler {
         t.n0 = sn * p.Wn + jn * bn; t.n1 = min(t.n0 + bn, (sn + 1) * p.Wn);
         return true;
     }
-    template <int RAG>
+    template <int RAG, bool FULL>
     __device__ bool get(int it, TileCoord& t) const {
         if (RAG == 1 && rag) return get_ragged(it, t);
         int g, i;
@@ -346,7 +350,7 @@ struct Scheduler {
         t.split = 0;
         if (p.splits > 1) { int ii; p.fd_splits.divmod(i, ii, t.split); i = ii; }   // the splits of one tile are neighbours in the walk
         t.e = 0;
-        if (p.batch > 1) { int ii; p.fd_tiles_per_problem.divmod(i, t.e, ii); i = ii; }
+        if (FULL && p.batch > 1) { int ii; p.fd_tiles_per_problem.divmod(i, t.e, ii); i = ii; }
         int pn, rem;
         p.fd_per_panel.divmod(i, pn, rem);
         const bool tail = gm - pn * p.panel < p.panel;   // the last panel may be lower
@@ -374,7 +378,7 @@ struct Scheduler {
 
 // RAG: 1 = ragged M (ccl_gemm_grouped), 2 = ragged K (ccl_gemm_grouped_k) -- instantiations of their own, so that the tile
 // walk and the k loops of all other calls stay as they are (the extra branches cost 1-1.5 us on a 15-30 us GEMM)
-template <int BN, int CTAS, bool SWIGLU = false, int RAG = 0>
+template <int BN, int CTAS, bool SWIGLU = false, int RAG = 0, bool FULL = true>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                 const __grid_constant__ CUtensorMap map_c, const __grid_constant__ GemmParams gp) {
@@ -475,7 +479,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         // K runs along the tensor map's x for a K-contiguous operand and along y otherwise; unless the
         // operand is split along K itself (rare) only that coordinate changes from one k block to the next
         // (a page-interleaved operand recomputes its coordinates every k block as well)
-        const bool ksplit = (mn ? om.split == 1 : om.split == 2) || om.il_mode != 0;
+        const bool ksplit = FULL && ((mn ? om.split == 1 : om.split == 2) || om.il_mode != 0);
         uint32_t soff;                                        // byte offset of the box inside a stage
         int off;                                              // offset of the box along M (A) or N (B) from the tile origin
         int hsel = 0;                                         // sub-tile of a B box
@@ -492,13 +496,13 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         const int stages = p.stages, num_kb = p.num_kb, kbps = p.kb_per_split;
         const uint32_t stage_bytes = p.stage_bytes;
         const bool post_tx = lane == 0 && leader;
-        for (int it = 0; ok && sched.template get<RAG>(it, t); ++it) {
+        for (int it = 0; ok && sched.template get<RAG, FULL>(it, t); ++it) {
             if (t.skip) continue;
             int base = (isA ? t.m0 : t.n0) + off;
             // output column n0 of strip g -> B column n0 + g * pair_dist (gate) and one pair_dist further (up)
             if (SWIGLU && !isA) base += (p.fd_wn.div(t.n0) + hsel) * p.pair_dist;
             int x, y, z, u;
-            if (mn) to_coords(om, 0, base, x, y, z, u); else to_coords(om, base, 0, x, y, z, u);
+            if (mn) to_coords<FULL>(om, 0, base, x, y, z, u); else to_coords<FULL>(om, base, 0, x, y, z, u);
             int kb0 = t.split * kbps, kb1 = min(num_kb, kb0 + kbps), kbase = 0;
             if (RAG == 2) { const KRange kr = k_range(p.k_offs, t.e, p.K); kb0 = 0; kb1 = kr.nkb; kbase = kr.k0; }
             if (lane == 0 && it == 0) CCL_TRACE(11);
@@ -511,7 +515,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 // (the byte count may be posted after a copy has completed: the phase cannot end before this arrival)
                 if (post_tx) mbar_expect_tx(&full[stage], stage_bytes * CTAS);
                 const int k0 = kbase + kb * BK;
-                if (ksplit) { if (mn) to_coords(om, k0, base, x, y, z, u); else to_coords(om, base, k0, x, y, z, u); }
+                if (ksplit) { if (mn) to_coords<FULL>(om, k0, base, x, y, z, u); else to_coords<FULL>(om, base, k0, x, y, z, u); }
                 else if (mn) y = k0; else x = k0;
                 if (lane == 0 && it == 0 && kb == kb0) CCL_TRACE(13);
                 if (active) tma_load<CTAS>(smem + (size_t)stage * stage_bytes + soff, map, full0 + (uint32_t)stage * 8u, x, y, z, u, t.e * om.batched);
@@ -534,7 +538,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             const int stages = p.stages, num_kb = p.num_kb, kbps = p.kb_per_split;
             const uint32_t stage_bytes = p.stage_bytes, a_bytes = p.a_bytes, idesc = p.idesc, smem0 = smem_u32(smem);
             int done = 0;                                   // tiles computed so far (empty tiles of a ragged batch do not count)
-            for (int it = 0; ok && sched.template get<RAG>(it, t); ++it) {
+            for (int it = 0; ok && sched.template get<RAG, FULL>(it, t); ++it) {
                 if (t.skip) continue;
                 // NSUB == 1: TMEM half (done & 1) is this tile's accumulator, the other half is being drained.
                 // NSUB == 2: both halves belong to this tile; half h may be overwritten once the epilogue
@@ -606,7 +610,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         bool alive = true;
         uint32_t epi_count = 0;                          // TMA-stored pieces so far (selects the staging buffer)
         int done = 0;                                    // tiles drained so far
-        for (int it = 0; alive && sched.template get<RAG>(it, t); ++it) {
+        for (int it = 0; alive && sched.template get<RAG, FULL>(it, t); ++it) {
           if (t.skip) continue;
           const int tile_no = done++;
           const int m = t.m0 + (int)rank * BM + quad * 32 + lane;
@@ -630,8 +634,8 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             // C map coordinates of (row0, nb): a tile lies inside one strip, so only x moves from piece to piece
             // (unless a strip row is cut into chunks, which puts the chunk index in y as well)
             int cx0, cy0, cz0, cu0;
-            to_coords(p.c, row0, nb, cx0, cy0, cz0, cu0);
-            const bool c_chunked = p.c.il_mode == 2;
+            to_coords<FULL>(p.c, row0, nb, cx0, cy0, cz0, cu0);
+            const bool c_chunked = FULL && p.c.il_mode == 2;
             // One 64-column piece: registers -> C.  `r` holds 64 fp32 accumulators of this thread's row.
             // One 64-column piece of this warp's 32 rows -> C.  `pk` holds the piece already rounded to bf16 (two
             // values per word); full pieces go through shared memory and a TMA tile store, ragged ones are stored
@@ -661,7 +665,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     CCL_TRACE2(warp == 2 && lane == 0 && epi_count < 12, epi_count * 5 + 3);
                     if (lane == 0) {
                         int cx = cx0 + c * 64, cy = cy0, cz = cz0, cu = cu0;
-                        if (c_chunked) to_coords(p.c, row0, n64, cx, cy, cz, cu);
+                        if (c_chunked) to_coords<FULL>(p.c, row0, n64, cx, cy, cz, cu);
                         tma_store_5d(&map_c, buf, cx, cy, cz, cu, t.e * p.c.batched);
                         tma_store_commit();
                     }
@@ -673,7 +677,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 // compute the address of its last row and store nothing (the row test only ever predicates a store:
                 // the TMEM loads and waits around this code are warp-wide)
                 const bool row_ok = m < t.m1;
-                unsigned short* dst = p.C + c_offset(p, min(m, t.m1 - 1), n64) + (int64_t)t.e * p.c_batch_stride;
+                unsigned short* dst = p.C + c_offset<FULL>(p, min(m, t.m1 - 1), n64) + (int64_t)t.e * p.c_batch_stride;
 #pragma unroll
                 for (int j = 0; j < 8; ++j)
                     if (n64 + j * 8 < t.n1)              // the same for the whole warp; n1 - n0 is a multiple of 8
@@ -693,7 +697,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             auto axpby_piece = [&](uint32_t (&r)[64], int c) {
                 const int n64 = nb + c * 64;
                 const bool row_ok = m < t.m1;
-                const unsigned short* src = p.C + c_offset(p, min(m, t.m1 - 1), n64) + (int64_t)t.e * p.c_batch_stride;
+                const unsigned short* src = p.C + c_offset<FULL>(p, min(m, t.m1 - 1), n64) + (int64_t)t.e * p.c_batch_stride;
                 const float alpha = p.alpha, beta = p.beta;
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
@@ -710,7 +714,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             };
             auto store_piece = [&](uint32_t (&r)[64], int c) {
                 if (p.splits > 1) { store_partial(r, c); return; }
-                if (p.axpby) axpby_piece(r, c);
+                if (FULL && p.axpby) axpby_piece(r, c);
                 uint32_t pk[32];
                 pack(r, pk);
                 store_packed(pk, c);
@@ -845,6 +849,7 @@ struct GemmPlan {
     size_t ws_bytes;
     MatView va, vb, vc;
     uint32_t smem_bytes;
+    bool lean;                 // no optional feature in use (see FULL)
     unsigned grid;
 };
 
@@ -1148,19 +1153,19 @@ static ccl_status operand_tmap(CUtensorMap* m, const MatView& v, const void* bas
     return encode_tmap(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, base, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
-template <int BN, int CTAS, bool SWIGLU = false, int RAG = 0>
+template <int BN, int CTAS, bool SWIGLU = false, int RAG = 0, bool FULL = true>
 static ccl_status configure(uint32_t smem_bytes) {
     static uint32_t configured_for = 0;
     if (configured_for < smem_bytes) {
-        CCL_CUDA_TRY(cudaFuncSetAttribute(ccl_gemm_kernel<BN, CTAS, SWIGLU, RAG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes));
+        CCL_CUDA_TRY(cudaFuncSetAttribute(ccl_gemm_kernel<BN, CTAS, SWIGLU, RAG, FULL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes));
         configured_for = smem_bytes;
     }
     return CCL_OK;
 }
 
-template <int BN, int CTAS, bool SWIGLU = false, int RAG = 0>
+template <int BN, int CTAS, bool SWIGLU = false, int RAG = 0, bool FULL = true>
 static ccl_status launch(const GemmPlan& plan, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, cudaStream_t st) {
-    ccl_status s = configure<BN, CTAS, SWIGLU, RAG>(plan.smem_bytes);
+    ccl_status s = configure<BN, CTAS, SWIGLU, RAG, FULL>(plan.smem_bytes);
     if (s) return s;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(plan.grid, 1, 1);
@@ -1181,7 +1186,7 @@ static ccl_status launch(const GemmPlan& plan, const CUtensorMap& ma, const CUte
         attr[1].val.programmaticStreamSerializationAllowed = 1;
         cfg.numAttrs = 2;
     }
-    CCL_CUDA_TRY(cudaLaunchKernelEx(&cfg, ccl_gemm_kernel<BN, CTAS, SWIGLU, RAG>, ma, mb, mc, plan.p));
+    CCL_CUDA_TRY(cudaLaunchKernelEx(&cfg, ccl_gemm_kernel<BN, CTAS, SWIGLU, RAG, FULL>, ma, mb, mc, plan.p));
     count_launch();
     return CCL_OK;
 }
@@ -1333,6 +1338,11 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
         plan.p.k_offs = k_offs;
         plan.p.c_batch_stride = batch4[3] / 2;
         plan.p.alpha = alpha; plan.p.beta = beta; plan.p.axpby = (alpha != 1.0f || beta != 0.0f) ? 1 : 0;
+        {
+            const GemmParams& q = plan.p;
+            const bool ks = (q.a_mn ? q.a.split == 1 : q.a.split == 2) || (q.b_mn ? q.b.split == 1 : q.b.split == 2);
+            plan.lean = !q.axpby && batch == 1 && !q.a.il_mode && !q.b.il_mode && !q.c.il_mode && !ks && !m_offs && !k_offs && !swiglu;
+        }
         const uint32_t bnh = (uint32_t)(plan.subn / plan.ctas);   // B rows of one K-major box
         if (!plan.p.a_mn) s = operand_tmap(&prep.ma, plan.va, A_dev, BK, BM, batch, batch4[1]); else s = operand_tmap(&prep.ma, plan.va, A_dev, 64, BK, batch, batch4[1]);
         if (s) return s;
@@ -1368,7 +1378,15 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
         else if (plan.bn == 192) s = launch<192, 1, false, 1>(plan, ma, mb, mc, st);
         else s = launch<128, 1, false, 1>(plan, ma, mb, mc, st);
     } else if (swiglu) s = launch<512, 2, true>(plan, ma, mb, mc, st);
-    else if (plan.ctas == 2) {
+    else if (plan.lean) {                                // nothing optional in use: the instantiation without those branches
+        if (plan.ctas == 2) {
+            if (plan.bn == 512) s = launch<512, 2, false, 0, false>(plan, ma, mb, mc, st);
+            else if (plan.bn == 192) s = launch<192, 2, false, 0, false>(plan, ma, mb, mc, st);
+            else s = plan.bn == 256 ? launch<256, 2, false, 0, false>(plan, ma, mb, mc, st) : launch<128, 2, false, 0, false>(plan, ma, mb, mc, st);
+        } else if (plan.bn == 256) s = launch<256, 1, false, 0, false>(plan, ma, mb, mc, st);
+        else if (plan.bn == 192) s = launch<192, 1, false, 0, false>(plan, ma, mb, mc, st);
+        else s = launch<128, 1, false, 0, false>(plan, ma, mb, mc, st);
+    } else if (plan.ctas == 2) {
         if (plan.bn == 512) s = launch<512, 2>(plan, ma, mb, mc, st);
         else if (plan.bn == 192) s = launch<192, 2>(plan, ma, mb, mc, st);
         else s = plan.bn == 256 ? launch<256, 2>(plan, ma, mb, mc, st) : launch<128, 2>(plan, ma, mb, mc, st);
