@@ -409,10 +409,18 @@ def extras(out_dir, quick, only=None):
                     if bounds[e + 1] > bounds[e]:
                         torch.matmul(Av[bounds[e]:bounds[e + 1]], Bv[e].t() if bt else Bv[e])
             t_t = timed(torch_loop, 3)
+            t_lib = None                                           # the library's own grouped GEMM, where this torch has one
+            try:
+                Bk = Bv.transpose(1, 2) if bt else Bv              # [E, K, N] view
+                ends = offs[1:].contiguous()
+                t_lib = timed(lambda: torch._grouped_mm(Av, Bk, offs=ends), 20)
+            except Exception as err:                               # noqa: BLE001 (absent or unsupported: report and go on)
+                print(f"extras grouped: torch._grouped_mm not usable here ({type(err).__name__})", flush=True)
             tf = 2.0 * T * N * K / (t_g * 1e-3) / 1e12
-            rows.append(dict(what="grouped", experts=E, tokens=T, N=N, K=K, counts=label, max_count=cap, grouped_ms=t_g, torch_loop_ms=t_t, tflops=tf))
+            rows.append(dict(what="grouped", experts=E, tokens=T, N=N, K=K, counts=label, max_count=cap, grouped_ms=t_g, torch_loop_ms=t_t,
+                             torch_grouped_mm_ms=t_lib, tflops=tf))
             print(f"extras grouped {E} experts, {T} tokens x {N} x {K}, {label} (max {cap}): one launch {t_g * 1e3:8.1f} us ({tf:6.0f} TFLOP/s) | "
-                  f"torch.matmul per expert {t_t * 1e3:8.1f} us", flush=True)
+                  f"torch.matmul per expert {t_t * 1e3:8.1f} us" + (f" | torch._grouped_mm {t_lib * 1e3:8.1f} us" if t_lib else ""), flush=True)
     # 1c. a whole MoE expert FFN forward on routed tokens: gate/up with the activation fused, then down -- two launches
     for E, T, H, I in (((128, 32768, 2048, 768),) if not quick else ((32, 8192, 2048, 768),)) if want("moe_ffn") else ():
         import numpy as np
@@ -463,10 +471,16 @@ def extras(out_dir, quick, only=None):
                     if bounds[e + 1] > bounds[e]:
                         torch.matmul(Av[bounds[e]:bounds[e + 1]].t(), Bv[bounds[e]:bounds[e + 1]])
             t_t = timed(torch_loop, 3)
+            t_lib = None
+            try:
+                ends = offs[1:].contiguous()
+                t_lib = timed(lambda: torch._grouped_mm(Av.t(), Bv, offs=ends), 20)
+            except Exception as err:                               # noqa: BLE001
+                print(f"extras MoE weight gradient: torch._grouped_mm not usable here ({type(err).__name__})", flush=True)
             tf = 2.0 * T * M * N / (t_g * 1e-3) / 1e12
-            rows.append(dict(what="moe_wgrad", name=name, experts=E, tokens=T, M=M, N=N, grouped_k_ms=t_g, torch_loop_ms=t_t, tflops=tf))
+            rows.append(dict(what="moe_wgrad", name=name, experts=E, tokens=T, M=M, N=N, grouped_k_ms=t_g, torch_loop_ms=t_t, torch_grouped_mm_ms=t_lib, tflops=tf))
             print(f"extras MoE weight gradient ({name}), {E} experts, {T} routed tokens, {M} x {N} each: one launch {t_g * 1e3:8.1f} us ({tf:6.0f} TFLOP/s) | "
-                  f"torch.matmul per expert {t_t * 1e3:8.1f} us", flush=True)
+                  f"torch.matmul per expert {t_t * 1e3:8.1f} us" + (f" | torch._grouped_mm {t_lib * 1e3:8.1f} us" if t_lib else ""), flush=True)
     # 2. gate/up GEMM with the gated activation in the epilogue against GEMM + elementwise kernel
     for M, N, K in (((8192, 57344, 8192), (16384, 1536, 2048)) if not quick else ((1024, 57344, 8192),)) if want("swiglu") else ():
         d0, d1 = desc(M, N, K, 4), desc(M, N, K, 4, c_cols=N // 2)
