@@ -41,8 +41,9 @@ FLOP_PER_STEP = sum(2 * g["M"] * g["N"] * g["K"] for g in GEMMS)
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the two GEMM launches of one step, from the
 # single-pass ncu capture of this very workload (profiles/ccl_gemm_kernel_llama_gateup_1024tok.md, second
-# table): gate+up 12.70 + 0.93 GB, down 5.30 + 0.12 GB.  Only valid for the default configuration.
-GEMM_DRAM_BYTES_PER_STEP = {(8192, 4, 4096): 19.05e9}
+# table): gate+up 6.40 + 0.93 GB, down 3.03 + 0.12 GB (19.05 GB before the CTAs were kept in step between rounds
+# of tiles).  Only valid for the default configuration.
+GEMM_DRAM_BYTES_PER_STEP = {(8192, 4, 4096): 10.48e9}
 
 
 def set_tokens(t):

@@ -26,6 +26,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <atomic>
 #include <mutex>
 
 #include <cuda_bf16.h>
@@ -48,6 +49,8 @@ constexpr int64_t kRaggedDense = 4096;         // problems of a ragged batch who
 constexpr uint32_t kEpiBytes = 4 * 2 * 32 * 128; // epilogue staging: per warp two buffers of 32 rows x 128 B
 
 __device__ int g_gemm_status = 0;
+constexpr int kWaveSlots = 64;
+__device__ unsigned int g_wave_ctr[kWaveSlots];
 
 #ifdef CCL_GEMM_TRACE   // development aid: per-CTA timestamps of the kernel's phases (not compiled into the library)
 __device__ unsigned long long g_trace[296][32];
@@ -124,6 +127,10 @@ struct GemmParams {
     int64_t c_batch_stride;         // elements between the C buffers of consecutive problems
     // ragged batch (ccl_gemm_grouped): problem e owns rows [m_offs[e], m_offs[e + 1]) of A and C; the tile grid of a
     // problem is laid out for Wm rows (the caller's bound) and tiles past a problem's last row are skipped
+    // soft wave barrier (large problems): the producers of all CTAs meet here between full rounds of the tile walk, so
+    // that the CTAs that share operand rows / columns stay close enough in time to find each other's lines in L2
+    unsigned int* wave_ctr;
+    int32_t wave_period, wave_wait_ns;
     const int32_t* m_offs;
     // ragged K (ccl_gemm_grouped_k): problem e contracts rows [k_offs[e], k_offs[e + 1]) of A [K x M] and B [K x N]
     const int32_t* k_offs;
@@ -285,6 +292,12 @@ __device__ __forceinline__ int64_t c_offset(const GemmParams& p, int64_t m, int6
 
 // Ragged K: first row, k blocks and rows of the last block of problem e (an empty or out-of-range problem: one block of
 // zero rows, so that its output is written as zeros).
+__device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
 struct KRange { int k0, nkb, rem; };
 __device__ __forceinline__ KRange k_range(const int32_t* k_offs, int e, int Ktot) {
     const int o0 = __ldg(k_offs + e), o1 = __ldg(k_offs + e + 1);
@@ -498,6 +511,15 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         const bool post_tx = lane == 0 && leader;
         for (int it = 0; ok && sched.template get<RAG, FULL>(it, t); ++it) {
             if (t.skip) continue;
+            if (p.wave_ctr && it >= 1 && it < p.sch_rounds && it % p.wave_period == 0) {   // wait (bounded) until every CTA has issued its previous tiles
+                if (lane == 0) {
+                    atomicAdd(p.wave_ctr, 1u);
+                    const unsigned int target = gridDim.x * (unsigned int)(it / p.wave_period);
+                    const uint64_t t0 = global_timer_ns();
+                    while (ld_acquire_u32(p.wave_ctr) < target && global_timer_ns() - t0 < (uint64_t)p.wave_wait_ns) { }
+                }
+                __syncwarp();
+            }
             int base = (isA ? t.m0 : t.n0) + off;
             // output column n0 of strip g -> B column n0 + g * pair_dist (gate) and one pair_dist further (up)
             if (SWIGLU && !isA) base += (p.fd_wn.div(t.n0) + hsel) * p.pair_dist;
@@ -1364,6 +1386,25 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     }
     plan.p.ws = static_cast<float*>(ws_dev);
     cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    // Soft wave barrier for problems of three or more full rounds of tiles (CCL_GEMM_WAVESYNC=0 turns it off, =n syncs
+    // every n-th round; CCL_GEMM_WAVEWAIT = bound of one wait in ns): without it the CTAs that share an A panel or B
+    // columns drift apart by more than the L2 holds and fetch the same lines from DRAM 2-3 times.
+    plan.p.wave_ctr = nullptr;
+    {
+        static const int wave_sync = []() { const char* f = std::getenv("CCL_GEMM_WAVESYNC"); return f ? atoi(f) : 1; }();
+        static const int wave_wait = []() { const char* f = std::getenv("CCL_GEMM_WAVEWAIT"); return f ? atoi(f) : 20000; }();
+        plan.p.wave_period = wave_sync > 0 ? wave_sync : 1; plan.p.wave_wait_ns = wave_wait;
+        if (wave_sync > 0 && plan.p.sch_rounds >= 3 && !m_offs && !k_offs) {
+            static std::atomic<unsigned int> next{0};
+            static unsigned int* base[64] = {};                  // address of the counters, per device
+            int dev = 0;
+            CCL_CUDA_TRY(cudaGetDevice(&dev));
+            if (dev < 0 || dev >= 64) dev = 0;
+            if (!base[dev]) CCL_CUDA_TRY(cudaGetSymbolAddress(reinterpret_cast<void**>(&base[dev]), g_wave_ctr));
+            plan.p.wave_ctr = base[dev] + next.fetch_add(1) % kWaveSlots;
+            CCL_CUDA_TRY(cudaMemsetAsync(plan.p.wave_ctr, 0, sizeof(unsigned int), st));
+        }
+    }
     if (k_offs) {                                        // ragged K: one CTA per tile (make_plan)
         if (plan.bn == 256) s = launch<256, 1, false, 2>(plan, ma, mb, mc, st);
         else if (plan.bn == 192) s = launch<192, 1, false, 2>(plan, ma, mb, mc, st);
