@@ -117,3 +117,37 @@ def test_ragged_batch_in_a_graph_follows_the_offsets_on_the_device():
         assert err.max() <= 1e-2 * (K / 1024.0) ** 0.5 + 2.0 ** -8
         assert (got[owned:] == 0).all()
     assert ccl.ccl_gemm_status()[0] == ccl.OK
+
+
+def test_large_gemm_with_its_wave_barrier_replays_from_a_graph():
+    """A problem of several rounds of tiles zeroes its meeting-point counter with a memset node in front of the launch:
+    captured and replayed, it gives the bits of the eager call every time."""
+    M, N, K, P = 4096, 8192, 512, 4
+    A, B = synth.gemm_operands(M, N, K, 0, 0, seed=61, tag="graph_big")
+    d = gemm_desc(M, N, K, P, ("row", "ccl", "ccl"), 0, 0, 2, 1)
+    assert ccl.ccl_gemm_workspace(d) == 0
+    a = A.cuda()
+    b_ccl = torch.empty(ccl.ccl_buffer_bytes(d.B) // 2, dtype=torch.bfloat16, device="cuda")
+    ccl.ccl_repack(d.B, B.cuda(), b_ccl, 0)
+    c = torch.zeros(ccl.ccl_buffer_bytes(d.C) // 2, dtype=torch.bfloat16, device="cuda")
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        ccl.ccl_gemm(d, a, b_ccl, c)
+        side.synchronize()
+        want = c.clone()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            ccl.ccl_gemm(d, a, b_ccl, c)
+            ccl.ccl_gemm(d, a, b_ccl, c)                               # twice in a row: each launch has its own counter
+    for _ in range(3):
+        c.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(c, want)
+    assert ccl.ccl_gemm_status()[0] == ccl.OK
+    # sampled against the oracle
+    rows = [0, 1, 777, 4095]
+    ref32, _, _ = orc.gemm(synth.bits(A)[rows], synth.bits(B), len(rows), N, K, 0, 0)
+    from test_gpu_gemm import from_layout, tol
+    got = synth.from_bits(from_layout(c.view(torch.int16), d.C)).to(torch.float32).numpy()[rows]
+    assert (np.abs(got - ref32) / np.maximum(1.0, np.abs(ref32))).max() <= tol(K)
