@@ -1394,7 +1394,9 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
         static const int wave_sync = []() { const char* f = std::getenv("CCL_GEMM_WAVESYNC"); return f ? atoi(f) : 1; }();
         static const int wave_wait = []() { const char* f = std::getenv("CCL_GEMM_WAVEWAIT"); return f ? atoi(f) : 20000; }();
         plan.p.wave_period = wave_sync > 0 ? wave_sync : 1; plan.p.wave_wait_ns = wave_wait;
-        if (wave_sync > 0 && plan.p.sch_rounds >= 3 && !m_offs && !k_offs) {
+        // (long tiles only: with K below 4096, or a batch of small problems, the CTAs share little and the waits only cost --
+        // measured -9 % on 128 batched expert GEMMs and on a 16384 x 1536 x 2048 fused gate/up GEMM)
+        if (wave_sync > 0 && plan.p.sch_rounds >= 3 && plan.p.kb_per_split >= 64 && batch == 1 && !m_offs && !k_offs) {
             static std::atomic<unsigned int> next{0};
             static unsigned int* base[64] = {};                  // address of the counters, per device
             int dev = 0;
