@@ -21,6 +21,18 @@
  *    ccl_last_error() gives a thread-local message for the last failing call.
  *  - There is no CPU fallback: without a CUDA device the device entry points return
  *    CCL_ERR_CUDA.
+ *
+ * Test / diagnostic switches (environment variables, read by the library; none changes a result beyond the
+ * rounding order of a split-K sum):
+ *   CCL_GEMM_CTAS = 1|2            force one CTA per tile or a cta_group::2 pair
+ *   CCL_GEMM_BN = 64|128|192|256|512   force the tile width
+ *   CCL_GEMM_SPLITK = n            force the number of K splits
+ *   CCL_GEMM_WAVESYNC = 0|n        soft wave barrier off / every n-th round of tiles
+ *   CCL_GEMM_PDL = 0               no programmatic dependent launch
+ *   CCL_GEMM_RAGGED_DENSE = 0      ragged batches walk the fixed grid of max_rows per problem
+ *   CCL_REPACK_PATH = vec|tma      force a repack kernel
+ *   CCL_GEMM_VERBOSE = 1           print the chosen plan of every newly planned GEMM to stderr -- the one
+ *                                  exception to "never prints"
  */
 #ifndef CCL_H_
 #define CCL_H_
@@ -59,9 +71,9 @@ typedef enum { CCL_PART_NONE = 0, CCL_PART_ROWS = 1, CCL_PART_COLS = 2 } ccl_par
  *       which Sec. 2.2 calls coarse-grained: already contiguous):
  *       h = rows/P, offset = (r / h)*stride + (r mod h)*cols + c, stride = h*cols
  *       (rounded up likewise).
- *   layout = CCL_CCL_INTERLEAVED (either part): the page-interleaved form of CCL that makes a plain
- *       address-driven round-robin mapping local (Sec. 3.3 / 4.1: "4 KB round-robin interleaving
- *       achieves the fine-grained locality").  strip_align_bytes is the chunk size S (> 0).  Element
+ *   layout = CCL_CCL_INTERLEAVED (either part): the page-interleaved form of CCL, under which a plain
+ *       address-driven round-robin mapping at the chunk size already puts every strip on its own
+ *       chiplet (the setting Sec. 3.3 / 4.1 evaluate).  strip_align_bytes is the chunk size S (> 0).  Element
  *       o of strip g's packed contents (o = r*w + c' resp. (r mod h)*cols + c, as above) sits in that
  *       strip's chunk j = o*e / S, and chunk j of strip g is stored as chunk j*P + g of the buffer:
  *       byte offset = (j*P + g)*S + (o*e mod S).  The buffer holds ceil(strip bytes / S)*P chunks;
@@ -124,7 +136,7 @@ ccl_status ccl_repack_batched(const ccl_mat* m, int32_t batch, const void* src_d
  */
 ccl_status ccl_repack_transpose(const ccl_mat* m, const void* src_dev, void* dst_dev, void* cuda_stream);
 
-/* ---- GEMM on CCL operands (Sec. 2.2 execution model, Sec. 3.3 "only the address map changes") */
+/* ---- GEMM on CCL operands (Sec. 2.2 execution model; Sec. 3.3: the layout changes addresses only) */
 
 /*
  * C[M x N] = A[M x K] * B[K x N]; bf16 inputs, fp32 accumulation, bf16 output rounded to
@@ -203,8 +215,8 @@ ccl_status ccl_gemm_grouped_k(const ccl_gemm_desc* d, int32_t groups, const int3
                               const void* B_dev, void* C_dev, int64_t c_stride_bytes, void* cuda_stream);
 
 /*
- * The BLAS form (Sec. 2.2: "the extension to alpha*A*B + beta*C is straightforward, since the scalars do not affect
- * placement and the C read shares the same partitioning as the output write"):
+ * The BLAS form (Sec. 2.2 notes that alpha and beta change nothing for placement: C is read under the partition it
+ * is written under):
  *   C <- bf16( alpha * (A*B) + beta * C ),  fp32 arithmetic on the fp32 accumulator, one rounding.
  * C is read (only when beta != 0) and written through the same descriptor d->C; every tile reads its own part
  * of C before it writes it, so C_dev may hold anything when beta = 0.  alpha = 1, beta = 0 is ccl_gemm, bit for
@@ -230,8 +242,8 @@ ccl_status ccl_gemm_batched(const ccl_gemm_desc* d, int32_t batch, const void* A
                             void* ws_dev, size_t ws_bytes, void* cuda_stream);
 /*
  * GEMM on a fused gate/up weight with the gated activation applied in the epilogue, so that the activation the
- * next GEMM consumes is produced directly in its layout (Sec. 3.3: activations are "produced directly by upstream
- * kernels in CCL layout"; Fig. 3 shows the fused up/gate operand and its per-chiplet strips).  The activation
+ * next GEMM consumes is produced directly in its layout (Sec. 3.3 has the kernel upstream of a GEMM write its
+ * activations in CCL; Fig. 3 shows the fused up/gate operand and its per-chiplet strips).  The activation
  * itself, silu(x) = x / (1 + exp(-x)), is the standard one of these FFNs; the paper does not define it.
  *   H[M x N] = A * B as in ccl_gemm (fp32 accumulation), N even.  The N columns form S strips of width Wp = N/S,
  *   S = d->P if d->out_part == CCL_PART_COLS and d->P > 1, else S = 1; a strip holds its gate columns in its first
@@ -244,9 +256,11 @@ ccl_status ccl_gemm_batched(const ccl_gemm_desc* d, int32_t batch, const void* A
  */
 ccl_status ccl_gemm_swiglu(const ccl_gemm_desc* d, const void* A_dev, const void* B_dev, void* C_dev, void* cuda_stream);
 /*
- * Synchronises `cuda_stream`, then reports and clears the status word of GEMMs finished on
- * the current device: CCL_OK, or CCL_ERR_TIMEOUT with *detail = the raw device code.
- * detail may be NULL.
+ * Synchronises `cuda_stream` (the one entry point that does), then reports and clears the status word of the
+ * GEMMs and repacks finished on the current device: CCL_OK, or CCL_ERR_TIMEOUT with *detail = the raw device code
+ * (1-6: a GEMM wait, 101: a repack wait), or CCL_ERR_SHAPE (detail 5) for bad offsets of a ragged batch.
+ * detail may be NULL.  There is ONE status word per device, shared by every stream: with several streams in flight
+ * the first caller after an expiry gets the report, whichever stream's kernel it was.
  */
 ccl_status ccl_gemm_status(void* cuda_stream, int32_t* detail);
 
@@ -340,8 +354,8 @@ ccl_status ccl_traffic_l2(const ccl_traffic_desc* d, const int32_t* cta_chiplet_
                           void* cuda_stream);
 
 /*
- * The same count behind a FINITE private L2 per chiplet: the metric of Sec. 4.1 ("remote operand reads that miss in
- * L2, and remote output writes"; 8 MB, 128-byte lines, 16 ways per chiplet).  The paper's simulator is not public;
+ * The same count behind a FINITE private L2 per chiplet: the metric of Sec. 4.1 (operand reads from a remote
+ * chiplet's memory that miss the L2, plus output writes to one; 8 MB, 128-byte lines, 16 ways per chiplet).  The paper's simulator is not public;
  * this is a tile-level model with everything it leaves open stated here:
  *   - a chiplet's CTAs (its tiles under `assign`) are taken in row-major order of the tile grid (traversal = 0,
  *     n fastest) or column-major (traversal = 1, m fastest); the paper sweeps the traversal and reports the best;
@@ -383,6 +397,17 @@ ccl_status ccl_traffic_lru(const ccl_traffic_desc* d, const ccl_l2_model* m, uin
  */
 ccl_status ccl_probe_l2_latency(const void* zero_buf_dev, int32_t nlines, int64_t stride_bytes, int32_t nctas, float* lat_dev,
                                 int32_t* smid_dev, void* cuda_stream);
+
+/*
+ * Test support for the bounded device-side waits (no counterpart in the paper).  Launches one small CTA whose wait
+ * CANNOT be satisfied, with a limit of limit_us microseconds (1..100000) instead of the library's 2 s, so that the
+ * expiry path runs: the wait gives up by itself, the kernel records its code and leaves the way the real kernels do,
+ * and the next ccl_gemm_status() returns CCL_ERR_TIMEOUT once.  Nothing is left waiting and the context stays usable.
+ *   which = 0: the GEMM's path -- TMEM allocated, an mbarrier nobody arrives at, status code 6, TMEM released;
+ *   which = 1: the repack's TMA ring -- four slots, the load of one slot left out, status code 101; the loads still in
+ *              flight are drained before the CTA exits.  src_dev: 2048 readable bytes, 16-byte aligned (which = 1 only).
+ */
+ccl_status ccl_selftest_wait_timeout(int32_t which, uint32_t limit_us, const void* src_dev, void* cuda_stream);
 
 /* Message for the last non-OK status returned on this thread ("" if none). Static storage. */
 const char* ccl_last_error(void);

@@ -15,7 +15,7 @@
 //   Sec. 2.2: C = A*B, one CTA per output tile streaming A and B along K;
 //            a column region of a column-major operand is already contiguous
 //            (PART_ROWS below)
-//   Sec. 3.3 / 4.1 ("plain 4 KB round-robin interleaving achieves the fine-grained locality"): the
+//   Sec. 3.3 / 4.1 (the evaluated setting: plain 4 KB round-robin over address bits already gives the locality): the
 //            page-interleaved variant of CCL (layout ORC_CCL_INTERLEAVED): strip g's j-th chunk of
 //            strip_align_bytes is stored at chunk j*G + g, so an address-driven "chunk mod G" mapping
 //            sends every strip to its own chiplet
@@ -541,8 +541,8 @@ int orc_traffic_ideal_l2(const orc_traffic_desc* d, const int32_t* explicit_q, u
 // The same count taken run by run (a stored row of a tile is one contiguous run per strip,
 // cut at page boundaries).  Validated against orc_traffic_elem in the tests; used at sizes
 // where the element walk would take minutes.
-// Remote traffic behind a FINITE private L2 per chiplet (Sec. 4.1: "per-chiplet L2 caches", 8 MB, 128-byte lines,
-// 16 ways; the metric counts "remote operand reads that miss in L2, and remote output writes").  What the paper
+// Remote traffic behind a FINITE private L2 per chiplet (Sec. 4.1: one L2 per chiplet, 8 MB, 128-byte lines,
+// 16 ways; the metric counts operand reads from a remote chiplet that miss the L2, plus output writes to one).  What the paper
 // leaves open is fixed here as the simplest tile-level model:
 //   * every chiplet has its own cache of capacity_bytes / (line_bytes * ways) sets, LRU replacement inside a set;
 //     the lines of A and of B are numbered from the start of their own buffers (assumed line-aligned) and carry the

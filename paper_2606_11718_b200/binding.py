@@ -20,7 +20,7 @@ PLACE_RR, PLACE_BLOCK, PLACE_BEST = 0, 1, 2
 ASSIGN_N_STRIPS, ASSIGN_M_STRIPS, ASSIGN_EXPLICIT = 0, 1, 2
 
 EXPORTS = ["ccl_map_offset", "ccl_map_inverse", "ccl_buffer_bytes", "ccl_strip_stride", "ccl_repack", "ccl_repack_batched", "ccl_repack_transpose", "ccl_gemm_workspace",
-           "ccl_gemm", "ccl_gemm_batched_workspace", "ccl_gemm_batched", "ccl_gemm_grouped", "ccl_gemm_grouped_swiglu", "ccl_gemm_grouped_k", "ccl_gemm_axpby", "ccl_gemm_swiglu", "ccl_gemm_static_ws", "ccl_gemm_status", "ccl_traffic_sizes", "ccl_traffic", "ccl_traffic_l2", "ccl_traffic_lru", "ccl_probe_l2_latency", "ccl_last_error", "ccl_launch_count", "ccl_version"]
+           "ccl_gemm", "ccl_gemm_batched_workspace", "ccl_gemm_batched", "ccl_gemm_grouped", "ccl_gemm_grouped_swiglu", "ccl_gemm_grouped_k", "ccl_gemm_axpby", "ccl_gemm_swiglu", "ccl_gemm_static_ws", "ccl_gemm_status", "ccl_selftest_wait_timeout", "ccl_traffic_sizes", "ccl_traffic", "ccl_traffic_l2", "ccl_traffic_lru", "ccl_probe_l2_latency", "ccl_last_error", "ccl_launch_count", "ccl_version"]
 
 
 class CclError(RuntimeError):
@@ -95,6 +95,7 @@ def lib():
         l.ccl_gemm_swiglu.argtypes = [C.POINTER(GemmDesc), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         l.ccl_gemm_static_ws.argtypes = [C.POINTER(GemmDesc), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         l.ccl_gemm_status.argtypes = [C.c_void_p, C.POINTER(C.c_int32)]
+        l.ccl_selftest_wait_timeout.argtypes = [C.c_int32, C.c_uint32, C.c_void_p, C.c_void_p]
         l.ccl_traffic_sizes.argtypes = [C.POINTER(TrafficDesc), C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
         l.ccl_traffic.argtypes = [C.POINTER(TrafficDesc), C.c_void_p, C.c_void_p, C.POINTER(C.c_void_p), C.POINTER(C.c_void_p),
                                   C.c_void_p, C.c_void_p]
@@ -277,6 +278,11 @@ def ccl_gemm_status():
     detail = C.c_int32()
     st = lib().ccl_gemm_status(_stream(), C.byref(detail))
     return st, detail.value
+
+
+def ccl_selftest_wait_timeout(which, limit_us, src=None):
+    """Test support: launches a CTA whose bounded wait runs out after limit_us (0: the GEMM's path, 1: the repack ring)."""
+    _check(lib().ccl_selftest_wait_timeout(which, limit_us, _ptr(src), _stream()))
 
 
 def ccl_traffic_sizes(d):

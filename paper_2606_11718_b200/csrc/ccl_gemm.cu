@@ -52,16 +52,6 @@ __device__ int g_gemm_status = 0;
 constexpr int kWaveSlots = 64;
 __device__ unsigned int g_wave_ctr[kWaveSlots];
 
-#ifdef CCL_GEMM_TRACE   // development aid: per-CTA timestamps of the kernel's phases (not compiled into the library)
-__device__ unsigned long long g_trace[296][32];
-#define CCL_TRACE(slot) do { g_trace[blockIdx.x][slot] = global_timer_ns(); g_trace[blockIdx.x][16 + (slot)] = (unsigned long long)clock64(); } while (0)
-__device__ unsigned long long g_trace2[296][128];
-#define CCL_TRACE2(cond, slot) do { if (cond) g_trace2[blockIdx.x][slot] = (unsigned long long)clock64(); } while (0)
-#else
-#define CCL_TRACE(slot) do { } while (0)
-#define CCL_TRACE2(cond, slot) do { } while (0)
-#endif
-
 // Division of a non-negative int by a launch constant as a multiply-high and a shift (an integer division costs a few
 // hundred cycles, and the tile walk of a short GEMM is nothing but divisions).  For d >= 2: l = ceil(log2 d),
 // mul = ceil(2^(31+l) / d), n / d = umulhi(n, mul) >> (l - 1), exact for 0 <= n < 2^31; d = 1: mul = 0, shr = 0.
@@ -429,7 +419,6 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     const bool leader = rank == 0;
 
     if (threadIdx.x == 0) {
-        CCL_TRACE(0);
         prefetch_tmap(&map_a);
         prefetch_tmap(&map_b);
         prefetch_tmap(&map_c);
@@ -443,7 +432,6 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     if (CTAS == 2) cluster_sync();                   // the peer's barriers exist before anything remote touches them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_ptr;
-    if (threadIdx.x == 0) CCL_TRACE(1);
     asm volatile("griddepcontrol.wait;" ::: "memory");   // everything before this overlapped the previous kernel's tail
 
     // Ragged batch with a dense walk: m-tiles of every problem, as an exclusive prefix over the problems.
@@ -473,7 +461,6 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         __syncthreads();
     }
     Scheduler sched(p, (int)(blockIdx.x / CTAS), BM * CTAS, TILE_N, rag_prefix);
-    if (threadIdx.x == 0) CCL_TRACE(10);
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -527,22 +514,16 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             if (mn) to_coords<FULL>(om, 0, base, x, y, z, u); else to_coords<FULL>(om, base, 0, x, y, z, u);
             int kb0 = t.split * kbps, kb1 = min(num_kb, kb0 + kbps), kbase = 0;
             if (RAG == 2) { const KRange kr = k_range(p.k_offs, t.e, p.K); kb0 = 0; kb1 = kr.nkb; kbase = kr.k0; }
-            if (lane == 0 && it == 0) CCL_TRACE(11);
             for (int kb = kb0; kb < kb1; ++kb) {
                 ok = mbar_wait_bounded(&empty[stage], phase ^ 1);
                 ok = __all_sync(0xffffffffu, ok);
-                if (lane == 0 && it == 0 && kb == kb0) CCL_TRACE(12);
-                CCL_TRACE2(lane == 0 && it == 0 && kb - kb0 < 16, 64 + (kb - kb0) * 2);
                 if (!ok) { if (lane == 0) atomicExch(&g_gemm_status, 1); break; }
                 // (the byte count may be posted after a copy has completed: the phase cannot end before this arrival)
                 if (post_tx) mbar_expect_tx(&full[stage], stage_bytes * CTAS);
                 const int k0 = kbase + kb * BK;
                 if (ksplit) { if (mn) to_coords<FULL>(om, k0, base, x, y, z, u); else to_coords<FULL>(om, base, k0, x, y, z, u); }
                 else if (mn) y = k0; else x = k0;
-                if (lane == 0 && it == 0 && kb == kb0) CCL_TRACE(13);
                 if (active) tma_load<CTAS>(smem + (size_t)stage * stage_bytes + soff, map, full0 + (uint32_t)stage * 8u, x, y, z, u, t.e * om.batched);
-                if (lane == 0 && it == 0 && kb == kb0) CCL_TRACE(2);
-                CCL_TRACE2(lane == 0 && it == 0 && kb - kb0 < 16, 64 + (kb - kb0) * 2 + 1);
                 if (++stage == stages) { stage = 0; phase ^= 1; }
             }
         }
@@ -574,8 +555,6 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     // (the copies' completion on the barrier orders the operand bytes before the MMAs that read them;
                     // tcgen05 fences are only needed around the accumulator hand-over below)
                     if (!mbar_wait_bounded(&full[stage], phase)) { atomicExch(&g_gemm_status, 3); ok = false; break; }
-                    if (it == 0 && kb == kb0) CCL_TRACE(3);
-                    CCL_TRACE2(it == 0 && kb - kb0 < 16, 96 + (kb - kb0) * 2);
                     const uint32_t sa = smem0 + (uint32_t)stage * stage_bytes;
                     const uint64_t adesc = smem_desc(sa, a_lbo, 1024);
                     // Ragged K, last block of a problem: only the 16-row k steps that hold rows of this problem are
@@ -613,12 +592,10 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     }
                     if (!ok) break;
                     umma_commit<CTAS>(&empty[stage]);          // frees the stage (in both CTAs) once these MMAs have read it
-                    CCL_TRACE2(it == 0 && kb - kb0 < 16, 96 + (kb - kb0) * 2 + 1);
                     if (++stage == stages) { stage = 0; phase ^= 1; }
                 }
                 if (ok) {
                     umma_commit<CTAS>(&tmem_full[acc0]);   // accumulator(s) complete (both CTAs); the sub-tiles of a wide tile finish together
-                    if (it == 0) CCL_TRACE(4);
                 }
             }
         }
@@ -645,8 +622,6 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) { if (lane == 0) atomicExch(&g_gemm_status, 4); alive = false; break; }
             tc_fence_after();
-            if (warp == 2 && lane == 0 && it == 0 && h == 0) CCL_TRACE(5);
-            if (warp == 2 && lane == 0 && it == 0 && h == 1) CCL_TRACE(14);
             const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * ACC_COLS);
             // Full 32-row x 64-column pieces go through shared memory (128-byte swizzle) and a TMA tile store
             // addressed through C's own tensor map; ragged pieces (tile clipped by a strip or the matrix edge)
@@ -675,23 +650,18 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 if (rows_full && n64 + 64 <= t.n1) {
                     // staging: 32 KB in all -- two buffers per warp with four warps, one with eight
                     unsigned char* buf = epi + (size_t)(EW == 1 ? (warp - 2) * 2 + (epi_count & 1) : (warp - 2)) * (32 * 128);
-                    CCL_TRACE2(warp == 2 && lane == 0 && epi_count < 12, epi_count * 5 + 0);
                     if (epi_count >= 2 / EW) { if (lane == 0) tma_store_wait_read<2 / EW - 1>(); __syncwarp(); }   // buffer free again
-                    CCL_TRACE2(warp == 2 && lane == 0 && epi_count < 12, epi_count * 5 + 1);
 #pragma unroll
                     for (int u = 0; u < 8; ++u)
                         *reinterpret_cast<uint4*>(buf + lane * 128 + ((u ^ (lane & 7)) << 4)) = make_uint4(pk[4 * u], pk[4 * u + 1], pk[4 * u + 2], pk[4 * u + 3]);
-                    CCL_TRACE2(warp == 2 && lane == 0 && epi_count < 12, epi_count * 5 + 2);
                     fence_proxy_async();
                     __syncwarp();
-                    CCL_TRACE2(warp == 2 && lane == 0 && epi_count < 12, epi_count * 5 + 3);
                     if (lane == 0) {
                         int cx = cx0 + c * 64, cy = cy0, cz = cz0, cu = cu0;
                         if (c_chunked) to_coords<FULL>(p.c, row0, n64, cx, cy, cz, cu);
                         tma_store_5d(&map_c, buf, cx, cy, cz, cu, t.e * p.c.batched);
                         tma_store_commit();
                     }
-                    CCL_TRACE2(warp == 2 && lane == 0 && epi_count < 12, epi_count * 5 + 4);
                     ++epi_count;
                     return;
                 }
@@ -796,8 +766,6 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             }
             tc_fence_before();
             __syncwarp();
-            if (warp == 2 && lane == 0 && it == 0 && h == NSUB - 1) CCL_TRACE(6);
-            if (warp == 2 && lane == 0 && it == 0 && h == 0) CCL_TRACE(15);
             if (lane == 0) {
                 if (CTAS == 2) mbar_arrive_cluster(tmem_empty0 + (uint32_t)acc * 8u);
                 else mbar_arrive(&tmem_empty[acc]);
@@ -811,17 +779,14 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         // every tile store has read its shared-memory source; the writes themselves are complete, like any other
         // store of the kernel, when the kernel is
         if (lane == 0) tma_store_wait_read<0>();
-        if (warp == 2 && lane == 0) CCL_TRACE(7);
     }
 
     tc_fence_before();
     __syncthreads();
     if (CTAS == 2) cluster_sync();                   // neither CTA frees TMEM or exits while the other may still use it
-    if (threadIdx.x == 0) CCL_TRACE(8);
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc<CTAS>(tmem_base, kTmemCols);
-        if (lane == 0) CCL_TRACE(9);
     }
 }
 
@@ -1231,6 +1196,26 @@ static int resident_pairs() {
 }
 
 ccl_status repack_status_take(int* code);   // ccl_repack.cu
+ccl_status repack_selftest_launch(const void* src_dev, uint64_t limit_ns, cudaStream_t st);   // ccl_repack.cu
+
+// Self-test of the GEMM's expiry path (ccl_selftest_wait_timeout, which = 0): one CTA allocates TMEM like the GEMM,
+// one thread waits -- bounded -- on an mbarrier nobody ever arrives at, records code 6 in the status word when the wait
+// gives up, and the CTA leaves the way the GEMM does: block-wide sync, TMEM released.
+__global__ void __launch_bounds__(64) wait_selftest_kernel(uint64_t limit_ns) {
+    __shared__ uint64_t bar;
+    __shared__ uint32_t tmem_slot;
+    const int warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) { mbar_init(&bar, 1); fence_barrier_init(); }
+    if (warp == 1) tmem_alloc<1>(&tmem_slot, 32);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_slot;
+    if (threadIdx.x == 0 && !mbar_wait_bounded(&bar, 0u, limit_ns)) atomicExch(&g_gemm_status, 6);
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) { tc_fence_after(); tmem_dealloc<1>(tmem_base, 32); }
+}
 
 }  // namespace ccl
 
@@ -1307,11 +1292,39 @@ static ccl_status workspace_impl(const ccl_gemm_desc* d, int64_t batch, size_t* 
 extern "C" ccl_status ccl_gemm_workspace(const ccl_gemm_desc* d, size_t* bytes) { return workspace_impl(d, 1, bytes); }
 extern "C" ccl_status ccl_gemm_batched_workspace(const ccl_gemm_desc* d, int32_t batch, size_t* bytes) { return workspace_impl(d, batch, bytes); }
 
+// Scratch for the split-K partial sums, part of the library image: every GPU that loads the library
+// holds these bytes until the process ends.  Only device code may use the name as an address; on the
+// host the name is merely a handle that cudaGetSymbolAddress turns into the device pointer.
+static __device__ __align__(256) unsigned char g_static_ws[CCL_GEMM_STATIC_WS_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_ws_mutex;
+void* g_static_ws_addr[kMaxDevices] = {};
+
+// Device address of g_static_ws on the current device, looked up once per device.
+ccl_status static_ws_address(void** out) {
+    int dev = -1;
+    CCL_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return ccl::fail(CCL_ERR_UNSUPPORTED, "ccl_gemm_static_ws: device ordinal %d is beyond the %d this library tracks", dev, kMaxDevices);
+    std::lock_guard<std::mutex> lock(g_static_ws_mutex);
+    if (!g_static_ws_addr[dev]) {
+        void* ptr = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_ws);
+        if (e != cudaSuccess || !ptr)
+            return ccl::fail(CCL_ERR_CUDA, "ccl_gemm_static_ws: cudaGetSymbolAddress failed: %s", cudaGetErrorString(e));
+        g_static_ws_addr[dev] = ptr;
+    }
+    *out = g_static_ws_addr[dev];
+    return CCL_OK;
+}
+}  // namespace
+
 // strides[X]: bytes between the buffers of operand X (A, B, C) of consecutive problems; 0 = shared (A and B only)
 // m_offs / cap: ragged batch (ccl_gemm_grouped), else nullptr / 0
 static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, const int64_t* strides, const void* A_dev, const void* B_dev, void* C_dev,
                             void* ws_dev, size_t ws_bytes, void* cuda_stream, float alpha = 1.0f, float beta = 0.0f, const int32_t* m_offs = nullptr,
-                            int64_t cap = 0, const int32_t* k_offs = nullptr) {
+                            int64_t cap = 0, const int32_t* k_offs = nullptr, bool static_ws = false) {
     if (!A_dev || !B_dev || !C_dev) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: NULL operand");
     if (!d) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: NULL descriptor");
     if (batch < 1 || batch > kMaxBatch) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: batch must be in [1, %lld]", (long long)kMaxBatch);
@@ -1379,6 +1392,16 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     GemmPlan& plan = prep.plan;
     const CUtensorMap &ma = prep.ma, &mb = prep.mb, &mc = prep.mc;
     const int sms = prep.sms;
+    if (static_ws) {                                     // ccl_gemm_static_ws: the scratch compiled into the library image
+        if (plan.ws_bytes > (size_t)CCL_GEMM_STATIC_WS_BYTES)
+            return fail(CCL_ERR_WORKSPACE, "ccl_gemm_static_ws: this problem needs %zu bytes of split-K workspace, the built-in scratch holds %u; "
+                        "use ccl_gemm with a caller-provided workspace", plan.ws_bytes, (unsigned)CCL_GEMM_STATIC_WS_BYTES);
+        ws_dev = nullptr; ws_bytes = 0;
+        if (plan.ws_bytes) {
+            if ((s = static_ws_address(&ws_dev))) return s;
+            ws_bytes = (size_t)CCL_GEMM_STATIC_WS_BYTES;
+        }
+    }
     if (plan.ws_bytes) {
         if (!ws_dev || ws_bytes < plan.ws_bytes)
             return fail(CCL_ERR_WORKSPACE, "ccl_gemm: this problem is split along K and needs %zu bytes of workspace (got %zu)", plan.ws_bytes, ws_dev ? ws_bytes : (size_t)0);
@@ -1387,24 +1410,34 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     plan.p.ws = static_cast<float*>(ws_dev);
     cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
     // Soft wave barrier for problems of three or more full rounds of tiles (CCL_GEMM_WAVESYNC=0 turns it off, =n syncs
-    // every n-th round; CCL_GEMM_WAVEWAIT = bound of one wait in ns): without it the CTAs that share an A panel or B
+    // every n-th round): without it the CTAs that share an A panel or B
     // columns drift apart by more than the L2 holds and fetch the same lines from DRAM 2-3 times.
     plan.p.wave_ctr = nullptr;
     {
         static const int wave_sync = []() { const char* f = std::getenv("CCL_GEMM_WAVESYNC"); return f ? atoi(f) : 1; }();
-        static const int wave_wait = []() { const char* f = std::getenv("CCL_GEMM_WAVEWAIT"); return f ? atoi(f) : 20000; }();
-        plan.p.wave_period = wave_sync > 0 ? wave_sync : 1; plan.p.wave_wait_ns = wave_wait;
+        plan.p.wave_period = wave_sync > 0 ? wave_sync : 1; plan.p.wave_wait_ns = 20000;        // one wait gives up after 20 us
         // (long tiles only: with K below 4096, or a batch of small problems, the CTAs share little and the waits only cost --
         // measured -9 % on 128 batched expert GEMMs and on a 16384 x 1536 x 2048 fused gate/up GEMM)
         if (wave_sync > 0 && plan.p.sch_rounds >= 3 && plan.p.kb_per_split >= 64 && batch == 1 && !m_offs && !k_offs) {
+            // One of kWaveSlots counters in the library image, handed out round-robin: a launch recorded into a CUDA graph
+            // keeps its slot for good while eager calls rotate through all of them, so two GEMMs that overlap on the GPU
+            // can land on one counter -- the barrier is soft (a wait just ends early or runs into its 20 us bound), results
+            // never depend on it.  A device ordinal beyond the table runs without the barrier.
             static std::atomic<unsigned int> next{0};
+            static std::mutex base_mutex;
             static unsigned int* base[64] = {};                  // address of the counters, per device
             int dev = 0;
             CCL_CUDA_TRY(cudaGetDevice(&dev));
-            if (dev < 0 || dev >= 64) dev = 0;
-            if (!base[dev]) CCL_CUDA_TRY(cudaGetSymbolAddress(reinterpret_cast<void**>(&base[dev]), g_wave_ctr));
-            plan.p.wave_ctr = base[dev] + next.fetch_add(1) % kWaveSlots;
-            CCL_CUDA_TRY(cudaMemsetAsync(plan.p.wave_ctr, 0, sizeof(unsigned int), st));
+            unsigned int* ctr0 = nullptr;
+            if (dev >= 0 && dev < 64) {
+                std::lock_guard<std::mutex> lock(base_mutex);
+                if (!base[dev]) CCL_CUDA_TRY(cudaGetSymbolAddress(reinterpret_cast<void**>(&base[dev]), g_wave_ctr));
+                ctr0 = base[dev];
+            }
+            if (ctr0) {
+                plan.p.wave_ctr = ctr0 + next.fetch_add(1) % kWaveSlots;
+                CCL_CUDA_TRY(cudaMemsetAsync(plan.p.wave_ctr, 0, sizeof(unsigned int), st));
+            }
         }
     }
     if (k_offs) {                                        // ragged K: one CTA per tile (make_plan)
@@ -1518,57 +1551,25 @@ extern "C" ccl_status ccl_gemm_status(void* cuda_stream, int32_t* detail) {
     return CCL_OK;
 }
 
+extern "C" ccl_status ccl_selftest_wait_timeout(int32_t which, uint32_t limit_us, const void* src_dev, void* cuda_stream) {
+    if (which != 0 && which != 1) return fail(CCL_ERR_INVALID_ARG, "ccl_selftest_wait_timeout: which must be 0 (GEMM) or 1 (repack ring)");
+    if (limit_us < 1 || limit_us > 100000) return fail(CCL_ERR_INVALID_ARG, "ccl_selftest_wait_timeout: limit_us must be in [1, 100000]");
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    const uint64_t limit_ns = (uint64_t)limit_us * 1000ull;
+    if (which == 1) return repack_selftest_launch(src_dev, limit_ns, st);
+    wait_selftest_kernel<<<1, 64, 0, st>>>(limit_ns);
+    count_launch();
+    CCL_CUDA_TRY(cudaGetLastError());
+    return CCL_OK;
+}
+
 // ------------------------------------------------------------------------------------------
 // ccl_gemm_static_ws: the split-K GEMM for callers that cannot allocate
 // ------------------------------------------------------------------------------------------
-// Scratch for the split-K partial sums, part of the library image: every GPU that loads the library
-// holds these bytes until the process ends.  Only device code may use the name as an address; on the
-// host the name is merely a handle that cudaGetSymbolAddress turns into the device pointer.
-static __device__ __align__(256) unsigned char g_static_ws[CCL_GEMM_STATIC_WS_BYTES];
-
-namespace {
-constexpr int kMaxDevices = 64;
-std::mutex g_static_ws_mutex;
-void* g_static_ws_addr[kMaxDevices] = {};
-
-// Device address of g_static_ws on the current device, looked up once per device.
-ccl_status static_ws_address(void** out) {
-    int dev = -1;
-    CCL_CUDA_TRY(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= kMaxDevices) return ccl::fail(CCL_ERR_UNSUPPORTED, "ccl_gemm_static_ws: device ordinal %d is beyond the %d this library tracks", dev, kMaxDevices);
-    std::lock_guard<std::mutex> lock(g_static_ws_mutex);
-    if (!g_static_ws_addr[dev]) {
-        void* ptr = nullptr;
-        cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_ws);
-        if (e != cudaSuccess || !ptr)
-            return ccl::fail(CCL_ERR_CUDA, "ccl_gemm_static_ws: cudaGetSymbolAddress failed: %s", cudaGetErrorString(e));
-        g_static_ws_addr[dev] = ptr;
-    }
-    *out = g_static_ws_addr[dev];
-    return CCL_OK;
-}
-}  // namespace
-
 extern "C" ccl_status ccl_gemm_static_ws(const ccl_gemm_desc* d, const void* A_dev, const void* B_dev, void* C_dev,
                                          void* cuda_stream) {
-    size_t need = 0;
-    ccl_status s = ccl_gemm_workspace(d, &need);
-    if (s) return s;
-    if (need > (size_t)CCL_GEMM_STATIC_WS_BYTES)
-        return ccl::fail(CCL_ERR_WORKSPACE, "ccl_gemm_static_ws: this problem needs %zu bytes of split-K workspace, the built-in scratch holds %u; "
-                         "use ccl_gemm with a caller-provided workspace", need, (unsigned)CCL_GEMM_STATIC_WS_BYTES);
-    void* ws = nullptr;
-    if (need) {
-        if ((s = static_ws_address(&ws))) return s;
-    }
-    return ccl_gemm(d, A_dev, B_dev, C_dev, ws, need ? (size_t)CCL_GEMM_STATIC_WS_BYTES : 0, cuda_stream);
+    // (the plan -- from the prepared-call cache on every call but the first -- says how much scratch the problem needs)
+    const int64_t none[3] = {0, 0, 0};
+    return gemm_impl(d, 1, false, none, A_dev, B_dev, C_dev, nullptr, 0, cuda_stream, 1.0f, 0.0f, nullptr, 0, nullptr, true);
 }
 
-#ifdef CCL_GEMM_TRACE
-extern "C" int ccl_debug_trace_read(void* host_out, size_t bytes) {
-    return (int)cudaMemcpyFromSymbol(host_out, ccl::g_trace, bytes < sizeof(ccl::g_trace) ? bytes : sizeof(ccl::g_trace));
-}
-extern "C" int ccl_debug_trace2_read(void* host_out, size_t bytes) {
-    return (int)cudaMemcpyFromSymbol(host_out, ccl::g_trace2, bytes < sizeof(ccl::g_trace2) ? bytes : sizeof(ccl::g_trace2));
-}
-#endif

@@ -101,7 +101,6 @@ __global__ void zero_pad_kernel(char* dst, int64_t pad_g, int64_t pad_off, int64
 // ------------------------------------------------------------------------------------------
 // TMA path: tile = box of (bx 8-byte units) x (by rows) of one strip
 // ------------------------------------------------------------------------------------------
-constexpr int kTmaMaxStages = 16;
 
 struct TmaTiling {
     uint32_t bx, by;              // box extents (8-byte units, rows)
@@ -122,6 +121,17 @@ __device__ __forceinline__ Coord5 tile_coord(const TmaTiling& t, bool il_side, u
     else if (t.il_mode == 1) { r.c[0] = (int)x; r.c[1] = (int)(y % t.il_kr); r.c[2] = (int)g; r.c[3] = (int)(y / t.il_kr); r.c[4] = (int)b; }
     else { r.c[0] = (int)(x % t.il_s8); r.c[1] = (int)(x / t.il_s8); r.c[2] = (int)y; r.c[3] = (int)g; r.c[4] = (int)b; }
     return r;
+}
+
+// After a wait on ring slot `it % stages` has run out: the loads of iterations it+1 .. (those issued so far) may still
+// be in flight into this CTA's shared memory, and a CTA must not exit under them.  Gives each of them a further,
+// short, bounded wait.  Loads are issued `stages` ahead at the start and then one per iteration, one iteration late
+// (see the loop of repack_tma_kernel); `left` = iterations from `it` to the end of this CTA's tiles.
+constexpr uint64_t kDrainLimitNs = 50000000ull;   // 50 ms per outstanding load
+__device__ __forceinline__ void ring_drain(uint64_t* full, uint64_t it, uint32_t stages, uint64_t left) {
+    const uint64_t issued_end = it == 0 ? stages : it + stages - 1;      // first iteration whose load is not issued yet
+    for (uint64_t j = it + 1; j < issued_end && j - it < left; ++j)
+        (void)mbar_wait_bounded(&full[j % stages], (uint32_t)((j / stages) & 1), kDrainLimitNs);
 }
 
 // RANK 3: one matrix, no interleaved side (maps {x, row, strip}); RANK 4: a batch of those, or one matrix with an
@@ -174,7 +184,12 @@ __global__ void __launch_bounds__(32) repack_tma_kernel(const __grid_constant__ 
         if (tile >= t.ntiles) break;
         uint32_t slot = (uint32_t)(it % t.stages);
         uint32_t parity = (uint32_t)((it / t.stages) & 1);
-        if (!mbar_wait_bounded(&full[slot], parity)) { atomicExch(&g_repack_status, 1); break; }
+        if (!mbar_wait_bounded(&full[slot], parity)) {
+            atomicExch(&g_repack_status, 1);
+            // the loads already issued into the other slots may still be writing this CTA's shared memory
+            ring_drain(full, it, t.stages, (t.ntiles - tile + gridDim.x - 1) / gridDim.x);
+            break;
+        }
         const Tile ti = decode(tile);
         const void* buf = stage0 + (size_t)slot * t.stage_bytes;
         if (RANK == 3) tma_store_3d(&dst_map, buf, (int)ti.x, (int)ti.y, (int)ti.g);
@@ -343,10 +358,6 @@ static ccl_status launch_tma(const char* src, char* dst, const CopyPlan& p, int 
     TmaTiling t;
     t.stages = 4; t.stage_bytes = 49152;                  // 4 x 48 KB measured best (6 x 32 KB: -3 %, 12 x 16 KB: -10 %)
     int ctas_per_sm = 1, max_bx = 256;
-    if (const char* f = std::getenv("CCL_REPACK_TUNE")) {   // "stages,stage_kb,ctas_per_sm,max_bx"
-        int a = 0, b = 0, c = 0, d2 = 0;
-        if (sscanf(f, "%d,%d,%d,%d", &a, &b, &c, &d2) == 4 && a > 0 && a <= kTmaMaxStages && b > 0 && c > 0 && d2 > 0) { t.stages = a; t.stage_bytes = b * 1024; ctas_per_sm = c; max_bx = d2; }
-    }
     t.bx = (uint32_t)std::min<uint64_t>((uint64_t)max_bx, dims[0]);
     t.il_mode = t.il_src = 0; t.il_kr = t.il_s8 = 1; t.nstrips = (uint32_t)p.nstrips;
     if (p.il_chunk) {
@@ -407,6 +418,41 @@ static ccl_status launch_tma(const char* src, char* dst, const CopyPlan& p, int 
     if (rank == 3) repack_tma_kernel<3><<<grid, 32, smem, st>>>(sm, dm, t);
     else if (rank == 4) repack_tma_kernel<4><<<grid, 32, smem, st>>>(sm, dm, t);
     else repack_tma_kernel<5><<<grid, 32, smem, st>>>(sm, dm, t);
+    count_launch();
+    CCL_CUDA_TRY(cudaGetLastError());
+    return CCL_OK;
+}
+
+// Self-test of the expiry path of the ring above (ccl_selftest_wait_timeout, which = 1): the same ring of mbarriers,
+// four slots of 512 bytes filled by plain bulk copies from src; the load of iteration 2 is left out on purpose, so the
+// consumer's wait on it runs out after limit_ns, the status word gets its code, ring_drain() waits for the load of
+// iteration 3 that is still outstanding, and the CTA returns.  Nothing waits on anything that cannot happen.
+constexpr uint32_t kSelfSlots = 4, kSelfBytes = 512;
+__global__ void __launch_bounds__(32) ring_selftest_kernel(const unsigned char* src, uint64_t limit_ns) {
+    __shared__ __align__(128) unsigned char buf[kSelfSlots][kSelfBytes];
+    __shared__ uint64_t full[kSelfSlots];
+    if (threadIdx.x != 0) return;
+    for (uint32_t s = 0; s < kSelfSlots; ++s) mbar_init(&full[s], 1);
+    fence_barrier_init();
+    for (uint32_t it = 0; it < kSelfSlots; ++it) {
+        if (it == 2) continue;                                   // the load that never comes
+        mbar_expect_tx(&full[it], kSelfBytes);
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"(smem_u32(buf[it])), "l"(src + (size_t)it * kSelfBytes), "r"(kSelfBytes), "r"(smem_u32(&full[it])) : "memory");
+    }
+    for (uint64_t it = 0; it < kSelfSlots; ++it) {
+        if (!mbar_wait_bounded(&full[it % kSelfSlots], 0u, limit_ns)) {
+            atomicExch(&g_repack_status, 1);
+            ring_drain(full, it, kSelfSlots, kSelfSlots - it);
+            break;
+        }
+    }
+}
+
+ccl_status repack_selftest_launch(const void* src_dev, uint64_t limit_ns, cudaStream_t st) {
+    if (!src_dev || (reinterpret_cast<uintptr_t>(src_dev) & 15))
+        return fail(CCL_ERR_ALIGN, "ccl_selftest_wait_timeout: src_dev must be a 16-byte aligned device buffer of %u bytes", kSelfSlots * kSelfBytes);
+    ring_selftest_kernel<<<1, 32, 0, st>>>(static_cast<const unsigned char*>(src_dev), limit_ns);
     count_launch();
     CCL_CUDA_TRY(cudaGetLastError());
     return CCL_OK;
@@ -561,7 +607,6 @@ extern "C" ccl_status ccl_repack_transpose(const ccl_mat* m, const void* src_dev
     int64_t run = kTrStages - 1;
     int il_shift = -1;
     if (v.ichunk && (v.ichunk & (v.ichunk - 1)) == 0) { il_shift = 0; while ((INT64_C(1) << il_shift) < v.ichunk) ++il_shift; }
-    if (const char* f = std::getenv("CCL_TRANSPOSE_RUN")) { const int n = std::atoi(f); if (n > 0) run = n; }
     (void)sms;
     const unsigned grid = (unsigned)std::min<int64_t>((ntiles + run - 1) / run, INT64_C(1) << 30);
     static bool carveout_set = false;

@@ -255,8 +255,8 @@ __global__ void traffic_owner_kernel(TrafficParams p) {
 }
 
 // ---- finite private L2 per chiplet (tile-level LRU model) --------------------------------------------------
-// Sec. 4.1 scores "remote operand reads that miss in L2, and remote output writes" with an 8 MB, 16-way, 128-byte-line
-// L2 per chiplet.  Model: the CTAs of a chiplet are taken in row-major (traversal 0) or column-major (traversal 1)
+// Sec. 4.1 scores the operand reads from a remote chiplet that miss the L2, and the output writes to one, with an 8 MB,
+// 16-way, 128-byte-line L2 per chiplet.  Model: the CTAs of a chiplet are taken in row-major (traversal 0) or column-major (traversal 1)
 // order of the tile grid and run in waves of `wave` consecutive CTAs that step through K together, `ks` elements at
 // a time; in each step every CTA of the wave in turn touches the lines of the k range of its A rectangle in address
 // order, then those of its B rectangle (wave = 1, ks = K: one CTA after the other); lines are numbered from the start of each operand's buffer and the operand is part of the tag,

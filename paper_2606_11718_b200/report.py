@@ -157,7 +157,7 @@ LRU_EXEC = dict(wave_ctas=1, k_slice=0)       # how a chiplet's CTAs run in the 
 
 def traffic_lru_best(g, layout_bc, place_bc, S, model_kw, e=2):
     """Remote bytes (A, B, C) behind a finite LRU L2 per chiplet: the best of both output partitions and both CTA
-    traversals, as the paper reports (Sec. 4.1: "we sweep CTA traversal and output-partition choices")."""
+    traversals, as the paper reports (Sec. 4.1 sweeps the CTA traversal and the output partition and keeps the best)."""
     best = None
     for assign in (ccl.ASSIGN_N_STRIPS, ccl.ASSIGN_M_STRIPS):
         td = traffic_desc(g, layout_bc, place_bc, S, assign, align=S, e=e)

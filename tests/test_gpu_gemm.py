@@ -212,23 +212,19 @@ def sample_blocks(M, N, P, rng, n_random=8, bm=128, bn=128):
     return [(m, m + bm, n, n + bn) for m, n in sorted(blocks)]
 
 
-@pytest.mark.parametrize("name,P", [("llama_fwd_down", 4), ("llama_wgrad", 2)])
-def test_gemm_llama_full_size_sampled(name, P):
-    """Full Llama-70B-size GEMM in the benchmark's launch configuration (CCL B and C, grouped raster): sampled
-    128x128 blocks against the oracle, plus a randomised projection check over the whole output."""
-    g = {x["name"]: x for x in synth.llama_fwd_gemms() + synth.llama_bwd_gemms()}[name]
-    M, N, K = g["M"], g["N"], g["K"]
-    A, B = synth.gemm_operands(M, N, K, g["a_trans"], g["b_trans"], seed=0, tag=name, a_std=g["a_std"], b_std=g["b_std"])
-    d = gemm_desc(M, N, K, P, ("row", "ccl", "ccl"), g["a_trans"], g["b_trans"], 2, 1)
+def check_sampled(d, A, B, g, P, rng, n_random=8):
+    """Sampled 128x128 blocks element by element against the oracle, plus the +-1 projection over every output."""
+    M, N, K = d.M, d.N, d.K
     got = run_gemm(d, A, B)
     gf = synth.from_bits(got).to(torch.float32)
     assert torch.isfinite(gf).all()
-    rng = np.random.default_rng(0)
-    for blk in sample_blocks(M, N, P, rng):
+    worst = 0.0
+    for blk in sample_blocks(M, N, P, rng, n_random):
         ref32, _, _ = orc.gemm(synth.bits(A), synth.bits(B), M, N, K, g["a_trans"], g["b_trans"], block=blk)
         sub = gf[blk[0]:blk[1], blk[2]:blk[3]].numpy()
         err = np.abs(sub - ref32) / np.maximum(1.0, np.abs(ref32))
         assert err.max() <= tol(K), (blk, err.max())
+        worst = max(worst, float(err.max()))
     # property over every output element: C v = A (B v) for random +-1 vectors (exact arithmetic up to rounding)
     Al = (A.T if g["a_trans"] else A).to(torch.float32)
     Bl = (B.T if g["b_trans"] else B).to(torch.float32)
@@ -241,6 +237,33 @@ def test_gemm_llama_full_size_sampled(name, P):
         # bf16 rounding of C: each element off by <= 2^-9 relative; random signs -> sqrt(N) growth, 8 sigma margin
         bound = 8 * math.sqrt(N) * sigma_c * 2.0 ** -8
         assert (lhs - rhs).abs().max().item() <= bound
+    return worst
+
+
+# name, P, strip alignment: the benchmark's own launch is the first (B and C in CCL, P = 4, strips aligned to 4 KB pages)
+LLAMA_FULL = [("llama_fwd_gateup", 4, 4096), ("llama_fwd_gateup", 2, 4096), ("llama_fwd_down", 4, 0), ("llama_fwd_down", 2, 4096),
+              ("llama_dgrad", 4, 4096), ("llama_wgrad", 2, 0), ("llama_wgrad", 4, 4096)]
+
+
+@pytest.mark.parametrize("name,P,align", LLAMA_FULL)
+def test_gemm_llama_full_size_sampled(name, P, align):
+    """Full Llama-70B-size GEMMs in the benchmark's launch configuration (CCL B and C, grouped raster): sampled
+    128x128 blocks against the oracle, plus a randomised projection check over the whole output."""
+    g = {x["name"]: x for x in synth.llama_fwd_gemms() + synth.llama_bwd_gemms()}[name]
+    M, N, K = g["M"], g["N"], g["K"]
+    A, B = synth.gemm_operands(M, N, K, g["a_trans"], g["b_trans"], seed=0, tag=name, a_std=g["a_std"], b_std=g["b_std"])
+    d = gemm_desc(M, N, K, P, ("row", "ccl", "ccl"), g["a_trans"], g["b_trans"], 2, 1, align=align)
+    check_sampled(d, A, B, g, P, np.random.default_rng(0))
+
+
+@pytest.mark.parametrize("name,P", [("llama_fwd_gateup", 4), ("llama_fwd_gateup", 8), ("llama_fwd_down", 2), ("llama_fwd_down", 4)])
+def test_gemm_m1024_llama_weights(name, P):
+    """The 1024-token row of the token-count sweep on the full Llama weights (CCL B and C, 4 KB-aligned strips)."""
+    g = dict({x["name"]: x for x in synth.llama_fwd_gemms()}[name])
+    M, N, K = 1024, g["N"], g["K"]
+    A, B = synth.gemm_operands(M, N, K, 0, 0, seed=0, tag=name + "/m1024")
+    d = gemm_desc(M, N, K, P, ("row", "ccl", "ccl"), 0, 0, 2, 1, align=4096)
+    check_sampled(d, A, B, g, P, np.random.default_rng(1), n_random=6)
 
 
 @pytest.fixture(params=[(1, 128), (1, 192), (1, 256), (2, 128), (2, 192), (2, 256), (2, 512)], ids=lambda v: f"c{v[0]}b{v[1]}")

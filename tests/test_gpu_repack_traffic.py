@@ -345,3 +345,32 @@ def test_traffic_llama_gateup_full_size_closed_form():
     do1, _ = traffic_pair(128, 57344, 8192, 4, 4096)
     want = orc.traffic(do1, level="runs")["per_cta"]
     np.testing.assert_array_equal(pc[:448, 1:], want[:, 1:])          # B and C columns of tile row 0
+
+
+@pytest.mark.parametrize("P", [4, 2])
+def test_traffic_llama_gateup_full_size_ccl_block(P):
+    """The benchmark's own count: the gate+up GEMM with B and C in CCL (strips aligned to 4 KB pages) and
+    page -> strip placement.  Totals against the closed form; the per-CTA numbers of sampled tile rows against the
+    oracle run on a descriptor restricted to one tile row (B's and C's strips then have other strides, so only the
+    quantities that do not depend on the stride are compared: every B and C byte local, A as in the full problem)."""
+    M, N, K, S = 8192, 57344, 8192, 4096
+    do, dl = traffic_pair(M, N, K, P, S, lay=("row", "ccl", "ccl"), place=(0, 1, 1), align=S)
+    nt, pages = ccl.ccl_traffic_sizes(dl)
+    per_cta = torch.zeros((nt, 3, 2), dtype=torch.int64, device="cuda")
+    totals = torch.zeros((3, 2), dtype=torch.int64, device="cuda")
+    ccl.ccl_traffic(dl, per_cta, totals)
+    t = host(totals, np.uint64)
+    tiles_n = N // 128
+    assert int(t[1, 1]) == 0 and int(t[2, 1]) == 0                       # the central claim: B and C fully local
+    assert int(t[1, 0]) == (M // 128) * K * N * 2 and int(t[2, 0]) == M * N * 2
+    assert int(t[0].sum()) == tiles_n * M * K * 2
+    assert int(t[0, 1]) * P == int(t[0].sum()) * (P - 1)                 # A row-major under round-robin: (P-1)/P remote
+    pc = host(per_cta, np.uint64)
+    assert (pc.sum(axis=2) == np.array([128 * K * 2, K * 128 * 2, 128 * 128 * 2], dtype=np.uint64)).all()
+    do1, _ = traffic_pair(128, N, K, P, S, lay=("row", "ccl", "ccl"), place=(0, 1, 1), align=S)
+    want = orc.traffic(do1, level="runs")["per_cta"]
+    for tm in (0, 17, 63):                                              # sampled tile rows
+        got = pc[tm * tiles_n:(tm + 1) * tiles_n]
+        np.testing.assert_array_equal(got[:, 1:], want[:, 1:])
+        # A: tile row tm reads rows [128 tm, 128 tm + 128) of A = pages 4 * (128 tm + r) + j: the same owner pattern
+        np.testing.assert_array_equal(got[:, 0], want[:, 0])

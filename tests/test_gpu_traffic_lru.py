@@ -126,3 +126,32 @@ def test_lru_rejections():
     assert rc(ccl.L2Model(), di) == ccl.ERR_UNSUPPORTED
     _, de = traffic_pair(256, 512, 128, 2, 4096, assign=2)
     assert rc(ccl.L2Model(), de) == ccl.ERR_UNSUPPORTED
+
+
+def _skew_cases():
+    out = []
+    for line in open(os.path.join(HERE, "golden", "lru_skew_index.txt")):
+        f = line.split()
+        if f and f[0] == "CASE":
+            out.append((f[1], *[int(x) for x in f[2:]]))
+    return out
+
+
+@pytest.mark.parametrize("case", _skew_cases(), ids=lambda c: c[0])
+def test_skewed_set_index_hand_cases_on_the_gpu(case):
+    """The hand-worked access strings that pin the skewed set index (their hit / miss outcome depends on it)."""
+    _, sets, hash_, M, N, K, BM, BN, bt, bstrips, balign, want_a, want_b = case
+    d = ccl.TrafficDesc()
+    d.M, d.N, d.K, d.BM, d.BN = M, N, K, BM, BN
+    d.A, d.C = ccl.Mat(M, K, 2), ccl.Mat(M, N, 2)
+    if bstrips > 1:
+        d.B = ccl.Mat(N, K, 2, bstrips, ccl.PART_ROWS, ccl.CCL, balign) if bt else ccl.Mat(K, N, 2, bstrips, ccl.PART_COLS, ccl.CCL, balign)
+    else:
+        d.B = ccl.Mat(N, K, 2) if bt else ccl.Mat(K, N, 2)
+    d.a_trans, d.b_trans, d.P, d.page_bytes = 0, bt, 1, 16
+    d.place[0] = d.place[1] = d.place[2] = ccl.PLACE_RR
+    d.assign, d.strip_tiling = ccl.ASSIGN_N_STRIPS, 1
+    t = run(d, ccl.L2Model(sets * 16, 16, 1, 0, hash_, 1, 0))
+    assert int(t[0, 0]) == want_a and int(t[0, 1]) == 0
+    if want_b >= 0:
+        assert int(t[1, 0]) == want_b
