@@ -39,11 +39,19 @@ GEMMS = [dict(name="gateup", M=T, N=2 * I, K=H), dict(name="down", M=T, N=H, K=I
 FLOP_PER_STEP = sum(2 * g["M"] * g["N"] * g["K"] for g in GEMMS)
 
 
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the two GEMM launches of one step, from the
-# single-pass ncu capture of this very workload (profiles/ccl_gemm_kernel_llama_gateup_1024tok.md, second
-# table): gate+up 6.40 + 0.93 GB, down 3.03 + 0.12 GB (19.05 GB before the CTAs were kept in step between rounds
-# of tiles).  Only valid for the default configuration.
-GEMM_DRAM_BYTES_PER_STEP = {(8192, 4, 4096): 10.48e9}
+def gemm_dram_traffic(tokens, P, page):
+    """DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the two GEMM launches of one step, as measured by
+    ncu: read from profiles/ccl_gemm_kernel_dram_traffic.json, which names the captured case, the capture command and the
+    rule that scales a reduced capture to the full launch.  None when the file does not cover this configuration."""
+    path = os.path.join(ROOT, "profiles", "ccl_gemm_kernel_dram_traffic.json")
+    try:
+        rec = json.load(open(path))
+    except (OSError, ValueError):
+        return None
+    for row in rec.get("configs", []):
+        if (row.get("tokens"), row.get("P"), row.get("page_bytes")) == (tokens, P, page):
+            return row.get("bytes_per_step")
+    return None
 
 
 def set_tokens(t):
@@ -58,8 +66,17 @@ def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         p = json.load(open(path))
-        return dict(hbm_gbs=p["hbm_gbs"], tf_burst=p["bf16_tflops"], tf_sustained=p["bf16_tflops_sustained"], source="measured")
-    return dict(hbm_gbs=6650.0, tf_burst=1590.0, tf_sustained=1400.0, source="fallback")
+        return dict(hbm_gbs=p["hbm_gbs"], tf_burst=p["bf16_tflops"], tf_sustained=p["bf16_tflops_sustained"], source="measured",
+                    sustained_sm_mhz=(p.get("clocks_under_load") or {}).get("sm_mhz_median"))
+    return dict(hbm_gbs=6650.0, tf_burst=1590.0, tf_sustained=1400.0, source="fallback", sustained_sm_mhz=1300.0)
+
+
+def tensor_peak(peaks, timed_seconds, sm_mhz):
+    """Which measured bf16 peak a GEMM timed here is held against.  The sustained figure was taken in a seconds-long loop
+    at the power cap (clock well below maximum); a timed region shorter than ~2 s, or one whose sampled SM clock is above the
+    clock of that loop, ran in the burst regime and is held against the burst figure."""
+    burst = timed_seconds < 2.0 or (sm_mhz is not None and peaks.get("sustained_sm_mhz") and sm_mhz > 1.05 * peaks["sustained_sm_mhz"])
+    return (peaks["tf_burst"], "burst") if burst else (peaks["tf_sustained"], "sustained")
 
 
 # ---------------------------------------------------------------------------------------------
@@ -281,6 +298,7 @@ def run_cuda(args):
     e2e_value = world * FLOP_PER_STEP / (e2e_ms * 1e-3) / 1e12
 
     peaks = measured_peaks()
+    peak_tf, peak_kind = tensor_peak(peaks, ms_total / 1e3, clocks.get("sm_mhz"))
     gemm_tf = FLOP_PER_STEP / (kms["gemm"] * 1e-3) / 1e12
     repack_bytes = sum(2 * g["K"] * g["N"] * 2 for g in GEMMS)
     repack_gbs = repack_bytes / (kms["repack"] * 1e-3) / 1e9
@@ -295,21 +313,136 @@ def run_cuda(args):
         "e2e": {"value": round(e2e_value, 2), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": round(e2e_ms, 3)},
         "gpu_launches": int(launches),
-        "roofline": {"kernel": "ccl_gemm_kernel", "bound": "tensor", "achieved": round(gemm_tf, 1), "peak": peaks["tf_sustained"],
-                     "unit": "TFLOP/s", "frac": round(gemm_tf / peaks["tf_sustained"], 4), "traffic": GEMM_DRAM_BYTES_PER_STEP.get((T, P, page)),
+        "roofline": {"kernel": "ccl_gemm_kernel", "bound": "tensor", "achieved": round(gemm_tf, 1), "peak": peak_tf,
+                     "unit": "TFLOP/s", "frac": round(gemm_tf / peak_tf, 4), "traffic": gemm_dram_traffic(T, P, page),
                      "traffic_unit": "bytes per step (2 launches), ncu", "algorithmic_bytes_per_step": sum(2 * (g["M"] * g["K"] + g["K"] * g["N"] + g["M"] * g["N"]) for g in GEMMS),
-                     "peak_source": f"bf16 sustained, {peaks['source']}", "frac_of_burst": round(gemm_tf / peaks["tf_burst"], 4),
+                     "peak_source": f"bf16 {peak_kind}, {peaks['source']} (timed region {ms_total / 1e3:.2f} s at {clocks.get('sm_mhz')} MHz)",
+                     "frac_of_burst": round(gemm_tf / peaks["tf_burst"], 4), "frac_of_sustained": round(gemm_tf / peaks["tf_sustained"], 4),
                      "frac_of_nominal_2250": round(gemm_tf / 2250.0, 4), "ms_per_step": round(kms["gemm"], 4)},
         "kernels": {"gemm_tflops": round(gemm_tf, 1), "repack_gbs": round(repack_gbs, 1),
-                    "repack_frac_of_hbm": round(repack_gbs / peaks["hbm_gbs"], 4), "repack_ms": round(kms["repack"], 4),
+                    "repack_frac_of_hbm": round(repack_gbs / peaks["hbm_gbs"], 4), "repack_frac_of_nominal_8TBs": round(repack_gbs / 8000.0, 4),
+                    "repack_ms": round(kms["repack"], 4),
                     "traffic_ms": round(kms["traffic"], 4),
                     "remote_traffic_ratio_ccl_vs_rr4k": round(ratio, 4), "remote_bytes": remote},
     }
+    if world == 1 and not args.no_by_config:
+        line["kernels"]["by_config"] = by_config(ccl, torch, descs, devb, peaks, P, page, uuid)
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
-            line["cpu_baseline"] = oracle_sample(P, page, synth, host)
+            # the step's own gate+up output, brought back to row-major by the library's repack, for the parity check
+            # that the oracle leg makes on its slab
+            d0 = descs[0]
+            ccl.ccl_repack(d0["mB"], devb[d0["w"]], d0["w_ccl"], 0)
+            ccl.ccl_gemm(d0["gd"], devb[d0["a"]], d0["w_ccl"], d0["c_ccl"])
+            c_row = torch.empty(T * d0["g"]["N"], dtype=torch.bfloat16, device="cuda")
+            ccl.ccl_repack(d0["mC"], d0["c_ccl"], c_row, 1)
+            c_slab = c_row.view(T, d0["g"]["N"])[:SAMPLE_ROWS].float().cpu().numpy()
+            line["cpu_baseline"], line["parity"] = oracle_sample(P, page, synth, host, c_slab=c_slab)
         print(json.dumps(line), flush=True)
     group.close()
+
+
+# ---------------------------------------------------------------------------------------------
+# the other configurations, kernel by kernel (outside the timed step and outside `value`)
+# ---------------------------------------------------------------------------------------------
+def by_config(ccl, torch, descs, devb, peaks, P, page, uuid):
+    """GEMM TFLOP/s and repack GB/s of the configurations the step does not cover: the single Qwen expert GEMM, the six
+    Qwen FFN GEMMs (forward, data and weight gradients), the Llama backward GEMMs and the weight-streaming rows
+    (M = 1, 16, 128) of the token sweep on both Llama weights.  B and C in CCL (P strips aligned to the page size),
+    grouped raster.  Each figure: CUDA events around back-to-back launches on one stream (100 for kernels under a
+    millisecond, 10 above), operands rotated through enough copies to exceed the L2 where one set would fit in it.
+    roofline_frac = time at min(tensor, HBM) roofline / measured time, against the measured burst peaks."""
+    from paper_2606_11718_b200 import synth
+    L2_BYTES = 126e6
+    sampler = ClockSampler(uuid)
+    sampler.start()
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def rand(rows, cols, std):
+        return (torch.randn(rows, cols, device="cuda", dtype=torch.float32) * std).to(torch.bfloat16)
+
+    def time_gemm(M, N, K, at, bt, a_src=None, b_src=None, P_=P):
+        lay_b = ccl.Mat(N, K, 2, P_, ccl.PART_ROWS, ccl.CCL, page) if bt else ccl.Mat(K, N, 2, P_, ccl.PART_COLS, ccl.CCL, page)
+        lay_c = ccl.Mat(M, N, 2, P_, ccl.PART_COLS, ccl.CCL, page)
+        gd = ccl.GemmDesc()
+        gd.M, gd.N, gd.K = M, N, K
+        gd.A, gd.B, gd.C = ccl.Mat(K, M, 2) if at else ccl.Mat(M, K, 2), lay_b, lay_c
+        gd.a_trans, gd.b_trans, gd.out_part, gd.P, gd.grouped_raster = at, bt, ccl.PART_COLS, P_, 1
+        one_set = 2 * (M * K + K * N + M * N)
+        copies = 1 if one_set > 2 * L2_BYTES else int(min(16, 2 * L2_BYTES // one_set + 2))
+        sets = []
+        for i in range(copies):
+            a = a_src if a_src is not None else rand(K if at else M, M if at else K, synth.ACT_STD)
+            if b_src is not None:
+                b = b_src
+            else:
+                b_row = rand(N if bt else K, K if bt else N, synth.WEIGHT_STD)
+                b = torch.empty(ccl.ccl_buffer_bytes(lay_b) // 2, dtype=torch.bfloat16, device="cuda")
+                ccl.ccl_repack(lay_b, b_row, b, 0)
+            c = torch.empty(ccl.ccl_buffer_bytes(lay_c) // 2, dtype=torch.bfloat16, device="cuda")
+            sets.append((a, b, c))
+        need = ccl.ccl_gemm_workspace(gd)
+        ws = torch.empty(max(need, 16) // 4, dtype=torch.float32, device="cuda")
+        flop = 2.0 * M * N * K
+        n = 100 if flop / 1.4e15 < 1e-3 else 10
+        for i in range(3):
+            ccl.ccl_gemm(gd, *sets[i % copies], ws)
+        e0, e1 = ev(), ev()
+        e0.record()
+        for i in range(n):
+            ccl.ccl_gemm(gd, *sets[i % copies], ws)
+        e1.record()
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) * 1e3 / n
+        roof_us = max(flop / (peaks["tf_burst"] * 1e12), one_set / (peaks["hbm_gbs"] * 1e9)) * 1e6
+        return {"M": M, "N": N, "K": K, "us": round(us, 2), "tflops": round(flop / us / 1e6, 1), "roofline_frac": round(roof_us / us, 4),
+                "bound": "tensor" if flop / (peaks["tf_burst"] * 1e12) > one_set / (peaks["hbm_gbs"] * 1e9) else "hbm",
+                "launches": n, "operand_sets": copies}
+
+    def time_repack(rows, cols):
+        m = ccl.Mat(rows, cols, 2, P, ccl.PART_COLS, ccl.CCL, page)
+        nbytes = rows * cols * 2
+        copies = 1 if nbytes > L2_BYTES else int(2 * L2_BYTES // nbytes + 2)
+        srcs = [rand(rows, cols, synth.WEIGHT_STD) for _ in range(copies)]
+        dsts = [torch.empty(ccl.ccl_buffer_bytes(m) // 2, dtype=torch.bfloat16, device="cuda") for _ in range(copies)]
+        n = 100 if nbytes < 1e8 else 20
+        for i in range(3):
+            ccl.ccl_repack(m, srcs[i % copies], dsts[i % copies], 0)
+        e0, e1 = ev(), ev()
+        e0.record()
+        for i in range(n):
+            ccl.ccl_repack(m, srcs[i % copies], dsts[i % copies], 0)
+        e1.record()
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) * 1e3 / n
+        gbs = 2 * nbytes / us / 1e3
+        return {"rows": rows, "cols": cols, "us": round(us, 2), "gbs": round(gbs, 1), "frac_of_hbm": round(gbs / peaks["hbm_gbs"], 4),
+                "launches": n, "operand_sets": copies}
+
+    out = {"layout": f"B and C in CCL, P={P}, strips aligned to {page} B, grouped raster", "peaks": "measured burst bf16 / measured HBM copy"}
+    g = synth.config1_gemm()
+    out["config1"] = {g["name"]: time_gemm(g["M"], g["N"], g["K"], g["a_trans"], g["b_trans"])}
+    out["config2"] = {g["name"]: time_gemm(g["M"], g["N"], g["K"], g["a_trans"], g["b_trans"]) for g in synth.qwen_ffn_gemms()}
+    out["config2_P2"] = {g["name"]: time_gemm(g["M"], g["N"], g["K"], g["a_trans"], g["b_trans"], P_=2) for g in synth.qwen_ffn_gemms()}
+    X, Z = devb["X"], devb["Z"]
+    wd_ccl = descs[1]["w_ccl"]
+    out["config4"] = {"llama_dgrad": time_gemm(T, H, I, 0, 0, a_src=Z, b_src=wd_ccl)}
+    x_ccl = torch.empty(ccl.ccl_buffer_bytes(ccl.Mat(T, H, 2, P, ccl.PART_COLS, ccl.CCL, page)) // 2, dtype=torch.bfloat16, device="cuda")
+    ccl.ccl_repack(ccl.Mat(T, H, 2, P, ccl.PART_COLS, ccl.CCL, page), X, x_ccl, 0)
+    out["config4"]["llama_wgrad"] = time_gemm(I, H, T, 1, 0, a_src=Z, b_src=x_ccl)
+    del x_ccl
+    out["config5"] = {}
+    for d, nm in zip(descs, ("gateup", "down")):
+        for M in (1, 16, 128):
+            a = rand(M, d["g"]["K"], synth.ACT_STD)
+            out["config5"][f"llama_{nm}_M{M}"] = time_gemm(M, d["g"]["N"], d["g"]["K"], 0, 0, a_src=a, b_src=d["w_ccl"])
+    out["repack"] = {"qwen_gateup_weight": time_repack(2048, 1536), "qwen_down_weight": time_repack(768, 2048),
+                     "llama_down_weight": time_repack(I, H), "llama_x": time_repack(T, H)}
+    st, detail = ccl.ccl_gemm_status()
+    if st != ccl.OK:
+        raise SystemExit(f"bench.py: device-side wait expired in the per-configuration runs (code {detail})")
+    out["clocks"] = sampler.stop()
+    return out
 
 
 # ---------------------------------------------------------------------------------------------
@@ -320,8 +453,10 @@ SAMPLE_REPACK_ROWS = 1024  # repack slab: the first 1024 rows of the gate+up wei
 REFERENCE_COLS = 16384     # --impl reference: each step covers this many output columns of the slab
 
 
-def oracle_sample(P, page, synth, host=None, ncols=None):
-    """Times the oracle, as it stands, on a slab of the workload.  Returns the cpu_baseline object."""
+def oracle_sample(P, page, synth, host=None, ncols=None, c_slab=None):
+    """Times the oracle, as it stands, on a slab of the workload.  Returns the cpu_baseline object; with c_slab (rows
+    [0, SAMPLE_ROWS) of the gate+up output the CUDA path computed, fp32) also the parity of that slab against the
+    oracle's fp32 sums, in the tolerance the tests use."""
     import oracle as orc
     g = GEMMS[0]
     M, N, K = g["M"], g["N"], g["K"]
@@ -336,7 +471,7 @@ def oracle_sample(P, page, synth, host=None, ncols=None):
     t0 = time.perf_counter()
     orc.repack(orc.Mat(SAMPLE_REPACK_ROWS, N, 2, P, orc.PART_COLS, orc.CCL, page), wb[:SAMPLE_REPACK_ROWS], 0)
     t1 = time.perf_counter()
-    orc.gemm(xb, wb, SAMPLE_ROWS, N, K, 0, 0, block=(0, SAMPLE_ROWS, 0, ncols), threads=cores)
+    ref32, _, _ = orc.gemm(xb, wb, SAMPLE_ROWS, N, K, 0, 0, block=(0, SAMPLE_ROWS, 0, ncols), threads=cores)
     t2 = time.perf_counter()
     td = orc.TrafficDesc()
     td.M, td.N, td.K, td.BM, td.BN = SAMPLE_ROWS, N, K, 128, 128
@@ -350,11 +485,21 @@ def oracle_sample(P, page, synth, host=None, ncols=None):
     t3 = time.perf_counter()
     flop = 2.0 * SAMPLE_ROWS * ncols * K
     total = t3 - t0
-    return {"value": round(flop / total / 1e12, 6), "unit": UNIT, "cores": cores, "kind": "oracle",
+    parity = None
+    if c_slab is not None:
+        import math
+        import numpy as np
+        err = np.abs(c_slab[:, :ncols] - ref32) / np.maximum(1.0, np.abs(ref32))
+        tol = 1e-2 * math.sqrt(K / 1024.0)
+        parity = {"max_err": float(err.max()), "tol": tol, "ok": bool(np.isfinite(c_slab).all() and err.max() <= tol),
+                  "blocks": f"gate+up output rows [0,{SAMPLE_ROWS}) x all {ncols} columns ({SAMPLE_ROWS * ncols} elements, every strip), "
+                            "err = |C - ref32| / max(1, |ref32|) against the fp32 oracle"}
+    base = {"value": round(flop / total / 1e12, 6), "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"gate+up GEMM rows [0,{SAMPLE_ROWS}) x columns [0,{ncols}) of {N} (fp32 oracle, {cores} threads), repack of the first "
                       f"{SAMPLE_REPACK_ROWS} weight rows and the traffic count of one tile row (both single-threaded)",
             "seconds": {"repack": round(t1 - t0, 3), "gemm": round(t2 - t1, 3), "traffic": round(t3 - t2, 3)},
             "gemm_only_tflops": round(flop / (t2 - t1) / 1e12, 6)}
+    return (base, parity) if c_slab is not None else base
 
 
 def run_reference(args):
@@ -396,8 +541,16 @@ def main():
     ap.add_argument("--page", type=int, default=4096, help="page / interleave bytes")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--tokens", type=int, default=8192, help="tokens per GPU (8192 = the benchmark workload)")
+    ap.add_argument("--no-by-config", action="store_true", help="skip the per-configuration kernel timings")
     args = ap.parse_args()
     set_tokens(args.tokens)
+    from paper_2606_11718_b200 import dist as ccl_dist
+    if args.impl == "ccl" and args.gpus > 1 and not ccl_dist.launched_by_a_launcher():
+        # no launcher set the environment: start the ranks here, one per GPU; rank 0 prints the line
+        env = {}
+        if "NCCL_DEBUG" not in os.environ:       # the communicator's own log (rank count, transports), kept off stdout
+            env = {"NCCL_DEBUG": "INFO", "NCCL_DEBUG_SUBSYS": "INIT", "NCCL_DEBUG_FILE": "/dev/stderr"}
+        sys.exit(ccl_dist.spawn_ranks(args.gpus, [sys.executable, os.path.abspath(__file__)] + sys.argv[1:], extra_env=env))
     if args.impl == "reference":
         args.steps = args.steps if args.steps is not None else 2
         args.warmup = args.warmup if args.warmup is not None else 1

@@ -4,6 +4,9 @@ Only the barrier, the max-over-ranks of a time and the aggregation of the per-ra
 ranks.  The functions are backend-agnostic (NCCL on GPUs, gloo in the CPU tests).
 """
 import os
+import socket
+import subprocess
+import sys
 
 import torch
 
@@ -67,3 +70,49 @@ def shard(items, rank, world):
     n = len(items)
     lo, hi = (n * rank) // world, (n * (rank + 1)) // world
     return items[lo:hi]
+
+
+def free_port():
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    return port
+
+
+def spawn_ranks(nproc, argv, extra_env=None, timeout=None):
+    """Runs `argv` (a command line) as `nproc` ranks on this node, one process per GPU: RANK = LOCAL_RANK = 0..nproc-1,
+    WORLD_SIZE, MASTER_ADDR = 127.0.0.1 and a free MASTER_PORT in the environment -- what a launcher would set.  The
+    children inherit stdout / stderr (rank 0 prints the result line).  Returns the largest exit code; if a rank
+    fails the others are terminated (by their own PIDs)."""
+    port = free_port()
+    procs = []
+    for r in range(nproc):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(nproc), MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        if extra_env:
+            env.update(extra_env)
+        procs.append(subprocess.Popen(list(argv), env=env))
+    worst, pending = 0, set(range(nproc))
+    import time
+    t0 = time.monotonic()
+    while pending:
+        for r in sorted(pending):
+            rc = procs[r].poll()
+            if rc is not None:
+                pending.discard(r)
+                worst = max(worst, abs(rc))
+        if worst or (timeout is not None and time.monotonic() - t0 > timeout):
+            for r in pending:
+                procs[r].terminate()
+            for r in pending:
+                try:
+                    procs[r].wait(timeout=10)
+                except subprocess.TimeoutExpired:
+                    procs[r].kill()
+            return worst or 124
+        time.sleep(0.05)
+    return worst
+
+
+def launched_by_a_launcher():
+    return "WORLD_SIZE" in os.environ and "RANK" in os.environ

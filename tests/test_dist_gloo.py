@@ -68,3 +68,40 @@ def test_reference_arm_rank1_prints_nothing():
     out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "1", "--warmup", "0"],
                          env=env, capture_output=True, text=True, timeout=120)
     assert out.returncode == 0 and out.stdout.strip() == ""
+
+
+SPAWNED = textwrap.dedent("""
+    import json, os, sys
+    sys.path.insert(0, %r)
+    from paper_2606_11718_b200 import dist
+    g = dist.Group("gloo")
+    ups, ms = dist.job_throughput(5.0, 1.0 + g.rank, g)
+    if g.rank == 0:
+        print(json.dumps({"n_gpus": g.world, "ups": ups, "ms": ms, "local": g.local}), flush=True)
+    g.close()
+""") % ROOT
+
+
+def test_spawn_helper_runs_two_gloo_ranks():
+    """The helper behind `bench.py --gpus N` when no launcher set the environment: N children, rank 0 prints one line."""
+    driver = textwrap.dedent("""
+        import sys
+        sys.path.insert(0, %r)
+        from paper_2606_11718_b200 import dist
+        sys.exit(dist.spawn_ranks(2, [sys.executable, "-c", %r], timeout=120))
+    """) % (ROOT, SPAWNED)
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_PORT", "MASTER_ADDR")}
+    out = subprocess.run([sys.executable, "-c", driver], env=env, capture_output=True, text=True, timeout=180)
+    assert out.returncode == 0, out.stderr
+    import json
+    lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    res = json.loads(lines[0])
+    assert res == {"n_gpus": 2, "ups": 10.0 / 2e-3, "ms": 2.0, "local": 0}
+
+
+def test_spawn_helper_reports_a_failing_rank():
+    sys.path.insert(0, ROOT)
+    from paper_2606_11718_b200 import dist
+    code = "import os, sys, time\nsys.exit(3) if os.environ['RANK'] == '1' else time.sleep(30)"
+    assert dist.spawn_ranks(2, [sys.executable, "-c", code], timeout=60) == 3
