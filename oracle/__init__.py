@@ -14,7 +14,7 @@ from . import build as _build
 ROWMAJOR, CCL, CCL_INTERLEAVED = 0, 1, 2
 PART_NONE, PART_ROWS, PART_COLS = 0, 1, 2
 PLACE_RR, PLACE_BLOCK, PLACE_BEST = 0, 1, 2
-ASSIGN_N, ASSIGN_M, ASSIGN_EXPLICIT = 0, 1, 2
+ASSIGN_N, ASSIGN_M, ASSIGN_EXPLICIT, ASSIGN_2D = 0, 1, 2, 3
 
 
 class Mat(C.Structure):
@@ -29,7 +29,7 @@ class TrafficDesc(C.Structure):
     _fields_ = [("M", C.c_int64), ("N", C.c_int64), ("K", C.c_int64), ("BM", C.c_int32), ("BN", C.c_int32),
                 ("A", Mat), ("B", Mat), ("C", Mat), ("a_trans", C.c_int32), ("b_trans", C.c_int32),
                 ("P", C.c_int32), ("page_bytes", C.c_int64), ("place", C.c_int32 * 3), ("assign", C.c_int32),
-                ("strip_tiling", C.c_int32)]
+                ("strip_tiling", C.c_int32), ("part_m", C.c_int32)]
 
 
 _lib = None

@@ -8,6 +8,9 @@
 //
 // Every function cites the passage of the paper it restates:
 //   Eq. 1  : g = floor(n / w), n' = n mod w, w = N / G
+//            (reading for N not a multiple of G, which the paper leaves out: w = ceil(N / G), Eq. 1 unchanged, the
+//            last strip is narrower -- N - (G-1)*w columns, at least one -- and every strip stays a contiguous
+//            rows x width block, strip g starting g strides in: a packed buffer is still a bijection onto [0, K*N))
 //   Eq. 2  : index_row(k, n) = k*N + n
 //   Eq. 3  : index_CCL(k, n) = g*K*w + k*w + n'
 //   Sec. 3.2 (last paragraph): a strip of K*w elements may be aligned to the
@@ -54,7 +57,7 @@ extern "C" {
 enum { ORC_ROWMAJOR = 0, ORC_CCL = 1, ORC_CCL_INTERLEAVED = 2 };
 enum { ORC_PART_NONE = 0, ORC_PART_ROWS = 1, ORC_PART_COLS = 2 };
 enum { ORC_PLACE_RR = 0, ORC_PLACE_BLOCK = 1, ORC_PLACE_BEST = 2 };
-enum { ORC_ASSIGN_N = 0, ORC_ASSIGN_M = 1, ORC_ASSIGN_EXPLICIT = 2 };
+enum { ORC_ASSIGN_N = 0, ORC_ASSIGN_M = 1, ORC_ASSIGN_EXPLICIT = 2, ORC_ASSIGN_2D = 3 };
 
 // A stored matrix: rows x cols, cols contiguous in the row-major view.
 typedef struct {
@@ -77,6 +80,7 @@ typedef struct {
     int32_t place[3];
     int32_t assign;
     int32_t strip_tiling;
+    int32_t part_m;             // ORC_ASSIGN_2D: the output is cut into part_m x (P / part_m) blocks, one per chiplet
 } orc_traffic_desc;
 
 }  // extern "C"
@@ -89,9 +93,9 @@ bool mat_ok(const orc_mat& m) {
     if (m.layout != ORC_ROWMAJOR && m.layout != ORC_CCL && m.layout != ORC_CCL_INTERLEAVED) return false;
     if (m.part < 0 || m.part > 2) return false;
     if (m.strip_align_bytes < 0 || m.strip_align_bytes % m.elem_bytes) return false;
-    if (m.layout != ORC_ROWMAJOR) {
-        if (m.part == ORC_PART_COLS && m.cols % m.P) return false;  // w = N/G must be whole
-        if (m.part == ORC_PART_ROWS && m.rows % m.P) return false;
+    if (m.layout != ORC_ROWMAJOR) {                    // every strip holds at least one column / row
+        if (m.part == ORC_PART_COLS && (int64_t)(m.P - 1) * ((m.cols + m.P - 1) / m.P) >= m.cols) return false;
+        if (m.part == ORC_PART_ROWS && (int64_t)(m.P - 1) * ((m.rows + m.P - 1) / m.P) >= m.rows) return false;
     }
     if (m.layout == ORC_CCL_INTERLEAVED && m.part != ORC_PART_NONE && m.strip_align_bytes <= 0) return false;
     return true;
@@ -100,11 +104,19 @@ bool mat_ok(const orc_mat& m) {
 bool is_ccl(const orc_mat& m) { return m.layout != ORC_ROWMAJOR && m.part != ORC_PART_NONE; }
 bool is_interleaved(const orc_mat& m) { return m.layout == ORC_CCL_INTERLEAVED && m.part != ORC_PART_NONE; }
 
-// Elements of one strip (K*w in the paper's notation).
-int64_t strip_elems(const orc_mat& m) {
-    return (m.part == ORC_PART_COLS) ? m.rows * (m.cols / m.P) : (m.rows / m.P) * m.cols;
+// Per-chiplet width w of Eq. 1 (split along columns) / rows per strip (split along rows): N / G, rounded up when N is
+// not a multiple of G; the last strip then holds what is left.
+int64_t strip_w(const orc_mat& m) { return (m.cols + m.P - 1) / m.P; }
+int64_t strip_h(const orc_mat& m) { return (m.rows + m.P - 1) / m.P; }
+int64_t strip_w_of(const orc_mat& m, int64_t g) { return std::min(strip_w(m), m.cols - g * strip_w(m)); }
+int64_t strip_h_of(const orc_mat& m, int64_t g) { return std::min(strip_h(m), m.rows - g * strip_h(m)); }
+
+// Elements of strip g, and of the largest strip (K*w in the paper's notation).
+int64_t strip_elems_of(const orc_mat& m, int64_t g) {
+    return (m.part == ORC_PART_COLS) ? m.rows * strip_w_of(m, g) : strip_h_of(m, g) * m.cols;
 }
-// Interleaved layout: chunks of strip_align_bytes each strip needs.
+int64_t strip_elems(const orc_mat& m) { return strip_elems_of(m, 0); }
+// Interleaved layout: chunks of strip_align_bytes each strip gets (those of the largest strip).
 int64_t strip_chunks(const orc_mat& m) {
     return (strip_elems(m) * m.elem_bytes + m.strip_align_bytes - 1) / m.strip_align_bytes;
 }
@@ -122,7 +134,10 @@ int64_t strip_stride(const orc_mat& m) {
 int64_t buffer_elems(const orc_mat& m) {
     if (!is_ccl(m)) return m.rows * m.cols;
     if (is_interleaved(m)) return strip_chunks(m) * m.P * (m.strip_align_bytes / m.elem_bytes);
-    return (int64_t)m.P * strip_stride(m);
+    // P-1 strides, then the last strip (rounded up like the others when strips are aligned)
+    int64_t last = strip_elems_of(m, m.P - 1);
+    if (m.strip_align_bytes) last = (last * m.elem_bytes + m.strip_align_bytes - 1) / m.strip_align_bytes * m.strip_align_bytes / m.elem_bytes;
+    return (int64_t)(m.P - 1) * strip_stride(m) + last;
 }
 
 // Interleaved layout: element `o` of strip g's packed contents (Eq. 3 inside the strip) lives in that strip's chunk
@@ -136,14 +151,15 @@ int64_t interleave(const orc_mat& m, int64_t g, int64_t o) {
 int64_t map_offset(const orc_mat& m, int64_t r, int64_t c) {
     if (!is_ccl(m)) return r * m.cols + c;            // Eq. 2
     if (m.part == ORC_PART_COLS) {
-        int64_t w = m.cols / m.P;                      // per-chiplet width
+        int64_t w = strip_w(m);                        // per-chiplet width
         int64_t g = c / w;                             // Eq. 1
         int64_t cp = c % w;                            // Eq. 1
-        if (is_interleaved(m)) return interleave(m, g, r * w + cp);
-        return g * strip_stride(m) + r * w + cp;       // Eq. 3
+        int64_t wg = strip_w_of(m, g);                 // = w, except in a narrower last strip
+        if (is_interleaved(m)) return interleave(m, g, r * wg + cp);
+        return g * strip_stride(m) + r * wg + cp;      // Eq. 3
     }
     // Split along rows: each strip is h whole rows, already contiguous (Sec. 2.2).
-    int64_t h = m.rows / m.P;
+    int64_t h = strip_h(m);
     if (is_interleaved(m)) return interleave(m, r / h, (r % h) * m.cols + c);
     return (r / h) * strip_stride(m) + (r % h) * m.cols + c;
 }
@@ -151,25 +167,21 @@ int64_t map_offset(const orc_mat& m, int64_t r, int64_t c) {
 int map_inverse(const orc_mat& m, int64_t off, int64_t* r, int64_t* c) {
     if (off < 0 || off >= buffer_elems(m)) return -1;
     if (!is_ccl(m)) { *r = off / m.cols; *c = off % m.cols; return 0; }
-    int64_t st, g, rem;
+    int64_t g, rem;
     if (is_interleaved(m)) {                           // undo the chunk interleave, then proceed as for a packed strip
         int64_t S = m.strip_align_bytes, b = off * m.elem_bytes, chunk = b / S;
         g = chunk % m.P;
         rem = (chunk / m.P * S + b % S) / m.elem_bytes;
-        st = strip_elems(m);
-        if (rem >= st) return -2;
     } else {
-        st = strip_stride(m);
+        int64_t st = strip_stride(m);
         g = off / st; rem = off % st;
     }
+    if (rem >= strip_elems_of(m, g)) return -2;        // inside the padding of strip g
     if (m.part == ORC_PART_COLS) {
-        int64_t w = m.cols / m.P;
-        if (rem >= m.rows * w) return -2;              // inside the padding of strip g
-        *r = rem / w; *c = g * w + rem % w; return 0;
+        int64_t wg = strip_w_of(m, g);
+        *r = rem / wg; *c = g * strip_w(m) + rem % wg; return 0;
     }
-    int64_t h = m.rows / m.P;
-    if (rem >= h * m.cols) return -2;
-    *r = g * h + rem / m.cols; *c = rem % m.cols; return 0;
+    *r = g * strip_h(m) + rem / m.cols; *c = rem % m.cols; return 0;
 }
 
 inline float bf16_to_f32(uint16_t h) { uint32_t u = (uint32_t)h << 16; float f; std::memcpy(&f, &u, 4); return f; }
@@ -182,35 +194,48 @@ inline uint16_t f32_to_bf16_rne(float f) {
 // ---- tile grid of the execution model (Sec. 2.2 / Sec. 4.1: one CTA per output tile) ----
 struct Seg { int64_t lo, hi; };
 
-// Tiles of one dimension.  strip_tiled: every strip of len/P is tiled on its own,
-// so that no tile straddles two strips; otherwise plain ceil(len/B) tiles.
+// Tiles of one dimension cut into P strips of ceil(len/P) (the last one holds the rest).  strip_tiled: every strip is
+// tiled on its own, so that no tile straddles two strips; otherwise plain ceil(len/B) tiles.
 std::vector<Seg> tile_dim(int64_t len, int64_t B, int P, bool strip_tiled) {
     std::vector<Seg> v;
     if (!strip_tiled) { for (int64_t s = 0; s < len; s += B) v.push_back({s, std::min(len, s + B)}); return v; }
-    int64_t w = len / P;
-    for (int g = 0; g < P; ++g)
-        for (int64_t s = 0; s < w; s += B) v.push_back({g * w + s, g * w + std::min(w, s + B)});
+    int64_t w = (len + P - 1) / P;
+    for (int g = 0; g < P; ++g) {
+        const int64_t wg = std::min(w, len - g * w);
+        for (int64_t s = 0; s < wg; s += B) v.push_back({g * w + s, g * w + std::min(wg, s + B)});
+    }
     return v;
 }
 
 struct Tile { int64_t m0, m1, n0, n1; int32_t q; };
 
+// every strip of a dimension of length len cut into P holds at least one element
+bool strips_ok(int64_t len, int64_t P) { return P >= 1 && (P - 1) * ((len + P - 1) / P) < len; }
+
+// Sec. 3.1 / 4.1: the output is partitioned over the chiplets and a CTA runs on the chiplet that owns its tile.
+// N strips, M strips, an explicit table, or a 2-D partition into part_m x (P / part_m) blocks (chiplet qm * Pn + qn
+// owns block (qm, qn)) -- Sec. 4.1 sweeps the output partition and keeps the best.
 int enumerate_tiles(const orc_traffic_desc& d, const int32_t* explicit_q, std::vector<Tile>& out) {
     if (d.M <= 0 || d.N <= 0 || d.K <= 0 || d.BM <= 0 || d.BN <= 0 || d.P < 1) return -1;
-    bool n_strips = d.assign == ORC_ASSIGN_N, m_strips = d.assign == ORC_ASSIGN_M;
-    if (n_strips && d.N % d.P) return -1;
-    if (m_strips && d.M % d.P) return -1;
+    if (d.assign < 0 || d.assign > 3) return -1;
+    int Pm = 1, Pn = 1;
+    if (d.assign == ORC_ASSIGN_N) Pn = d.P;
+    else if (d.assign == ORC_ASSIGN_M) Pm = d.P;
+    else if (d.assign == ORC_ASSIGN_2D) {
+        if (d.part_m < 1 || d.P % d.part_m) return -1;
+        Pm = d.part_m; Pn = d.P / d.part_m;
+    }
+    if (!strips_ok(d.N, Pn) || !strips_ok(d.M, Pm)) return -1;
     if (d.assign == ORC_ASSIGN_EXPLICIT && !explicit_q) return -1;
-    if (d.assign < 0 || d.assign > 2) return -1;
-    auto tm = tile_dim(d.M, d.BM, d.P, m_strips && d.strip_tiling);
-    auto tn = tile_dim(d.N, d.BN, d.P, n_strips && d.strip_tiling);
+    const int64_t wM = (d.M + Pm - 1) / Pm, wN = (d.N + Pn - 1) / Pn;
+    auto tm = tile_dim(d.M, d.BM, Pm, Pm > 1 && d.strip_tiling);
+    auto tn = tile_dim(d.N, d.BN, Pn, Pn > 1 && d.strip_tiling);
     for (size_t i = 0; i < tm.size(); ++i)
         for (size_t j = 0; j < tn.size(); ++j) {
             Tile t{tm[i].lo, tm[i].hi, tn[j].lo, tn[j].hi, 0};
             int64_t idx = (int64_t)i * (int64_t)tn.size() + (int64_t)j;
-            if (n_strips) t.q = (int32_t)(t.n0 / (d.N / d.P));       // chiplet owning the tile's columns
-            else if (m_strips) t.q = (int32_t)(t.m0 / (d.M / d.P));
-            else { t.q = explicit_q[idx]; if (t.q < 0 || t.q >= d.P) return -1; }
+            if (d.assign == ORC_ASSIGN_EXPLICIT) { t.q = explicit_q[idx]; if (t.q < 0 || t.q >= d.P) return -1; }
+            else t.q = (int32_t)((t.m0 / wM) * Pn + t.n0 / wN);      // the block holding the tile's first element
             out.push_back(t);
         }
     return 0;
@@ -262,15 +287,15 @@ void for_each_piece_elem(const orc_traffic_desc& d, const orc_mat& m, int64_t r0
 template <class F>
 void for_each_piece_run(const orc_traffic_desc& d, const orc_mat& m, int64_t r0, int64_t r1, int64_t c0, int64_t c1, F&& f) {
     int64_t S = d.page_bytes, e = m.elem_bytes;
-    int64_t w = (is_ccl(m) && m.part == ORC_PART_COLS) ? m.cols / m.P : m.cols;
+    int64_t w = (is_ccl(m) && m.part == ORC_PART_COLS) ? strip_w(m) : m.cols;
     for (int64_t r = r0; r < r1; ++r) {
         int64_t c = c0;
         while (c < c1) {
             int64_t cend = std::min(c1, (c / w + 1) * w);
             if (is_interleaved(m)) {                   // contiguity also ends at every chunk of the interleave
                 int64_t Si = m.strip_align_bytes;
-                int64_t rr = (m.part == ORC_PART_ROWS) ? r % (m.rows / m.P) : r;
-                int64_t roww = (m.part == ORC_PART_COLS) ? w : m.cols;
+                int64_t rr = (m.part == ORC_PART_ROWS) ? r % strip_h(m) : r;
+                int64_t roww = (m.part == ORC_PART_COLS) ? strip_w_of(m, c / w) : m.cols;
                 int64_t packed = (rr * roww + (m.part == ORC_PART_COLS ? c % w : c)) * e;   // byte inside the strip
                 int64_t sub = std::min<int64_t>((cend - c) * e, (packed / Si + 1) * Si - packed);
                 cend = c + sub / e;

@@ -17,7 +17,7 @@ OK, ERR_INVALID_ARG, ERR_SHAPE, ERR_ALIGN, ERR_UNSUPPORTED, ERR_CUDA, ERR_WORKSP
 ROWMAJOR, CCL, CCL_INTERLEAVED = 0, 1, 2
 PART_NONE, PART_ROWS, PART_COLS = 0, 1, 2
 PLACE_RR, PLACE_BLOCK, PLACE_BEST = 0, 1, 2
-ASSIGN_N_STRIPS, ASSIGN_M_STRIPS, ASSIGN_EXPLICIT = 0, 1, 2
+ASSIGN_N_STRIPS, ASSIGN_M_STRIPS, ASSIGN_EXPLICIT, ASSIGN_2D = 0, 1, 2, 3
 
 EXPORTS = ["ccl_map_offset", "ccl_map_inverse", "ccl_buffer_bytes", "ccl_strip_stride", "ccl_repack", "ccl_repack_batched", "ccl_repack_transpose", "ccl_gemm_workspace",
            "ccl_gemm", "ccl_gemm_batched_workspace", "ccl_gemm_batched", "ccl_gemm_grouped", "ccl_gemm_grouped_swiglu", "ccl_gemm_grouped_k", "ccl_gemm_axpby", "ccl_gemm_swiglu", "ccl_gemm_static_ws", "ccl_gemm_status", "ccl_selftest_wait_timeout", "ccl_traffic_sizes", "ccl_traffic", "ccl_traffic_l2", "ccl_traffic_lru", "ccl_probe_l2_latency", "ccl_last_error", "ccl_launch_count", "ccl_version"]
@@ -49,7 +49,8 @@ class TrafficDesc(C.Structure):
     """ccl_traffic_desc"""
     _fields_ = [("M", C.c_int64), ("N", C.c_int64), ("K", C.c_int64), ("BM", C.c_int32), ("BN", C.c_int32),
                 ("A", Mat), ("B", Mat), ("C", Mat), ("a_trans", C.c_int32), ("b_trans", C.c_int32), ("P", C.c_int32),
-                ("page_bytes", C.c_int64), ("place", C.c_int32 * 3), ("assign", C.c_int32), ("strip_tiling", C.c_int32)]
+                ("page_bytes", C.c_int64), ("place", C.c_int32 * 3), ("assign", C.c_int32), ("strip_tiling", C.c_int32),
+                ("part_m", C.c_int32)]
 
 
 class L2Model(C.Structure):

@@ -108,13 +108,85 @@ def test_inverse_packed_roundtrip():
 
 def test_rejects_bad_descriptors():
     with pytest.raises(ValueError):
-        orc.map_table(ccl_cols(4, 10, 4))          # w = N/G not whole
+        orc.map_table(ccl_cols(4, 9, 4))           # w = ceil(9/4) = 3: the fourth strip would be empty
     with pytest.raises(ValueError):
-        orc.map_table(ccl_rows(5, 8, 2))
+        orc.map_table(ccl_rows(4, 8, 3))           # h = 2: the third strip would be empty
     with pytest.raises(ValueError):
         orc.map_offset(ccl_cols(4, 8, 2), 4, 0)    # out of range
     with pytest.raises(ValueError):
         orc.map_table(orc.Mat(4, 8, 3))            # element size
+
+
+# ---------------------------------------------------------------- widths the chiplet count does not divide
+
+def test_ragged_worked_example():
+    rows = [l.split() for l in open(os.path.join(GOLD, "ragged_ccl_index.txt")) if l.strip() and not l.startswith("#")]
+    hdr = {k: int(v) for k, v in rows[:3]}
+    table = np.array(rows[3:], dtype=np.int64)
+    m = ccl_cols(hdr["K"], hdr["N"], hdr["G"])
+    np.testing.assert_array_equal(orc.map_table(m), table)
+    assert orc.buffer_bytes(m) == hdr["K"] * hdr["N"] * 2 and orc.strip_stride(m) == 9
+    np.testing.assert_array_equal(orc.map_table(ccl_rows(3, 7, 2)), np.arange(21).reshape(3, 7))
+
+
+@pytest.mark.parametrize("R,Cc,P", [(3, 7, 3), (4, 10, 4), (5, 200, 3), (64, 1537, 4), (33, 770, 8), (17, 9, 2), (6, 1000, 7)])
+def test_ragged_bijection_strips_and_slices(R, Cc, P):
+    """Packed ragged CCL is a bijection onto [0, R*C); strip g is the contiguous block after the g strips before it and
+    holds, row-major, the column slice [g w, min(C, (g+1) w)) -- written here with numpy slices, not with the map."""
+    m = ccl_cols(R, Cc, P)
+    t = orc.map_table(m)
+    np.testing.assert_array_equal(np.sort(t.reshape(-1)), np.arange(R * Cc))
+    w = -(-Cc // P)
+    x = _rand_u16(R, Cc, seed=R + Cc)
+    want = np.concatenate([x[:, g * w:min(Cc, (g + 1) * w)].reshape(-1) for g in range(P)])
+    np.testing.assert_array_equal(orc.repack(m, x, 0), want)
+    np.testing.assert_array_equal(orc.repack(m, orc.repack(m, x, 0), 1).reshape(R, Cc), x)
+    for off in range(0, R * Cc, max(1, R * Cc // 97)):
+        rc, r, c = orc.map_inverse(m, off)
+        assert rc == 0 and t[r, c] == off
+    # split along rows: strips of ceil(R/P) whole rows stay where they are
+    if (P - 1) * -(-R // P) < R:
+        np.testing.assert_array_equal(orc.map_table(ccl_rows(R, Cc, P)), np.arange(R * Cc).reshape(R, Cc))
+
+
+@pytest.mark.parametrize("R,Cc,P,align", [(3, 7, 3, 64), (5, 200, 3, 4096), (9, 1537, 4, 256)])
+def test_ragged_aligned_strips(R, Cc, P, align):
+    """Aligned strips: every strip base is a multiple of the alignment, the map stays injective, padding holes invert to -2
+    and the repack writes zeros there."""
+    m = ccl_cols(R, Cc, P, align=align)
+    t = orc.map_table(m)
+    w = -(-Cc // P)
+    st = orc.strip_stride(m)
+    assert (st * 2) % align == 0 and st >= R * w
+    assert len(np.unique(t)) == R * Cc
+    for g in range(P):
+        assert t[0, g * w] == g * st
+    n = orc.buffer_bytes(m) // 2
+    assert n == (P - 1) * st + -(-(R * (Cc - (P - 1) * w) * 2) // align) * align // 2
+    x = np.random.default_rng(1).integers(1, 65536, size=(R, Cc), dtype=np.uint16)
+    buf = orc.repack(m, x, 0)
+    used = np.zeros(n, dtype=bool)
+    used[t.reshape(-1)] = True
+    assert (buf[~used] == 0).all() and (buf[used] != 0).all()
+    holes = np.flatnonzero(~used)
+    for off in holes[:: max(1, len(holes) // 50)]:
+        assert orc.map_inverse(m, int(off))[0] == -2
+
+
+def test_ragged_interleaved_is_a_chunk_permutation_of_aligned():
+    """Page-interleaved ragged CCL: chunk j of strip g sits at chunk j*G + g; every strip gets the chunk count of the widest."""
+    R, Cc, P, S = 5, 202, 3, 128
+    mi = orc.Mat(R, Cc, 2, P, orc.PART_COLS, orc.CCL_INTERLEAVED, S)
+    x = _rand_u16(R, Cc, seed=5)
+    w = -(-Cc // P)
+    chunks = -(-(R * w * 2) // S)
+    buf = orc.repack(mi, x, 0).reshape(chunks, P, S // 2)
+    for g in range(P):
+        strip = x[:, g * w:min(Cc, (g + 1) * w)].reshape(-1)
+        got = buf[:, g, :].reshape(-1)
+        np.testing.assert_array_equal(got[:strip.size], strip)
+        assert (got[strip.size:] == 0).all()
+    np.testing.assert_array_equal(orc.repack(mi, buf.reshape(-1), 1).reshape(R, Cc), x)
 
 
 # ---------------------------------------------------------------- repack

@@ -196,8 +196,90 @@ def test_explicit_assignment_and_bad_descriptors():
     with pytest.raises(ValueError):
         orc.traffic(d, explicit_q=np.array([2, 0, 0, 1], dtype=np.int32))
     with pytest.raises(ValueError):
-        orc.traffic(desc(8, 9, 4, 2, 16))          # N % P != 0
+        orc.traffic(desc(8, 9, 4, 4, 16))          # strips of ceil(9/4) = 3 columns would leave the fourth chiplet none
     bad = desc(8, 8, 4, 2, 16)
     bad.A.rows = 9
     with pytest.raises(ValueError):
         orc.traffic(bad)
+
+
+# ---------------------------------------------------------------- 2-D output partitions and ragged strips
+
+def desc_2d(M, N, K, P, Pm, S, **kw):
+    d = desc(M, N, K, P, S, assign=orc.ASSIGN_N, parts=(orc.PART_NONE,) * 3, **kw)
+    d.assign, d.part_m = orc.ASSIGN_2D, Pm
+    return d
+
+
+def test_hand_enumerated_2d_partition():
+    rows = [l.split() for l in open(os.path.join(GOLD, "tiny_traffic_2d.txt")) if l.strip() and not l.startswith("#")]
+    cases = {"rr": desc_2d(4, 8, 4, 4, 2, 16, BM=2, BN=4), "best": desc_2d(4, 8, 4, 4, 2, 16, BM=2, BN=4, place=(orc.PLACE_BEST,) * 3)}
+    for level in ("elem", "runs"):
+        res = {k: orc.traffic(v, level=level) for k, v in cases.items()}
+        for case, op, tile, loc, rem in rows:
+            assert tuple(res[case]["per_cta"][int(tile), "ABC".index(op)]) == (int(loc), int(rem)), (case, op, tile)
+    np.testing.assert_array_equal(orc.traffic_tiles(cases["rr"])[:, 4], [0, 1, 2, 3])
+    np.testing.assert_array_equal(orc.traffic(cases["best"])["owner"][A_], [0, 2])
+    np.testing.assert_array_equal(orc.traffic(cases["best"])["owner"][C_], [0, 0, 2, 2])
+
+
+@pytest.mark.parametrize("M,N,K,P,S,BM,BN", [(128, 256, 64, 4, 256, 32, 32), (96, 384, 48, 8, 128, 16, 64), (130, 200, 40, 2, 64, 64, 64)])
+def test_2d_partition_degenerates_to_strips(M, N, K, P, S, BM, BN):
+    """part_m = 1 is the N-strip partition and part_m = P the M-strip partition, tile for tile."""
+    for Pm, assign in ((1, orc.ASSIGN_N), (P, orc.ASSIGN_M)):
+        if assign == orc.ASSIGN_M and (P - 1) * -(-M // P) >= M:
+            continue
+        a = orc.traffic(desc_2d(M, N, K, P, Pm, S, BM=BM, BN=BN), level="runs")
+        b = orc.traffic(desc(M, N, K, P, S, assign=assign, parts=(orc.PART_NONE,) * 3, BM=BM, BN=BN), level="runs")
+        for k in ("per_cta", "totals"):
+            np.testing.assert_array_equal(a[k], b[k])
+
+
+@pytest.mark.parametrize("kw", [dict(M=128, N=256, K=64, P=4, Pm=2, S=256, BM=32, BN=32), dict(M=120, N=200, K=40, P=6, Pm=3, S=64, BM=16, BN=32),
+                                dict(M=130, N=384, K=96, P=8, Pm=2, S=512, BM=64, BN=64, strip_tiling=0),
+                                dict(M=131, N=203, K=24, P=6, Pm=2, S=128, BM=32, BN=32)])
+def test_2d_partition_invariants(kw):
+    Pm = kw["Pm"]
+    for place in PLACES:
+        d = desc_2d(place=place, **kw)
+        res, runs = orc.traffic(d, level="elem"), orc.traffic(d, level="runs")
+        tiles = orc.traffic_tiles(d)
+        np.testing.assert_array_equal(res["per_cta"], runs["per_cta"])
+        np.testing.assert_array_equal(res["per_cta"].sum(axis=2), touched_bytes(d, tiles))
+        Pn = d.P // Pm
+        wM, wN = -(-d.M // Pm), -(-d.N // Pn)
+        np.testing.assert_array_equal(tiles[:, 4], (tiles[:, 0] // wM) * Pn + tiles[:, 2] // wN)
+        if d.strip_tiling:                               # no tile straddles a block
+            assert ((tiles[:, 1] - 1) // wM == tiles[:, 0] // wM).all() and ((tiles[:, 3] - 1) // wN == tiles[:, 2] // wN).all()
+        for X in range(3):
+            assert res["per_page"][X].sum() == res["per_cta"][:, X].sum()
+    with pytest.raises(ValueError):
+        bad = desc_2d(**kw)
+        bad.part_m = 5 if kw["P"] % 5 else 7
+        orc.traffic(bad)
+
+
+@pytest.mark.parametrize("N,P", [(200, 3), (1000, 7), (385, 4)])
+def test_ragged_strips_in_the_counter(N, P):
+    """N not a multiple of P: strips of ceil(N/P) columns and a narrower last one; element- and run-level counts agree, every
+    byte is accounted for, tiles stay inside their strips, and CCL keeps each strip one contiguous block."""
+    M, K, S = 96, 40, 256
+    w = -(-N // P)
+    for lay in LAYS:
+        for place in PLACES[:3]:
+            d = desc(M, N, K, P, S, lay, place, BM=32, BN=32)
+            res, runs = orc.traffic(d, level="elem"), orc.traffic(d, level="runs")
+            tiles = orc.traffic_tiles(d)
+            np.testing.assert_array_equal(res["per_cta"], runs["per_cta"])
+            np.testing.assert_array_equal(res["per_cta"].sum(axis=2), touched_bytes(d, tiles))
+            np.testing.assert_array_equal(tiles[:, 4], tiles[:, 2] // w)
+            assert ((tiles[:, 3] - 1) // w == tiles[:, 2] // w).all()
+            assert sorted(set(tiles[:, 4])) == list(range(P))
+    # CCL B: the bytes a strip's tiles read are exactly the strip's block [g K w, g K w + K w_g) of the buffer
+    d = desc(M, N, K, P, S, ("row", "ccl", "row"), (orc.PLACE_RR,) * 3, BM=32, BN=32)
+    pp = orc.traffic(d)["per_page"][B_]                  # [pages, P] bytes of each page demanded by each chiplet
+    for g in range(P):
+        lo, hi = g * K * w * 2, (g * K * w + K * min(w, N - g * w)) * 2
+        touched = np.flatnonzero(pp[:, g])
+        assert touched.min() == lo // S and touched.max() == (hi - 1) // S
+        assert pp[:, g].sum() == (M // 32) * (hi - lo)
