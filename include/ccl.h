@@ -57,7 +57,8 @@ typedef enum {
 } ccl_status;
 
 typedef enum { CCL_ROWMAJOR = 0, CCL_CCL = 1, CCL_CCL_INTERLEAVED = 2 } ccl_layout; /* physical order of a buffer */
-typedef enum { CCL_PART_NONE = 0, CCL_PART_ROWS = 1, CCL_PART_COLS = 2 } ccl_part; /* stored dim split over chiplets */
+typedef enum { CCL_PART_NONE = 0, CCL_PART_ROWS = 1, CCL_PART_COLS = 2, /* stored dim split over chiplets */
+               CCL_PART_2D = 3 /* only as the out_part of a GEMM: the output cut into blocks along both dimensions */ } ccl_part;
 
 /*
  * Descriptor of one stored matrix.
@@ -67,10 +68,15 @@ typedef enum { CCL_PART_NONE = 0, CCL_PART_ROWS = 1, CCL_PART_COLS = 2 } ccl_par
  *       stride = rows*w when strip_align_bytes == 0 (packed, Eq. 3 literally), else
  *       rows*w*e rounded up to strip_align_bytes (Sec. 3.2: a strip can be aligned to
  *       the placement granularity).  Padding elements belong to no (r,c).
+ *       cols not a multiple of P (the paper assumes it is; this library's reading): w = ceil(cols/P),
+ *       Eq. 1 unchanged, the last strip keeps the cols - (P-1)*w >= 1 columns that are left and is a
+ *       contiguous rows x (its width) block like the others: offset = g*stride + r*w_g + c' with w_g the
+ *       width of strip g.  A packed buffer is still exactly rows*cols elements.  Map, repack and traffic
+ *       take such matrices; ccl_gemm returns CCL_ERR_UNSUPPORTED for them.
  *   layout = CCL_CCL, part = CCL_PART_ROWS (split along the non-contiguous dimension,
  *       which Sec. 2.2 calls coarse-grained: already contiguous):
- *       h = rows/P, offset = (r / h)*stride + (r mod h)*cols + c, stride = h*cols
- *       (rounded up likewise).
+ *       h = rows/P (rounded up, the last strip keeping the rest, as above), offset = (r / h)*stride +
+ *       (r mod h)*cols + c, stride = h*cols (rounded up likewise).
  *   layout = CCL_CCL_INTERLEAVED (either part): the page-interleaved form of CCL, under which a plain
  *       address-driven round-robin mapping at the chunk size already puts every strip on its own
  *       chiplet (the setting Sec. 3.3 / 4.1 evaluate).  strip_align_bytes is the chunk size S (> 0).  Element
@@ -81,8 +87,8 @@ typedef enum { CCL_PART_NONE = 0, CCL_PART_ROWS = 1, CCL_PART_COLS = 2 } ccl_par
  *       Map, repack and traffic take every such layout; ccl_gemm takes those whose chunks line up with the
  *       strip rows (see ccl_gemm).
  *   A CCL layout with part = CCL_PART_NONE behaves as CCL_ROWMAJOR.
- * Requirements: rows, cols > 0; elem_bytes in {1,2,4}; P >= 1; the split dimension
- * divisible by P (else CCL_ERR_SHAPE); strip_align_bytes >= 0 and a multiple of e.
+ * Requirements: rows, cols > 0; elem_bytes in {1,2,4}; P >= 1; every strip of the split dimension
+ * non-empty, i.e. (P-1)*ceil(dim/P) < dim (else CCL_ERR_SHAPE); strip_align_bytes >= 0 and a multiple of e.
  */
 typedef struct ccl_mat {
     int64_t rows, cols;
@@ -145,7 +151,9 @@ ccl_status ccl_repack_transpose(const ccl_mat* m, const void* src_dev, void* dst
  *   B stored [K x N] (b_trans = 0) or [N x K] (b_trans = 1);   C stored [M x N].
  * out_part / P / grouped_raster describe how C is partitioned over chiplets and whether CTA
  * group g computes only strip g of C (Sec. 3.1: each CTA runs on the chiplet that owns its
- * output tile): out_part = CCL_PART_COLS splits N, CCL_PART_ROWS splits M, CCL_PART_NONE (or
+ * output tile): out_part = CCL_PART_COLS splits N, CCL_PART_ROWS splits M, CCL_PART_2D cuts C into
+ * part_m x (P / part_m) blocks (group qm * (P / part_m) + qn computes block (qm, qn); M divisible by
+ * part_m and N by P / part_m -- the output-partition choices Sec. 4.1 sweeps), CCL_PART_NONE (or
  * grouped_raster = 0) uses one plain raster.  The result does not depend on these choices.
  * Requirements (else CCL_ERR_UNSUPPORTED / CCL_ERR_ALIGN, nothing launched): elem_bytes = 2;
  * every contiguous extent a tile row lives in (cols, or w for CCL_PART_COLS) a multiple of 8
@@ -164,6 +172,7 @@ typedef struct ccl_gemm_desc {
     int32_t out_part; /* ccl_part */
     int32_t P;
     int32_t grouped_raster;
+    int32_t part_m;   /* out_part == CCL_PART_2D: blocks along M (a divisor of P); ignored otherwise */
 } ccl_gemm_desc;
 
 /* Bytes of device workspace ccl_gemm needs for this problem (0 when none). */
@@ -295,7 +304,7 @@ ccl_status ccl_gemm_static_ws(const ccl_gemm_desc* d, const void* A_dev, const v
 /* ---- remote-traffic counter (Sec. 4.1 metric, every touched byte counted: no L2 filter) */
 
 typedef enum { CCL_PLACE_RR = 0, CCL_PLACE_BLOCK = 1, CCL_PLACE_BEST = 2 } ccl_place;
-typedef enum { CCL_ASSIGN_N_STRIPS = 0, CCL_ASSIGN_M_STRIPS = 1, CCL_ASSIGN_EXPLICIT = 2 } ccl_assign;
+typedef enum { CCL_ASSIGN_N_STRIPS = 0, CCL_ASSIGN_M_STRIPS = 1, CCL_ASSIGN_EXPLICIT = 2, CCL_ASSIGN_2D = 3 } ccl_assign;
 
 /*
  * One CTA per BM x BN output tile (Sec. 2.2); it reads its rows of A over all K, its
@@ -307,9 +316,13 @@ typedef enum { CCL_ASSIGN_N_STRIPS = 0, CCL_ASSIGN_M_STRIPS = 1, CCL_ASSIGN_EXPL
  *                     strips are whole pages this is "page -> its strip's chiplet"
  *   CCL_PLACE_BEST  : owner = the chiplet that demands most bytes of the page (ties: lowest
  *                     index; untouched pages: 0): the best any page-granular mapping can do.
- * Tile -> chiplet: CCL_ASSIGN_N_STRIPS: the strip (width N/P) holding the tile's first column;
- * CCL_ASSIGN_M_STRIPS likewise along M; CCL_ASSIGN_EXPLICIT: cta_chiplet_dev[tile].
- * strip_tiling = 1 tiles every strip of the assignment dimension on its own (tiles never
+ * Tile -> chiplet: CCL_ASSIGN_N_STRIPS: the strip (width N/P, rounded up; the last strip holds the
+ * rest) holding the tile's first column; CCL_ASSIGN_M_STRIPS likewise along M; CCL_ASSIGN_2D: the
+ * output is cut into part_m x (P / part_m) blocks of ceil(M / part_m) x ceil(N / (P / part_m)) and the
+ * tile belongs to chiplet qm * (P / part_m) + qn of the block (qm, qn) holding its first element
+ * (Sec. 4.1 sweeps the output partition and reports the best); CCL_ASSIGN_EXPLICIT: cta_chiplet_dev[tile].
+ * Every strip / block must be non-empty (else CCL_ERR_SHAPE).
+ * strip_tiling = 1 tiles every strip of a partitioned dimension on its own (tiles never
  * straddle strips, the last tile of a strip may be partial); 0 tiles globally.  Tiles are
  * numbered tile_m * tiles_n + tile_n.  Partial tiles touch only valid elements.
  */
@@ -323,6 +336,7 @@ typedef struct ccl_traffic_desc {
     int32_t place[3];   /* ccl_place for A, B, C */
     int32_t assign;     /* ccl_assign */
     int32_t strip_tiling;
+    int32_t part_m;     /* CCL_ASSIGN_2D: blocks along M (a divisor of P); ignored otherwise */
 } ccl_traffic_desc;
 
 /* Number of tiles and of pages per operand (sizes of the output arrays below). */
@@ -372,7 +386,7 @@ ccl_status ccl_traffic_l2(const ccl_traffic_desc* d, const int32_t* cta_chiplet_
  *   - C is written once, past the cache.
  * totals_dev: uint64[3][2] (A, B, C) x (local, remote) bytes.
  * Requirements: capacity a whole number of sets, ways <= 32, wave_ctas in [1, 256], page_bytes a multiple of line_bytes (else
- * CCL_ERR_INVALID_ARG / CCL_ERR_UNSUPPORTED); fixed placements only; CCL_ASSIGN_N_STRIPS or _M_STRIPS;
+ * CCL_ERR_INVALID_ARG / CCL_ERR_UNSUPPORTED); fixed placements only; any assignment but CCL_ASSIGN_EXPLICIT;
  * A and B row-major or CCL (page-interleaved -> CCL_ERR_UNSUPPORTED).
  * One warp simulates one cache set of one chiplet; cost grows with tiles x K steps x lines per tile / sets.
  */

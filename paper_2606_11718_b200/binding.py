@@ -15,7 +15,7 @@ LIB_PATH = os.path.join(HERE, "libccl.so")
 
 OK, ERR_INVALID_ARG, ERR_SHAPE, ERR_ALIGN, ERR_UNSUPPORTED, ERR_CUDA, ERR_WORKSPACE, ERR_TIMEOUT, ERR_PADDING = range(9)
 ROWMAJOR, CCL, CCL_INTERLEAVED = 0, 1, 2
-PART_NONE, PART_ROWS, PART_COLS = 0, 1, 2
+PART_NONE, PART_ROWS, PART_COLS, PART_2D = 0, 1, 2, 3
 PLACE_RR, PLACE_BLOCK, PLACE_BEST = 0, 1, 2
 ASSIGN_N_STRIPS, ASSIGN_M_STRIPS, ASSIGN_EXPLICIT, ASSIGN_2D = 0, 1, 2, 3
 
@@ -42,7 +42,7 @@ class GemmDesc(C.Structure):
     """ccl_gemm_desc"""
     _fields_ = [("M", C.c_int64), ("N", C.c_int64), ("K", C.c_int64), ("A", Mat), ("B", Mat), ("C", Mat),
                 ("a_trans", C.c_int32), ("b_trans", C.c_int32), ("out_part", C.c_int32), ("P", C.c_int32),
-                ("grouped_raster", C.c_int32)]
+                ("grouped_raster", C.c_int32), ("part_m", C.c_int32)]
 
 
 class TrafficDesc(C.Structure):

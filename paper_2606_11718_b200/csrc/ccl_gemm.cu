@@ -97,7 +97,9 @@ struct GemmParams {
     int32_t tps_m, tps_n;           // tiles per strip (a tile is 128*CTAS x BN)
     int32_t tiles_m, tiles_n;
     int32_t num_kb;
-    int32_t groups, group_dim;      // chiplet-grouped raster: number of CTA groups, 0 = along N, 1 = along M
+    int32_t groups, group_dim;      // chiplet-grouped raster: number of CTA groups, 0 = along N, 1 = along M, 2 = blocks (2-D)
+    int32_t groups_n;               // 2-D partition: blocks along N (group g owns block (g / groups_n, g % groups_n))
+    FastDiv fd_groups_n;
     int32_t panel;                  // m-tiles per raster panel
     // raster constants the host derives from the grid it launches (see Scheduler)
     int32_t sch_units, sch_gm, sch_gn, sch_upg, sch_floaters, sch_rounds, sch_per_group, sch_pool_per_group;
@@ -362,6 +364,7 @@ struct Scheduler {
         if (tail) { ln = rem / ph; lr = rem - ln * ph; } else p.fd_panel.divmod(rem, ln, lr);
         int lm = pn * p.panel + lr;
         int tm = lm + (p.group_dim == 1 ? g * gm : 0), tn = ln + (p.group_dim == 0 && p.groups > 1 ? g * gn : 0);
+        if (FULL && p.group_dim == 2) { int qm, qn; p.fd_groups_n.divmod(g, qm, qn); tm += qm * gm; tn += qn * gn; }
         int sm, jm, sn, jn;
         p.fd_tps_m.divmod(tm, sm, jm);
         p.fd_tps_n.divmod(tn, sn, jn);
@@ -854,6 +857,7 @@ static int interleave_mode(const MatView& v, int64_t* kr) {
 // k_along_rows: the GEMM's K dimension runs along the stored rows of this operand (never for C)
 static ccl_status check_operand(const MatView& v, const void* ptr, const char* name, bool k_along_rows, int64_t K) {
     if (v.e != 2) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: %s: only 2-byte (bf16) elements are supported", name);
+    if (ragged(v)) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: %s: strips of unequal size (the split dimension is not a multiple of P) are not supported", name);
     int64_t inner = v.split == 2 ? v.w : v.cols;
     if (inner % 8) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: %s: contiguous extent %lld is not a multiple of 8 elements", name, (long long)inner);
     if (v.ichunk) {
@@ -899,7 +903,9 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     if (!d) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: NULL descriptor");
     if (d->M <= 0 || d->N <= 0 || d->K <= 0) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: M, N, K must be positive");
     if (d->M >= (INT64_C(1) << 31) || d->N >= (INT64_C(1) << 31) || d->K >= (INT64_C(1) << 31)) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: dimension too large");
-    if (d->out_part < 0 || d->out_part > 2) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: unknown out_part");
+    if (d->out_part < 0 || d->out_part > 3) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: unknown out_part");
+    if (d->out_part == CCL_PART_2D && (d->part_m < 1 || d->P % d->part_m)) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: part_m (%d) must divide P (%d)", d->part_m, d->P);
+    if (d->out_part == CCL_PART_2D && swiglu) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm_swiglu: a 2-D output partition is not supported");
     if (d->P < 1 || d->P > 255) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: P must be in [1,255]");
     ccl_status s;
     if ((s = make_view(&d->A, "ccl_gemm: A", &plan->va))) return s;
@@ -938,9 +944,15 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
         }
     } else if ((s = merge_width(&Wn, split_width(vb, bt), "N"))) return s;
     if ((s = merge_width(&Wn, split_width(vc, false), "N"))) return s;
-    int groups = 1, group_dim = 0;
+    int groups = 1, group_dim = 0, groups_n = 1;
     if (d->grouped_raster && d->P > 1 && d->out_part != CCL_PART_NONE) {
-        if (d->out_part == CCL_PART_COLS) {
+        if (d->out_part == CCL_PART_2D) {                 // part_m x (P / part_m) blocks of the output, one CTA group each
+            const int pm = d->part_m, pn = d->P / d->part_m;
+            if (d->M % pm || Nc % pn) return fail(CCL_ERR_SHAPE, "ccl_gemm: M / N not divisible by the %d x %d output partition", pm, pn);
+            if (pm > 1 && (s = merge_width(&Wm, d->M / pm, "M"))) return s;
+            if (pn > 1 && (s = merge_width(&Wn, Nc / pn, "N"))) return s;
+            groups = d->P; group_dim = 2; groups_n = pn;
+        } else if (d->out_part == CCL_PART_COLS) {
             if (Nc % d->P) return fail(CCL_ERR_SHAPE, "ccl_gemm: N not divisible by P");
             if ((s = merge_width(&Wn, Nc / d->P, "N"))) return s;
             groups = d->P; group_dim = 0;
@@ -1066,13 +1078,16 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     int units = (int)std::min<int64_t>(ntiles, ctas == 2 ? pairs : sms);
     plan->grid = (unsigned)(units * ctas);
     // grouped raster needs at least one unit per group and whole strips per group
-    if (groups > 1 && units >= groups && (group_dim == 0 ? p.tiles_n % groups == 0 : p.tiles_m % groups == 0)) {
-        p.groups = groups; p.group_dim = group_dim;
-    } else { p.groups = 1; p.group_dim = 0; }
+    const bool whole = group_dim == 0 ? p.tiles_n % groups == 0 : group_dim == 1 ? p.tiles_m % groups == 0
+                                      : (p.tiles_n % groups_n == 0 && p.tiles_m % (groups / groups_n) == 0);
+    if (groups > 1 && units >= groups && whole) {
+        p.groups = groups; p.group_dim = group_dim; p.groups_n = groups_n;
+    } else { p.groups = 1; p.group_dim = 0; p.groups_n = 1; }
+    p.fd_groups_n = make_fastdiv(p.groups_n);
     {   // raster constants (see Scheduler): equal-size groups, floaters, full rounds and the pooled tail
         if (ntiles >= (INT64_C(1) << 31) - 2 * units) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: too many tiles");
-        const int gm = p.group_dim == 1 && p.groups > 1 ? p.tiles_m / p.groups : p.tiles_m;
-        const int gn = p.group_dim == 0 && p.groups > 1 ? p.tiles_n / p.groups : p.tiles_n;
+        const int gm = p.group_dim == 1 && p.groups > 1 ? p.tiles_m / p.groups : p.group_dim == 2 ? p.tiles_m / (p.groups / p.groups_n) : p.tiles_m;
+        const int gn = p.group_dim == 0 && p.groups > 1 ? p.tiles_n / p.groups : p.group_dim == 2 ? p.tiles_n / p.groups_n : p.tiles_n;
         const int64_t per_group = (int64_t)gm * gn * splits * batch;
         p.fd_tiles_per_problem = make_fastdiv((int64_t)gm * gn);
         const int upg = units / p.groups;
@@ -1086,11 +1101,12 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     // pick the panel that minimises them; ties go to the taller panel.
     {
         const int upg = std::max(1, units / p.groups);
-        const int gm = p.group_dim == 1 && p.groups > 1 ? p.tiles_m / p.groups : p.tiles_m;
+        const int gm = p.sch_gm;
         int64_t best_fp = -1;
         for (int pnl = 1; pnl <= std::min(gm, 64); ++pnl) {
             int64_t fp = (int64_t)pnl * bm + (int64_t)p.groups * ((upg + pnl - 1) / pnl) * bn;
             if (p.group_dim == 1 && p.groups > 1) fp = (int64_t)p.groups * pnl * bm + (int64_t)((upg + pnl - 1) / pnl) * bn;
+            if (p.group_dim == 2) fp = (int64_t)(p.groups / p.groups_n) * pnl * bm + (int64_t)p.groups_n * ((upg + pnl - 1) / pnl) * bn;
             if (best_fp < 0 || fp <= best_fp) { best_fp = fp; p.panel = pnl; }
         }
     }
@@ -1249,7 +1265,8 @@ static void make_key(const ccl_gemm_desc* d, const int64_t* batch4, const void* 
     for (int i = 0; i < 4; ++i) k->f[32 + i] = batch4[i];          // batch, strides of A, B, C
     k->f[0] = d->M; k->f[1] = d->N; k->f[2] = d->K;
     put_mat(d->A, k->f + 3); put_mat(d->B, k->f + 10); put_mat(d->C, k->f + 17);
-    k->f[24] = d->a_trans; k->f[25] = d->b_trans; k->f[26] = d->out_part; k->f[27] = d->P; k->f[28] = d->grouped_raster;
+    k->f[24] = d->a_trans; k->f[25] = d->b_trans; k->f[26] = d->out_part; k->f[27] = d->P;
+    k->f[28] = d->grouped_raster + ((int64_t)(d->out_part == CCL_PART_2D ? d->part_m : 0) << 8);
     k->f[29] = (int64_t)reinterpret_cast<uintptr_t>(A); k->f[30] = (int64_t)reinterpret_cast<uintptr_t>(B);
     k->f[31] = (int64_t)reinterpret_cast<uintptr_t>(C);
     k->dev = -1;
@@ -1376,7 +1393,7 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
         {
             const GemmParams& q = plan.p;
             const bool ks = (q.a_mn ? q.a.split == 1 : q.a.split == 2) || (q.b_mn ? q.b.split == 1 : q.b.split == 2);
-            plan.lean = !q.axpby && batch == 1 && !q.a.il_mode && !q.b.il_mode && !q.c.il_mode && !ks && !m_offs && !k_offs && !swiglu;
+            plan.lean = q.group_dim != 2 && !q.axpby && batch == 1 && !q.a.il_mode && !q.b.il_mode && !q.c.il_mode && !ks && !m_offs && !k_offs && !swiglu;
         }
         const uint32_t bnh = (uint32_t)(plan.subn / plan.ctas);   // B rows of one K-major box
         if (!plan.p.a_mn) s = operand_tmap(&prep.ma, plan.va, A_dev, BK, BM, batch, batch4[1]); else s = operand_tmap(&prep.ma, plan.va, A_dev, 64, BK, batch, batch4[1]);

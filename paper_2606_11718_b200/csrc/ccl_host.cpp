@@ -39,15 +39,19 @@ ccl_status make_view(const ccl_mat* m, const char* what, MatView* out) {
         return fail(CCL_ERR_INVALID_ARG, "%s: matrix too large", what);
     MatView v;
     v.rows = m->rows; v.cols = m->cols; v.e = m->elem_bytes;
-    v.w = m->cols; v.h = m->rows; v.stride = 0; v.nstrips = 1; v.split = 0; v.ichunk = 0; v.ichunks = 0;
+    v.w = m->cols; v.h = m->rows; v.wlast = v.w; v.hlast = v.h; v.last_span = 0; v.stride = 0; v.nstrips = 1; v.split = 0; v.ichunk = 0; v.ichunks = 0;
     if (m->layout != CCL_ROWMAJOR && m->part != CCL_PART_NONE) {
-        int64_t packed;
+        // Eq. 1 with w = N / G rounded up: when P does not divide the split dimension the last strip keeps what is left
+        // (at least one column / row, else CCL_ERR_SHAPE)
+        int64_t packed, packed_last;
         if (m->part == CCL_PART_COLS) {
-            if (m->cols % m->P) return fail(CCL_ERR_SHAPE, "%s: cols (%lld) not divisible by P (%d)", what, (long long)m->cols, m->P);
-            v.w = m->cols / m->P; packed = m->rows * v.w; v.split = 2;
+            v.w = (m->cols + m->P - 1) / m->P; v.wlast = m->cols - (int64_t)(m->P - 1) * v.w;
+            if (v.wlast <= 0) return fail(CCL_ERR_SHAPE, "%s: %lld columns cannot be cut into %d strips of %lld (a strip would be empty)", what, (long long)m->cols, m->P, (long long)v.w);
+            packed = m->rows * v.w; packed_last = m->rows * v.wlast; v.split = 2;
         } else {
-            if (m->rows % m->P) return fail(CCL_ERR_SHAPE, "%s: rows (%lld) not divisible by P (%d)", what, (long long)m->rows, m->P);
-            v.h = m->rows / m->P; packed = v.h * m->cols; v.split = 1;
+            v.h = (m->rows + m->P - 1) / m->P; v.hlast = m->rows - (int64_t)(m->P - 1) * v.h;
+            if (v.hlast <= 0) return fail(CCL_ERR_SHAPE, "%s: %lld rows cannot be cut into %d strips of %lld (a strip would be empty)", what, (long long)m->rows, m->P, (long long)v.h);
+            packed = v.h * m->cols; packed_last = v.hlast * m->cols; v.split = 1;
         }
         v.nstrips = m->P;
         if (m->layout == CCL_CCL_INTERLEAVED) {
@@ -55,11 +59,13 @@ ccl_status make_view(const ccl_mat* m, const char* what, MatView* out) {
             v.ichunk = m->strip_align_bytes / m->elem_bytes;
             v.ichunks = (packed + v.ichunk - 1) / v.ichunk;
             v.stride = packed;                 // strip-local extent; strips are not stored one after the other
+            v.last_span = packed_last;
         } else if (m->strip_align_bytes) {
-            int64_t a = m->strip_align_bytes, bytes = packed * m->elem_bytes;
-            v.stride = (bytes + a - 1) / a * a / m->elem_bytes;
+            int64_t a = m->strip_align_bytes;
+            v.stride = (packed * m->elem_bytes + a - 1) / a * a / m->elem_bytes;
+            v.last_span = (packed_last * m->elem_bytes + a - 1) / a * a / m->elem_bytes;
         } else {
-            v.stride = packed;
+            v.stride = packed; v.last_span = packed_last;
         }
     }
     *out = v;
@@ -94,15 +100,11 @@ ccl_status ccl_map_inverse(const ccl_mat* m, int64_t off, int64_t* r, int64_t* c
         int64_t chunk = off / v.ichunk;
         g = chunk % v.nstrips;
         rem = (chunk / v.nstrips) * v.ichunk + off % v.ichunk;
-        if (rem >= v.stride) return fail(CCL_ERR_PADDING, "ccl_map_inverse: offset lies in the padding of strip %lld", (long long)g);
     } else { g = off / v.stride; rem = off % v.stride; }
-    if (v.split == 2) {
-        if (rem >= v.rows * v.w) return fail(CCL_ERR_PADDING, "ccl_map_inverse: offset lies in the padding of strip %lld", (long long)g);
-        *r = rem / v.w; *c = g * v.w + rem % v.w;
-    } else {
-        if (rem >= v.h * v.cols) return fail(CCL_ERR_PADDING, "ccl_map_inverse: offset lies in the padding of strip %lld", (long long)g);
-        *r = g * v.h + rem / v.cols; *c = rem % v.cols;
-    }
+    const int64_t wg = strip_w_of(v, g), hg = strip_h_of(v, g);
+    if (rem >= (v.split == 2 ? v.rows * wg : hg * v.cols)) return fail(CCL_ERR_PADDING, "ccl_map_inverse: offset lies in the padding of strip %lld", (long long)g);
+    if (v.split == 2) { *r = rem / wg; *c = g * v.w + rem % wg; }
+    else { *r = g * v.h + rem / v.cols; *c = rem % v.cols; }
     return CCL_OK;
 }
 

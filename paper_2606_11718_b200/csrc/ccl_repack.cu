@@ -27,6 +27,8 @@ struct CopyPlan {
     int64_t il_chunk, il_P;
     int32_t il_shift, il_dst;                 // log2(il_chunk) or -1; 1 = the destination is the interleaved side
     int64_t batch, src_b, dst_b;              // matrices per launch and the byte strides between them
+    int64_t g0;                               // index of the first strip this launch covers (the narrower last strip of a
+                                              // width that P does not divide is copied by a launch of its own)
 };
 
 __device__ __forceinline__ int64_t interleaved_off(const CopyPlan& p, int64_t g, int64_t b) {
@@ -58,7 +60,7 @@ constexpr int kVecUnroll = 4;
 template <typename V, typename IDX>
 __global__ void __launch_bounds__(kVecThreads) repack_vec_kernel(const char* __restrict__ src, char* __restrict__ dst, CopyPlan p,
                                                                  IDX chunks_per_row, IDX chunks_per_strip) {
-    const int64_t g = blockIdx.y;
+    const int64_t g = blockIdx.y + p.g0;
     const char* s = src + (int64_t)blockIdx.z * p.src_b + g * p.src_g;
     char* d = dst + (int64_t)blockIdx.z * p.dst_b + g * p.dst_g;
     const IDX step = (IDX)gridDim.x * kVecThreads * kVecUnroll;
@@ -541,6 +543,33 @@ static ccl_status repack_impl(const ccl_mat* m, int64_t batch, const void* src_d
 
     const char* src = static_cast<const char*>(src_dev);
     char* dst = static_cast<char*>(dst_dev);
+    if (ragged(v)) {
+        // The split dimension is not a multiple of P: the first P - 1 strips are one strided copy, the narrower (or
+        // shorter) last strip another; padding (aligned strips, chunk tails) is cleared by zeroing the destination first.
+        if (dir == 0 && (m->strip_align_bytes || v.ichunk))
+            CCL_CUDA_TRY(cudaMemset2DAsync(dst, batch > 1 ? (size_t)dst_b : (size_t)(buffer_elems(v) * e), 0, (size_t)(buffer_elems(v) * e), (size_t)batch, st));
+        for (int pass = 0; pass < 2; ++pass) {
+            CopyPlan q = p;
+            q.pad_bytes = 0;
+            if (pass == 0) { q.nstrips = v.nstrips - 1; if (q.nstrips == 0) continue; }
+            else {
+                q.nstrips = 1; q.g0 = v.nstrips - 1;
+                if (v.split == 2) {
+                    q.row_bytes = v.wlast * e;
+                    if (dir == 0) q.dst_r = v.wlast * e; else q.src_r = v.wlast * e;
+                } else q.rows = v.hlast;
+            }
+            const int64_t addr = (int64_t)((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst)) & 15);
+            const int64_t vq = pow2_divisor(q.row_bytes | q.src_g | q.src_r | q.dst_g | q.dst_r | q.il_chunk | q.src_b | q.dst_b | addr, 16);
+            if (vq == 16) s = launch_vec<uint4>(src, dst, q, sms, st);
+            else if (vq == 8) s = launch_vec<uint2>(src, dst, q, sms, st);
+            else if (vq == 4) s = launch_vec<unsigned int>(src, dst, q, sms, st);
+            else if (vq == 2) s = launch_vec<unsigned short>(src, dst, q, sms, st);
+            else s = launch_vec<unsigned char>(src, dst, q, sms, st);
+            if (s) return s;
+        }
+        return CCL_OK;
+    }
     int64_t addr_bits = (int64_t)((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst)) & 15);
     int64_t vec = pow2_divisor(p.row_bytes | p.src_g | p.src_r | p.dst_g | p.dst_r | p.il_chunk | p.src_b | p.dst_b | addr_bits, 16);
 
@@ -598,7 +627,9 @@ extern "C" ccl_status ccl_repack_transpose(const ccl_mat* m, const void* src_dev
     set_padding(v, &p);
     char* dst = static_cast<char*>(dst_dev);
     const bool aligned16 = ((reinterpret_cast<uintptr_t>(src_dev) | reinterpret_cast<uintptr_t>(dst_dev)) & 15) == 0;
-    const bool vec = v.e == 2 && aligned16 && v.rows % 8 == 0 && v.cols % 8 == 0 && v.w % 8 == 0 && v.stride % 8 == 0 && v.ichunk % 8 == 0 &&
+    if (ragged(v) && (m->strip_align_bytes || v.ichunk))      // strips of unequal size: the padding is cleared by zeroing the destination first
+        CCL_CUDA_TRY(cudaMemsetAsync(dst, 0, (size_t)(buffer_elems(v) * v.e), st));
+    const bool vec = !ragged(v) && v.e == 2 && aligned16 && v.rows % 8 == 0 && v.cols % 8 == 0 && v.w % 8 == 0 && v.stride % 8 == 0 && v.ichunk % 8 == 0 &&
                      v.rows < (INT64_C(1) << 31) && v.cols < (INT64_C(1) << 31) && ((v.rows + 63) / 64) * ((v.cols + 63) / 64) < (INT64_C(1) << 31);
     const int64_t T = vec ? kTrTile : 32;
     const int64_t tiles_r = (v.rows + T - 1) / T, tiles_c = (v.cols + T - 1) / T, ntiles = tiles_r * tiles_c;
@@ -621,5 +652,5 @@ extern "C" ccl_status ccl_repack_transpose(const ccl_mat* m, const void* src_dev
     else return fail(CCL_ERR_UNSUPPORTED, "ccl_repack_transpose: elem_bytes must be 1, 2 or 4");
     count_launch();
     CCL_CUDA_TRY(cudaGetLastError());
-    return zero_padding(dst, p, st);
+    return ragged(v) ? CCL_OK : zero_padding(dst, p, st);
 }

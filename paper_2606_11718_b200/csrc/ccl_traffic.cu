@@ -30,6 +30,7 @@ struct TrafficParams {
     int32_t assign;
     int32_t m_strip_tiled, n_strip_tiled;
     int64_t tiles_m, tiles_n, tps_m, tps_n, wM, wN;
+    int32_t pm, pn;               // blocks of the output partition along M and N (pm * pn = P, or 1 x 1 for an explicit table)
     int64_t ntiles;
     int64_t pages[3];
     int64_t bytes_total[3];
@@ -53,16 +54,16 @@ struct TileInfo { int64_t m0, m1, n0, n1; int32_t q; };
 __device__ __forceinline__ TileInfo decode_tile(const TrafficParams& p, int64_t t) {
     TileInfo ti;
     int64_t tm = t / p.tiles_n, tn = t - tm * p.tiles_n;
-    if (p.m_strip_tiled) {
-        int64_t g = tm / p.tps_m, j = tm - g * p.tps_m;
-        ti.m0 = g * p.wM + j * p.BM; ti.m1 = min(ti.m0 + p.BM, (g + 1) * p.wM);
+    if (p.m_strip_tiled) {                        // strips of wM rows (the last one may be shorter), each tiled on its own
+        int64_t g = min(tm / p.tps_m, (int64_t)p.pm - 1), j = tm - g * p.tps_m;
+        ti.m0 = g * p.wM + j * p.BM; ti.m1 = min(ti.m0 + p.BM, min(p.M, (g + 1) * p.wM));
     } else { ti.m0 = tm * p.BM; ti.m1 = min(p.M, ti.m0 + p.BM); }
     if (p.n_strip_tiled) {
-        int64_t g = tn / p.tps_n, j = tn - g * p.tps_n;
-        ti.n0 = g * p.wN + j * p.BN; ti.n1 = min(ti.n0 + p.BN, (g + 1) * p.wN);
+        int64_t g = min(tn / p.tps_n, (int64_t)p.pn - 1), j = tn - g * p.tps_n;
+        ti.n0 = g * p.wN + j * p.BN; ti.n1 = min(ti.n0 + p.BN, min(p.N, (g + 1) * p.wN));
     } else { ti.n0 = tn * p.BN; ti.n1 = min(p.N, ti.n0 + p.BN); }
-    if (p.assign == CCL_ASSIGN_N_STRIPS) ti.q = (int32_t)(ti.n0 / p.wN);
-    else if (p.assign == CCL_ASSIGN_M_STRIPS) ti.q = (int32_t)(ti.m0 / p.wM);
+    // the block of the output partition that holds the tile's first element (N strips: 1 x P, M strips: P x 1)
+    if (p.assign != CCL_ASSIGN_EXPLICIT) ti.q = (int32_t)((ti.m0 / p.wM) * p.pn + ti.n0 / p.wN);
     else { int32_t q = p.q[t]; ti.q = q < 0 ? 0 : (q >= p.P ? p.P - 1 : q); }
     return ti;
 }
@@ -83,11 +84,12 @@ __device__ __forceinline__ void walk_row(const TrafficParams& p, const MatView& 
         if (v.split == 2) {
             int64_t g = c / v.w;
             cend = min(c1, (g + 1) * v.w);
+            const int64_t wg = strip_w_of(v, g);   // the last strip of a ragged width has its own row pitch
             if (v.ichunk) {                        // page-interleaved CCL: contiguity also ends at every chunk
-                const int64_t o = r * v.w + (c - g * v.w);
+                const int64_t o = r * wg + (c - g * v.w);
                 cend = min(cend, c + (o / v.ichunk + 1) * v.ichunk - o);
                 off = interleave(v, g, o);
-            } else off = g * v.stride + r * v.w + (c - g * v.w);
+            } else off = g * v.stride + r * wg + (c - g * v.w);
         } else if (v.ichunk) {                     // split along rows, page-interleaved
             const int64_t g = r / v.h, o = (r - g * v.h) * v.cols + c;
             cend = min(c1, c + (o / v.ichunk + 1) * v.ichunk - o);
@@ -351,8 +353,8 @@ __global__ void __launch_bounds__(32 * kLruWarps) traffic_lru_kernel(TrafficPara
         if (k_is_rows) { r0 = k0; r1 = k1; } else { c0 = k0; c1 = k1; }
         if (v.split == 2) {                                           // strips of columns: one piece per strip touched
             for (int64_t g = c0 / v.w; g * v.w < c1; ++g) {
-                const int64_t ca = max(c0, g * v.w), cb = min(c1, (g + 1) * v.w);
-                piece(X, (g * v.stride + r0 * v.w + (ca - g * v.w)) * v.e, r1 - r0, v.w * v.e, (cb - ca) * v.e);
+                const int64_t ca = max(c0, g * v.w), cb = min(c1, (g + 1) * v.w), wg = strip_w_of(v, g);
+                piece(X, (g * v.stride + r0 * wg + (ca - g * v.w)) * v.e, r1 - r0, wg * v.e, (cb - ca) * v.e);
             }
         } else if (v.split == 1) {                                    // strips of rows
             for (int64_t g = r0 / v.h; g * v.h < r1; ++g) {
@@ -399,7 +401,7 @@ static ccl_status fill_params(const ccl_traffic_desc* d, TrafficParams* p) {
     if (d->M <= 0 || d->N <= 0 || d->K <= 0 || d->BM <= 0 || d->BN <= 0) return fail(CCL_ERR_INVALID_ARG, "ccl_traffic: sizes must be positive");
     if (d->P < 1 || d->P > 255) return fail(CCL_ERR_INVALID_ARG, "ccl_traffic: P must be in [1,255]");
     if (d->page_bytes <= 0) return fail(CCL_ERR_INVALID_ARG, "ccl_traffic: page_bytes must be positive");
-    if (d->assign < 0 || d->assign > 2) return fail(CCL_ERR_INVALID_ARG, "ccl_traffic: unknown assign");
+    if (d->assign < 0 || d->assign > 3) return fail(CCL_ERR_INVALID_ARG, "ccl_traffic: unknown assign");
     const ccl_mat* ms[3] = {&d->A, &d->B, &d->C};
     const char* names[3] = {"ccl_traffic: A", "ccl_traffic: B", "ccl_traffic: C"};
     for (int X = 0; X < 3; ++X) {
@@ -416,21 +418,30 @@ static ccl_status fill_params(const ccl_traffic_desc* d, TrafficParams* p) {
     int64_t br = d->b_trans ? d->N : d->K, bc = d->b_trans ? d->K : d->N;
     if (d->A.rows != ar || d->A.cols != ac || d->B.rows != br || d->B.cols != bc || d->C.rows != d->M || d->C.cols != d->N)
         return fail(CCL_ERR_SHAPE, "ccl_traffic: operand shapes do not match M, N, K and the transpose flags");
-    if (d->assign == CCL_ASSIGN_N_STRIPS && d->N % d->P) return fail(CCL_ERR_SHAPE, "ccl_traffic: N not divisible by P");
-    if (d->assign == CCL_ASSIGN_M_STRIPS && d->M % d->P) return fail(CCL_ERR_SHAPE, "ccl_traffic: M not divisible by P");
+    // output partition: pm x pn blocks of ceil(M / pm) x ceil(N / pn) (the last ones hold what is left)
+    int64_t pm = 1, pn = 1;
+    if (d->assign == CCL_ASSIGN_N_STRIPS) pn = d->P;
+    else if (d->assign == CCL_ASSIGN_M_STRIPS) pm = d->P;
+    else if (d->assign == CCL_ASSIGN_2D) {
+        if (d->part_m < 1 || d->P % d->part_m) return fail(CCL_ERR_INVALID_ARG, "ccl_traffic: part_m (%d) must divide P (%d)", d->part_m, d->P);
+        pm = d->part_m; pn = d->P / d->part_m;
+    }
     p->M = d->M; p->N = d->N; p->K = d->K; p->BM = d->BM; p->BN = d->BN;
+    p->wM = (d->M + pm - 1) / pm; p->wN = (d->N + pn - 1) / pn;
+    if ((pn - 1) * p->wN >= d->N) return fail(CCL_ERR_SHAPE, "ccl_traffic: N (%lld) cannot be cut into %lld strips (one would be empty)", (long long)d->N, (long long)pn);
+    if ((pm - 1) * p->wM >= d->M) return fail(CCL_ERR_SHAPE, "ccl_traffic: M (%lld) cannot be cut into %lld strips (one would be empty)", (long long)d->M, (long long)pm);
+    p->pm = (int32_t)pm; p->pn = (int32_t)pn;
     p->a_trans = d->a_trans != 0; p->b_trans = d->b_trans != 0; p->P = d->P; p->S = d->page_bytes;
     p->s_shift = -1;
     if ((d->page_bytes & (d->page_bytes - 1)) == 0) { int sh = 0; while ((INT64_C(1) << sh) < d->page_bytes) ++sh; p->s_shift = sh; }
     p->assign = d->assign;
-    p->m_strip_tiled = d->assign == CCL_ASSIGN_M_STRIPS && d->strip_tiling;
-    p->n_strip_tiled = d->assign == CCL_ASSIGN_N_STRIPS && d->strip_tiling;
-    p->wM = d->assign == CCL_ASSIGN_M_STRIPS ? d->M / d->P : d->M;
-    p->wN = d->assign == CCL_ASSIGN_N_STRIPS ? d->N / d->P : d->N;
+    p->m_strip_tiled = pm > 1 && d->strip_tiling;
+    p->n_strip_tiled = pn > 1 && d->strip_tiling;
     p->tps_m = p->m_strip_tiled ? (p->wM + d->BM - 1) / d->BM : 0;
     p->tps_n = p->n_strip_tiled ? (p->wN + d->BN - 1) / d->BN : 0;
-    p->tiles_m = p->m_strip_tiled ? p->tps_m * d->P : (d->M + d->BM - 1) / d->BM;
-    p->tiles_n = p->n_strip_tiled ? p->tps_n * d->P : (d->N + d->BN - 1) / d->BN;
+    const int64_t m_last = d->M - (pm - 1) * p->wM, n_last = d->N - (pn - 1) * p->wN;
+    p->tiles_m = p->m_strip_tiled ? p->tps_m * (pm - 1) + (m_last + d->BM - 1) / d->BM : (d->M + d->BM - 1) / d->BM;
+    p->tiles_n = p->n_strip_tiled ? p->tps_n * (pn - 1) + (n_last + d->BN - 1) / d->BN : (d->N + d->BN - 1) / d->BN;
     p->ntiles = p->tiles_m * p->tiles_n;
     return CCL_OK;
 }

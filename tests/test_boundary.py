@@ -53,6 +53,11 @@ MAP_CASES = [
     dict(rows=7, cols=24, P=3, part=2, layout=2, align=64),
     dict(rows=12, cols=40, P=4, part=1, layout=2, align=48, e=4),
     dict(rows=33, cols=96, P=4, part=2, layout=2, align=256, e=1),
+    dict(rows=3, cols=7, P=3, part=2, layout=1),                           # widths P does not divide: the hand example
+    dict(rows=9, cols=1537, P=4, part=2, layout=1, align=256),
+    dict(rows=13, cols=40, P=4, part=1, layout=1, align=64),
+    dict(rows=5, cols=202, P=3, part=2, layout=2, align=128),
+    dict(rows=11, cols=30, P=4, part=1, layout=2, align=48, e=4),
 ]
 
 
@@ -94,8 +99,8 @@ def expect(status, fn, *a, **k):
 
 
 def test_map_error_codes():
-    expect(ccl.ERR_SHAPE, ccl.ccl_map_offset, ccl.Mat(4, 10, 2, 4, 2, 1), 0, 0)
-    expect(ccl.ERR_SHAPE, ccl.ccl_buffer_bytes, ccl.Mat(5, 8, 2, 2, 1, 1))
+    expect(ccl.ERR_SHAPE, ccl.ccl_map_offset, ccl.Mat(4, 9, 2, 4, 2, 1), 0, 0)       # 4 strips of ceil(9/4) = 3: the last would be empty
+    expect(ccl.ERR_SHAPE, ccl.ccl_buffer_bytes, ccl.Mat(4, 8, 2, 3, 1, 1))
     expect(ccl.ERR_INVALID_ARG, ccl.ccl_map_offset, ccl.Mat(4, 8, 2, 2, 2, 1), 4, 0)
     expect(ccl.ERR_INVALID_ARG, ccl.ccl_map_offset, ccl.Mat(4, 8, 3, 2, 2, 1), 0, 0)
     expect(ccl.ERR_INVALID_ARG, ccl.ccl_map_offset, ccl.Mat(4, 8, 2, 0, 2, 1), 0, 0)
@@ -112,7 +117,7 @@ def test_repack_rejects_bad_input_before_any_launch():
     assert l.ccl_repack(C.byref(m), C.c_void_p(256), C.c_void_p(512), 2, None) == ccl.ERR_INVALID_ARG
     assert l.ccl_repack(C.byref(m), C.c_void_p(256), C.c_void_p(256), 0, None) == ccl.ERR_INVALID_ARG
     assert l.ccl_repack(C.byref(m), C.c_void_p(257), C.c_void_p(512), 0, None) == ccl.ERR_ALIGN
-    bad = ccl.Mat(4, 9, 2, 2, 2, 1)
+    bad = ccl.Mat(4, 9, 2, 4, 2, 1)
     assert l.ccl_repack(C.byref(bad), C.c_void_p(256), C.c_void_p(512), 0, None) == ccl.ERR_SHAPE
     # a batch: count in range, outputs that do not overlap, strides in whole elements
     rb = lambda batch, ss, ds, d=0: l.ccl_repack_batched(C.byref(m), batch, C.c_void_p(256), ss, C.c_void_p(4096), ds, d, None)
@@ -179,6 +184,13 @@ def test_gemm_rejects_bad_input_before_any_launch():
     assert gemm_rc(d) == ccl.ERR_UNSUPPORTED
     d = gemm_desc(128, 256, 64, 3, ("row", "row", "row"))
     assert gemm_rc(d) == ccl.ERR_SHAPE                                                               # N % P with a grouped raster
+    assert gemm_rc(gemm_desc(128, 264, 64, 4, ("row", "ccl", "row"), grouped=0)) == ccl.ERR_UNSUPPORTED   # strips of unequal width (264 = 3 * 72 + 48)
+    d = gemm_desc(256, 512, 64, 4, ("row", "row", "row"), out_part=3)
+    d.part_m = 3
+    assert gemm_rc(d) == ccl.ERR_INVALID_ARG                                                         # part_m must divide P
+    d.part_m = 2
+    d.M = 255; d.A.rows = 255; d.C.rows = 255
+    assert gemm_rc(d) == ccl.ERR_SHAPE                                                               # M not divisible by part_m
     # page-interleaved operands: chunks must line up with the strip rows (w = 96 elements = 192 bytes here)
     assert gemm_rc(gemm_desc(128, 192, 64, 2, ("row", "ileave", "ccl"), align=256)) == ccl.ERR_UNSUPPORTED    # neither divides
     assert gemm_rc(gemm_desc(128, 192, 64, 2, ("row", "ileave", "ccl"), align=576)) == ccl.ERR_UNSUPPORTED    # 3 rows per chunk
@@ -202,13 +214,21 @@ def test_traffic_sizes_and_rejections():
     do, dl = traffic_pair(128, 256, 64, 8, 512, assign=1, BM=16, BN=64, lay=("ccl", "row", "ccl"), align=1024)
     assert ccl.ccl_traffic_sizes(dl) == tuple(orc.traffic_sizes(do))
     l = ccl.lib()
-    _, bad = traffic_pair(8, 9, 4, 2, 16)
+    _, bad = traffic_pair(8, 9, 4, 4, 16)
     assert l.ccl_traffic(C.byref(bad), None, C.c_void_p(256), None, None, C.c_void_p(512), None) == ccl.ERR_SHAPE
+    do, dl = traffic_pair(8, 9, 4, 2, 16)                                                            # strips of 5 and 4 columns
+    assert ccl.ccl_traffic_sizes(dl) == tuple(orc.traffic_sizes(do))
+    do, dl = traffic_pair(131, 203, 24, 6, 128, assign=3, part_m=2, BM=32, BN=32)                    # 2 x 3 blocks, ragged both ways
+    assert ccl.ccl_traffic_sizes(dl) == tuple(orc.traffic_sizes(do))
+    _, d = traffic_pair(128, 256, 24, 6, 128, assign=3, part_m=4)
+    assert l.ccl_traffic(C.byref(d), None, C.c_void_p(256), None, None, C.c_void_p(512), None) == ccl.ERR_INVALID_ARG
     _, d = traffic_pair(8, 8, 4, 2, 16)
     assert l.ccl_traffic(C.byref(d), None, None, None, None, C.c_void_p(512), None) == ccl.ERR_INVALID_ARG
     _, d = traffic_pair(8, 8, 4, 2, 16, place=(2, 2, 2))
     assert l.ccl_traffic(C.byref(d), None, C.c_void_p(256), None, None, C.c_void_p(512), None) == ccl.ERR_WORKSPACE
     _, d = traffic_pair(8, 8, 4, 2, 16, assign=2)
+    assert l.ccl_traffic(C.byref(d), None, C.c_void_p(256), None, None, C.c_void_p(512), None) == ccl.ERR_INVALID_ARG
+    _, d = traffic_pair(8, 8, 4, 2, 16, assign=4)
     assert l.ccl_traffic(C.byref(d), None, C.c_void_p(256), None, None, C.c_void_p(512), None) == ccl.ERR_INVALID_ARG
     _, d = traffic_pair(8, 8, 4, 2, 3)
     assert l.ccl_traffic(C.byref(d), None, C.c_void_p(256), None, None, C.c_void_p(512), None) == ccl.ERR_INVALID_ARG

@@ -87,6 +87,28 @@ SMALL = [
 ]
 
 
+PART_2D = [
+    # M, N, K, P, part_m, layouts(A,B,C), strips of (A, B, C), splits of (A, B, C), a_trans, b_trans
+    (512, 1024, 256, 4, 2, ("row", "row", "row"), (1, 1, 1), (0, 0, 0), 0, 0),       # 2 x 2 blocks of a row-major C
+    (512, 1024, 256, 4, 2, ("ccl", "ccl", "ccl"), (2, 2, 2), (1, 2, 1), 0, 0),       # A, C in 2 row strips, B in 2 column strips
+    (768, 1536, 200, 8, 2, ("ccl", "ccl", "ccl"), (2, 4, 4), (1, 2, 2), 0, 0),       # 2 x 4 blocks, C split along N into 4
+    (768, 1536, 328, 8, 4, ("ccl", "ccl", "row"), (4, 2, 1), (2, 1, 0), 1, 1),       # A [K x M] split along cols, B [N x K] along rows
+    (1536, 768, 192, 6, 3, ("row", "ccl", "ccl"), (1, 2, 3), (0, 2, 1), 0, 0),       # 3 x 2 blocks
+    (2048, 4096, 512, 4, 2, ("row", "ccl", "ccl"), (1, 2, 2), (0, 2, 2), 0, 0),      # several tiles per group
+]
+
+
+@pytest.mark.parametrize("M,N,K,P,pm,lay,mp,parts,at,bt", PART_2D)
+def test_gemm_2d_output_partition(M, N, K, P, pm, lay, mp, parts, at, bt):
+    """Sec. 4.1 (output-partition choices): CTA group (qm, qn) computes block (qm, qn) of C; the result is the plain product,
+    bit for bit the one of the plain raster."""
+    A, B = synth.gemm_operands(M, N, K, at, bt, seed=0, tag="2d")
+    d = gemm_desc(M, N, K, P, lay, at, bt, out_part=3, grouped=1, parts=parts, part_m=pm, mat_P=mp)
+    got, _ = check(d, A, B)
+    d0 = gemm_desc(M, N, K, P, lay, at, bt, out_part=3, grouped=0, parts=parts, part_m=pm, mat_P=mp)
+    np.testing.assert_array_equal(got, run_gemm(d0, A, B))
+
+
 @pytest.fixture(params=["auto", "1", "2"])
 def cta_mode(request):
     """Forces the 1-CTA or the 2-CTA (cta_group::2 pair) kernel, or leaves the library's own choice."""

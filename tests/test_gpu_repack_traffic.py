@@ -86,6 +86,15 @@ REPACK_CASES = [
     dict(rows=1001, cols=1024, P=4, part=2, layout=2, align=4096),     # a chunk holds 8 strip rows, the last chunk 1
     dict(rows=1001, cols=1024, P=4, part=2, layout=2, align=16384, e=4),   # ... 16 rows of 4-byte elements
     dict(rows=2100, cols=2048, P=4, part=1, layout=2, align=8192),     # strips of rows: a chunk holds two rows
+    dict(rows=3, cols=7, P=3, part=2, layout=1),                       # widths P does not divide: the hand example
+    dict(rows=64, cols=1537, P=4, part=2, layout=1),                   # w = 385, last strip 382
+    dict(rows=130, cols=1000, P=7, part=2, layout=1, align=4096),      # w = 143, last 142; aligned strips
+    dict(rows=513, cols=2050, P=4, part=2, layout=1, e=4, align=256),
+    dict(rows=1001, cols=768, P=3, part=1, layout=1),                  # strips of 334 rows, the last 333
+    dict(rows=1001, cols=768, P=8, part=1, layout=1, align=65536),
+    dict(rows=77, cols=202, P=3, part=2, layout=2, align=128),         # page-interleaved, unequal strips
+    dict(rows=301, cols=1030, P=4, part=2, layout=2, align=4096, e=1),
+    dict(rows=1001, cols=96, P=6, part=1, layout=2, align=512),
 ]
 
 
@@ -266,6 +275,12 @@ SHAPES = [
     dict(M=130, N=384, K=96, P=4, S=256, strip_tiling=0),
     dict(M=1, N=512, K=256, P=4, S=4096),
     dict(M=16, N=512, K=256, P=1, S=4096),
+    dict(M=96, N=200, K=40, P=3, S=256, BM=32, BN=32),                 # strips of 67, 67, 66 columns
+    dict(M=97, N=385, K=72, P=4, S=128, BM=32, BN=64, assign=1),       # strips of 25, 25, 25, 22 rows
+    dict(M=4, N=8, K=4, P=4, S=16, BM=2, BN=4, assign=3, part_m=2),    # the hand-enumerated 2 x 2 partition
+    dict(M=128, N=256, K=64, P=4, S=256, BM=32, BN=32, assign=3, part_m=2),
+    dict(M=131, N=203, K=24, P=6, S=128, BM=32, BN=32, assign=3, part_m=2),     # 2 x 3 blocks, ragged both ways
+    dict(M=130, N=384, K=96, P=8, S=512, BM=64, BN=64, assign=3, part_m=4, strip_tiling=0),
 ]
 LAYS = [("row", "row", "row"), ("row", "ccl", "ccl"), ("ccl", "ccl", "ccl"), ("row", "ileave", "ileave"), ("ileave", "ileave", "ileave")]
 PLACES = [(0, 0, 0), (1, 1, 1), (2, 2, 2), (0, 1, 2)]
@@ -289,6 +304,15 @@ def test_traffic_interleaved_ccl_is_local_under_literal_round_robin(P):
         r = run_traffic(*traffic_pair(lay=("row", "ileave", "ileave"), place=(0, 0, 0), align=4096, **base), level="runs")
         assert r["totals"][1, 1] == 0 and r["totals"][2, 1] == 0
         r = run_traffic(*traffic_pair(lay=("row", "ileave", "ileave"), place=(0, 0, 0), align=65536, **base), level="runs")
+
+
+def test_traffic_2d_partition_with_matching_layouts():
+    """A 2 x 2 output partition with A and C in CCL split along rows into 2 strips and B along columns into 2 strips
+    (each operand's own P): the counter takes any mix of operand strips and output blocks."""
+    for place in PLACES:
+        do, dl = traffic_pair(256, 512, 128, 4, 1024, lay=("ccl", "ccl", "ccl"), place=place, assign=3, part_m=2, BM=64, BN=64,
+                              parts=(1, 2, 1), mat_P=(2, 2, 2), align=1024)
+        run_traffic(do, dl, "elem")
 
 
 def test_traffic_explicit_assignment():

@@ -56,11 +56,11 @@ CACHES = [(128, 128, 1), (8 * 1024, 128, 4), (96 * 1024, 128, 16), (48 * 128 * 3
 
 
 @pytest.mark.parametrize("M,N,K,P,S,lay,place,BM,BN,at,bt", SHAPES)
-@pytest.mark.parametrize("assign", [0, 1])
+@pytest.mark.parametrize("assign", [0, 1, 3])
 def test_lru_bit_exact(M, N, K, P, S, lay, place, BM, BN, at, bt, assign):
-    if assign == 1 and M % P:
-        pytest.skip("M not divisible by P")
-    do, dl = traffic_pair(M, N, K, P, S, lay, place, a_trans=at, b_trans=bt, assign=assign, BM=BM, BN=BN, align=S)
+    if assign == 3 and P < 4:
+        pytest.skip("a 2-D partition needs at least 2 x 2 chiplets")
+    do, dl = traffic_pair(M, N, K, P, S, lay, place, a_trans=at, b_trans=bt, assign=assign, BM=BM, BN=BN, align=S, part_m=2 if assign == 3 else 0)
     for cap, line, ways in CACHES:
         if S % line:
             continue
