@@ -103,7 +103,7 @@ struct GemmParams {
     int32_t panel;                  // m-tiles per raster panel
     // raster constants the host derives from the grid it launches (see Scheduler)
     int32_t sch_units, sch_gm, sch_gn, sch_upg, sch_floaters, sch_rounds, sch_per_group, sch_pool_per_group;
-    FastDiv fd_upg, fd_groups, fd_splits, fd_per_panel, fd_panel, fd_tps_m, fd_tps_n;
+    FastDiv fd_upg, fd_groups, fd_splits, fd_per_panel, fd_panel, fd_tps_m, fd_tps_n, fd_num_kb;
     // batch of independent problems of one shape (ccl_gemm_batched): the tile walk of a group runs through its
     // tiles of problem 0, then of problem 1, ...; problem e is coordinate e of every tensor map's last dimension
     int32_t batch;
@@ -139,6 +139,13 @@ struct GemmParams {
     uint32_t stage_bytes, a_bytes;  // bytes per stage per CTA, bytes of its A part
     int32_t splits, kb_per_split;   // split-K: each tile is computed by `splits` units over disjoint k-block ranges
     float* ws;                      // split-K partial sums, [splits][M][N] fp32 (row-major, logical coordinates)
+    // balanced split: the k blocks of the first bal_tiles tiles of a group, laid end to end, are cut into equal shares, one
+    // for each of the group's first bal_units units; bal_q / bal_r = quotient and remainder of that division
+    int32_t bal, bal_q, bal_r, bal_units, bal_tiles;
+    // "partial sums written" flags, one per (CTA, epilogue warp), behind the partial sums in the workspace; zeroed by a
+    // memset node in front of the launch (so a replayed CUDA graph clears them as well) and set to bal_mark by the kernel
+    unsigned long long bal_mark;
+    unsigned long long* bal_flags;
 };
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
@@ -290,6 +297,12 @@ __device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
     return v;
 }
 
+__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+
 struct KRange { int k0, nkb, rem; };
 __device__ __forceinline__ KRange k_range(const int32_t* k_offs, int e, int Ktot) {
     const int o0 = __ldg(k_offs + e), o1 = __ldg(k_offs + e + 1);
@@ -300,7 +313,11 @@ __device__ __forceinline__ KRange k_range(const int32_t* k_offs, int e, int Ktot
     return r;
 }
 
-struct TileCoord { int m0, m1, n0, n1, split, e; bool skip; };   // e: problem of the batch; skip: an empty tile of a ragged batch
+// e: problem of the batch; skip: an empty tile of a ragged batch.  Balanced split: the unit computes k blocks [kb0, kb1) of
+// the tile; part = 0: all of them (a plain tile), 1: a share -- the tile is split among `nshare` consecutive units, of
+// which this one is number `mine` (0 holds k = 0); every sharer writes its partial sums to its slot of the workspace and
+// then reduces and stores every nshare-th 64-column piece of the tile.
+struct TileCoord { int m0, m1, n0, n1, split, e; bool skip; int kb0, kb1, part, nshare, mine, round; };   // round: of whole tiles (-1: a share)
 
 // Tiles of this CTA (pair).  The schedulable units (CTAs, or CTA pairs) serve `groups` strip ranges
 // (chiplet-grouped raster): group g owns the tiles of strip range g and walks them in panels of
@@ -334,28 +351,48 @@ struct Scheduler {
         const int o0 = __ldg(p.m_offs + lo), o1 = __ldg(p.m_offs + lo + 1);
         int sn, jn;
         p.fd_tps_n.divmod(tn, sn, jn);
-        t.e = lo; t.split = 0; t.skip = false;
+        t.e = lo; t.split = 0; t.skip = false; t.part = 0; t.round = it;
         t.m0 = o0 + (mt - rag[lo]) * bm; t.m1 = min(t.m0 + bm, o1);
         t.n0 = sn * p.Wn + jn * bn; t.n1 = min(t.n0 + bn, (sn + 1) * p.Wn);
         return true;
     }
-    template <int RAG, bool FULL>
-    __device__ bool get(int it, TileCoord& t) const {
-        if (RAG == 1 && rag) return get_ragged(it, t);
-        int g, i;
-        if (it < rounds && my_g >= 0) { g = my_g; i = idx + it * upg; }
-        else {
-            const int q = it < rounds ? idx + it * floaters : floaters * rounds + unit + (it - rounds) * units;
-            int j = q;
-            g = 0;
-            if (p.groups > 1) p.fd_groups.divmod(q, j, g);
-            if (j >= pool_per_group) return false;
-            i = rounds * upg + j;
+    // Balanced split.  A group's tiles that do not fill a whole round of its units -- the first bal_tiles tiles of its walk --
+    // are laid end to end along K and cut into equal shares of k blocks, one per unit (the first bal_units units; share of
+    // unit u = [lo(u), lo(u + 1)), lo(u) = u * q + min(u, r)): every unit starts with its share, then walks whole tiles
+    // round by round like everybody else.  A tile of the first kind is thus split among consecutive units; each of them
+    // hands its partial sums to the others through the workspace and reduces its part of the tile's columns (epilogue
+    // warps only: the tensor cores are on the unit's next tile by then).
+    __device__ int bal_lo(int u) const { u = min(u, p.bal_units); return u * p.bal_q + min(u, p.bal_r); }
+    template <bool FULL>
+    __device__ bool get_balanced(int it, TileCoord& t) const {
+        if (my_g < 0) return false;
+        const int nkb = p.num_kb, lo = bal_lo(idx), hi = bal_lo(idx + 1);
+        const int first = p.fd_num_kb.div(lo), shares = hi > lo ? p.fd_num_kb.div(hi - 1) - first + 1 : 0;
+        t.split = 0; t.e = 0; t.skip = false; t.nshare = 1; t.mine = 0;
+        if (it < shares) {
+            const int tile = first + it, k0 = tile * nkb;
+            t.kb0 = max(lo, k0) - k0; t.kb1 = min(hi, k0 + nkb) - k0;
+            t.part = (t.kb0 > 0 || t.kb1 < nkb) ? 1 : 0;
+            t.round = -1;
+            if (t.part) {                                  // the units whose shares meet this tile: u0 holds k0, the last one k0 + nkb - 1
+                int u0 = idx;
+                while (bal_lo(u0) > k0) --u0;
+                int u1 = idx;
+                while (bal_lo(u1 + 1) < k0 + nkb) ++u1;
+                t.mine = idx - u0; t.nshare = u1 - u0 + 1;
+            }
+            coords<FULL>(my_g, tile, t);
+            return true;
         }
-        t.split = 0;
-        if (p.splits > 1) { int ii; p.fd_splits.divmod(i, ii, t.split); i = ii; }   // the splits of one tile are neighbours in the walk
-        t.e = 0;
-        if (FULL && p.batch > 1) { int ii; p.fd_tiles_per_problem.divmod(i, t.e, ii); i = ii; }
+        const int tile = p.bal_tiles + idx + (it - shares) * upg;
+        if (tile >= p.sch_per_group) return false;
+        t.kb0 = 0; t.kb1 = nkb; t.part = 0; t.round = it - shares;
+        coords<FULL>(my_g, tile, t);
+        return true;
+    }
+    // tile i of group g's walk -> its rows and columns
+    template <bool FULL>
+    __device__ void coords(int g, int i, TileCoord& t) const {
         int pn, rem;
         p.fd_per_panel.divmod(i, pn, rem);
         const bool tail = gm - pn * p.panel < p.panel;   // the last panel may be lower
@@ -370,6 +407,27 @@ struct Scheduler {
         p.fd_tps_n.divmod(tn, sn, jn);
         t.m0 = sm * p.Wm + jm * bm; t.m1 = min(t.m0 + bm, (sm + 1) * p.Wm);
         t.n0 = sn * p.Wn + jn * bn; t.n1 = min(t.n0 + bn, (sn + 1) * p.Wn);
+    }
+    template <int RAG, bool FULL>
+    __device__ bool get(int it, TileCoord& t) const {
+        if (RAG == 1 && rag) return get_ragged(it, t);
+        if (RAG == 0 && p.bal) return get_balanced<FULL>(it, t);
+        t.part = 0; t.round = it;
+        int g, i;
+        if (it < rounds && my_g >= 0) { g = my_g; i = idx + it * upg; }
+        else {
+            const int q = it < rounds ? idx + it * floaters : floaters * rounds + unit + (it - rounds) * units;
+            int j = q;
+            g = 0;
+            if (p.groups > 1) p.fd_groups.divmod(q, j, g);
+            if (j >= pool_per_group) return false;
+            i = rounds * upg + j;
+        }
+        t.split = 0;
+        if (p.splits > 1) { int ii; p.fd_splits.divmod(i, ii, t.split); i = ii; }   // the splits of one tile are neighbours in the walk
+        t.e = 0;
+        if (FULL && p.batch > 1) { int ii; p.fd_tiles_per_problem.divmod(i, t.e, ii); i = ii; }
+        coords<FULL>(g, i, t);
         t.skip = false;
         if (RAG == 1 && p.m_offs) {                      // rows of this problem inside the concatenated A and C
             const int o0 = __ldg(p.m_offs + t.e), o1 = __ldg(p.m_offs + t.e + 1);
@@ -501,10 +559,10 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         const bool post_tx = lane == 0 && leader;
         for (int it = 0; ok && sched.template get<RAG, FULL>(it, t); ++it) {
             if (t.skip) continue;
-            if (p.wave_ctr && it >= 1 && it < p.sch_rounds && it % p.wave_period == 0) {   // wait (bounded) until every CTA has issued its previous tiles
+            if (p.wave_ctr && t.round >= 1 && t.round < p.sch_rounds && t.round % p.wave_period == 0) {   // wait (bounded) until every CTA has issued its previous tiles
                 if (lane == 0) {
                     atomicAdd(p.wave_ctr, 1u);
-                    const unsigned int target = gridDim.x * (unsigned int)(it / p.wave_period);
+                    const unsigned int target = gridDim.x * (unsigned int)(t.round / p.wave_period);
                     const uint64_t t0 = global_timer_ns();
                     while (ld_acquire_u32(p.wave_ctr) < target && global_timer_ns() - t0 < (uint64_t)p.wave_wait_ns) { }
                 }
@@ -516,6 +574,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             int x, y, z, u;
             if (mn) to_coords<FULL>(om, 0, base, x, y, z, u); else to_coords<FULL>(om, base, 0, x, y, z, u);
             int kb0 = t.split * kbps, kb1 = min(num_kb, kb0 + kbps), kbase = 0;
+            if (RAG == 0 && p.bal) { kb0 = t.kb0; kb1 = t.kb1; }
             if (RAG == 2) { const KRange kr = k_range(p.k_offs, t.e, p.K); kb0 = 0; kb1 = kr.nkb; kbase = kr.k0; }
             for (int kb = kb0; kb < kb1; ++kb) {
                 ok = mbar_wait_bounded(&empty[stage], phase ^ 1);
@@ -553,6 +612,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 const uint32_t acc_phase = NSUB == 1 ? ((uint32_t)(done >> 1) & 1) : ((uint32_t)done & 1);
                 ++done;
                 int kb0 = t.split * kbps, kb1 = min(num_kb, kb0 + kbps), tail = BK;
+                if (RAG == 0 && p.bal) { kb0 = t.kb0; kb1 = t.kb1; }
                 if (RAG == 2) { const KRange kr = k_range(p.k_offs, t.e, p.K); kb0 = 0; kb1 = kr.nkb; tail = kr.rem; }
                 for (int kb = kb0; ok && kb < kb1; ++kb) {
                     // (the copies' completion on the barrier orders the operand bytes before the MMAs that read them;
@@ -612,25 +672,29 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         bool alive = true;
         uint32_t epi_count = 0;                          // TMA-stored pieces so far (selects the staging buffer)
         int done = 0;                                    // tiles drained so far
+        TileCoord pend[2];                               // balanced split: shares written but not yet reduced
+        int npend = 0;
         for (int it = 0; alive && sched.template get<RAG, FULL>(it, t); ++it) {
           if (t.skip) continue;
           const int tile_no = done++;
-          const int m = t.m0 + (int)rank * BM + quad * 32 + lane;
+          int m = t.m0 + (int)rank * BM + quad * 32 + lane;
 #pragma unroll 1                                         // one copy of the (large) drain code: a short GEMM pays for every instruction-cache miss
           for (int h = 0; h < (SWIGLU ? 1 : NSUB); ++h) {
             const int acc = NSUB == 1 ? (tile_no & 1) : h;
             const uint32_t acc_phase = NSUB == 1 ? ((uint32_t)(tile_no >> 1) & 1) : ((uint32_t)tile_no & 1);
-            const int nb = t.n0 + h * SUBN;              // first (output) column of this sub-tile
+            int nb = t.n0 + h * SUBN;                    // first (output) column of this sub-tile
             bool ok = h > 0 || mbar_wait_bounded(&tmem_full[acc], acc_phase);   // one "full" barrier per tile
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) { if (lane == 0) atomicExch(&g_gemm_status, 4); alive = false; break; }
             tc_fence_after();
+            const bool bal = RAG == 0 && !SWIGLU && p.bal;
+            bool released = false;                                 // the accumulator has been handed back already
             const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * ACC_COLS);
             // Full 32-row x 64-column pieces go through shared memory (128-byte swizzle) and a TMA tile store
             // addressed through C's own tensor map; ragged pieces (tile clipped by a strip or the matrix edge)
             // and split-K partial sums are stored from registers.
-            const int row0 = t.m0 + (int)rank * BM + quad * 32;
-            const bool rows_full = row0 + 32 <= t.m1;
+            int row0 = t.m0 + (int)rank * BM + quad * 32;
+            bool rows_full = row0 + 32 <= t.m1;
             // C map coordinates of (row0, nb): a tile lies inside one strip, so only x moves from piece to piece
             // (unless a strip row is cut into chunks, which puts the chunk index in y as well)
             int cx0, cy0, cz0, cu0;
@@ -743,6 +807,98 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     }
                     store_packed(pk, c);
                 }
+            } else if (bal && t.part != 0) {
+                // Balanced split, a tile shared by t.nshare units.  A unit's slot of the workspace holds one CTA's 128 x BN
+                // partial sums as [epilogue warp][64-column piece][16][lane] float4 -- the registers of a piece exactly as
+                // tcgen05.ld hands them out, so a warp reads and writes 512 contiguous bytes per instruction; the flags of all
+                // CTAs follow the slots.
+                // A unit's share can end in one tile and go on in the next: a CTA has two slots (and two sets of flags), the
+                // first for a share that starts inside a tile, the second for the share that starts a tile (k = 0).
+                const size_t slot_floats = (size_t)BM * BN, quad_off = (size_t)quad * 32 * BN;
+                constexpr int PPS = SUBN / 64;                     // pieces per sub-tile
+                const size_t my_slot = (size_t)blockIdx.x * 2 + (t.mine == 0 ? 1 : 0);
+                // (1) this sub-tile's partial sums -> own slot; the accumulator goes back to the tensor cores at once
+#pragma unroll 1
+                for (int c = 0; c < npieces; ++c) {
+                    load_piece(ra, c);
+                    tmem_ld_wait();
+                    tmem_regs_ready(ra);
+                    float* dst = p.ws + my_slot * slot_floats + quad_off + (size_t)(h * PPS + c) * (32 * 64) + (size_t)lane * 4;
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        *reinterpret_cast<uint4*>(dst + j * 128) = make_uint4(ra[4 * j], ra[4 * j + 1], ra[4 * j + 2], ra[4 * j + 3]);
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    if (CTAS == 2) mbar_arrive_cluster(tmem_empty0 + (uint32_t)acc * 8u);
+                    else mbar_arrive(&tmem_empty[acc]);
+                }
+                released = true;
+                if (h == NSUB - 1) {
+                    // (2) mark this warp's rows of the share as written
+                    __threadfence();
+                    __syncwarp();
+                    if (lane == 0) asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p.bal_flags + my_slot * 4 + quad), "l"(p.bal_mark) : "memory");
+                    // (3) the reduction of a shared tile waits for the other sharers; if this unit's next piece of work is
+                    // another share, that one is written first -- its sharers wait for it in turn, and a unit that reduced
+                    // before writing would make them queue up one behind the other across the whole group
+                    pend[npend++] = t;
+                    TileCoord nx;
+                    const bool more = sched.template get<RAG, FULL>(it + 1, nx);
+                    if (!(more && nx.part != 0)) {
+                        for (int q = 0; q < npend && alive; ++q) {
+                            t = pend[q];
+                            m = t.m0 + (int)rank * BM + quad * 32 + lane;
+                            row0 = t.m0 + (int)rank * BM + quad * 32;
+                            rows_full = row0 + 32 <= t.m1;
+                            const int cta0 = (int)blockIdx.x - t.mine * CTAS;       // the first sharer's CTA of this rank
+                            bool seen = true;                                       // bounded wait for the same rows of the other sharers
+                            const uint64_t t0 = global_timer_ns();
+                            for (int o = 0; seen && o < t.nshare; ++o) {
+                                if (o == t.mine) continue;
+                                const unsigned long long* f = p.bal_flags + ((size_t)(cta0 + o * CTAS) * 2 + (o == 0 ? 1 : 0)) * 4 + quad;
+                                while (ld_acquire_u64(f) != p.bal_mark)
+                                    if (global_timer_ns() - t0 > kWaitLimitNs) { seen = false; break; }
+                            }
+                            seen = __all_sync(0xffffffffu, seen);
+                            if (!seen) { if (lane == 0) atomicExch(&g_gemm_status, 7); alive = false; break; }
+                            // every nshare-th piece of the tile is this unit's: sum the sharers' partial sums in the order of
+                            // their k ranges (the same bits on every run) and store the piece as usual
+#pragma unroll 1
+                            for (int hh = 0; hh < NSUB; ++hh) {
+                                nb = t.n0 + hh * SUBN;
+                                to_coords<FULL>(p.c, row0, nb, cx0, cy0, cz0, cu0);
+                                const int np = min(PPS, (t.n1 - nb + 63) / 64);
+#pragma unroll 1
+                                for (int c = 0; c < np; ++c) {
+                                    const int pc = hh * PPS + c;
+                                    if (pc % t.nshare != t.mine) continue;
+                                    const size_t piece_off = quad_off + (size_t)pc * (32 * 64) + (size_t)lane * 4;
+#pragma unroll 1
+                                    for (int o = 0; o < t.nshare; ++o) {
+                                        const float* src = p.ws + ((size_t)(cta0 + o * CTAS) * 2 + (o == 0 ? 1 : 0)) * slot_floats + piece_off;
+#pragma unroll
+                                        for (int j = 0; j < 16; ++j) {             // sixteen loads in flight, then the sums
+                                            const uint4 v = __ldcg(reinterpret_cast<const uint4*>(src + j * 128));
+                                            rb[4 * j] = v.x; rb[4 * j + 1] = v.y; rb[4 * j + 2] = v.z; rb[4 * j + 3] = v.w;
+                                        }
+                                        if (o == 0) {
+#pragma unroll
+                                            for (int i = 0; i < 64; ++i) ra[i] = rb[i];
+                                        } else {
+#pragma unroll
+                                            for (int i = 0; i < 64; ++i) ra[i] = __float_as_uint(__uint_as_float(ra[i]) + __uint_as_float(rb[i]));
+                                        }
+                                    }
+                                    store_piece(ra, c);
+                                }
+                            }
+                        }
+                        npend = 0;
+                        if (!alive) break;
+                    }
+                }
             } else if (EW > 1) {
 #pragma unroll 1
                 for (int c = hf; c < npieces; c += EW) {
@@ -769,7 +925,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) {
+            if (lane == 0 && !released) {
                 if (CTAS == 2) mbar_arrive_cluster(tmem_empty0 + (uint32_t)acc * 8u);
                 else mbar_arrive(&tmem_empty[acc]);
                 if (SWIGLU) {                            // both accumulators of the tile have been read
@@ -899,7 +1055,7 @@ static ccl_status merge_width(int64_t* cur, int64_t w, const char* dim) {
 // cap > 0: a ragged batch -- the tile grid of one problem covers `cap` rows, d->M is the total row count of A and C
 // ragk: a batch with ragged K -- d->K is the total row count of the concatenated A [K x M] and B [K x N]
 static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, const void* A, const void* B, const void* C, int sms, int pairs, GemmPlan* plan,
-                            int64_t cap = 0, bool ragk = false) {
+                            int64_t cap = 0, bool ragk = false, size_t max_ws = ~(size_t)0) {
     if (!d) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: NULL descriptor");
     if (d->M <= 0 || d->N <= 0 || d->K <= 0) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: M, N, K must be positive");
     if (d->M >= (INT64_C(1) << 31) || d->N >= (INT64_C(1) << 31) || d->K >= (INT64_C(1) << 31)) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: dimension too large");
@@ -1032,9 +1188,61 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
         }
     }
     if (best < 0) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: no kernel variant matches the forced CCL_GEMM_* settings");
+    // Balanced split: instead of whole tiles, every unit of a group gets the same number of k blocks of the group's tiles
+    // laid end to end (at most `share`), so nothing is lost to a last round that fills a fraction of the machine or to a
+    // tile count below the unit count.  A tile cut between units costs one unit its partial sums (written to the
+    // workspace while its next tile computes) and the finishing unit a read of them; with shares shorter than a tile the
+    // shares of a tile run side by side and the finishing one reads several.  Modelled in the same cycles as above.
+    bool balanced = false;
+    {
+        const char* force_bal = std::getenv("CCL_GEMM_BALANCED");   // 0: never, 1: whenever the call qualifies
+        const int want = force_bal ? atoi(force_bal) : -1;
+        const bool can = want != 0 && batch == 1 && !swiglu && cap == 0 && !ragk && num_kb >= 2 && !(force_split && atoi(force_split) > 1);
+        double best_bal = -1.0;
+        int bc = 0, bb = 0;
+        int64_t bal_rounds = 0;
+        for (int c = 1; can && c <= 2; ++c) {
+            if (c == 2 && pairs <= 0) continue;
+            if (force_ctas && atoi(force_ctas) != c) continue;
+            const int units = c == 2 ? pairs : sms;
+            for (int b : {512, 256, 192, 128}) {
+                if (c == 1 && b > 256) continue;
+                if (c == 2 && b == 192 && !bt) continue;
+                if (b == 192 && (c == 2 ? no_192_pair : no_192)) continue;
+                if (force_bn && atoi(force_bn) != b) continue;
+                const int64_t tm = strips_m * ((Wm + BM * c - 1) / (BM * c)), tn = strips_n * ((Wn + b - 1) / b);
+                if (tm == 1 && want != 1) continue;              // one row of tiles streams B from HBM: the split-K plans above are tuned for it
+                int G = 1;
+                if (groups > 1 && units >= groups && (group_dim == 0 ? tn % groups == 0 : group_dim == 1 ? tm % groups == 0
+                                                                    : (tn % groups_n == 0 && tm % (groups / groups_n) == 0))) G = groups;
+                const int64_t tiles_g = tm * tn / G;
+                const int upg = units / G;
+                const int64_t rounds = tiles_g / upg, rest = tiles_g - rounds * upg;     // whole rounds, tiles of the shared part
+                if (rest == 0 || rest * num_kb >= (INT64_C(1) << 30)) continue;
+                const int64_t sharers = std::max<int64_t>(1, std::min<int64_t>(upg, rest * num_kb / 4));   // a share is at least four k blocks
+                const int64_t share = (rest * num_kb + sharers - 1) / sharers;
+                const size_t ws = (size_t)G * upg * c * 2 * ((size_t)BM * b * 4 + 32);
+                if (ws > max_ws) continue;
+                const double t_kb = b == 512 ? 1050.0 : (c == 1 && b == 256 ? 680.0 : (c == 1 ? 570.0 : 620.0));
+                const double t_drain = b == 512 ? 7000.0 : 1500.0;
+                // every sharer writes its partial sums and reads as much back (its part of the columns from every
+                // sharer), all of them at the same time: measured ~17 B/clk per SM then (the L2's write side saturates);
+                // this runs behind the unit's next tile if it has one (costing that tile a little of its operand
+                // bandwidth), and is the tail of the kernel if the shares are all there is
+                const double fix = 2.0 * (double)BM * b * 4 / 17.0;
+                const double cost = ((double)share + (double)rounds * num_kb) * t_kb + t_drain + (rounds == 0 ? fix : 0.15 * fix) + 3000.0 + 2500.0;
+                if (best_bal < 0 || cost < best_bal) { best_bal = cost; bc = c; bb = b; bal_rounds = rounds; }
+            }
+        }
+        // Measured (B200): the shares pay off only where a last round would leave most of the machine idle, K is long enough
+        // to dwarf the partial-sum traffic and the kernel is too short to run into the power cap (a long GEMM at the cap
+        // turns fewer idle cycles into lower clocks, not less time): taken on its own only with whole rounds behind the
+        // shares, a modelled gain of 10 % and under ~200 us; CCL_GEMM_BALANCED=1 forces it wherever it is legal.
+        if (best_bal > 0 && (want == 1 || (bal_rounds >= 1 && best_bal < 0.90 * best && best_bal < 400000.0))) { ctas = bc; bn = bb; splits = 1; balanced = true; best = best_bal; }
+    }
     if (std::getenv("CCL_GEMM_VERBOSE"))
-        std::fprintf(stderr, "ccl_gemm plan: %lld x %lld x %lld batch %lld -> %d CTA(s) per tile, tile width %d, %d K split(s), modelled %.0f cycles\n",
-                     (long long)d->M, (long long)d->N, (long long)d->K, (long long)batch, ctas, bn, splits, best);
+        std::fprintf(stderr, "ccl_gemm plan: %lld x %lld x %lld batch %lld -> %d CTA(s) per tile, tile width %d, %d K split(s)%s, modelled %.0f cycles\n",
+                     (long long)d->M, (long long)d->N, (long long)d->K, (long long)batch, ctas, bn, splits, balanced ? ", balanced split" : "", best);
     const int subn = bn > 256 ? 256 : bn;                // columns of one MMA / one TMEM accumulator
     plan->subn = subn;
     const int bm = BM * ctas;
@@ -1095,6 +1303,21 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
         p.sch_units = units; p.sch_gm = gm; p.sch_gn = gn; p.sch_upg = upg; p.sch_floaters = units - upg * p.groups;
         p.sch_rounds = (int32_t)rounds; p.sch_per_group = (int32_t)per_group; p.sch_pool_per_group = (int32_t)(per_group - rounds * upg);
     }
+    if (balanced) {                                      // balanced split of the tiles that do not fill a round (see Scheduler)
+        units = ctas == 2 ? pairs : sms;
+        units -= units % p.groups;
+        const int upg = units / p.groups;
+        const int64_t rest = p.sch_per_group % upg, work = rest * p.num_kb;
+        if (rest > 0) {
+            const int64_t sharers = std::max<int64_t>(1, std::min<int64_t>(upg, work / 4));
+            plan->grid = (unsigned)(units * ctas);
+            p.bal = 1; p.bal_units = (int32_t)sharers; p.bal_tiles = (int32_t)rest;
+            p.bal_q = (int32_t)(work / sharers); p.bal_r = (int32_t)(work % sharers);
+            p.sch_units = units; p.sch_upg = upg; p.sch_floaters = 0; p.sch_rounds = (int32_t)(p.sch_per_group / upg); p.sch_pool_per_group = 0;
+            plan->ws_bytes = (size_t)plan->grid * 2 * ((size_t)BM * bn * 4 + 32);   // two slots of partial sums per CTA, then a flag per slot and epilogue warp
+        }
+    }
+    p.fd_num_kb = make_fastdiv(p.num_kb);
     // Raster panel height: the units of a group that run at the same time cover `panel` m-tiles by
     // ceil(upg / panel) n-tiles; all groups walk the same m-panel.  The operand rows + columns such a wave
     // touches are what it pulls from DRAM (the L2 does not hold a wave's footprint until the next wave), so
@@ -1239,7 +1462,7 @@ using namespace ccl;
 
 // ---- host-side cache of prepared calls (plan + encoded tensor maps) --------------------------------------
 struct PreparedKey {
-    int64_t f[38];          // every field of the descriptor, the batch, the three pointers, the ragged-batch arguments
+    int64_t f[40];          // every field of the descriptor, the batch, the three pointers, the ragged-batch arguments, the workspace at hand
     int dev;
     int mode;               // 0 plain, 1 gated activation
     float alpha, beta;
@@ -1272,7 +1495,7 @@ static void make_key(const ccl_gemm_desc* d, const int64_t* batch4, const void* 
     k->dev = -1;
     (void)cudaGetDevice(&k->dev);
     size_t pos = 0;
-    for (const char* name : {"CCL_GEMM_CTAS", "CCL_GEMM_BN", "CCL_GEMM_SPLITK", "CCL_GEMM_PANEL", "CCL_GEMM_RAGGED_DENSE"}) {
+    for (const char* name : {"CCL_GEMM_CTAS", "CCL_GEMM_BN", "CCL_GEMM_SPLITK", "CCL_GEMM_PANEL", "CCL_GEMM_RAGGED_DENSE", "CCL_GEMM_BALANCED"}) {
         const char* v = std::getenv(name);
         for (const char* c = v ? v : ""; *c && pos + 2 < sizeof(k->env); ++c) k->env[pos++] = *c;
         if (pos + 1 < sizeof(k->env)) k->env[pos++] = ';';
@@ -1350,8 +1573,12 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     // reuse the plan and the two encoded tensor maps: a host-side cache only, nothing is kept on the device.
     PreparedKey key;
     make_key(d, batch4, A_dev, B_dev, C_dev, &key);
-    key.mode = swiglu ? 1 : 0; key.alpha = alpha; key.beta = beta;
+    key.mode = (swiglu ? 1 : 0) | (static_ws ? 2 : 0); key.alpha = alpha; key.beta = beta;
     key.f[36] = (int64_t)reinterpret_cast<uintptr_t>(m_offs) ^ ((int64_t)reinterpret_cast<uintptr_t>(k_offs) << 1); key.f[37] = cap + (k_offs ? (INT64_C(1) << 62) : 0);
+    // The balanced split is optional: it is planned only when the workspace at hand holds its partial sums (the caller's
+    // ws_bytes; the scratch array for ccl_gemm_static_ws).  A caller that passes none gets whole-tile plans, as before.
+    const size_t max_ws = static_ws ? (size_t)CCL_GEMM_STATIC_WS_BYTES : (ws_dev ? ws_bytes : 0);
+    key.f[38] = (int64_t)max_ws;
     Prepared prep;
     bool hit = false;
     {
@@ -1362,7 +1589,7 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     ccl_status s;
     if (!hit) {
         GemmPlan& plan = prep.plan;
-        s = make_plan(d, batch, swiglu, A_dev, B_dev, C_dev, 148, 74, &plan, cap, k_offs != nullptr);     // validation first: no CUDA call on bad input
+        s = make_plan(d, batch, swiglu, A_dev, B_dev, C_dev, 148, 74, &plan, cap, k_offs != nullptr, max_ws);     // validation first: no CUDA call on bad input
         if (s) return s;
         if (batch > 1) {
             const MatView* views[3] = {&plan.va, &plan.vb, &plan.vc};
@@ -1380,10 +1607,10 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
         CCL_CUDA_TRY(cudaDeviceGetAttribute(&prep.sms, cudaDevAttrMultiProcessorCount, dev));
         if (dev != key.dev) {
             make_key(d, batch4, A_dev, B_dev, C_dev, &key);
-            key.mode = swiglu ? 1 : 0; key.alpha = alpha; key.beta = beta;
+            key.mode = (swiglu ? 1 : 0) | (static_ws ? 2 : 0); key.alpha = alpha; key.beta = beta; key.f[38] = (int64_t)max_ws;
             key.f[36] = (int64_t)reinterpret_cast<uintptr_t>(m_offs) ^ ((int64_t)reinterpret_cast<uintptr_t>(k_offs) << 1); key.f[37] = cap + (k_offs ? (INT64_C(1) << 62) : 0);
         }
-        if ((s = make_plan(d, batch, swiglu, A_dev, B_dev, C_dev, prep.sms, resident_pairs(), &plan, cap, k_offs != nullptr))) return s;
+        if ((s = make_plan(d, batch, swiglu, A_dev, B_dev, C_dev, prep.sms, resident_pairs(), &plan, cap, k_offs != nullptr, max_ws))) return s;
         plan.p.C = static_cast<uint16_t*>(C_dev);
         plan.p.a.batched = batch4[1] != 0; plan.p.b.batched = batch4[2] != 0; plan.p.c.batched = m_offs ? 0 : 1;
         plan.p.m_offs = m_offs;
@@ -1426,6 +1653,11 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     }
     plan.p.ws = static_cast<float*>(ws_dev);
     cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    if (plan.p.bal) {                                    // flags behind the partial sums, cleared in front of the launch
+        plan.p.bal_flags = reinterpret_cast<unsigned long long*>(static_cast<char*>(ws_dev) + (size_t)plan.grid * 2 * ((size_t)BM * plan.bn * 4));
+        plan.p.bal_mark = 1ull;
+        CCL_CUDA_TRY(cudaMemsetAsync(plan.p.bal_flags, 0, (size_t)plan.grid * 2 * 32, st));
+    }
     // Soft wave barrier for problems of three or more full rounds of tiles (CCL_GEMM_WAVESYNC=0 turns it off, =n syncs
     // every n-th round): without it the CTAs that share an A panel or B
     // columns drift apart by more than the L2 holds and fetch the same lines from DRAM 2-3 times.

@@ -81,32 +81,53 @@ def timed(fn, reps, warm=2):
     return e0.elapsed_time(e1) / reps
 
 
-def traffic_remote(g, layout_bc, place_bc, S, assign, align=0):
-    """Remote bytes (A, B, C) of one policy; None if the partition does not apply (M % P != 0)."""
+def partitions(g):
+    """Output partitions swept per GEMM (Sec. 4.1 sweeps them and reports the best): N strips, M strips where M divides,
+    and the 2-D cuts pm x pn of P with both factors above 1.  Entries: (label, assign, part_m)."""
+    M, N, P = g["M"], g["N"], g["P"]
+    out = [("N", ccl.ASSIGN_N_STRIPS, 0)]
+    if M % P == 0 and M >= P:
+        out.append(("M", ccl.ASSIGN_M_STRIPS, 0))
+    for pm in range(2, P):
+        if P % pm == 0 and M % pm == 0 and N % (P // pm) == 0:
+            out.append((f"{pm}x{P // pm}", ccl.ASSIGN_2D, pm))
+    return out
+
+
+def operand_mats(g, layout_bc, assign, part_m, align, e=2):
+    """Descriptors of A, B, C under one output partition: the operands whose rows / columns the partition cuts follow it in
+    the given layout (strips = the blocks along that dimension), the others stay row-major.  Returns (mats, parts)."""
     M, N, K, P = g["M"], g["N"], g["K"], g["P"]
-    if assign == ccl.ASSIGN_M_STRIPS and (M % P or M < P):
-        return None
     at, bt = g["a_trans"], g["b_trans"]
-    td = ccl.TrafficDesc()
-    td.M, td.N, td.K, td.BM, td.BN = M, N, K, 128, 128
-    a_shape = (K, M) if at else (M, K)
-    b_shape = (N, K) if bt else (K, N)
-    if assign == ccl.ASSIGN_N_STRIPS:                       # C split along N: B and C follow, A is shared
-        parts = (ccl.PART_NONE, ccl.PART_ROWS if bt else ccl.PART_COLS, ccl.PART_COLS)
-    else:                                                   # C split along M: A and C follow, B is shared
-        parts = (ccl.PART_COLS if at else ccl.PART_ROWS, ccl.PART_NONE, ccl.PART_ROWS)
-    shapes = (a_shape, b_shape, (M, N))
+    pm = P if assign == ccl.ASSIGN_M_STRIPS else (part_m if assign == ccl.ASSIGN_2D else 1)
+    pn = P if assign == ccl.ASSIGN_N_STRIPS else (P // part_m if assign == ccl.ASSIGN_2D else 1)
+    a_part = (ccl.PART_COLS if at else ccl.PART_ROWS) if pm > 1 else ccl.PART_NONE
+    b_part = (ccl.PART_ROWS if bt else ccl.PART_COLS) if pn > 1 else ccl.PART_NONE
+    c_part = ccl.PART_COLS if pn > 1 and pm == 1 else (ccl.PART_ROWS if pm > 1 else ccl.PART_NONE)   # 2-D: C's rows follow A
+    parts = (a_part, b_part, c_part)
+    strips = (pm, pn, pn if c_part == ccl.PART_COLS else pm)
+    shapes = ((K, M) if at else (M, K), (N, K) if bt else (K, N), (M, N))
     ms = []
     for X in range(3):
         is_ccl = layout_bc != ccl.ROWMAJOR and parts[X] != ccl.PART_NONE
-        ms.append(ccl.Mat(shapes[X][0], shapes[X][1], 2, P, parts[X] if is_ccl else ccl.PART_NONE,
+        ms.append(ccl.Mat(shapes[X][0], shapes[X][1], e, strips[X] if is_ccl else 1, parts[X] if is_ccl else ccl.PART_NONE,
                           layout_bc if is_ccl else ccl.ROWMAJOR, align if is_ccl else 0))
+    return ms, parts
+
+
+def traffic_remote(g, layout_bc, place_bc, S, assign, align=0, part_m=0):
+    """Remote bytes (A, B, C) of one policy under one output partition."""
+    M, N, K, P = g["M"], g["N"], g["K"], g["P"]
+    at, bt = g["a_trans"], g["b_trans"]
+    td = ccl.TrafficDesc()
+    td.M, td.N, td.K, td.BM, td.BN = M, N, K, 128, 128
+    ms, parts = operand_mats(g, layout_bc, assign, part_m, align)
     td.A, td.B, td.C = ms
     td.a_trans, td.b_trans, td.P, td.page_bytes = at, bt, P, S
     for X in range(3):
         split = parts[X] != ccl.PART_NONE
         td.place[X] = place_bc if split else (ccl.PLACE_RR if place_bc != ccl.PLACE_BEST else ccl.PLACE_BEST)
-    td.assign, td.strip_tiling = assign, 1
+    td.assign, td.strip_tiling, td.part_m = assign, 1, part_m
     nt, pages = ccl.ccl_traffic_sizes(td)
     per_cta = torch.empty((nt, 3, 2), dtype=torch.int64, device="cuda")
     totals = torch.empty((3, 2), dtype=torch.int64, device="cuda")
@@ -124,31 +145,17 @@ def traffic_remote(g, layout_bc, place_bc, S, assign, align=0):
     return out
 
 
-def traffic_desc(g, layout_bc, place_bc, S, assign, align=0, e=2):
-    """Library descriptor of one placement policy; None if the partition does not apply (M % P != 0)."""
+def traffic_desc(g, layout_bc, place_bc, S, assign, align=0, e=2, part_m=0):
+    """Library descriptor of one placement policy under one output partition."""
     M, N, K, P = g["M"], g["N"], g["K"], g["P"]
-    if assign == ccl.ASSIGN_M_STRIPS and (M % P or M < P):
-        return None
-    at, bt = g["a_trans"], g["b_trans"]
     td = ccl.TrafficDesc()
     td.M, td.N, td.K, td.BM, td.BN = M, N, K, 128, 128
-    a_shape = (K, M) if at else (M, K)
-    b_shape = (N, K) if bt else (K, N)
-    if assign == ccl.ASSIGN_N_STRIPS:
-        parts = (ccl.PART_NONE, ccl.PART_ROWS if bt else ccl.PART_COLS, ccl.PART_COLS)
-    else:
-        parts = (ccl.PART_COLS if at else ccl.PART_ROWS, ccl.PART_NONE, ccl.PART_ROWS)
-    shapes = (a_shape, b_shape, (M, N))
-    ms = []
-    for X in range(3):
-        is_ccl = layout_bc != ccl.ROWMAJOR and parts[X] != ccl.PART_NONE
-        ms.append(ccl.Mat(shapes[X][0], shapes[X][1], e, P, parts[X] if is_ccl else ccl.PART_NONE,
-                          layout_bc if is_ccl else ccl.ROWMAJOR, align if is_ccl else 0))
+    ms, parts = operand_mats(g, layout_bc, assign, part_m, align, e)
     td.A, td.B, td.C = ms
-    td.a_trans, td.b_trans, td.P, td.page_bytes = at, bt, P, S
+    td.a_trans, td.b_trans, td.P, td.page_bytes = g["a_trans"], g["b_trans"], P, S
     for X in range(3):
         td.place[X] = place_bc if parts[X] != ccl.PART_NONE else ccl.PLACE_RR
-    td.assign, td.strip_tiling = assign, 1
+    td.assign, td.strip_tiling, td.part_m = assign, 1, part_m
     return td
 
 
@@ -156,19 +163,17 @@ LRU_EXEC = dict(wave_ctas=1, k_slice=0)       # how a chiplet's CTAs run in the 
 
 
 def traffic_lru_best(g, layout_bc, place_bc, S, model_kw, e=2):
-    """Remote bytes (A, B, C) behind a finite LRU L2 per chiplet: the best of both output partitions and both CTA
+    """Remote bytes (A, B, C) behind a finite LRU L2 per chiplet: the best of the output partitions (N strips, M strips, 2-D cuts) and both CTA
     traversals, as the paper reports (Sec. 4.1 sweeps the CTA traversal and the output partition and keeps the best)."""
     best = None
-    for assign in (ccl.ASSIGN_N_STRIPS, ccl.ASSIGN_M_STRIPS):
-        td = traffic_desc(g, layout_bc, place_bc, S, assign, align=S, e=e)
-        if td is None:
-            continue
+    for label, assign, pm in partitions(g):
+        td = traffic_desc(g, layout_bc, place_bc, S, assign, align=S, e=e, part_m=pm)
         for traversal in (0, 1):
             t = torch.empty((3, 2), dtype=torch.int64, device="cuda")
             ccl.ccl_traffic_lru(td, ccl.L2Model(traversal=traversal, **model_kw, **LRU_EXEC), t)
             r = [int(x) for x in t.cpu()[:, 1]]
             if best is None or sum(r) < sum(best["remote"]):
-                best = dict(remote=r, partition="N" if assign == ccl.ASSIGN_N_STRIPS else "M", traversal=traversal)
+                best = dict(remote=r, partition=label, traversal=traversal)
     return best
 
 
@@ -226,11 +231,9 @@ def run_gemm(g, pk, reps, lru=False):
                                 ("row_best", ccl.ROWMAJOR, ccl.PLACE_BEST, S), ("ccl_block", ccl.CCL, ccl.PLACE_BLOCK, S),
                                 ("ccl_rr", ccl.CCL, ccl.PLACE_RR, S), ("ileave_rr", ccl.CCL_INTERLEAVED, ccl.PLACE_RR, S)):
         best = None
-        for assign in (ccl.ASSIGN_N_STRIPS, ccl.ASSIGN_M_STRIPS):
-            r = traffic_remote(g, lay, place, Sp, assign, align=Sp)
-            if r is None:
-                continue
-            r["partition"] = "N" if assign == ccl.ASSIGN_N_STRIPS else "M"
+        for label, assign, pm in partitions(g):
+            r = traffic_remote(g, lay, place, Sp, assign, align=Sp, part_m=pm)
+            r["partition"] = label
             if best is None or sum(r["remote"]) < sum(best["remote"]):
                 best = r
         pol[tag] = best

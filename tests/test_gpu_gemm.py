@@ -433,3 +433,76 @@ def test_gemm_axpby_identity_scalars_equal_plain_gemm():
     with pytest.raises(ccl.CclError) as ei:
         ccl.ccl_gemm_axpby(d, float("nan"), 0.0, a_dev, b_dev, c_dev)
     assert ei.value.status == ccl.ERR_INVALID_ARG
+
+
+# ---------------------------------------------------------------------------------------------
+# balanced split: every unit gets the same number of k blocks; tiles cut between units are summed in the order of k
+# ---------------------------------------------------------------------------------------------
+@pytest.fixture
+def balanced():
+    keys = ("CCL_GEMM_BALANCED", "CCL_GEMM_CTAS", "CCL_GEMM_BN")
+    old = {k: os.environ.pop(k, None) for k in keys}
+    os.environ["CCL_GEMM_BALANCED"] = "1"
+    yield
+    for k in keys:
+        os.environ.pop(k, None)
+        if old[k] is not None:
+            os.environ[k] = old[k]
+
+
+BALANCED = [
+    # M, N, K, P, layouts, a_trans, b_trans, out_part
+    (768, 2048, 4096, 4, ("row", "ccl", "ccl"), 1, 0, 2),      # fewer tiles than units: the shares of a tile run side by side
+    (256, 768, 2048, 4, ("row", "ccl", "ccl"), 0, 1, 2),       # the single-expert GEMM: many shares per tile
+    (4096, 1536, 2048, 4, ("row", "ccl", "ccl"), 0, 0, 2),     # 1.3 rounds of tiles: a unit finishes the tile its neighbour began
+    (4096, 768, 2048, 2, ("row", "ccl", "ccl"), 0, 1, 2),
+    (520, 1536, 328, 4, ("row", "ccl", "ccl"), 0, 0, 2),       # ragged tiles in M, K not a multiple of 64
+    (300, 2304, 512, 2, ("row", "ccl", "row"), 0, 1, 2),
+    (1032, 1024, 1096, 1, ("row", "row", "row"), 1, 1, 0),     # plain raster
+    (2048, 2048, 2048, 4, ("ccl", "row", "ccl"), 0, 0, 1),     # M strips
+    (130, 384, 4096, 4, ("row", "ccl", "ccl"), 0, 0, 2),       # strips of 96 columns: every tile partial in N
+    (1024, 1024, 1024, 4, ("row", "ileave", "ileave"), 0, 0, 2),   # page-interleaved operands
+]
+
+
+@pytest.mark.parametrize("M,N,K,P,lay,at,bt,op", BALANCED)
+@pytest.mark.parametrize("variant", [None, (1, 128), (1, 256), (2, 256), (2, 512)], ids=lambda v: "auto" if v is None else f"c{v[0]}b{v[1]}")
+def test_gemm_balanced_split(balanced, M, N, K, P, lay, at, bt, op, variant):
+    """The balanced split forced on: parity with the oracle, the same bits on every run, flags left clear."""
+    if variant is not None:
+        os.environ["CCL_GEMM_CTAS"], os.environ["CCL_GEMM_BN"] = str(variant[0]), str(variant[1])
+    A, B = synth.gemm_operands(M, N, K, at, bt, seed=5, tag="balanced")
+    d = gemm_desc(M, N, K, P, lay, at, bt, op, 1, align=4096 if "ileave" in lay else 0)
+    got1, _ = check(d, A, B)
+    got2, _ = check(d, A, B)
+    np.testing.assert_array_equal(got1, got2)
+
+
+def test_gemm_balanced_split_needs_its_workspace_or_steps_aside(balanced):
+    """Without a workspace the call runs whole tiles (the balanced split is optional); with one that is too small for the
+    partial sums but not empty, likewise; results agree within the tolerance either way."""
+    M, N, K, P = 768, 2048, 4096, 4
+    A, B = synth.gemm_operands(M, N, K, 1, 0, seed=6, tag="balanced-ws")
+    d = gemm_desc(M, N, K, P, ("row", "ccl", "ccl"), 1, 0, 2, 1)
+    need = ccl.ccl_gemm_workspace(d)
+    a_dev, b_dev = to_layout(synth.bits(A), d.A), to_layout(synth.bits(B), d.B)
+    ref32, _, _ = orc.gemm(synth.bits(A), synth.bits(B), M, N, K, 1, 0)
+    os.environ.pop("CCL_GEMM_BALANCED")                      # the planner's own choice from here on
+    for ws in (None, torch.empty(1024, dtype=torch.float32, device="cuda"), torch.empty(need // 4, dtype=torch.float32, device="cuda")):
+        c_dev = torch.zeros(M * N, dtype=torch.int16, device="cuda")
+        if ws is not None and ws.numel() * 4 < ccl.ccl_gemm_workspace(d):
+            try:
+                ccl.ccl_gemm(d, a_dev, b_dev, c_dev, ws)
+            except ccl.CclError as e:                         # a plan split along K in the old way insists on its workspace
+                assert e.status == ccl.ERR_WORKSPACE
+                continue
+        else:
+            try:
+                ccl.ccl_gemm(d, a_dev, b_dev, c_dev, ws)
+            except ccl.CclError as e:
+                assert ws is None and e.status == ccl.ERR_WORKSPACE
+                continue
+        assert ccl.ccl_gemm_status()[0] == ccl.OK
+        g = synth.from_bits(from_layout(c_dev, d.C)).to(torch.float32).numpy()
+        err = np.abs(g - ref32) / np.maximum(1.0, np.abs(ref32))
+        assert err.max() <= tol(K)
