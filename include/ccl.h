@@ -25,8 +25,9 @@
  * Test / diagnostic switches (environment variables, read by the library; none changes a result beyond the
  * rounding order of a split-K sum):
  *   CCL_GEMM_CTAS = 1|2            force one CTA per tile or a cta_group::2 pair
- *   CCL_GEMM_BN = 64|128|192|256|512   force the tile width
+ *   CCL_GEMM_BN = 128|192|256|512  force the tile width
  *   CCL_GEMM_SPLITK = n            force the number of K splits
+ *   CCL_GEMM_BALANCED = 0|1        never / always (where legal) cut the tiles that do not fill a round into equal shares
  *   CCL_GEMM_WAVESYNC = 0|n        soft wave barrier off / every n-th round of tiles
  *   CCL_GEMM_PDL = 0               no programmatic dependent launch
  *   CCL_GEMM_RAGGED_DENSE = 0      ragged batches walk the fixed grid of max_rows per problem
@@ -175,7 +176,14 @@ typedef struct ccl_gemm_desc {
     int32_t part_m;   /* out_part == CCL_PART_2D: blocks along M (a divisor of P); ignored otherwise */
 } ccl_gemm_desc;
 
-/* Bytes of device workspace ccl_gemm needs for this problem (0 when none). */
+/*
+ * Bytes of device workspace the preferred plan of this problem uses (0 when none): fp32 partial sums of a problem split
+ * along K.  Two kinds of plan use it: the classic split (every tile computed by several units over disjoint k ranges,
+ * summed by a second kernel) INSISTS on it -- ccl_gemm returns CCL_ERR_WORKSPACE without it --, the balanced split
+ * (the tiles that do not fill a round of the machine are cut into equal shares of k blocks, one per unit, and reduced
+ * inside the kernel, in the order of k: the same bits on every run) is OPTIONAL: given less than it needs, ccl_gemm
+ * falls back to a whole-tile plan.  Calls that can overlap on the GPU must not share a workspace.
+ */
 ccl_status ccl_gemm_workspace(const ccl_gemm_desc* d, size_t* bytes);
 /*
  * Enqueue the GEMM.  ws_dev may be NULL when ccl_gemm_workspace reports 0.

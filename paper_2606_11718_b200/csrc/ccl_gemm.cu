@@ -1146,8 +1146,7 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     const int64_t strips_m = Mt / Wm, strips_n = Nc / Wn;
     int ctas = 1, bn = 256, splits = 1;
     double best = -1.0;
-    // Tuning / test overrides (environment): CCL_GEMM_CTAS = 1|2, CCL_GEMM_BN = 128|192|256|512,
-    // CCL_GEMM_SPLITK = number of K splits, CCL_GEMM_PANEL = raster panel height in m-tiles.
+    // Test overrides (environment): CCL_GEMM_CTAS = 1|2, CCL_GEMM_BN = 128|192|256|512, CCL_GEMM_SPLITK = number of K splits.
     const char* force_ctas = std::getenv("CCL_GEMM_CTAS");
     const char* force_bn = std::getenv("CCL_GEMM_BN");
     const char* force_split = std::getenv("CCL_GEMM_SPLITK");
@@ -1333,7 +1332,6 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
             if (best_fp < 0 || fp <= best_fp) { best_fp = fp; p.panel = pnl; }
         }
     }
-    if (const char* f = std::getenv("CCL_GEMM_PANEL")) p.panel = std::max(1, atoi(f));
     p.fd_upg = make_fastdiv(p.sch_upg); p.fd_groups = make_fastdiv(p.groups); p.fd_splits = make_fastdiv(p.splits);
     p.fd_per_panel = make_fastdiv((int64_t)p.panel * p.sch_gn); p.fd_panel = make_fastdiv(p.panel);
     p.fd_tps_m = make_fastdiv(p.tps_m); p.fd_tps_n = make_fastdiv(p.tps_n);
@@ -1495,7 +1493,7 @@ static void make_key(const ccl_gemm_desc* d, const int64_t* batch4, const void* 
     k->dev = -1;
     (void)cudaGetDevice(&k->dev);
     size_t pos = 0;
-    for (const char* name : {"CCL_GEMM_CTAS", "CCL_GEMM_BN", "CCL_GEMM_SPLITK", "CCL_GEMM_PANEL", "CCL_GEMM_RAGGED_DENSE", "CCL_GEMM_BALANCED"}) {
+    for (const char* name : {"CCL_GEMM_CTAS", "CCL_GEMM_BN", "CCL_GEMM_SPLITK", "CCL_GEMM_RAGGED_DENSE", "CCL_GEMM_BALANCED"}) {
         const char* v = std::getenv(name);
         for (const char* c = v ? v : ""; *c && pos + 2 < sizeof(k->env); ++c) k->env[pos++] = *c;
         if (pos + 1 < sizeof(k->env)) k->env[pos++] = ';';

@@ -538,6 +538,27 @@ def extras(out_dir, quick, only=None):
     json.dump(rows, open(os.path.join(out_dir, "report_extras.json"), "w"), indent=1)
 
 
+def one_gemm(args):
+    f = [int(x) for x in args.gemm.split(",")]
+    M, N, K = f[:3]
+    at, bt = (f[3], f[4]) if len(f) >= 5 else (0, 0)
+    P, page = 4, 4096
+    mB = ccl.Mat(N, K, 2, P, ccl.PART_ROWS, ccl.CCL, page) if bt else ccl.Mat(K, N, 2, P, ccl.PART_COLS, ccl.CCL, page)
+    mC = ccl.Mat(M, N, 2, P, ccl.PART_COLS, ccl.CCL, page)
+    d = ccl.GemmDesc()
+    d.M, d.N, d.K, d.A, d.B, d.C = M, N, K, (ccl.Mat(K, M, 2) if at else ccl.Mat(M, K, 2)), mB, mC
+    d.a_trans, d.b_trans, d.out_part, d.P, d.grouped_raster = at, bt, ccl.PART_COLS, P, 1
+    a = torch.empty((K, M) if at else (M, K), dtype=torch.bfloat16, device="cuda").normal_(0, 1)
+    b = torch.empty(ccl.ccl_buffer_bytes(mB) // 2, dtype=torch.bfloat16, device="cuda").normal_(0, 0.02)
+    c = torch.empty(ccl.ccl_buffer_bytes(mC) // 2, dtype=torch.bfloat16, device="cuda")
+    need = ccl.ccl_gemm_workspace(d)
+    ws = torch.empty(max(need, 16) // 4, dtype=torch.float32, device="cuda")
+    ms = timed(lambda: ccl.ccl_gemm(d, a, b, c, ws), args.reps, 1)
+    st, detail = ccl.ccl_gemm_status()
+    print(f"gemm {M}x{N}x{K} a_trans {at} b_trans {bt}: {ms * 1e3:.1f} us, {2.0 * M * N * K / ms / 1e9:.1f} TFLOP/s, "
+          f"algorithmic bytes {2 * (M * K + K * N + M * N)}, status {st}", flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--config", default="all")
@@ -550,6 +571,9 @@ def main():
     ap.add_argument("--paper-sweep", action="store_true", help="the 2 x 18-GEMM sweep of Sec. 4.2 under the finite-L2 model, both execution models (then exit)")
     ap.add_argument("--topology", action="store_true", help="experiment: split the SMs into the two dies by their latency to the L2 (then exit)")
     ap.add_argument("--extras", action="store_true", help="time the batched, gated-activation, alpha/beta, transposing- and batched-repack entry points (then exit)")
+    ap.add_argument("--gemm", default=None, help="M,N,K[,a_trans,b_trans]: run just this GEMM (B and C in CCL, P = 4, strips aligned to 4 KB, "
+                                                   "grouped raster) --reps times and print its time (e.g. for a profiler capture), then exit")
+    ap.add_argument("--reps", type=int, default=3)
     ap.add_argument("--only", default=None, help="run only the GEMMs whose name contains this text (e.g. for a profiler capture)")
     args = ap.parse_args()
     assert torch.cuda.is_available(), "report needs a CUDA device"
@@ -558,6 +582,9 @@ def main():
     LRU_EXEC.update(wave_ctas=args.lru_wave, k_slice=args.lru_kslice)
     if args.paper_sweep:
         paper_sweep(args.out, args.quick)
+        return
+    if args.gemm:
+        one_gemm(args)
         return
     if args.topology:
         topology(args.out)

@@ -41,7 +41,19 @@ def test_step_replays_from_a_cuda_graph():
     per_cta = torch.zeros((nt, 3, 2), dtype=torch.int64, device="cuda")
     totals = torch.zeros((3, 2), dtype=torch.int64, device="cuda")
 
+    # a GEMM whose last round is cut into equal shares (partial sums and their flags in the workspace)
+    db = gemm_desc(4096, 2048, 1536, P, ("row", "ccl", "ccl"), 0, 1, 2, 1)
+    Ab, Bb = synth.gemm_operands(4096, 2048, 1536, 0, 1, seed=33, tag="graphb")
+    import os
+    os.environ["CCL_GEMM_BALANCED"] = "1"
+    needbal = ccl.ccl_gemm_workspace(db)
+    abal, bbal = Ab.cuda(), torch.from_numpy(orc.repack(orc.Mat(2048, 1536, 2, P, orc.PART_ROWS, orc.CCL, 0), synth.bits(Bb), 0).view(np.int16)).cuda()
+    cbal = torch.zeros(ccl.ccl_buffer_bytes(db.C) // 2, dtype=torch.bfloat16, device="cuda")
+    wsbal = torch.empty(needbal // 4, dtype=torch.float32, device="cuda")
+    assert needbal > 0
+
     def step():
+        ccl.ccl_gemm(db, abal, bbal, cbal, wsbal)
         ccl.ccl_repack(d.B, b, b_ccl, 0)
         ccl.ccl_repack(dk.B, bk_row, bk_ccl, 0)
         ccl.ccl_gemm(d, a, b_ccl, c1)
@@ -50,7 +62,7 @@ def test_step_replays_from_a_cuda_graph():
         ccl.ccl_gemm_batched(d, E, ab, M * K * 2, b_ccl, 0, cb, nc * 2, wsb if needb else None)
         ccl.ccl_traffic(td, per_cta, totals)
 
-    outs = (c1, c2, ck, cb, per_cta, totals)
+    outs = (c1, c2, ck, cb, per_cta, totals, cbal)
     side = torch.cuda.Stream()
     with torch.cuda.stream(side):
         step()                                                   # eager: plans cached, kernels configured
@@ -70,6 +82,11 @@ def test_step_replays_from_a_cuda_graph():
         for o, w in zip(outs, want):
             assert torch.equal(o, w)
     assert ccl.ccl_gemm_status()[0] == ccl.OK
+    os.environ.pop("CCL_GEMM_BALANCED", None)
+    ref32, _, _ = orc.gemm(synth.bits(Ab), synth.bits(Bb), 4096, 2048, 1536, 0, 1, block=(0, 256, 0, 2048))
+    got = orc.repack(orc.Mat(4096, 2048, 2, P, orc.PART_COLS, orc.CCL, 0), cbal.view(torch.int16).cpu().numpy().view(np.uint16), 1).reshape(4096, 2048)
+    g = synth.from_bits(got[:256]).to(torch.float32).numpy()
+    assert (np.abs(g - ref32) / np.maximum(1.0, np.abs(ref32))).max() <= 1e-2 * (1536 / 1024.0) ** 0.5
 
 
 def test_ragged_batch_in_a_graph_follows_the_offsets_on_the_device():
