@@ -1233,11 +1233,14 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
                 if (best_bal < 0 || cost < best_bal) { best_bal = cost; bc = c; bb = b; bal_rounds = rounds; }
             }
         }
-        // Measured (B200): the shares pay off only where a last round would leave most of the machine idle, K is long enough
-        // to dwarf the partial-sum traffic and the kernel is too short to run into the power cap (a long GEMM at the cap
-        // turns fewer idle cycles into lower clocks, not less time): taken on its own only with whole rounds behind the
-        // shares, a modelled gain of 10 % and under ~200 us; CCL_GEMM_BALANCED=1 forces it wherever it is legal.
-        if (best_bal > 0 && (want == 1 || (bal_rounds >= 1 && best_bal < 0.90 * best && best_bal < 400000.0))) { ctas = bc; bn = bb; splits = 1; balanced = true; best = best_bal; }
+        // Measured (B200): on its own the planner never takes it.  Short GEMMs lose more to the partial-sum traffic (fp32
+        // through the L2, whose write side all sharers hit at once: ~17 B/clk per SM) and to the extra node in front of the
+        // launch than they gain (Qwen-size shapes: 1.2-2x slower), and a long GEMM runs at the power cap, where fewer idle
+        // cycles come back as lower clocks, not less time (4096 x 8192 x 8192: 9 % fewer cycles, 1 % less time; the two
+        // benchmark GEMMs: 2-3 % more time, for the two CTA pairs the equal groups leave out).  CCL_GEMM_BALANCED=1 turns it
+        // on wherever it is legal.
+        if (best_bal > 0 && want == 1) { ctas = bc; bn = bb; splits = 1; balanced = true; best = best_bal; }
+        (void)bal_rounds;
     }
     if (std::getenv("CCL_GEMM_VERBOSE"))
         std::fprintf(stderr, "ccl_gemm plan: %lld x %lld x %lld batch %lld -> %d CTA(s) per tile, tile width %d, %d K split(s)%s, modelled %.0f cycles\n",
