@@ -1240,7 +1240,7 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
         // benchmark GEMMs: 2-3 % more time, for the two CTA pairs the equal groups leave out).  CCL_GEMM_BALANCED=1 turns it
         // on wherever it is legal.
         if (best_bal > 0 && want == 1) { ctas = bc; bn = bb; splits = 1; balanced = true; best = best_bal; }
-        (void)bal_rounds;
+        (void)bal_rounds;                                   // (kept in the model for the record)
     }
     if (std::getenv("CCL_GEMM_VERBOSE"))
         std::fprintf(stderr, "ccl_gemm plan: %lld x %lld x %lld batch %lld -> %d CTA(s) per tile, tile width %d, %d K split(s)%s, modelled %.0f cycles\n",
