@@ -350,7 +350,8 @@ def by_config(ccl, torch, descs, devb, peaks, P, page, uuid):
     Qwen FFN GEMMs (forward, data and weight gradients), the Llama backward GEMMs and the weight-streaming rows
     (M = 1, 16, 128) of the token sweep on both Llama weights.  B and C in CCL (P strips aligned to the page size),
     grouped raster.  Each figure: CUDA events around back-to-back launches on one stream (100 for kernels under a
-    millisecond, 10 above), operands rotated through enough copies to exceed the L2 where one set would fit in it.
+    millisecond, queued behind a device-side spin so that the host's issue rate does not show; 10 above), operands
+    rotated through enough copies to exceed the L2 where one set would fit in it.
     roofline_frac = time at min(tensor, HBM) roofline / measured time, against the measured burst peaks."""
     from paper_2606_11718_b200 import synth
     L2_BYTES = 126e6
@@ -388,7 +389,10 @@ def by_config(ccl, torch, descs, devb, peaks, P, page, uuid):
         for i in range(3):
             ccl.ccl_gemm(gd, *sets[i % copies], ws)
         e0, e1 = ev(), ev()
-        e0.record()
+        torch.cuda.synchronize()
+        if n == 100:
+            torch.cuda._sleep(6_000_000)           # ~3 ms of device-side spin: the launches queue up behind it, so a kernel of
+        e0.record()                                # a few microseconds is timed on the device, not at the host's issue rate
         for i in range(n):
             ccl.ccl_gemm(gd, *sets[i % copies], ws)
         e1.record()
@@ -409,6 +413,9 @@ def by_config(ccl, torch, descs, devb, peaks, P, page, uuid):
         for i in range(3):
             ccl.ccl_repack(m, srcs[i % copies], dsts[i % copies], 0)
         e0, e1 = ev(), ev()
+        torch.cuda.synchronize()
+        if n == 100:
+            torch.cuda._sleep(6_000_000)
         e0.record()
         for i in range(n):
             ccl.ccl_repack(m, srcs[i % copies], dsts[i % copies], 0)

@@ -142,6 +142,9 @@ struct GemmParams {
     // balanced split: the k blocks of the first bal_tiles tiles of a group, laid end to end, are cut into equal shares, one
     // for each of the group's first bal_units units; bal_q / bal_r = quotient and remainder of that division
     int32_t bal, bal_q, bal_r, bal_units, bal_tiles;
+    // cluster split: a cluster of `ks` CTAs computes ONE 128 x BN tile, CTA r of it the r-th kb_per_split k blocks; the
+    // partial sums meet in distributed shared memory (see the epilogue)
+    int32_t ks;
     // "partial sums written" flags, one per (CTA, epilogue warp), behind the partial sums in the workspace; zeroed by a
     // memset node in front of the launch (so a replayed CUDA graph clears them as well) and set to bal_mark by the kernel
     unsigned long long bal_mark;
@@ -413,6 +416,14 @@ struct Scheduler {
         if (RAG == 1 && rag) return get_ragged(it, t);
         if (RAG == 0 && p.bal) return get_balanced<FULL>(it, t);
         t.part = 0; t.round = it;
+        if (RAG == 0 && p.ks) {                           // cluster split: unit = cluster, one tile each
+            if (it > 0) return false;
+            int g = 0, i = unit;
+            if (p.groups > 1) { g = unit / p.sch_per_group; i = unit - g * p.sch_per_group; }
+            t.split = 0; t.e = 0; t.skip = false;
+            coords<FULL>(g, i, t);
+            return true;
+        }
         int g, i;
         if (it < rounds && my_g >= 0) { g = my_g; i = idx + it * upg; }
         else {
@@ -442,7 +453,8 @@ struct Scheduler {
 
 // RAG: 1 = ragged M (ccl_gemm_grouped), 2 = ragged K (ccl_gemm_grouped_k) -- instantiations of their own, so that the tile
 // walk and the k loops of all other calls stay as they are (the extra branches cost 1-1.5 us on a 15-30 us GEMM)
-template <int BN, int CTAS, bool SWIGLU = false, int RAG = 0, bool FULL = true>
+// KS > 0: cluster split along K (CTAS = 1): the KS CTAs of a cluster share one tile
+template <int BN, int CTAS, bool SWIGLU = false, int RAG = 0, bool FULL = true, int KS = 0>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                 const __grid_constant__ CUtensorMap map_c, const __grid_constant__ GemmParams gp) {
@@ -478,6 +490,8 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = CTAS == 2 ? cluster_ctarank() : 0;
     const bool leader = rank == 0;
+    static_assert(KS == 0 || (CTAS == 1 && BN <= 256 && !SWIGLU && RAG == 0 && !FULL), "the cluster split is a plain 1-CTA-per-tile kernel");
+    const uint32_t krank = KS ? cluster_ctarank() : 0;   // cluster split: which part of K this CTA computes
 
     if (threadIdx.x == 0) {
         prefetch_tmap(&map_a);
@@ -521,7 +535,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         for (int e = lo; e < hi; ++e) { rag_prefix[e] = run; run += tiles_of(e); }
         __syncthreads();
     }
-    Scheduler sched(p, (int)(blockIdx.x / CTAS), BM * CTAS, TILE_N, rag_prefix);
+    Scheduler sched(p, (int)(blockIdx.x / (KS ? KS : CTAS)), BM * CTAS, TILE_N, rag_prefix);
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -559,6 +573,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         const bool post_tx = lane == 0 && leader;
         for (int it = 0; ok && sched.template get<RAG, FULL>(it, t); ++it) {
             if (t.skip) continue;
+            if (KS) t.split = (int)krank;
             if (p.wave_ctr && t.round >= 1 && t.round < p.sch_rounds && t.round % p.wave_period == 0) {   // wait (bounded) until every CTA has issued its previous tiles
                 if (lane == 0) {
                     atomicAdd(p.wave_ctr, 1u);
@@ -589,6 +604,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 if (++stage == stages) { stage = 0; phase ^= 1; }
             }
         }
+        if (KS) { __syncwarp(); cluster_sync(); cluster_sync(); }   // the two meetings of the cluster split (see the epilogue)
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (leader CTA only)
         if (lane == 0 && leader) {
@@ -605,6 +621,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             int done = 0;                                   // tiles computed so far (empty tiles of a ragged batch do not count)
             for (int it = 0; ok && sched.template get<RAG, FULL>(it, t); ++it) {
                 if (t.skip) continue;
+                if (KS) t.split = (int)krank;
                 // NSUB == 1: TMEM half (done & 1) is this tile's accumulator, the other half is being drained.
                 // NSUB == 2: both halves belong to this tile; half h may be overwritten once the epilogue
                 //            of the previous tile has drained it.
@@ -662,6 +679,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 }
             }
         }
+        if (KS) { __syncwarp(); cluster_sync(); cluster_sync(); }
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..5)
         const int quad = warp & 3;                       // TMEM lane quadrant this warp may read
@@ -685,7 +703,11 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             int nb = t.n0 + h * SUBN;                    // first (output) column of this sub-tile
             bool ok = h > 0 || mbar_wait_bounded(&tmem_full[acc], acc_phase);   // one "full" barrier per tile
             ok = __all_sync(0xffffffffu, ok);
-            if (!ok) { if (lane == 0) atomicExch(&g_gemm_status, 4); alive = false; break; }
+            if (!ok) {
+                if (lane == 0) atomicExch(&g_gemm_status, 4);
+                if (KS) { cluster_sync(); cluster_sync(); }        // the others are waiting at the cluster's meetings
+                alive = false; break;
+            }
             tc_fence_after();
             const bool bal = RAG == 0 && !SWIGLU && p.bal;
             bool released = false;                                 // the accumulator has been handed back already
@@ -807,6 +829,54 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     }
                     store_packed(pk, c);
                 }
+            } else if (KS > 0) {
+                // Cluster split: the KS CTAs of the cluster hold the partial sums of ONE tile, each over its part of K.  They
+                // are exchanged in distributed shared memory -- no workspace, no second launch: of every 64-column piece,
+                // CTA k of the cluster owns the 4-column groups [k JS, k JS + JS) (JS = 16 / KS); a warp instruction writes
+                // one group of its 32 rows -- 512 contiguous bytes -- into the owner's copy of the operand ring, which all
+                // MMAs are done with by then (first meeting of the cluster); after the second meeting every CTA sums its
+                // column groups over the KS sources in the order of their k ranges (the same bits on every run), rounds
+                // and stores them through C's layout.
+                constexpr int JS = 16 / (KS > 0 ? KS : 1), PP = BN / 64;
+                cluster_sync();
+                float* rbuf = reinterpret_cast<float*>(smem);                       // [source][quarter][piece][group in slice][lane] float4
+#pragma unroll 1
+                for (int c = 0; c < npieces; ++c) {
+                    load_piece(ra, c);
+                    tmem_ld_wait();
+                    tmem_regs_ready(ra);
+                    const uint32_t local = smem_u32(rbuf + ((((size_t)krank * 4 + quad) * PP + c) * JS * 32 + lane) * 4);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const uint32_t remote = map_to_cta(local + (uint32_t)(j % JS) * 512u, (uint32_t)(j / JS));
+                        asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(remote), "r"(ra[4 * j]), "r"(ra[4 * j + 1]),
+                                     "r"(ra[4 * j + 2]), "r"(ra[4 * j + 3]) : "memory");
+                    }
+                }
+                cluster_sync();
+                // (a tile lies inside one strip of C: the columns of a row follow each other from the tile's first column on)
+                const int row = t.m0 + quad * 32 + lane;
+                unsigned short* crow = p.C + c_offset<FULL>(p, min(row, t.m1 - 1), nb) + (int)krank * JS * 4;
+#pragma unroll 1
+                for (int c = 0; c < npieces; ++c)
+#pragma unroll
+                    for (int js = 0; js < JS; js += 2) {           // two 4-column groups = one 16-byte store
+                        float4 a0 = make_float4(0.0f, 0.0f, 0.0f, 0.0f), a1 = a0;
+#pragma unroll
+                        for (int src = 0; src < KS; ++src) {
+                            const float* g0 = rbuf + ((((size_t)src * 4 + quad) * PP + c) * JS * 32 + js * 32 + lane) * 4;
+                            const float4 v0 = *reinterpret_cast<const float4*>(g0), v1 = *reinterpret_cast<const float4*>(g0 + 128);
+                            a0.x += v0.x; a0.y += v0.y; a0.z += v0.z; a0.w += v0.w;
+                            a1.x += v1.x; a1.y += v1.y; a1.z += v1.z; a1.w += v1.w;
+                        }
+                        const int col = nb + c * 64 + ((int)krank * JS + js) * 4;
+                        const __nv_bfloat162 h0 = __floats2bfloat162_rn(a0.x, a0.y), h1 = __floats2bfloat162_rn(a0.z, a0.w);
+                        const __nv_bfloat162 h2 = __floats2bfloat162_rn(a1.x, a1.y), h3 = __floats2bfloat162_rn(a1.z, a1.w);
+                        uint4 o;
+                        o.x = *reinterpret_cast<const uint32_t*>(&h0); o.y = *reinterpret_cast<const uint32_t*>(&h1);
+                        o.z = *reinterpret_cast<const uint32_t*>(&h2); o.w = *reinterpret_cast<const uint32_t*>(&h3);
+                        st_global_v4_if(crow + c * 64 + js * 4, o, row < t.m1 && col < t.n1);
+                    }
             } else if (bal && t.part != 0) {
                 // Balanced split, a tile shared by t.nshare units.  A unit's slot of the workspace holds one CTA's 128 x BN
                 // partial sums as [epilogue warp][64-column piece][16][lane] float4 -- the registers of a piece exactly as
@@ -997,6 +1067,7 @@ struct GemmPlan {
     uint32_t smem_bytes;
     bool lean;                 // no optional feature in use (see FULL)
     unsigned grid;
+    int ks;                    // cluster split along K: CTAs per cluster (0: none)
 };
 
 // How a page-interleaved operand is expressed as a rank-4 tensor map (OpMap::il_mode): 0 = not interleaved,
@@ -1054,8 +1125,11 @@ static ccl_status merge_width(int64_t* cur, int64_t w, const char* dim) {
 // units = schedulable CTAs (1-CTA kernel) or CTA pairs (2-CTA kernel) the device can hold at once
 // cap > 0: a ragged batch -- the tile grid of one problem covers `cap` rows, d->M is the total row count of A and C
 // ragk: a batch with ragged K -- d->K is the total row count of the concatenated A [K x M] and B [K x N]
+static int resident_clusters(int ks, bool have_device);
+
+// have_device: the unit counts come from the current device (else the figures of a B200); plain: no alpha / beta
 static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, const void* A, const void* B, const void* C, int sms, int pairs, GemmPlan* plan,
-                            int64_t cap = 0, bool ragk = false, size_t max_ws = ~(size_t)0) {
+                            int64_t cap = 0, bool ragk = false, size_t max_ws = ~(size_t)0, bool have_device = false, bool plain = true) {
     if (!d) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: NULL descriptor");
     if (d->M <= 0 || d->N <= 0 || d->K <= 0) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: M, N, K must be positive");
     if (d->M >= (INT64_C(1) << 31) || d->N >= (INT64_C(1) << 31) || d->K >= (INT64_C(1) << 31)) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: dimension too large");
@@ -1242,9 +1316,38 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
         if (best_bal > 0 && want == 1) { ctas = bc; bn = bb; splits = 1; balanced = true; best = best_bal; }
         (void)bal_rounds;                                   // (kept in the model for the record)
     }
+    // Cluster split: a problem of few tiles and a long K -- fewer tiles than a fraction of the SMs -- is split along K
+    // inside a cluster of 2, 4 or 8 CTAs per 128 x BN tile, the partial sums meeting in distributed shared memory: no
+    // workspace, no second launch.  Plain calls only (no batch, activation, alpha / beta, page-interleaved or K-split
+    // operand); CCL_GEMM_CLUSTERK = 0 turns it off, = 2|4|8 forces the cluster size.
+    int ks = 0;
+    {
+        const char* force_ks = std::getenv("CCL_GEMM_CLUSTERK");
+        const int want_ks = force_ks ? atoi(force_ks) : -1;
+        const bool can = want_ks != 0 && plain && batch == 1 && !swiglu && cap == 0 && !ragk && !il_a && !il_b && !il_c && !ka && !kb &&
+                         !(force_split && atoi(force_split) > 1) && !balanced && !(force_ctas && atoi(force_ctas) != 1) && d->out_part != CCL_PART_2D;
+        double best_ks = -1.0;
+        int kb_ = 0, kk = 0;
+        for (int b : {256, 192, 128}) {
+            if (!can) break;
+            if (b == 192 && no_192) continue;
+            if (force_bn && atoi(force_bn) != b) continue;
+            const int64_t tiles = strips_m * ((Wm + BM - 1) / BM) * strips_n * ((Wn + b - 1) / b);
+            for (int k : {2, 4, 8}) {
+                if (want_ks > 0 && want_ks != k) continue;
+                if (tiles > resident_clusters(k, have_device) || tiles * k > sms) continue;
+                const int64_t kbps = (num_kb + k - 1) / k;
+                if ((num_kb + kbps - 1) / kbps != k || kbps < 2) continue;           // every CTA of the cluster owns k blocks
+                const double t_kb = b == 256 ? 680.0 : 570.0;
+                const double cost = (double)kbps * t_kb + 1500.0 + 3500.0 + 3000.0;    // drain, the exchange and its two meetings, launch
+                if (best_ks < 0 || cost < best_ks) { best_ks = cost; kb_ = b; kk = k; }
+            }
+        }
+        if (best_ks > 0 && (want_ks > 0 || best_ks < 0.85 * best)) { ctas = 1; bn = kb_; splits = 1; ks = kk; best = best_ks; }
+    }
     if (std::getenv("CCL_GEMM_VERBOSE"))
         std::fprintf(stderr, "ccl_gemm plan: %lld x %lld x %lld batch %lld -> %d CTA(s) per tile, tile width %d, %d K split(s)%s, modelled %.0f cycles\n",
-                     (long long)d->M, (long long)d->N, (long long)d->K, (long long)batch, ctas, bn, splits, balanced ? ", balanced split" : "", best);
+                     (long long)d->M, (long long)d->N, (long long)d->K, (long long)batch, ctas, bn, splits, balanced ? ", balanced split" : (ks ? ", cluster split along K" : ""), best);
     const int subn = bn > 256 ? 256 : bn;                // columns of one MMA / one TMEM accumulator
     plan->subn = subn;
     const int bm = BM * ctas;
@@ -1319,6 +1422,12 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
             plan->ws_bytes = (size_t)plan->grid * 2 * ((size_t)BM * bn * 4 + 32);   // two slots of partial sums per CTA, then a flag per slot and epilogue warp
         }
     }
+    if (ks) {                                            // cluster split: one cluster per tile, every CTA a part of K
+        p.ks = ks; p.kb_per_split = (int32_t)((num_kb + ks - 1) / ks);
+        plan->grid = (unsigned)(ntiles * ks);
+        p.sch_units = (int32_t)ntiles;
+    }
+    plan->ks = ks;
     p.fd_num_kb = make_fastdiv(p.num_kb);
     // Raster panel height: the units of a group that run at the same time cover `panel` m-tiles by
     // ceil(upg / panel) n-tiles; all groups walk the same m-panel.  The operand rows + columns such a wave
@@ -1380,19 +1489,19 @@ static ccl_status operand_tmap(CUtensorMap* m, const MatView& v, const void* bas
     return encode_tmap(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, base, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
-template <int BN, int CTAS, bool SWIGLU = false, int RAG = 0, bool FULL = true>
+template <int BN, int CTAS, bool SWIGLU = false, int RAG = 0, bool FULL = true, int KS = 0>
 static ccl_status configure(uint32_t smem_bytes) {
     static uint32_t configured_for = 0;
     if (configured_for < smem_bytes) {
-        CCL_CUDA_TRY(cudaFuncSetAttribute(ccl_gemm_kernel<BN, CTAS, SWIGLU, RAG, FULL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes));
+        CCL_CUDA_TRY(cudaFuncSetAttribute(ccl_gemm_kernel<BN, CTAS, SWIGLU, RAG, FULL, KS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes));
         configured_for = smem_bytes;
     }
     return CCL_OK;
 }
 
-template <int BN, int CTAS, bool SWIGLU = false, int RAG = 0, bool FULL = true>
+template <int BN, int CTAS, bool SWIGLU = false, int RAG = 0, bool FULL = true, int KS = 0>
 static ccl_status launch(const GemmPlan& plan, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, cudaStream_t st) {
-    ccl_status s = configure<BN, CTAS, SWIGLU, RAG, FULL>(plan.smem_bytes);
+    ccl_status s = configure<BN, CTAS, SWIGLU, RAG, FULL, KS>(plan.smem_bytes);
     if (s) return s;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(plan.grid, 1, 1);
@@ -1401,7 +1510,7 @@ static ccl_status launch(const GemmPlan& plan, const CUtensorMap& ma, const CUte
     cfg.stream = st;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = CTAS; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[0].val.clusterDim.x = KS ? KS : CTAS; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     // Programmatic dependent launch (CCL_GEMM_PDL=0 turns it off): this kernel's CTAs may be placed, and run their set-up
@@ -1413,7 +1522,7 @@ static ccl_status launch(const GemmPlan& plan, const CUtensorMap& ma, const CUte
         attr[1].val.programmaticStreamSerializationAllowed = 1;
         cfg.numAttrs = 2;
     }
-    CCL_CUDA_TRY(cudaLaunchKernelEx(&cfg, ccl_gemm_kernel<BN, CTAS, SWIGLU, RAG, FULL>, ma, mb, mc, plan.p));
+    CCL_CUDA_TRY(cudaLaunchKernelEx(&cfg, ccl_gemm_kernel<BN, CTAS, SWIGLU, RAG, FULL, KS>, ma, mb, mc, plan.p));
     count_launch();
     return CCL_OK;
 }
@@ -1433,6 +1542,30 @@ static int resident_pairs() {
     int n = 0;
     if (cudaOccupancyMaxActiveClusters(&n, ccl_gemm_kernel<256, 2>, &cfg) != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
     return pairs = n;
+}
+
+// Clusters of `ks` CTAs of the cluster-split kernel that can be resident at once (a tile per cluster); the figures of a
+// B200 (16 clusters of 8, 32 of 4, 64 of 2: clusters do not span GPCs) when no device can be asked.
+template <int KS>
+static int query_clusters() {
+    uint32_t smem = kSmemBudget + kEpiBytes + 2048;
+    if (configure<256, 1, false, 0, false, KS>(smem) != CCL_OK) { clear_error(); return 0; }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(KS, 1, 1); cfg.blockDim = dim3(kGemmThreads, 1, 1); cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = KS; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, ccl_gemm_kernel<256, 1, false, 0, false, KS>, &cfg) != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
+    return n;
+}
+static int resident_clusters(int ks, bool have_device) {
+    static int cached[3] = {-1, -1, -1};
+    const int i = ks == 2 ? 0 : (ks == 4 ? 1 : 2);
+    if (!have_device) return ks == 2 ? 64 : (ks == 4 ? 32 : 16);
+    if (cached[i] < 0) cached[i] = ks == 2 ? query_clusters<2>() : (ks == 4 ? query_clusters<4>() : query_clusters<8>());
+    return cached[i];
 }
 
 ccl_status repack_status_take(int* code);   // ccl_repack.cu
@@ -1496,7 +1629,7 @@ static void make_key(const ccl_gemm_desc* d, const int64_t* batch4, const void* 
     k->dev = -1;
     (void)cudaGetDevice(&k->dev);
     size_t pos = 0;
-    for (const char* name : {"CCL_GEMM_CTAS", "CCL_GEMM_BN", "CCL_GEMM_SPLITK", "CCL_GEMM_RAGGED_DENSE", "CCL_GEMM_BALANCED"}) {
+    for (const char* name : {"CCL_GEMM_CTAS", "CCL_GEMM_BN", "CCL_GEMM_SPLITK", "CCL_GEMM_RAGGED_DENSE", "CCL_GEMM_BALANCED", "CCL_GEMM_CLUSTERK"}) {
         const char* v = std::getenv(name);
         for (const char* c = v ? v : ""; *c && pos + 2 < sizeof(k->env); ++c) k->env[pos++] = *c;
         if (pos + 1 < sizeof(k->env)) k->env[pos++] = ';';
@@ -1505,14 +1638,15 @@ static void make_key(const ccl_gemm_desc* d, const int64_t* batch4, const void* 
 
 // SM count and resident CTA pairs of the current device; the figures of a B200 when no device is usable
 // (the planner then still validates and sizes the workspace the same way a B200 would).
-static void device_units(int* sms, int* pairs) {
+static bool device_units(int* sms, int* pairs) {
     int dev = 0, n = 0;
     if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) {
         *sms = n; *pairs = resident_pairs();
-    } else {
-        (void)cudaGetLastError();
-        *sms = 148; *pairs = 74;
+        return true;
     }
+    (void)cudaGetLastError();
+    *sms = 148; *pairs = 74;
+    return false;
 }
 
 constexpr int64_t kMaxBatch = 65536;
@@ -1524,8 +1658,8 @@ static ccl_status workspace_impl(const ccl_gemm_desc* d, int64_t batch, size_t* 
     if (s) return s;
     if (!bytes) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm_workspace: NULL output");
     int sms, pairs;
-    device_units(&sms, &pairs);
-    if ((s = make_plan(d, batch, false, nullptr, nullptr, nullptr, sms, pairs, &plan))) return s;
+    const bool have_device = device_units(&sms, &pairs);
+    if ((s = make_plan(d, batch, false, nullptr, nullptr, nullptr, sms, pairs, &plan, 0, false, ~(size_t)0, have_device))) return s;
     *bytes = plan.ws_bytes;
     return CCL_OK;
 }
@@ -1611,7 +1745,8 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
             key.mode = (swiglu ? 1 : 0) | (static_ws ? 2 : 0); key.alpha = alpha; key.beta = beta; key.f[38] = (int64_t)max_ws;
             key.f[36] = (int64_t)reinterpret_cast<uintptr_t>(m_offs) ^ ((int64_t)reinterpret_cast<uintptr_t>(k_offs) << 1); key.f[37] = cap + (k_offs ? (INT64_C(1) << 62) : 0);
         }
-        if ((s = make_plan(d, batch, swiglu, A_dev, B_dev, C_dev, prep.sms, resident_pairs(), &plan, cap, k_offs != nullptr, max_ws))) return s;
+        if ((s = make_plan(d, batch, swiglu, A_dev, B_dev, C_dev, prep.sms, resident_pairs(), &plan, cap, k_offs != nullptr, max_ws, true,
+                           alpha == 1.0f && beta == 0.0f))) return s;
         plan.p.C = static_cast<uint16_t*>(C_dev);
         plan.p.a.batched = batch4[1] != 0; plan.p.b.batched = batch4[2] != 0; plan.p.c.batched = m_offs ? 0 : 1;
         plan.p.m_offs = m_offs;
@@ -1704,7 +1839,18 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
         else if (plan.bn == 192) s = launch<192, 1, false, 1>(plan, ma, mb, mc, st);
         else s = launch<128, 1, false, 1>(plan, ma, mb, mc, st);
     } else if (swiglu) s = launch<512, 2, true>(plan, ma, mb, mc, st);
-    else if (plan.lean) {                                // nothing optional in use: the instantiation without those branches
+    else if (plan.ks) {                                  // cluster split along K (plain calls only)
+        const int key = plan.bn * 10 + plan.ks;
+        if (key == 2562) s = launch<256, 1, false, 0, false, 2>(plan, ma, mb, mc, st);
+        else if (key == 2564) s = launch<256, 1, false, 0, false, 4>(plan, ma, mb, mc, st);
+        else if (key == 2568) s = launch<256, 1, false, 0, false, 8>(plan, ma, mb, mc, st);
+        else if (key == 1922) s = launch<192, 1, false, 0, false, 2>(plan, ma, mb, mc, st);
+        else if (key == 1924) s = launch<192, 1, false, 0, false, 4>(plan, ma, mb, mc, st);
+        else if (key == 1928) s = launch<192, 1, false, 0, false, 8>(plan, ma, mb, mc, st);
+        else if (key == 1282) s = launch<128, 1, false, 0, false, 2>(plan, ma, mb, mc, st);
+        else if (key == 1284) s = launch<128, 1, false, 0, false, 4>(plan, ma, mb, mc, st);
+        else s = launch<128, 1, false, 0, false, 8>(plan, ma, mb, mc, st);
+    } else if (plan.lean) {                                // nothing optional in use: the instantiation without those branches
         if (plan.ctas == 2) {
             if (plan.bn == 512) s = launch<512, 2, false, 0, false>(plan, ma, mb, mc, st);
             else if (plan.bn == 192) s = launch<192, 2, false, 0, false>(plan, ma, mb, mc, st);

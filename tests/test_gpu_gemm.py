@@ -506,3 +506,41 @@ def test_gemm_balanced_split_needs_its_workspace_or_steps_aside(balanced):
         g = synth.from_bits(from_layout(c_dev, d.C)).to(torch.float32).numpy()
         err = np.abs(g - ref32) / np.maximum(1.0, np.abs(ref32))
         assert err.max() <= tol(K)
+
+
+# ---------------------------------------------------------------------------------------------
+# cluster split: the CTAs of a cluster share one tile along K, partial sums meet in distributed shared memory
+# ---------------------------------------------------------------------------------------------
+CLUSTERK = [
+    # M, N, K, P, layouts, a_trans, b_trans, out_part
+    (256, 768, 2048, 4, ("row", "ccl", "ccl"), 0, 1, 2),       # the single-expert GEMM (configuration 1)
+    (256, 768, 2048, 4, ("row", "ccl", "ccl"), 0, 0, 2),       # ... with the weight materialised [K x N]: strips of 192 columns
+    (768, 2048, 4096, 4, ("row", "ccl", "ccl"), 1, 0, 2),      # the Qwen down-projection weight gradient
+    (130, 384, 1096, 2, ("row", "ccl", "ccl"), 0, 0, 2),       # ragged rows, K not a multiple of 64
+    (304, 520, 512, 1, ("row", "row", "row"), 1, 1, 0),        # ragged columns, plain raster, both operands transposed
+    (512, 512, 8192, 4, ("ccl", "row", "ccl"), 0, 0, 1),       # M strips
+    (1, 1024, 4096, 4, ("row", "ccl", "ccl"), 0, 0, 2),        # one row
+]
+
+
+@pytest.mark.parametrize("M,N,K,P,lay,at,bt,op", CLUSTERK)
+@pytest.mark.parametrize("ks", [2, 4, 8])
+@pytest.mark.parametrize("bn", [None, 128, 192, 256])
+def test_gemm_cluster_split(M, N, K, P, lay, at, bt, op, ks, bn):
+    """The cluster split forced on (cluster size and tile width): parity with the oracle, the same bits on every run."""
+    keys = ("CCL_GEMM_CLUSTERK", "CCL_GEMM_BN")
+    old = {k: os.environ.pop(k, None) for k in keys}
+    os.environ["CCL_GEMM_CLUSTERK"] = str(ks)
+    if bn is not None:
+        os.environ["CCL_GEMM_BN"] = str(bn)
+    try:
+        A, B = synth.gemm_operands(M, N, K, at, bt, seed=9, tag="clusterk")
+        d = gemm_desc(M, N, K, P, lay, at, bt, op, 1)
+        got1, _ = check(d, A, B)
+        got2, _ = check(d, A, B)
+        np.testing.assert_array_equal(got1, got2)
+    finally:
+        for k in keys:
+            os.environ.pop(k, None)
+            if old[k] is not None:
+                os.environ[k] = old[k]
