@@ -86,9 +86,13 @@ struct OpMap {          // how stored coordinates (r, c) of an operand become te
     //   il_mode 1: a chunk holds il_kr whole strip rows  -> map {x, row % kr, strip, row / kr}
     //   il_mode 2: a strip row spans whole chunks        -> map {x % sc, x / sc, row, strip}
     //   il_mode 0: strips stored one after the other     -> map {x, row, strip, 1}
+    //   il_mode 3: neither (e.g. strip rows of 3.5 chunks): no affine box exists; a 64-element piece of a row at a
+    //              64-aligned column is still contiguous, so the buffer is mapped as 128-byte lines {64, line} and a tile is
+    //              fetched row by row (see line_of())
     int32_t il_mode;
     FastDiv il_kr, il_sc;
     int32_t batched;    // 1: each problem of a batch has its own buffer, 0: all problems share this operand
+    int32_t rows, cols, roww, nstrips, lines;   // il_mode 3: stored shape, elements of a strip row, strips, 128-byte lines of the buffer
 };
 
 struct GemmParams {
@@ -272,6 +276,18 @@ __device__ __forceinline__ void to_coords(const OpMap& o, int r, int c, int& x, 
     else if (FULL && o.il_mode == 2) { o.il_sc.divmod(xx, y, x); z = rr; u = g; }
     else { x = xx; y = rr; z = g; u = 0; }
 }
+// il_mode 3: the 128-byte line of the buffer that holds the 64 elements from stored (r, c) on, c a multiple of 64; a piece
+// outside the matrix gets a line past the end of the tensor map, which the copy engine fills with zeros.
+__device__ __forceinline__ int line_of(const OpMap& o, int r, int c) {
+    if (r >= o.rows || c >= o.cols) return o.lines;
+    int g = 0, rr = r, xx = c;
+    if (o.split == 2) o.w.divmod(c, g, xx);
+    else if (o.split == 1) o.h.divmod(r, g, rr);
+    const int e = rr * o.roww + xx;                  // element of the strip's packed contents (< 2^31: checked on the host)
+    int j, x;
+    o.il_sc.divmod(e, j, x);
+    return (int)((((int64_t)j * o.nstrips + g) * (int64_t)o.il_sc.d + x) >> 6);
+}
 // Element offset of C[m][n] in its buffer (any layout).
 template <bool FULL = true>
 __device__ __forceinline__ int64_t c_offset(const GemmParams& p, int64_t m, int64_t n) {
@@ -283,6 +299,11 @@ __device__ __forceinline__ int64_t c_offset(const GemmParams& p, int64_t m, int6
         int j, y;
         p.c.il_kr.divmod(rr, j, y);
         return ((int64_t)j * p.c_nstrips + g) * p.c_ichunk + (int64_t)y * p.c_row + xx;
+    }
+    if (FULL && p.c.il_mode == 3) {                  // chunks and strip rows do not line up: the general form
+        int j, x;
+        p.c.il_sc.divmod(rr * p.c.roww + xx, j, x);
+        return ((int64_t)j * p.c_nstrips + g) * p.c_ichunk + x;
     }
     if (FULL && p.c.il_mode == 2) {                  // a strip row spans c_cpr whole chunks
         int cj, x;
@@ -555,6 +576,8 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         // operand is split along K itself (rare) only that coordinate changes from one k block to the next
         // (a page-interleaved operand recomputes its coordinates every k block as well)
         const bool ksplit = FULL && ((mn ? om.split == 1 : om.split == 2) || om.il_mode != 0);
+        const bool gather_a = FULL && p.a.il_mode == 3, gather_b = FULL && p.b.il_mode == 3;
+        const bool box = active && !(isA ? gather_a : gather_b);     // this lane issues one box per stage
         uint32_t soff;                                        // byte offset of the box inside a stage
         int off;                                              // offset of the box along M (A) or N (B) from the tile origin
         int hsel = 0;                                         // sub-tile of a B box
@@ -600,7 +623,35 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 const int k0 = kbase + kb * BK;
                 if (ksplit) { if (mn) to_coords<FULL>(om, k0, base, x, y, z, u); else to_coords<FULL>(om, base, k0, x, y, z, u); }
                 else if (mn) y = k0; else x = k0;
-                if (active) tma_load<CTAS>(smem + (size_t)stage * stage_bytes + soff, map, full0 + (uint32_t)stage * 8u, x, y, z, u, t.e * om.batched);
+                if (box) tma_load<CTAS>(smem + (size_t)stage * stage_bytes + soff, map, full0 + (uint32_t)stage * 8u, x, y, z, u, t.e * om.batched);
+                if (FULL && (gather_a || gather_b)) {
+                    // An operand whose chunks and strip rows do not line up: its part of the stage is fetched as single
+                    // 128-byte rows (the swizzle is a function of the shared-memory address, so the rows land exactly
+                    // where a box would have put them), the 32 lanes taking turns.
+                    unsigned char* st0 = smem + (size_t)stage * stage_bytes;
+                    const uint32_t bar = full0 + (uint32_t)stage * 8u;
+                    if (gather_a)
+                        for (int i = lane; i < BM; i += 32) {
+                            int r, c; uint32_t so;
+                            if (p.a_mn) { const int ch = i >> 6, kr = i & 63; r = k0 + kr; c = t.m0 + (int)rank * BM + 64 * ch; so = (uint32_t)(ch * 64 * BK * 2 + kr * 128); }
+                            else { r = t.m0 + (int)rank * BM + i; c = k0; so = (uint32_t)i * 128u; }
+                            tma_load<CTAS>(st0 + so, &map_a, bar, 0, line_of(p.a, r, c), 0, 0, 0);
+                        }
+                    if (gather_b)
+                        for (int i = lane; i < NSUB * SUBH; i += 32) {
+                            int r, c; uint32_t so;
+                            if (p.b_mn) {
+                                const int ch = i >> 6, kr = i & 63, h = ch / NC, cc = ch - h * NC;
+                                r = k0 + kr; c = t.n0 + h * SUBN + (int)rank * SUBH + 64 * cc;
+                                so = p.a_bytes + (uint32_t)(h * SUBH * BK * 2 + cc * 64 * BK * 2 + kr * 128);
+                            } else {
+                                const int h = i / SUBH, rr = i - h * SUBH;
+                                r = t.n0 + h * SUBN + (int)rank * SUBH + rr; c = k0;
+                                so = p.a_bytes + (uint32_t)(h * SUBH * BK * 2 + rr * 128);
+                            }
+                            tma_load<CTAS>(st0 + so, &map_b, bar, 0, line_of(p.b, r, c), 0, 0, 0);
+                        }
+                }
                 if (++stage == stages) { stage = 0; phase ^= 1; }
             }
         }
@@ -736,7 +787,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             };
             auto store_packed = [&](const uint32_t (&pk)[32], int c) {
                 const int n64 = nb + c * 64;
-                if (rows_full && n64 + 64 <= t.n1) {
+                if (rows_full && n64 + 64 <= t.n1 && !(FULL && p.c.il_mode == 3)) {
                     // staging: 32 KB in all -- two buffers per warp with four warps, one with eight
                     unsigned char* buf = epi + (size_t)(EW == 1 ? (warp - 2) * 2 + (epi_count & 1) : (warp - 2)) * (32 * 128);
                     if (epi_count >= 2 / EW) { if (lane == 0) tma_store_wait_read<2 / EW - 1>(); __syncwarp(); }   // buffer free again
@@ -872,6 +923,14 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                             a1.x += v1.x; a1.y += v1.y; a1.z += v1.z; a1.w += v1.w;
                         }
                         const int col = nb + c * 64 + ((int)krank * JS + js) * 4;
+                        if (p.axpby) {                             // C <- alpha * sum + beta * C (C read through its own layout)
+                            const uint4 cv = ld_global_v4_if(crow + c * 64 + js * 4, p.beta != 0.0f && row < t.m1 && col < t.n1);
+                            const float al = p.alpha, be = p.beta;
+                            a0.x = fmaf(al, a0.x, be * __uint_as_float(cv.x << 16)); a0.y = fmaf(al, a0.y, be * __uint_as_float(cv.x & 0xFFFF0000u));
+                            a0.z = fmaf(al, a0.z, be * __uint_as_float(cv.y << 16)); a0.w = fmaf(al, a0.w, be * __uint_as_float(cv.y & 0xFFFF0000u));
+                            a1.x = fmaf(al, a1.x, be * __uint_as_float(cv.z << 16)); a1.y = fmaf(al, a1.y, be * __uint_as_float(cv.z & 0xFFFF0000u));
+                            a1.z = fmaf(al, a1.z, be * __uint_as_float(cv.w << 16)); a1.w = fmaf(al, a1.w, be * __uint_as_float(cv.w & 0xFFFF0000u));
+                        }
                         const __nv_bfloat162 h0 = __floats2bfloat162_rn(a0.x, a0.y), h1 = __floats2bfloat162_rn(a0.z, a0.w);
                         const __nv_bfloat162 h2 = __floats2bfloat162_rn(a1.x, a1.y), h3 = __floats2bfloat162_rn(a1.z, a1.w);
                         uint4 o;
@@ -1080,11 +1139,12 @@ static int interleave_mode(const MatView& v, int64_t* kr) {
     const int64_t row = v.split == 2 ? v.w : v.cols;
     if (v.ichunk % row == 0) { *kr = v.ichunk / row; return 1; }
     if (row % v.ichunk == 0 && v.ichunk % 64 == 0) return 2;
+    if (row % 64 == 0 && v.ichunk % 64 == 0) return 3;      // no affine box, but every 128-byte piece of a row lies inside one chunk
     return -1;
 }
 
 // k_along_rows: the GEMM's K dimension runs along the stored rows of this operand (never for C)
-static ccl_status check_operand(const MatView& v, const void* ptr, const char* name, bool k_along_rows, int64_t K) {
+static ccl_status check_operand(const MatView& v, const void* ptr, const char* name, bool k_along_rows, int64_t K, bool is_c = false) {
     if (v.e != 2) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: %s: only 2-byte (bf16) elements are supported", name);
     if (ragged(v)) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: %s: strips of unequal size (the split dimension is not a multiple of P) are not supported", name);
     int64_t inner = v.split == 2 ? v.w : v.cols;
@@ -1094,7 +1154,15 @@ static ccl_status check_operand(const MatView& v, const void* ptr, const char* n
         const int mode = interleave_mode(v, &kr);
         if (mode < 0)
             return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: %s: page-interleaved layout: a chunk (%lld elements) must hold whole strip rows (%lld elements), "
-                        "or a strip row whole chunks of a multiple of 64 elements", name, (long long)v.ichunk, (long long)inner);
+                        "or a strip row whole chunks of a multiple of 64 elements, or both must be multiples of 64 elements", name, (long long)v.ichunk, (long long)inner);
+        if (mode == 3) {                     // fetched row by row (see line_of): what that path assumes
+            if (k_along_rows ? v.split == 1 : (v.split == 2 && !is_c))
+                return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: %s: a page-interleaved operand whose chunks and strip rows do not line up must not be split along K", name);
+            if (!k_along_rows && !is_c && K % BK)
+                return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: %s: page-interleaved layout: K (%lld) must be a multiple of %d when chunks and strip rows do not line up", name, (long long)K, BK);
+            if ((double)(v.split == 1 ? v.h : v.rows) * (double)inner >= 2147483648.0 || buffer_elems(v) / 64 >= (INT64_C(1) << 31))
+                return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: %s: strip too large for the row-by-row path", name);
+        }
         if (mode == 1 && (kr & (kr - 1)))
             return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: %s: page-interleaved layout: %lld strip rows per chunk is not a power of two", name, (long long)kr);
         const int64_t R = v.split == 1 ? v.h : v.rows;
@@ -1129,9 +1197,9 @@ static ccl_status merge_width(int64_t* cur, int64_t w, const char* dim) {
 // ragk: a batch with ragged K -- d->K is the total row count of the concatenated A [K x M] and B [K x N]
 static int resident_clusters(int ks, bool have_device);
 
-// have_device: the unit counts come from the current device (else the figures of a B200); plain: no alpha / beta
+// have_device: the unit counts come from the current device (else the figures of a B200)
 static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, const void* A, const void* B, const void* C, int sms, int pairs, GemmPlan* plan,
-                            int64_t cap = 0, bool ragk = false, size_t max_ws = ~(size_t)0, bool have_device = false, bool plain = true) {
+                            int64_t cap = 0, bool ragk = false, size_t max_ws = ~(size_t)0, bool have_device = false) {
     if (!d) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: NULL descriptor");
     if (d->M <= 0 || d->N <= 0 || d->K <= 0) return fail(CCL_ERR_INVALID_ARG, "ccl_gemm: M, N, K must be positive");
     if (d->M >= (INT64_C(1) << 31) || d->N >= (INT64_C(1) << 31) || d->K >= (INT64_C(1) << 31)) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: dimension too large");
@@ -1154,9 +1222,11 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
         return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm_swiglu: page-interleaved operands are not supported");
     if ((s = check_operand(va, A, "A", at, d->K))) return s;
     if ((s = check_operand(vb, B, "B", !bt, d->K))) return s;
-    if ((s = check_operand(vc, C, "C", false, d->K))) return s;
+    if ((s = check_operand(vc, C, "C", false, d->K, true))) return s;
     int64_t kr_a, kr_b, kr_c;
     const int il_a = interleave_mode(va, &kr_a), il_b = interleave_mode(vb, &kr_b), il_c = interleave_mode(vc, &kr_c);
+    if ((il_a == 3 || il_b == 3 || il_c == 3) && (batch > 1 || cap > 0 || ragk))
+        return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: a batch with a page-interleaved operand whose chunks and strip rows do not line up is not supported");
     // a 192-row (96-row for a CTA pair) box of a K-contiguous B cannot be cut into chunks of more than 64 (32) rows
     const bool no_192 = il_b == 1 && bt && kr_b > 64, no_192_pair = il_b == 1 && bt && kr_b > 32;
 
@@ -1320,13 +1390,12 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     }
     // Cluster split: a problem of few tiles and a long K -- fewer tiles than a fraction of the SMs -- is split along K
     // inside a cluster of 2, 4 or 8 CTAs per 128 x BN tile, the partial sums meeting in distributed shared memory: no
-    // workspace, no second launch.  Plain calls only (no batch, activation, alpha / beta, page-interleaved or K-split
-    // operand); CCL_GEMM_CLUSTERK = 0 turns it off, = 2|4|8 forces the cluster size.
+    // workspace, no second launch.  No batch, fused activation, page-interleaved or K-split operand; CCL_GEMM_CLUSTERK = 0 turns it off, = 2|4|8 forces the cluster size.
     int ks = 0;
     {
         const char* force_ks = std::getenv("CCL_GEMM_CLUSTERK");
         const int want_ks = force_ks ? atoi(force_ks) : -1;
-        const bool can = want_ks != 0 && plain && batch == 1 && !swiglu && cap == 0 && !ragk && !il_a && !il_b && !il_c && !ka && !kb &&
+        const bool can = want_ks != 0 && batch == 1 && !swiglu && cap == 0 && !ragk && !il_a && !il_b && !il_c && !ka && !kb &&
                          !(force_split && atoi(force_split) > 1) && !balanced && !(force_ctas && atoi(force_ctas) != 1) && d->out_part != CCL_PART_2D;
         double best_ks = -1.0;
         int kb_ = 0, kk = 0;
@@ -1373,6 +1442,15 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     p.b.il_mode = il_b; p.b.il_kr = make_fastdiv(kr_b); p.b.il_sc = make_fastdiv(vb.ichunk);
     p.c.split = vc.split; p.c.w = make_fastdiv(vc.w); p.c.h = make_fastdiv(vc.h);
     p.c.il_mode = il_c; p.c.il_kr = make_fastdiv(kr_c); p.c.il_sc = make_fastdiv(vc.ichunk);
+    {
+        const MatView* vs[3] = {&va, &vb, &vc};
+        OpMap* os[3] = {&p.a, &p.b, &p.c};
+        for (int X = 0; X < 3; ++X) {
+            os[X]->rows = (int32_t)vs[X]->rows; os[X]->cols = (int32_t)vs[X]->cols;
+            os[X]->roww = (int32_t)(vs[X]->split == 2 ? vs[X]->w : vs[X]->cols); os[X]->nstrips = (int32_t)vs[X]->nstrips;
+            os[X]->lines = os[X]->il_mode == 3 ? (int32_t)(buffer_elems(*vs[X]) / 64) : 0;
+        }
+    }
     p.c_row = vc.split == 2 ? vc.w : vc.cols; p.c_stride = vc.stride;
     p.c_ichunk = vc.ichunk; p.c_nstrips = vc.nstrips;
     p.c_cpr = il_c == 2 ? (int32_t)(p.c_row / vc.ichunk) : 0;
@@ -1482,6 +1560,10 @@ static ccl_status operand_tmap(CUtensorMap* m, const MatView& v, const void* bas
         dims[0] = sc; dims[1] = row / sc; dims[2] = R; dims[3] = S;
         strides[0] = S * sc * 2; strides[1] = row * S * 2; strides[2] = sc * 2;
         box[0] = box_inner; box[1] = 1; box[2] = box_rows; box[3] = 1;
+    } else if (mode == 3) {                              // the buffer as 128-byte lines, fetched one row of a tile at a time
+        dims[0] = 64; dims[1] = (uint64_t)(buffer_elems(v) / 64); dims[2] = 1; dims[3] = 1; dims[4] = 1;
+        strides[0] = 128; strides[1] = 128; strides[2] = 128;
+        box[0] = 64; box[1] = 1; box[2] = 1; box[3] = 1;
     } else if (mode == 0) {
         dims[0] = row; dims[1] = R; dims[2] = v.split ? S : 1; dims[3] = 1;
         strides[0] = row * 2; strides[1] = v.split ? (uint64_t)v.stride * 2 : row * 2; strides[2] = strides[1];
@@ -1747,8 +1829,7 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
             key.mode = (swiglu ? 1 : 0) | (static_ws ? 2 : 0); key.alpha = alpha; key.beta = beta; key.f[38] = (int64_t)max_ws;
             key.f[36] = (int64_t)reinterpret_cast<uintptr_t>(m_offs) ^ ((int64_t)reinterpret_cast<uintptr_t>(k_offs) << 1); key.f[37] = cap + (k_offs ? (INT64_C(1) << 62) : 0);
         }
-        if ((s = make_plan(d, batch, swiglu, A_dev, B_dev, C_dev, prep.sms, resident_pairs(), &plan, cap, k_offs != nullptr, max_ws, true,
-                           alpha == 1.0f && beta == 0.0f))) return s;
+        if ((s = make_plan(d, batch, swiglu, A_dev, B_dev, C_dev, prep.sms, resident_pairs(), &plan, cap, k_offs != nullptr, max_ws, true))) return s;
         plan.p.C = static_cast<uint16_t*>(C_dev);
         plan.p.a.batched = batch4[1] != 0; plan.p.b.batched = batch4[2] != 0; plan.p.c.batched = m_offs ? 0 : 1;
         plan.p.m_offs = m_offs;

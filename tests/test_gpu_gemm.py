@@ -150,12 +150,21 @@ INTERLEAVED = [
     (16, 1024, 2048, 2, ("row", "ileave", "ileave"), 0, 0, 2, 4096),    # split along K: the reduction writes interleaved C
     (640, 2560, 512, 2, ("row", "ileave", "ileave"), 0, 0, 2, 10240),   # several tiles per CTA group, 4 rows per chunk
     (256, 4096, 512, 4, ("row", "ileave", "ileave"), 0, 0, 2, 4096),    # the common case: 4 KB pages, 2 KB strip rows
+    # chunks and strip rows that do not line up (no affine box: the operand ring is filled row by row)
+    (264, 3584, 512, 4, ("row", "ileave", "ileave"), 0, 0, 2, 4096),    # w = 896: a strip row is 1792 B = 0.4375 chunks
+    (264, 3584, 328, 4, ("row", "ileave", "row"), 0, 0, 2, 4096),       # ... K not a multiple of 64 (K runs along B's rows)
+    (1024, 7168, 256, 8, ("row", "ileave", "ileave"), 0, 0, 2, 1024),   # w = 896 against 512-element chunks, P = 8
+    (300, 1792, 512, 2, ("row", "ileave", "ileave"), 0, 1, 2, 768),     # B stored [N x K]: rows of 512 elements, chunks of 384
+    (768, 512, 320, 2, ("ileave", "row", "ileave"), 1, 0, 1, 640),      # A stored [K x M] split along its columns (w = 384), chunks of 320
+    (1792, 512, 256, 2, ("ileave", "row", "ileave"), 0, 0, 1, 768),     # A [M x K] split along rows: rows of 256, chunks of 384 elements
 ]
 
 
 @pytest.mark.parametrize("M,N,K,P,lay,at,bt,op,chunk", INTERLEAVED)
-def test_gemm_page_interleaved_operands(M, N, K, P, lay, at, bt, op, chunk, cta_mode):
-    """The page-interleaved form of CCL changes the address map only: same bits as from packed CCL operands."""
+def test_gemm_page_interleaved_operands(M, N, K, P, lay, at, bt, op, chunk, cta_mode, monkeypatch):
+    """The page-interleaved form of CCL changes the address map only: same bits as from packed CCL operands (under the
+    same plan: the cluster split, which page-interleaved operands do not take, sums K in another order)."""
+    monkeypatch.setenv("CCL_GEMM_CLUSTERK", "0")
     A, B = synth.gemm_operands(M, N, K, at, bt, seed=5, tag="ileave")
     plain = tuple("ccl" if l == "ileave" else l for l in lay)
     want = run_gemm(gemm_desc(M, N, K, P, plain, at, bt, op, 1), A, B)

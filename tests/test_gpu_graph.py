@@ -29,9 +29,8 @@ def test_step_replays_from_a_cuda_graph():
     c1 = torch.zeros(nc, dtype=torch.bfloat16, device="cuda")
     c2 = torch.zeros(ccl.ccl_buffer_bytes(ds.C) // 2, dtype=torch.bfloat16, device="cuda")
     ck = torch.zeros(ccl.ccl_buffer_bytes(dk.C) // 2, dtype=torch.bfloat16, device="cuda")
-    need = ccl.ccl_gemm_workspace(dk)
-    assert need > 0
-    ws = torch.empty(need // 4, dtype=torch.float32, device="cuda")
+    need = ccl.ccl_gemm_workspace(dk)                      # (a short problem: split along K in one way or another)
+    ws = torch.empty(max(need, 16) // 4, dtype=torch.float32, device="cuda")
     ab = a.repeat(E, 1).contiguous()
     cb = torch.zeros(E * nc, dtype=torch.bfloat16, device="cuda")
     needb = ccl.ccl_gemm_batched_workspace(d, E)
