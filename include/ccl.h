@@ -28,6 +28,8 @@
  *   CCL_GEMM_BN = 128|192|256|512  force the tile width
  *   CCL_GEMM_SPLITK = n            force the number of K splits
  *   CCL_GEMM_BALANCED = 0|1        never / always (where legal) cut the tiles that do not fill a round into equal shares
+ *   CCL_GEMM_CLUSTERK = 0|2|4|8    never / always (where legal) let the CTAs of a cluster of that size share one tile,
+ *                                  each over its own part of K (the default picks it for problems of few tiles)
  *   CCL_GEMM_WAVESYNC = 0|n        soft wave barrier off / every n-th round of tiles
  *   CCL_GEMM_PDL = 0               no programmatic dependent launch
  *   CCL_GEMM_RAGGED_DENSE = 0      ragged batches walk the fixed grid of max_rows per problem
@@ -163,8 +165,11 @@ ccl_status ccl_repack_transpose(const ccl_mat* m, const void* src_dev, void* dst
  * affine box of the buffer: either a chunk holds a power-of-two number of whole strip rows, or a strip row is
  * made of whole chunks of a multiple of 64 elements; the chunk size a multiple of 16 bytes.  (With chunks of
  * whole rows, an operand whose rows run along K must have K a multiple of 64 or rows-per-strip a multiple of
- * the rows per chunk: the padding of a strip's last chunk is not read as zero.)  Other chunkings ->
- * CCL_ERR_UNSUPPORTED.
+ * the rows per chunk: the padding of a strip's last chunk is not read as zero.)  When neither holds but a strip row
+ * and a chunk are both multiples of 64 elements (say rows of 3.5 chunks), every 128-byte piece of a row still lies
+ * inside one chunk and the operand is fetched and written row by row in such pieces -- correct, slower; it then
+ * must not be split along K, an A or B whose rows run along M or N needs K a multiple of 64, and a strip must hold
+ * fewer than 2^31 elements.  Other chunkings -> CCL_ERR_UNSUPPORTED.
  */
 typedef struct ccl_gemm_desc {
     int64_t M, N, K;
@@ -178,7 +183,8 @@ typedef struct ccl_gemm_desc {
 
 /*
  * Bytes of device workspace the preferred plan of this problem uses (0 when none): fp32 partial sums of a problem split
- * along K.  Two kinds of plan use it: the classic split (every tile computed by several units over disjoint k ranges,
+ * along K.  (A problem of few tiles is split inside thread-block clusters instead -- the partial sums meet in the
+ * cluster's shared memory, in a fixed order -- and needs none.)  Two kinds of plan use it: the classic split (every tile computed by several units over disjoint k ranges,
  * summed by a second kernel) INSISTS on it -- ccl_gemm returns CCL_ERR_WORKSPACE without it --, the balanced split
  * (the tiles that do not fill a round of the machine are cut into equal shares of k blocks, one per unit, and reduced
  * inside the kernel, in the order of k: the same bits on every run) is OPTIONAL: given less than it needs, ccl_gemm
@@ -246,8 +252,8 @@ ccl_status ccl_gemm_axpby(const ccl_gemm_desc* d, float alpha, float beta, const
  * projections of a mixture-of-experts FFN (Sec. 4.1 evaluates the Qwen expert GEMMs one at a time; the
  * paper has no batched call: the batch only amortises the launch and fills the machine with small problems).
  * Problem e (0 <= e < batch) reads A_dev + e*a_stride_bytes and B_dev + e*b_stride_bytes and writes
- * C_dev + e*c_stride_bytes, each buffer laid out as `d` says; results are those of `batch` ccl_gemm calls,
- * bit for bit.  A stride of 0 for A or B means every problem shares that operand.  Otherwise a stride must
+ * C_dev + e*c_stride_bytes, each buffer laid out as `d` says; results are those of `batch` ccl_gemm calls
+ * (bit for bit unless one of the two plans splits K, which changes the order of the fp32 sum).  A stride of 0 for A or B means every problem shares that operand.  Otherwise a stride must
  * be a multiple of 16 bytes and at least ccl_buffer_bytes of the operand (CCL_ERR_ALIGN / CCL_ERR_INVALID_ARG);
  * 1 <= batch <= 65536.  With batch = 1 the strides are ignored and the call equals ccl_gemm.
  * Workspace: ccl_gemm_batched_workspace bytes (0 when the plan does not split K).  All buffers are the

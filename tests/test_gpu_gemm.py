@@ -398,6 +398,8 @@ AXPBY = [
     (16, 1024, 2048, 2, ("row", "ccl", "ccl"), 0, 0, 2, 2.0, -0.5),        # split along K: the reduction applies the scalars
     (300, 1024, 256, 4, ("row", "ileave", "ileave"), 0, 0, 2, 0.25, 3.0),  # page-interleaved C
     (640, 2560, 512, 2, ("row", "ccl", "ccl"), 0, 0, 2, 3.0, 0.0),         # beta = 0: C is not read
+    (256, 768, 2048, 4, ("row", "ccl", "ccl"), 0, 1, 2, 0.5, 2.0),         # few tiles: split inside clusters, the owners of the sums apply the scalars
+    (130, 392, 4096, 2, ("row", "ccl", "ccl"), 0, 0, 2, -2.0, 1.0),        # ... with ragged rows and columns
 ]
 
 
