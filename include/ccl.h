@@ -25,7 +25,7 @@
  * Test / diagnostic switches (environment variables, read by the library; none changes a result beyond the
  * rounding order of a split-K sum):
  *   CCL_GEMM_CTAS = 1|2            force one CTA per tile or a cta_group::2 pair
- *   CCL_GEMM_BN = 128|192|256|512  force the tile width
+ *   CCL_GEMM_BN = 128|192|256|384|512  force the tile width
  *   CCL_GEMM_SPLITK = n            force the number of K splits
  *   CCL_GEMM_BALANCED = 0|1        never / always (where legal) cut the tiles that do not fill a round into equal shares
  *   CCL_GEMM_CLUSTERK = 0|2|4|8    never / always (where legal) let the CTAs of a cluster of that size share one tile,

@@ -489,15 +489,23 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         uint32_t* dst = reinterpret_cast<uint32_t*>(&p);
         for (int i = threadIdx.x; i < (int)(sizeof(GemmParams) / 4); i += kGemmThreads) dst[i] = src[i];
     }
-    // A tile wider than 256 columns is computed as NSUB sub-tiles of SUBN columns (one MMA each per
-    // k step) that fill TMEM; narrower tiles use the two 256-column halves of TMEM as a double buffer.
-    constexpr int NSUB = BN > 256 ? BN / 256 : 1;
-    constexpr int SUBN = BN / NSUB;
-    constexpr int ACC_COLS = NSUB == 1 ? 256 : SUBN;  // TMEM columns between accumulators
-    constexpr int NACC = NSUB == 1 ? 2 : NSUB;        // accumulator barriers in use
-    static_assert(!SWIGLU || NSUB == 2, "the gated activation pairs the two accumulators of a wide tile");
+    // A tile wider than 256 columns is computed as two sub-tiles (one MMA each per k step), the first 256 columns wide,
+    // the second the rest (256 or 128), each with a 256-column half of TMEM; narrower tiles use the two halves as a
+    // double buffer.
+    static_assert(BN <= 256 || BN == 384 || BN == 512, "tile widths");
+    constexpr int NSUB = BN > 256 ? 2 : 1;
+    constexpr int SUBN = NSUB == 1 ? BN : 256;        // width of the first sub-tile = columns from one sub-tile to the next
+    constexpr int SUBN1 = NSUB == 1 ? 0 : BN - 256;   // width of the second
+    constexpr int ACC_COLS = 256;                     // TMEM columns between accumulators
+    constexpr int NACC = 2;                           // accumulator barriers in use
+    static_assert(!SWIGLU || BN == 512, "the gated activation pairs the two accumulators of a wide tile");
     constexpr int TILE_N = SWIGLU ? SUBN : BN;        // tile width in the columns the tile walk counts (output columns)
-    constexpr int SUBH = SUBN / CTAS;                // B columns of one sub-tile this CTA stages
+    constexpr int SUBH = SUBN / CTAS;                // B columns of the first sub-tile this CTA stages
+    constexpr int SUBH1 = SUBN1 / CTAS;              // ... of the second
+    static_assert(BN != 384 || CTAS == 2, "the 384-wide tile is a CTA-pair tile");
+    // B boxes are 64 columns wide for an N-contiguous B; a K-contiguous B is staged in one box per sub-tile, except in
+    // the 384-wide tile, whose sub-tiles differ in width: 64-row boxes there (same place in shared memory either way)
+    constexpr bool B64 = BN == 384;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     unsigned char* epi = smem + (size_t)gp.stages * gp.stage_bytes;     // 1024-byte aligned: stage sizes are multiples of 1 KB
@@ -528,7 +536,10 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     if (CTAS == 2) cluster_sync();                   // the peer's barriers exist before anything remote touches them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_ptr;
-    asm volatile("griddepcontrol.wait;" ::: "memory");   // everything before this overlapped the previous kernel's tail
+    // Everything before the dependency wait overlaps the previous kernel's tail.  A ragged batch reads its offsets from
+    // global memory right away and waits here; otherwise every role waits where it first needs global memory -- the
+    // producer only after it has worked out its first tile's coordinates.
+    if (RAG != 0) asm volatile("griddepcontrol.wait;" ::: "memory");
 
     // Ragged batch with a dense walk: m-tiles of every problem, as an exclusive prefix over the problems.
     int* rag_prefix = nullptr;
@@ -563,9 +574,10 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         // One lane per TMA box of a stage (at most 6): the whole warp walks the tile/k loop, every lane
         // polls the stage's "empty" barrier, lane 0 posts the byte count and each active lane issues its
         // own box, so a stage is refilled in one issue slot instead of a serial chain.
-        constexpr int NA = BM / 64, NC = SUBH / 64;          // 64-wide boxes per MN-major A tile / B sub-tile
+        constexpr int NA = BM / 64, NC = SUBH / 64, NC1 = SUBH1 / 64;   // 64-wide boxes per MN-major A tile / B sub-tile
+        const bool b64 = B64 || p.b_mn;
         const int nA = p.a_mn ? NA : 1;
-        const int nB = p.b_mn ? NSUB * NC : NSUB;
+        const int nB = b64 ? NC + NC1 : NSUB;
         const bool active = lane < nA + nB;
         const bool isA = lane < nA;
         const int bi = isA ? lane : lane - nA;                // box index within its operand
@@ -582,7 +594,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         int off;                                              // offset of the box along M (A) or N (B) from the tile origin
         int hsel = 0;                                         // sub-tile of a B box
         if (isA) { soff = mn ? (uint32_t)bi * (64 * BK * 2) : 0u; off = (int)rank * BM + (mn ? 64 * bi : 0); }
-        else if (mn) { const int h = bi / NC, c = bi - h * NC; hsel = h; soff = p.a_bytes + (uint32_t)(h * SUBH * BK * 2 + c * 64 * BK * 2); off = h * SUBN + (int)rank * SUBH + 64 * c; }
+        else if (b64) { const int h = bi >= NC ? 1 : 0, c = bi - h * NC; hsel = h; soff = p.a_bytes + (uint32_t)(h * SUBH * BK * 2 + c * 64 * BK * 2); off = h * SUBN + (int)rank * (h ? SUBH1 : SUBH) + 64 * c; }
         else { hsel = bi; soff = p.a_bytes + (uint32_t)(bi * SUBH * BK * 2); off = bi * SUBN + (int)rank * SUBH; }
         if (SWIGLU && !isA) off -= hsel * SUBN;               // sub-tile 1 is not 256 columns on but pair_dist (below)
         const uint32_t full0 = CTAS == 2 ? map_to_cta(smem_u32(&full[0]), 0) : smem_u32(&full[0]);
@@ -614,6 +626,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             int kb0 = t.split * kbps, kb1 = min(num_kb, kb0 + kbps), kbase = 0;
             if (RAG == 0 && p.bal) { kb0 = t.kb0; kb1 = t.kb1; }
             if (RAG == 2) { const KRange kr = k_range(p.k_offs, t.e, p.K); kb0 = 0; kb1 = kr.nkb; kbase = kr.k0; }
+            if (RAG == 0 && it == 0) asm volatile("griddepcontrol.wait;" ::: "memory");   // the first operand load is next
             for (int kb = kb0; kb < kb1; ++kb) {
                 ok = mbar_wait_bounded(&empty[stage], phase ^ 1);
                 ok = __all_sync(0xffffffffu, ok);
@@ -638,15 +651,15 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                             tma_load<CTAS>(st0 + so, &map_a, bar, 0, line_of(p.a, r, c), 0, 0, 0);
                         }
                     if (gather_b)
-                        for (int i = lane; i < NSUB * SUBH; i += 32) {
+                        for (int i = lane; i < SUBH + SUBH1; i += 32) {
                             int r, c; uint32_t so;
                             if (p.b_mn) {
-                                const int ch = i >> 6, kr = i & 63, h = ch / NC, cc = ch - h * NC;
-                                r = k0 + kr; c = t.n0 + h * SUBN + (int)rank * SUBH + 64 * cc;
+                                const int ch = i >> 6, kr = i & 63, h = ch >= NC ? 1 : 0, cc = ch - h * NC;
+                                r = k0 + kr; c = t.n0 + h * SUBN + (int)rank * (h ? SUBH1 : SUBH) + 64 * cc;
                                 so = p.a_bytes + (uint32_t)(h * SUBH * BK * 2 + cc * 64 * BK * 2 + kr * 128);
                             } else {
-                                const int h = i / SUBH, rr = i - h * SUBH;
-                                r = t.n0 + h * SUBN + (int)rank * SUBH + rr; c = k0;
+                                const int h = i >= SUBH ? 1 : 0, rr = i - h * SUBH;
+                                r = t.n0 + h * SUBN + (int)rank * (h ? SUBH1 : SUBH) + rr; c = k0;
                                 so = p.a_bytes + (uint32_t)(h * SUBH * BK * 2 + rr * 128);
                             }
                             tma_load<CTAS>(st0 + so, &map_b, bar, 0, line_of(p.b, r, c), 0, 0, 0);
@@ -658,6 +671,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         if (KS) { __syncwarp(); cluster_sync(); cluster_sync(); }   // the two meetings of the cluster split (see the epilogue)
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+        if (RAG == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
         if (lane == 0 && leader) {
             int stage = 0;
             uint32_t phase = 0;
@@ -711,14 +725,16 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                         }
                         const uint32_t tmem_d = tmem_base + (uint32_t)((acc0 + h) * ACC_COLS);
                         const uint64_t bdesc = smem_desc(sa + a_bytes + h * (SUBH * BK * 2), b_lbo, 1024);
+                        // (the instruction descriptor carries the width of the first sub-tile: N >> 3 in bits 17-22)
+                        const uint32_t idesc_h = (NSUB == 2 && SUBN1 != SUBN && h == 1) ? (idesc & ~(0x3Fu << 17)) | ((uint32_t)(SUBN1 >> 3) << 17) : idesc;
                         if (!cut) {                           // (the common path keeps its four back-to-back MMAs)
 #pragma unroll
                             for (int k = 0; k < BK / 16; ++k)
-                                umma_bf16<CTAS>(tmem_d, adesc + (uint64_t)(k * a_kstep), bdesc + (uint64_t)(k * b_kstep), idesc, ((kb - kb0) | k) != 0);
+                                umma_bf16<CTAS>(tmem_d, adesc + (uint64_t)(k * a_kstep), bdesc + (uint64_t)(k * b_kstep), idesc_h, ((kb - kb0) | k) != 0);
                         } else {
 #pragma unroll 1
                             for (int k = 0; k < ksteps; ++k)
-                                umma_bf16<CTAS>(tmem_d, adesc + (uint64_t)(k * a_kstep), bdesc + (uint64_t)(k * b_kstep), idesc, ((kb - kb0) | k) != 0);
+                                umma_bf16<CTAS>(tmem_d, adesc + (uint64_t)(k * a_kstep), bdesc + (uint64_t)(k * b_kstep), idesc_h, ((kb - kb0) | k) != 0);
                         }
                     }
                     if (!ok) break;
@@ -733,6 +749,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         if (KS) { __syncwarp(); cluster_sync(); cluster_sync(); }
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..5)
+        if (RAG == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
         const int quad = warp & 3;                       // TMEM lane quadrant this warp may read
         constexpr int EW = kEpiWarps / 4;                // warps per quadrant
         const int hf = (warp - 2) >> 2;                  // which of them this one is
@@ -853,7 +870,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             };
             // TMEM reads are software-pipelined: the load of piece c+1 is in flight while piece c is converted
             // and stored (two register sets, so the loop is unrolled by two).
-            const int npieces = min(SUBN / 64, (t.n1 - nb + 63) / 64);      // warp-uniform
+            const int npieces = min((h == 0 ? SUBN : SUBN1) / 64, (t.n1 - nb + 63) / 64);      // warp-uniform
             uint32_t ra[64], rb[64];
             auto load_piece = [&](uint32_t (&r)[64], int c) {
                 tmem_ld32(taddr + (uint32_t)(c * 64), *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
@@ -1292,7 +1309,7 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     const int64_t strips_m = Mt / Wm, strips_n = Nc / Wn;
     int ctas = 1, bn = 256, splits = 1;
     double best = -1.0;
-    // Test overrides (environment): CCL_GEMM_CTAS = 1|2, CCL_GEMM_BN = 128|192|256|512, CCL_GEMM_SPLITK = number of K splits.
+    // Test overrides (environment): CCL_GEMM_CTAS = 1|2, CCL_GEMM_BN = 128|192|256|384|512, CCL_GEMM_SPLITK = number of K splits.
     const char* force_ctas = std::getenv("CCL_GEMM_CTAS");
     const char* force_bn = std::getenv("CCL_GEMM_BN");
     const char* force_split = std::getenv("CCL_GEMM_SPLITK");
@@ -1300,17 +1317,18 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
         if (c == 2 && (pairs <= 0 || ragk)) continue;          // (a ragged-K tail is zeroed by the CTA that issues the MMAs)
         if (force_ctas && atoi(force_ctas) != c) continue;
         const int units = c == 2 ? pairs : sms;
-        for (int b : {512, 256, 192, 128}) {
+        for (int b : {512, 384, 256, 192, 128}) {
             if (c == 1 && b > 256) continue;
             if (c == 2 && b == 192 && !bt) continue;             // 96 columns per CTA are not made of 64-column boxes of an N-contiguous B
             if (b == 192 && (c == 2 ? no_192_pair : no_192)) continue;
+            if (b == 384 && (cap > 0 || ragk)) continue;            // (no ragged-batch instantiation of the 256 + 128 tile)
             if (force_bn && atoi(force_bn) != b) continue;
             if (swiglu && !(c == 2 && b == 512)) continue;          // the gated activation pairs the two accumulators of the wide tile
             const int64_t tiles_m_all = strips_m * ((Wm + BM * c - 1) / (BM * c));
             const int bs = swiglu ? 256 : b;                        // tile width in C columns
             const int64_t tiles = tiles_m_all * strips_n * ((Wn + bs - 1) / bs) * batch;
-            const double t_kb = b == 512 ? 1050.0 : (c == 1 && b == 256 ? 680.0 : (c == 1 ? 570.0 : 620.0));
-            const double t_drain = b == 512 ? 7000.0 : 1500.0;
+            const double t_kb = b == 512 ? 1050.0 : (b == 384 ? 800.0 : (c == 1 && b == 256 ? 680.0 : (c == 1 ? 570.0 : 620.0)));
+            const double t_drain = b == 512 ? 7000.0 : (b == 384 ? 5500.0 : 1500.0);
             // one row of tiles: nobody shares the B columns, the problem streams B from HBM at ~29 B/clk per SM in
             // aggregate however the units are cut (a ragged last wave still saturates the memory); wider boxes are
             // fetched a little more efficiently (measured: 128 / 192 columns cost ~10 % / ~4 % more time per byte)
@@ -1841,7 +1859,7 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
             const bool ks = (q.a_mn ? q.a.split == 1 : q.a.split == 2) || (q.b_mn ? q.b.split == 1 : q.b.split == 2);
             plan.lean = q.group_dim != 2 && !q.axpby && batch == 1 && !q.a.il_mode && !q.b.il_mode && !q.c.il_mode && !ks && !m_offs && !k_offs && !swiglu;
         }
-        const uint32_t bnh = (uint32_t)(plan.subn / plan.ctas);   // B rows of one K-major box
+        const uint32_t bnh = plan.bn == 384 ? 64u : (uint32_t)(plan.subn / plan.ctas);   // B rows of one K-major box
         if (!plan.p.a_mn) s = operand_tmap(&prep.ma, plan.va, A_dev, BK, BM, batch, batch4[1]); else s = operand_tmap(&prep.ma, plan.va, A_dev, 64, BK, batch, batch4[1]);
         if (s) return s;
         if (!plan.p.b_mn) s = operand_tmap(&prep.mb, plan.vb, B_dev, BK, bnh, batch, batch4[2]); else s = operand_tmap(&prep.mb, plan.vb, B_dev, 64, BK, batch, batch4[2]);
@@ -1936,6 +1954,7 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     } else if (plan.lean) {                                // nothing optional in use: the instantiation without those branches
         if (plan.ctas == 2) {
             if (plan.bn == 512) s = launch<512, 2, false, 0, false>(plan, ma, mb, mc, st);
+            else if (plan.bn == 384) s = launch<384, 2, false, 0, false>(plan, ma, mb, mc, st);
             else if (plan.bn == 192) s = launch<192, 2, false, 0, false>(plan, ma, mb, mc, st);
             else s = plan.bn == 256 ? launch<256, 2, false, 0, false>(plan, ma, mb, mc, st) : launch<128, 2, false, 0, false>(plan, ma, mb, mc, st);
         } else if (plan.bn == 256) s = launch<256, 1, false, 0, false>(plan, ma, mb, mc, st);
@@ -1943,6 +1962,7 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
         else s = launch<128, 1, false, 0, false>(plan, ma, mb, mc, st);
     } else if (plan.ctas == 2) {
         if (plan.bn == 512) s = launch<512, 2>(plan, ma, mb, mc, st);
+        else if (plan.bn == 384) s = launch<384, 2>(plan, ma, mb, mc, st);
         else if (plan.bn == 192) s = launch<192, 2>(plan, ma, mb, mc, st);
         else s = plan.bn == 256 ? launch<256, 2>(plan, ma, mb, mc, st) : launch<128, 2>(plan, ma, mb, mc, st);
     } else if (plan.bn == 256) s = launch<256, 1>(plan, ma, mb, mc, st);

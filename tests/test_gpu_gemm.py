@@ -297,7 +297,7 @@ def test_gemm_m1024_llama_weights(name, P):
     check_sampled(d, A, B, g, P, np.random.default_rng(1), n_random=6)
 
 
-@pytest.fixture(params=[(1, 128), (1, 192), (1, 256), (2, 128), (2, 192), (2, 256), (2, 512)], ids=lambda v: f"c{v[0]}b{v[1]}")
+@pytest.fixture(params=[(1, 128), (1, 192), (1, 256), (2, 128), (2, 192), (2, 256), (2, 384), (2, 512)], ids=lambda v: f"c{v[0]}b{v[1]}")
 def tile_mode(request):
     """Forces one kernel variant: CTAs per tile (1, or a cta_group::2 pair) and tile width."""
     keys = ("CCL_GEMM_CTAS", "CCL_GEMM_BN")
@@ -322,6 +322,43 @@ def test_gemm_every_tile_shape(M, N, K, P, at, bt, tile_mode):
         assert e.status == ccl.ERR_UNSUPPORTED
         pytest.skip("variant not available for this operand layout")
     check(d, A, B)
+
+
+WIDE384 = [
+    # M, N, K, P, layouts, a_trans, b_trans, out_part, chunk bytes (page-interleaved operands), alpha, beta
+    (4096, 1536, 256, 4, ("row", "ccl", "ccl"), 0, 0, 2, 0, 1.0, 0.0),          # strips of exactly one tile width (the Qwen gate+up shape, short K)
+    (520, 1536, 328, 2, ("row", "ccl", "ccl"), 0, 1, 2, 0, 1.0, 0.0),           # B stored [N x K]: three 64-row boxes per CTA; two tiles per strip
+    (304, 1000, 512, 1, ("row", "row", "row"), 1, 1, 0, 0, 1.0, 0.0),           # ragged in M and N: a last tile that ends inside its first sub-tile ... (1000 = 2 * 384 + 232)
+    (300, 1096, 512, 1, ("row", "row", "row"), 0, 0, 0, 0, 1.0, 0.0),           # ... and one that ends inside its second (1096 = 2 * 384 + 256 + 72)
+    (264, 1536, 328, 4, ("row", "ileave", "ileave"), 0, 0, 2, 256, 1.0, 0.0),   # a strip row of 3 chunks
+    (200, 768, 256, 2, ("row", "ileave", "ileave"), 0, 1, 2, 4096, 1.0, 0.0),   # B stored [N x K] in chunks of 8 rows
+    (264, 3584, 512, 4, ("row", "ileave", "ileave"), 0, 0, 2, 4096, 1.0, 0.0),  # chunks and strip rows that do not line up: row-by-row fetch
+    (512, 768, 256, 4, ("ileave", "row", "ileave"), 0, 0, 1, 2048, 1.0, 0.0),   # M-partition
+    (520, 1536, 328, 4, ("row", "ccl", "ccl"), 0, 0, 2, 0, 0.5, 2.0),           # alpha / beta
+]
+
+
+@pytest.mark.parametrize("M,N,K,P,lay,at,bt,op,chunk,alpha,beta", WIDE384)
+def test_gemm_384_wide_pair_tile(M, N, K, P, lay, at, bt, op, chunk, alpha, beta, monkeypatch):
+    """The 256 x 384 pair tile (a 256-wide and a 128-wide MMA per k step) forced on: parity with the oracle; with K split too."""
+    monkeypatch.setenv("CCL_GEMM_CTAS", "2")
+    monkeypatch.setenv("CCL_GEMM_BN", "384")
+    monkeypatch.setenv("CCL_GEMM_CLUSTERK", "0")
+    A, B = synth.gemm_operands(M, N, K, at, bt, seed=11, tag="w384")
+    d = gemm_desc(M, N, K, P, lay, at, bt, op, 1, align=chunk)
+    if alpha == 1.0 and beta == 0.0:
+        check(d, A, B)
+        monkeypatch.setenv("CCL_GEMM_SPLITK", "2")
+        check(d, A, B)
+        return
+    Cin = synth.randn_bf16(M, N, 1.0, 11, "w384/C")
+    a_dev, b_dev, c_dev = to_layout(synth.bits(A), d.A), to_layout(synth.bits(B), d.B), to_layout(synth.bits(Cin), d.C)
+    ccl.ccl_gemm_axpby(d, alpha, beta, a_dev, b_dev, c_dev)
+    assert ccl.ccl_gemm_status()[0] == ccl.OK
+    got = synth.from_bits(from_layout(c_dev, d.C)).to(torch.float32).numpy()
+    ref32, _ = orc.gemm_axpby(synth.bits(A), synth.bits(B), synth.bits(Cin), M, N, K, alpha, beta, at, bt)
+    err = np.abs(got - ref32) / np.maximum(1.0, np.abs(ref32))
+    assert err.max() <= abs(alpha) * tol(K) + 2.0 ** -8, err.max()
 
 
 @pytest.fixture(params=["auto", "1", "2", "4", "8", "2p", "4p"])
@@ -399,7 +436,7 @@ AXPBY = [
     (300, 1024, 256, 4, ("row", "ileave", "ileave"), 0, 0, 2, 0.25, 3.0),  # page-interleaved C
     (640, 2560, 512, 2, ("row", "ccl", "ccl"), 0, 0, 2, 3.0, 0.0),         # beta = 0: C is not read
     (256, 768, 2048, 4, ("row", "ccl", "ccl"), 0, 1, 2, 0.5, 2.0),         # few tiles: split inside clusters, the owners of the sums apply the scalars
-    (130, 392, 4096, 2, ("row", "ccl", "ccl"), 0, 0, 2, -2.0, 1.0),        # ... with ragged rows and columns
+    (130, 400, 4096, 2, ("row", "ccl", "ccl"), 0, 0, 2, -2.0, 1.0),        # ... with ragged rows and columns
 ]
 
 
