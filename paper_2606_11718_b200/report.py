@@ -50,7 +50,8 @@ def configs(which, quick):
             for P in ((4,) if quick else (2, 4, 8)):
                 sweep.append(dict(g, name=f"{g['name']}_M{M}", M=M, P=P, S=4096))
     out[5] = sweep
-    return {k: v for k, v in out.items() if which in ("all", str(k))}
+    want = [w.strip() for w in str(which).split(",")]
+    return {k: v for k, v in out.items() if "all" in want or str(k) in want}
 
 
 def mats(g, layout_bc, align=0):
@@ -62,6 +63,24 @@ def mats(g, layout_bc, align=0):
     mB = ccl.Mat(b_shape[0], b_shape[1], 2, P, b_part, layout_bc, align if layout_bc == ccl.CCL else 0)
     mC = ccl.Mat(M, N, 2, P, ccl.PART_COLS, layout_bc, align if layout_bc == ccl.CCL else 0)
     return mA, mB, mC
+
+
+_NVML = {}
+LAST_CLOCK = dict(sm_mhz=None, sm_max_mhz=None)
+
+
+def sm_clock():
+    """SM clock of the current device in MHz (read through NVML; None where that is not possible).  Reading only."""
+    try:
+        import pynvml
+        if "h" not in _NVML:
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(torch.cuda.current_device()).uuid)
+            _NVML["h"] = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + uuid if not uuid.startswith("GPU-") else uuid).encode())
+            _NVML["max"] = pynvml.nvmlDeviceGetMaxClockInfo(_NVML["h"], pynvml.NVML_CLOCK_SM)
+        return dict(sm_mhz=pynvml.nvmlDeviceGetClockInfo(_NVML["h"], pynvml.NVML_CLOCK_SM), sm_max_mhz=_NVML["max"])
+    except Exception:
+        return dict(sm_mhz=None, sm_max_mhz=None)
 
 
 def timed(fn, reps, warm=2):
@@ -77,6 +96,7 @@ def timed(fn, reps, warm=2):
     for _ in range(reps):
         fn()
     e1.record()
+    LAST_CLOCK.update(sm_clock())            # sampled while the queued launches run
     torch.cuda.synchronize()
     return e0.elapsed_time(e1) / reps
 
@@ -209,7 +229,7 @@ def run_gemm(g, pk, reps, lru=False):
         ms_g = timed(lambda: ccl.ccl_gemm(d, A, Bl, Cb, ws), reps)
         st, detail = ccl.ccl_gemm_status()
         tf = flop / ms_g / 1e9
-        res[tag] = dict(ms=ms_g, tflops=tf, frac_of_roofline=tf / roof_tf, split_k_workspace=need, status=st)
+        res[tag] = dict(ms=ms_g, tflops=tf, frac_of_roofline=tf / roof_tf, split_k_workspace=need, status=st, **LAST_CLOCK)
         if lay == ccl.CCL:
             Cr = torch.empty(M * N, dtype=torch.bfloat16, device=dev)
             ccl.ccl_repack(mC, Cb, Cr, 1)
@@ -561,7 +581,7 @@ def one_gemm(args):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--config", default="all")
+    ap.add_argument("--config", default="all", help="all, one configuration (1-5) or a comma-separated list (e.g. 1,2)")
     ap.add_argument("--out", default=os.path.join(ROOT, "report_out"))
     ap.add_argument("--quick", action="store_true", help="fewer repetitions and P = 4 only in the sweep")
     ap.add_argument("--lru", action="store_true", help="also score the placements behind a finite LRU L2 per chiplet (slow at Llama sizes)")
@@ -607,7 +627,7 @@ def main():
             t = r["traffic"]
             print(f"cfg{cfg} {r['name']:24s} M{r['M']:5d} N{r['N']:5d} K{r['K']:5d} P{r['P']} S{r['page']:7d} | "
                   f"gemm ccl {c.get('tflops', float('nan')):7.1f} row {rw.get('tflops', float('nan')):7.1f} torch {r['torch_matmul_tflops']:7.1f} TF "
-                  f"(roof {r['roofline_tflops']:6.1f} {r['roofline_bound']}, {100 * c.get('frac_of_roofline', float('nan')):5.1f}%) "
+                  f"(roof {r['roofline_tflops']:6.1f} {r['roofline_bound']}, {100 * c.get('frac_of_roofline', float('nan')):5.1f}%, {c.get('ms', float('nan')) * 1e3:.1f} us at {c.get('sm_mhz')} MHz) "
                   f"bits_equal={r.get('ccl_equals_rowmajor_bits')} | repack {r.get('repack', {}).get('gbs', float('nan')):7.1f} GB/s | "
                   f"remote/rr4k: rr64k {t['row_rr64k']['ratio_vs_rr4k']:.3f} rr2m {t['row_rr2m']['ratio_vs_rr4k']:.3f} "
                   f"block {t['row_block']['ratio_vs_rr4k']:.3f} best {t['row_best']['ratio_vs_rr4k']:.3f} "
