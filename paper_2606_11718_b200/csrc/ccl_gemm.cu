@@ -197,6 +197,41 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint6
         asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}"
                      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// The four MMAs of one k block (UMMA_K = 16 each).  The MMA-issuing thread is the pacemaker of a short GEMM: its scalar
+// instructions run one dependent step at a time, and ~300 cycles of address arithmetic, barrier polling and hand-back
+// around ~300 cycles of MMA issue made every k block cost ~600 cycles whatever the tile width (measured), while a
+// 256-wide block keeps the tensor pipe busy for 512.  So the descriptors are carried as 32-bit halves (only the low
+// word, which holds the shared-memory address in 16-byte units, changes from step to step and from stage to stage),
+// and, with PROBE, a look at the NEXT stage's barrier is started before the MMAs and read after them, so that its
+// latency passes behind their issue.  Returns whether phase `probe_parity` of that barrier has completed (acquire).
+// Called by a whole, converged warp with the same arguments in every lane (so that the compiler can keep them in
+// uniform registers, which is where the MMA instruction takes its operands from); one elected lane issues the MMAs.
+template <int CTAS, bool PROBE>
+__device__ __forceinline__ uint32_t umma_bf16_x4(uint32_t tmem_d, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi, uint32_t a_kstep,
+                                                 uint32_t b_kstep, uint32_t idesc, uint32_t accumulate, uint32_t probe_bar, uint32_t probe_parity) {
+    uint32_t done = 0;
+#define CCL_UMMA_X4(GROUP, PROBE_INSTR, PROBE_READ)                                                                     \
+    asm volatile("{\n .reg .pred p, q, t, e;\n .reg .b32 x, y;\n .reg .b64 da, db;\n" PROBE_INSTR                         \
+                 " elect.sync _|e, 0xffffffff;\n"                                                                        \
+                 " setp.ne.b32 p, %9, 0;\n setp.eq.b32 t, 0, 0;\n"                                                       \
+                 " mov.b64 da, {%2, %3};\n mov.b64 db, {%4, %5};\n"                                                      \
+                 " @e tcgen05.mma.cta_group::" GROUP ".kind::f16 [%1], da, db, %8, p;\n"                                 \
+                 " add.u32 x, %2, %6;\n add.u32 y, %4, %7;\n mov.b64 da, {x, %3};\n mov.b64 db, {y, %5};\n"             \
+                 " @e tcgen05.mma.cta_group::" GROUP ".kind::f16 [%1], da, db, %8, t;\n"                                 \
+                 " add.u32 x, x, %6;\n add.u32 y, y, %7;\n mov.b64 da, {x, %3};\n mov.b64 db, {y, %5};\n"               \
+                 " @e tcgen05.mma.cta_group::" GROUP ".kind::f16 [%1], da, db, %8, t;\n"                                 \
+                 " add.u32 x, x, %6;\n add.u32 y, y, %7;\n mov.b64 da, {x, %3};\n mov.b64 db, {y, %5};\n"               \
+                 " @e tcgen05.mma.cta_group::" GROUP ".kind::f16 [%1], da, db, %8, t;\n" PROBE_READ "}"                  \
+                 : "+r"(done)                                                                                            \
+                 : "r"(tmem_d), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(a_kstep), "r"(b_kstep), "r"(idesc), "r"(accumulate),   \
+                   "r"(probe_bar), "r"(probe_parity) : "memory")
+    if (CTAS == 1 && PROBE) CCL_UMMA_X4("1", " mbarrier.test_wait.parity.shared::cta.b64 q, [%10], %11;\n", " selp.u32 %0, 1, 0, q;\n");
+    else if (CTAS == 1) CCL_UMMA_X4("1", "", "");
+    else if (PROBE) CCL_UMMA_X4("2", " mbarrier.test_wait.parity.shared::cta.b64 q, [%10], %11;\n", " selp.u32 %0, 1, 0, q;\n");
+    else CCL_UMMA_X4("2", "", "");
+#undef CCL_UMMA_X4
+    return done;
+}
 // Arrive on an mbarrier once every MMA issued so far by this thread has completed.  With two CTAs
 // the arrival is delivered to the barrier at the same offset in both CTAs of the pair.
 template <int CTAS>
@@ -206,6 +241,15 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
     else
         asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
                      ::"r"(smem_u32(bar)), "h"((unsigned short)3) : "memory");
+}
+// (called by a whole, converged warp: one elected lane issues the commit)
+template <int CTAS>
+__device__ __forceinline__ void umma_commit_addr(uint32_t bar_addr) {
+    if (CTAS == 1)
+        asm volatile("{\n .reg .pred e;\n elect.sync _|e, 0xffffffff;\n @e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n}" ::"r"(bar_addr) : "memory");
+    else
+        asm volatile("{\n .reg .pred e;\n elect.sync _|e, 0xffffffff;\n @e tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;\n}"
+                     ::"r"(bar_addr), "h"((unsigned short)3) : "memory");
 }
 // TMA tile load whose completion bytes are credited to `bar_addr` (a shared::cluster address; with two
 // CTAs this is the leader's barrier, which the cta_group::2 form of the copy is allowed to signal).
@@ -574,7 +618,10 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         // One lane per TMA box of a stage (at most 6): the whole warp walks the tile/k loop, every lane
         // polls the stage's "empty" barrier, lane 0 posts the byte count and each active lane issues its
         // own box, so a stage is refilled in one issue slot instead of a serial chain.
-        constexpr int NA = BM / 64, NC = SUBH / 64, NC1 = SUBH1 / 64;   // 64-wide boxes per MN-major A tile / B sub-tile
+        // 64-wide boxes per MN-major A tile / B sub-tile.  (The 96 columns a CTA of a 256 x 192 pair tile stages of an
+        // N-contiguous B are fetched as two boxes, the second of which is half used: what it holds beyond the 96th
+        // column -- the peer's columns, the next tile's, or the zero fill past the strip's end -- is never read.)
+        constexpr int NA = BM / 64, NC = (SUBH + 63) / 64, NC1 = (SUBH1 + 63) / 64;
         const bool b64 = B64 || p.b_mn;
         const int nA = p.a_mn ? NA : 1;
         const int nB = b64 ? NC + NC1 : NSUB;
@@ -672,20 +719,34 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (leader CTA only)
         if (RAG == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
-        if (lane == 0 && leader) {
+        // The whole warp runs the loop with the same values in every lane and one elected lane issues the tcgen05
+        // instructions: values the compiler can prove warp-uniform (kernel parameters, shuffles, votes) live in uniform
+        // registers, which is where the MMA takes its descriptors from -- a single diverged lane had to move every
+        // operand across for every instruction.
+        if (leader) {
+            const uint32_t FULLMASK = 0xffffffffu;
             int stage = 0;
             uint32_t phase = 0;
             TileCoord t;
             bool ok = true;
-            const uint32_t a_lbo = p.a_mn ? 64 * BK * 2 : 16, b_lbo = p.b_mn ? 64 * BK * 2 : 16;
-            const uint32_t a_kstep = p.a_mn ? (16 * 128) >> 4 : (16 * 2) >> 4;     // descriptor units (16 B) per UMMA_K = 16
-            const uint32_t b_kstep = p.b_mn ? (16 * 128) >> 4 : (16 * 2) >> 4;
-            // loop constants in registers (the asm statements below are memory barriers to the compiler)
-            const int stages = p.stages, num_kb = p.num_kb, kbps = p.kb_per_split;
-            const uint32_t stage_bytes = p.stage_bytes, a_bytes = p.a_bytes, idesc = p.idesc, smem0 = smem_u32(smem);
+            const uint32_t a_lbo = gp.a_mn ? 64 * BK * 2 : 16, b_lbo = gp.b_mn ? 64 * BK * 2 : 16;
+            const uint32_t a_kstep = gp.a_mn ? (16 * 128) >> 4 : (16 * 2) >> 4;     // descriptor units (16 B) per UMMA_K = 16
+            const uint32_t b_kstep = gp.b_mn ? (16 * 128) >> 4 : (16 * 2) >> 4;
+            const int stages = gp.stages, num_kb = gp.num_kb, kbps = gp.kb_per_split;
+            const uint32_t stage_bytes = gp.stage_bytes, a_bytes = gp.a_bytes, idesc = gp.idesc, smem0 = smem_u32(smem);
+            const uint32_t tmem_b = __shfl_sync(FULLMASK, tmem_base, 0);
             int done = 0;                                   // tiles computed so far (empty tiles of a ragged batch do not count)
-            for (int it = 0; ok && sched.template get<RAG, FULL>(it, t); ++it) {
-                if (t.skip) continue;
+            bool ready = false;
+            // running values of the current stage: descriptor low words (the address field counts 16-byte units; a stage
+            // is a multiple of 1 KB), the shared-memory addresses of its two barriers
+            const uint64_t adesc0 = smem_desc(smem0, a_lbo, 1024), bdesc0 = smem_desc(smem0 + a_bytes, b_lbo, 1024);
+            const uint32_t a_hi = (uint32_t)(adesc0 >> 32), b_hi = (uint32_t)(bdesc0 >> 32), a_lo0 = (uint32_t)adesc0, b_lo0 = (uint32_t)bdesc0;
+            const uint32_t st_units = stage_bytes >> 4, fbar0 = smem_u32(&full[0]), ebar0 = smem_u32(&empty[0]);
+            uint32_t a_lo = a_lo0, b_lo = b_lo0, fbar = fbar0, ebar = ebar0;
+            for (int it = 0; ok; ++it) {
+                const bool more = sched.template get<RAG, FULL>(it, t);
+                if (!__shfl_sync(FULLMASK, (int)more, 0)) break;
+                if (RAG != 0 && __shfl_sync(FULLMASK, (int)t.skip, 0)) continue;
                 if (KS) t.split = (int)krank;
                 // NSUB == 1: TMEM half (done & 1) is this tile's accumulator, the other half is being drained.
                 // NSUB == 2: both halves belong to this tile; half h may be overwritten once the epilogue
@@ -694,14 +755,21 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 const uint32_t acc_phase = NSUB == 1 ? ((uint32_t)(done >> 1) & 1) : ((uint32_t)done & 1);
                 ++done;
                 int kb0 = t.split * kbps, kb1 = min(num_kb, kb0 + kbps), tail = BK;
-                if (RAG == 0 && p.bal) { kb0 = t.kb0; kb1 = t.kb1; }
+                if (RAG == 0 && gp.bal) { kb0 = t.kb0; kb1 = t.kb1; }
                 if (RAG == 2) { const KRange kr = k_range(p.k_offs, t.e, p.K); kb0 = 0; kb1 = kr.nkb; tail = kr.rem; }
+                kb0 = __shfl_sync(FULLMASK, kb0, 0); kb1 = __shfl_sync(FULLMASK, kb1, 0);
+                if (RAG == 2) tail = __shfl_sync(FULLMASK, tail, 0);
                 for (int kb = kb0; ok && kb < kb1; ++kb) {
                     // (the copies' completion on the barrier orders the operand bytes before the MMAs that read them;
                     // tcgen05 fences are only needed around the accumulator hand-over below)
-                    if (!mbar_wait_bounded(&full[stage], phase)) { atomicExch(&g_gemm_status, 3); ok = false; break; }
-                    const uint32_t sa = smem0 + (uint32_t)stage * stage_bytes;
-                    const uint64_t adesc = smem_desc(sa, a_lbo, 1024);
+                    // `ready`: this stage's barrier was already seen complete by the look-ahead of the previous k block
+                    if (!ready) {
+                        ok = __all_sync(FULLMASK, mbar_wait_bounded_addr(fbar, phase));
+                        if (!ok) { if (lane == 0) atomicExch(&g_gemm_status, 3); break; }
+                    }
+                    // the stage after this one (its barrier is looked at while this block's MMAs are issued)
+                    uint32_t n_a_lo = a_lo + st_units, n_b_lo = b_lo + st_units, n_fbar = fbar + 8, n_ebar = ebar + 8, n_phase = phase;
+                    if (++stage == stages) { stage = 0; n_a_lo = a_lo0; n_b_lo = b_lo0; n_fbar = fbar0; n_ebar = ebar0; n_phase = phase ^ 1; }
                     // Ragged K, last block of a problem: only the 16-row k steps that hold rows of this problem are
                     // issued, and the rows of the last step that belong to the next problem are zeroed in shared memory
                     // (both operands are [k][64 columns] boxes of 128-byte rows here, so a k row is a whole line).
@@ -709,41 +777,48 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     int ksteps = BK / 16;
                     if (cut) {
                         ksteps = tail > 0 ? (tail + 15) / 16 : 1;
+                        const uint32_t sa = (a_lo & 0x3FFFu) << 4;          // the stage's shared-memory address, back from the descriptor
                         const int nboxes = (int)(stage_bytes / (64 * BK * 2));
-                        for (int r = tail; r < ksteps * 16; ++r)
-                            for (int b = 0; b < nboxes; ++b)
+                        for (int i = tail * nboxes + lane; i < ksteps * 16 * nboxes; i += 32) {     // the lanes share the (row, box) pairs
+                            const int r = i / nboxes, b = i - r * nboxes;
 #pragma unroll
-                                for (int c = 0; c < 8; ++c)
-                                    asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(sa + (uint32_t)(b * 64 * BK * 2 + r * 128 + c * 16)), "r"(0u) : "memory");
+                            for (int c = 0; c < 8; ++c)
+                                asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(sa + (uint32_t)(b * 64 * BK * 2 + r * 128 + c * 16)), "r"(0u) : "memory");
+                        }
                         fence_proxy_async();
+                        __syncwarp();
                     }
+                    ready = false;
 #pragma unroll
                     for (int h = 0; h < NSUB; ++h) {
                         if (kb == kb0) {
-                            if (!mbar_wait_bounded(&tmem_empty[acc0 + h], acc_phase ^ 1)) { atomicExch(&g_gemm_status, 2); ok = false; break; }
+                            ok = __all_sync(FULLMASK, mbar_wait_bounded(&tmem_empty[acc0 + h], acc_phase ^ 1));
+                            if (!ok) { if (lane == 0) atomicExch(&g_gemm_status, 2); break; }
                             tc_fence_after();
                         }
-                        const uint32_t tmem_d = tmem_base + (uint32_t)((acc0 + h) * ACC_COLS);
-                        const uint64_t bdesc = smem_desc(sa + a_bytes + h * (SUBH * BK * 2), b_lbo, 1024);
+                        const uint32_t tmem_d = tmem_b + (uint32_t)((acc0 + h) * ACC_COLS);
+                        const uint32_t b_lo_h = b_lo + (uint32_t)(h * ((SUBH * BK * 2) >> 4));
                         // (the instruction descriptor carries the width of the first sub-tile: N >> 3 in bits 17-22)
                         const uint32_t idesc_h = (NSUB == 2 && SUBN1 != SUBN && h == 1) ? (idesc & ~(0x3Fu << 17)) | ((uint32_t)(SUBN1 >> 3) << 17) : idesc;
-                        if (!cut) {                           // (the common path keeps its four back-to-back MMAs)
-#pragma unroll
-                            for (int k = 0; k < BK / 16; ++k)
-                                umma_bf16<CTAS>(tmem_d, adesc + (uint64_t)(k * a_kstep), bdesc + (uint64_t)(k * b_kstep), idesc_h, ((kb - kb0) | k) != 0);
+                        if (!cut) {                           // (the common path: four back-to-back MMAs and a look at the next stage's barrier)
+                            static_assert(BK / 16 == 4, "four MMAs per k block");
+                            if (h == 0) ready = __all_sync(FULLMASK, umma_bf16_x4<CTAS, true>(tmem_d, a_lo, a_hi, b_lo_h, b_hi, a_kstep, b_kstep, idesc_h, kb != kb0, n_fbar, n_phase) != 0);
+                            else umma_bf16_x4<CTAS, false>(tmem_d, a_lo, a_hi, b_lo_h, b_hi, a_kstep, b_kstep, idesc_h, kb != kb0, 0u, 0u);
                         } else {
+                            const uint64_t adesc = ((uint64_t)a_hi << 32) | a_lo, bdesc = ((uint64_t)b_hi << 32) | b_lo_h;
+                            if (lane == 0) {
 #pragma unroll 1
-                            for (int k = 0; k < ksteps; ++k)
-                                umma_bf16<CTAS>(tmem_d, adesc + (uint64_t)(k * a_kstep), bdesc + (uint64_t)(k * b_kstep), idesc_h, ((kb - kb0) | k) != 0);
+                                for (int k = 0; k < ksteps; ++k)
+                                    umma_bf16<CTAS>(tmem_d, adesc + (uint64_t)(k * a_kstep), bdesc + (uint64_t)(k * b_kstep), idesc_h, ((kb - kb0) | k) != 0);
+                            }
+                            __syncwarp();
                         }
                     }
                     if (!ok) break;
-                    umma_commit<CTAS>(&empty[stage]);          // frees the stage (in both CTAs) once these MMAs have read it
-                    if (++stage == stages) { stage = 0; phase ^= 1; }
+                    umma_commit_addr<CTAS>(ebar);              // frees the stage (in both CTAs) once these MMAs have read it
+                    a_lo = n_a_lo; b_lo = n_b_lo; fbar = n_fbar; ebar = n_ebar; phase = n_phase;
                 }
-                if (ok) {
-                    umma_commit<CTAS>(&tmem_full[acc0]);   // accumulator(s) complete (both CTAs); the sub-tiles of a wide tile finish together
-                }
+                if (ok) umma_commit_addr<CTAS>(smem_u32(&tmem_full[acc0]));   // accumulator(s) complete (both CTAs); the sub-tiles of a wide tile finish together
             }
         }
         if (KS) { __syncwarp(); cluster_sync(); cluster_sync(); }
@@ -1214,6 +1289,16 @@ static ccl_status merge_width(int64_t* cur, int64_t w, const char* dim) {
 // ragk: a batch with ragged K -- d->K is the total row count of the concatenated A [K x M] and B [K x N]
 static int resident_clusters(int ks, bool have_device);
 
+// Modelled cycles of one k block (64 of K) of a tile `b` columns wide on `c` CTAs: the tensor pipe needs 2 cycles per tile
+// column (128 rows per SM, UMMA_K = 16, four steps); the SM pulls its share of the operands (its 128 rows of A and its
+// columns of B, whole 64-column boxes of an N-contiguous B) from the L2 at ~70 B/clk; the producer and MMA-issue loops
+// need ~450 cycles per block whatever the tile (all measured with per-role timestamps); the longest of the three, plus
+// the hand-over.
+static double kblock_cycles(int b, int c, bool b_kmajor) {
+    const double b_cols = (double)(b_kmajor ? b / c : (b / c + 63) / 64 * 64);
+    return std::max(std::max(2.0 * b, (BM + b_cols) * (BK * 2) / 70.0), 450.0) + 15.0;
+}
+
 // have_device: the unit counts come from the current device (else the figures of a B200)
 static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, const void* A, const void* B, const void* C, int sms, int pairs, GemmPlan* plan,
                             int64_t cap = 0, bool ragk = false, size_t max_ws = ~(size_t)0, bool have_device = false) {
@@ -1319,7 +1404,7 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
         const int units = c == 2 ? pairs : sms;
         for (int b : {512, 384, 256, 192, 128}) {
             if (c == 1 && b > 256) continue;
-            if (c == 2 && b == 192 && !bt) continue;             // 96 columns per CTA are not made of 64-column boxes of an N-contiguous B
+            if (c == 2 && b == 192 && !bt && il_b) continue;    // 96 columns per CTA of an N-contiguous B: a box and a half (see the kernel), not across chunks
             if (b == 192 && (c == 2 ? no_192_pair : no_192)) continue;
             if (b == 384 && (cap > 0 || ragk)) continue;            // (no ragged-batch instantiation of the 256 + 128 tile)
             if (force_bn && atoi(force_bn) != b) continue;
@@ -1327,7 +1412,10 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
             const int64_t tiles_m_all = strips_m * ((Wm + BM * c - 1) / (BM * c));
             const int bs = swiglu ? 256 : b;                        // tile width in C columns
             const int64_t tiles = tiles_m_all * strips_n * ((Wn + bs - 1) / bs) * batch;
-            const double t_kb = b == 512 ? 1050.0 : (b == 384 ? 800.0 : (c == 1 && b == 256 ? 680.0 : (c == 1 ? 570.0 : 620.0)));
+            // a k block: the tensor pipe needs 2 cycles per tile column (128 rows per SM, UMMA_K = 16, four steps), the
+            // SM pulls its share of the operands (its 128 rows of A and its columns of B, whole 64-column boxes of an
+            // N-contiguous B) from the L2 at ~70 B/clk; whichever is longer, plus the hand-over
+            const double t_kb = kblock_cycles(b, c, bt);
             const double t_drain = b == 512 ? 7000.0 : (b == 384 ? 5500.0 : 1500.0);
             // one row of tiles: nobody shares the B columns, the problem streams B from HBM at ~29 B/clk per SM in
             // aggregate however the units are cut (a ragged last wave still saturates the memory); wider boxes are
@@ -1345,6 +1433,10 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
                 const double last = (double)(tiles * sp - (waves - 1) * units) / (double)units;
                 double cost = std::max((double)waves * ((double)kbps * t_kb + (sp > 1 ? 2.0 * t_drain : t_drain)),
                                        stream_clk * (1.0 + 0.1 * (1.0 - last))) + 3000.0;
+                // a problem that runs for long runs at the power cap, where the clock follows the energy a k block costs:
+                // measured, 256 x 256 pair tiles (a third more operand bytes per flop than 256 x 512) take 3-6 % longer on
+                // the Llama-size GEMMs although they need fewer cycles
+                if (cost > 3.0e5) cost *= 1.0 + 0.25 * ((BM + (double)b / c) / ((double)b / c) / 1.5 - 1.0);
                 if (sp > 1) cost += ((double)sp + 0.5) * (double)batch * (double)Mt * (double)d->N * 4.0 / 3400.0 + 14000.0;
                 if (best < 0 || cost < best) { best = cost; ctas = c; bn = b; splits = sp; }
             }
@@ -1427,12 +1519,11 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
                 if (tiles > resident_clusters(k, have_device) || tiles * k > sms) continue;
                 const int64_t kbps = (num_kb + k - 1) / k;
                 if ((num_kb + kbps - 1) / kbps != k || kbps < 2) continue;           // every CTA of the cluster owns k blocks
-                const double t_kb = b == 256 ? 680.0 : 570.0;
-                const double cost = (double)kbps * t_kb + 1500.0 + 3500.0 + 3000.0;    // drain, the exchange and its two meetings, launch
+                const double cost = (double)kbps * kblock_cycles(b, 1, bt) + 1500.0 + 3500.0 + 3000.0;    // drain, the exchange and its two meetings, launch
                 if (best_ks < 0 || cost < best_ks) { best_ks = cost; kb_ = b; kk = k; }
             }
         }
-        if (best_ks > 0 && (want_ks > 0 || best_ks < 0.85 * best)) { ctas = 1; bn = kb_; splits = 1; ks = kk; best = best_ks; }
+        if (best_ks > 0 && (want_ks > 0 || best_ks < 0.95 * best)) { ctas = 1; bn = kb_; splits = 1; ks = kk; best = best_ks; }
     }
     if (std::getenv("CCL_GEMM_VERBOSE"))
         std::fprintf(stderr, "ccl_gemm plan: %lld x %lld x %lld batch %lld -> %d CTA(s) per tile, tile width %d, %d K split(s)%s, modelled %.0f cycles\n",
@@ -1475,7 +1566,7 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     // instruction descriptor: D = f32, A = B = bf16, operand majors, N >> 3, M >> 4 (M spans the CTA pair)
     p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)p.a_mn << 15) | ((uint32_t)p.b_mn << 16) |
               ((uint32_t)(subn >> 3) << 17) | ((uint32_t)(bm >> 4) << 24);
-    p.a_bytes = BM * BK * 2; p.stage_bytes = p.a_bytes + (uint32_t)(bn / ctas) * BK * 2;
+    p.a_bytes = BM * BK * 2; p.stage_bytes = p.a_bytes + (uint32_t)(p.b_mn ? (bn / ctas + 63) / 64 * 64 : bn / ctas) * BK * 2;   // (an N-contiguous B comes in whole 64-column boxes)
     // a ragged batch of up to kRaggedDense problems walks only real tiles: the prefix of their tile counts sits behind
     // the barriers in shared memory, and the operand ring gives up that room
     // (CCL_GEMM_RAGGED_DENSE=0: the fixed grid of max_rows per problem with empty tiles skipped, as for larger batches)
