@@ -141,6 +141,7 @@ struct GemmParams {
     uint32_t idesc;
     int32_t stages;
     uint32_t stage_bytes, a_bytes;  // bytes per stage per CTA, bytes of its A part
+    uint32_t tx_bytes;              // bytes the copies of a stage deliver per CTA (stage_bytes unless the A box is cut short, see a_box_rows)
     int32_t splits, kb_per_split;   // split-K: each tile is computed by `splits` units over disjoint k-block ranges
     float* ws;                      // split-K partial sums, [splits][M][N] fp32 (row-major, logical coordinates)
     // balanced split: the k blocks of the first bal_tiles tiles of a group, laid end to end, are cut into equal shares, one
@@ -651,7 +652,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         bool ok = true;
         // loop constants in registers (the asm statements below are memory barriers to the compiler)
         const int stages = p.stages, num_kb = p.num_kb, kbps = p.kb_per_split;
-        const uint32_t stage_bytes = p.stage_bytes;
+        const uint32_t stage_bytes = p.stage_bytes, tx_bytes = p.tx_bytes;
         const bool post_tx = lane == 0 && leader;
         for (int it = 0; ok && sched.template get<RAG, FULL>(it, t); ++it) {
             if (t.skip) continue;
@@ -679,7 +680,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) { if (lane == 0) atomicExch(&g_gemm_status, 1); break; }
                 // (the byte count may be posted after a copy has completed: the phase cannot end before this arrival)
-                if (post_tx) mbar_expect_tx(&full[stage], stage_bytes * CTAS);
+                if (post_tx) mbar_expect_tx(&full[stage], tx_bytes * CTAS);
                 const int k0 = kbase + kb * BK;
                 if (ksplit) { if (mn) to_coords<FULL>(om, k0, base, x, y, z, u); else to_coords<FULL>(om, base, k0, x, y, z, u); }
                 else if (mn) y = k0; else x = k0;
@@ -1215,6 +1216,7 @@ __global__ void __launch_bounds__(256) splitk_reduce_kernel(const GemmParams p) 
 struct GemmPlan {
     GemmParams p;
     int bn, ctas, subn;
+    int a_box_rows;            // rows of A's TMA box (BM unless A has fewer than 8 rows)
     size_t ws_bytes;
     MatView va, vb, vc;
     uint32_t smem_bytes;
@@ -1566,10 +1568,16 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     // instruction descriptor: D = f32, A = B = bf16, operand majors, N >> 3, M >> 4 (M spans the CTA pair)
     p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)p.a_mn << 15) | ((uint32_t)p.b_mn << 16) |
               ((uint32_t)(subn >> 3) << 17) | ((uint32_t)(bm >> 4) << 24);
+    // Fewer than 8 rows of a K-contiguous A (a decode step): the box holds just those rows.  Measured, a 128-row box of
+    // which fewer than one 8-row swizzle group exists makes the weight-streaming GEMM 57344 x 8192 take 170 us at
+    // M = 1 ... 7 against 147 us at M = 8 ... 33.  The rows of the stage the box no longer writes keep what was there:
+    // they only feed accumulator rows past M, which no epilogue stores.
+    plan->a_box_rows = (!at && cap == 0 && !ragk && !il_a && d->M < 8) ? (int)d->M : BM;
     p.a_bytes = BM * BK * 2; p.stage_bytes = p.a_bytes + (uint32_t)(p.b_mn ? (bn / ctas + 63) / 64 * 64 : bn / ctas) * BK * 2;   // (an N-contiguous B comes in whole 64-column boxes)
     // a ragged batch of up to kRaggedDense problems walks only real tiles: the prefix of their tile counts sits behind
     // the barriers in shared memory, and the operand ring gives up that room
     // (CCL_GEMM_RAGGED_DENSE=0: the fixed grid of max_rows per problem with empty tiles skipped, as for larger batches)
+    p.tx_bytes = p.stage_bytes - (uint32_t)(BM - plan->a_box_rows) * BK * 2;
     const char* rag_env = std::getenv("CCL_GEMM_RAGGED_DENSE");
     const uint32_t rag_bytes = cap > 0 && batch <= kRaggedDense && !(rag_env && atoi(rag_env) == 0) ? (uint32_t)(4 * (kGemmThreads + batch + 1) + 1023) & ~1023u : 0;
     p.rag_dense = rag_bytes ? 1 : 0;
@@ -1951,7 +1959,7 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
             plan.lean = q.group_dim != 2 && !q.axpby && batch == 1 && !q.a.il_mode && !q.b.il_mode && !q.c.il_mode && !ks && !m_offs && !k_offs && !swiglu;
         }
         const uint32_t bnh = plan.bn == 384 ? 64u : (uint32_t)(plan.subn / plan.ctas);   // B rows of one K-major box
-        if (!plan.p.a_mn) s = operand_tmap(&prep.ma, plan.va, A_dev, BK, BM, batch, batch4[1]); else s = operand_tmap(&prep.ma, plan.va, A_dev, 64, BK, batch, batch4[1]);
+        if (!plan.p.a_mn) s = operand_tmap(&prep.ma, plan.va, A_dev, BK, (uint32_t)plan.a_box_rows, batch, batch4[1]); else s = operand_tmap(&prep.ma, plan.va, A_dev, 64, BK, batch, batch4[1]);
         if (s) return s;
         if (!plan.p.b_mn) s = operand_tmap(&prep.mb, plan.vb, B_dev, BK, bnh, batch, batch4[2]); else s = operand_tmap(&prep.mb, plan.vb, B_dev, 64, BK, batch, batch4[2]);
         if (s) return s;
