@@ -28,7 +28,7 @@
  *   CCL_GEMM_BN = 128|192|256|384|512  force the tile width
  *   CCL_GEMM_SPLITK = n            force the number of K splits
  *   CCL_GEMM_BALANCED = 0|1        never / always (where legal) cut the tiles that do not fill a round into equal shares
- *   CCL_GEMM_CLUSTERK = 0|2|4|8    never / always (where legal) let the CTAs of a cluster of that size share one tile,
+ *   CCL_GEMM_CLUSTERK = 0|2|4|8        never / always (where legal) let the CTAs of a cluster of that size share one tile,
  *                                  each over its own part of K (the default picks it for problems of few tiles)
  *   CCL_GEMM_WAVESYNC = 0|n        soft wave barrier off / every n-th round of tiles
  *   CCL_GEMM_PDL = 0               no programmatic dependent launch
