@@ -66,16 +66,25 @@ CASES = [
 
 
 @pytest.mark.parametrize("M,N,K,P,lay,at,bt,op,batch", CASES)
-@pytest.mark.parametrize("ctas", ["auto", "1", "2"])
-def test_batched_equals_oracle_and_single_calls(M, N, K, P, lay, at, bt, op, batch, ctas):
+@pytest.mark.parametrize("ctas", ["auto", "1", "2", "2/384", "2/192"])
+def test_batched_equals_oracle_and_single_calls(M, N, K, P, lay, at, bt, op, batch, ctas, monkeypatch):
+    """ctas: CTAs per tile, optionally with the tile width forced too (the 256 + 128 pair tile; 256 x 192 pairs, whose CTAs
+    stage a box and a half of an N-contiguous B)."""
     old = os.environ.pop("CCL_GEMM_CTAS", None)
     if ctas != "auto":
-        os.environ["CCL_GEMM_CTAS"] = ctas
+        os.environ["CCL_GEMM_CTAS"] = ctas.split("/")[0]
+        if "/" in ctas:
+            monkeypatch.setenv("CCL_GEMM_BN", ctas.split("/")[1])
     try:
         ops = [synth.gemm_operands(M, N, K, at, bt, seed=11 + e, tag="batched") for e in range(batch)]
         As, Bs = [o[0] for o in ops], [o[1] for o in ops]
         align = 1024 if "ileave" in lay else 0
         d = gemm_desc(M, N, K, P, lay, at, bt, op, 1, align=align)
+        try:
+            ccl.ccl_gemm_batched_workspace(d, batch)
+        except ccl.CclError as e:                      # a forced variant that this operand layout does not take
+            assert "/" in ctas and e.status == ccl.ERR_UNSUPPORTED
+            pytest.skip("variant not available for this operand layout")
         got = run_batched(d, batch, As, Bs, gap=64)
         for e in range(batch):
             ref32, _, _ = orc.gemm(synth.bits(As[e]), synth.bits(Bs[e]), M, N, K, at, bt)
