@@ -167,7 +167,8 @@ ccl_status ccl_repack_transpose(const ccl_mat* m, const void* src_dev, void* dst
  * whole rows, an operand whose rows run along K must have K a multiple of 64 or rows-per-strip a multiple of
  * the rows per chunk: the padding of a strip's last chunk is not read as zero.)  When neither holds but a strip row
  * and a chunk are both multiples of 64 elements (say rows of 3.5 chunks), every 128-byte piece of a row still lies
- * inside one chunk and the operand is fetched and written row by row in such pieces -- correct, slower; it then
+ * inside one chunk and the operand is fetched and written row by row in such pieces -- correct, ~10x slower for A or B
+ * (store the operand with K along its rows, or pick a chunk size that divides the strip row, where speed matters); it then
  * must not be split along K, an A or B whose rows run along M or N needs K a multiple of 64, and a strip must hold
  * fewer than 2^31 elements.  Other chunkings -> CCL_ERR_UNSUPPORTED.
  */
