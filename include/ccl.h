@@ -160,7 +160,13 @@ ccl_status ccl_repack_transpose(const ccl_mat* m, const void* src_dev, void* dst
  * grouped_raster = 0) uses one plain raster.  The result does not depend on these choices.
  * Requirements (else CCL_ERR_UNSUPPORTED / CCL_ERR_ALIGN, nothing launched): elem_bytes = 2;
  * every contiguous extent a tile row lives in (cols, or w for CCL_PART_COLS) a multiple of 8
- * elements; strip strides multiples of 16 bytes; base pointers 16-byte aligned.
+ * elements; strip strides multiples of 16 bytes; base pointers 16-byte aligned; where the tile grid follows strips
+ * along N (of B, of C, or of out_part with a grouped raster), strips of a multiple of 8 columns -- likewise strips along
+ * M when A is stored [K x M].
+ * Strips of unequal size (the split dimension not a multiple of P: strips of ceil(. / P), the last one shorter) are
+ * taken by ccl_gemm / ccl_gemm_axpby / ccl_gemm_static_ws: not along K, not page-interleaved, a narrower last strip
+ * a multiple of 8 columns wide (with the rule above that means P >= 9 for strips along N; strips of rows -- an
+ * M-partition with A stored [M x K] -- have no such limit).  K is then never split.
  * A CCL_CCL_INTERLEAVED operand is taken when its chunks line up with its strip rows, so that a tile is an
  * affine box of the buffer: either a chunk holds a power-of-two number of whole strip rows, or a strip row is
  * made of whole chunks of a multiple of 64 elements; the chunk size a multiple of 16 bytes.  (With chunks of

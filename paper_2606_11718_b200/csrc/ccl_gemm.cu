@@ -93,6 +93,8 @@ struct OpMap {          // how stored coordinates (r, c) of an operand become te
     FastDiv il_kr, il_sc;
     int32_t batched;    // 1: each problem of a batch has its own buffer, 0: all problems share this operand
     int32_t rows, cols, roww, nstrips, lines;   // il_mode 3: stored shape, elements of a strip row, strips, 128-byte lines of the buffer
+    int32_t rag;        // 1: the last strip is narrower / lower than the others (the split dimension is not a multiple of P):
+                        // it has a tensor map of its own (the kernel's second set of maps), addressed with strip coordinate 0
 };
 
 struct GemmParams {
@@ -138,6 +140,7 @@ struct GemmParams {
     int64_t c_row, c_stride, c_ichunk, c_nstrips;   // C: elements of a strip row, between strips, per chunk; strips
     int32_t c_cpr;                  // page-interleaved C whose strip rows span chunks: chunks per strip row
     uint16_t* C;
+    int32_t c_wlast;                // elements of a row of C's last strip when that strip is narrower (else 0)
     uint32_t idesc;
     int32_t stages;
     uint32_t stage_bytes, a_bytes;  // bytes per stage per CTA, bytes of its A part
@@ -355,6 +358,7 @@ __device__ __forceinline__ int64_t c_offset(const GemmParams& p, int64_t m, int6
         p.c.il_sc.divmod(xx, cj, x);
         return (((int64_t)rr * p.c_cpr + cj) * p.c_nstrips + g) * p.c_ichunk + x;
     }
+    if (FULL && p.c_wlast && g == p.c.nstrips - 1) return (int64_t)g * p.c_stride + (int64_t)rr * p.c_wlast + xx;   // a narrower last strip
     return (int64_t)g * p.c_stride + (int64_t)rr * p.c_row + xx;
 }
 
@@ -476,6 +480,7 @@ struct Scheduler {
         p.fd_tps_n.divmod(tn, sn, jn);
         t.m0 = sm * p.Wm + jm * bm; t.m1 = min(t.m0 + bm, (sm + 1) * p.Wm);
         t.n0 = sn * p.Wn + jn * bn; t.n1 = min(t.n0 + bn, (sn + 1) * p.Wn);
+        if (FULL) { t.m1 = min(t.m1, p.M); t.n1 = min(t.n1, p.N); }     // (a last strip that is lower / narrower than the others)
     }
     template <int RAG, bool FULL>
     __device__ bool get(int it, TileCoord& t) const {
@@ -505,7 +510,7 @@ struct Scheduler {
         t.e = 0;
         if (FULL && p.batch > 1) { int ii; p.fd_tiles_per_problem.divmod(i, t.e, ii); i = ii; }
         coords<FULL>(g, i, t);
-        t.skip = false;
+        t.skip = FULL && RAG == 0 && (t.m0 >= p.M || t.n0 >= p.N);   // the tile grid of a shorter last strip has empty places
         if (RAG == 1 && p.m_offs) {                      // rows of this problem inside the concatenated A and C
             const int o0 = __ldg(p.m_offs + t.e), o1 = __ldg(p.m_offs + t.e + 1);
             const bool bad = o0 < 0 || o1 > p.M || o1 - o0 > p.Wm;   // outside A / C, or more rows than the caller's bound:
@@ -523,7 +528,11 @@ struct Scheduler {
 template <int BN, int CTAS, bool SWIGLU = false, int RAG = 0, bool FULL = true, int KS = 0>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                const __grid_constant__ CUtensorMap map_c, const __grid_constant__ GemmParams gp) {
+                const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_a2,
+                const __grid_constant__ CUtensorMap map_b2, const __grid_constant__ CUtensorMap map_c2,
+                const __grid_constant__ GemmParams gp) {
+    // map_a2 / map_b2 / map_c2: the last strip of an operand whose strips are not all alike (OpMap::rag); copies of the
+    // first three otherwise
     // The parameters are read from shared memory: the threads fetch the block's words side by side, so
     // the cold constant-cache misses at kernel start overlap instead of queueing up in every role's set-up.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel's CTAs may be placed as SMs free up
@@ -654,6 +663,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         const int stages = p.stages, num_kb = p.num_kb, kbps = p.kb_per_split;
         const uint32_t stage_bytes = p.stage_bytes, tx_bytes = p.tx_bytes;
         const bool post_tx = lane == 0 && leader;
+        bool dep_pending = RAG == 0;                          // the previous kernel has not been waited for yet
         for (int it = 0; ok && sched.template get<RAG, FULL>(it, t); ++it) {
             if (t.skip) continue;
             if (KS) t.split = (int)krank;
@@ -671,10 +681,12 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             if (SWIGLU && !isA) base += (p.fd_wn.div(t.n0) + hsel) * p.pair_dist;
             int x, y, z, u;
             if (mn) to_coords<FULL>(om, 0, base, x, y, z, u); else to_coords<FULL>(om, base, 0, x, y, z, u);
+            const CUtensorMap* mp = map;
+            if (FULL && om.rag && z == om.nstrips - 1) { mp = isA ? &map_a2 : &map_b2; z = 0; }
             int kb0 = t.split * kbps, kb1 = min(num_kb, kb0 + kbps), kbase = 0;
             if (RAG == 0 && p.bal) { kb0 = t.kb0; kb1 = t.kb1; }
             if (RAG == 2) { const KRange kr = k_range(p.k_offs, t.e, p.K); kb0 = 0; kb1 = kr.nkb; kbase = kr.k0; }
-            if (RAG == 0 && it == 0) asm volatile("griddepcontrol.wait;" ::: "memory");   // the first operand load is next
+            if (dep_pending) { asm volatile("griddepcontrol.wait;" ::: "memory"); dep_pending = false; }   // the first operand load is next
             for (int kb = kb0; kb < kb1; ++kb) {
                 ok = mbar_wait_bounded(&empty[stage], phase ^ 1);
                 ok = __all_sync(0xffffffffu, ok);
@@ -684,7 +696,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 const int k0 = kbase + kb * BK;
                 if (ksplit) { if (mn) to_coords<FULL>(om, k0, base, x, y, z, u); else to_coords<FULL>(om, base, k0, x, y, z, u); }
                 else if (mn) y = k0; else x = k0;
-                if (box) tma_load<CTAS>(smem + (size_t)stage * stage_bytes + soff, map, full0 + (uint32_t)stage * 8u, x, y, z, u, t.e * om.batched);
+                if (box) tma_load<CTAS>(smem + (size_t)stage * stage_bytes + soff, mp, full0 + (uint32_t)stage * 8u, x, y, z, u, t.e * om.batched);
                 if (FULL && (gather_a || gather_b)) {
                     // An operand whose chunks and strip rows do not line up: its part of the stage is fetched as single
                     // 128-byte rows (the swizzle is a function of the shared-memory address, so the rows land exactly
@@ -747,7 +759,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             for (int it = 0; ok; ++it) {
                 const bool more = sched.template get<RAG, FULL>(it, t);
                 if (!__shfl_sync(FULLMASK, (int)more, 0)) break;
-                if (RAG != 0 && __shfl_sync(FULLMASK, (int)t.skip, 0)) continue;
+                if ((RAG != 0 || FULL) && __shfl_sync(FULLMASK, (int)t.skip, 0)) continue;
                 if (KS) t.split = (int)krank;
                 // NSUB == 1: TMEM half (done & 1) is this tile's accumulator, the other half is being drained.
                 // NSUB == 2: both halves belong to this tile; half h may be overwritten once the epilogue
@@ -865,6 +877,8 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             // (unless a strip row is cut into chunks, which puts the chunk index in y as well)
             int cx0, cy0, cz0, cu0;
             to_coords<FULL>(p.c, row0, nb, cx0, cy0, cz0, cu0);
+            const CUtensorMap* mpc = &map_c;
+            if (FULL && p.c.rag && cz0 == p.c.nstrips - 1) { mpc = &map_c2; cz0 = 0; }
             const bool c_chunked = FULL && p.c.il_mode == 2;
             // One 64-column piece: registers -> C.  `r` holds 64 fp32 accumulators of this thread's row.
             // One 64-column piece of this warp's 32 rows -> C.  `pk` holds the piece already rounded to bf16 (two
@@ -892,7 +906,7 @@ ccl_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     if (lane == 0) {
                         int cx = cx0 + c * 64, cy = cy0, cz = cz0, cu = cu0;
                         if (c_chunked) to_coords<FULL>(p.c, row0, n64, cx, cy, cz, cu);
-                        tma_store_5d(&map_c, buf, cx, cy, cz, cu, t.e * p.c.batched);
+                        tma_store_5d(mpc, buf, cx, cy, cz, cu, t.e * p.c.batched);
                         tma_store_commit();
                     }
                     ++epi_count;
@@ -1217,6 +1231,7 @@ struct GemmPlan {
     GemmParams p;
     int bn, ctas, subn;
     int a_box_rows;            // rows of A's TMA box (BM unless A has fewer than 8 rows)
+    CUtensorMap ma2, mb2, mc2; // the last strips of operands whose strips are not all alike (else copies of the operands' maps)
     size_t ws_bytes;
     MatView va, vb, vc;
     uint32_t smem_bytes;
@@ -1240,7 +1255,12 @@ static int interleave_mode(const MatView& v, int64_t* kr) {
 // k_along_rows: the GEMM's K dimension runs along the stored rows of this operand (never for C)
 static ccl_status check_operand(const MatView& v, const void* ptr, const char* name, bool k_along_rows, int64_t K, bool is_c = false) {
     if (v.e != 2) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: %s: only 2-byte (bf16) elements are supported", name);
-    if (ragged(v)) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: %s: strips of unequal size (the split dimension is not a multiple of P) are not supported", name);
+    if (ragged(v)) {                     // a last strip narrower / lower than the others: it gets a tensor map of its own
+        if (v.ichunk) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: %s: a page-interleaved operand with strips of unequal size is not supported", name);
+        if (!is_c && (k_along_rows ? v.split == 1 : v.split == 2))
+            return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: %s: strips of unequal size along K are not supported", name);
+        if (v.split == 2 && v.wlast % 8) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: %s: the last strip's %lld columns are not a multiple of 8", name, (long long)v.wlast);
+    }
     int64_t inner = v.split == 2 ? v.w : v.cols;
     if (inner % 8) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: %s: contiguous extent %lld is not a multiple of 8 elements", name, (long long)inner);
     if (v.ichunk) {
@@ -1359,12 +1379,13 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
             if (pn > 1 && (s = merge_width(&Wn, Nc / pn, "N"))) return s;
             groups = d->P; group_dim = 2; groups_n = pn;
         } else if (d->out_part == CCL_PART_COLS) {
-            if (Nc % d->P) return fail(CCL_ERR_SHAPE, "ccl_gemm: N not divisible by P");
-            if ((s = merge_width(&Wn, Nc / d->P, "N"))) return s;
+            // (N not a multiple of P: the strips are those of the operands -- ceil(N / P) wide, the last one narrower)
+            if (Nc % d->P) { if (!(Wn > 0 && (Nc + Wn - 1) / Wn == d->P)) return fail(CCL_ERR_SHAPE, "ccl_gemm: N not divisible by P"); }
+            else if ((s = merge_width(&Wn, Nc / d->P, "N"))) return s;
             groups = d->P; group_dim = 0;
         } else {
-            if (d->M % d->P) return fail(CCL_ERR_SHAPE, "ccl_gemm: M not divisible by P");
-            if ((s = merge_width(&Wm, d->M / d->P, "M"))) return s;
+            if (d->M % d->P) { if (!(Wm > 0 && (d->M + Wm - 1) / Wm == d->P)) return fail(CCL_ERR_SHAPE, "ccl_gemm: M not divisible by P"); }
+            else if ((s = merge_width(&Wm, d->M / d->P, "M"))) return s;
             groups = d->P; group_dim = 1;
         }
     }
@@ -1372,6 +1393,9 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     if ((ka && ka % BK) || (kb && kb % BK)) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: an operand split along K needs strips that are multiples of %d", BK);
     if (ragk && (!at || bt || ka || kb || il_a || il_b))
         return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm_grouped_k: A must be stored [K x M] and B [K x N], neither split along K nor page-interleaved");
+    const bool any_rag = ragged(va) || ragged(vb) || ragged(vc);
+    if (any_rag && (batch > 1 || cap > 0 || ragk || swiglu || d->out_part == CCL_PART_2D))
+        return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: strips of unequal size are taken by the plain call only (no batch, fused activation or 2-D partition)");
     const int64_t Mt = cap > 0 ? cap : d->M;            // rows the tile grid of one problem covers
     if (cap > 0 && Wm) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm_grouped: A and C must not be split along M");
     if (!Wm) Wm = Mt;
@@ -1393,7 +1417,11 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     // 256 x 512 pair tiles move the fewest bytes per flop and win once K is long; short problems prefer the
     // variant whose tile count fills the machine.
     const int64_t num_kb = ((ragk ? std::max<int64_t>(1, d->K / batch) : d->K) + BK - 1) / BK;   // (ragged K: the mean, for the cost model only)
-    const int64_t strips_m = Mt / Wm, strips_n = Nc / Wn;
+    const int64_t strips_m = (Mt + Wm - 1) / Wm, strips_n = (Nc + Wn - 1) / Wn;
+    // a tile starts at a multiple of the strip width: where that is the contiguous coordinate of a tensor map -- the columns of
+    // C (and of an N-contiguous B), the columns of an A stored [K x M] -- it must be a multiple of 8 elements (16 bytes)
+    if (strips_n > 1 && Wn % 8) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: strips of %lld columns of N are not a multiple of 8", (long long)Wn);
+    if (strips_m > 1 && at && Wm % 8) return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: strips of %lld columns of an A stored [K x M] are not a multiple of 8", (long long)Wm);
     int ctas = 1, bn = 256, splits = 1;
     double best = -1.0;
     // Test overrides (environment): CCL_GEMM_CTAS = 1|2, CCL_GEMM_BN = 128|192|256|384|512, CCL_GEMM_SPLITK = number of K splits.
@@ -1425,7 +1453,7 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
             const double stream_clk = tiles_m_all == 1 ? (double)tiles * (double)num_kb * (double)b * (BK * 2) / (sms * 29.0) *
                                                              (b <= 128 ? 1.10 : (b <= 192 ? 1.04 : 1.0)) : 0.0;
             for (int sp : {1, 2, 3, 4, 6, 8, 12, 16}) {
-                if (sp > 1 && (swiglu || cap > 0 || ragk || num_kb / sp < 2)) continue;
+                if (sp > 1 && (swiglu || cap > 0 || ragk || any_rag || num_kb / sp < 2)) continue;
                 if (force_split && atoi(force_split) != sp) continue;
                 const int64_t kbps = (num_kb + sp - 1) / sp;
                 const int64_t sp_eff = (num_kb + kbps - 1) / kbps;          // every split owns at least one k block
@@ -1454,7 +1482,7 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     {
         const char* force_bal = std::getenv("CCL_GEMM_BALANCED");   // 0: never, 1: whenever the call qualifies
         const int want = force_bal ? atoi(force_bal) : -1;
-        const bool can = want != 0 && batch == 1 && !swiglu && cap == 0 && !ragk && num_kb >= 2 && !(force_split && atoi(force_split) > 1);
+        const bool can = want != 0 && batch == 1 && !swiglu && cap == 0 && !ragk && !any_rag && num_kb >= 2 && !(force_split && atoi(force_split) > 1);
         double best_bal = -1.0;
         int bc = 0, bb = 0;
         int64_t bal_rounds = 0;
@@ -1507,7 +1535,7 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     {
         const char* force_ks = std::getenv("CCL_GEMM_CLUSTERK");
         const int want_ks = force_ks ? atoi(force_ks) : -1;
-        const bool can = want_ks != 0 && batch == 1 && !swiglu && cap == 0 && !ragk && !il_a && !il_b && !il_c && !ka && !kb &&
+        const bool can = want_ks != 0 && batch == 1 && !swiglu && cap == 0 && !ragk && !any_rag && !il_a && !il_b && !il_c && !ka && !kb &&
                          !(force_split && atoi(force_split) > 1) && !balanced && !(force_ctas && atoi(force_ctas) != 1) && d->out_part != CCL_PART_2D;
         double best_ks = -1.0;
         int kb_ = 0, kk = 0;
@@ -1545,7 +1573,7 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
     p.pair_dist = swiglu ? (int32_t)Wn : 0; p.fd_wn = make_fastdiv(Wn);
     p.Wm = (int32_t)Wm; p.Wn = (int32_t)Wn;
     p.tps_m = (int32_t)((Wm + bm - 1) / bm); p.tps_n = (int32_t)((Wn + bn_walk - 1) / bn_walk);
-    p.tiles_m = (int32_t)(Mt / Wm) * p.tps_m; p.tiles_n = (int32_t)(Nc / Wn) * p.tps_n;
+    p.tiles_m = (int32_t)((Mt + Wm - 1) / Wm) * p.tps_m; p.tiles_n = (int32_t)((Nc + Wn - 1) / Wn) * p.tps_n;
     p.num_kb = (int32_t)num_kb;
     p.splits = splits; p.kb_per_split = (int32_t)((num_kb + splits - 1) / splits);
     p.a.split = va.split; p.a.w = make_fastdiv(va.w); p.a.h = make_fastdiv(va.h);
@@ -1562,9 +1590,11 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
             os[X]->rows = (int32_t)vs[X]->rows; os[X]->cols = (int32_t)vs[X]->cols;
             os[X]->roww = (int32_t)(vs[X]->split == 2 ? vs[X]->w : vs[X]->cols); os[X]->nstrips = (int32_t)vs[X]->nstrips;
             os[X]->lines = os[X]->il_mode == 3 ? (int32_t)(buffer_elems(*vs[X]) / 64) : 0;
+            os[X]->rag = ragged(*vs[X]) ? 1 : 0;
         }
     }
     p.c_row = vc.split == 2 ? vc.w : vc.cols; p.c_stride = vc.stride;
+    p.c_wlast = ragged(vc) && vc.split == 2 ? (int32_t)vc.wlast : 0;
     p.c_ichunk = vc.ichunk; p.c_nstrips = vc.nstrips;
     p.c_cpr = il_c == 2 ? (int32_t)(p.c_row / vc.ichunk) : 0;
     // instruction descriptor: D = f32, A = B = bf16, operand majors, N >> 3, M >> 4 (M spans the CTA pair)
@@ -1657,10 +1687,21 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
 //   interleaved, mode 1        : {strip row extent, rows per chunk kr, strips, chunk index}; a box of more than kr
 //                                rows takes kr rows from each of box_rows / kr consecutive chunks of its strip
 //   interleaved, mode 2        : {chunk extent, chunks per strip row, rows per strip, strips}
-static ccl_status operand_tmap(CUtensorMap* m, const MatView& v, const void* base, uint32_t box_inner, uint32_t box_rows, int64_t batch, int64_t batch_stride_bytes) {
-    const uint64_t row = (uint64_t)(v.split == 2 ? v.w : v.cols);      // elements of a strip row
-    const uint64_t R = (uint64_t)(v.split == 1 ? v.h : v.rows);        // rows per strip
-    const uint64_t S = (uint64_t)v.nstrips, sc = (uint64_t)v.ichunk;
+//   last_strip: of an operand whose last strip is narrower / lower than the others, the map of that strip alone (the
+//                map of the others leaves it out)
+static ccl_status operand_tmap(CUtensorMap* m, const MatView& v, const void* base, uint32_t box_inner, uint32_t box_rows, int64_t batch, int64_t batch_stride_bytes,
+                               bool last_strip = false) {
+    uint64_t row = (uint64_t)(v.split == 2 ? v.w : v.cols);      // elements of a strip row
+    uint64_t R = (uint64_t)(v.split == 1 ? v.h : v.rows);        // rows per strip
+    uint64_t S = (uint64_t)v.nstrips;
+    const uint64_t sc = (uint64_t)v.ichunk;
+    if (ragged(v)) {
+        if (last_strip) {
+            base = static_cast<const unsigned char*>(base) + (size_t)(v.nstrips - 1) * (size_t)v.stride * 2;
+            if (v.split == 2) row = (uint64_t)v.wlast; else R = (uint64_t)v.hlast;
+            S = 1;
+        } else S -= 1;
+    }
     uint64_t dims[5], strides[4];
     uint32_t box[5];
     int64_t kr;
@@ -1686,6 +1727,7 @@ static ccl_status operand_tmap(CUtensorMap* m, const MatView& v, const void* bas
     } else if (mode == 0) {
         dims[0] = row; dims[1] = R; dims[2] = v.split ? S : 1; dims[3] = 1;
         strides[0] = row * 2; strides[1] = v.split ? (uint64_t)v.stride * 2 : row * 2; strides[2] = strides[1];
+        // (the last strip alone: one strip, so the strip stride is never applied; keep it a multiple of 16 bytes)
         box[0] = box_inner; box[1] = box_rows; box[2] = 1; box[3] = 1;
     } else return fail(CCL_ERR_UNSUPPORTED, "ccl_gemm: this page-interleaved layout has no tensor map");
     strides[3] = dims[4] > 1 ? (uint64_t)batch_stride_bytes : strides[0];
@@ -1725,7 +1767,7 @@ static ccl_status launch(const GemmPlan& plan, const CUtensorMap& ma, const CUte
         attr[1].val.programmaticStreamSerializationAllowed = 1;
         cfg.numAttrs = 2;
     }
-    CCL_CUDA_TRY(cudaLaunchKernelEx(&cfg, ccl_gemm_kernel<BN, CTAS, SWIGLU, RAG, FULL, KS>, ma, mb, mc, plan.p));
+    CCL_CUDA_TRY(cudaLaunchKernelEx(&cfg, ccl_gemm_kernel<BN, CTAS, SWIGLU, RAG, FULL, KS>, ma, mb, mc, plan.ma2, plan.mb2, plan.mc2, plan.p));
     count_launch();
     return CCL_OK;
 }
@@ -1957,7 +1999,8 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
         {
             const GemmParams& q = plan.p;
             const bool ks = (q.a_mn ? q.a.split == 1 : q.a.split == 2) || (q.b_mn ? q.b.split == 1 : q.b.split == 2);
-            plan.lean = q.group_dim != 2 && !q.axpby && batch == 1 && !q.a.il_mode && !q.b.il_mode && !q.c.il_mode && !ks && !m_offs && !k_offs && !swiglu;
+            plan.lean = q.group_dim != 2 && !q.axpby && batch == 1 && !q.a.il_mode && !q.b.il_mode && !q.c.il_mode && !ks && !m_offs && !k_offs && !swiglu &&
+                        !q.a.rag && !q.b.rag && !q.c.rag;
         }
         const uint32_t bnh = plan.bn == 384 ? 64u : (uint32_t)(plan.subn / plan.ctas);   // B rows of one K-major box
         if (!plan.p.a_mn) s = operand_tmap(&prep.ma, plan.va, A_dev, BK, (uint32_t)plan.a_box_rows, batch, batch4[1]); else s = operand_tmap(&prep.ma, plan.va, A_dev, 64, BK, batch, batch4[1]);
@@ -1965,6 +2008,13 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
         if (!plan.p.b_mn) s = operand_tmap(&prep.mb, plan.vb, B_dev, BK, bnh, batch, batch4[2]); else s = operand_tmap(&prep.mb, plan.vb, B_dev, 64, BK, batch, batch4[2]);
         if (s) return s;
         if ((s = operand_tmap(&prep.mc, plan.vc, C_dev, 64, 32, batch, batch4[3]))) return s;   // C: 64-column x 32-row store boxes
+        // the last strips of operands whose strips are not all alike (else copies)
+        plan.ma2 = prep.ma; plan.mb2 = prep.mb; plan.mc2 = prep.mc;
+        if (ragged(plan.va) && (s = plan.p.a_mn ? operand_tmap(&plan.ma2, plan.va, A_dev, 64, BK, batch, batch4[1], true)
+                                              : operand_tmap(&plan.ma2, plan.va, A_dev, BK, (uint32_t)plan.a_box_rows, batch, batch4[1], true))) return s;
+        if (ragged(plan.vb) && (s = plan.p.b_mn ? operand_tmap(&plan.mb2, plan.vb, B_dev, 64, BK, batch, batch4[2], true)
+                                              : operand_tmap(&plan.mb2, plan.vb, B_dev, BK, bnh, batch, batch4[2], true))) return s;
+        if (ragged(plan.vc) && (s = operand_tmap(&plan.mc2, plan.vc, C_dev, 64, 32, batch, batch4[3], true))) return s;
         prep.key = key; prep.valid = true;
         std::lock_guard<std::mutex> lock(g_prepared_mutex);
         g_prepared[g_prepared_next] = prep;
@@ -2004,7 +2054,8 @@ static ccl_status gemm_impl(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
         plan.p.wave_period = wave_sync > 0 ? wave_sync : 1; plan.p.wave_wait_ns = 20000;        // one wait gives up after 20 us
         // (long tiles only: with K below 4096, or a batch of small problems, the CTAs share little and the waits only cost --
         // measured -9 % on 128 batched expert GEMMs and on a 16384 x 1536 x 2048 fused gate/up GEMM)
-        if (wave_sync > 0 && plan.p.sch_rounds >= 3 && plan.p.kb_per_split >= 64 && batch == 1 && !m_offs && !k_offs) {
+        const bool any_rag = plan.p.a.rag || plan.p.b.rag || plan.p.c.rag;      // (CTAs that skip the empty places of a short last strip would miss the meeting)
+        if (wave_sync > 0 && plan.p.sch_rounds >= 3 && plan.p.kb_per_split >= 64 && batch == 1 && !m_offs && !k_offs && !any_rag) {
             // One of kWaveSlots counters in the library image, handed out round-robin: a launch recorded into a CUDA graph
             // keeps its slot for good while eager calls rotate through all of them, so two GEMMs that overlap on the GPU
             // can land on one counter -- the barrier is soft (a wait just ends early or runs into its 20 us bound), results

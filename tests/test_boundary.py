@@ -185,7 +185,9 @@ def test_gemm_rejects_bad_input_before_any_launch():
     assert gemm_rc(d) == ccl.ERR_UNSUPPORTED
     d = gemm_desc(128, 256, 64, 3, ("row", "row", "row"))
     assert gemm_rc(d) == ccl.ERR_SHAPE                                                               # N % P with a grouped raster
-    assert gemm_rc(gemm_desc(128, 264, 64, 4, ("row", "ccl", "row"), grouped=0)) == ccl.ERR_UNSUPPORTED   # strips of unequal width (264 = 3 * 72 + 48)
+    assert gemm_rc(gemm_desc(128, 264, 64, 4, ("row", "ccl", "row"), grouped=0)) == ccl.ERR_UNSUPPORTED   # strips of 66 columns
+    assert gemm_rc(gemm_desc(128, 1000, 64, 4, ("row", "row", "row"), out_part=2, grouped=1)) == ccl.ERR_UNSUPPORTED   # tiles would start at multiples of 250 columns
+    assert gemm_rc(gemm_desc(264, 1000, 64, 3, ("row", "ccl", "row"), b_trans=1)) == ccl.ERR_UNSUPPORTED   # B [N x K] in strips of 334 rows: C's tiles would start there
     d = gemm_desc(256, 512, 64, 4, ("row", "row", "row"), out_part=3)
     d.part_m = 3
     assert gemm_rc(d) == ccl.ERR_INVALID_ARG                                                         # part_m must divide P

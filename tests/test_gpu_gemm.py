@@ -324,6 +324,42 @@ def test_gemm_every_tile_shape(M, N, K, P, at, bt, tile_mode):
     check(d, A, B)
 
 
+RAGGED_STRIPS = [
+    # M, N, K, P, layouts, a_trans, b_trans, out_part -- the split dimension is not a multiple of P: strips of ceil(./P), the last one shorter
+    (330, 512, 256, 4, ("ccl", "row", "ccl"), 0, 0, 1),        # M-partition: A and C in strips of 83 rows, the last of 81
+    (1301, 256, 200, 3, ("ccl", "row", "ccl"), 0, 0, 1),       # ... strips of 434 rows (several tiles each), the last of 433; ragged K
+    (264, 1016, 328, 16, ("row", "ccl", "row"), 0, 1, 2),      # B stored [N x K] in strips of 64 rows, the last of 56; C row-major
+    (130, 1016, 192, 16, ("row", "ccl", "ccl"), 0, 0, 2),      # column strips of 64, the last of 56 (P = 16)
+    (1016, 256, 128, 16, ("ccl", "row", "row"), 1, 0, 1),      # A stored [K x M] in column strips of 64, the last of 56
+    (700, 2040, 512, 16, ("row", "ccl", "ccl"), 0, 0, 2),      # column strips of 128, the last of 120; several tiles per CTA
+]
+
+
+@pytest.mark.parametrize("M,N,K,P,lay,at,bt,op", RAGGED_STRIPS)
+def test_gemm_strips_of_unequal_size(M, N, K, P, lay, at, bt, op, cta_mode):
+    """Operands whose last strip is narrower / lower than the others (reading: w = ceil(N / P)): the last strip has a tensor
+    map of its own.  Parity with the oracle, grouped and plain raster; the guard zone behind C stays untouched."""
+    A, B = synth.gemm_operands(M, N, K, at, bt, seed=13, tag="ragstrips")
+    for grouped in (1, 0):
+        check(gemm_desc(M, N, K, P, lay, at, bt, op, grouped), A, B)
+    if "ccl" in lay:
+        check(gemm_desc(M, N, K, P, lay, at, bt, op, 1, align=4096), A, B)   # page-aligned strips
+
+
+def test_gemm_strips_of_unequal_size_axpby():
+    M, N, K, P = 330, 512, 256, 4
+    A, B = synth.gemm_operands(M, N, K, 0, 0, seed=14, tag="ragstrips/axpby")
+    Cin = synth.randn_bf16(M, N, 1.0, 14, "ragstrips/C")
+    d = gemm_desc(M, N, K, P, ("ccl", "row", "ccl"), 0, 0, 1, 1)
+    a_dev, b_dev, c_dev = to_layout(synth.bits(A), d.A), to_layout(synth.bits(B), d.B), to_layout(synth.bits(Cin), d.C)
+    ccl.ccl_gemm_axpby(d, 0.5, 2.0, a_dev, b_dev, c_dev)
+    assert ccl.ccl_gemm_status()[0] == ccl.OK
+    got = synth.from_bits(from_layout(c_dev, d.C)).to(torch.float32).numpy()
+    ref32, _ = orc.gemm_axpby(synth.bits(A), synth.bits(B), synth.bits(Cin), M, N, K, 0.5, 2.0, 0, 0)
+    err = np.abs(got - ref32) / np.maximum(1.0, np.abs(ref32))
+    assert err.max() <= 0.5 * tol(K) + 2.0 ** -8, err.max()
+
+
 WIDE384 = [
     # M, N, K, P, layouts, a_trans, b_trans, out_part, chunk bytes (page-interleaved operands), alpha, beta
     (4096, 1536, 256, 4, ("row", "ccl", "ccl"), 0, 0, 2, 0, 1.0, 0.0),          # strips of exactly one tile width (the Qwen gate+up shape, short K)
