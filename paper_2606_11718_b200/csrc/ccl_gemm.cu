@@ -1313,12 +1313,14 @@ static int resident_clusters(int ks, bool have_device);
 
 // Modelled cycles of one k block (64 of K) of a tile `b` columns wide on `c` CTAs: the tensor pipe needs 2 cycles per tile
 // column (128 rows per SM, UMMA_K = 16, four steps); the SM pulls its share of the operands (its 128 rows of A and its
-// columns of B, whole 64-column boxes of an N-contiguous B) from the L2 at ~70 B/clk; the producer and MMA-issue loops
-// need ~450 cycles per block whatever the tile (all measured with per-role timestamps); the longest of the three, plus
-// the hand-over.
-static double kblock_cycles(int b, int c, bool b_kmajor) {
+// columns of B, whole 64-column boxes of an N-contiguous B) from the L2 at ~70 B/clk on its own and at its share of
+// ~9 KB/clk when `active` CTAs pull at once (61 B/clk with all 148: 128 x 192 tiles measured 670 cycles per block in a
+// batch that fills the machine, 585 alone); the producer and MMA-issue loops need ~450 cycles per block whatever the
+// tile (all measured with per-role timestamps); the longest of the three, plus the hand-over.
+static double kblock_cycles(int b, int c, bool b_kmajor, int64_t active) {
     const double b_cols = (double)(b_kmajor ? b / c : (b / c + 63) / 64 * 64);
-    return std::max(std::max(2.0 * b, (BM + b_cols) * (BK * 2) / 70.0), 450.0) + 15.0;
+    const double rate = std::min(70.0, 9000.0 / (double)std::max<int64_t>(1, active));
+    return std::max(std::max(2.0 * b, (BM + b_cols) * (BK * 2) / rate), 450.0) + 15.0;
 }
 
 // have_device: the unit counts come from the current device (else the figures of a B200)
@@ -1445,7 +1447,7 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
             // a k block: the tensor pipe needs 2 cycles per tile column (128 rows per SM, UMMA_K = 16, four steps), the
             // SM pulls its share of the operands (its 128 rows of A and its columns of B, whole 64-column boxes of an
             // N-contiguous B) from the L2 at ~70 B/clk; whichever is longer, plus the hand-over
-            const double t_kb = kblock_cycles(b, c, bt);
+            const double t_kb = kblock_cycles(b, c, bt, std::min<int64_t>(tiles, units) * c);
             const double t_drain = b == 512 ? 7000.0 : (b == 384 ? 5500.0 : 1500.0);
             // one row of tiles: nobody shares the B columns, the problem streams B from HBM at ~29 B/clk per SM in
             // aggregate however the units are cut (a ragged last wave still saturates the memory); wider boxes are
@@ -1551,7 +1553,7 @@ static ccl_status make_plan(const ccl_gemm_desc* d, int64_t batch, bool swiglu, 
                 if ((num_kb + kbps - 1) / kbps != k || kbps < 2) continue;           // every CTA of the cluster owns k blocks
                 // drain, the exchange (every CTA sends (k - 1) / k of its sums and adds up k sources: ~1000 cycles per CTA of
                 // the cluster, measured on 256 x 768 x 2048: 7.0 / 7.4 / 7.9 / 8.5 us with clusters of 4 / 3 / 6 / 8), launch
-                const double cost = (double)kbps * kblock_cycles(b, 1, bt) + 1500.0 + (1000.0 + 1000.0 * k) + 3000.0;
+                const double cost = (double)kbps * kblock_cycles(b, 1, bt, tiles * k) + 1500.0 + (1000.0 + 1000.0 * k) + 3000.0;
                 if (best_ks < 0 || cost < best_ks) { best_ks = cost; kb_ = b; kk = k; }
             }
         }
